@@ -1,0 +1,190 @@
+/*
+ * hotline.h -- C boundary of the B200 (sm_100a) library for the data-parallel hot path of the Hotline
+ * heterogeneous embedding pipeline (arXiv 2204.05436).
+ *
+ * The path, per mini-batch (paper Section IV "Acceleration Phase", Fig. 8):
+ *   hl_fragment        split mini-batch M into the popular micro-batch O (every lookup hits a popular row)
+ *                      and the non-popular micro-batch X                              (Sections I, V-A, V-C; Eq. 3)
+ *   hl_gather_cold     stage X's non-popular working rows from the host-DRAM table behind the hot cache,
+ *                      on a side stream, while O executes                              (Sections IV, V-A)
+ *   hl_embbag_fwd      sum-pool the rows of every bag                                 (the Reducer, Section V-D)
+ *   hl_embbag_bwd_sgd  scatter-add the pooled gradients per distinct row, one SGD update per row (Section IV)
+ *   hl_scatter_cold    write X's updated cold rows back to the host table              (Section IV, dma_wr)
+ * and, once per learning phase (Section IV "Learning Phase", Section V-B):
+ *   hl_profile_hot     count row accesses over sampled mini-batches and select the popular rows
+ *   hl_build_remap     build the popular-row lookup structure and load the popular rows into HBM.
+ *
+ * Conventions
+ *   - Pointers named d_* are DEVICE pointers (16-byte aligned); h_* are HOST pointers; `host_table` must be
+ *     readable/writable from the device (pinned, mapped host memory; device memory also works).
+ *   - The caller owns every buffer.  The library allocates nothing on the device: its scratch lives in the
+ *     caller-provided workspace given to hl_create (size from hl_workspace_bytes).
+ *   - Every call returns an int32 status (HL_OK = 0, negative = error) for what the host can check.  Calls are
+ *     asynchronous on `stream` (a cudaStream_t passed as void*); errors found on the device (an index outside
+ *     its table, a capacity overflow) never trap: the offending item is skipped, a status word is set, and
+ *     hl_status() returns it.
+ *   - No call synchronises the host, so sizes that depend on the data (number of popular inputs, number of
+ *     cold rows, lookups per micro-batch) stay in device memory and are passed between calls as pointers.
+ *   - Mini-batch layout: table-major CSR.  Bag beta(t, b, s) = (t*B + b)*S + s for table t, input b, step s
+ *     holds indices[offsets[beta] .. offsets[beta+1]), table-local int32 row ids.  Global row id
+ *     g = base_t + index, base_t = rows of all earlier tables.  N = total rows < 2^31.
+ *   - fp32 values; dim % 4 == 0.
+ *   - Calls that share a context may overlap on different streams only as stated per call (each call names
+ *     the scratch region it uses).
+ */
+#ifndef HOTLINE_H_
+#define HOTLINE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define HL_API __attribute__((visibility("default")))
+#else
+#define HL_API
+#endif
+
+#define HL_OK          0
+#define HL_EINVAL    (-1)   /* bad argument, shape or alignment (host check), or malformed device data          */
+#define HL_EBOUNDS   (-2)   /* an index outside its table / a slot outside the cache (device; item skipped)      */
+#define HL_ECAPACITY (-3)   /* an output buffer, the hot cache or the staging area is too small (device; clamped)*/
+#define HL_ECUDA     (-4)   /* a CUDA runtime call failed                                                        */
+#define HL_ETIMEOUT  (-5)   /* reserved: a bounded device-side wait gave up                                      */
+
+typedef struct hl_ctx hl_ctx;
+
+/* Model geometry.  table_rows is a HOST array of num_tables row counts. */
+typedef struct {
+    int32_t        num_tables;       /* T                                                         */
+    int32_t        dim;              /* D, fp32 columns per row, multiple of 4                    */
+    int32_t        bags_per_sample;  /* S: bags per input and table (21 time steps, else 1)       */
+    const int64_t* table_rows;       /* host, [T]                                                 */
+} hl_geometry;
+
+/* One mini-batch in device memory (table-major CSR, see above). */
+typedef struct {
+    const int32_t* indices;          /* device, [nnz]                                             */
+    const int32_t* offsets;          /* device, [T*batch*S + 1], offsets[0] = 0                   */
+    int32_t        batch;            /* B inputs                                                  */
+    int64_t        nnz;              /* total lookups L = offsets[T*batch*S]                      */
+} hl_batch;
+
+/* One micro-batch in device memory, caller-sized for the worst case (all inputs land in it). */
+typedef struct {
+    int32_t* offsets;                /* device, [T*max_batch*S + 1]                               */
+    int32_t* ids;                    /* device, [cap_ids]: cache slots, or global rows (X before hl_gather_cold) */
+    int64_t  cap_ids;
+} hl_ubatch;
+
+/* How hl_profile_hot turns counts into a popular set.  All policies rank rows seen at least once by
+ * (count descending, global id ascending), one ranking across all tables, and clip to the hot capacity. */
+enum {
+    HL_HOT_TOPK_ROWS     = 0,        /* keep p_num rows                                           */
+    HL_HOT_BUDGET_BYTES  = 1,        /* keep floor(p_num / (4*D)) rows (row payload only)         */
+    HL_HOT_FRACTION_ROWS = 2,        /* keep floor(N * p_num / p_den) rows                        */
+    HL_HOT_MIN_SHARE     = 3         /* keep rows with count/total >= p_num/p_den (the paper's
+                                        1-in-100,000 criterion, Fig. 4), exact integer test       */
+};
+
+/* ---------------------------------------------------------------------------------------------------------
+ * Support calls (no counterpart in the paper; they carry the address registers of the Data Dispatcher,
+ * Section V-A: one base per table).
+ * ------------------------------------------------------------------------------------------------------- */
+
+/* Bytes of device workspace a context needs for mini-batches of at most max_batch inputs and max_nnz
+ * lookups, hot_cap_rows cache slots and staging_cap_rows staging slots.  0 on invalid arguments. */
+HL_API size_t hl_workspace_bytes(const hl_geometry* geom, int32_t max_batch, int64_t max_nnz,
+                          int64_t hot_cap_rows, int64_t staging_cap_rows);
+
+/* Creates a context on the current device.  d_workspace (device, 256-byte aligned, ws_bytes long) stays
+ * owned by the caller and must outlive the context.  Synchronous (initialises the workspace).
+ * The cache the other calls take is fp32 [(hot_cap_rows + staging_cap_rows), D]: slots [0, hot_cap_rows) hold
+ * popular rows, slot hot_cap_rows + i holds the i-th staged cold row. */
+HL_API int32_t hl_create(hl_ctx** out, const hl_geometry* geom, int32_t max_batch, int64_t max_nnz,
+                  int64_t hot_cap_rows, int64_t staging_cap_rows, void* d_workspace, size_t ws_bytes);
+HL_API int32_t hl_destroy(hl_ctx* ctx);
+
+/* Synchronises the device, returns the first device-side error recorded since the last call (HL_OK if
+ * none) and clears it. */
+HL_API int32_t hl_status(hl_ctx* ctx);
+
+HL_API const char* hl_strerror(int32_t status);
+
+/* ---------------------------------------------------------------------------------------------------------
+ * Learning phase
+ * ------------------------------------------------------------------------------------------------------- */
+
+/* Section IV "Learning Phase" / Section V-B (the exact counter the paper calls the Oracle LFU logger).
+ * If reset != 0 the per-row access counters are cleared first.  If b != NULL every lookup of the mini-batch
+ * adds one to its row's counter (repeats inside a bag count again).  If finalize != 0 the popular rows are
+ * selected by `policy` (see the enum) and written in ASCENDING global id to d_hot_rows [hot_cap_rows], their
+ * number to *d_n_hot.  Scratch: the profile region.  Must not overlap with other calls on this context. */
+HL_API int32_t hl_profile_hot(hl_ctx* ctx, const hl_batch* b, int32_t reset, int32_t finalize,
+                       int32_t policy, int64_t p_num, int64_t p_den,
+                       int32_t* d_hot_rows, int64_t* d_n_hot, void* stream);
+
+/* Section IV: popular rows are replicated in GPU memory, the classifier keeps only their indices.
+ * Builds the lookup structure for the popular set d_hot_rows[0 .. *d_n_hot) (strictly ascending global ids;
+ * any such set is allowed, misclassification never affects fidelity): the cache slot of a popular row is its
+ * rank in that list.  If host_table != NULL also loads cache[i, :] = host_table[hot_rows[i], :] (bit copy).
+ * If d_remap_out != NULL writes the dense map remap[g] = slot or -1, int32 [N].
+ * Must not overlap with other calls on this context. */
+HL_API int32_t hl_build_remap(hl_ctx* ctx, const int32_t* d_hot_rows, const int64_t* d_n_hot,
+                       const float* host_table, float* d_cache, int32_t* d_remap_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------------------
+ * Acceleration phase
+ * ------------------------------------------------------------------------------------------------------- */
+
+/* Sections I, V-A (Input Classifier), V-C (Lookup Engine), Eq. 3.
+ * An input is popular iff every lookup of it, over all tables and steps, addresses a popular row (an input
+ * without lookups is popular).  Outputs:
+ *   d_perm   [B]   inputs of O in ascending order, then inputs of X in ascending order
+ *   d_counts [4]   { n_pop, n_non, lookups in O, lookups in X }
+ *   pop            O as table-major CSR over its n_pop inputs; ids = cache slots
+ *   non            X as table-major CSR over its n_non inputs; ids = GLOBAL row ids (-1 for an index that was
+ *                  outside its table: such a lookup counts as a miss and is ignored downstream)
+ *   d_dense_out    optional [B, n_dense]: d_dense rows in d_perm order (values untouched)
+ * Scratch: the fragment region (may overlap with embbag/cold calls of an earlier mini-batch). */
+HL_API int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_dense, int32_t n_dense,
+                    int32_t* d_perm, int32_t* d_counts, hl_ubatch* pop, hl_ubatch* non,
+                    float* d_dense_out, void* stream);
+
+/* Section V-D (Reducer: sparse-length element-wise sum).
+ * out[beta, :] = sum over the bag's lookups of cache[ids[j], :], for the T * (*d_n_samples) * S bags of the
+ * micro-batch; an empty bag gives zeros; negative ids are skipped.  d_out is [T*max_batch*S, D].
+ * Uses no scratch: may overlap with anything that does not write the rows it reads. */
+HL_API int32_t hl_embbag_fwd(hl_ctx* ctx, const float* d_cache, const hl_ubatch* ub, const int32_t* d_n_samples,
+                      float* d_out, void* stream);
+
+/* Section IV (popular rows are updated in GPU memory; plain SGD as the optimizer).
+ * For every distinct id u of the micro-batch: G_u = sum over lookups j with ids[j] == u of
+ * d_grad_out[bag(j), :], then cache[u, :] -= lr * G_u, exactly one read-modify-write per row, deterministic
+ * (duplicates are segmented by a sort, no floating-point atomics).  Rows not referenced keep their bits.
+ * Scratch: the backward region (may overlap with hl_gather_cold / hl_fragment, not with itself). */
+HL_API int32_t hl_embbag_bwd_sgd(hl_ctx* ctx, float* d_cache, const hl_ubatch* ub, const int32_t* d_n_samples,
+                          const float* d_grad_out, float lr, void* stream);
+
+/* Sections IV and V-A (dma_rd of non-popular rows; popular rows of X are read from GPU memory).
+ * In:  non->ids = global rows of X (from hl_fragment), *d_n_non = inputs in X.
+ * Out: d_cold_rows[0 .. *d_n_cold) = the distinct non-popular rows referenced by X, ascending (each staged
+ *      once); non->ids rewritten to unified cache slots (hot slot, or hot_cap_rows + rank in d_cold_rows);
+ *      cache[hot_cap_rows + i, :] = host_table[d_cold_rows[i], :].
+ * Touches only the staging part of the cache: may run on a side stream while O's forward/backward run.
+ * Scratch: the cold region. */
+HL_API int32_t hl_gather_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const float* host_table,
+                       float* d_cache, int32_t* d_cold_rows, int64_t* d_n_cold, void* stream);
+
+/* Section IV (non-popular rows are updated in CPU memory by DMA write).
+ * host_table[d_cold_rows[i], :] = cache[hot_cap_rows + i, :] for i < *d_n_cold.  No scratch. */
+HL_API int32_t hl_scatter_cold(hl_ctx* ctx, const float* d_cache, const int32_t* d_cold_rows,
+                        const int64_t* d_n_cold, float* host_table, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HOTLINE_H_ */

@@ -1,0 +1,184 @@
+"""ctypes binding of libhotline.so: the same names and arguments as include/hotline.h, marshalling only.
+
+Pointers are passed as integers (``tensor.data_ptr()``), as objects with a ``data_ptr()`` method, or None.
+A negative status raises :class:`HotlineError`.  There is no fallback: if the library is missing, importing
+this module fails and says how to build it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhotline.so")
+
+HL_OK, HL_EINVAL, HL_EBOUNDS, HL_ECAPACITY, HL_ECUDA, HL_ETIMEOUT = 0, -1, -2, -3, -4, -5
+HL_HOT_TOPK_ROWS, HL_HOT_BUDGET_BYTES, HL_HOT_FRACTION_ROWS, HL_HOT_MIN_SHARE = 0, 1, 2, 3
+
+EXPORTS = (
+    "hl_workspace_bytes", "hl_create", "hl_destroy", "hl_status", "hl_strerror", "hl_profile_hot",
+    "hl_build_remap", "hl_fragment", "hl_embbag_fwd", "hl_embbag_bwd_sgd", "hl_gather_cold", "hl_scatter_cold",
+)
+
+
+class HotlineError(RuntimeError):
+    def __init__(self, call: str, status: int):
+        self.status = status
+        super().__init__(f"{call} failed with status {status} ({strerror(status)})")
+
+
+class hl_geometry(ctypes.Structure):
+    _fields_ = [("num_tables", ctypes.c_int32), ("dim", ctypes.c_int32), ("bags_per_sample", ctypes.c_int32),
+                ("table_rows", ctypes.POINTER(ctypes.c_int64))]
+
+
+class hl_batch(ctypes.Structure):
+    _fields_ = [("indices", ctypes.c_void_p), ("offsets", ctypes.c_void_p), ("batch", ctypes.c_int32),
+                ("nnz", ctypes.c_int64)]
+
+
+class hl_ubatch(ctypes.Structure):
+    _fields_ = [("offsets", ctypes.c_void_p), ("ids", ctypes.c_void_p), ("cap_ids", ctypes.c_int64)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(_LIB_PATH):
+        raise ImportError(
+            f"{_LIB_PATH} is missing: build it with `python -m paper_2204_05436_b200.build` "
+            "(needs nvcc; there is no CPU fallback)")
+    lib = ctypes.CDLL(_LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    geo = ctypes.POINTER(hl_geometry)
+    lib.hl_workspace_bytes.restype = ctypes.c_size_t
+    lib.hl_workspace_bytes.argtypes = [geo, i32, i64, i64, i64]
+    lib.hl_create.restype = i32
+    lib.hl_create.argtypes = [ctypes.POINTER(vp), geo, i32, i64, i64, i64, vp, ctypes.c_size_t]
+    lib.hl_destroy.restype = i32
+    lib.hl_destroy.argtypes = [vp]
+    lib.hl_status.restype = i32
+    lib.hl_status.argtypes = [vp]
+    lib.hl_strerror.restype = ctypes.c_char_p
+    lib.hl_strerror.argtypes = [i32]
+    lib.hl_profile_hot.restype = i32
+    lib.hl_profile_hot.argtypes = [vp, ctypes.POINTER(hl_batch), i32, i32, i32, i64, i64, vp, vp, vp]
+    lib.hl_build_remap.restype = i32
+    lib.hl_build_remap.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.hl_fragment.restype = i32
+    lib.hl_fragment.argtypes = [vp, ctypes.POINTER(hl_batch), vp, i32, vp, vp, ctypes.POINTER(hl_ubatch),
+                                ctypes.POINTER(hl_ubatch), vp, vp]
+    lib.hl_embbag_fwd.restype = i32
+    lib.hl_embbag_fwd.argtypes = [vp, vp, ctypes.POINTER(hl_ubatch), vp, vp, vp]
+    lib.hl_embbag_bwd_sgd.restype = i32
+    lib.hl_embbag_bwd_sgd.argtypes = [vp, vp, ctypes.POINTER(hl_ubatch), vp, vp, ctypes.c_float, vp]
+    lib.hl_gather_cold.restype = i32
+    lib.hl_gather_cold.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, vp, vp, vp, vp, vp]
+    lib.hl_scatter_cold.restype = i32
+    lib.hl_scatter_cold.argtypes = [vp, vp, vp, vp, vp, vp]
+    return lib
+
+
+_lib = _load()
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def _ptr(x) -> Optional[int]:
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    return int(x.data_ptr())
+
+
+def _check(call: str, status: int) -> int:
+    if status < 0:
+        raise HotlineError(call, status)
+    return status
+
+
+def strerror(status: int) -> str:
+    return _lib.hl_strerror(int(status)).decode()
+
+
+def make_geometry(table_rows: Sequence[int], dim: int, bags_per_sample: int = 1) -> hl_geometry:
+    arr = (ctypes.c_int64 * len(table_rows))(*[int(r) for r in table_rows])
+    g = hl_geometry(len(table_rows), int(dim), int(bags_per_sample), arr)
+    g._keepalive = arr
+    return g
+
+
+def make_batch(indices, offsets, batch: int, nnz: int) -> hl_batch:
+    return hl_batch(_ptr(indices), _ptr(offsets), int(batch), int(nnz))
+
+
+def make_ubatch(offsets, ids, cap_ids: int) -> hl_ubatch:
+    return hl_ubatch(_ptr(offsets), _ptr(ids), int(cap_ids))
+
+
+def hl_workspace_bytes(geom: hl_geometry, max_batch: int, max_nnz: int, hot_cap_rows: int,
+                       staging_cap_rows: int) -> int:
+    n = _lib.hl_workspace_bytes(ctypes.byref(geom), max_batch, max_nnz, hot_cap_rows, staging_cap_rows)
+    if n == 0:
+        raise HotlineError("hl_workspace_bytes", HL_EINVAL)
+    return int(n)
+
+
+def hl_create(geom: hl_geometry, max_batch: int, max_nnz: int, hot_cap_rows: int, staging_cap_rows: int,
+              d_workspace, ws_bytes: int) -> int:
+    ctx = ctypes.c_void_p()
+    _check("hl_create", _lib.hl_create(ctypes.byref(ctx), ctypes.byref(geom), max_batch, max_nnz, hot_cap_rows,
+                                       staging_cap_rows, _ptr(d_workspace), ws_bytes))
+    return ctx.value
+
+
+def hl_destroy(ctx: int) -> None:
+    _check("hl_destroy", _lib.hl_destroy(ctx))
+
+
+def hl_status(ctx: int, raise_on_error: bool = True) -> int:
+    st = _lib.hl_status(ctx)
+    if raise_on_error:
+        _check("hl_status", st)
+    return st
+
+
+def hl_profile_hot(ctx: int, batch: Optional[hl_batch], reset: bool, finalize: bool, policy: int, p_num: int,
+                   p_den: int, d_hot_rows, d_n_hot, stream: int) -> None:
+    b = ctypes.byref(batch) if batch is not None else None
+    _check("hl_profile_hot", _lib.hl_profile_hot(ctx, b, int(reset), int(finalize), policy, p_num, p_den,
+                                                 _ptr(d_hot_rows), _ptr(d_n_hot), stream))
+
+
+def hl_build_remap(ctx: int, d_hot_rows, d_n_hot, host_table, d_cache, d_remap_out, stream: int) -> None:
+    _check("hl_build_remap", _lib.hl_build_remap(ctx, _ptr(d_hot_rows), _ptr(d_n_hot), _ptr(host_table),
+                                                 _ptr(d_cache), _ptr(d_remap_out), stream))
+
+
+def hl_fragment(ctx: int, batch: hl_batch, d_dense, n_dense: int, d_perm, d_counts, pop: hl_ubatch,
+                non: hl_ubatch, d_dense_out, stream: int) -> None:
+    _check("hl_fragment", _lib.hl_fragment(ctx, ctypes.byref(batch), _ptr(d_dense), n_dense, _ptr(d_perm),
+                                           _ptr(d_counts), ctypes.byref(pop), ctypes.byref(non),
+                                           _ptr(d_dense_out), stream))
+
+
+def hl_embbag_fwd(ctx: int, d_cache, ub: hl_ubatch, d_n_samples, d_out, stream: int) -> None:
+    _check("hl_embbag_fwd", _lib.hl_embbag_fwd(ctx, _ptr(d_cache), ctypes.byref(ub), _ptr(d_n_samples),
+                                               _ptr(d_out), stream))
+
+
+def hl_embbag_bwd_sgd(ctx: int, d_cache, ub: hl_ubatch, d_n_samples, d_grad_out, lr: float, stream: int) -> None:
+    _check("hl_embbag_bwd_sgd", _lib.hl_embbag_bwd_sgd(ctx, _ptr(d_cache), ctypes.byref(ub), _ptr(d_n_samples),
+                                                       _ptr(d_grad_out), float(lr), stream))
+
+
+def hl_gather_cold(ctx: int, non: hl_ubatch, d_n_non, host_table, d_cache, d_cold_rows, d_n_cold,
+                   stream: int) -> None:
+    _check("hl_gather_cold", _lib.hl_gather_cold(ctx, ctypes.byref(non), _ptr(d_n_non), _ptr(host_table),
+                                                 _ptr(d_cache), _ptr(d_cold_rows), _ptr(d_n_cold), stream))
+
+
+def hl_scatter_cold(ctx: int, d_cache, d_cold_rows, d_n_cold, host_table, stream: int) -> None:
+    _check("hl_scatter_cold", _lib.hl_scatter_cold(ctx, _ptr(d_cache), _ptr(d_cold_rows), _ptr(d_n_cold),
+                                                   _ptr(host_table), stream))

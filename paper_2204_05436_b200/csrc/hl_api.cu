@@ -1,0 +1,177 @@
+// Context, workspace carving and status of the Hotline library.
+#include <stdlib.h>
+#include <string.h>
+
+#include "hl_common.cuh"
+
+namespace hl {
+namespace {
+
+struct Carver {
+    char* base;
+    size_t off = 0;
+    template <typename T>
+    T* take(int64_t count) {
+        off = (off + 255) & ~size_t(255);
+        T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+        off += (size_t)count * sizeof(T);
+        return p;
+    }
+};
+
+bool geometry_ok(const hl_geometry* g, int64_t* total_rows) {
+    if (!g || g->num_tables < 1 || g->dim < 4 || (g->dim & 3) || g->bags_per_sample < 1 || !g->table_rows)
+        return false;
+    int64_t n = 0;
+    for (int t = 0; t < g->num_tables; ++t) {
+        if (g->table_rows[t] < 1) return false;
+        n += g->table_rows[t];
+        if (n >= (int64_t(1) << 31)) return false;   // global row ids are int32
+    }
+    *total_rows = n;
+    return true;
+}
+
+int64_t hist_words(int64_t max_nnz) {
+    const int64_t n_tiles = div_up(max_nnz > 0 ? max_nnz : 1, kSortTile);
+    const int64_t n_hist = 256 * n_tiles;
+    return n_hist + 1 + n_hist / kScanTile + 8;
+}
+
+// Lays the regions out over `base` (nullptr: size only).  Returns the bytes used.
+size_t carve(char* base, const hl_geometry* g, int64_t N, int32_t max_batch, int64_t max_nnz, int64_t hot_cap,
+             int64_t staging_cap, Regions* r, int64_t* n_remap_blocks, int64_t* n_sel_tiles) {
+    Carver c{base};
+    const int64_t T = g->num_tables, S = g->bags_per_sample, D = g->dim;
+    const int64_t max_bags = T * (int64_t)max_batch * S;
+    const int64_t nnz = max_nnz > 0 ? max_nnz : 1;
+    *n_remap_blocks = div_up(N, kRemapRowsPerBlock) + 1;
+    *n_sel_tiles = div_up(N, kSelTile);
+    r->status = c.take<int32_t>(8);
+    r->table_base = c.take<int64_t>(T + 1);
+    r->remap = c.take<RemapBlock>(*n_remap_blocks);
+    r->counts = c.take<uint32_t>(N);
+    r->sel = c.take<SelectState>(1);
+    r->sel_gt = c.take<uint32_t>(*n_sel_tiles + 2);
+    r->sel_eq = c.take<uint32_t>(*n_sel_tiles + 2);
+    r->frag_flags = c.take<uint8_t>(max_batch);
+    r->frag_scan = c.take<int32_t>(max_bags + 2);
+    r->frag_tiles = c.take<int32_t>(max_bags / kScanTile + 4);
+    for (int i = 0; i < 2; ++i) {
+        r->bwd_keys[i] = c.take<int32_t>(nnz);
+        r->bwd_vals[i] = c.take<int32_t>(nnz);
+    }
+    r->bwd_hist = c.take<uint32_t>(hist_words(nnz));
+    r->bwd_part = c.take<float>(2 * div_up(nnz, kBwdChunk) * D);
+    r->bwd_n = c.take<int32_t>(4);
+    for (int i = 0; i < 2; ++i) {
+        r->cold_keys[i] = c.take<int32_t>(nnz);
+        r->cold_vals[i] = c.take<int32_t>(nnz);
+    }
+    r->cold_hist = c.take<uint32_t>(hist_words(nnz));
+    r->cold_rank = c.take<int32_t>(nnz + 2);
+    r->cold_tiles = c.take<int32_t>(nnz / kScanTile + 4);
+    r->cold_n = c.take<int32_t>(4);
+    (void)hot_cap;
+    (void)staging_cap;
+    return (c.off + 255) & ~size_t(255);
+}
+
+}  // namespace
+}  // namespace hl
+
+using namespace hl;
+
+extern "C" size_t hl_workspace_bytes(const hl_geometry* geom, int32_t max_batch, int64_t max_nnz,
+                                     int64_t hot_cap_rows, int64_t staging_cap_rows) {
+    int64_t N;
+    if (!geometry_ok(geom, &N) || max_batch < 1 || max_nnz < 0 || hot_cap_rows < 0 || staging_cap_rows < 0) return 0;
+    Regions r;
+    int64_t a, b;
+    return carve(nullptr, geom, N, max_batch, max_nnz, hot_cap_rows, staging_cap_rows, &r, &a, &b);
+}
+
+extern "C" int32_t hl_create(hl_ctx** out, const hl_geometry* geom, int32_t max_batch, int64_t max_nnz,
+                             int64_t hot_cap_rows, int64_t staging_cap_rows, void* d_workspace, size_t ws_bytes) {
+    if (!out) return HL_EINVAL;
+    *out = nullptr;
+    int64_t N;
+    if (!geometry_ok(geom, &N) || max_batch < 1 || max_nnz < 0 || hot_cap_rows < 0 || staging_cap_rows < 0)
+        return HL_EINVAL;
+    const int64_t max_bags = (int64_t)geom->num_tables * max_batch * geom->bags_per_sample;
+    if (max_bags >= (int64_t(1) << 31) - 2 || max_nnz >= (int64_t(1) << 31) - 2) return HL_EINVAL;
+    if (hot_cap_rows + staging_cap_rows >= (int64_t(1) << 31) - 2) return HL_EINVAL;
+    if (!d_workspace || (reinterpret_cast<uintptr_t>(d_workspace) & 255)) return HL_EINVAL;
+
+    hl_ctx* ctx = static_cast<hl_ctx*>(calloc(1, sizeof(hl_ctx)));
+    if (!ctx) return HL_EINVAL;
+    ctx->T = geom->num_tables;
+    ctx->D = geom->dim;
+    ctx->S = geom->bags_per_sample;
+    ctx->N = N;
+    ctx->max_batch = max_batch;
+    ctx->max_nnz = max_nnz;
+    ctx->max_bags = max_bags;
+    ctx->hot_cap = hot_cap_rows;
+    ctx->staging_cap = staging_cap_rows;
+    const size_t need = carve(static_cast<char*>(d_workspace), geom, N, max_batch, max_nnz, hot_cap_rows,
+                              staging_cap_rows, &ctx->r, &ctx->n_remap_blocks, &ctx->n_sel_tiles);
+    if (need > ws_bytes) {
+        free(ctx);
+        return HL_ECAPACITY;
+    }
+    if (cudaGetDevice(&ctx->device) != cudaSuccess) {
+        free(ctx);
+        return HL_ECUDA;
+    }
+    ctx->h_table_base = static_cast<int64_t*>(malloc(sizeof(int64_t) * (ctx->T + 1)));
+    if (!ctx->h_table_base) {
+        free(ctx);
+        return HL_EINVAL;
+    }
+    ctx->h_table_base[0] = 0;
+    for (int t = 0; t < ctx->T; ++t) ctx->h_table_base[t + 1] = ctx->h_table_base[t] + geom->table_rows[t];
+
+    cudaError_t e = cudaMemcpy(ctx->r.table_base, ctx->h_table_base, sizeof(int64_t) * (ctx->T + 1),
+                               cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemset(ctx->r.status, 0, 8 * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->r.remap, 0, sizeof(RemapBlock) * ctx->n_remap_blocks);
+    if (e == cudaSuccess) e = cudaMemset(ctx->r.counts, 0, sizeof(uint32_t) * N);
+    if (e == cudaSuccess) e = cudaMemset(ctx->r.sel, 0, sizeof(SelectState));
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        free(ctx->h_table_base);
+        free(ctx);
+        return HL_ECUDA;
+    }
+    *out = ctx;
+    return HL_OK;
+}
+
+extern "C" int32_t hl_destroy(hl_ctx* ctx) {
+    if (!ctx) return HL_EINVAL;
+    free(ctx->h_table_base);
+    free(ctx);
+    return HL_OK;
+}
+
+extern "C" int32_t hl_status(hl_ctx* ctx) {
+    if (!ctx) return HL_EINVAL;
+    HL_CUDA_TRY(cudaDeviceSynchronize());
+    int32_t st = 0;
+    HL_CUDA_TRY(cudaMemcpy(&st, ctx->r.status, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    if (st != 0) HL_CUDA_TRY(cudaMemset(ctx->r.status, 0, sizeof(int32_t)));
+    return st;
+}
+
+extern "C" const char* hl_strerror(int32_t status) {
+    switch (status) {
+        case HL_OK: return "ok";
+        case HL_EINVAL: return "invalid argument or malformed data";
+        case HL_EBOUNDS: return "index outside its table or slot outside the cache";
+        case HL_ECAPACITY: return "output buffer, hot cache or staging area too small";
+        case HL_ECUDA: return "CUDA runtime error";
+        case HL_ETIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}

@@ -1,0 +1,150 @@
+// Shared declarations of the Hotline sm_100a library: context layout, status word, remap probe.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "hotline.h"
+
+namespace hl {
+
+constexpr int kSMs = 148;                  // B200: 2 dies x 74 SMs
+constexpr int kRemapRowsPerBlock = 224;    // 7 bitmap words per 32-byte remap block
+constexpr int kSortTile = 2048;            // keys per radix-sort tile (256 threads x 8)
+constexpr int kScanTile = 2048;            // elements per scan tile (256 threads x 8)
+constexpr int kSelTile = 4096;             // rows per hot-set selection tile (256 threads x 16)
+constexpr int kBwdChunk = 32;              // sorted lookups per backward chunk
+
+// One 32-byte sector per 224 rows: w[0] = number of popular rows before this block, w[1..7] = hit bitmap.
+struct __align__(32) RemapBlock {
+    uint32_t w[8];
+};
+
+// State of the count-threshold selection (device memory).
+struct SelectState {
+    unsigned long long hist[256];
+    unsigned long long k_remaining;    // rows still wanted among the current prefix class
+    unsigned long long quota_eq;       // rows with count == threshold to keep (in ascending id)
+    unsigned long long total;          // lookups counted so far
+    unsigned int prefix;               // high digits of the threshold found so far
+    unsigned int mask;                 // bits of `prefix` that are fixed
+    unsigned int c_min;                // smallest admissible count (>= 1)
+    unsigned int threshold;            // final: k-th largest admissible count
+    int take_all;                      // fewer admissible rows than wanted: keep them all
+};
+
+struct Regions {
+    // common
+    int32_t* status;                   // [8]  status[0] = first device error
+    int64_t* table_base;               // [T+1]
+    RemapBlock* remap;                 // [n_remap_blocks]
+    // profile
+    uint32_t* counts;                  // [N]
+    SelectState* sel;
+    uint32_t* sel_gt;                  // [n_sel_tiles + 1]
+    uint32_t* sel_eq;                  // [n_sel_tiles + 1]
+    // fragment
+    uint8_t* frag_flags;               // [max_batch]
+    int32_t* frag_scan;                // [max_bags + 1]
+    int32_t* frag_tiles;               // [scan tiles + 1]
+    // backward
+    int32_t* bwd_keys[2];              // [max_nnz]
+    int32_t* bwd_vals[2];              // [max_nnz]
+    uint32_t* bwd_hist;                // [256 * sort tiles]
+    float* bwd_part;                   // [2 * n_chunks * D]
+    int32_t* bwd_n;                    // [4] lookups in the micro-batch
+    // cold
+    int32_t* cold_keys[2];
+    int32_t* cold_vals[2];
+    uint32_t* cold_hist;
+    int32_t* cold_rank;                // [max_nnz + 1]
+    int32_t* cold_tiles;               // [scan tiles + 1]
+    int32_t* cold_n;                   // [4] cold lookups
+};
+
+}  // namespace hl
+
+struct hl_ctx {
+    int32_t T, D, S;
+    int64_t N;
+    int32_t max_batch;
+    int64_t max_nnz, max_bags;
+    int64_t hot_cap, staging_cap;
+    int64_t n_remap_blocks, n_sel_tiles;
+    int device;
+    int64_t* h_table_base;             // host copy [T+1]
+    hl::Regions r;
+};
+
+namespace hl {
+
+#define HL_CUDA_TRY(expr)                         \
+    do {                                          \
+        cudaError_t e__ = (expr);                 \
+        if (e__ != cudaSuccess) return HL_ECUDA;  \
+    } while (0)
+
+#define HL_LAUNCH_CHECK()                                  \
+    do {                                                   \
+        if (cudaGetLastError() != cudaSuccess) return HL_ECUDA; \
+    } while (0)
+
+__device__ __forceinline__ void set_status(int32_t* status, int32_t code) {
+    atomicCAS(status, 0, code);
+}
+
+// Hit test only: one 4-byte load.
+__device__ __forceinline__ bool remap_hit(const RemapBlock* __restrict__ remap, int64_t g) {
+    const uint32_t blk = (uint32_t)(g / kRemapRowsPerBlock);
+    const uint32_t r = (uint32_t)(g - (int64_t)blk * kRemapRowsPerBlock);
+    const uint32_t word = __ldg(&remap[blk].w[1 + (r >> 5)]);
+    return (word >> (r & 31)) & 1u;
+}
+
+// Slot of global row g, or -1: one 32-byte sector.
+__device__ __forceinline__ int32_t remap_slot(const RemapBlock* __restrict__ remap, int64_t g) {
+    const uint32_t blk = (uint32_t)(g / kRemapRowsPerBlock);
+    const uint32_t r = (uint32_t)(g - (int64_t)blk * kRemapRowsPerBlock);
+    const uint4 lo = __ldg(reinterpret_cast<const uint4*>(&remap[blk].w[0]));
+    const uint4 hi = __ldg(reinterpret_cast<const uint4*>(&remap[blk].w[4]));
+    const uint32_t w[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+    const uint32_t wi = 1 + (r >> 5), bit = r & 31;
+    uint32_t slot = w[0];
+    uint32_t word = 0;
+#pragma unroll
+    for (uint32_t i = 1; i < 8; ++i) {
+        if (i < wi) slot += __popc(w[i]);
+        if (i == wi) word = w[i];
+    }
+    if (!((word >> bit) & 1u)) return -1;
+    slot += __popc(word & ((1u << bit) - 1u));
+    return (int32_t)slot;
+}
+
+__device__ __forceinline__ unsigned lanemask_lt() {
+    unsigned m;
+    asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+    return m;
+}
+
+// ---- primitives implemented in hl_prims.cu -----------------------------------------------------------------
+// Exclusive scan of in[0 .. n) into out[0 .. n] (out[n] = total); n = *d_n if d_n != nullptr (clamped to
+// n_max), else n_max.  in may alias out.  tiles: scratch of n_max / kScanTile + 2 ints.
+int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, int64_t n_max, int32_t* tiles,
+                           cudaStream_t stream);
+
+// Stable LSD radix sort of (key, value) pairs by the low key_bits bits of the non-negative keys.
+// n = *d_n (clamped to n_max).  Returns in *out_keys / *out_vals which of the two buffers holds the result.
+int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n, int64_t n_max, int key_bits,
+                         uint32_t* hist, int32_t** out_keys, int32_t** out_vals, cudaStream_t stream);
+
+inline int64_t div_up(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline int grid_for(int64_t work_items, int per_block, int max_blocks) {
+    int64_t b = div_up(work_items, per_block);
+    if (b < 1) b = 1;
+    if (b > max_blocks) b = max_blocks;
+    return (int)b;
+}
+
+}  // namespace hl

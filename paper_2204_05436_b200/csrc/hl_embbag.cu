@@ -1,0 +1,436 @@
+// Embedding bag over the HBM cache: sum-pooling forward, and scatter-add + SGD backward with one update per
+// distinct row.  Rows are fp32 [*, D]; a group of G lanes owns one row at a time, each lane NV float4 columns,
+// so that a row is read with 128-bit loads that coalesce into whole sectors.
+#include "hl_common.cuh"
+
+namespace hl {
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ float4 f4_zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+__device__ __forceinline__ void f4_add(float4& a, const float4& b) {
+    a.x += b.x;
+    a.y += b.y;
+    a.z += b.z;
+    a.w += b.w;
+}
+
+__device__ __forceinline__ int clamp_samples(const int32_t* d_n_samples, int max_batch) {
+    int n = *d_n_samples;
+    if (n < 0) n = 0;
+    return n < max_batch ? n : max_batch;
+}
+
+// ---- forward ------------------------------------------------------------------------------------------------
+// Each group takes UB consecutive bags per trip and walks them in lock step, so that UB independent row loads
+// are in flight per lane.
+template <int G, int NV, int UB>
+__global__ void __launch_bounds__(kThreads) k_embbag_fwd(const float* __restrict__ cache,
+                                                         const int32_t* __restrict__ ids,
+                                                         const int32_t* __restrict__ offsets,
+                                                         const int32_t* __restrict__ d_n_samples, int max_batch,
+                                                         int bags_per_sample_all /* T*S */, int D4, int64_t n_slots,
+                                                         float* __restrict__ out, int32_t* status) {
+    const int64_t n_bags = (int64_t)clamp_samples(d_n_samples, max_batch) * bags_per_sample_all;
+    const int sub = threadIdx.x % G;
+    const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+    const int64_t n_groups = (int64_t)gridDim.x * kThreads / G;
+    const float4* __restrict__ rows = reinterpret_cast<const float4*>(cache);
+    float4* __restrict__ out4 = reinterpret_cast<float4*>(out);
+
+    for (int64_t bag0 = group * UB; bag0 < n_bags; bag0 += n_groups * UB) {
+        int32_t lo[UB], len[UB];
+        int32_t max_len = 0;
+#pragma unroll
+        for (int u = 0; u < UB; ++u) {
+            const int64_t bag = bag0 + u;
+            const bool valid = bag < n_bags;
+            lo[u] = valid ? __ldg(&offsets[bag]) : 0;
+            len[u] = valid ? __ldg(&offsets[bag + 1]) - lo[u] : 0;
+            max_len = max(max_len, len[u]);
+        }
+        // p-th lookup of each of the UB bags: UB independent row loads per lane
+        auto load_rows = [&](int32_t p, float4 (&r)[UB][NV]) {
+            int32_t id[UB];
+#pragma unroll
+            for (int u = 0; u < UB; ++u) id[u] = p < len[u] ? __ldg(&ids[lo[u] + p]) : -1;
+#pragma unroll
+            for (int u = 0; u < UB; ++u) {
+                const bool ok = id[u] >= 0 && id[u] < n_slots;
+                if (id[u] >= n_slots) set_status(status, HL_EBOUNDS);
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const int c = sub + v * G;
+                    r[u][v] = (ok && c < D4) ? __ldg(&rows[(int64_t)id[u] * D4 + c]) : f4_zero();
+                }
+            }
+        };
+        float4 first[UB][NV];
+        load_rows(0, first);
+        if (max_len <= 1) {
+            // bags of at most one lookup: the pooled vector is the row itself (or zeros), a plain copy
+#pragma unroll
+            for (int u = 0; u < UB; ++u) {
+                const int64_t bag = bag0 + u;
+                if (bag < n_bags) {
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        const int c = sub + v * G;
+                        if (c < D4) __stcs(&out4[bag * D4 + c], first[u][v]);
+                    }
+                }
+            }
+            continue;
+        }
+        // longer bags: add in lookup order in fp64 and round once, so that the result does not depend on
+        // cancellation between the rows of a bag
+        double acc[UB][NV][4];
+#pragma unroll
+        for (int u = 0; u < UB; ++u)
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                acc[u][v][0] = first[u][v].x;
+                acc[u][v][1] = first[u][v].y;
+                acc[u][v][2] = first[u][v].z;
+                acc[u][v][3] = first[u][v].w;
+            }
+        for (int32_t p = 1; p < max_len; ++p) {
+            float4 r[UB][NV];
+            load_rows(p, r);
+#pragma unroll
+            for (int u = 0; u < UB; ++u)
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    acc[u][v][0] += (double)r[u][v].x;
+                    acc[u][v][1] += (double)r[u][v].y;
+                    acc[u][v][2] += (double)r[u][v].z;
+                    acc[u][v][3] += (double)r[u][v].w;
+                }
+        }
+#pragma unroll
+        for (int u = 0; u < UB; ++u) {
+            const int64_t bag = bag0 + u;
+            if (bag < n_bags) {
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const int c = sub + v * G;
+                    if (c < D4)
+                        __stcs(&out4[bag * D4 + c], make_float4((float)acc[u][v][0], (float)acc[u][v][1],
+                                                               (float)acc[u][v][2], (float)acc[u][v][3]));
+                }
+            }
+        }
+    }
+}
+
+// ---- backward -----------------------------------------------------------------------------------------------
+// (slot, bag) pair per lookup; a negative id becomes the sentinel n_slots, which sorts last and is ignored.
+template <int GROUP>
+__global__ void __launch_bounds__(kThreads) k_bwd_pairs(const int32_t* __restrict__ ids,
+                                                        const int32_t* __restrict__ offsets,
+                                                        const int32_t* __restrict__ d_n_samples, int max_batch,
+                                                        int bags_per_sample_all, int64_t n_slots, int64_t max_nnz,
+                                                        int32_t* __restrict__ keys, int32_t* __restrict__ vals,
+                                                        int32_t* __restrict__ d_n_lookups, int32_t* status) {
+    const int64_t n_bags = (int64_t)clamp_samples(d_n_samples, max_batch) * bags_per_sample_all;
+    const int sub = threadIdx.x % GROUP;
+    const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / GROUP;
+    const int64_t n_groups = (int64_t)gridDim.x * kThreads / GROUP;
+    if (group == 0 && sub == 0) {
+        int32_t L = offsets[n_bags];
+        if (L > max_nnz) {
+            set_status(status, HL_ECAPACITY);
+            L = (int32_t)max_nnz;
+        }
+        d_n_lookups[0] = L;
+    }
+    for (int64_t bag = group; bag < n_bags; bag += n_groups) {
+        const int32_t lo = offsets[bag], hi = offsets[bag + 1];
+        for (int32_t j = lo + sub; j < hi; j += GROUP) {
+            if (j >= max_nnz) break;
+            const int32_t id = ids[j];
+            if (id >= n_slots) set_status(status, HL_EBOUNDS);
+            keys[j] = (id < 0 || id >= n_slots) ? (int32_t)n_slots : id;
+            vals[j] = (int32_t)bag;
+        }
+    }
+}
+
+template <int G, int NV>
+struct RowOps {
+    // cache[key, :] -= lr * acc  (this group's columns)
+    static __device__ __forceinline__ void sgd(float* cache, int64_t key, int D4, int sub, float lr,
+                                               const float4 (&acc)[NV]) {
+        float4* row = reinterpret_cast<float4*>(cache) + key * D4;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int c = sub + v * G;
+            if (c < D4) {
+                float4 w = row[c];
+                w.x -= lr * acc[v].x;
+                w.y -= lr * acc[v].y;
+                w.z -= lr * acc[v].z;
+                w.w -= lr * acc[v].w;
+                row[c] = w;
+            }
+        }
+    }
+};
+
+// The sorted lookups are cut into chunks of kBwdChunk.  One group per chunk sums, in order, the gradient rows of
+// each run of equal slots inside its chunk.  A run that lies wholly inside the chunk is finished here (one
+// read-modify-write of its row).  A run that crosses a chunk border leaves a partial sum: part[chunk][0] for the
+// piece that continues a run from the previous chunk, part[chunk][1] for the piece that starts a run continuing
+// into the next chunk.  k_bwd_spans adds those up.
+template <int G, int NV>
+__global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cache,
+                                                         const int32_t* __restrict__ keys,
+                                                         const int32_t* __restrict__ vals,
+                                                         const int32_t* __restrict__ d_n_lookups,
+                                                         const float* __restrict__ grad_out, int D4, int64_t n_slots,
+                                                         float lr, float* __restrict__ part) {
+    constexpr int U = NV >= 8 ? 1 : (NV >= 4 ? 2 : (NV >= 2 ? 4 : 8));
+    const int64_t n = d_n_lookups[0];
+    const int sub = threadIdx.x % G;
+    const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+    const int64_t n_groups = (int64_t)gridDim.x * kThreads / G;
+    const float4* __restrict__ grad4 = reinterpret_cast<const float4*>(grad_out);
+    float4* __restrict__ part4 = reinterpret_cast<float4*>(part);
+
+    for (int64_t chunk = group; chunk * kBwdChunk < n; chunk += n_groups) {
+        const int64_t start = chunk * kBwdChunk;
+        const int64_t end = min(start + (int64_t)kBwdChunk, n);
+        int32_t cur = keys[start];
+        bool seg_left_open = start > 0 && keys[start - 1] == cur;
+        float4 acc[NV];
+#pragma unroll
+        for (int v = 0; v < NV; ++v) acc[v] = f4_zero();
+
+        auto flush = [&](bool right_open) {
+            if (cur >= n_slots) return;   // sentinel: lookups that were skipped
+            if (!seg_left_open && !right_open) {
+                RowOps<G, NV>::sgd(cache, cur, D4, sub, lr, acc);
+            } else {
+                const int64_t slot = chunk * 2 + (seg_left_open ? 0 : 1);
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const int c = sub + v * G;
+                    if (c < D4) part4[slot * D4 + c] = acc[v];
+                }
+            }
+        };
+
+        for (int64_t p0 = start; p0 < end; p0 += U) {
+            int32_t k[U], b[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const bool valid = p0 + u < end;
+                k[u] = valid ? keys[p0 + u] : -1;
+                b[u] = valid ? vals[p0 + u] : 0;
+            }
+            float4 g[U][NV];
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const int c = sub + v * G;
+                    g[u][v] = (k[u] >= 0 && k[u] < n_slots && c < D4) ? __ldg(&grad4[(int64_t)b[u] * D4 + c])
+                                                                      : f4_zero();
+                }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (p0 + u < end) {
+                    if (k[u] != cur) {
+                        flush(false);
+#pragma unroll
+                        for (int v = 0; v < NV; ++v) acc[v] = f4_zero();
+                        cur = k[u];
+                        seg_left_open = false;
+                    }
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) f4_add(acc[v], g[u][v]);
+                }
+            }
+        }
+        flush(end < n && keys[end] == cur);
+    }
+}
+
+// One group per chunk; it acts only if a run STARTS in its chunk and continues into the next one.  It finds the
+// run's end by a galloping search over the sorted keys, adds the continuation pieces in chunk order, and applies
+// the single SGD update of that row.
+template <int G, int NV>
+__global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cache, const int32_t* __restrict__ keys,
+                                                        const int32_t* __restrict__ d_n_lookups, int D4,
+                                                        int64_t n_slots, float lr, const float* __restrict__ part) {
+    const int64_t n = d_n_lookups[0];
+    const int sub = threadIdx.x % G;
+    const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+    const int64_t n_groups = (int64_t)gridDim.x * kThreads / G;
+    const float4* __restrict__ part4 = reinterpret_cast<const float4*>(part);
+
+    for (int64_t chunk = group; chunk * kBwdChunk < n; chunk += n_groups) {
+        const int64_t start = chunk * kBwdChunk;
+        const int64_t end = min(start + (int64_t)kBwdChunk, n);
+        if (end >= n) continue;
+        const int32_t key = keys[end - 1];
+        if (key >= n_slots || keys[end] != key) continue;                        // not right-open
+        if (keys[start] == key && start > 0 && keys[start - 1] == key) continue;   // run started earlier
+
+        // e = one past the run's last lookup
+        int64_t lo = end, hi, step = kBwdChunk;
+        for (;;) {
+            hi = lo + step;
+            if (hi >= n) {
+                hi = n;
+                break;
+            }
+            if (keys[hi] != key) break;
+            lo = hi;
+            step <<= 1;
+        }
+        while (hi - lo > 1) {
+            const int64_t mid = (lo + hi) >> 1;
+            if (keys[mid] == key) lo = mid;
+            else hi = mid;
+        }
+        const int64_t last_chunk = (hi - 1) / kBwdChunk;
+
+        // the pieces of one run are added in chunk order in fp64 (runs of many thousands of lookups occur)
+        double dacc[NV][4];
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int c = sub + v * G;
+            const float4 t = c < D4 ? part4[(chunk * 2 + 1) * D4 + c] : f4_zero();
+            dacc[v][0] = t.x;
+            dacc[v][1] = t.y;
+            dacc[v][2] = t.z;
+            dacc[v][3] = t.w;
+        }
+        int64_t c2 = chunk + 1;
+        for (; c2 + 3 <= last_chunk; c2 += 4) {
+            float4 t[4][NV];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const int c = sub + v * G;
+                    t[u][v] = c < D4 ? part4[((c2 + u) * 2) * D4 + c] : f4_zero();
+                }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    dacc[v][0] += (double)t[u][v].x;
+                    dacc[v][1] += (double)t[u][v].y;
+                    dacc[v][2] += (double)t[u][v].z;
+                    dacc[v][3] += (double)t[u][v].w;
+                }
+        }
+        for (; c2 <= last_chunk; ++c2)
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int c = sub + v * G;
+                if (c < D4) {
+                    const float4 t = part4[(c2 * 2) * D4 + c];
+                    dacc[v][0] += (double)t.x;
+                    dacc[v][1] += (double)t.y;
+                    dacc[v][2] += (double)t.z;
+                    dacc[v][3] += (double)t.w;
+                }
+            }
+        float4 acc[NV];
+#pragma unroll
+        for (int v = 0; v < NV; ++v)
+            acc[v] = make_float4((float)dacc[v][0], (float)dacc[v][1], (float)dacc[v][2], (float)dacc[v][3]);
+        RowOps<G, NV>::sgd(cache, key, D4, sub, lr, acc);
+    }
+}
+
+template <int G, int NV>
+int32_t launch_fwd(hl_ctx* ctx, const float* cache, const hl_ubatch* ub, const int32_t* d_n, float* out,
+                   cudaStream_t stream) {
+    constexpr int UB = NV >= 8 ? 1 : (NV >= 4 ? 2 : 4);
+    const int64_t max_bags = ctx->max_bags;
+    const int grid = grid_for(div_up(max_bags, UB) * G, kThreads, kSMs * 8);
+    k_embbag_fwd<G, NV, UB><<<grid, kThreads, 0, stream>>>(cache, ub->ids, ub->offsets, d_n, ctx->max_batch,
+                                                          ctx->T * ctx->S, ctx->D / 4,
+                                                          ctx->hot_cap + ctx->staging_cap, out, ctx->r.status);
+    HL_LAUNCH_CHECK();
+    return HL_OK;
+}
+
+template <int G, int NV>
+int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t* vals, const float* grad, float lr,
+                   cudaStream_t stream) {
+    const int64_t max_chunks = div_up(ctx->max_nnz, kBwdChunk);
+    const int grid = grid_for(max_chunks * G, kThreads, kSMs * 8);
+    const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
+    k_bwd_chunks<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, vals, ctx->r.bwd_n, grad, ctx->D / 4, n_slots,
+                                                      lr, ctx->r.bwd_part);
+    k_bwd_spans<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, ctx->r.bwd_n, ctx->D / 4, n_slots, lr,
+                                                     ctx->r.bwd_part);
+    HL_LAUNCH_CHECK();
+    return HL_OK;
+}
+
+int bits_for(int64_t max_value) {
+    int b = 1;
+    while ((int64_t(1) << b) <= max_value) ++b;
+    return b;
+}
+
+}  // namespace
+}  // namespace hl
+
+using namespace hl;
+
+#define HL_DISPATCH_ROW_SHAPE(D4, CALL)                  \
+    do {                                                 \
+        if ((D4) <= 4) return CALL(4, 1);                \
+        if ((D4) <= 8) return CALL(8, 1);                \
+        if ((D4) <= 16) return CALL(16, 1);              \
+        if ((D4) <= 32) return CALL(32, 1);              \
+        if ((D4) <= 64) return CALL(32, 2);              \
+        if ((D4) <= 128) return CALL(32, 4);             \
+        if ((D4) <= 256) return CALL(32, 8);             \
+        return HL_EINVAL;                                \
+    } while (0)
+
+extern "C" int32_t hl_embbag_fwd(hl_ctx* ctx, const float* d_cache, const hl_ubatch* ub, const int32_t* d_n_samples,
+                                 float* d_out, void* stream_) {
+    if (!ctx || !d_cache || !ub || !ub->offsets || !d_n_samples || !d_out) return HL_EINVAL;
+    if (ctx->max_nnz > 0 && !ub->ids) return HL_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+#define HL_FWD(G, NV) launch_fwd<G, NV>(ctx, d_cache, ub, d_n_samples, d_out, stream)
+    HL_DISPATCH_ROW_SHAPE(ctx->D / 4, HL_FWD);
+#undef HL_FWD
+}
+
+extern "C" int32_t hl_embbag_bwd_sgd(hl_ctx* ctx, float* d_cache, const hl_ubatch* ub, const int32_t* d_n_samples,
+                                     const float* d_grad_out, float lr, void* stream_) {
+    if (!ctx || !d_cache || !ub || !ub->offsets || !d_n_samples || !d_grad_out) return HL_EINVAL;
+    if (ctx->max_nnz == 0) return HL_OK;
+    if (!ub->ids) return HL_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Regions& r = ctx->r;
+    const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
+    const bool short_bags = ctx->max_nnz <= 4 * ctx->max_bags;
+    if (short_bags)
+        k_bwd_pairs<1><<<grid_for(ctx->max_bags, kThreads, kSMs * 8), kThreads, 0, stream>>>(
+            ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, r.bwd_keys[0],
+            r.bwd_vals[0], r.bwd_n, r.status);
+    else
+        k_bwd_pairs<32><<<grid_for(ctx->max_bags, kThreads / 32, kSMs * 8), kThreads, 0, stream>>>(
+            ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, r.bwd_keys[0],
+            r.bwd_vals[0], r.bwd_n, r.status);
+    HL_LAUNCH_CHECK();
+    int32_t *keys, *vals;
+    int32_t st = radix_sort_pairs(r.bwd_keys, r.bwd_vals, r.bwd_n, ctx->max_nnz, bits_for(n_slots), r.bwd_hist,
+                                  &keys, &vals, stream);
+    if (st != HL_OK) return st;
+#define HL_BWD(G, NV) launch_bwd<G, NV>(ctx, d_cache, keys, vals, d_grad_out, lr, stream)
+    HL_DISPATCH_ROW_SHAPE(ctx->D / 4, HL_BWD);
+#undef HL_BWD
+}

@@ -1,0 +1,269 @@
+// Fragmenting a mini-batch into the popular micro-batch O and the non-popular micro-batch X.
+//
+//   1. k_frag_flags     one warp per input: probe the popular-row bitmap for every lookup of the input,
+//                       all-hit decided by a warp vote
+//   2. k_frag_partition one block: ballot + prefix sums over the flags -> stable partition `perm`, n_pop
+//   3. k_frag_sizes     size of every destination bag (O's bags, then X's bags), then an exclusive scan
+//   4. k_frag_emit      copy every bag's lookups to its place, mapped to a cache slot (O) or global row (X)
+#include "hl_common.cuh"
+
+namespace hl {
+namespace {
+
+constexpr int kThreads = 256;
+
+// LANE_PER_TABLE: lane l walks the lookups of tables l, l+32, ... of its input (short bags: pooling 1).
+// otherwise the warp walks table after table with the lanes striding over the table's lookups of the input
+// (its S bags are contiguous in the table-major layout).
+template <bool LANE_PER_TABLE>
+__global__ void __launch_bounds__(kThreads) k_frag_flags(const int32_t* __restrict__ indices,
+                                                         const int32_t* __restrict__ offsets, int B, int T, int S,
+                                                         const int64_t* __restrict__ table_base,
+                                                         const RemapBlock* __restrict__ remap,
+                                                         uint8_t* __restrict__ flags, int32_t* status) {
+    const int lane = threadIdx.x & 31;
+    const int warps_per_block = kThreads / 32;
+    for (int b = blockIdx.x * warps_per_block + (threadIdx.x >> 5); b < B; b += gridDim.x * warps_per_block) {
+        bool miss = false;
+        if (LANE_PER_TABLE) {
+            for (int t = lane; t < T; t += 32) {
+                const int64_t first_bag = ((int64_t)t * B + b) * S;
+                const int32_t lo = offsets[first_bag], hi = offsets[first_bag + S];
+                const int64_t base = table_base[t], rows = table_base[t + 1] - base;
+                for (int32_t j = lo; j < hi; ++j) {
+                    const int32_t idx = indices[j];
+                    if (idx < 0 || idx >= rows) {
+                        set_status(status, HL_EBOUNDS);
+                        miss = true;
+                    } else if (!remap_hit(remap, base + idx)) {
+                        miss = true;
+                    }
+                }
+            }
+        } else {
+            for (int t = 0; t < T; ++t) {
+                const int64_t first_bag = ((int64_t)t * B + b) * S;
+                const int32_t lo = offsets[first_bag], hi = offsets[first_bag + S];
+                const int64_t base = table_base[t], rows = table_base[t + 1] - base;
+                for (int32_t j = lo + lane; j < hi; j += 32) {
+                    const int32_t idx = indices[j];
+                    if (idx < 0 || idx >= rows) {
+                        set_status(status, HL_EBOUNDS);
+                        miss = true;
+                    } else if (!remap_hit(remap, base + idx)) {
+                        miss = true;
+                    }
+                }
+            }
+        }
+        const unsigned any_miss = __ballot_sync(0xffffffffu, miss);
+        if (lane == 0) flags[b] = any_miss == 0;
+    }
+}
+
+// One block of 1024 threads.  Pass 1 counts the popular inputs; pass 2 places every input: a popular one at
+// its rank among the popular, a non-popular one behind all popular ones at its rank among the non-popular.
+__global__ void __launch_bounds__(1024) k_frag_partition(const uint8_t* __restrict__ flags, int B,
+                                                         int32_t* __restrict__ perm, int32_t* __restrict__ counts) {
+    __shared__ int warp_sum[32];
+    __shared__ int s_total;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned lt = lanemask_lt();
+
+    int mine = 0;
+    for (int b = threadIdx.x; b < B; b += 1024) mine += flags[b];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, d);
+    if (lane == 0) warp_sum[warp] = mine;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int s = 0;
+        for (int w = 0; w < 32; ++w) s += warp_sum[w];
+        s_total = s;
+    }
+    __syncthreads();
+    const int n_pop = s_total;
+    __syncthreads();
+
+    int before = 0;   // popular inputs in earlier chunks
+    for (int start = 0; start < B; start += 1024) {
+        const int b = start + threadIdx.x;
+        const bool valid = b < B;
+        const bool pop = valid && flags[b];
+        const unsigned vote = __ballot_sync(0xffffffffu, pop);
+        if (lane == 0) warp_sum[warp] = __popc(vote);
+        __syncthreads();
+        if (warp == 0) {
+            const int c = warp_sum[lane];
+            int incl = c;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                int o = __shfl_up_sync(0xffffffffu, incl, d);
+                if (lane >= d) incl += o;
+            }
+            warp_sum[lane] = incl - c;
+            if (lane == 31) s_total = incl;
+        }
+        __syncthreads();
+        if (valid) {
+            const int rank_pop = before + warp_sum[warp] + __popc(vote & lt);   // popular inputs before b
+            if (pop) perm[rank_pop] = b;
+            else perm[n_pop + (b - rank_pop)] = b;
+        }
+        before += s_total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        counts[0] = n_pop;
+        counts[1] = B - n_pop;
+    }
+}
+
+struct DestBag {
+    int64_t src_bag;
+    int t;
+    bool is_pop;
+};
+
+// Destination bags: O's T*l*S bags, then X's T*k*S bags, each table-major over the micro-batch's inputs.
+__device__ __forceinline__ DestBag decode_dest_bag(int64_t dst, int B, int S, int n_pop, int64_t pop_bags,
+                                                   const int32_t* __restrict__ perm) {
+    DestBag d;
+    d.is_pop = dst < pop_bags;
+    const int64_t local = d.is_pop ? dst : dst - pop_bags;
+    const int n = d.is_pop ? n_pop : B - n_pop;
+    const int64_t per_table = (int64_t)n * S;
+    d.t = (int)(local / per_table);
+    const int64_t rem = local - (int64_t)d.t * per_table;
+    const int i = (int)(rem / S), s = (int)(rem - (int64_t)i * S);
+    const int b = perm[(d.is_pop ? 0 : n_pop) + i];
+    d.src_bag = ((int64_t)d.t * B + b) * S + s;
+    return d;
+}
+
+__global__ void __launch_bounds__(kThreads) k_frag_sizes(const int32_t* __restrict__ offsets, int B, int T, int S,
+                                                         const int32_t* __restrict__ perm,
+                                                         const int32_t* __restrict__ counts,
+                                                         int32_t* __restrict__ sizes) {
+    const int n_pop = counts[0];
+    const int64_t n_bags = (int64_t)T * B * S, pop_bags = (int64_t)T * n_pop * S;
+    for (int64_t dst = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; dst < n_bags;
+         dst += (int64_t)gridDim.x * blockDim.x) {
+        const DestBag d = decode_dest_bag(dst, B, S, n_pop, pop_bags, perm);
+        sizes[dst] = offsets[d.src_bag + 1] - offsets[d.src_bag];
+    }
+}
+
+// GROUP lanes cooperate on one destination bag (1 for short bags, 32 for long ones).
+template <int GROUP>
+__global__ void __launch_bounds__(kThreads) k_frag_emit(const int32_t* __restrict__ indices,
+                                                        const int32_t* __restrict__ offsets, int B, int T, int S,
+                                                        const int32_t* __restrict__ perm,
+                                                        int32_t* __restrict__ counts,
+                                                        const int32_t* __restrict__ dst_start,   // scanned sizes
+                                                        const int64_t* __restrict__ table_base,
+                                                        const RemapBlock* __restrict__ remap,
+                                                        int32_t* __restrict__ pop_offsets, int32_t* __restrict__ pop_ids,
+                                                        int64_t pop_cap, int32_t* __restrict__ non_offsets,
+                                                        int32_t* __restrict__ non_ids, int64_t non_cap,
+                                                        int32_t* status) {
+    const int n_pop = counts[0];
+    const int64_t n_bags = (int64_t)T * B * S, pop_bags = (int64_t)T * n_pop * S;
+    const int32_t L_pop = dst_start[pop_bags], L_all = dst_start[n_bags];
+    const int sub = threadIdx.x % GROUP;
+    const int64_t group = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / GROUP;
+    const int64_t n_groups = (int64_t)gridDim.x * blockDim.x / GROUP;
+    if (group == 0 && sub == 0) {
+        counts[2] = L_pop;
+        counts[3] = L_all - L_pop;
+        pop_offsets[pop_bags] = L_pop;
+        non_offsets[n_bags - pop_bags] = L_all - L_pop;
+    }
+    for (int64_t dst = group; dst < n_bags; dst += n_groups) {
+        const DestBag d = decode_dest_bag(dst, B, S, n_pop, pop_bags, perm);
+        const int32_t src_lo = offsets[d.src_bag], src_hi = offsets[d.src_bag + 1];
+        const int64_t base = table_base[d.t], rows = table_base[d.t + 1] - base;
+        if (d.is_pop) {
+            const int32_t out_lo = dst_start[dst];
+            if (sub == 0) pop_offsets[dst] = out_lo;
+            for (int32_t j = sub; j < src_hi - src_lo; j += GROUP) {
+                if (out_lo + j >= pop_cap) {
+                    set_status(status, HL_ECAPACITY);
+                    break;
+                }
+                const int32_t idx = indices[src_lo + j];
+                // every lookup of a popular input was tested to be in range and popular
+                pop_ids[out_lo + j] = remap_slot(remap, base + idx);
+            }
+        } else {
+            const int32_t out_lo = dst_start[dst] - L_pop;
+            if (sub == 0) non_offsets[dst - pop_bags] = out_lo;
+            for (int32_t j = sub; j < src_hi - src_lo; j += GROUP) {
+                if (out_lo + j >= non_cap) {
+                    set_status(status, HL_ECAPACITY);
+                    break;
+                }
+                const int32_t idx = indices[src_lo + j];
+                non_ids[out_lo + j] = (idx < 0 || idx >= rows) ? -1 : (int32_t)(base + idx);
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(kThreads) k_permute_dense(const float* __restrict__ dense, int B, int n_dense,
+                                                            const int32_t* __restrict__ perm,
+                                                            float* __restrict__ out) {
+    const int64_t total = (int64_t)B * n_dense;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int i = (int)(e / n_dense), c = (int)(e - (int64_t)i * n_dense);
+        out[e] = dense[(int64_t)perm[i] * n_dense + c];
+    }
+}
+
+}  // namespace
+}  // namespace hl
+
+using namespace hl;
+
+extern "C" int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_dense, int32_t n_dense,
+                               int32_t* d_perm, int32_t* d_counts, hl_ubatch* pop, hl_ubatch* non,
+                               float* d_dense_out, void* stream_) {
+    if (!ctx || !b || !d_perm || !d_counts || !pop || !non) return HL_EINVAL;
+    if (b->batch < 1 || b->batch > ctx->max_batch || b->nnz < 0 || b->nnz > ctx->max_nnz || !b->offsets ||
+        (b->nnz > 0 && !b->indices))
+        return HL_EINVAL;
+    if (!pop->offsets || !non->offsets || (b->nnz > 0 && (!pop->ids || !non->ids))) return HL_EINVAL;
+    if ((d_dense == nullptr) != (d_dense_out == nullptr) || (d_dense && n_dense < 1)) return HL_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Regions& r = ctx->r;
+    const int B = b->batch, T = ctx->T, S = ctx->S;
+    const int64_t n_bags = (int64_t)T * B * S;
+    const bool short_bags = b->nnz <= 4 * (int64_t)T * B;   // on average at most 4 lookups per input and table
+
+    const int flag_grid = grid_for(B, kThreads / 32, kSMs * 16);
+    if (short_bags)
+        k_frag_flags<true><<<flag_grid, kThreads, 0, stream>>>(b->indices, b->offsets, B, T, S, r.table_base,
+                                                               r.remap, r.frag_flags, r.status);
+    else
+        k_frag_flags<false><<<flag_grid, kThreads, 0, stream>>>(b->indices, b->offsets, B, T, S, r.table_base,
+                                                                r.remap, r.frag_flags, r.status);
+    k_frag_partition<<<1, 1024, 0, stream>>>(r.frag_flags, B, d_perm, d_counts);
+    k_frag_sizes<<<grid_for(n_bags, kThreads, kSMs * 8), kThreads, 0, stream>>>(b->offsets, B, T, S, d_perm,
+                                                                               d_counts, r.frag_scan);
+    HL_LAUNCH_CHECK();
+    int32_t st = exclusive_scan_i32(r.frag_scan, r.frag_scan, nullptr, n_bags, r.frag_tiles, stream);
+    if (st != HL_OK) return st;
+    if (b->nnz <= 4 * n_bags)
+        k_frag_emit<1><<<grid_for(n_bags, kThreads, kSMs * 8), kThreads, 0, stream>>>(
+            b->indices, b->offsets, B, T, S, d_perm, d_counts, r.frag_scan, r.table_base, r.remap, pop->offsets,
+            pop->ids, pop->cap_ids, non->offsets, non->ids, non->cap_ids, r.status);
+    else
+        k_frag_emit<32><<<grid_for(n_bags, kThreads / 32, kSMs * 8), kThreads, 0, stream>>>(
+            b->indices, b->offsets, B, T, S, d_perm, d_counts, r.frag_scan, r.table_base, r.remap, pop->offsets,
+            pop->ids, pop->cap_ids, non->offsets, non->ids, non->cap_ids, r.status);
+    if (d_dense)
+        k_permute_dense<<<grid_for((int64_t)B * n_dense, kThreads, kSMs * 8), kThreads, 0, stream>>>(
+            d_dense, B, n_dense, d_perm, d_dense_out);
+    HL_LAUNCH_CHECK();
+    return HL_OK;
+}

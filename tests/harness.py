@@ -1,0 +1,210 @@
+"""Runs one synthetic workload through the CUDA library and through the CPU oracle, call by call, and compares.
+
+Integer outputs (hot set, remap, perm, counts, micro-batch CSRs, cold rows, unified slots) must match bit for
+bit; fp32 outputs (pooled vectors, updated rows) within rtol 1e-5 / atol 1e-6, the tolerance the benchmark spec states.
+The oracle never sees a value produced by the CUDA path: both start from the same generated inputs.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import gen
+from oracle import hotline_oracle as orc
+
+RTOL, ATOL = 1e-5, 1e-6
+
+
+def _t(x, device):
+    return torch.from_numpy(np.ascontiguousarray(x)).to(device)
+
+
+def max_nnz_of(spec: gen.WorkloadSpec, geom: gen.Geometry, batch: int) -> int:
+    bags = geom.num_tables * batch * geom.bags_per_sample
+    return bags if spec.pooling[0] == "one" else bags * int(spec.pooling[2])
+
+
+def mu_grad(grad_full, samples, T, B, S):
+    """Rows of the whole-batch gradient that belong to a micro-batch's bags, in the micro-batch's bag order."""
+    samples = np.asarray(samples, dtype=np.int64)
+    src = ((np.arange(T)[:, None, None] * B + samples[None, :, None]) * S + np.arange(S)[None, None, :]).reshape(-1)
+    return grad_full[src], src
+
+
+def policy_args(policy):
+    import paper_2204_05436_b200 as hl
+    if policy[0] == "topk":
+        return hl.HL_HOT_TOPK_ROWS, int(policy[1]), 1
+    if policy[0] == "budget":
+        return hl.HL_HOT_BUDGET_BYTES, int(policy[1]), 1
+    if policy[0] == "fraction":
+        return hl.HL_HOT_FRACTION_ROWS, int(policy[1]), int(policy[2])
+    if policy[0] == "share":
+        return hl.HL_HOT_MIN_SHARE, int(policy[1]), int(policy[2])
+    raise ValueError(policy)
+
+
+def assert_close(got, want, what):
+    np.testing.assert_allclose(got, want, rtol=RTOL, atol=ATOL, err_msg=what)
+
+
+def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: bool = False, hot_override=None,
+                     deferred: bool = False, overlap: bool = True, profile_batches=None, verbose: bool = False,
+                     device: str = "cuda:0", resync: bool = True):
+    """Profiles, builds the remap, then runs ``steps`` mini-batches: the first call by call with a comparison
+    after every call, the others through Hotline.step().  ``hot_override``: None (profiled), "empty", "full",
+    or ("random", fraction).  With ``resync`` every step after the first starts from the oracle's tables
+    (copied to the device and the host table), so that each step is a parity check on identical inputs; without
+    it the two sides drift apart by their accumulated fp32 rounding.  Returns a dict of workload statistics."""
+    import paper_2204_05436_b200 as hl
+
+    if isinstance(spec, str):
+        spec = gen.CONFIGS[spec]
+    geom = gen.make_geometry(spec, scale_rows)
+    T, D, S, B = geom.num_tables, geom.dim, geom.bags_per_sample, spec.batch
+    N = geom.total_rows
+    n_bags = T * B * S
+    P = spec.profile_batches if profile_batches is None else profile_batches
+    lr = 0.125 if integer else spec.lr
+    max_nnz = max_nnz_of(spec, geom, B)
+    K = N if spec.hot_policy[0] == "share" else orc.hot_capacity(spec.hot_policy, N, D)
+    hot_cap = max(1, min(K, N))
+    staging_cap = max(1, min(N, max_nnz))
+
+    table0 = gen.table_values(np.arange(N), D, spec.seed, integer=integer)
+    host_table = torch.from_numpy(table0.copy()).pin_memory()
+    h = hl.Hotline(geom.table_rows, D, S, B, max_nnz, hot_cap, staging_cap, host_table, n_dense=spec.n_dense,
+                   device=device)
+    stats = {}
+    try:
+        with torch.cuda.stream(h.main):
+            # ---------------- learning phase ----------------
+            prof = [gen.make_batch(spec, geom, i) for i in range(P)]
+            cnt = orc.access_counts([(b.indices, b.offsets) for b in prof], B, geom.table_rows, S)
+            if hot_override is None:
+                min_share = (spec.hot_policy[1], spec.hot_policy[2]) if spec.hot_policy[0] == "share" else None
+                k_sel = hot_cap if spec.hot_policy[0] == "share" else min(K, hot_cap)
+                hot_o = orc.select_hot(cnt, k_sel, min_share)
+                pol, p_num, p_den = policy_args(spec.hot_policy)
+                for i, b in enumerate(prof):
+                    h.profile(_t(b.indices, device), _t(b.offsets, device), B, reset=(i == 0))
+                h.profile(None, None, reset=(P == 0), finalize=True, policy=pol, p_num=p_num, p_den=p_den)
+                h.status()
+                n_hot = int(h.n_hot.item())
+                assert n_hot == len(hot_o), ("n_hot", n_hot, len(hot_o))
+                assert np.array_equal(h.hot_rows[:n_hot].cpu().numpy(), hot_o.astype(np.int32)), "hot_rows"
+            else:
+                rng = np.random.default_rng(spec.seed + 99)
+                if hot_override == "empty":
+                    hot_o = np.zeros(0, dtype=np.int64)
+                elif hot_override == "full":
+                    hot_o = np.arange(min(N, hot_cap), dtype=np.int64)
+                else:
+                    hot_o = np.sort(rng.choice(N, int(min(hot_cap, N * hot_override[1])), replace=False)).astype(np.int64)
+                h.set_hot_rows(_t(hot_o, device))
+                n_hot = len(hot_o)
+            remap_o = orc.build_remap(hot_o, N)
+            remap_g = torch.empty(N, dtype=torch.int32, device=device)
+            h.build_remap(load_rows=True, remap_out=remap_g)
+            h.status()
+            assert np.array_equal(remap_g.cpu().numpy(), remap_o), "remap"
+            cache_o = np.zeros((hot_cap + staging_cap, D), dtype=np.float32)
+            cache_o[:n_hot] = orc.load_hot_cache(table0, hot_o)
+            assert np.array_equal(h.cache[:n_hot].cpu().numpy().view(np.uint32), cache_o[:n_hot].view(np.uint32)), "cache"
+            table_o = table0.copy()
+
+            # ---------------- acceleration phase ----------------
+            for step in range(steps):
+                bid = P + step
+                if step > 0 and resync:
+                    h.cache.copy_(_t(cache_o, device))
+                    h.host_table.copy_(torch.from_numpy(table_o))
+                    torch.cuda.synchronize()
+                batch = gen.make_batch(spec, geom, bid)
+                grad_full = gen.grad_values(spec.seed, bid, 2, n_bags, D, integer=integer)
+                perm_o, n_pop_o, O, X, dense_o = orc.fragment(batch.indices, batch.offsets, B, geom.table_rows, remap_o, S,
+                                                              batch.dense)
+                g_pop, _ = mu_grad(grad_full, perm_o[:n_pop_o], T, B, S)
+                g_non, _ = mu_grad(grad_full, perm_o[n_pop_o:], T, B, S)
+                out = orc.hotline_step(table_o, cache_o, hot_cap, remap_o, batch.indices, batch.offsets, B,
+                                       geom.table_rows, S, g_pop, g_non, lr, deferred=deferred)
+                _, _, _, X_slots, C, pooled_pop_o, pooled_non_o = out
+                n_non_o = B - n_pop_o
+                bags_pop, bags_non = T * n_pop_o * S, T * n_non_o * S
+
+                d_idx, d_off = _t(batch.indices, device), _t(batch.offsets, device)
+                d_dense = _t(batch.dense, device) if batch.dense is not None else None
+                d_gpop = torch.zeros((n_bags, D), dtype=torch.float32, device=device)
+                d_gnon = torch.zeros((n_bags, D), dtype=torch.float32, device=device)
+                d_gpop[:bags_pop] = _t(g_pop, device)
+                d_gnon[:bags_non] = _t(g_non, device)
+                torch.cuda.synchronize()
+
+                def check_fragment():
+                    counts = h.counts.cpu().numpy()
+                    assert counts.tolist() == [n_pop_o, n_non_o, len(O.ids), len(X.ids)], ("counts", counts.tolist())
+                    assert np.array_equal(h.perm[:B].cpu().numpy(), perm_o), "perm"
+                    assert np.array_equal(h.pop_offsets[:bags_pop + 1].cpu().numpy(), O.offsets), "pop offsets"
+                    assert np.array_equal(h.pop_ids[:len(O.ids)].cpu().numpy(), O.ids), "pop slots"
+                    assert np.array_equal(h.non_offsets[:bags_non + 1].cpu().numpy(), X.offsets), "non offsets"
+                    if dense_o is not None:
+                        assert np.array_equal(h.dense_out[:B].cpu().numpy().view(np.uint32), dense_o.view(np.uint32)), "dense"
+
+                def check_gather():
+                    assert int(h.n_cold.item()) == len(C), ("n_cold", int(h.n_cold.item()), len(C))
+                    assert np.array_equal(h.cold_rows[:len(C)].cpu().numpy(), C.astype(np.int32)), "cold rows"
+                    assert np.array_equal(h.non_ids[:len(X.ids)].cpu().numpy(), X_slots.ids), "non slots"
+
+                if step == 0:
+                    if True:
+                        h.fragment(d_idx, d_off, B, d_dense)
+                        h.status()
+                        check_fragment()
+                        assert np.array_equal(h.non_ids[:len(X.ids)].cpu().numpy(), X.ids), "non rows"
+                        h.gather_cold()
+                        h.status()
+                        check_gather()
+                        staged = h.cache[hot_cap:hot_cap + len(C)].cpu().numpy()
+                        assert np.array_equal(staged.view(np.uint32), table0[C].view(np.uint32)) or step > 0, "staging"
+                        h.fwd_pop()
+                        if deferred:
+                            h.fwd_non()
+                            h.bwd_pop(d_gpop, lr)
+                        else:
+                            h.bwd_pop(d_gpop, lr)
+                            h.fwd_non()
+                        h.bwd_non(d_gnon, lr)
+                        h.scatter_cold()
+                        h.status()
+                else:
+                    h.step(d_idx, d_off, B, d_gpop, d_gnon, lr, dense=d_dense, deferred=deferred, overlap=overlap)
+                    h.status()
+                    check_fragment()
+                    check_gather()
+
+                pp = h.pooled_pop[:bags_pop].cpu().numpy()
+                pn = h.pooled_non[:bags_non].cpu().numpy()
+                assert_close(pp, pooled_pop_o, "pooled_pop")
+                assert_close(pn, pooled_non_o, "pooled_non")
+                assert_close(h.cache[:n_hot].cpu().numpy(), cache_o[:n_hot], "hot rows after update")
+                assert_close(h.cache[hot_cap:hot_cap + len(C)].cpu().numpy(), cache_o[hot_cap:hot_cap + len(C)],
+                             "staged rows after update")
+                assert_close(h.host_table.numpy(), table_o, "host table after scatter")
+                if integer:
+                    assert np.array_equal(pp, pooled_pop_o) and np.array_equal(pn, pooled_non_o), "integer pooled"
+                    assert np.array_equal(h.cache[:n_hot].cpu().numpy(), cache_o[:n_hot]), "integer hot rows"
+                    assert np.array_equal(h.host_table.numpy(), table_o), "integer host table"
+                if spec.pooling[0] == "one" and step == 0:   # a bag of one lookup is a row copy: bit-exact
+                    assert np.array_equal(pp.view(np.uint32), pooled_pop_o.view(np.uint32)), "pooled_pop bits"
+                # rows nobody touched keep their bits
+                touched = np.zeros(N, dtype=bool)
+                touched[C] = True
+                assert np.array_equal(h.host_table.numpy()[~touched].view(np.uint32), table0[~touched].view(np.uint32)) \
+                    or step > 0, "untouched host rows"
+                stats = dict(n_pop=n_pop_o, n_non=n_non_o, n_cold=len(C), n_hot=n_hot, L_pop=len(O.ids), L_non=len(X.ids),
+                             batch=B, N=N)
+                if verbose:
+                    print(f"[{spec.name}] step {step}: {stats}")
+    finally:
+        h.close()
+    return stats

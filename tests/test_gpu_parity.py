@@ -1,0 +1,95 @@
+"""CUDA path vs CPU oracle, call by call, through the C boundary (needs a B200)."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import gen
+from tests.harness import run_config_check
+
+pytestmark = pytest.mark.gpu
+
+
+def test_tiny_config():
+    stats = run_config_check("tiny", steps=3)
+    assert 0 < stats["n_pop"] < stats["batch"]
+
+
+def test_tiny_config_three_steps_without_resync():
+    """The two sides are never re-aligned: their rounding differences accumulate over the steps and must still
+    stay inside the tolerance on this pooling-1 workload."""
+    run_config_check("tiny", steps=3, resync=False)
+
+
+def test_tiny_config_deferred_order_and_no_overlap():
+    run_config_check("tiny", steps=2, deferred=True, overlap=False)
+
+
+def test_tiny_integer_data_is_bit_exact():
+    run_config_check("tiny", steps=2, integer=True)
+
+
+@pytest.mark.parametrize("hot", ["empty", "full", ("random", 0.3), ("random", 0.9)])
+def test_arbitrary_hot_sets(hot):
+    """Misclassifying a row never changes the result (Section V-B): any hot set must give the oracle's answer."""
+    spec = dataclasses.replace(gen.CONFIGS["tiny"], hot_policy=("topk", 80_000))
+    stats = run_config_check(spec, steps=2, hot_override=hot)
+    if hot == "empty":
+        assert stats["n_pop"] == 0
+    if hot == "full":
+        assert stats["n_non"] == 0 and stats["n_cold"] == 0
+
+
+def test_min_share_policy():
+    spec = dataclasses.replace(gen.CONFIGS["tiny"], hot_policy=("share", 1, 2000))
+    run_config_check(spec, steps=1)
+
+
+@pytest.mark.parametrize("dim", [4, 8, 32, 64, 128, 200])
+def test_row_widths(dim):
+    spec = dataclasses.replace(gen.CONFIGS["tiny"], dim=dim, batch=333, rows=("fixed", 3001))
+    run_config_check(spec, steps=2)
+
+
+def test_ragged_shapes_many_tables():
+    spec = gen.WorkloadSpec(name="ragged", num_tables=37, dim=16, batch=1237, rows=("loguniform", 4, 50_000, 7),
+                            alpha=tuple([1.1] * 37), n_dense=5, hot_policy=("fraction", 20, 100), profile_batches=6,
+                            seed=11)
+    run_config_check(spec, steps=2)
+
+
+def test_multi_hot_bags():
+    spec = dataclasses.replace(gen.CONFIGS["multi_hot"], batch=2048, rows=("fixed", 50_000),
+                               hot_policy=("fraction", 30, 100), profile_batches=4)
+    stats = run_config_check(spec, steps=2)
+    assert stats["L_non"] > 0
+
+
+def test_multi_hot_integer_data_long_runs():
+    spec = dataclasses.replace(gen.CONFIGS["multi_hot"], batch=4096, dim=64, rows=("fixed", 500),
+                               hot_policy=("fraction", 50, 100), profile_batches=2)
+    run_config_check(spec, steps=1, integer=True)
+
+
+def test_time_series_shape():
+    spec = dataclasses.replace(gen.CONFIGS["tbsm"], batch=512, rows=("list", (20_000, 80_000, 1000)),
+                               hot_policy=("fraction", 60, 100), profile_batches=8)
+    stats = run_config_check(spec, steps=2)
+    assert stats["n_pop"] > 0
+
+
+def test_dlrm_small_scaled():
+    stats = run_config_check("dlrm_small", steps=2, scale_rows=0.05, profile_batches=8)
+    assert stats["n_pop"] > 0 and stats["n_cold"] > 0
+
+
+def test_dlrm_large_scaled():
+    spec = dataclasses.replace(gen.CONFIGS["dlrm_large"], batch=4096)
+    run_config_check(spec, steps=1, scale_rows=0.002, profile_batches=4)
+
+
+def test_batch_of_one_and_single_table():
+    spec = gen.WorkloadSpec(name="one", num_tables=1, dim=16, batch=1, rows=("fixed", 50), alpha=(1.5,),
+                            hot_policy=("topk", 10), profile_batches=3, seed=3)
+    run_config_check(spec, steps=2)
