@@ -1,0 +1,508 @@
+#!/usr/bin/env python
+"""Benchmark of the Hotline hot path on B200: samples/s through fragment + embedding-bag forward/backward
+(+ cold gather/scatter), one process per GPU, synthetic inputs.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A "step" is one mini-batch through the whole path: hl_fragment, hl_gather_cold (side stream), hl_embbag_fwd and
+hl_embbag_bwd_sgd for the popular and then the non-popular micro-batch, hl_scatter_cold.  Rank 0 prints ONE JSON
+line.  `--impl reference` times the CPU oracle on the host cores instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+METRIC = "samples/sec through fragment+embbag fwd/bwd"
+UNIT = "samples/s"
+L2_BYTES = 126 << 20
+FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the roofline kernel, from the ncu capture summarised
+# under profiles/ (None until a capture of that workload exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+# ----------------------------------------------------------------------------------------------------------
+# workload
+# ----------------------------------------------------------------------------------------------------------
+def mem_available_bytes() -> int:
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable"):
+                return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return 0
+
+
+def pick_workload(requested: str, world: int):
+    """(config name, row scale).  The metric is quoted on the DLRM-large-like configuration; every rank keeps its
+    own host table, so with several ranks (or little host RAM) the table is shrunk, or DLRM-small-like is used."""
+    if requested != "auto":
+        return requested, 1.0
+    need = gen.make_geometry(gen.CONFIGS["dlrm_large"]).total_rows * 64 * 4
+    avail = mem_available_bytes()
+    if avail and need * world <= 0.7 * avail:
+        return "dlrm_large", 1.0
+    return "dlrm_small", 1.0
+
+
+def max_nnz_of(spec, geom) -> int:
+    bags = geom.num_tables * spec.batch * geom.bags_per_sample
+    return bags if spec.pooling[0] == "one" else bags * int(spec.pooling[2])
+
+
+def fill_table(table, dim: int, seed: int, device, chunk_rows: int = 1 << 21) -> None:
+    """table[g, :] = gen.table_values(g) for every row, computed on the device in chunks and copied down."""
+    import torch
+    n = table.shape[0]
+    for r0 in range(0, n, chunk_rows):
+        r1 = min(n, r0 + chunk_rows)
+        table[r0:r1].copy_(gen.table_values_torch(r0, r1 - r0, dim, seed, device))
+    if str(device) != "cpu":
+        torch.cuda.synchronize()
+
+
+class Workload:
+    """Everything both arms need: geometry, the host table, profiling and timed batches (host copies)."""
+
+    def __init__(self, name: str, scale: float, n_batches: int, profile_batches, device, threads: int):
+        import torch
+        import paper_2204_05436_b200 as hl
+        self.spec = gen.CONFIGS[name]
+        self.geom = gen.make_geometry(self.spec, scale)
+        self.name, self.scale = name, scale
+        g, s = self.geom, self.spec
+        self.T, self.D, self.S, self.B, self.N = g.num_tables, g.dim, g.bags_per_sample, s.batch, g.total_rows
+        self.n_bags = self.T * self.B * self.S
+        self.max_nnz = max_nnz_of(s, g)
+        self.P = s.profile_batches if profile_batches is None else profile_batches
+        self.hot_cap = max(1, min(self.N, self._policy_rows()))
+        self.staging_cap = max(1, min(self.N, self.max_nnz))
+        t0 = time.time()
+        self.table = hl.host_table_tensor(self.N, self.D)
+        fill_table(self.table, self.D, s.seed, device)
+        log(f"[bench] host table {self.N} x {self.D} fp32 = {self.N * self.D * 4 / 2**30:.1f} GiB pinned+filled "
+            f"in {time.time() - t0:.1f}s")
+        t0 = time.time()
+        self.profile = [gen.make_batch(s, g, i, threads) for i in range(self.P)]
+        self.batches = [gen.make_batch(s, g, self.P + i, threads) for i in range(n_batches)]
+        log(f"[bench] drew {self.P} profiling + {n_batches} timed batches in {time.time() - t0:.1f}s")
+
+    def _policy_rows(self) -> int:
+        p = self.spec.hot_policy
+        if p[0] == "budget":
+            return int(p[1]) // (4 * self.D)
+        if p[0] == "fraction":
+            return self.N * int(p[1]) // int(p[2])
+        return int(p[1])
+
+    def policy_args(self):
+        import paper_2204_05436_b200 as hl
+        p = self.spec.hot_policy
+        if p[0] == "budget":
+            return hl.HL_HOT_BUDGET_BYTES, int(p[1]), 1
+        if p[0] == "fraction":
+            return hl.HL_HOT_FRACTION_ROWS, int(p[1]), int(p[2])
+        return hl.HL_HOT_TOPK_ROWS, int(p[1]), 1
+
+    def free(self):
+        import paper_2204_05436_b200 as hl
+        ptr = self.table.data_ptr()
+        self.table = None
+        hl.hl_host_free(ptr)
+
+
+# ----------------------------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(prefix="hl_clocks_", suffix=".csv")
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------------------
+# CPU oracle legs (cpu_baseline of the CUDA arm, and the whole `--impl reference` arm)
+# ----------------------------------------------------------------------------------------------------------
+def take_samples(batch: gen.Batch, T: int, B: int, S: int, n: int) -> gen.Batch:
+    """The first n inputs of a table-major CSR mini-batch, as a mini-batch of n inputs."""
+    if n >= B:
+        return batch
+    off = batch.offsets.astype(np.int64)
+    idx_parts, sizes = [], []
+    for t in range(T):
+        lo_bag, hi_bag = t * B * S, (t * B + n) * S
+        idx_parts.append(batch.indices[off[lo_bag]:off[hi_bag]])
+        sizes.append(np.diff(off[lo_bag:hi_bag + 1]))
+    new_off = np.concatenate([[0], np.cumsum(np.concatenate(sizes))]).astype(np.int32)
+    dense = None if batch.dense is None else batch.dense[:n]
+    return gen.Batch(np.concatenate(idx_parts).astype(np.int32), new_off, dense, n)
+
+
+class OracleRunner:
+    """Runs the CPU oracle, as it stands, on the workload: learning phase once, then one step per call."""
+
+    def __init__(self, wl: Workload):
+        from oracle import hotline_oracle as orc
+        self.orc, self.wl = orc, wl
+        t0 = time.time()
+        cnt = orc.access_counts([(b.indices, b.offsets) for b in wl.profile], wl.B, wl.geom.table_rows, wl.S)
+        k = min(wl.hot_cap, orc.hot_capacity(wl.spec.hot_policy, wl.N, wl.D))
+        self.hot = orc.select_hot(cnt, k)
+        del cnt
+        self.remap = orc.build_remap(self.hot, wl.N)
+        self.table = wl.table.numpy()
+        self.cache = np.zeros((wl.hot_cap + wl.staging_cap, wl.D), dtype=np.float32)
+        self.cache[: len(self.hot)] = orc.load_hot_cache(self.table, self.hot)
+        self.rng = np.random.default_rng(1234)
+        log(f"[bench] oracle learning phase: {len(self.hot)} hot rows in {time.time() - t0:.1f}s")
+
+    def step(self, batch: gen.Batch) -> float:
+        """Seconds the oracle needs for one mini-batch (fragment, gather, fwd/bwd of O and X, scatter)."""
+        wl, orc = self.wl, self.orc
+        n_bags = wl.T * batch.batch * wl.S
+        grad = self.rng.standard_normal((n_bags, wl.D), dtype=np.float32)
+        # the split of the gradient rows between O and X is input marshalling, outside the timed part
+        _, n_pop, _, _, _ = orc.fragment(batch.indices, batch.offsets, batch.batch, wl.geom.table_rows, self.remap,
+                                         wl.S)
+        bags_pop = wl.T * n_pop * wl.S
+        t0 = time.perf_counter()
+        orc.hotline_step(self.table, self.cache, wl.hot_cap, self.remap, batch.indices, batch.offsets, batch.batch,
+                         wl.geom.table_rows, wl.S, grad[:bags_pop], grad[bags_pop:], wl.spec.lr)
+        return time.perf_counter() - t0
+
+
+def threads_in_use() -> int:
+    """numpy does the oracle's work on the calling thread (no BLAS call is involved)."""
+    return 1
+
+
+def run_reference(args, rank: int, world: int) -> None:
+    if rank != 0:
+        return
+    import torch
+    device = "cuda:0" if torch.cuda.is_available() else "cpu"
+    name, scale = pick_workload(args.workload, 1)
+    wl = Workload(name, scale, n_batches=min(8, args.steps + args.warmup), profile_batches=args.profile_batches,
+                  device=device, threads=args.threads)
+    runner = OracleRunner(wl)
+    # size the per-step sample so that the whole run ends within a few minutes
+    probe = take_samples(wl.batches[0], wl.T, wl.B, wl.S, min(wl.B, 2048))
+    t_probe = runner.step(probe)
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    n = int(min(wl.B, max(256, probe.batch * budget / max(t_probe, 1e-6))))
+    n = 1 << (n.bit_length() - 1) if n < wl.B else wl.B
+    sample = [take_samples(b, wl.T, wl.B, wl.S, n) for b in wl.batches]
+    for i in range(args.warmup):
+        runner.step(sample[i % len(sample)])
+    times = [runner.step(sample[(args.warmup + i) % len(sample)]) for i in range(args.steps)]
+    total = sum(times)
+    value = n * args.steps / total
+    sample_txt = f"first {n} of {wl.B} inputs of each mini-batch, {args.steps} mini-batches"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "row_scale": wl.scale, "batch": wl.B, "sample_inputs_per_step": n,
+                   "tables": wl.T, "dim": wl.D, "total_rows": wl.N},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads_in_use(), "kind": "oracle",
+                         "sample": sample_txt},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+    wl.free()
+
+
+# ----------------------------------------------------------------------------------------------------------
+# CUDA arm
+# ----------------------------------------------------------------------------------------------------------
+def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
+    import torch
+    import torch.distributed as dist
+    import paper_2204_05436_b200 as hl
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    device = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(device)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+
+    name, scale = pick_workload(args.workload, world)
+    n_batches = 8
+    wl = Workload(name, scale, n_batches, args.profile_batches, device, args.threads)
+    T, D, S, B = wl.T, wl.D, wl.S, wl.B
+    h = hl.Hotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
+                   n_dense=wl.spec.n_dense, device=str(device))
+    lr = wl.spec.lr
+
+    with torch.cuda.stream(h.main):
+        # ---- learning phase (setup, timed separately) ----
+        t0 = time.time()
+        for i, b in enumerate(wl.profile):
+            h.profile(torch.from_numpy(b.indices).to(device), torch.from_numpy(b.offsets).to(device), B, reset=(i == 0))
+        pol, p_num, p_den = wl.policy_args()
+        h.profile(None, None, finalize=True, policy=pol, p_num=p_num, p_den=p_den)
+        h.build_remap(load_rows=True)
+        h.status()
+        n_hot = int(h.n_hot.item())
+        log(f"[bench] learning phase on the device: {n_hot} hot rows of {wl.hot_cap} slots in {time.time() - t0:.1f}s")
+
+        # ---- resident inputs ----
+        pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()   # noqa: E731
+        h_idx = [pin(b.indices) for b in wl.batches]
+        h_off = [pin(b.offsets) for b in wl.batches]
+        h_dense = [pin(b.dense) if b.dense is not None else None for b in wl.batches]
+        d_idx = [x.to(device) for x in h_idx]
+        d_off = [x.to(device) for x in h_off]
+        d_dense = [x.to(device) if x is not None else None for x in h_dense]
+        gen_t = torch.Generator(device=device)
+        gen_t.manual_seed(wl.spec.seed + 1000 + rank)
+        d_grad = torch.randn((wl.n_bags, D), generator=gen_t, device=device, dtype=torch.float32)
+        h_grad = d_grad.cpu().pin_memory()
+        torch.cuda.synchronize()
+
+        def one_step(i, timers=None):
+            k = i % n_batches
+            h.step(d_idx[k], d_off[k], B, d_grad, d_grad, lr, dense=d_dense[k], timers=timers)
+
+        # per-batch sizes (they depend only on the indices and the hot set): one untimed pass
+        sizes = []
+        for k in range(n_batches):
+            one_step(k)
+            h.status()
+            c = h.counts.cpu().tolist()
+            sizes.append(dict(n_pop=c[0], n_non=c[1], L_pop=c[2], L_non=c[3], n_cold=int(h.n_cold.item())))
+
+        # ---- timed region: device-resident inputs ----
+        for i in range(args.warmup):
+            one_step(i)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        timers = {}
+        launches0 = hl.hl_launch_count()
+        clocks = ClockSampler(local_rank)
+        clocks.start()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        ev0.record(h.main)
+        for i in range(args.steps):
+            one_step(args.warmup + i, timers)
+        ev1.record(h.main)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        clock_info = clocks.stop()
+        launches = hl.hl_launch_count() - launches0
+        h.status()
+        ms_total = ev0.elapsed_time(ev1)
+
+        # ---- end to end: host buffers in, results out, copies inside the timed region ----
+        e2e = None
+        if not args.no_e2e:
+            out_pop = torch.empty((wl.n_bags, D), dtype=torch.float32).pin_memory()
+            out_non = torch.empty((wl.n_bags, D), dtype=torch.float32).pin_memory()
+            out_counts = torch.empty(4, dtype=torch.int32).pin_memory()
+            out_perm = torch.empty(B, dtype=torch.int32).pin_memory()
+            h2d = d2h = 0
+
+            def e2e_step(i):
+                nonlocal h2d, d2h
+                k = i % n_batches
+                d_idx[k].copy_(h_idx[k], non_blocking=True)
+                d_off[k].copy_(h_off[k], non_blocking=True)
+                h2d_now = h_idx[k].numel() * 4 + h_off[k].numel() * 4 + h_grad.numel() * 4
+                if d_dense[k] is not None:
+                    d_dense[k].copy_(h_dense[k], non_blocking=True)
+                    h2d_now += h_dense[k].numel() * 4
+                d_grad.copy_(h_grad, non_blocking=True)
+                h.step(d_idx[k], d_off[k], B, d_grad, d_grad, lr, dense=d_dense[k])
+                out_counts.copy_(h.counts, non_blocking=True)
+                out_perm.copy_(h.perm[:B], non_blocking=True)
+                h.main.synchronize()
+                bags_pop, bags_non = T * int(out_counts[0]) * S, T * int(out_counts[1]) * S
+                out_pop[:bags_pop].copy_(h.pooled_pop[:bags_pop], non_blocking=True)
+                out_non[:bags_non].copy_(h.pooled_non[:bags_non], non_blocking=True)
+                h.main.synchronize()
+                h2d, d2h = h2d_now, 16 + B * 4 + (bags_pop + bags_non) * D * 4
+
+            for i in range(max(3, min(args.warmup, 5))):
+                e2e_step(i)
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(h.main)
+            for i in range(args.steps):
+                e2e_step(args.warmup + i)
+            e1.record(h.main)
+            torch.cuda.synchronize()
+            e2e_ms = e0.elapsed_time(e1)
+            e2e = {"ms_total": e2e_ms, "h2d": h2d, "d2h": d2h}
+        h.status()
+
+    # ---- reduce over ranks (max time) ----
+    if world > 1:
+        t = torch.tensor([ms_total, e2e["ms_total"] if e2e else 0.0], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t[0])
+        if e2e:
+            e2e["ms_total"] = float(t[1])
+
+    if rank == 0:
+        ms_per_step = ms_total / args.steps
+        value = B * world * args.steps / (ms_total * 1e-3)
+
+        def mean_us(name):
+            ev = timers.get(name, [])
+            return 1e3 * sum(a.elapsed_time(b) for a, b in ev) / max(1, len(ev))
+
+        breakdown = {k: round(mean_us(k), 2) for k in timers}
+        used = [sizes[(args.warmup + i) % n_batches] for i in range(args.steps)]
+        mean = lambda key: sum(u[key] for u in used) / len(used)   # noqa: E731
+        # roofline of the popular micro-batch's embedding-bag forward (one kernel per call): per lookup a row
+        # (4*D bytes) and its slot (4 bytes) are read, per bag a pooled row (4*D) is written and an offset read.
+        bags_pop = T * mean("n_pop") * S
+        fwd_bytes = mean("L_pop") * (4 * D + 4) + bags_pop * (4 * D + 4)
+        fwd_us = mean_us("fwd_pop")
+        peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(peaks_path):
+            peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        else:
+            peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+        achieved = fwd_bytes / (fwd_us * 1e-6) / 1e9 if fwd_us > 0 else 0.0
+        roofline = {"kernel": "k_embbag_fwd (popular micro-batch)", "bound": "hbm", "achieved": achieved,
+                    "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+                    "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "algorithmic_bytes_per_launch": fwd_bytes,
+                    "us_per_launch": fwd_us}
+        link_us = mean_us("gather_cold")
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "row_scale": wl.scale, "batch": B, "tables": T, "dim": D,
+                       "bags_per_sample": S, "total_rows": wl.N, "table_gib": round(wl.N * D * 4 / 2 ** 30, 2),
+                       "hot_rows": n_hot, "hot_cap_rows": wl.hot_cap, "profile_batches": wl.P,
+                       "popular_fraction": round(mean("n_pop") / B, 4), "cold_rows_per_step": round(mean("n_cold"), 1),
+                       "l2": "no explicit flush: a step reads and writes more than the 126 MB L2 "
+                             f"({(2 * wl.n_bags * D * 4 + fwd_bytes) / 2**20:.0f} MB of pooled vectors, gradients and rows)"
+                             if 2 * wl.n_bags * D * 4 > L2_BYTES else
+                             "per-step working set is smaller than L2 on this workload; batches rotate over 8 buffers",
+                       "replicas": "independent replica per GPU, no collective"},
+            "clocks": clock_info, "gpu_launches": int(launches),
+            "launches_per_step": launches / args.steps, "breakdown_us": breakdown, "roofline": roofline,
+            "cold_gather": {"rows_per_step": mean("n_cold"), "bytes_per_step": mean("n_cold") * D * 4,
+                            "call_us": link_us},
+        }
+        if e2e:
+            line["e2e"] = {"value": B * world * args.steps / (e2e["ms_total"] * 1e-3), "unit": UNIT,
+                           "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                           "ms_per_step": e2e["ms_total"] / args.steps}
+        if world == 1 and not args.no_cpu_baseline:
+            h.close()
+            runner = OracleRunner(wl)
+            t_first = runner.step(wl.batches[0])
+            n_more = int(max(1, min(len(wl.batches) - 1, 15.0 / max(t_first, 1e-3))))
+            times = [t_first] + [runner.step(wl.batches[1 + i]) for i in range(n_more)]
+            line["cpu_baseline"] = {"value": B * len(times) / sum(times), "unit": UNIT, "cores": threads_in_use(),
+                                    "kind": "oracle",
+                                    "sample": f"{len(times)} whole mini-batches of {B} inputs ({sum(times):.1f} s)"}
+        print(json.dumps(line), flush=True)
+    h.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    wl.free()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="auto", choices=["auto"] + sorted(gen.CONFIGS))
+    ap.add_argument("--profile-batches", type=int, default=None)
+    ap.add_argument("--threads", type=int, default=min(16, os.cpu_count() or 1))
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        log("[bench] warm-up raised to 3 steps")
+        args.warmup = 3
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_cuda(args, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()

@@ -114,6 +114,15 @@ HL_API int32_t hl_status(hl_ctx* ctx);
 
 HL_API const char* hl_strerror(int32_t status);
 
+/* Pinned, device-mapped host memory for the host-DRAM table (exactly `bytes`, no rounding): the device reads
+ * and writes it over the host link at the same address.  The caller owns it and frees it with hl_host_free.
+ * Returns NULL on failure. */
+HL_API void* hl_host_alloc(size_t bytes);
+HL_API int32_t hl_host_free(void* p);
+
+/* Number of kernels this library has launched in this process so far (all contexts). */
+HL_API uint64_t hl_launch_count(void);
+
 /* ---------------------------------------------------------------------------------------------------------
  * Learning phase
  * ------------------------------------------------------------------------------------------------------- */

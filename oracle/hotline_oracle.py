@@ -58,12 +58,12 @@ def access_counts(batches: Iterable, batch: int, table_rows, bags_per_sample: in
     also repeats inside one bag (the access logger "tracks the frequency of access", Section V-B; this is
     the exact counter the paper calls the Oracle LFU logger)."""
     N = int(np.sum(np.asarray(table_rows, dtype=np.int64)))
-    cnt = np.zeros(N, dtype=np.int64)
+    rows = [np.zeros(0, dtype=np.int64)]
     for indices, offsets in batches:
         g, _, _, _ = lookups_of(indices, offsets, batch, table_rows, bags_per_sample)
         assert ((np.asarray(indices) >= 0)).all() and (g < N).all()
-        cnt += np.bincount(g, minlength=N)
-    return cnt
+        rows.append(g)
+    return np.bincount(np.concatenate(rows), minlength=N).astype(np.int64)
 
 
 def select_hot(cnt: np.ndarray, k_max: int, min_share: Optional[tuple] = None) -> np.ndarray:

@@ -16,7 +16,8 @@ HL_OK, HL_EINVAL, HL_EBOUNDS, HL_ECAPACITY, HL_ECUDA, HL_ETIMEOUT = 0, -1, -2, -
 HL_HOT_TOPK_ROWS, HL_HOT_BUDGET_BYTES, HL_HOT_FRACTION_ROWS, HL_HOT_MIN_SHARE = 0, 1, 2, 3
 
 EXPORTS = (
-    "hl_workspace_bytes", "hl_create", "hl_destroy", "hl_status", "hl_strerror", "hl_profile_hot",
+    "hl_workspace_bytes", "hl_create", "hl_destroy", "hl_status", "hl_strerror", "hl_launch_count", "hl_host_alloc",
+    "hl_host_free", "hl_profile_hot",
     "hl_build_remap", "hl_fragment", "hl_embbag_fwd", "hl_embbag_bwd_sgd", "hl_gather_cold", "hl_scatter_cold",
 )
 
@@ -44,7 +45,7 @@ class hl_ubatch(ctypes.Structure):
 def _load() -> ctypes.CDLL:
     if not os.path.exists(_LIB_PATH):
         raise ImportError(
-            f"{_LIB_PATH} is missing: build it with `python -m paper_2204_05436_b200.build` "
+            f"{_LIB_PATH} is missing: build it with `python paper_2204_05436_b200/csrc/build.py` "
             "(needs nvcc; there is no CPU fallback)")
     lib = ctypes.CDLL(_LIB_PATH)
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
@@ -59,6 +60,12 @@ def _load() -> ctypes.CDLL:
     lib.hl_status.argtypes = [vp]
     lib.hl_strerror.restype = ctypes.c_char_p
     lib.hl_strerror.argtypes = [i32]
+    lib.hl_launch_count.restype = ctypes.c_uint64
+    lib.hl_launch_count.argtypes = []
+    lib.hl_host_alloc.restype = vp
+    lib.hl_host_alloc.argtypes = [ctypes.c_size_t]
+    lib.hl_host_free.restype = i32
+    lib.hl_host_free.argtypes = [vp]
     lib.hl_profile_hot.restype = i32
     lib.hl_profile_hot.argtypes = [vp, ctypes.POINTER(hl_batch), i32, i32, i32, i64, i64, vp, vp, vp]
     lib.hl_build_remap.restype = i32
@@ -100,6 +107,32 @@ def _check(call: str, status: int) -> int:
 
 def strerror(status: int) -> str:
     return _lib.hl_strerror(int(status)).decode()
+
+
+def hl_launch_count() -> int:
+    return int(_lib.hl_launch_count())
+
+
+def hl_host_alloc(nbytes: int) -> int:
+    p = _lib.hl_host_alloc(int(nbytes))
+    if not p:
+        raise HotlineError("hl_host_alloc", HL_ECUDA)
+    return int(p)
+
+
+def hl_host_free(ptr: int) -> None:
+    _check("hl_host_free", _lib.hl_host_free(ptr))
+
+
+def host_table_tensor(n_rows: int, dim: int):
+    """fp32 [n_rows, dim] torch tensor over memory from hl_host_alloc (exact size).  Free it with
+    ``hl_host_free(t.data_ptr())`` once no tensor or kernel uses it any more."""
+    import numpy as np
+    import torch
+    nbytes = int(n_rows) * int(dim) * 4
+    ptr = hl_host_alloc(nbytes)
+    buf = (ctypes.c_float * (int(n_rows) * int(dim))).from_address(ptr)
+    return torch.from_numpy(np.frombuffer(buf, dtype=np.float32).reshape(int(n_rows), int(dim)))
 
 
 def make_geometry(table_rows: Sequence[int], dim: int, bags_per_sample: int = 1) -> hl_geometry:

@@ -1,4 +1,8 @@
-"""Builds libhotline.so (sm_100a) in-tree with nvcc.  `python -m paper_2204_05436_b200.build [--force]`."""
+"""Builds libhotline.so (sm_100a) in-tree with nvcc:  python paper_2204_05436_b200/csrc/build.py [--force] [-v]
+
+Kept outside the package's import path on purpose: importing the package loads the library, so the script that
+creates the library must be runnable before the library exists.
+"""
 from __future__ import annotations
 
 import os
@@ -7,9 +11,9 @@ import subprocess
 import sys
 from concurrent.futures import ThreadPoolExecutor
 
-PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+CSRC = os.path.dirname(os.path.abspath(__file__))
+PKG_DIR = os.path.dirname(CSRC)
 ROOT = os.path.dirname(PKG_DIR)
-CSRC = os.path.join(PKG_DIR, "csrc")
 OBJ_DIR = os.path.join(CSRC, "build")
 LIB_PATH = os.path.join(PKG_DIR, "libhotline.so")
 INCLUDE = os.path.join(ROOT, "include")

@@ -164,6 +164,27 @@ extern "C" int32_t hl_status(hl_ctx* ctx) {
     return st;
 }
 
+namespace hl {
+unsigned long long launches_so_far();
+}
+
+extern "C" uint64_t hl_launch_count(void) { return hl::launches_so_far(); }
+
+extern "C" void* hl_host_alloc(size_t bytes) {
+    void* p = nullptr;
+    if (bytes == 0 || cudaHostAlloc(&p, bytes, cudaHostAllocMapped | cudaHostAllocPortable) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return p;
+}
+
+extern "C" int32_t hl_host_free(void* p) {
+    if (!p) return HL_OK;
+    HL_CUDA_TRY(cudaFreeHost(p));
+    return HL_OK;
+}
+
 extern "C" const char* hl_strerror(int32_t status) {
     switch (status) {
         case HL_OK: return "ok";

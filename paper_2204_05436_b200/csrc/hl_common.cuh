@@ -139,6 +139,9 @@ int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, 
 int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n, int64_t n_max, int key_bits,
                          uint32_t* hist, int32_t** out_keys, int32_t** out_vals, cudaStream_t stream);
 
+// Process-wide count of kernels this library has launched (read by hl_launch_count).
+void note_launches(int n);
+
 inline int64_t div_up(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int grid_for(int64_t work_items, int per_block, int max_blocks) {
     int64_t b = div_up(work_items, per_block);

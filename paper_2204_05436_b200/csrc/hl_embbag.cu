@@ -357,6 +357,7 @@ int32_t launch_fwd(hl_ctx* ctx, const float* cache, const hl_ubatch* ub, const i
     k_embbag_fwd<G, NV, UB><<<grid, kThreads, 0, stream>>>(cache, ub->ids, ub->offsets, d_n, ctx->max_batch,
                                                           ctx->T * ctx->S, ctx->D / 4,
                                                           ctx->hot_cap + ctx->staging_cap, out, ctx->r.status);
+    note_launches(1);
     HL_LAUNCH_CHECK();
     return HL_OK;
 }
@@ -371,6 +372,7 @@ int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t
                                                       lr, ctx->r.bwd_part);
     k_bwd_spans<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, ctx->r.bwd_n, ctx->D / 4, n_slots, lr,
                                                      ctx->r.bwd_part);
+    note_launches(2);
     HL_LAUNCH_CHECK();
     return HL_OK;
 }
@@ -425,6 +427,7 @@ extern "C" int32_t hl_embbag_bwd_sgd(hl_ctx* ctx, float* d_cache, const hl_ubatc
         k_bwd_pairs<32><<<grid_for(ctx->max_bags, kThreads / 32, kSMs * 8), kThreads, 0, stream>>>(
             ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, r.bwd_keys[0],
             r.bwd_vals[0], r.bwd_n, r.status);
+    note_launches(1);
     HL_LAUNCH_CHECK();
     int32_t *keys, *vals;
     int32_t st = radix_sort_pairs(r.bwd_keys, r.bwd_vals, r.bwd_n, ctx->max_nnz, bits_for(n_slots), r.bwd_hist,

@@ -250,6 +250,7 @@ extern "C" int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_de
     k_frag_partition<<<1, 1024, 0, stream>>>(r.frag_flags, B, d_perm, d_counts);
     k_frag_sizes<<<grid_for(n_bags, kThreads, kSMs * 8), kThreads, 0, stream>>>(b->offsets, B, T, S, d_perm,
                                                                                d_counts, r.frag_scan);
+    note_launches(3);   // flags, partition, sizes
     HL_LAUNCH_CHECK();
     int32_t st = exclusive_scan_i32(r.frag_scan, r.frag_scan, nullptr, n_bags, r.frag_tiles, stream);
     if (st != HL_OK) return st;
@@ -264,6 +265,7 @@ extern "C" int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_de
     if (d_dense)
         k_permute_dense<<<grid_for((int64_t)B * n_dense, kThreads, kSMs * 8), kThreads, 0, stream>>>(
             d_dense, B, n_dense, d_perm, d_dense_out);
+    note_launches(d_dense ? 2 : 1);   // emit (+ dense permutation)
     HL_LAUNCH_CHECK();
     return HL_OK;
 }

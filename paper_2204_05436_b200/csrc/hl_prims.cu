@@ -1,8 +1,14 @@
 // Device-wide primitives used by several steps: exclusive scan and stable LSD radix sort of pairs.
 // Both take their element count from device memory, so that no step has to synchronise the host.
+#include <atomic>
+
 #include "hl_common.cuh"
 
 namespace hl {
+
+static std::atomic<unsigned long long> g_launches{0};
+void note_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+unsigned long long launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
 
 namespace {
 
@@ -200,6 +206,7 @@ int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, 
     k_scan_tile_sums<<<(unsigned)n_tiles, kThreads, 0, stream>>>(in, d_n, n_max, tiles);
     k_scan_spine<<<1, 1024, 0, stream>>>(tiles, n_tiles);
     k_scan_apply<<<(unsigned)n_tiles, kThreads, 0, stream>>>(in, out, d_n, n_max, tiles, n_tiles);
+    note_launches(3);
     HL_LAUNCH_CHECK();
     return HL_OK;
 }
@@ -216,6 +223,7 @@ int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n,
             k_sort_hist<<<(unsigned)n_tiles, kThreads, 0, stream>>>(keys[cur], d_n, n_max, shift, hist, n_tiles);
             if (n_hist <= 65536) {
                 k_scan_spine<<<1, 1024, 0, stream>>>(reinterpret_cast<int32_t*>(hist), n_hist);
+                note_launches(1);
             } else {
                 // the scan's tile sums live right behind the histogram (the workspace reserves the room)
                 int32_t* tiles = reinterpret_cast<int32_t*>(hist) + n_hist + 1;
@@ -226,6 +234,7 @@ int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n,
             k_sort_scatter<<<(unsigned)n_tiles, kThreads, 0, stream>>>(keys[cur], vals[cur], keys[cur ^ 1],
                                                                       vals[cur ^ 1], d_n, n_max, shift, hist,
                                                                       n_tiles);
+            note_launches(2);   // histogram + scatter
             cur ^= 1;
         }
         HL_LAUNCH_CHECK();

@@ -337,6 +337,7 @@ extern "C" int32_t hl_profile_hot(hl_ctx* ctx, const hl_batch* b, int32_t reset,
         const int64_t n_bags = bags_per_table * ctx->T;
         k_count<<<grid_for(n_bags, kThreads, kSMs * 8), kThreads, 0, stream>>>(
             b->indices, b->offsets, n_bags, bags_per_table, r.table_base, r.counts, r.sel, r.status);
+        note_launches(1);
         HL_LAUNCH_CHECK();
     }
     if (finalize) {
@@ -370,6 +371,7 @@ extern "C" int32_t hl_profile_hot(hl_ctx* ctx, const hl_batch* b, int32_t reset,
         k_select_spine<<<1, 1024, 0, stream>>>(r.sel_gt, r.sel_eq, ctx->n_sel_tiles);
         k_select_emit<<<tiles, kThreads, 0, stream>>>(r.counts, ctx->N, r.sel, r.sel_gt, r.sel_eq, ctx->n_sel_tiles,
                                                       ctx->hot_cap, d_hot_rows, d_n_hot, r.status);
+        note_launches(12);   // begin, 4 x (histogram, pick), tile counts, spine, emit
         HL_LAUNCH_CHECK();
     }
     return HL_OK;
@@ -385,9 +387,11 @@ extern "C" int32_t hl_build_remap(hl_ctx* ctx, const int32_t* d_hot_rows, const 
     if (ctx->hot_cap > 0) {
         k_remap_bits<<<grid_for(ctx->hot_cap, kThreads, kSMs * 8), kThreads, 0, stream>>>(
             d_hot_rows, d_n_hot, ctx->hot_cap, ctx->N, r.remap, r.status);
+        note_launches(1);
     }
     k_remap_prefix<<<grid_for(ctx->n_remap_blocks, kThreads, kSMs * 8), kThreads, 0, stream>>>(
         d_hot_rows, d_n_hot, ctx->hot_cap, ctx->n_remap_blocks, r.remap);
+    note_launches(d_remap_out ? 2 : 1);
     if (d_remap_out)
         k_remap_dense<<<grid_for(ctx->N, kThreads * 4, kSMs * 16), kThreads, 0, stream>>>(r.remap, ctx->N,
                                                                                          d_remap_out);

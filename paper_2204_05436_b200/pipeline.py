@@ -140,28 +140,42 @@ class Hotline:
 
     # ---- acceleration phase: one mini-batch --------------------------------------------------------------------
     def step(self, indices, offsets, batch: int, grad_pop: torch.Tensor, grad_non: torch.Tensor, lr: float,
-             dense: Optional[torch.Tensor] = None, deferred: bool = False, overlap: bool = True) -> None:
+             dense: Optional[torch.Tensor] = None, deferred: bool = False, overlap: bool = True,
+             timers: Optional[dict] = None) -> None:
         """One mini-batch through the pipeline.  ``grad_pop`` / ``grad_non`` are the upstream gradients of the
         pooled outputs of O and X (rows in the micro-batches' own bag order).  ``deferred`` runs both forwards
-        before both backwards; ``overlap=False`` keeps the cold gather on the main stream."""
-        self.fragment(indices, offsets, batch, dense)
+        before both backwards; ``overlap=False`` keeps the cold gather on the main stream.  ``timers``: a dict
+        that receives, per call name, a list of (start, end) CUDA events recorded on the stream of that call."""
+
+        def timed(name, stream, fn):
+            if timers is None:
+                fn()
+                return
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            timers.setdefault(name, []).append((a, b))
+
+        m = self.main
+        timed("fragment", m, lambda: self.fragment(indices, offsets, batch, dense))
         if overlap:
-            self.ev_frag.record(self.main)
+            self.ev_frag.record(m)
             self.side.wait_event(self.ev_frag)
-            self.gather_cold(self.side)
+            timed("gather_cold", self.side, lambda: self.gather_cold(self.side))
             self.ev_gather.record(self.side)
         else:
-            self.gather_cold(self.main)
-        self.fwd_pop()
+            timed("gather_cold", m, lambda: self.gather_cold(m))
+        timed("fwd_pop", m, self.fwd_pop)
         if not deferred:
-            self.bwd_pop(grad_pop, lr)
+            timed("bwd_pop", m, lambda: self.bwd_pop(grad_pop, lr))
         if overlap:
-            self.main.wait_event(self.ev_gather)
-        self.fwd_non()
+            m.wait_event(self.ev_gather)
+        timed("fwd_non", m, self.fwd_non)
         if deferred:
-            self.bwd_pop(grad_pop, lr)
-        self.bwd_non(grad_non, lr)
-        self.scatter_cold()
+            timed("bwd_pop", m, lambda: self.bwd_pop(grad_pop, lr))
+        timed("bwd_non", m, lambda: self.bwd_non(grad_non, lr))
+        timed("scatter_cold", m, self.scatter_cold)
 
     def synchronize(self) -> None:
         self.main.synchronize()

@@ -10,8 +10,12 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 @pytest.fixture(scope="module")
 def lib_path():
-    from paper_2204_05436_b200.build import build_library
-    return build_library()
+    import importlib.util
+    spec = importlib.util.spec_from_file_location(
+        "hotline_build", os.path.join(ROOT, "paper_2204_05436_b200", "csrc", "build.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod.build_library()
 
 
 def declared_functions():
