@@ -193,6 +193,35 @@ HL_API int32_t hl_gather_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_no
 HL_API int32_t hl_scatter_cold(hl_ctx* ctx, const float* d_cache, const int32_t* d_cold_rows,
                         const int64_t* d_n_cold, float* host_table, void* stream);
 
+/* No counterpart in the paper: an addition for callers that cannot allocate.
+ *
+ * Some callers have no way to hand the library a workspace: code that runs where device allocation is forbidden
+ * or unavailable (a plug-in inside a host application that owns all device memory and gives none away, a
+ * latency-critical loop that must never enter the allocator, a process whose memory budget is already committed).
+ * For them this variant of hl_embbag_bwd_sgd needs neither a context nor a workspace: its scratch (sort buffers,
+ * histograms, partial sums) is a fixed array of about 3 MB inside the library image, which every GPU that loads
+ * the library holds until the process exits.  It calls no cudaMalloc/cudaFree and no allocating routine.
+ *
+ * Same result as hl_embbag_bwd_sgd: for every distinct id u, cache[u, :] -= lr * sum of d_grad_out[bag(j), :]
+ * over the lookups j with ids[j] == u.  d_cache is fp32 [cache_rows, dim]; d_offsets [n_bags + 1] and d_ids [nnz]
+ * are a CSR over the bags; d_grad_out is [n_bags, dim]; all device pointers.  n_bags and nnz are given by the
+ * host.  d_status (device, may be NULL) receives HL_OK or the first device-side error (HL_EBOUNDS for an id
+ * outside the cache; that lookup is skipped).
+ *
+ * Limits: nnz <= HL_STATIC_MAX_NNZ, n_bags <= HL_STATIC_MAX_NNZ, dim <= HL_STATIC_MAX_DIM; anything larger is
+ * refused with HL_ECAPACITY before any work is queued.
+ * The first call on a device looks up the device address of the array (cudaGetSymbolAddress, with that device
+ * current); make that first call outside any stream capture.
+ * All calls on a device share the one array, which still holds the previous call's data: what must start at
+ * zero is cleared by the call itself, but two calls that overlap on the GPU (different streams, or different
+ * threads) race on it -- serialise them. */
+#define HL_STATIC_MAX_NNZ 65536
+#define HL_STATIC_MAX_DIM 128
+HL_API int32_t hl_embbag_bwd_sgd_static(float* d_cache, int64_t cache_rows, int32_t dim,
+                                        const int32_t* d_offsets, const int32_t* d_ids, int32_t n_bags,
+                                        int64_t nnz, const float* d_grad_out, float lr, int32_t* d_status,
+                                        void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -19,6 +19,7 @@ EXPORTS = (
     "hl_workspace_bytes", "hl_create", "hl_destroy", "hl_status", "hl_strerror", "hl_launch_count", "hl_host_alloc",
     "hl_host_free", "hl_profile_hot",
     "hl_build_remap", "hl_fragment", "hl_embbag_fwd", "hl_embbag_bwd_sgd", "hl_gather_cold", "hl_scatter_cold",
+    "hl_embbag_bwd_sgd_static",
 )
 
 
@@ -81,6 +82,8 @@ def _load() -> ctypes.CDLL:
     lib.hl_gather_cold.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, vp, vp, vp, vp, vp]
     lib.hl_scatter_cold.restype = i32
     lib.hl_scatter_cold.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.hl_embbag_bwd_sgd_static.restype = i32
+    lib.hl_embbag_bwd_sgd_static.argtypes = [vp, i64, i32, vp, vp, i32, i64, vp, ctypes.c_float, vp, vp]
     return lib
 
 
@@ -215,3 +218,15 @@ def hl_gather_cold(ctx: int, non: hl_ubatch, d_n_non, host_table, d_cache, d_col
 def hl_scatter_cold(ctx: int, d_cache, d_cold_rows, d_n_cold, host_table, stream: int) -> None:
     _check("hl_scatter_cold", _lib.hl_scatter_cold(ctx, _ptr(d_cache), _ptr(d_cold_rows), _ptr(d_n_cold),
                                                    _ptr(host_table), stream))
+
+
+HL_STATIC_MAX_NNZ, HL_STATIC_MAX_DIM = 65536, 128
+
+
+def hl_embbag_bwd_sgd_static(d_cache, cache_rows: int, dim: int, d_offsets, d_ids, n_bags: int, nnz: int,
+                             d_grad_out, lr: float, d_status, stream: int) -> None:
+    """Backward + SGD for callers that cannot allocate device memory: no context, no workspace; the scratch is a
+    fixed array inside the library (see include/hotline.h for the limits and the sharing rule)."""
+    _check("hl_embbag_bwd_sgd_static", _lib.hl_embbag_bwd_sgd_static(
+        _ptr(d_cache), int(cache_rows), int(dim), _ptr(d_offsets), _ptr(d_ids), int(n_bags), int(nnz),
+        _ptr(d_grad_out), float(lr), _ptr(d_status), stream))

@@ -32,11 +32,7 @@ bool geometry_ok(const hl_geometry* g, int64_t* total_rows) {
     return true;
 }
 
-int64_t hist_words(int64_t max_nnz) {
-    const int64_t n_tiles = div_up(max_nnz > 0 ? max_nnz : 1, kSortTile);
-    const int64_t n_hist = 256 * n_tiles;
-    return n_hist + 1 + n_hist / kScanTile + 8;
-}
+int64_t hist_words(int64_t max_nnz) { return sort_hist_words(max_nnz); }
 
 // Lays the regions out over `base` (nullptr: size only).  Returns the bytes used.
 size_t carve(char* base, const hl_geometry* g, int64_t N, int32_t max_batch, int64_t max_nnz, int64_t hot_cap,

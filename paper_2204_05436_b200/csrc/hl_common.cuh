@@ -139,6 +139,13 @@ int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, 
 int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n, int64_t n_max, int key_bits,
                          uint32_t* hist, int32_t** out_keys, int32_t** out_vals, cudaStream_t stream);
 
+// 32-bit words of histogram scratch radix_sort_pairs needs for at most max_nnz pairs.
+constexpr int64_t sort_hist_words(int64_t max_nnz) {
+    const int64_t n_tiles = ((max_nnz > 0 ? max_nnz : 1) + kSortTile - 1) / kSortTile;
+    const int64_t n_hist = 256 * n_tiles;
+    return n_hist + 1 + n_hist / kScanTile + 8;
+}
+
 // Process-wide count of kernels this library has launched (read by hl_launch_count).
 void note_launches(int n);
 

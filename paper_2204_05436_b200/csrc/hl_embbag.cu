@@ -1,6 +1,8 @@
 // Embedding bag over the HBM cache: sum-pooling forward, and scatter-add + SGD backward with one update per
 // distinct row.  Rows are fp32 [*, D]; a group of G lanes owns one row at a time, each lane NV float4 columns,
 // so that a row is read with 128-bit loads that coalesce into whole sectors.
+#include <mutex>
+
 #include "hl_common.cuh"
 
 namespace hl {
@@ -436,4 +438,110 @@ extern "C" int32_t hl_embbag_bwd_sgd(hl_ctx* ctx, float* d_cache, const hl_ubatc
 #define HL_BWD(G, NV) launch_bwd<G, NV>(ctx, d_cache, keys, vals, d_grad_out, lr, stream)
     HL_DISPATCH_ROW_SHAPE(ctx->D / 4, HL_BWD);
 #undef HL_BWD
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Backward without a context or a workspace: the scratch is a fixed array inside the library image.
+// ---------------------------------------------------------------------------------------------------------------
+namespace hl {
+namespace {
+
+constexpr int64_t kStaticMaxNnz = HL_STATIC_MAX_NNZ;
+constexpr int64_t kStaticMaxDim = HL_STATIC_MAX_DIM;
+
+constexpr size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+// layout of the static scratch: [header: status (8 ints), bag count word + lookup count (8 ints)] [keys x2]
+// [vals x2] [histogram] [partial sums]
+constexpr size_t kStaticHeaderBytes = 256;
+constexpr size_t kStaticPairBytes = align256(size_t(kStaticMaxNnz) * sizeof(int32_t));
+constexpr int64_t kStaticHistWords = sort_hist_words(kStaticMaxNnz);
+constexpr size_t kStaticHistBytes = align256(size_t(kStaticHistWords) * sizeof(uint32_t));
+constexpr size_t kStaticPartBytes =
+    align256(size_t(2) * ((kStaticMaxNnz + kBwdChunk - 1) / kBwdChunk) * kStaticMaxDim * sizeof(float));
+constexpr size_t kStaticScratchBytes = kStaticHeaderBytes + 4 * kStaticPairBytes + kStaticHistBytes + kStaticPartBytes;
+
+// Lives in every device's copy of the library image from load to exit (about 3 MB).  The name below is only a
+// host-side handle for cudaGetSymbolAddress; kernels get the real device address as an argument.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+std::mutex g_static_mutex;
+unsigned char* g_static_ptr[64] = {};   // device address of g_static_scratch, per device ordinal
+
+__global__ void k_static_begin(int32_t* header, int32_t n_bags) {
+    header[0] = 0;        // status word: every call starts clean
+    header[8] = n_bags;   // the backward kernels read their bag count from device memory
+}
+
+__global__ void k_static_end(const int32_t* header, int32_t* d_status) { *d_status = header[0]; }
+
+}  // namespace
+}  // namespace hl
+
+extern "C" int32_t hl_embbag_bwd_sgd_static(float* d_cache, int64_t cache_rows, int32_t dim,
+                                            const int32_t* d_offsets, const int32_t* d_ids, int32_t n_bags,
+                                            int64_t nnz, const float* d_grad_out, float lr, int32_t* d_status,
+                                            void* stream_) {
+    if (!d_cache || !d_offsets || !d_grad_out || cache_rows < 1 || cache_rows >= (int64_t(1) << 31) - 2)
+        return HL_EINVAL;
+    if (dim < 4 || (dim & 3) || n_bags < 0 || nnz < 0 || (nnz > 0 && !d_ids)) return HL_EINVAL;
+    if (nnz > kStaticMaxNnz || n_bags > kStaticMaxNnz || dim > kStaticMaxDim) return HL_ECAPACITY;
+    if (sort_hist_words(nnz) > kStaticHistWords) return HL_ECAPACITY;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    // set-up, once per device: ask the runtime where this device keeps the array
+    int dev = 0;
+    HL_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return HL_EINVAL;
+    unsigned char* base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[dev]) {
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return HL_ECUDA;
+            g_static_ptr[dev] = static_cast<unsigned char*>(p);
+        }
+        base = g_static_ptr[dev];
+    }
+    if (nnz == 0 || n_bags == 0) {
+        if (d_status) HL_CUDA_TRY(cudaMemsetAsync(d_status, 0, sizeof(int32_t), stream));
+        return HL_OK;
+    }
+
+    // a context on the stack whose backward region points into the static array; nothing else is used
+    hl_ctx tmp{};
+    tmp.T = 1;
+    tmp.S = 1;
+    tmp.D = dim;
+    tmp.N = cache_rows;
+    tmp.max_batch = n_bags;
+    tmp.max_bags = n_bags;
+    tmp.max_nnz = nnz;
+    tmp.hot_cap = cache_rows;
+    tmp.staging_cap = 0;
+    int32_t* header = reinterpret_cast<int32_t*>(base);
+    unsigned char* p = base + kStaticHeaderBytes;
+    tmp.r.status = header;
+    tmp.r.bwd_n = header + 12;
+    for (int i = 0; i < 2; ++i) {
+        tmp.r.bwd_keys[i] = reinterpret_cast<int32_t*>(p);
+        p += kStaticPairBytes;
+        tmp.r.bwd_vals[i] = reinterpret_cast<int32_t*>(p);
+        p += kStaticPairBytes;
+    }
+    tmp.r.bwd_hist = reinterpret_cast<uint32_t*>(p);
+    p += kStaticHistBytes;
+    tmp.r.bwd_part = reinterpret_cast<float*>(p);
+
+    k_static_begin<<<1, 1, 0, stream>>>(header, n_bags);
+    note_launches(1);
+    HL_LAUNCH_CHECK();
+    hl_ubatch ub{const_cast<int32_t*>(d_offsets), const_cast<int32_t*>(d_ids), nnz};
+    const int32_t st = hl_embbag_bwd_sgd(&tmp, d_cache, &ub, header + 8, d_grad_out, lr, stream_);
+    if (st != HL_OK) return st;
+    if (d_status) {
+        k_static_end<<<1, 1, 0, stream>>>(header, d_status);
+        note_launches(1);
+        HL_LAUNCH_CHECK();
+    }
+    return HL_OK;
 }
