@@ -480,6 +480,70 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
     wl.free()
 
 
+# ----------------------------------------------------------------------------------------------------------
+# single-call micro runs (the small cases the ncu captures under profiles/ are taken on)
+# ----------------------------------------------------------------------------------------------------------
+def run_micro(args) -> None:
+    """`--micro fwd|bwd`: one library call in isolation on an all-popular ("hot-only") micro-batch with the
+    DLRM-large-like shape (26 tables x `--micro-batch` inputs, dim 64, one lookup per bag) over a 1 GiB cache.
+    Slots are uniform over the cache (`--micro-dist uniform`: no reuse, every row comes from HBM) or Zipf(1.2)
+    within each table's share of the cache (`zipf`: long runs of equal slots, as in the real workload)."""
+    import torch
+    import paper_2204_05436_b200 as hl
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    T, D, S, B = 26, args.micro_dim, 1, args.micro_batch
+    H = (1 << 30) // (4 * D)
+    n_bags = T * B
+    rng = np.random.default_rng(5)
+    if args.micro_dist == "uniform":
+        ids = rng.integers(0, H, n_bags, dtype=np.int64)
+    else:
+        per = H // T
+        ids = np.concatenate([t * per + gen.feistel_permute(gen.zipf_ranks(rng, 1.2, per, B) - 1, per, 17 + t)
+                              for t in range(T)])
+    geom = hl.make_geometry([H], D, 1)            # one "table" as large as the cache: slots are what matter here
+    ws_bytes = hl.hl_workspace_bytes(geom, n_bags, n_bags, H, 0)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    ctx = hl.hl_create(geom, n_bags, n_bags, H, 0, ws, ws_bytes)
+    cache = torch.rand((H, D), device=dev, dtype=torch.float32) - 0.5
+    d_ids = torch.from_numpy(ids.astype(np.int32)).to(dev)
+    d_off = torch.arange(n_bags + 1, dtype=torch.int32, device=dev)
+    d_n = torch.tensor([n_bags], dtype=torch.int32, device=dev)
+    out = torch.empty((n_bags, D), dtype=torch.float32, device=dev)
+    grad = torch.randn((n_bags, D), dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    ub = hl.make_ubatch(d_off, d_ids, n_bags)
+    stream = torch.cuda.current_stream().cuda_stream
+    distinct = int(np.unique(ids).shape[0])
+    if args.micro == "fwd":
+        call = lambda: hl.hl_embbag_fwd(ctx, cache, ub, d_n, out, stream)   # noqa: E731
+        nbytes = n_bags * (4 * D + 4) + n_bags * (4 * D + 4)
+    else:
+        call = lambda: hl.hl_embbag_bwd_sgd(ctx, cache, ub, d_n, grad, 1e-3, stream)   # noqa: E731
+        nbytes = n_bags * (4 * D + 8) + distinct * 2 * 4 * D
+    for _ in range(max(3, args.warmup)):
+        call()
+    times = []
+    for _ in range(args.steps):
+        flush.zero_()                      # write 256 MB: nothing of the previous call is left in the 126 MB L2
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        call()
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b) * 1e3)
+    hl.hl_status(ctx)
+    us = statistics.median(times)
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak = float(json.load(open(peaks_path))["hbm_gbs"]) if os.path.exists(peaks_path) else FALLBACK_HBM_GBS
+    print(json.dumps({"micro": args.micro, "dist": args.micro_dist, "bags": n_bags, "dim": D, "distinct_rows": distinct,
+                      "us_median": us, "us_min": min(times), "algorithmic_bytes": nbytes,
+                      "gbs": nbytes / us / 1e3, "frac_of_hbm_peak": nbytes / us / 1e3 / peak, "peak_gbs": peak,
+                      "l2": "flushed between calls (256 MB write)"}), flush=True)
+    hl.hl_destroy(ctx)
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -491,7 +555,14 @@ def main() -> None:
     ap.add_argument("--threads", type=int, default=min(16, os.cpu_count() or 1))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--micro", default=None, choices=["fwd", "bwd"], help="time one library call in isolation")
+    ap.add_argument("--micro-dist", default="uniform", choices=["uniform", "zipf"])
+    ap.add_argument("--micro-batch", type=int, default=16384)
+    ap.add_argument("--micro-dim", type=int, default=64)
     args = ap.parse_args()
+    if args.micro:
+        run_micro(args)
+        return
     if args.warmup < 3:
         log("[bench] warm-up raised to 3 steps")
         args.warmup = 3

@@ -52,7 +52,7 @@ size_t carve(char* base, const hl_geometry* g, int64_t N, int32_t max_batch, int
     r->sel_eq = c.take<uint32_t>(*n_sel_tiles + 2);
     r->frag_flags = c.take<uint8_t>(max_batch);
     r->frag_scan = c.take<int32_t>(max_bags + 2);
-    r->frag_tiles = c.take<int32_t>(max_bags / kScanTile + 4);
+    r->frag_tiles = c.take<int32_t>(scan_tile_words(max_bags));
     for (int i = 0; i < 2; ++i) {
         r->bwd_keys[i] = c.take<int32_t>(nnz);
         r->bwd_vals[i] = c.take<int32_t>(nnz);
@@ -66,7 +66,7 @@ size_t carve(char* base, const hl_geometry* g, int64_t N, int32_t max_batch, int
     }
     r->cold_hist = c.take<uint32_t>(hist_words(nnz));
     r->cold_rank = c.take<int32_t>(nnz + 2);
-    r->cold_tiles = c.take<int32_t>(nnz / kScanTile + 4);
+    r->cold_tiles = c.take<int32_t>(scan_tile_words(nnz));
     r->cold_n = c.take<int32_t>(4);
     (void)hot_cap;
     (void)staging_cap;
@@ -95,7 +95,7 @@ extern "C" int32_t hl_create(hl_ctx** out, const hl_geometry* geom, int32_t max_
     if (!geometry_ok(geom, &N) || max_batch < 1 || max_nnz < 0 || hot_cap_rows < 0 || staging_cap_rows < 0)
         return HL_EINVAL;
     const int64_t max_bags = (int64_t)geom->num_tables * max_batch * geom->bags_per_sample;
-    if (max_bags >= (int64_t(1) << 31) - 2 || max_nnz >= (int64_t(1) << 31) - 2) return HL_EINVAL;
+    if (max_bags >= (int64_t(1) << 30) || max_nnz >= (int64_t(1) << 30)) return HL_EINVAL;   // 30-bit chain values
     if (hot_cap_rows + staging_cap_rows >= (int64_t(1) << 31) - 2) return HL_EINVAL;
     if (!d_workspace || (reinterpret_cast<uintptr_t>(d_workspace) & 255)) return HL_EINVAL;
 

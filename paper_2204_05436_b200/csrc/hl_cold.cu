@@ -200,12 +200,12 @@ extern "C" int32_t hl_gather_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_
     HL_LAUNCH_CHECK();
     int32_t *keys, *vals;
     int32_t st = radix_sort_pairs(r.cold_keys, r.cold_vals, r.cold_n, ctx->max_nnz, bits_for(ctx->N - 1),
-                                  r.cold_hist, &keys, &vals, stream);
+                                  r.cold_hist, r.status, &keys, &vals, stream);
     if (st != HL_OK) return st;
     k_cold_heads<<<grid, kThreads, 0, stream>>>(keys, r.cold_n, ctx->max_nnz, r.cold_rank);
     note_launches(1);
     HL_LAUNCH_CHECK();
-    st = exclusive_scan_i32(r.cold_rank, r.cold_rank, r.cold_n, ctx->max_nnz, r.cold_tiles, stream);
+    st = exclusive_scan_i32(r.cold_rank, r.cold_rank, r.cold_n, ctx->max_nnz, r.cold_tiles, r.status, stream);
     if (st != HL_OK) return st;
     k_cold_assign<<<grid, kThreads, 0, stream>>>(keys, vals, r.cold_n, ctx->max_nnz, r.cold_rank, ctx->hot_cap,
                                                  ctx->staging_cap, non->ids, d_cold_rows, d_n_cold, r.status);

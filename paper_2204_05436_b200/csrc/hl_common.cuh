@@ -130,21 +130,25 @@ __device__ __forceinline__ unsigned lanemask_lt() {
 
 // ---- primitives implemented in hl_prims.cu -----------------------------------------------------------------
 // Exclusive scan of in[0 .. n) into out[0 .. n] (out[n] = total); n = *d_n if d_n != nullptr (clamped to
-// n_max), else n_max.  in may alias out.  tiles: scratch of n_max / kScanTile + 2 ints.
+// n_max), else n_max.  in may alias out.  tiles: scratch of scan_tile_words(n_max) ints.  A chain poll that
+// gives up records HL_ETIMEOUT in *status.
 int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, int64_t n_max, int32_t* tiles,
-                           cudaStream_t stream);
+                           int32_t* status, cudaStream_t stream);
 
 // Stable LSD radix sort of (key, value) pairs by the low key_bits bits of the non-negative keys.
 // n = *d_n (clamped to n_max).  Returns in *out_keys / *out_vals which of the two buffers holds the result.
 int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n, int64_t n_max, int key_bits,
-                         uint32_t* hist, int32_t** out_keys, int32_t** out_vals, cudaStream_t stream);
+                         uint32_t* hist, int32_t* status, int32_t** out_keys, int32_t** out_vals,
+                         cudaStream_t stream);
 
 // 32-bit words of histogram scratch radix_sort_pairs needs for at most max_nnz pairs.
 constexpr int64_t sort_hist_words(int64_t max_nnz) {
     const int64_t n_tiles = ((max_nnz > 0 ? max_nnz : 1) + kSortTile - 1) / kSortTile;
-    const int64_t n_hist = 256 * n_tiles;
-    return n_hist + 1 + n_hist / kScanTile + 8;
+    return 4 * 256 + 8 + 4 * n_tiles * 256;   // digit counts, tickets, tile status words for up to 4 passes
 }
+
+// ints of scratch exclusive_scan_i32 needs for at most n_max elements (64-bit ticket + status words).
+constexpr int64_t scan_tile_words(int64_t n_max) { return 2 * ((n_max > 0 ? n_max : 1) / kScanTile + 3); }
 
 // Process-wide count of kernels this library has launched (read by hl_launch_count).
 void note_launches(int n);

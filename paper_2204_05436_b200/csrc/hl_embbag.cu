@@ -25,8 +25,52 @@ __device__ __forceinline__ int clamp_samples(const int32_t* d_n_samples, int max
 }
 
 // ---- forward ------------------------------------------------------------------------------------------------
-// Each group takes UB consecutive bags per trip and walks them in lock step, so that UB independent row loads
-// are in flight per lane.
+// A bag of several lookups, finished by one group of G lanes: rows are added in lookup order in fp64, four loads
+// in flight, and the sum is rounded once (so cancellation between the rows of a bag costs no accuracy).
+template <int G, int NV>
+__device__ __forceinline__ void pool_long_bag(const float4* __restrict__ rows, const int32_t* __restrict__ ids,
+                                           int32_t lo, int32_t len, int sub, int D4, int64_t n_slots,
+                                           float4* __restrict__ dst, int32_t* status) {
+    double acc[NV][4];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0.0;
+    for (int32_t p = 0; p < len; p += 4) {
+        int32_t id[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) id[k] = p + k < len ? __ldg(&ids[lo + p + k]) : -1;
+        float4 r[4][NV];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const bool ok = id[k] >= 0 && id[k] < n_slots;
+            if (id[k] >= n_slots) set_status(status, HL_EBOUNDS);
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int c = sub + v * G;
+                r[k][v] = (ok && c < D4) ? __ldg(&rows[(int64_t)id[k] * D4 + c]) : f4_zero();
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                acc[v][0] += (double)r[k][v].x;
+                acc[v][1] += (double)r[k][v].y;
+                acc[v][2] += (double)r[k][v].z;
+                acc[v][3] += (double)r[k][v].w;
+            }
+    }
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c = sub + v * G;
+        if (c < D4)
+            __stcs(&dst[c], make_float4((float)acc[v][0], (float)acc[v][1], (float)acc[v][2], (float)acc[v][3]));
+    }
+}
+
+// A group of G lanes takes UB consecutive bags per trip.  Bags of at most one lookup (the one-hot case) are plain
+// row copies: the UB rows are loaded at once (UB independent 128-bit loads per lane), and the offsets and ids of
+// the NEXT trip are requested before those rows are consumed, so that the offsets -> id -> row chain of one trip
+// hides behind the rows of another.  Longer bags go through pool_long_bag one after the other.
 template <int G, int NV, int UB>
 __global__ void __launch_bounds__(kThreads) k_embbag_fwd(const float* __restrict__ cache,
                                                          const int32_t* __restrict__ ids,
@@ -41,87 +85,60 @@ __global__ void __launch_bounds__(kThreads) k_embbag_fwd(const float* __restrict
     const float4* __restrict__ rows = reinterpret_cast<const float4*>(cache);
     float4* __restrict__ out4 = reinterpret_cast<float4*>(out);
 
-    for (int64_t bag0 = group * UB; bag0 < n_bags; bag0 += n_groups * UB) {
-        int32_t lo[UB], len[UB];
-        int32_t max_len = 0;
+    // lo/len of the UB bags of a trip, and the id of every bag that has exactly one lookup (-1 otherwise)
+    auto load_index = [&](int64_t bag0, int32_t (&lo)[UB], int32_t (&len)[UB], int32_t (&id1)[UB]) {
 #pragma unroll
         for (int u = 0; u < UB; ++u) {
             const int64_t bag = bag0 + u;
             const bool valid = bag < n_bags;
             lo[u] = valid ? __ldg(&offsets[bag]) : 0;
-            len[u] = valid ? __ldg(&offsets[bag + 1]) - lo[u] : 0;
-            max_len = max(max_len, len[u]);
+            len[u] = valid ? __ldg(&offsets[bag + 1]) - lo[u] : -1;
         }
-        // p-th lookup of each of the UB bags: UB independent row loads per lane
-        auto load_rows = [&](int32_t p, float4 (&r)[UB][NV]) {
-            int32_t id[UB];
 #pragma unroll
-            for (int u = 0; u < UB; ++u) id[u] = p < len[u] ? __ldg(&ids[lo[u] + p]) : -1;
-#pragma unroll
-            for (int u = 0; u < UB; ++u) {
-                const bool ok = id[u] >= 0 && id[u] < n_slots;
-                if (id[u] >= n_slots) set_status(status, HL_EBOUNDS);
-#pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    const int c = sub + v * G;
-                    r[u][v] = (ok && c < D4) ? __ldg(&rows[(int64_t)id[u] * D4 + c]) : f4_zero();
-                }
-            }
-        };
-        float4 first[UB][NV];
-        load_rows(0, first);
-        if (max_len <= 1) {
-            // bags of at most one lookup: the pooled vector is the row itself (or zeros), a plain copy
-#pragma unroll
-            for (int u = 0; u < UB; ++u) {
-                const int64_t bag = bag0 + u;
-                if (bag < n_bags) {
-#pragma unroll
-                    for (int v = 0; v < NV; ++v) {
-                        const int c = sub + v * G;
-                        if (c < D4) __stcs(&out4[bag * D4 + c], first[u][v]);
-                    }
-                }
-            }
-            continue;
-        }
-        // longer bags: add in lookup order in fp64 and round once, so that the result does not depend on
-        // cancellation between the rows of a bag
-        double acc[UB][NV][4];
-#pragma unroll
-        for (int u = 0; u < UB; ++u)
-#pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                acc[u][v][0] = first[u][v].x;
-                acc[u][v][1] = first[u][v].y;
-                acc[u][v][2] = first[u][v].z;
-                acc[u][v][3] = first[u][v].w;
-            }
-        for (int32_t p = 1; p < max_len; ++p) {
-            float4 r[UB][NV];
-            load_rows(p, r);
-#pragma unroll
-            for (int u = 0; u < UB; ++u)
-#pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    acc[u][v][0] += (double)r[u][v].x;
-                    acc[u][v][1] += (double)r[u][v].y;
-                    acc[u][v][2] += (double)r[u][v].z;
-                    acc[u][v][3] += (double)r[u][v].w;
-                }
-        }
+        for (int u = 0; u < UB; ++u) id1[u] = len[u] == 1 ? __ldg(&ids[lo[u]]) : -1;
+    };
+
+    int32_t lo[UB], len[UB], id1[UB];
+    int64_t bag0 = group * UB;
+    if (bag0 < n_bags) load_index(bag0, lo, len, id1);
+    for (; bag0 < n_bags; bag0 += n_groups * UB) {
+        float4 row[UB][NV];
 #pragma unroll
         for (int u = 0; u < UB; ++u) {
-            const int64_t bag = bag0 + u;
-            if (bag < n_bags) {
+            const bool ok = id1[u] >= 0 && id1[u] < n_slots;
+            if (id1[u] >= n_slots) set_status(status, HL_EBOUNDS);
 #pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    const int c = sub + v * G;
-                    if (c < D4)
-                        __stcs(&out4[bag * D4 + c], make_float4((float)acc[u][v][0], (float)acc[u][v][1],
-                                                               (float)acc[u][v][2], (float)acc[u][v][3]));
-                }
+            for (int v = 0; v < NV; ++v) {
+                const int c = sub + v * G;
+                row[u][v] = (ok && c < D4) ? __ldg(&rows[(int64_t)id1[u] * D4 + c]) : f4_zero();
             }
+        }
+        int32_t cur_len[UB];
+#pragma unroll
+        for (int u = 0; u < UB; ++u) cur_len[u] = len[u];
+        const int64_t next0 = bag0 + n_groups * UB;
+        if (next0 < n_bags) load_index(next0, lo, len, id1);   // in flight while this trip's rows arrive
+        unsigned long_bags = 0;   // bit u: bag u of this trip has more than one lookup
+#pragma unroll
+        for (int u = 0; u < UB; ++u) {
+            if (cur_len[u] < 0) continue;   // past the last bag
+            if (cur_len[u] > 1) {
+                long_bags |= 1u << u;
+                continue;
+            }
+            float4* dst = out4 + (bag0 + u) * D4;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int c = sub + v * G;
+                if (c < D4) __stcs(&dst[c], row[u][v]);
+            }
+        }
+        while (long_bags) {   // one copy of the pooling loop, whichever bag of the trip it serves
+            const int u = __ffs(long_bags) - 1;
+            long_bags &= long_bags - 1;
+            const int64_t bag = bag0 + u;
+            const int32_t b_lo = __ldg(&offsets[bag]), b_len = __ldg(&offsets[bag + 1]) - b_lo;
+            pool_long_bag<G, NV>(rows, ids, b_lo, b_len, sub, D4, n_slots, out4 + bag * D4, status);
         }
     }
 }
@@ -353,9 +370,18 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
 template <int G, int NV>
 int32_t launch_fwd(hl_ctx* ctx, const float* cache, const hl_ubatch* ub, const int32_t* d_n, float* out,
                    cudaStream_t stream) {
-    constexpr int UB = NV >= 8 ? 1 : (NV >= 4 ? 2 : 4);
+    constexpr int UB = NV >= 4 ? 1 : (NV >= 2 ? 2 : 4);
+    // persistent grid: as many CTAs as fit on the chip at once (a whole number per SM), never more than the work
+    static int ctas_per_sm = 0;
+    if (ctas_per_sm == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_embbag_fwd<G, NV, UB>, kThreads, 0) != cudaSuccess ||
+            n < 1)
+            n = 2;
+        ctas_per_sm = n;
+    }
     const int64_t max_bags = ctx->max_bags;
-    const int grid = grid_for(div_up(max_bags, UB) * G, kThreads, kSMs * 8);
+    const int grid = grid_for(div_up(max_bags, UB) * G, kThreads, kSMs * ctas_per_sm);
     k_embbag_fwd<G, NV, UB><<<grid, kThreads, 0, stream>>>(cache, ub->ids, ub->offsets, d_n, ctx->max_batch,
                                                           ctx->T * ctx->S, ctx->D / 4,
                                                           ctx->hot_cap + ctx->staging_cap, out, ctx->r.status);
@@ -433,7 +459,7 @@ extern "C" int32_t hl_embbag_bwd_sgd(hl_ctx* ctx, float* d_cache, const hl_ubatc
     HL_LAUNCH_CHECK();
     int32_t *keys, *vals;
     int32_t st = radix_sort_pairs(r.bwd_keys, r.bwd_vals, r.bwd_n, ctx->max_nnz, bits_for(n_slots), r.bwd_hist,
-                                  &keys, &vals, stream);
+                                  r.status, &keys, &vals, stream);
     if (st != HL_OK) return st;
 #define HL_BWD(G, NV) launch_bwd<G, NV>(ctx, d_cache, keys, vals, d_grad_out, lr, stream)
     HL_DISPATCH_ROW_SHAPE(ctx->D / 4, HL_BWD);

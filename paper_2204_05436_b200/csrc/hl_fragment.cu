@@ -252,7 +252,7 @@ extern "C" int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_de
                                                                                d_counts, r.frag_scan);
     note_launches(3);   // flags, partition, sizes
     HL_LAUNCH_CHECK();
-    int32_t st = exclusive_scan_i32(r.frag_scan, r.frag_scan, nullptr, n_bags, r.frag_tiles, stream);
+    int32_t st = exclusive_scan_i32(r.frag_scan, r.frag_scan, nullptr, n_bags, r.frag_tiles, r.status, stream);
     if (st != HL_OK) return st;
     if (b->nnz <= 4 * n_bags)
         k_frag_emit<1><<<grid_for(n_bags, kThreads, kSMs * 8), kThreads, 0, stream>>>(

@@ -1,4 +1,5 @@
-// Device-wide primitives used by several steps: exclusive scan and stable LSD radix sort of pairs.
+// Device-wide primitives used by several steps: single-pass exclusive scan and stable LSD radix sort of pairs
+// (one kernel per digit; tiles chained through status words instead of a separate scan of tile histograms).
 // Both take their element count from device memory, so that no step has to synchronise the host.
 #include <atomic>
 
@@ -53,53 +54,46 @@ __device__ __forceinline__ int64_t clamp_n(const int32_t* d_n, int64_t n_max) {
     return n < n_max ? n : n_max;
 }
 
+// ---- single-pass chaining between tiles --------------------------------------------------------------------
+// Tiles are handed out by a ticket counter, so a tile's predecessors are always held by blocks that have
+// started.  A tile first publishes its own sum (AGGREGATE), then walks back over its predecessors adding their
+// sums until it meets one that already knows its inclusive prefix (PREFIX), and finally publishes its own
+// prefix.  Publishing never waits on anything, so the walk always terminates; every poll is bounded all the same,
+// and a poll that runs out records HL_ETIMEOUT and carries on with what it has (positions are range-checked).
+constexpr uint32_t kFlagAgg = 1u << 30, kFlagPrefix = 1u << 31, kValueMask = kFlagAgg - 1u;
+constexpr unsigned long long kFlagAgg64 = 1ull << 62, kFlagPrefix64 = 1ull << 63, kValueMask64 = kFlagAgg64 - 1ull;
+constexpr int kMaxPolls = 1 << 20;
+
+__device__ __forceinline__ uint32_t ld_relaxed(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed(uint32_t* p, uint32_t v) {
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long ld_relaxed64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
 // ---- scan ---------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) k_scan_tile_sums(const int32_t* __restrict__ in, const int32_t* d_n,
-                                                             int64_t n_max, int32_t* __restrict__ tiles) {
+// st[0] = ticket counter, st[1 + tile] = status word of the tile; all zero on entry.
+__global__ void __launch_bounds__(kThreads) k_scan_chained(const int32_t* in, int32_t* out, const int32_t* d_n,
+                                                           int64_t n_max, unsigned long long* st, int32_t* status) {
     __shared__ int smem[40];
+    __shared__ long long s_tile, s_excl;
+    if (threadIdx.x == 0) s_tile = (long long)atomicAdd(&st[0], 1ull);
+    __syncthreads();
+    const int64_t tile = s_tile;
     const int64_t n = clamp_n(d_n, n_max);
-    const int64_t base = (int64_t)blockIdx.x * kScanTile + (int64_t)threadIdx.x * kItems;
-    int s = 0;
-#pragma unroll
-    for (int i = 0; i < kItems; ++i)
-        if (base + i < n) s += in[base + i];
-    int total;
-    block_exclusive_scan(s, smem, total);
-    if (threadIdx.x == 0) tiles[blockIdx.x] = total;
-}
-
-// Single block: exclusive scan of vals[0 .. count) in place, vals[count] = total.
-__global__ void __launch_bounds__(1024) k_scan_spine(int32_t* __restrict__ vals, int64_t count) {
-    __shared__ int smem[40];
-    constexpr int kPer = 16;
-    int carry = 0;
-    for (int64_t start = 0; start < count; start += 1024 * kPer) {
-        const int64_t base = start + (int64_t)threadIdx.x * kPer;
-        int v[kPer];
-        int s = 0;
-#pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            v[i] = base + i < count ? vals[base + i] : 0;
-            s += v[i];
-        }
-        int total;
-        int excl = block_exclusive_scan(s, smem, total) + carry;
-#pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-            if (base + i < count) vals[base + i] = excl;
-            excl += v[i];
-        }
-        carry += total;
-    }
-    if (threadIdx.x == 0) vals[count] = carry;
-}
-
-__global__ void __launch_bounds__(kThreads) k_scan_apply(const int32_t* in, int32_t* out, const int32_t* d_n,
-                                                         int64_t n_max, const int32_t* __restrict__ tiles,
-                                                         int64_t n_tiles) {
-    __shared__ int smem[40];
-    const int64_t n = clamp_n(d_n, n_max);
-    const int64_t base = (int64_t)blockIdx.x * kScanTile + (int64_t)threadIdx.x * kItems;
+    const int64_t tile_base = tile * kScanTile;
+    if (tile_base > n) return;   // the tile at tile_base == n has no element but still writes out[n]
+    const int64_t base = tile_base + (int64_t)threadIdx.x * kItems;
     int v[kItems];
     int s = 0;
 #pragma unroll
@@ -108,49 +102,80 @@ __global__ void __launch_bounds__(kThreads) k_scan_apply(const int32_t* in, int3
         s += v[i];
     }
     int total;
-    int excl = block_exclusive_scan(s, smem, total) + tiles[blockIdx.x];
+    int excl = block_exclusive_scan(s, smem, total);
+    if (threadIdx.x == 0) {
+        long long before = 0;
+        if (tile > 0) {
+            st_relaxed64(&st[1 + tile], kFlagAgg64 | (unsigned long long)total);
+            for (int64_t t = tile - 1; t >= 0; --t) {
+                unsigned long long w = 0;
+                int polls = 0;
+                while (((w = ld_relaxed64(&st[1 + t])) & (kFlagAgg64 | kFlagPrefix64)) == 0) {
+                    if (++polls > kMaxPolls) {
+                        set_status(status, HL_ETIMEOUT);
+                        break;
+                    }
+                    __nanosleep(20);
+                }
+                before += (long long)(w & kValueMask64);
+                if ((w & kFlagPrefix64) || polls > kMaxPolls) break;
+            }
+        }
+        st_relaxed64(&st[1 + tile], kFlagPrefix64 | (unsigned long long)(before + total));
+        s_excl = before;
+        if (n < tile_base + kScanTile) out[n] = (int32_t)(before + total);
+    }
+    __syncthreads();
+    excl += (int)s_excl;
 #pragma unroll
     for (int i = 0; i < kItems; ++i) {
         if (base + i < n) out[base + i] = excl;
         excl += v[i];
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) out[n] = tiles[n_tiles];
 }
 
 // ---- radix sort ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) k_sort_hist(const int32_t* __restrict__ keys, const int32_t* d_n,
-                                                        int64_t n_max, int shift, uint32_t* __restrict__ hist,
-                                                        int64_t n_tiles) {
-    __shared__ uint32_t h[256];
-    h[threadIdx.x] = 0;
+// Digit histograms of all passes in one sweep over the keys.
+__global__ void __launch_bounds__(kThreads) k_sort_digit_hist(const int32_t* __restrict__ keys, const int32_t* d_n,
+                                                              int64_t n_max, int passes,
+                                                              uint32_t* __restrict__ ghist /* [passes][256] */) {
+    __shared__ uint32_t h[4][256];
+    for (int i = threadIdx.x; i < 4 * 256; i += kThreads) (&h[0][0])[i] = 0;
     __syncthreads();
     const int64_t n = clamp_n(d_n, n_max);
-    const int64_t base = (int64_t)blockIdx.x * kSortTile;
-#pragma unroll
-    for (int i = 0; i < kItems; ++i) {
-        const int64_t idx = base + (int64_t)i * kThreads + threadIdx.x;
-        if (idx < n) atomicAdd(&h[((uint32_t)keys[idx] >> shift) & 255u], 1u);
+    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (int64_t)gridDim.x * kThreads) {
+        const uint32_t k = (uint32_t)keys[i];
+        for (int p = 0; p < passes; ++p) atomicAdd(&h[p][(k >> (8 * p)) & 255u], 1u);
     }
     __syncthreads();
-    hist[(int64_t)threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];
+    for (int i = threadIdx.x; i < passes * 256; i += kThreads) {
+        const uint32_t c = (&h[0][0])[i];
+        if (c) atomicAdd(&ghist[i], c);
+    }
 }
 
-// Stable scatter.  Order of the items of a tile: warp-major, then round, then lane.
-__global__ void __launch_bounds__(kThreads) k_sort_scatter(const int32_t* __restrict__ keys_in,
-                                                           const int32_t* __restrict__ vals_in,
-                                                           int32_t* __restrict__ keys_out,
-                                                           int32_t* __restrict__ vals_out, const int32_t* d_n,
-                                                           int64_t n_max, int shift,
-                                                           const uint32_t* __restrict__ hist, int64_t n_tiles) {
+// One pass: stable scatter by one digit.  Order of the items of a tile: warp-major, then round, then lane.
+// ghist: this pass's 256 digit counts; ticket: tile counter; tstat[tile][256]: status words, zero on entry.
+__global__ void __launch_bounds__(kThreads) k_sort_pass(const int32_t* __restrict__ keys_in,
+                                                        const int32_t* __restrict__ vals_in,
+                                                        int32_t* __restrict__ keys_out, int32_t* __restrict__ vals_out,
+                                                        const int32_t* d_n, int64_t n_max, int shift,
+                                                        const uint32_t* __restrict__ ghist, uint32_t* ticket,
+                                                        uint32_t* tstat, int32_t* status) {
     constexpr int kWarps = kThreads / 32;
     __shared__ uint32_t cnt[kWarps][256];
     __shared__ uint32_t digit_base[256];
+    __shared__ int scan_smem[40];
+    __shared__ uint32_t s_tile;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
     for (int i = threadIdx.x; i < kWarps * 256; i += kThreads) (&cnt[0][0])[i] = 0;
     __syncthreads();
-
+    const int64_t tile = s_tile;
     const int64_t n = clamp_n(d_n, n_max);
-    const int64_t warp_base = (int64_t)blockIdx.x * kSortTile + (int64_t)warp * (32 * kItems);
+    if (tile * kSortTile >= n) return;
+
+    const int64_t warp_base = tile * kSortTile + (int64_t)warp * (32 * kItems);
     int32_t key[kItems], val[kItems];
     uint32_t rank[kItems];
     const unsigned lt = lanemask_lt();
@@ -170,26 +195,48 @@ __global__ void __launch_bounds__(kThreads) k_sort_scatter(const int32_t* __rest
         __syncwarp();
     }
     __syncthreads();
-    {   // one thread per digit: exclusive prefix over the warps, plus this tile's global base for the digit
-        const int d = threadIdx.x;
-        uint32_t run = 0;
+    // one thread per digit: prefix over the warps; then chain with the earlier tiles
+    const int d = threadIdx.x;
+    uint32_t total = 0;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const uint32_t c = cnt[w][d];
-            cnt[w][d] = run;
-            run += c;
-        }
-        digit_base[d] = hist[(int64_t)d * n_tiles + blockIdx.x];
+    for (int w = 0; w < kWarps; ++w) {
+        const uint32_t c = cnt[w][d];
+        cnt[w][d] = total;
+        total += c;
     }
+    uint32_t before = 0;
+    uint32_t* my = tstat + tile * 256 + d;
+    if (tile > 0) {
+        st_relaxed(my, kFlagAgg | total);
+        for (int64_t t = tile - 1; t >= 0; --t) {
+            uint32_t w = 0;
+            int polls = 0;
+            while (((w = ld_relaxed(tstat + t * 256 + d)) & (kFlagAgg | kFlagPrefix)) == 0) {
+                if (++polls > kMaxPolls) {
+                    set_status(status, HL_ETIMEOUT);
+                    break;
+                }
+                __nanosleep(20);
+            }
+            before += w & kValueMask;
+            if ((w & kFlagPrefix) || polls > kMaxPolls) break;
+        }
+    }
+    st_relaxed(my, kFlagPrefix | ((before + total) & kValueMask));
+    int all;
+    const int gbase = block_exclusive_scan((int)ghist[d], scan_smem, all);   // keys with a smaller digit
+    digit_base[d] = (uint32_t)gbase + before;
     __syncthreads();
 #pragma unroll
     for (int r = 0; r < kItems; ++r) {
         const int64_t idx = warp_base + r * 32 + lane;
         if (idx < n) {
-            const uint32_t d = ((uint32_t)key[r] >> shift) & 255u;
-            const int64_t pos = (int64_t)digit_base[d] + cnt[warp][d] + rank[r];
-            keys_out[pos] = key[r];
-            vals_out[pos] = val[r];
+            const uint32_t dg = ((uint32_t)key[r] >> shift) & 255u;
+            const int64_t pos = (int64_t)digit_base[dg] + cnt[warp][dg] + rank[r];
+            if (pos < n) {   // always true unless a chain poll gave up
+                keys_out[pos] = key[r];
+                vals_out[pos] = val[r];
+            }
         }
     }
 }
@@ -197,46 +244,43 @@ __global__ void __launch_bounds__(kThreads) k_sort_scatter(const int32_t* __rest
 }  // namespace
 
 int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, int64_t n_max, int32_t* tiles,
-                           cudaStream_t stream) {
+                           int32_t* status, cudaStream_t stream) {
     if (n_max <= 0) {
         HL_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(int32_t), stream));
         return HL_OK;
     }
-    const int64_t n_tiles = div_up(n_max, kScanTile);
-    k_scan_tile_sums<<<(unsigned)n_tiles, kThreads, 0, stream>>>(in, d_n, n_max, tiles);
-    k_scan_spine<<<1, 1024, 0, stream>>>(tiles, n_tiles);
-    k_scan_apply<<<(unsigned)n_tiles, kThreads, 0, stream>>>(in, out, d_n, n_max, tiles, n_tiles);
-    note_launches(3);
+    const int64_t n_tiles = n_max / kScanTile + 1;   // one more than needed when n is a multiple of the tile
+    unsigned long long* st = reinterpret_cast<unsigned long long*>(tiles);
+    HL_CUDA_TRY(cudaMemsetAsync(st, 0, sizeof(unsigned long long) * (n_tiles + 1), stream));
+    k_scan_chained<<<(unsigned)n_tiles, kThreads, 0, stream>>>(in, out, d_n, n_max, st, status);
+    note_launches(1);
     HL_LAUNCH_CHECK();
     return HL_OK;
 }
 
 int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n, int64_t n_max, int key_bits,
-                         uint32_t* hist, int32_t** out_keys, int32_t** out_vals, cudaStream_t stream) {
+                         uint32_t* hist, int32_t* status, int32_t** out_keys, int32_t** out_vals,
+                         cudaStream_t stream) {
     int cur = 0;
     if (n_max > 0) {
         const int64_t n_tiles = div_up(n_max, kSortTile);
-        const int64_t n_hist = 256 * n_tiles;
         const int passes = (key_bits + 7) / 8;
+        if (passes > 4) return HL_EINVAL;
+        // scratch: [4][256] digit counts, 8 ticket words, [4][n_tiles][256] tile status words
+        uint32_t* ghist = hist;
+        uint32_t* ticket = hist + 4 * 256;
+        uint32_t* tstat = hist + 4 * 256 + 8;
+        HL_CUDA_TRY(cudaMemsetAsync(hist, 0, sizeof(uint32_t) * (4 * 256 + 8 + (size_t)passes * n_tiles * 256),
+                                    stream));
+        k_sort_digit_hist<<<grid_for(n_max, kThreads * 8, kSMs * 2), kThreads, 0, stream>>>(keys[0], d_n, n_max,
+                                                                                            passes, ghist);
         for (int p = 0; p < passes; ++p) {
-            const int shift = 8 * p;
-            k_sort_hist<<<(unsigned)n_tiles, kThreads, 0, stream>>>(keys[cur], d_n, n_max, shift, hist, n_tiles);
-            if (n_hist <= 65536) {
-                k_scan_spine<<<1, 1024, 0, stream>>>(reinterpret_cast<int32_t*>(hist), n_hist);
-                note_launches(1);
-            } else {
-                // the scan's tile sums live right behind the histogram (the workspace reserves the room)
-                int32_t* tiles = reinterpret_cast<int32_t*>(hist) + n_hist + 1;
-                int32_t st = exclusive_scan_i32(reinterpret_cast<int32_t*>(hist), reinterpret_cast<int32_t*>(hist),
-                                                nullptr, n_hist, tiles, stream);
-                if (st != HL_OK) return st;
-            }
-            k_sort_scatter<<<(unsigned)n_tiles, kThreads, 0, stream>>>(keys[cur], vals[cur], keys[cur ^ 1],
-                                                                      vals[cur ^ 1], d_n, n_max, shift, hist,
-                                                                      n_tiles);
-            note_launches(2);   // histogram + scatter
+            k_sort_pass<<<(unsigned)n_tiles, kThreads, 0, stream>>>(keys[cur], vals[cur], keys[cur ^ 1], vals[cur ^ 1],
+                                                                    d_n, n_max, 8 * p, ghist + 256 * p, ticket + p,
+                                                                    tstat + (size_t)p * n_tiles * 256, status);
             cur ^= 1;
         }
+        note_launches(1 + passes);
         HL_LAUNCH_CHECK();
     }
     *out_keys = keys[cur];
