@@ -33,9 +33,10 @@ UNIT = "samples/s"
 L2_BYTES = 126 << 20
 FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the roofline kernel, from the ncu capture summarised
-# under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {}
+# dram__bytes_read.sum + dram__bytes_write.sum of the forward kernel per bag at dim 64, from the ncu capture
+# summarised in profiles/k_embbag_fwd_micro_dim64.md (164.4 MB for 425,984 one-lookup bags).  The bench's own
+# launch is scaled from it by the number of bags it processes (traffic grows in proportion to the bags).
+NCU_FWD_TRAFFIC_BYTES_PER_BAG = {64: 164.4e6 / 425984}
 
 
 def log(*a):
@@ -137,51 +138,52 @@ class Workload:
 # clocks
 # ----------------------------------------------------------------------------------------------------------
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons of one GPU through NVML (read-only) every few milliseconds."""
 
-    def __init__(self, gpu_index: int):
-        self.path = tempfile.mktemp(prefix="hl_clocks_", suffix=".csv")
-        self.proc = None
-        self.gpu_index = gpu_index
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, gpu_index: int, period_s: float = 0.004):
+        self.period = period_s
+        self.samples, self.reasons = [], set()
+        self.stop_flag = threading.Event()
+        self.thread = None
+        self.handle = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = int(vis.split(",")[gpu_index]) if vis and vis.split(",")[gpu_index].isdigit() else gpu_index
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception as e:   # noqa: BLE001
+            self.err = repr(e)
+
+    def _run(self):
+        nv = self.nv
+        while not self.stop_flag.is_set():
+            try:
+                self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:   # noqa: BLE001
+                pass
+            time.sleep(self.period)
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
-        except OSError:
-            self.proc = None
+        if self.handle is not None:
+            self.thread = threading.Thread(target=self._run, daemon=True)
+            self.thread.start()
 
     def stop(self) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        try:
-            for line in open(self.path):
-                f = [x.strip() for x in line.split(",")]
-                if len(f) < 9:
-                    continue
-                try:
-                    sm.append(float(f[1]))
-                    mx.append(float(f[2]))
-                except ValueError:
-                    continue
-                for name, val in zip(names, f[5:9]):
-                    if val.lower().startswith("active"):
-                        reasons.add(name)
-            os.unlink(self.path)
-        except OSError:
-            pass
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        if self.thread is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["NVML unavailable"]}
+        self.stop_flag.set()
+        self.thread.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.sm_max,
+                "samples": len(self.samples), "reasons": sorted(self.reasons)}
 
 
 # ----------------------------------------------------------------------------------------------------------
@@ -362,6 +364,32 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         h.status()
         ms_total = ev0.elapsed_time(ev1)
 
+        # ---- kernel timers and host link (diagnostic pass, outside the timed region) ----
+        hl.hl_timing_enable(h.ctx, True)
+        kt = {"gather_move": [], "scatter_move": [], "bwd_reduce_non": [], "fwd_non": []}
+        for k in range(n_batches):
+            one_step(k)
+            torch.cuda.synchronize()
+            kt["gather_move"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_GATHER_MOVE), sizes[k]["n_cold"]))
+            kt["scatter_move"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_SCATTER_MOVE), sizes[k]["n_cold"]))
+            kt["bwd_reduce_non"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_BWD_REDUCE), sizes[k]["L_non"]))
+            kt["fwd_non"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_FWD), sizes[k]["L_non"]))
+        hl.hl_timing_enable(h.ctx, False)
+        link = {}
+        buf_h = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
+        buf_d = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        for nm, (dst, src) in {"h2d": (buf_d, buf_h), "d2h": (buf_h, buf_d)}.items():
+            best = 0.0
+            for _ in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                dst.copy_(src, non_blocking=True)
+                b.record()
+                torch.cuda.synchronize()
+                best = max(best, buf_h.numel() / (a.elapsed_time(b) * 1e-3) / 1e9)
+            link[nm] = best
+        del buf_h, buf_d
+
         # ---- end to end: host buffers in, results out, copies inside the timed region ----
         e2e = None
         if not args.no_e2e:
@@ -438,7 +466,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         achieved = fwd_bytes / (fwd_us * 1e-6) / 1e9 if fwd_us > 0 else 0.0
         roofline = {"kernel": "k_embbag_fwd (popular micro-batch)", "bound": "hbm", "achieved": achieved,
                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                    "traffic": NCU_TRAFFIC_BYTES.get(wl.name), "algorithmic_bytes_per_launch": fwd_bytes,
+                    "traffic": (NCU_FWD_TRAFFIC_BYTES_PER_BAG[D] * bags_pop if D in NCU_FWD_TRAFFIC_BYTES_PER_BAG else None),
+                    "traffic_source": "ncu capture of the hot-only micro case, scaled by bags", "algorithmic_bytes_per_launch": fwd_bytes,
                     "us_per_launch": fwd_us}
         link_us = mean_us("gather_cold")
         line = {
@@ -456,8 +485,18 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                        "replicas": "independent replica per GPU, no collective"},
             "clocks": clock_info, "gpu_launches": int(launches),
             "launches_per_step": launches / args.steps, "breakdown_us": breakdown, "roofline": roofline,
-            "cold_gather": {"rows_per_step": mean("n_cold"), "bytes_per_step": mean("n_cold") * D * 4,
-                            "call_us": link_us},
+            "host_link": {
+                "memcpy_h2d_gbs": link["h2d"], "memcpy_d2h_gbs": link["d2h"],
+                "cold_rows_per_step": mean("n_cold"), "bytes_per_step": mean("n_cold") * D * 4,
+                "gather_call_us": link_us,
+                "gather_move_kernel_us": 1e3 * statistics.mean(t for t, _ in kt["gather_move"]),
+                "gather_move_gbs": statistics.mean(n * D * 4 / (t * 1e-3) / 1e9 for t, n in kt["gather_move"] if t > 0),
+                "scatter_move_kernel_us": 1e3 * statistics.mean(t for t, _ in kt["scatter_move"]),
+                "scatter_move_gbs": statistics.mean(n * D * 4 / (t * 1e-3) / 1e9 for t, n in kt["scatter_move"] if t > 0),
+                "note": "fresh random rows of the host table every step; see `--micro gather` for the same kernel "
+                        "on rows whose address translations are resident"},
+            "kernels_us": {"bwd_reduce_non": 1e3 * statistics.mean(t for t, _ in kt["bwd_reduce_non"]),
+                           "fwd_non": 1e3 * statistics.mean(t for t, _ in kt["fwd_non"])},
         }
         if e2e:
             line["e2e"] = {"value": B * world * args.steps / (e2e["ms_total"] * 1e-3), "unit": UNIT,
@@ -483,6 +522,54 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
 # ----------------------------------------------------------------------------------------------------------
 # single-call micro runs (the small cases the ncu captures under profiles/ are taken on)
 # ----------------------------------------------------------------------------------------------------------
+def run_micro_gather(args) -> None:
+    """`--micro gather`: the row-move kernel alone, host table -> HBM, 65,536 rows of 256 bytes from a 16 GiB
+    pinned table: consecutive rows, random rows within the first 4 GiB, random rows over the whole table; each
+    pattern is gathered three times (the later repetitions find their address translations resident)."""
+    import torch
+    import paper_2204_05436_b200 as hl
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    N, D, K = 1 << 26, 64, 1 << 16
+    table = hl.host_table_tensor(N, D)
+    h = hl.Hotline([N], D, 1, 64, 64, K, 16, table)
+    rng = np.random.default_rng(0)
+    cases = {"consecutive": np.arange(K), "random_4GiB": np.sort(rng.choice(1 << 24, K, replace=False)),
+             "random_16GiB": np.sort(rng.choice(N, K, replace=False))}
+    buf_h = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
+    buf_d = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    best = 0.0
+    for _ in range(5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        buf_d.copy_(buf_h, non_blocking=True)
+        b.record()
+        torch.cuda.synchronize()
+        best = max(best, buf_h.numel() / (a.elapsed_time(b) * 1e-3) / 1e9)
+    res = {"micro": "gather", "rows": K, "row_bytes": 4 * D, "table_gib": N * D * 4 / 2 ** 30, "memcpy_h2d_gbs": best}
+
+    def timed(load):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(h.main)
+        h.build_remap(load_rows=load)
+        b.record(h.main)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+
+    with torch.cuda.stream(h.main):
+        for name, rows in cases.items():
+            h.set_hot_rows(torch.from_numpy(rows).to(dev))
+            torch.cuda.synchronize()
+            base = min(timed(False) for _ in range(3))          # remap kernels without the row load
+            runs = [timed(True) - base for _ in range(3)]
+            res[name] = {"first_gbs": K * D * 4 / runs[0] / 1e6, "best_gbs": K * D * 4 / min(runs) / 1e6,
+                         "best_frac_of_memcpy": K * D * 4 / min(runs) / 1e6 / best}
+    h.status()
+    h.close()
+    print(json.dumps(res), flush=True)
+    hl.hl_host_free(table.data_ptr())
+
+
 def run_micro(args) -> None:
     """`--micro fwd|bwd`: one library call in isolation on an all-popular ("hot-only") micro-batch with the
     DLRM-large-like shape (26 tables x `--micro-batch` inputs, dim 64, one lookup per bag) over a 1 GiB cache.
@@ -547,7 +634,7 @@ def run_micro(args) -> None:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="auto", choices=["auto"] + sorted(gen.CONFIGS))
@@ -555,11 +642,15 @@ def main() -> None:
     ap.add_argument("--threads", type=int, default=min(16, os.cpu_count() or 1))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--micro", default=None, choices=["fwd", "bwd"], help="time one library call in isolation")
+    ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather"],
+                    help="time one library call in isolation")
     ap.add_argument("--micro-dist", default="uniform", choices=["uniform", "zipf"])
     ap.add_argument("--micro-batch", type=int, default=16384)
     ap.add_argument("--micro-dim", type=int, default=64)
     args = ap.parse_args()
+    if args.micro == "gather":
+        run_micro_gather(args)
+        return
     if args.micro:
         run_micro(args)
         return

@@ -114,6 +114,19 @@ HL_API int32_t hl_status(hl_ctx* ctx);
 
 HL_API const char* hl_strerror(int32_t status);
 
+/* Optional kernel timers, off by default.  When enabled, the library records a CUDA event pair on the call's
+ * stream around: the row-move kernel of hl_gather_cold (HL_TIMER_GATHER_MOVE) and of hl_scatter_cold
+ * (HL_TIMER_SCATTER_MOVE), the segment-reduce + update kernel of hl_embbag_bwd_sgd (HL_TIMER_BWD_REDUCE), the
+ * kernel of hl_embbag_fwd (HL_TIMER_FWD).  hl_timing_read gives the milliseconds of the LAST recorded pair; the
+ * caller synchronises first (HL_EINVAL if the pair was never recorded or has not finished). */
+#define HL_TIMER_GATHER_MOVE  0
+#define HL_TIMER_SCATTER_MOVE 1
+#define HL_TIMER_BWD_REDUCE   2
+#define HL_TIMER_FWD          3
+#define HL_TIMER_COUNT        4
+HL_API int32_t hl_timing_enable(hl_ctx* ctx, int32_t on);
+HL_API int32_t hl_timing_read(hl_ctx* ctx, int32_t which, float* ms);
+
 /* Pinned, device-mapped host memory for the host-DRAM table (exactly `bytes`, no rounding): the device reads
  * and writes it over the host link at the same address.  The caller owns it and frees it with hl_host_free.
  * Returns NULL on failure. */

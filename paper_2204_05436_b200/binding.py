@@ -16,7 +16,7 @@ HL_OK, HL_EINVAL, HL_EBOUNDS, HL_ECAPACITY, HL_ECUDA, HL_ETIMEOUT = 0, -1, -2, -
 HL_HOT_TOPK_ROWS, HL_HOT_BUDGET_BYTES, HL_HOT_FRACTION_ROWS, HL_HOT_MIN_SHARE = 0, 1, 2, 3
 
 EXPORTS = (
-    "hl_workspace_bytes", "hl_create", "hl_destroy", "hl_status", "hl_strerror", "hl_launch_count", "hl_host_alloc",
+    "hl_workspace_bytes", "hl_create", "hl_destroy", "hl_status", "hl_strerror", "hl_launch_count", "hl_timing_enable", "hl_timing_read", "hl_host_alloc",
     "hl_host_free", "hl_profile_hot",
     "hl_build_remap", "hl_fragment", "hl_embbag_fwd", "hl_embbag_bwd_sgd", "hl_gather_cold", "hl_scatter_cold",
     "hl_embbag_bwd_sgd_static",
@@ -63,6 +63,10 @@ def _load() -> ctypes.CDLL:
     lib.hl_strerror.argtypes = [i32]
     lib.hl_launch_count.restype = ctypes.c_uint64
     lib.hl_launch_count.argtypes = []
+    lib.hl_timing_enable.restype = i32
+    lib.hl_timing_enable.argtypes = [vp, i32]
+    lib.hl_timing_read.restype = i32
+    lib.hl_timing_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_float)]
     lib.hl_host_alloc.restype = vp
     lib.hl_host_alloc.argtypes = [ctypes.c_size_t]
     lib.hl_host_free.restype = i32
@@ -114,6 +118,20 @@ def strerror(status: int) -> str:
 
 def hl_launch_count() -> int:
     return int(_lib.hl_launch_count())
+
+
+HL_TIMER_GATHER_MOVE, HL_TIMER_SCATTER_MOVE, HL_TIMER_BWD_REDUCE, HL_TIMER_FWD = 0, 1, 2, 3
+
+
+def hl_timing_enable(ctx: int, on: bool) -> None:
+    _check("hl_timing_enable", _lib.hl_timing_enable(ctx, int(on)))
+
+
+def hl_timing_read(ctx: int, which: int) -> float:
+    """Milliseconds of the last recorded event pair of timer ``which`` (synchronise first)."""
+    ms = ctypes.c_float()
+    _check("hl_timing_read", _lib.hl_timing_read(ctx, which, ctypes.byref(ms)))
+    return float(ms.value)
 
 
 def hl_host_alloc(nbytes: int) -> int:

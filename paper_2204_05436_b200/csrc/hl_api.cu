@@ -144,8 +144,30 @@ extern "C" int32_t hl_create(hl_ctx** out, const hl_geometry* geom, int32_t max_
     return HL_OK;
 }
 
+extern "C" int32_t hl_timing_enable(hl_ctx* ctx, int32_t on) {
+    if (!ctx) return HL_EINVAL;
+    if (on && !ctx->timer[0][0]) {
+        for (int w = 0; w < HL_TIMER_COUNT; ++w)
+            for (int e = 0; e < 2; ++e) HL_CUDA_TRY(cudaEventCreate(&ctx->timer[w][e]));
+    }
+    ctx->timing_on = on ? 1 : 0;
+    return HL_OK;
+}
+
+extern "C" int32_t hl_timing_read(hl_ctx* ctx, int32_t which, float* ms) {
+    if (!ctx || !ms || which < 0 || which >= HL_TIMER_COUNT || !ctx->timer[which][0]) return HL_EINVAL;
+    if (cudaEventElapsedTime(ms, ctx->timer[which][0], ctx->timer[which][1]) != cudaSuccess) {
+        cudaGetLastError();
+        return HL_EINVAL;   // never recorded, or not finished yet
+    }
+    return HL_OK;
+}
+
 extern "C" int32_t hl_destroy(hl_ctx* ctx) {
     if (!ctx) return HL_EINVAL;
+    for (int w = 0; w < HL_TIMER_COUNT; ++w)
+        for (int e = 0; e < 2; ++e)
+            if (ctx->timer[w][e]) cudaEventDestroy(ctx->timer[w][e]);
     free(ctx->h_table_base);
     free(ctx);
     return HL_OK;

@@ -211,14 +211,20 @@ extern "C" int32_t hl_gather_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_
                                                  ctx->staging_cap, non->ids, d_cold_rows, d_n_cold, r.status);
     note_launches(1);
     HL_LAUNCH_CHECK();
-    return launch_move_rows<false>(d_cache, ctx->hot_cap, const_cast<float*>(host_table), d_cold_rows, d_n_cold,
-                                   ctx->staging_cap, ctx->N, ctx->D, r.status, stream);
+    timer_mark(ctx, HL_TIMER_GATHER_MOVE, 0, stream);
+    st = launch_move_rows<false>(d_cache, ctx->hot_cap, const_cast<float*>(host_table), d_cold_rows, d_n_cold,
+                                 ctx->staging_cap, ctx->N, ctx->D, r.status, stream);
+    timer_mark(ctx, HL_TIMER_GATHER_MOVE, 1, stream);
+    return st;
 }
 
 extern "C" int32_t hl_scatter_cold(hl_ctx* ctx, const float* d_cache, const int32_t* d_cold_rows,
                                    const int64_t* d_n_cold, float* host_table, void* stream_) {
     if (!ctx || !d_cache || !d_cold_rows || !d_n_cold || !host_table) return HL_EINVAL;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    return launch_move_rows<true>(const_cast<float*>(d_cache), ctx->hot_cap, host_table, d_cold_rows, d_n_cold,
-                                  ctx->staging_cap, ctx->N, ctx->D, ctx->r.status, stream);
+    timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 0, stream);
+    const int32_t st = launch_move_rows<true>(const_cast<float*>(d_cache), ctx->hot_cap, host_table, d_cold_rows,
+                                              d_n_cold, ctx->staging_cap, ctx->N, ctx->D, ctx->r.status, stream);
+    timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 1, stream);
+    return st;
 }

@@ -75,6 +75,8 @@ struct hl_ctx {
     int device;
     int64_t* h_table_base;             // host copy [T+1]
     hl::Regions r;
+    int timing_on;                     // optional kernel timers (hl_timing_enable)
+    cudaEvent_t timer[HL_TIMER_COUNT][2];
 };
 
 namespace hl {
@@ -89,6 +91,11 @@ namespace hl {
     do {                                                   \
         if (cudaGetLastError() != cudaSuccess) return HL_ECUDA; \
     } while (0)
+
+// Records the start/end event of one of the optional kernel timers on `stream` (no-op unless enabled).
+inline void timer_mark(hl_ctx* ctx, int which, int end, cudaStream_t stream) {
+    if (ctx->timing_on && ctx->timer[which][end]) cudaEventRecord(ctx->timer[which][end], stream);
+}
 
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) {
     atomicCAS(status, 0, code);

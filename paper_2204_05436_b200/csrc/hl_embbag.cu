@@ -382,9 +382,11 @@ int32_t launch_fwd(hl_ctx* ctx, const float* cache, const hl_ubatch* ub, const i
     }
     const int64_t max_bags = ctx->max_bags;
     const int grid = grid_for(div_up(max_bags, UB) * G, kThreads, kSMs * ctas_per_sm);
+    timer_mark(ctx, HL_TIMER_FWD, 0, stream);
     k_embbag_fwd<G, NV, UB><<<grid, kThreads, 0, stream>>>(cache, ub->ids, ub->offsets, d_n, ctx->max_batch,
                                                           ctx->T * ctx->S, ctx->D / 4,
                                                           ctx->hot_cap + ctx->staging_cap, out, ctx->r.status);
+    timer_mark(ctx, HL_TIMER_FWD, 1, stream);
     note_launches(1);
     HL_LAUNCH_CHECK();
     return HL_OK;
@@ -396,8 +398,10 @@ int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t
     const int64_t max_chunks = div_up(ctx->max_nnz, kBwdChunk);
     const int grid = grid_for(max_chunks * G, kThreads, kSMs * 8);
     const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
+    timer_mark(ctx, HL_TIMER_BWD_REDUCE, 0, stream);
     k_bwd_chunks<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, vals, ctx->r.bwd_n, grad, ctx->D / 4, n_slots,
                                                       lr, ctx->r.bwd_part);
+    timer_mark(ctx, HL_TIMER_BWD_REDUCE, 1, stream);
     k_bwd_spans<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, ctx->r.bwd_n, ctx->D / 4, n_slots, lr,
                                                      ctx->r.bwd_part);
     note_launches(2);
