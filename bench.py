@@ -298,8 +298,13 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
     n_batches = 8
     wl = Workload(name, scale, n_batches, args.profile_batches, device, args.threads)
     T, D, S, B = wl.T, wl.D, wl.S, wl.B
-    h = hl.Hotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
-                   n_dense=wl.spec.n_dense, device=str(device))
+    pipelined = args.pipeline
+    if pipelined:
+        h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
+                                n_dense=wl.spec.n_dense, device=str(device))
+    else:
+        h = hl.Hotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
+                       n_dense=wl.spec.n_dense, device=str(device))
     lr = wl.spec.lr
 
     with torch.cuda.stream(h.main):
@@ -328,21 +333,42 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         h_grad = d_grad.cpu().pin_memory()
         torch.cuda.synchronize()
 
-        def one_step(i, timers=None):
+        cursor = [0]   # mini-batches issued so far; mini-batch i uses input buffers i % n_batches
+
+        def batch_args(k):
+            return (d_idx[k], d_off[k], B, d_dense[k])
+
+        def one_step(timers=None):
+            """Issues the next mini-batch; returns (its buffer index k, the object holding its outputs)."""
+            i = cursor[0]
+            cursor[0] += 1
             k = i % n_batches
+            if pipelined:
+                if h.j_submitted == h.j_done:
+                    h.start(*batch_args(k))
+                s = h.step(d_grad, d_grad, lr, next_batch=batch_args((i + 1) % n_batches), timers=timers)
+                return k, h.sets[s]
             h.step(d_idx[k], d_off[k], B, d_grad, d_grad, lr, dense=d_dense[k], timers=timers)
+            return k, h
+
+        def finish():
+            """Everything issued so far is complete, write-backs included."""
+            if pipelined:
+                h.drain()
+            torch.cuda.synchronize()
 
         # per-batch sizes (they depend only on the indices and the hot set): one untimed pass
-        sizes = []
-        for k in range(n_batches):
-            one_step(k)
+        sizes = [None] * n_batches
+        for _ in range(n_batches):
+            k, o = one_step()
+            finish()
             h.status()
-            c = h.counts.cpu().tolist()
-            sizes.append(dict(n_pop=c[0], n_non=c[1], L_pop=c[2], L_non=c[3], n_cold=int(h.n_cold.item())))
+            c = o.counts.cpu().tolist()
+            sizes[k] = dict(n_pop=c[0], n_non=c[1], L_pop=c[2], L_non=c[3], n_cold=int(o.n_cold.item()))
 
         # ---- timed region: device-resident inputs ----
         for i in range(args.warmup):
-            one_step(i)
+            one_step()
         torch.cuda.synchronize()
         if world > 1:
             dist.barrier()
@@ -352,11 +378,14 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         clocks.start()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
+        first_timed = cursor[0]
         ev0.record(h.main)
         for i in range(args.steps):
-            one_step(args.warmup + i, timers)
+            one_step(timers)
+        if pipelined:
+            h.main.wait_stream(h.wb)     # the last write-backs belong to the timed work
         ev1.record(h.main)
-        torch.cuda.synchronize()
+        finish()
         if world > 1:
             dist.barrier()
         clock_info = clocks.stop()
@@ -367,9 +396,9 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         # ---- kernel timers and host link (diagnostic pass, outside the timed region) ----
         hl.hl_timing_enable(h.ctx, True)
         kt = {"gather_move": [], "scatter_move": [], "bwd_reduce_non": [], "fwd_non": []}
-        for k in range(n_batches):
-            one_step(k)
-            torch.cuda.synchronize()
+        for _ in range(n_batches):
+            k, _o = one_step()
+            finish()
             kt["gather_move"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_GATHER_MOVE), sizes[k]["n_cold"]))
             kt["scatter_move"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_SCATTER_MOVE), sizes[k]["n_cold"]))
             kt["bwd_reduce_non"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_BWD_REDUCE), sizes[k]["L_non"]))
@@ -400,8 +429,10 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             h2d = d2h = 0
 
             def e2e_step(i):
+                # the inputs copied here are those of the mini-batch whose ahead-work this step issues (pipelined)
+                # or of this step's own mini-batch (sequential); the gradients are this step's
                 nonlocal h2d, d2h
-                k = i % n_batches
+                k = ((cursor[0] + 1) if pipelined else cursor[0]) % n_batches
                 d_idx[k].copy_(h_idx[k], non_blocking=True)
                 d_off[k].copy_(h_off[k], non_blocking=True)
                 h2d_now = h_idx[k].numel() * 4 + h_off[k].numel() * 4 + h_grad.numel() * 4
@@ -409,13 +440,13 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                     d_dense[k].copy_(h_dense[k], non_blocking=True)
                     h2d_now += h_dense[k].numel() * 4
                 d_grad.copy_(h_grad, non_blocking=True)
-                h.step(d_idx[k], d_off[k], B, d_grad, d_grad, lr, dense=d_dense[k])
-                out_counts.copy_(h.counts, non_blocking=True)
-                out_perm.copy_(h.perm[:B], non_blocking=True)
+                _k, o = one_step()
+                out_counts.copy_(o.counts, non_blocking=True)
+                out_perm.copy_(o.perm[:B], non_blocking=True)
                 h.main.synchronize()
                 bags_pop, bags_non = T * int(out_counts[0]) * S, T * int(out_counts[1]) * S
-                out_pop[:bags_pop].copy_(h.pooled_pop[:bags_pop], non_blocking=True)
-                out_non[:bags_non].copy_(h.pooled_non[:bags_non], non_blocking=True)
+                out_pop[:bags_pop].copy_(o.pooled_pop[:bags_pop], non_blocking=True)
+                out_non[:bags_non].copy_(o.pooled_non[:bags_non], non_blocking=True)
                 h.main.synchronize()
                 h2d, d2h = h2d_now, 16 + B * 4 + (bags_pop + bags_non) * D * 4
 
@@ -425,11 +456,14 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             if world > 1:
                 dist.barrier()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            finish()
             e0.record(h.main)
             for i in range(args.steps):
                 e2e_step(args.warmup + i)
+            if pipelined:
+                h.main.wait_stream(h.wb)
             e1.record(h.main)
-            torch.cuda.synchronize()
+            finish()
             e2e_ms = e0.elapsed_time(e1)
             e2e = {"ms_total": e2e_ms, "h2d": h2d, "d2h": d2h}
         h.status()
@@ -451,7 +485,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             return 1e3 * sum(a.elapsed_time(b) for a, b in ev) / max(1, len(ev))
 
         breakdown = {k: round(mean_us(k), 2) for k in timers}
-        used = [sizes[(args.warmup + i) % n_batches] for i in range(args.steps)]
+        used = [sizes[(first_timed + i) % n_batches] for i in range(args.steps)]
         mean = lambda key: sum(u[key] for u in used) / len(used)   # noqa: E731
         # roofline of the popular micro-batch's embedding-bag forward (one kernel per call): per lookup a row
         # (4*D bytes) and its slot (4 bytes) are read, per bag a pooled row (4*D) is written and an offset read.
@@ -482,6 +516,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                              f"({(2 * wl.n_bags * D * 4 + fwd_bytes) / 2**20:.0f} MB of pooled vectors, gradients and rows)"
                              if 2 * wl.n_bags * D * 4 > L2_BYTES else
                              "per-step working set is smaller than L2 on this workload; batches rotate over 8 buffers",
+                       "schedule": ("software-pipelined across mini-batches (PipelinedHotline)" if pipelined else
+                                    "one mini-batch after the other (Hotline.step)"),
                        "replicas": "independent replica per GPU, no collective"},
             "clocks": clock_info, "gpu_launches": int(launches),
             "launches_per_step": launches / args.steps, "breakdown_us": breakdown, "roofline": roofline,
@@ -641,6 +677,10 @@ def main() -> None:
     ap.add_argument("--profile-batches", type=int, default=None)
     ap.add_argument("--threads", type=int, default=min(16, os.cpu_count() or 1))
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--pipeline", action="store_true",
+                    help="software-pipeline the mini-batches (PipelinedHotline) instead of running one after the "
+                         "other (Hotline.step); kernels of different mini-batches then overlap, so the per-call "
+                         "times no longer describe a kernel running alone")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather"],
                     help="time one library call in isolation")

@@ -206,6 +206,38 @@ HL_API int32_t hl_gather_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_no
 HL_API int32_t hl_scatter_cold(hl_ctx* ctx, const float* d_cache, const int32_t* d_cold_rows,
                         const int64_t* d_n_cold, float* host_table, void* stream);
 
+/* ---------------------------------------------------------------------------------------------------------
+ * Software pipelining across mini-batches (Section IV: the gathering of the working parameters is pipelined with
+ * the execution on the GPU so that the GPU never stalls).  While mini-batch j-1 is still executing, mini-batch j
+ * can already be fragmented and its cold rows staged, provided that a cold row which j shares with j-1 is NOT
+ * read from the host (its update by j-1 has not been written back yet) but copied from j-1's staging area once
+ * j-1's backward has run.  The staging part of the cache is used as several windows (stage_row0, stage_rows):
+ * a row of rank r is staged at cache slot hot_cap_rows + stage_row0 + r.
+ * ------------------------------------------------------------------------------------------------------- */
+
+/* hl_gather_cold into the window [stage_row0, stage_row0 + stage_rows) of the staging area, with exclusion:
+ * d_prev_cold_rows[0 .. *d_n_prev) (ascending; may be NULL) is the cold set of the mini-batch still in flight.
+ * d_fwd_src[i] (out, [stage_rows]) = position of d_cold_rows[i] in that set, or -1; rows with d_fwd_src[i] >= 0
+ * are not read from the host (hl_forward_cold fills them in later).
+ * Optional CUDA events (cudaEvent_t as void*, may be NULL): record_after_index is recorded on the stream once
+ * d_cold_rows, *d_n_cold, d_fwd_src and the unified slots in non->ids are final; the stream waits for
+ * wait_before_move_a / _b right before the host rows are read (e.g. the write-back of an earlier mini-batch). */
+HL_API int32_t hl_gather_cold_ahead(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const float* host_table,
+                                    float* d_cache, int64_t stage_row0, int64_t stage_rows, int32_t* d_cold_rows,
+                                    int64_t* d_n_cold, const int32_t* d_prev_cold_rows, const int64_t* d_n_prev,
+                                    int32_t* d_fwd_src, void* record_after_index, void* wait_before_move_a,
+                                    void* wait_before_move_b, void* stream);
+
+/* cache[hot_cap + to_stage_row0 + i, :] = cache[hot_cap + from_stage_row0 + d_fwd_src[i], :] for every
+ * i < *d_n_cold with d_fwd_src[i] >= 0 (device-to-device; run it after the earlier mini-batch's backward). */
+HL_API int32_t hl_forward_cold(hl_ctx* ctx, float* d_cache, int64_t from_stage_row0, int64_t to_stage_row0,
+                               int64_t stage_rows, const int32_t* d_fwd_src, const int64_t* d_n_cold, void* stream);
+
+/* hl_scatter_cold from the window [stage_row0, stage_row0 + stage_rows) of the staging area. */
+HL_API int32_t hl_scatter_cold_at(hl_ctx* ctx, const float* d_cache, int64_t stage_row0, int64_t stage_rows,
+                                  const int32_t* d_cold_rows, const int64_t* d_n_cold, float* host_table,
+                                  void* stream);
+
 /* No counterpart in the paper: an addition for callers that cannot allocate.
  *
  * Some callers have no way to hand the library a workspace: code that runs where device allocation is forbidden

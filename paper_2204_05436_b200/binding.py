@@ -19,7 +19,7 @@ EXPORTS = (
     "hl_workspace_bytes", "hl_create", "hl_destroy", "hl_status", "hl_strerror", "hl_launch_count", "hl_timing_enable", "hl_timing_read", "hl_host_alloc",
     "hl_host_free", "hl_profile_hot",
     "hl_build_remap", "hl_fragment", "hl_embbag_fwd", "hl_embbag_bwd_sgd", "hl_gather_cold", "hl_scatter_cold",
-    "hl_embbag_bwd_sgd_static",
+    "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at",
 )
 
 
@@ -86,6 +86,13 @@ def _load() -> ctypes.CDLL:
     lib.hl_gather_cold.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, vp, vp, vp, vp, vp]
     lib.hl_scatter_cold.restype = i32
     lib.hl_scatter_cold.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.hl_gather_cold_ahead.restype = i32
+    lib.hl_gather_cold_ahead.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp,
+                                         vp]
+    lib.hl_forward_cold.restype = i32
+    lib.hl_forward_cold.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
+    lib.hl_scatter_cold_at.restype = i32
+    lib.hl_scatter_cold_at.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
     lib.hl_embbag_bwd_sgd_static.restype = i32
     lib.hl_embbag_bwd_sgd_static.argtypes = [vp, i64, i32, vp, vp, i32, i64, vp, ctypes.c_float, vp, vp]
     return lib
@@ -248,3 +255,33 @@ def hl_embbag_bwd_sgd_static(d_cache, cache_rows: int, dim: int, d_offsets, d_id
     _check("hl_embbag_bwd_sgd_static", _lib.hl_embbag_bwd_sgd_static(
         _ptr(d_cache), int(cache_rows), int(dim), _ptr(d_offsets), _ptr(d_ids), int(n_bags), int(nnz),
         _ptr(d_grad_out), float(lr), _ptr(d_status), stream))
+
+
+def _ev(e):
+    """A torch.cuda.Event (already recorded or created with its handle), a raw cudaEvent_t as int, or None."""
+    if e is None:
+        return None
+    if isinstance(e, int):
+        return e
+    return int(e.cuda_event)
+
+
+def hl_gather_cold_ahead(ctx: int, non: hl_ubatch, d_n_non, host_table, d_cache, stage_row0: int, stage_rows: int,
+                         d_cold_rows, d_n_cold, d_prev_cold_rows, d_n_prev, d_fwd_src, record_after_index,
+                         wait_before_move_a, wait_before_move_b, stream: int) -> None:
+    _check("hl_gather_cold_ahead", _lib.hl_gather_cold_ahead(
+        ctx, ctypes.byref(non), _ptr(d_n_non), _ptr(host_table), _ptr(d_cache), int(stage_row0), int(stage_rows),
+        _ptr(d_cold_rows), _ptr(d_n_cold), _ptr(d_prev_cold_rows), _ptr(d_n_prev), _ptr(d_fwd_src),
+        _ev(record_after_index), _ev(wait_before_move_a), _ev(wait_before_move_b), stream))
+
+
+def hl_forward_cold(ctx: int, d_cache, from_stage_row0: int, to_stage_row0: int, stage_rows: int, d_fwd_src, d_n_cold,
+                    stream: int) -> None:
+    _check("hl_forward_cold", _lib.hl_forward_cold(ctx, _ptr(d_cache), int(from_stage_row0), int(to_stage_row0),
+                                                   int(stage_rows), _ptr(d_fwd_src), _ptr(d_n_cold), stream))
+
+
+def hl_scatter_cold_at(ctx: int, d_cache, stage_row0: int, stage_rows: int, d_cold_rows, d_n_cold, host_table,
+                       stream: int) -> None:
+    _check("hl_scatter_cold_at", _lib.hl_scatter_cold_at(ctx, _ptr(d_cache), int(stage_row0), int(stage_rows),
+                                                         _ptr(d_cold_rows), _ptr(d_n_cold), _ptr(host_table), stream))

@@ -65,11 +65,11 @@ __global__ void __launch_bounds__(kThreads) k_cold_heads(const int32_t* __restri
 }
 
 // rank_excl[i] = number of run heads before i; the row at i has rank rank_excl[i] if it is a head, else
-// rank_excl[i] - 1.
+// rank_excl[i] - 1.  A row of rank r is staged at cache slot slot0 + r (slot0 = start of the staging window).
 __global__ void __launch_bounds__(kThreads) k_cold_assign(const int32_t* __restrict__ keys,
                                                           const int32_t* __restrict__ vals,
                                                           const int32_t* __restrict__ d_n, int64_t n_max,
-                                                          const int32_t* __restrict__ rank_excl, int64_t hot_cap,
+                                                          const int32_t* __restrict__ rank_excl, int64_t slot0,
                                                           int64_t staging_cap, int32_t* __restrict__ ids,
                                                           int32_t* __restrict__ cold_rows,
                                                           int64_t* __restrict__ d_n_cold, int32_t* status) {
@@ -88,20 +88,22 @@ __global__ void __launch_bounds__(kThreads) k_cold_assign(const int32_t* __restr
         const int64_t rank = head ? rank_excl[i] : rank_excl[i] - 1;
         if (rank < staging_cap) {
             if (head) cold_rows[rank] = keys[i];
-            ids[vals[i]] = (int32_t)(hot_cap + rank);
+            ids[vals[i]] = (int32_t)(slot0 + rank);
         } else {
             ids[vals[i]] = -1;   // no room to stage this row: the lookup is dropped and the status word says so
         }
     }
 }
 
-// dst[(dst_row0 + i), :] = table[rows[i], :]; G lanes per row, UR rows in flight per group.
+// dst[(dst_row0 + i), :] = table[rows[i], :] (or the other way round); G lanes per row, UR rows in flight per
+// group.  Rows i with skip[i] >= 0 are left alone.
 template <int G, bool TO_TABLE>
 __global__ void __launch_bounds__(kThreads) k_move_rows(float* __restrict__ dense_side, int64_t dense_row0,
                                                         float* __restrict__ table, const int32_t* __restrict__ rows,
                                                         const int64_t* __restrict__ d_n, int64_t n_max,
-                                                        int64_t table_rows, int D4, int32_t* status) {
-    constexpr int UR = 4;
+                                                        int64_t table_rows, int D4,
+                                                        const int32_t* __restrict__ skip, int32_t* status) {
+    constexpr int UR = 16;
     int64_t n = *d_n;
     n = n < 0 ? 0 : (n < n_max ? n : n_max);
     const int sub = threadIdx.x % G;
@@ -114,6 +116,7 @@ __global__ void __launch_bounds__(kThreads) k_move_rows(float* __restrict__ dens
 #pragma unroll
         for (int u = 0; u < UR; ++u) {
             g[u] = i0 + u < n ? (int64_t)rows[i0 + u] : -1;
+            if (skip != nullptr && g[u] >= 0 && skip[i0 + u] >= 0) g[u] = -1;   // row comes from elsewhere
             if (g[u] >= table_rows) {
                 set_status(status, HL_EBOUNDS);
                 g[u] = -1;
@@ -134,28 +137,193 @@ __global__ void __launch_bounds__(kThreads) k_move_rows(float* __restrict__ dens
     }
 }
 
+// src[i] = position of rows[i] in the ascending list prev[0 .. *d_n_prev), or -1.
+__global__ void __launch_bounds__(kThreads) k_cold_match(const int32_t* __restrict__ rows,
+                                                         const int64_t* __restrict__ d_n, int64_t n_max,
+                                                         const int32_t* __restrict__ prev,
+                                                         const int64_t* __restrict__ d_n_prev, int64_t n_prev_max,
+                                                         int32_t* __restrict__ src) {
+    int64_t n = *d_n, np = *d_n_prev;
+    n = n < 0 ? 0 : (n < n_max ? n : n_max);
+    np = np < 0 ? 0 : (np < n_prev_max ? np : n_prev_max);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        const int32_t g = rows[i];
+        int64_t lo = 0, hi = np;
+        while (lo < hi) {
+            const int64_t mid = (lo + hi) >> 1;
+            if (prev[mid] < g) lo = mid + 1;
+            else hi = mid;
+        }
+        src[i] = (lo < np && prev[lo] == g) ? (int32_t)lo : -1;
+    }
+}
+
+// cache[to_row0 + i, :] = cache[from_row0 + src[i], :] for every i < *d_n with src[i] >= 0.
+template <int G>
+__global__ void __launch_bounds__(kThreads) k_forward_rows(float* cache, int64_t from_row0, int64_t to_row0,
+                                                           const int32_t* __restrict__ src,
+                                                           const int64_t* __restrict__ d_n, int64_t n_max, int D4) {
+    int64_t n = *d_n;
+    n = n < 0 ? 0 : (n < n_max ? n : n_max);
+    const int sub = threadIdx.x % G;
+    const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+    const int64_t n_groups = (int64_t)gridDim.x * kThreads / G;
+    float4* c4 = reinterpret_cast<float4*>(cache);
+    for (int64_t i = group; i < n; i += n_groups) {
+        const int32_t j = src[i];
+        if (j < 0 || j >= n_max) continue;
+        for (int c = sub; c < D4; c += G) c4[(to_row0 + i) * D4 + c] = c4[(from_row0 + j) * D4 + c];
+    }
+}
+
+// ---- row mover on the bulk-copy (TMA) engine ----------------------------------------------------------------
+// The same copy as k_move_rows, issued as asynchronous bulk copies: every row is one cp.async.bulk from its
+// source into shared memory (completion counted in bytes on an mbarrier) and one cp.async.bulk from shared memory
+// to its destination.  The rows in flight are then requests of the copy engine of the SM, not pending loads of
+// its load-store unit, so that embedding-bag CTAs of another micro-batch that share the SM keep their own
+// loads moving while hundreds of host rows, each waiting microseconds for its address translation, are pending.
+// Source, destination and row size are multiples of 16 bytes (dim % 4 == 0, 16-byte aligned bases).
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* mbar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(smem_dst)),
+                 "l"(gmem_src), "r"(bytes), "r"(smem_u32(mbar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gmem_dst),
+                 "r"(smem_u32(smem_src)), "r"(bytes)
+                 : "memory");
+}
+
+constexpr int kBulkThreads = 128;
+constexpr int kBulkStages = 2;
+constexpr int kBulkStageBytes = 16384;
+constexpr int kBulkMaxPolls = 1 << 22;
+// CTAs of the mover.  8 CTAs x 2 stages x 16 KB keep 256 KB of rows in flight: enough for the link (measured: 50 GB/s
+// on rows whose translations are resident), and the fastest setting on fresh random rows (390 us for 18 K rows,
+// against 416-460 us with 16 to 64 CTAs).  More rows in flight do not go faster -- the link is waiting for address
+// translations -- but they slow every other kernel on the chip: a forward kernel that takes 49 us alone takes
+// 60 us next to 8 mover CTAs, 100 us next to 16, and over 300 us next to 32 or more.
+constexpr int kBulkCtas = 8;   // (the hot-cache load of hl_build_remap, which runs alone, uses 2 per SM)
+
+template <bool TO_TABLE>
+__global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_side, int64_t dense_row0, float* table,
+                                                                 const int32_t* __restrict__ rows,
+                                                                 const int64_t* __restrict__ d_n, int64_t n_max,
+                                                                 int64_t table_rows, int row_bytes,
+                                                                 int rows_per_stage,
+                                                                 const int32_t* __restrict__ skip, int32_t* status) {
+    __shared__ __align__(128) unsigned char stage[kBulkStages][kBulkStageBytes];
+    __shared__ __align__(8) uint64_t mbar[kBulkStages];
+    __shared__ unsigned int stage_bytes[kBulkStages];
+    int64_t n = *d_n;
+    n = n < 0 ? 0 : (n < n_max ? n : n_max);
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        for (int s = 0; s < kBulkStages; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&mbar[s])), "r"(1) : "memory");
+            stage_bytes[s] = 0;
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    unsigned char* dense = reinterpret_cast<unsigned char*>(dense_side) + dense_row0 * row_bytes;
+    unsigned char* tab = reinterpret_cast<unsigned char*>(table);
+    const int64_t n_batches = (n + rows_per_stage - 1) / rows_per_stage;
+    int it = 0;
+    for (int64_t b = blockIdx.x; b < n_batches; b += gridDim.x, ++it) {
+        const int s = it % kBulkStages;
+        const uint32_t parity = (uint32_t)(it / kBulkStages) & 1u;
+        const int64_t i0 = b * rows_per_stage;
+        const int cnt = (int)min((int64_t)rows_per_stage, n - i0);
+        // this thread's earlier stores out of stage s have finished reading shared memory
+        asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kBulkStages - 1) : "memory");
+        __syncthreads();
+        // which of my rows move, and how many bytes the stage expects
+        unsigned int my_bytes = 0;
+        for (int r = tid; r < cnt; r += kBulkThreads) {
+            const int64_t g = rows[i0 + r];
+            const bool ok = g >= 0 && g < table_rows && !(skip != nullptr && skip[i0 + r] >= 0);
+            if (g >= table_rows) set_status(status, HL_EBOUNDS);
+            if (ok) my_bytes += (unsigned int)row_bytes;
+        }
+        if (my_bytes) atomicAdd(&stage_bytes[s], my_bytes);
+        __syncthreads();
+        if (tid == 0) {
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&mbar[s])),
+                         "r"(stage_bytes[s])
+                         : "memory");
+            stage_bytes[s] = 0;
+        }
+        for (int r = tid; r < cnt; r += kBulkThreads) {
+            const int64_t g = rows[i0 + r];
+            const bool ok = g >= 0 && g < table_rows && !(skip != nullptr && skip[i0 + r] >= 0);
+            if (!ok) continue;
+            const unsigned char* src = TO_TABLE ? dense + (i0 + r) * row_bytes : tab + g * row_bytes;
+            bulk_load(&stage[s][r * row_bytes], src, (uint32_t)row_bytes, &mbar[s]);
+        }
+        // wait for the stage to fill (bounded)
+        uint32_t done = 0;
+        for (int polls = 0; !done; ++polls) {
+            asm volatile(
+                "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(done)
+                : "r"(smem_u32(&mbar[s])), "r"(parity)
+                : "memory");
+            if (!done && polls > kBulkMaxPolls) {
+                set_status(status, HL_ETIMEOUT);
+                break;
+            }
+        }
+        for (int r = tid; r < cnt; r += kBulkThreads) {
+            const int64_t g = rows[i0 + r];
+            const bool ok = done && g >= 0 && g < table_rows && !(skip != nullptr && skip[i0 + r] >= 0);
+            if (!ok) continue;   // (a stage whose wait gave up is not written; the status word says so)
+            unsigned char* dst = TO_TABLE ? tab + g * row_bytes : dense + (i0 + r) * row_bytes;
+            bulk_store(dst, &stage[s][r * row_bytes], (uint32_t)row_bytes);
+        }
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
 template <bool TO_TABLE>
 int32_t launch_move_rows(float* dense_side, int64_t dense_row0, float* table, const int32_t* rows,
-                         const int64_t* d_n, int64_t n_max, int64_t table_rows, int D, int32_t* status,
-                         cudaStream_t stream) {
+                         const int64_t* d_n, int64_t n_max, int64_t table_rows, int D, const int32_t* skip,
+                         int bulk_ctas, int32_t* status, cudaStream_t stream) {
     if (n_max <= 0) return HL_OK;
     const int D4 = D / 4;
-    // Two light CTAs per SM: random rows of a table of tens of GB miss the address translation of the host
-    // link on almost every row, and the link only reaches its rate with many such misses in flight at once
-    // (measured: 32 CTAs 19 GB/s, 296 and more 24 GB/s on random rows; 50 GB/s on rows within 4 GB either way).
-    const int grid = 2 * kSMs;
+    const int row_bytes = D * 4;
+    if (row_bytes <= kBulkStageBytes) {
+        const int rows_per_stage = kBulkStageBytes / row_bytes;
+        const int grid = grid_for(n_max, rows_per_stage, bulk_ctas);
+        k_move_rows_bulk<TO_TABLE><<<grid, kBulkThreads, 0, stream>>>(dense_side, dense_row0, table, rows, d_n, n_max,
+                                                                     table_rows, row_bytes, rows_per_stage, skip,
+                                                                     status);
+        note_launches(1);
+        HL_LAUNCH_CHECK();
+        return HL_OK;
+    }
+    // Few CTAs with many rows in flight each.  Random rows of a table of tens of GB miss the address translation
+    // of the host link on almost every row, so the link needs about a megabyte in flight to reach its rate; but
+    // this kernel runs next to the embedding-bag kernels of another micro-batch, whose grids are sized to fill the
+    // chip: every SM it sits on takes CTA slots and load-store queue entries away from them for hundreds of
+    // microseconds.  48 CTAs x 16 groups x 16 rows keeps 12 K rows in flight on a third of the SMs.
+    const int grid = 48;
     if (D4 <= 4)
         k_move_rows<4, TO_TABLE><<<grid, kThreads, 0, stream>>>(dense_side, dense_row0, table, rows, d_n, n_max,
-                                                               table_rows, D4, status);
+                                                               table_rows, D4, skip, status);
     else if (D4 <= 8)
         k_move_rows<8, TO_TABLE><<<grid, kThreads, 0, stream>>>(dense_side, dense_row0, table, rows, d_n, n_max,
-                                                               table_rows, D4, status);
+                                                               table_rows, D4, skip, status);
     else if (D4 <= 16)
         k_move_rows<16, TO_TABLE><<<grid, kThreads, 0, stream>>>(dense_side, dense_row0, table, rows, d_n, n_max,
-                                                                table_rows, D4, status);
+                                                                table_rows, D4, skip, status);
     else
         k_move_rows<32, TO_TABLE><<<grid, kThreads, 0, stream>>>(dense_side, dense_row0, table, rows, d_n, n_max,
-                                                                table_rows, D4, status);
+                                                                table_rows, D4, skip, status);
     note_launches(1);
     HL_LAUNCH_CHECK();
     return HL_OK;
@@ -172,27 +340,33 @@ int bits_for(int64_t max_value) {
 int32_t launch_gather_rows(float* dst, int64_t dst_row0, const float* table, const int32_t* rows,
                            const int64_t* d_n, int64_t n_max, int64_t table_rows, int D, int32_t* status,
                            cudaStream_t stream) {
-    return launch_move_rows<false>(dst, dst_row0, const_cast<float*>(table), rows, d_n, n_max, table_rows, D, status,
-                                   stream);
+    // loading the hot cache happens with nothing else on the chip: two mover CTAs per SM, for the link's full rate
+    return launch_move_rows<false>(dst, dst_row0, const_cast<float*>(table), rows, d_n, n_max, table_rows, D, nullptr,
+                                   2 * kSMs, status, stream);
 }
 
 }  // namespace hl
 
 using namespace hl;
 
-extern "C" int32_t hl_gather_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const float* host_table,
-                                  float* d_cache, int32_t* d_cold_rows, int64_t* d_n_cold, void* stream_) {
-    if (!ctx || !non || !non->offsets || !d_n_non || !host_table || !d_cache || !d_cold_rows || !d_n_cold)
-        return HL_EINVAL;
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+namespace hl {
+namespace {
+
+// Shared body of hl_gather_cold and hl_gather_cold_ahead.  Staging window: cache slots
+// [hot_cap + stage_row0, hot_cap + stage_row0 + stage_rows).
+int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const float* host_table, float* d_cache,
+                    int64_t stage_row0, int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold,
+                    const int32_t* d_prev_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
+                    cudaEvent_t record_after_index, cudaEvent_t wait_a, cudaEvent_t wait_b, cudaStream_t stream) {
     Regions& r = ctx->r;
     if (ctx->max_nnz == 0) {
         HL_CUDA_TRY(cudaMemsetAsync(d_n_cold, 0, sizeof(int64_t), stream));
+        if (record_after_index) HL_CUDA_TRY(cudaEventRecord(record_after_index, stream));
         return HL_OK;
     }
     if (!non->ids) return HL_EINVAL;
     HL_CUDA_TRY(cudaMemsetAsync(r.cold_n, 0, 4 * sizeof(int32_t), stream));
-    const int grid = grid_for(ctx->max_nnz, kThreads, kSMs * 4);
+    const int grid = grid_for(ctx->max_nnz, kThreads, kMaxGrid);
     k_cold_classify<<<grid, kThreads, 0, stream>>>(non->ids, non->offsets, d_n_non, ctx->max_batch, ctx->T * ctx->S,
                                                    non->cap_ids, ctx->N, r.remap, r.cold_keys[0], r.cold_vals[0],
                                                    r.cold_n, ctx->max_nnz, r.status);
@@ -207,24 +381,93 @@ extern "C" int32_t hl_gather_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_
     HL_LAUNCH_CHECK();
     st = exclusive_scan_i32(r.cold_rank, r.cold_rank, r.cold_n, ctx->max_nnz, r.cold_tiles, r.status, stream);
     if (st != HL_OK) return st;
-    k_cold_assign<<<grid, kThreads, 0, stream>>>(keys, vals, r.cold_n, ctx->max_nnz, r.cold_rank, ctx->hot_cap,
-                                                 ctx->staging_cap, non->ids, d_cold_rows, d_n_cold, r.status);
+    k_cold_assign<<<grid, kThreads, 0, stream>>>(keys, vals, r.cold_n, ctx->max_nnz, r.cold_rank,
+                                                 ctx->hot_cap + stage_row0, stage_rows, non->ids, d_cold_rows,
+                                                 d_n_cold, r.status);
     note_launches(1);
     HL_LAUNCH_CHECK();
+    if (d_prev_rows) {
+        k_cold_match<<<grid_for(stage_rows, kThreads, kMaxGrid), kThreads, 0, stream>>>(
+            d_cold_rows, d_n_cold, stage_rows, d_prev_rows, d_n_prev, ctx->staging_cap, d_fwd_src);
+        note_launches(1);
+        HL_LAUNCH_CHECK();
+    }
+    if (record_after_index) HL_CUDA_TRY(cudaEventRecord(record_after_index, stream));
+    if (wait_a) HL_CUDA_TRY(cudaStreamWaitEvent(stream, wait_a, 0));
+    if (wait_b) HL_CUDA_TRY(cudaStreamWaitEvent(stream, wait_b, 0));
     timer_mark(ctx, HL_TIMER_GATHER_MOVE, 0, stream);
-    st = launch_move_rows<false>(d_cache, ctx->hot_cap, const_cast<float*>(host_table), d_cold_rows, d_n_cold,
-                                 ctx->staging_cap, ctx->N, ctx->D, r.status, stream);
+    st = launch_move_rows<false>(d_cache, ctx->hot_cap + stage_row0, const_cast<float*>(host_table), d_cold_rows,
+                                 d_n_cold, stage_rows, ctx->N, ctx->D, d_prev_rows ? d_fwd_src : nullptr, kBulkCtas,
+                                 r.status, stream);
     timer_mark(ctx, HL_TIMER_GATHER_MOVE, 1, stream);
+    return st;
+}
+
+bool window_ok(const hl_ctx* ctx, int64_t row0, int64_t rows) {
+    return row0 >= 0 && rows >= 0 && row0 + rows <= ctx->staging_cap;
+}
+
+}  // namespace
+}  // namespace hl
+
+extern "C" int32_t hl_gather_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const float* host_table,
+                                  float* d_cache, int32_t* d_cold_rows, int64_t* d_n_cold, void* stream_) {
+    if (!ctx || !non || !non->offsets || !d_n_non || !host_table || !d_cache || !d_cold_rows || !d_n_cold)
+        return HL_EINVAL;
+    return gather_impl(ctx, non, d_n_non, host_table, d_cache, 0, ctx->staging_cap, d_cold_rows, d_n_cold, nullptr,
+                       nullptr, nullptr, nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int32_t hl_gather_cold_ahead(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const float* host_table,
+                                        float* d_cache, int64_t stage_row0, int64_t stage_rows, int32_t* d_cold_rows,
+                                        int64_t* d_n_cold, const int32_t* d_prev_cold_rows, const int64_t* d_n_prev,
+                                        int32_t* d_fwd_src, void* record_after_index, void* wait_before_move_a,
+                                        void* wait_before_move_b, void* stream_) {
+    if (!ctx || !non || !non->offsets || !d_n_non || !host_table || !d_cache || !d_cold_rows || !d_n_cold)
+        return HL_EINVAL;
+    if (!window_ok(ctx, stage_row0, stage_rows)) return HL_EINVAL;
+    if ((d_prev_cold_rows != nullptr) != (d_n_prev != nullptr) || (d_prev_cold_rows && !d_fwd_src)) return HL_EINVAL;
+    return gather_impl(ctx, non, d_n_non, host_table, d_cache, stage_row0, stage_rows, d_cold_rows, d_n_cold,
+                       d_prev_cold_rows, d_n_prev, d_fwd_src, static_cast<cudaEvent_t>(record_after_index),
+                       static_cast<cudaEvent_t>(wait_before_move_a), static_cast<cudaEvent_t>(wait_before_move_b),
+                       static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int32_t hl_forward_cold(hl_ctx* ctx, float* d_cache, int64_t from_stage_row0, int64_t to_stage_row0,
+                                   int64_t stage_rows, const int32_t* d_fwd_src, const int64_t* d_n_cold,
+                                   void* stream_) {
+    if (!ctx || !d_cache || !d_fwd_src || !d_n_cold) return HL_EINVAL;
+    if (!window_ok(ctx, from_stage_row0, stage_rows) || !window_ok(ctx, to_stage_row0, stage_rows)) return HL_EINVAL;
+    if (stage_rows == 0) return HL_OK;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int D4 = ctx->D / 4;
+    const int grid = 2 * kSMs;
+    const int64_t from = ctx->hot_cap + from_stage_row0, to = ctx->hot_cap + to_stage_row0;
+    if (D4 <= 4) k_forward_rows<4><<<grid, kThreads, 0, stream>>>(d_cache, from, to, d_fwd_src, d_n_cold, stage_rows, D4);
+    else if (D4 <= 8) k_forward_rows<8><<<grid, kThreads, 0, stream>>>(d_cache, from, to, d_fwd_src, d_n_cold, stage_rows, D4);
+    else if (D4 <= 16) k_forward_rows<16><<<grid, kThreads, 0, stream>>>(d_cache, from, to, d_fwd_src, d_n_cold, stage_rows, D4);
+    else k_forward_rows<32><<<grid, kThreads, 0, stream>>>(d_cache, from, to, d_fwd_src, d_n_cold, stage_rows, D4);
+    note_launches(1);
+    HL_LAUNCH_CHECK();
+    return HL_OK;
+}
+
+extern "C" int32_t hl_scatter_cold_at(hl_ctx* ctx, const float* d_cache, int64_t stage_row0, int64_t stage_rows,
+                                      const int32_t* d_cold_rows, const int64_t* d_n_cold, float* host_table,
+                                      void* stream_) {
+    if (!ctx || !d_cache || !d_cold_rows || !d_n_cold || !host_table) return HL_EINVAL;
+    if (!window_ok(ctx, stage_row0, stage_rows)) return HL_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 0, stream);
+    const int32_t st = launch_move_rows<true>(const_cast<float*>(d_cache), ctx->hot_cap + stage_row0, host_table,
+                                              d_cold_rows, d_n_cold, stage_rows, ctx->N, ctx->D, nullptr, kBulkCtas,
+                                              ctx->r.status, stream);
+    timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 1, stream);
     return st;
 }
 
 extern "C" int32_t hl_scatter_cold(hl_ctx* ctx, const float* d_cache, const int32_t* d_cold_rows,
                                    const int64_t* d_n_cold, float* host_table, void* stream_) {
-    if (!ctx || !d_cache || !d_cold_rows || !d_n_cold || !host_table) return HL_EINVAL;
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 0, stream);
-    const int32_t st = launch_move_rows<true>(const_cast<float*>(d_cache), ctx->hot_cap, host_table, d_cold_rows,
-                                              d_n_cold, ctx->staging_cap, ctx->N, ctx->D, ctx->r.status, stream);
-    timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 1, stream);
-    return st;
+    if (!ctx) return HL_EINVAL;
+    return hl_scatter_cold_at(ctx, d_cache, 0, ctx->staging_cap, d_cold_rows, d_n_cold, host_table, stream_);
 }

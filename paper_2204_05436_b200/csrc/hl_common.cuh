@@ -15,6 +15,10 @@ constexpr int kSortTile = 2048;            // keys per radix-sort tile (256 thre
 constexpr int kScanTile = 2048;            // elements per scan tile (256 threads x 8)
 constexpr int kSelTile = 4096;             // rows per hot-set selection tile (256 threads x 16)
 constexpr int kBwdChunk = 32;              // sorted lookups per backward chunk
+// Per-mini-batch kernels are launched with one CTA per tile of work rather than as chip-filling persistent grids:
+// they run next to the host-link movers of another micro-batch, which slow down the SMs they sit on, and the
+// hardware block scheduler then simply hands those SMs fewer CTAs.
+constexpr int kMaxGrid = 1 << 22;
 
 // One 32-byte sector per 224 rows: w[0] = number of popular rows before this block, w[1..7] = hit bitmap.
 struct __align__(32) RemapBlock {

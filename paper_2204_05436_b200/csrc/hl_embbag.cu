@@ -9,6 +9,7 @@ namespace hl {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kFwdTrips = 4;   // trips of the forward kernel per CTA
 
 __device__ __forceinline__ float4 f4_zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
 __device__ __forceinline__ void f4_add(float4& a, const float4& b) {
@@ -80,8 +81,6 @@ __global__ void __launch_bounds__(kThreads) k_embbag_fwd(const float* __restrict
                                                          float* __restrict__ out, int32_t* status) {
     const int64_t n_bags = (int64_t)clamp_samples(d_n_samples, max_batch) * bags_per_sample_all;
     const int sub = threadIdx.x % G;
-    const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
-    const int64_t n_groups = (int64_t)gridDim.x * kThreads / G;
     const float4* __restrict__ rows = reinterpret_cast<const float4*>(cache);
     float4* __restrict__ out4 = reinterpret_cast<float4*>(out);
 
@@ -98,10 +97,14 @@ __global__ void __launch_bounds__(kThreads) k_embbag_fwd(const float* __restrict
         for (int u = 0; u < UB; ++u) id1[u] = len[u] == 1 ? __ldg(&ids[lo[u]]) : -1;
     };
 
+    // this CTA's tile: kFwdTrips consecutive trips of (groups per CTA) x UB bags
+    constexpr int kGroups = kThreads / G;
     int32_t lo[UB], len[UB], id1[UB];
-    int64_t bag0 = group * UB;
-    if (bag0 < n_bags) load_index(bag0, lo, len, id1);
-    for (; bag0 < n_bags; bag0 += n_groups * UB) {
+    const int64_t tile0 = (int64_t)blockIdx.x * kFwdTrips * kGroups * UB;
+    const int64_t tile_end = min(n_bags, tile0 + (int64_t)kFwdTrips * kGroups * UB);
+    int64_t bag0 = tile0 + (int64_t)(threadIdx.x / G) * UB;
+    if (bag0 < tile_end) load_index(bag0, lo, len, id1);
+    for (; bag0 < tile_end; bag0 += kGroups * UB) {
         float4 row[UB][NV];
 #pragma unroll
         for (int u = 0; u < UB; ++u) {
@@ -116,8 +119,8 @@ __global__ void __launch_bounds__(kThreads) k_embbag_fwd(const float* __restrict
         int32_t cur_len[UB];
 #pragma unroll
         for (int u = 0; u < UB; ++u) cur_len[u] = len[u];
-        const int64_t next0 = bag0 + n_groups * UB;
-        if (next0 < n_bags) load_index(next0, lo, len, id1);   // in flight while this trip's rows arrive
+        const int64_t next0 = bag0 + kGroups * UB;
+        if (next0 < tile_end) load_index(next0, lo, len, id1);   // in flight while this trip's rows arrive
         unsigned long_bags = 0;   // bit u: bag u of this trip has more than one lookup
 #pragma unroll
         for (int u = 0; u < UB; ++u) {
@@ -176,32 +179,16 @@ __global__ void __launch_bounds__(kThreads) k_bwd_pairs(const int32_t* __restric
     }
 }
 
-template <int G, int NV>
-struct RowOps {
-    // cache[key, :] -= lr * acc  (this group's columns)
-    static __device__ __forceinline__ void sgd(float* cache, int64_t key, int D4, int sub, float lr,
-                                               const float4 (&acc)[NV]) {
-        float4* row = reinterpret_cast<float4*>(cache) + key * D4;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int c = sub + v * G;
-            if (c < D4) {
-                float4 w = row[c];
-                w.x -= lr * acc[v].x;
-                w.y -= lr * acc[v].y;
-                w.z -= lr * acc[v].z;
-                w.w -= lr * acc[v].w;
-                row[c] = w;
-            }
-        }
-    }
-};
-
 // The sorted lookups are cut into chunks of kBwdChunk.  One group per chunk sums, in order, the gradient rows of
 // each run of equal slots inside its chunk.  A run that lies wholly inside the chunk is finished here (one
 // read-modify-write of its row).  A run that crosses a chunk border leaves a partial sum: part[chunk][0] for the
 // piece that continues a run from the previous chunk, part[chunk][1] for the piece that starts a run continuing
 // into the next chunk.  k_bwd_spans adds those up.
+//
+// The group reads its chunk's 32 (slot, bag) pairs with one coalesced load per lane and passes them round by
+// shuffles, so that all gradient-row addresses are known at once; gradient rows are then loaded U at a time,
+// together with the cache row of every run that starts among those U lookups (the row is needed only when the
+// run closes, but asking for it up front takes its latency off the critical path).
 template <int G, int NV>
 __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cache,
                                                          const int32_t* __restrict__ keys,
@@ -209,27 +196,55 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
                                                          const int32_t* __restrict__ d_n_lookups,
                                                          const float* __restrict__ grad_out, int D4, int64_t n_slots,
                                                          float lr, float* __restrict__ part) {
-    constexpr int U = NV >= 8 ? 1 : (NV >= 4 ? 2 : (NV >= 2 ? 4 : 8));
+    constexpr int KPL = kBwdChunk / G;                       // pairs held per lane
+    constexpr int U = NV >= 4 ? 1 : (NV >= 2 ? 2 : 4);       // lookups in flight per lane
+    static_assert(G % U == 0, "batch must divide the group");
     const int64_t n = d_n_lookups[0];
-    const int sub = threadIdx.x % G;
+    const int lane = threadIdx.x & 31;
+    const int sub = lane % G;
+    const unsigned gmask = G == 32 ? 0xffffffffu : (((1u << G) - 1u) << (lane / G * G));
     const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
     const int64_t n_groups = (int64_t)gridDim.x * kThreads / G;
     const float4* __restrict__ grad4 = reinterpret_cast<const float4*>(grad_out);
+    float4* cache4 = reinterpret_cast<float4*>(cache);
     float4* __restrict__ part4 = reinterpret_cast<float4*>(part);
 
     for (int64_t chunk = group; chunk * kBwdChunk < n; chunk += n_groups) {
         const int64_t start = chunk * kBwdChunk;
         const int64_t end = min(start + (int64_t)kBwdChunk, n);
-        int32_t cur = keys[start];
-        bool seg_left_open = start > 0 && keys[start - 1] == cur;
-        float4 acc[NV];
+        int32_t kk[KPL], vv[KPL];
 #pragma unroll
-        for (int v = 0; v < NV; ++v) acc[v] = f4_zero();
+        for (int i = 0; i < KPL; ++i) {
+            const int64_t p = start + i * G + sub;
+            kk[i] = p < end ? keys[p] : -1;
+            vv[i] = p < end ? vals[p] : 0;
+        }
+        const int32_t prev_key = start > 0 ? keys[start - 1] : -3;   // -3: equal to no key
+        const int32_t next_key = end < n ? keys[end] : -2;
+
+        int32_t cur = prev_key;        // slot of the segment being summed
+        bool seg_left_open = true;     // it continues a run from the previous chunk (until the slot changes)
+        int seg_count = 0;             // lookups of this chunk summed into it so far
+        int32_t last_k = prev_key;     // slot of the previous lookup (to spot run heads)
+        float4 acc[NV], wrow[NV];
+#pragma unroll
+        for (int v = 0; v < NV; ++v) acc[v] = wrow[v] = f4_zero();
 
         auto flush = [&](bool right_open) {
-            if (cur >= n_slots) return;   // sentinel: lookups that were skipped
+            if (seg_count == 0 || cur >= n_slots) return;   // nothing summed, or the sentinel of skipped lookups
             if (!seg_left_open && !right_open) {
-                RowOps<G, NV>::sgd(cache, cur, D4, sub, lr, acc);
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const int c = sub + v * G;
+                    if (c < D4) {
+                        float4 w = wrow[v];
+                        w.x -= lr * acc[v].x;
+                        w.y -= lr * acc[v].y;
+                        w.z -= lr * acc[v].z;
+                        w.w -= lr * acc[v].w;
+                        cache4[(int64_t)cur * D4 + c] = w;
+                    }
+                }
             } else {
                 const int64_t slot = chunk * 2 + (seg_left_open ? 0 : 1);
 #pragma unroll
@@ -240,105 +255,117 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
             }
         };
 
-        for (int64_t p0 = start; p0 < end; p0 += U) {
-            int32_t k[U], b[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const bool valid = p0 + u < end;
-                k[u] = valid ? keys[p0 + u] : -1;
-                b[u] = valid ? vals[p0 + u] : 0;
-            }
-            float4 g[U][NV];
+        for (int i = 0; i < KPL; ++i) {
+            for (int j = 0; j < G; j += U) {
+                int32_t k[U], b[U];
+                bool head[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u)
+                for (int u = 0; u < U; ++u) {
+                    k[u] = __shfl_sync(gmask, kk[i], j + u, G);
+                    b[u] = __shfl_sync(gmask, vv[i], j + u, G);
+                    head[u] = k[u] != last_k;
+                    last_k = k[u] >= 0 ? k[u] : last_k;
+                }
+                float4 g[U][NV], wn[U][NV];
 #pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    const int c = sub + v * G;
-                    g[u][v] = (k[u] >= 0 && k[u] < n_slots && c < D4) ? __ldg(&grad4[(int64_t)b[u] * D4 + c])
-                                                                      : f4_zero();
+                for (int u = 0; u < U; ++u) {
+                    const bool ok = k[u] >= 0 && k[u] < n_slots;
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        const int c = sub + v * G;
+                        g[u][v] = (ok && c < D4) ? __ldg(&grad4[(int64_t)b[u] * D4 + c]) : f4_zero();
+                        wn[u][v] = (ok && head[u] && c < D4) ? cache4[(int64_t)k[u] * D4 + c] : f4_zero();
+                    }
                 }
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                if (p0 + u < end) {
+                for (int u = 0; u < U; ++u) {
+                    if (k[u] < 0) continue;   // past the end of the last chunk
                     if (k[u] != cur) {
                         flush(false);
-#pragma unroll
-                        for (int v = 0; v < NV; ++v) acc[v] = f4_zero();
                         cur = k[u];
                         seg_left_open = false;
+                        seg_count = 0;
+#pragma unroll
+                        for (int v = 0; v < NV; ++v) {
+                            acc[v] = f4_zero();
+                            wrow[v] = wn[u][v];
+                        }
                     }
 #pragma unroll
                     for (int v = 0; v < NV; ++v) f4_add(acc[v], g[u][v]);
+                    ++seg_count;
                 }
             }
         }
-        flush(end < n && keys[end] == cur);
+        flush(next_key == cur);
     }
 }
 
-// One group per chunk; it acts only if a run STARTS in its chunk and continues into the next one.  It finds the
-// run's end by a galloping search over the sorted keys, adds the continuation pieces in chunk order, and applies
-// the single SGD update of that row.
+// One WARP per chunk; it acts only if a run STARTS in its chunk and continues into the next one.  The lanes look
+// at the last slot of the next 32 chunks at once to find where the run ends, the warp's 32/G groups add the
+// run's continuation pieces in an interleaved, fixed order in fp64 (runs of many thousands of lookups occur), the
+// group sums are combined by shuffles in a fixed order, and group 0 applies the single SGD update of the row.
 template <int G, int NV>
 __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cache, const int32_t* __restrict__ keys,
                                                         const int32_t* __restrict__ d_n_lookups, int D4,
                                                         int64_t n_slots, float lr, const float* __restrict__ part) {
+    constexpr int GW = 32 / G;   // groups per warp
+    constexpr int U = NV >= 4 ? 1 : (NV >= 2 ? 2 : 4);
     const int64_t n = d_n_lookups[0];
-    const int sub = threadIdx.x % G;
-    const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
-    const int64_t n_groups = (int64_t)gridDim.x * kThreads / G;
+    const int lane = threadIdx.x & 31;
+    const int sub = lane % G, gi = lane / G;
+    const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * kThreads) >> 5;
     const float4* __restrict__ part4 = reinterpret_cast<const float4*>(part);
+    float4* cache4 = reinterpret_cast<float4*>(cache);
 
-    for (int64_t chunk = group; chunk * kBwdChunk < n; chunk += n_groups) {
+    for (int64_t chunk = warp; chunk * kBwdChunk < n; chunk += n_warps) {
         const int64_t start = chunk * kBwdChunk;
         const int64_t end = min(start + (int64_t)kBwdChunk, n);
         if (end >= n) continue;
         const int32_t key = keys[end - 1];
-        if (key >= n_slots || keys[end] != key) continue;                        // not right-open
-        if (keys[start] == key && start > 0 && keys[start - 1] == key) continue;   // run started earlier
+        if (key >= n_slots || keys[end] != key) continue;                         // not right-open
+        if (keys[start] == key && start > 0 && keys[start - 1] == key) continue;    // run started earlier
 
-        // e = one past the run's last lookup
-        int64_t lo = end, hi, step = kBwdChunk;
-        for (;;) {
-            hi = lo + step;
-            if (hi >= n) {
-                hi = n;
-                break;
-            }
-            if (keys[hi] != key) break;
-            lo = hi;
-            step <<= 1;
+        // last chunk that holds a piece of the run: a later chunk lies wholly inside the run iff its last slot is
+        // the run's slot
+        int64_t last_chunk;
+        for (int64_t base = chunk + 1;; base += 32) {
+            const int64_t cc = base + lane;
+            const bool in_range = cc * kBwdChunk < n;
+            const int64_t last_pos = min((cc + 1) * (int64_t)kBwdChunk, n) - 1;
+            const bool whole = in_range && keys[last_pos] == key;
+            const unsigned m = __ballot_sync(0xffffffffu, whole);
+            if (m == 0xffffffffu) continue;
+            const int first_not = __ffs(~m) - 1;
+            const int64_t cand = base + first_not;   // first chunk not wholly inside the run
+            last_chunk = (cand * kBwdChunk < n && keys[cand * kBwdChunk] == key) ? cand : cand - 1;
+            break;
         }
-        while (hi - lo > 1) {
-            const int64_t mid = (lo + hi) >> 1;
-            if (keys[mid] == key) lo = mid;
-            else hi = mid;
-        }
-        const int64_t last_chunk = (hi - 1) / kBwdChunk;
 
-        // the pieces of one run are added in chunk order in fp64 (runs of many thousands of lookups occur)
         double dacc[NV][4];
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             const int c = sub + v * G;
-            const float4 t = c < D4 ? part4[(chunk * 2 + 1) * D4 + c] : f4_zero();
+            const float4 t = (gi == 0 && c < D4) ? part4[(chunk * 2 + 1) * D4 + c] : f4_zero();
             dacc[v][0] = t.x;
             dacc[v][1] = t.y;
             dacc[v][2] = t.z;
             dacc[v][3] = t.w;
         }
-        int64_t c2 = chunk + 1;
-        for (; c2 + 3 <= last_chunk; c2 += 4) {
-            float4 t[4][NV];
+        for (int64_t c2 = chunk + 1 + gi; c2 <= last_chunk; c2 += (int64_t)GW * U) {
+            float4 t[U][NV];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < U; ++u)
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     const int c = sub + v * G;
-                    t[u][v] = c < D4 ? part4[((c2 + u) * 2) * D4 + c] : f4_zero();
+                    const int64_t cc = c2 + (int64_t)u * GW;
+                    t[u][v] = (cc <= last_chunk && c < D4) ? part4[(cc * 2) * D4 + c] : f4_zero();
                 }
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < U; ++u)
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     dacc[v][0] += (double)t[u][v].x;
@@ -347,23 +374,26 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
                     dacc[v][3] += (double)t[u][v].w;
                 }
         }
-        for (; c2 <= last_chunk; ++c2)
+#pragma unroll
+        for (int off = G; off < 32; off <<= 1)
+#pragma unroll
+            for (int v = 0; v < NV; ++v)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) dacc[v][e] += __shfl_xor_sync(0xffffffffu, dacc[v][e], off);
+        if (gi == 0) {
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
                 const int c = sub + v * G;
                 if (c < D4) {
-                    const float4 t = part4[(c2 * 2) * D4 + c];
-                    dacc[v][0] += (double)t.x;
-                    dacc[v][1] += (double)t.y;
-                    dacc[v][2] += (double)t.z;
-                    dacc[v][3] += (double)t.w;
+                    float4 w = cache4[(int64_t)key * D4 + c];
+                    w.x -= lr * (float)dacc[v][0];
+                    w.y -= lr * (float)dacc[v][1];
+                    w.z -= lr * (float)dacc[v][2];
+                    w.w -= lr * (float)dacc[v][3];
+                    cache4[(int64_t)key * D4 + c] = w;
                 }
             }
-        float4 acc[NV];
-#pragma unroll
-        for (int v = 0; v < NV; ++v)
-            acc[v] = make_float4((float)dacc[v][0], (float)dacc[v][1], (float)dacc[v][2], (float)dacc[v][3]);
-        RowOps<G, NV>::sgd(cache, key, D4, sub, lr, acc);
+        }
     }
 }
 
@@ -371,17 +401,8 @@ template <int G, int NV>
 int32_t launch_fwd(hl_ctx* ctx, const float* cache, const hl_ubatch* ub, const int32_t* d_n, float* out,
                    cudaStream_t stream) {
     constexpr int UB = NV >= 4 ? 1 : (NV >= 2 ? 2 : 4);
-    // persistent grid: as many CTAs as fit on the chip at once (a whole number per SM), never more than the work
-    static int ctas_per_sm = 0;
-    if (ctas_per_sm == 0) {
-        int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_embbag_fwd<G, NV, UB>, kThreads, 0) != cudaSuccess ||
-            n < 1)
-            n = 2;
-        ctas_per_sm = n;
-    }
-    const int64_t max_bags = ctx->max_bags;
-    const int grid = grid_for(div_up(max_bags, UB) * G, kThreads, kSMs * ctas_per_sm);
+    const int64_t bags_per_cta = (int64_t)kFwdTrips * (kThreads / G) * UB;
+    const int grid = grid_for(ctx->max_bags, (int)bags_per_cta, kMaxGrid);
     timer_mark(ctx, HL_TIMER_FWD, 0, stream);
     k_embbag_fwd<G, NV, UB><<<grid, kThreads, 0, stream>>>(cache, ub->ids, ub->offsets, d_n, ctx->max_batch,
                                                           ctx->T * ctx->S, ctx->D / 4,
@@ -396,14 +417,15 @@ template <int G, int NV>
 int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t* vals, const float* grad, float lr,
                    cudaStream_t stream) {
     const int64_t max_chunks = div_up(ctx->max_nnz, kBwdChunk);
-    const int grid = grid_for(max_chunks * G, kThreads, kSMs * 8);
+    const int grid = grid_for(max_chunks * G, kThreads, kMaxGrid);
     const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 0, stream);
     k_bwd_chunks<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, vals, ctx->r.bwd_n, grad, ctx->D / 4, n_slots,
                                                       lr, ctx->r.bwd_part);
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 1, stream);
-    k_bwd_spans<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, ctx->r.bwd_n, ctx->D / 4, n_slots, lr,
-                                                     ctx->r.bwd_part);
+    const int span_grid = grid_for(max_chunks * 32, kThreads, kMaxGrid);   // one warp per chunk
+    k_bwd_spans<G, NV><<<span_grid, kThreads, 0, stream>>>(cache, keys, ctx->r.bwd_n, ctx->D / 4, n_slots, lr,
+                                                          ctx->r.bwd_part);
     note_launches(2);
     HL_LAUNCH_CHECK();
     return HL_OK;
@@ -452,11 +474,11 @@ extern "C" int32_t hl_embbag_bwd_sgd(hl_ctx* ctx, float* d_cache, const hl_ubatc
     const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
     const bool short_bags = ctx->max_nnz <= 4 * ctx->max_bags;
     if (short_bags)
-        k_bwd_pairs<1><<<grid_for(ctx->max_bags, kThreads, kSMs * 8), kThreads, 0, stream>>>(
+        k_bwd_pairs<1><<<grid_for(ctx->max_bags, kThreads, kMaxGrid), kThreads, 0, stream>>>(
             ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, r.bwd_keys[0],
             r.bwd_vals[0], r.bwd_n, r.status);
     else
-        k_bwd_pairs<32><<<grid_for(ctx->max_bags, kThreads / 32, kSMs * 8), kThreads, 0, stream>>>(
+        k_bwd_pairs<32><<<grid_for(ctx->max_bags, kThreads / 32, kMaxGrid), kThreads, 0, stream>>>(
             ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, r.bwd_keys[0],
             r.bwd_vals[0], r.bwd_n, r.status);
     note_launches(1);

@@ -272,7 +272,7 @@ int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n,
         uint32_t* tstat = hist + 4 * 256 + 8;
         HL_CUDA_TRY(cudaMemsetAsync(hist, 0, sizeof(uint32_t) * (4 * 256 + 8 + (size_t)passes * n_tiles * 256),
                                     stream));
-        k_sort_digit_hist<<<grid_for(n_max, kThreads * 8, kSMs * 2), kThreads, 0, stream>>>(keys[0], d_n, n_max,
+        k_sort_digit_hist<<<grid_for(n_max, kThreads * 8, kMaxGrid), kThreads, 0, stream>>>(keys[0], d_n, n_max,
                                                                                             passes, ghist);
         for (int p = 0; p < passes; ++p) {
             k_sort_pass<<<(unsigned)n_tiles, kThreads, 0, stream>>>(keys[cur], vals[cur], keys[cur ^ 1], vals[cur ^ 1],

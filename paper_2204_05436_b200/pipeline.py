@@ -180,3 +180,138 @@ class Hotline:
     def synchronize(self) -> None:
         self.main.synchronize()
         self.side.synchronize()
+
+
+class _BatchSet:
+    """Index buffers and outputs of one mini-batch in flight."""
+
+    def __init__(self, h: "Hotline"):
+        dev, i32, i64, f32 = h.device, torch.int32, torch.int64, torch.float32
+        ids_cap = max(1, h.max_nnz)
+        self.perm = torch.zeros(h.max_batch, dtype=i32, device=dev)
+        self.counts = torch.zeros(4, dtype=i32, device=dev)
+        self.pop_offsets = torch.zeros(h.max_bags + 1, dtype=i32, device=dev)
+        self.pop_ids = torch.zeros(ids_cap, dtype=i32, device=dev)
+        self.non_offsets = torch.zeros(h.max_bags + 1, dtype=i32, device=dev)
+        self.non_ids = torch.zeros(ids_cap, dtype=i32, device=dev)
+        self.pop = B.make_ubatch(self.pop_offsets, self.pop_ids, h.max_nnz)
+        self.non = B.make_ubatch(self.non_offsets, self.non_ids, h.max_nnz)
+        self.cold_rows = torch.zeros(max(1, h.window_rows), dtype=i32, device=dev)
+        self.n_cold = torch.zeros(1, dtype=i64, device=dev)
+        self.fwd_src = torch.full((max(1, h.window_rows),), -1, dtype=i32, device=dev)
+        self.pooled_pop = torch.zeros((h.max_bags, h.D), dtype=f32, device=dev)
+        self.pooled_non = torch.zeros((h.max_bags, h.D), dtype=f32, device=dev)
+        self.dense_out = torch.zeros((h.max_batch, h.n_dense), dtype=f32, device=dev) if h.n_dense else None
+        # events whose handles the library records or waits on: record each once so that the handle exists
+        self.ev_index = torch.cuda.Event()
+        self.ev_gather = torch.cuda.Event()
+        self.ev_forward = torch.cuda.Event()
+        self.ev_x = torch.cuda.Event()
+        self.ev_scatter = torch.cuda.Event()
+        for e in (self.ev_index, self.ev_gather, self.ev_forward, self.ev_x, self.ev_scatter):
+            e.record(h.main)
+
+
+class PipelinedHotline(Hotline):
+    """The same path, software-pipelined across mini-batches: while mini-batch j executes on the main stream,
+    mini-batch j+1 is already fragmented and its cold rows staged on a side stream, and mini-batch j-1's cold rows
+    are written back on a third stream.  The result is that of processing the mini-batches one after the other:
+    a cold row that j+1 shares with j is not read from the host but copied from j's staging window after j's
+    backward (hl_forward_cold), and the host rows of j+1 are read only after j-1's write-back has finished.
+
+    Three sets of index buffers rotate over the mini-batches, two windows of the staging area alternate.
+
+        p.start(idx0, off0, B)                       # ahead-work of mini-batch 0
+        for j in range(n):
+            s = p.step(grad_pop, grad_non, lr, next_batch=(idx, off, B, dense) or None)
+            ... p.sets[s].pooled_pop / pooled_non are mini-batch j's outputs once the main stream gets there
+        p.drain()
+    """
+
+    def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
+                 n_dense: int = 0, device: str = "cuda:0"):
+        self.window_rows = int(window_rows)
+        super().__init__(table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, 2 * self.window_rows,
+                         host_table, n_dense=n_dense, device=device)
+        self.sets = [_BatchSet(self) for _ in range(3)]
+        self.sides = [self.side, torch.cuda.Stream(device=self.device)]
+        self.wb = torch.cuda.Stream(device=self.device)
+        self._ev_inputs = torch.cuda.Event()
+        self.j_submitted = 0      # mini-batches whose ahead-work has been issued
+        self.j_done = 0           # mini-batches whose main work has been issued
+        torch.cuda.synchronize(self.device)
+
+    @staticmethod
+    def _timed(timers, name, stream, fn):
+        if timers is None:
+            fn()
+            return
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        fn()
+        b.record(stream)
+        timers.setdefault(name, []).append((a, b))
+
+    def _submit(self, indices, offsets, batch: int, dense=None, timers=None) -> None:
+        j = self.j_submitted
+        st, side = self.sets[j % 3], self.sides[j % 2]
+        self._ev_inputs.record(self.main)                # the caller prepared the inputs on the main stream
+        side.wait_event(self._ev_inputs)
+        if j >= 3:
+            side.wait_event(st.ev_scatter)               # set j%3 was mini-batch j-3's: long done, stated anyway
+        prev = self.sets[(j - 1) % 3] if j >= 1 else None
+        if prev is not None:
+            side.wait_event(prev.ev_index)               # its cold set is final; fragment/cold scratch is free
+        self._timed(timers, "fragment", side, lambda: B.hl_fragment(
+            self.ctx, self._batch(indices, offsets, batch), dense, self.n_dense if dense is not None else 0,
+            st.perm, st.counts, st.pop, st.non, st.dense_out if dense is not None else None, side.cuda_stream))
+        self._timed(timers, "gather_cold", side, lambda: B.hl_gather_cold_ahead(
+            self.ctx, st.non, st.counts[1:], self.host_table, self.cache, (j % 2) * self.window_rows,
+            self.window_rows, st.cold_rows, st.n_cold,
+            prev.cold_rows if prev is not None else None, prev.n_cold if prev is not None else None, st.fwd_src,
+            st.ev_index,
+            self.sets[(j - 2) % 3].ev_scatter if j >= 2 else None,     # host rows of j-2 are final after its write-back
+            prev.ev_forward if prev is not None else None,             # j-1 has copied what it needs out of this window
+            side.cuda_stream))
+        st.ev_gather.record(side)
+        self.j_submitted += 1
+
+    def start(self, indices, offsets, batch: int, dense=None) -> None:
+        assert self.j_submitted == self.j_done, "start() only with nothing in flight"
+        self._submit(indices, offsets, batch, dense)
+
+    def step(self, grad_pop: torch.Tensor, grad_non: torch.Tensor, lr: float, next_batch=None, timers=None) -> int:
+        """Main work of the oldest submitted mini-batch; ``next_batch`` = (indices, offsets, batch, dense) of
+        the one after it (its ahead-work is issued here), or None at the end.  Returns the index of the buffer set
+        that holds this mini-batch's outputs."""
+        j = self.j_done
+        assert self.j_submitted == j + 1, "call start() first"
+        st, m = self.sets[j % 3], self.main
+        s_main = m.cuda_stream
+        w0, w1 = (j % 2) * self.window_rows, ((j + 1) % 2) * self.window_rows
+        m.wait_event(st.ev_index)
+        if j >= 1:   # rows shared with mini-batch j-1 come from its staging window (its backward ran on this stream)
+            B.hl_forward_cold(self.ctx, self.cache, w1, w0, self.window_rows, st.fwd_src, st.n_cold, s_main)
+        st.ev_forward.record(m)
+        if next_batch is not None:
+            self._submit(*next_batch, timers=timers)
+        t = lambda name, stream, fn: self._timed(timers, name, stream, fn)   # noqa: E731
+        t("fwd_pop", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.pop, st.counts, st.pooled_pop, s_main))
+        t("bwd_pop", m, lambda: B.hl_embbag_bwd_sgd(self.ctx, self.cache, st.pop, st.counts, grad_pop, lr, s_main))
+        m.wait_event(st.ev_gather)
+        t("fwd_non", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.non, st.counts[1:], st.pooled_non, s_main))
+        t("bwd_non", m, lambda: B.hl_embbag_bwd_sgd(self.ctx, self.cache, st.non, st.counts[1:], grad_non, lr,
+                                                    s_main))
+        st.ev_x.record(m)
+        self.wb.wait_event(st.ev_x)
+        t("scatter_cold", self.wb, lambda: B.hl_scatter_cold_at(
+            self.ctx, self.cache, w0, self.window_rows, st.cold_rows, st.n_cold, self.host_table,
+            self.wb.cuda_stream))
+        st.ev_scatter.record(self.wb)
+        self.j_done += 1
+        return j % 3
+
+    def drain(self) -> None:
+        """Waits until everything issued so far, write-backs included, has finished."""
+        for s in [self.main, self.wb] + self.sides:
+            s.synchronize()

@@ -208,3 +208,107 @@ def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: boo
     finally:
         h.close()
     return stats
+
+
+def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: bool = True, profile_batches=None,
+                        device: str = "cuda:0"):
+    """Software-pipelined CUDA path (PipelinedHotline) against the oracle processing the same mini-batches one
+    after the other.  With integer data every sum is exact, so pooled vectors, the hot cache and the host table
+    must agree bit for bit after any number of steps -- which they only do if rows shared by consecutive
+    mini-batches are forwarded and write-backs are ordered correctly."""
+    import paper_2204_05436_b200 as hl
+
+    if isinstance(spec, str):
+        spec = gen.CONFIGS[spec]
+    geom = gen.make_geometry(spec, scale_rows)
+    T, D, S, B = geom.num_tables, geom.dim, geom.bags_per_sample, spec.batch
+    N = geom.total_rows
+    n_bags = T * B * S
+    P = spec.profile_batches if profile_batches is None else profile_batches
+    lr = 0.125 if integer else spec.lr
+    max_nnz = max_nnz_of(spec, geom, B)
+    K = orc.hot_capacity(spec.hot_policy, N, D)
+    hot_cap = max(1, min(K, N))
+    window = max(1, min(N, max_nnz))
+
+    table0 = gen.table_values(np.arange(N), D, spec.seed, integer=integer)
+    prof = [gen.make_batch(spec, geom, i) for i in range(P)]
+    cnt = orc.access_counts([(b.indices, b.offsets) for b in prof], B, geom.table_rows, S)
+    hot_o = orc.select_hot(cnt, min(K, hot_cap))
+    remap_o = orc.build_remap(hot_o, N)
+    n_hot = len(hot_o)
+
+    # ---- oracle: one mini-batch after the other ----
+    table_o = table0.copy()
+    cache_o = np.zeros((hot_cap + window, D), dtype=np.float32)
+    cache_o[:n_hot] = orc.load_hot_cache(table0, hot_o)
+    batches, grads, expect = [], [], []
+    shared = 0
+    prev_C = np.zeros(0, dtype=np.int64)
+    for step in range(steps):
+        bid = P + step
+        batch = gen.make_batch(spec, geom, bid)
+        grad_full = gen.grad_values(spec.seed, bid, 2, n_bags, D, integer=integer)
+        perm_o, n_pop_o, _, _, _ = orc.fragment(batch.indices, batch.offsets, B, geom.table_rows, remap_o, S)
+        g_pop, _ = mu_grad(grad_full, perm_o[:n_pop_o], T, B, S)
+        g_non, _ = mu_grad(grad_full, perm_o[n_pop_o:], T, B, S)
+        out = orc.hotline_step(table_o, cache_o, hot_cap, remap_o, batch.indices, batch.offsets, B, geom.table_rows,
+                               S, g_pop, g_non, lr)
+        _, _, _, _, C, pooled_pop_o, pooled_non_o = out
+        shared += len(np.intersect1d(C, prev_C))
+        prev_C = C
+        batches.append(batch)
+        grads.append((g_pop, g_non))
+        expect.append((perm_o, n_pop_o, pooled_pop_o, pooled_non_o, len(C)))
+
+    # ---- CUDA: pipelined ----
+    host_table = torch.from_numpy(table0.copy()).pin_memory()
+    p = hl.PipelinedHotline(geom.table_rows, D, S, B, max_nnz, hot_cap, window, host_table, n_dense=spec.n_dense,
+                            device=device)
+    got = []
+    try:
+        with torch.cuda.stream(p.main):
+            p.set_hot_rows(_t(hot_o, device))
+            p.build_remap(load_rows=True)
+            d_batches = [(_t(b.indices, device), _t(b.offsets, device), B,
+                          _t(b.dense, device) if b.dense is not None else None) for b in batches]
+            d_grads = []
+            for (g_pop, g_non) in grads:
+                gp = torch.zeros((n_bags, D), dtype=torch.float32, device=device)
+                gn = torch.zeros((n_bags, D), dtype=torch.float32, device=device)
+                gp[:len(g_pop)] = _t(g_pop, device)
+                gn[:len(g_non)] = _t(g_non, device)
+                d_grads.append((gp, gn))
+            torch.cuda.synchronize()
+            p.start(*d_batches[0])
+            for step in range(steps):
+                nxt = d_batches[step + 1] if step + 1 < steps else None
+                s = p.step(d_grads[step][0], d_grads[step][1], lr, next_batch=nxt)
+                st = p.sets[s]
+                got.append((st.perm.clone(), st.counts.clone(), st.pooled_pop.clone(), st.pooled_non.clone(),
+                            st.n_cold.clone()))
+            p.drain()
+            p.status()
+        for step in range(steps):
+            perm_o, n_pop_o, pooled_pop_o, pooled_non_o, n_cold_o = expect[step]
+            perm_g, counts_g, pp, pn, n_cold_g = [x.cpu().numpy() for x in got[step]]
+            assert counts_g[0] == n_pop_o and counts_g[1] == B - n_pop_o, ("counts", step)
+            assert np.array_equal(perm_g[:B], perm_o), ("perm", step)
+            assert int(n_cold_g[0]) == n_cold_o, ("n_cold", step)
+            bags_pop, bags_non = T * n_pop_o * S, T * (B - n_pop_o) * S
+            if integer:
+                assert np.array_equal(pp[:bags_pop], pooled_pop_o), ("pooled_pop", step)
+                assert np.array_equal(pn[:bags_non], pooled_non_o), ("pooled_non", step)
+            else:
+                assert_close(pp[:bags_pop], pooled_pop_o, f"pooled_pop step {step}")
+                assert_close(pn[:bags_non], pooled_non_o, f"pooled_non step {step}")
+        hot_g = p.cache[:n_hot].cpu().numpy()
+        if integer:
+            assert np.array_equal(hot_g, cache_o[:n_hot]), "hot cache"
+            assert np.array_equal(p.host_table.numpy(), table_o), "host table"
+        else:
+            assert_close(hot_g, cache_o[:n_hot], "hot cache")
+            assert_close(p.host_table.numpy(), table_o, "host table")
+    finally:
+        p.close()
+    return dict(shared_cold_rows=shared, steps=steps)

@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import gen
-from tests.harness import run_config_check
+from tests.harness import run_config_check, run_pipelined_check
 
 pytestmark = pytest.mark.gpu
 
@@ -93,3 +93,22 @@ def test_batch_of_one_and_single_table():
     spec = gen.WorkloadSpec(name="one", num_tables=1, dim=16, batch=1, rows=("fixed", 50), alpha=(1.5,),
                             hot_policy=("topk", 10), profile_batches=3, seed=3)
     run_config_check(spec, steps=2)
+
+
+def test_pipelined_steps_equal_sequential_steps_integer_data():
+    """Six mini-batches through the software pipeline; with integer data the result must be bit-identical to the
+    oracle's one-after-the-other processing.  Consecutive Zipf mini-batches share cold rows, so this exercises the
+    forwarding of staged rows and the ordering of write-backs."""
+    stats = run_pipelined_check("tiny", steps=6, integer=True)
+    assert stats["shared_cold_rows"] > 50
+
+
+def test_pipelined_steps_real_data_and_dense_features():
+    run_pipelined_check("dlrm_small", steps=3, scale_rows=0.02, integer=False, profile_batches=6)
+
+
+def test_pipelined_multi_hot_integer_data():
+    spec = dataclasses.replace(gen.CONFIGS["multi_hot"], batch=1024, dim=32, rows=("fixed", 3000),
+                               hot_policy=("fraction", 40, 100), profile_batches=2)
+    stats = run_pipelined_check(spec, steps=5, integer=True)
+    assert stats["shared_cold_rows"] > 100
