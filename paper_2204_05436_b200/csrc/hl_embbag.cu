@@ -226,9 +226,15 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
         bool seg_left_open = true;     // it continues a run from the previous chunk (until the slot changes)
         int seg_count = 0;             // lookups of this chunk summed into it so far
         int32_t last_k = prev_key;     // slot of the previous lookup (to spot run heads)
-        float4 acc[NV], wrow[NV];
+        // a segment's sum is kept in fp64: a popular row can collect tens of thousands of gradient rows, and the
+        // rounding of many fp32 partial sums would show in the updated row
+        double acc[NV][4];
+        float4 wrow[NV];
 #pragma unroll
-        for (int v = 0; v < NV; ++v) acc[v] = wrow[v] = f4_zero();
+        for (int v = 0; v < NV; ++v) {
+            acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0.0;
+            wrow[v] = f4_zero();
+        }
 
         auto flush = [&](bool right_open) {
             if (seg_count == 0 || cur >= n_slots) return;   // nothing summed, or the sentinel of skipped lookups
@@ -238,10 +244,10 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
                     const int c = sub + v * G;
                     if (c < D4) {
                         float4 w = wrow[v];
-                        w.x -= lr * acc[v].x;
-                        w.y -= lr * acc[v].y;
-                        w.z -= lr * acc[v].z;
-                        w.w -= lr * acc[v].w;
+                        w.x -= lr * (float)acc[v][0];
+                        w.y -= lr * (float)acc[v][1];
+                        w.z -= lr * (float)acc[v][2];
+                        w.w -= lr * (float)acc[v][3];
                         cache4[(int64_t)cur * D4 + c] = w;
                     }
                 }
@@ -250,7 +256,9 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     const int c = sub + v * G;
-                    if (c < D4) part4[slot * D4 + c] = acc[v];
+                    if (c < D4)
+                        part4[slot * D4 + c] =
+                            make_float4((float)acc[v][0], (float)acc[v][1], (float)acc[v][2], (float)acc[v][3]);
                 }
             }
         };
@@ -288,12 +296,17 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
                         seg_count = 0;
 #pragma unroll
                         for (int v = 0; v < NV; ++v) {
-                            acc[v] = f4_zero();
+                            acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0.0;
                             wrow[v] = wn[u][v];
                         }
                     }
 #pragma unroll
-                    for (int v = 0; v < NV; ++v) f4_add(acc[v], g[u][v]);
+                    for (int v = 0; v < NV; ++v) {
+                        acc[v][0] += (double)g[u][v].x;
+                        acc[v][1] += (double)g[u][v].y;
+                        acc[v][2] += (double)g[u][v].z;
+                        acc[v][3] += (double)g[u][v].w;
+                    }
                     ++seg_count;
                 }
             }

@@ -312,3 +312,162 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
     finally:
         p.close()
     return dict(shared_cold_rows=shared, steps=steps)
+
+
+def run_fullsize_check(spec, scale_rows: float = 1.0, n_samples: int = 1500, profile_batches=None,
+                       device: str = "cuda:0", verbose: bool = False):
+    """A workload too large for an element-by-element float comparison, run in the launch configuration the
+    benchmark times (Hotline.step, cold gather on the side stream).  Every integer result is compared in full
+    (hot set, perm, counts, both CSRs, cold rows, unified slots); float results are compared on sampled outputs
+    that the oracle's definitions give one by one: sampled pooled vectors, sampled updated hot rows, sampled
+    written-back cold rows, and sampled rows nobody touched (which must keep their bits).  The host table lives in
+    pinned memory and is filled on the device from the same counter hash the oracle evaluates row by row."""
+    import bench
+    import paper_2204_05436_b200 as hl
+
+    if isinstance(spec, str):
+        spec = gen.CONFIGS[spec]
+    geom = gen.make_geometry(spec, scale_rows)
+    T, D, S, B = geom.num_tables, geom.dim, geom.bags_per_sample, spec.batch
+    N = geom.total_rows
+    n_bags = T * B * S
+    P = spec.profile_batches if profile_batches is None else profile_batches
+    lr = spec.lr
+    max_nnz = max_nnz_of(spec, geom, B)
+    K = orc.hot_capacity(spec.hot_policy, N, D)
+    hot_cap = max(1, min(K, N))
+    staging_cap = max(1, min(N, max_nnz))
+    rng = np.random.default_rng(spec.seed + 4242)
+    rows_of = lambda g: gen.table_values(np.asarray(g, dtype=np.int64), D, spec.seed)   # noqa: E731
+
+    table = hl.host_table_tensor(N, D)
+    h = None
+    try:
+        bench.fill_table(table, D, spec.seed, torch.device(device))
+        probe = rng.integers(0, N, 64)
+        assert np.array_equal(table.numpy()[probe].view(np.uint32), rows_of(probe).view(np.uint32)), "table fill"
+        h = hl.Hotline(geom.table_rows, D, S, B, max_nnz, hot_cap, staging_cap, table, n_dense=spec.n_dense,
+                       device=device)
+        with torch.cuda.stream(h.main):
+            # ---- learning phase: full comparison ----
+            prof = [gen.make_batch(spec, geom, i) for i in range(P)]
+            cnt = orc.access_counts([(b.indices, b.offsets) for b in prof], B, geom.table_rows, S)
+            hot_o = orc.select_hot(cnt, min(K, hot_cap))
+            del cnt
+            pol, p_num, p_den = policy_args(spec.hot_policy)
+            for i, b in enumerate(prof):
+                h.profile(_t(b.indices, device), _t(b.offsets, device), B, reset=(i == 0))
+            h.profile(None, None, finalize=True, policy=pol, p_num=p_num, p_den=p_den)
+            h.build_remap(load_rows=True)
+            h.status()
+            n_hot = int(h.n_hot.item())
+            assert n_hot == len(hot_o), ("n_hot", n_hot, len(hot_o))
+            assert np.array_equal(h.hot_rows[:n_hot].cpu().numpy(), hot_o.astype(np.int32)), "hot rows"
+            remap_o = orc.build_remap(hot_o, N)
+            pick = rng.integers(0, n_hot, n_samples)
+            got = h.cache[torch.from_numpy(pick).to(device)].cpu().numpy()
+            assert np.array_equal(got.view(np.uint32), rows_of(hot_o[pick]).view(np.uint32)), "hot cache load"
+
+            # ---- one mini-batch through Hotline.step ----
+            batch = gen.make_batch(spec, geom, P)
+            grad = gen.grad_values(spec.seed, P, 2, n_bags, D)
+            perm_o, n_pop_o, O, X, dense_o = orc.fragment(batch.indices, batch.offsets, B, geom.table_rows, remap_o,
+                                                          S, batch.dense)
+            C, x_slots = orc.gather_cold(X.ids, remap_o, hot_cap)
+            n_non_o = B - n_pop_o
+            bags_pop, bags_non = T * n_pop_o * S, T * n_non_o * S
+            d_grad = _t(grad, device)
+            d_dense = _t(batch.dense, device) if batch.dense is not None else None
+            d_idx, d_off = _t(batch.indices, device), _t(batch.offsets, device)
+            torch.cuda.synchronize()
+            h.step(d_idx, d_off, B, d_grad, d_grad, lr, dense=d_dense)
+            h.status()
+            assert h.counts.cpu().tolist() == [n_pop_o, n_non_o, len(O.ids), len(X.ids)], "counts"
+            assert np.array_equal(h.perm[:B].cpu().numpy(), perm_o), "perm"
+            assert np.array_equal(h.pop_offsets[:bags_pop + 1].cpu().numpy(), O.offsets), "pop offsets"
+            assert np.array_equal(h.pop_ids[:len(O.ids)].cpu().numpy(), O.ids), "pop slots"
+            assert np.array_equal(h.non_offsets[:bags_non + 1].cpu().numpy(), X.offsets), "non offsets"
+            assert int(h.n_cold.item()) == len(C), "n_cold"
+            assert np.array_equal(h.cold_rows[:len(C)].cpu().numpy(), C.astype(np.int32)), "cold rows"
+            assert np.array_equal(h.non_ids[:len(X.ids)].cpu().numpy(), x_slots), "unified slots"
+            if dense_o is not None:
+                assert np.array_equal(h.dense_out[:B].cpu().numpy().view(np.uint32), dense_o.view(np.uint32)), "dense"
+
+            # ---- sampled float results ----
+            lr64 = float(np.float32(lr))
+
+            def slot_row_id(slots):   # global row behind a unified slot
+                slots = np.asarray(slots, dtype=np.int64)
+                return np.where(slots < hot_cap, hot_o[np.minimum(slots, n_hot - 1)], C[np.maximum(slots - hot_cap, 0)
+                                                                                        % max(1, len(C))])
+
+            def row_grad(ids, offsets, u):   # sum of grad rows of the bags whose lookups address slot u (fp64)
+                pos = np.flatnonzero(ids == u)
+                bags = np.searchsorted(offsets, pos, side="right") - 1
+                return grad[bags].astype(np.float64).sum(axis=0)
+
+            # rows after O's update (needed by X's forward): start from the initial values
+            o_ids64, x_ids64 = O.ids.astype(np.int64), x_slots.astype(np.int64)
+            touched_by_o = np.zeros(hot_cap + staging_cap, dtype=bool)
+            touched_by_o[o_ids64] = True
+
+            def value_after_o(slots):
+                base = rows_of(slot_row_id(slots))
+                out = base.copy()
+                for i, u in enumerate(np.asarray(slots)):
+                    if touched_by_o[u]:
+                        out[i] = (base[i].astype(np.float64) - lr64 * row_grad(O.ids, O.offsets, u)).astype(np.float32)
+                return out
+
+            def pooled_expect(ids, offsets, bags, value_fn):
+                out = np.zeros((len(bags), D), dtype=np.float32)
+                for i, bag in enumerate(bags):
+                    sl = ids[offsets[bag]:offsets[bag + 1]]
+                    out[i] = value_fn(sl).astype(np.float64).sum(axis=0).astype(np.float32) if len(sl) else 0.0
+                return out
+
+            n_s = max(8, n_samples // 8)
+            if bags_pop:
+                bags = rng.integers(0, bags_pop, n_s)
+                want = pooled_expect(O.ids, O.offsets, bags, lambda sl: rows_of(slot_row_id(sl)))
+                got = h.pooled_pop[torch.from_numpy(bags).to(device)].cpu().numpy()
+                assert_close(got, want, "sampled pooled_pop")
+            if bags_non:
+                bags = rng.integers(0, bags_non, n_s)
+                want = pooled_expect(x_slots, X.offsets, bags, value_after_o)
+                got = h.pooled_non[torch.from_numpy(bags).to(device)].cpu().numpy()
+                assert_close(got, want, "sampled pooled_non")
+            # updated rows: O's update then X's update, each rounded to fp32 as the oracle does step by step
+            cand = np.unique(np.concatenate([o_ids64[rng.integers(0, max(1, len(o_ids64)), n_s)] if len(o_ids64) else
+                                             np.zeros(0, np.int64),
+                                             x_ids64[rng.integers(0, max(1, len(x_ids64)), n_s)] if len(x_ids64) else
+                                             np.zeros(0, np.int64)]))
+            touched_by_x = np.zeros(hot_cap + staging_cap, dtype=bool)
+            touched_by_x[x_ids64] = True
+            want = value_after_o(cand)
+            for i, u in enumerate(cand):
+                if touched_by_x[u]:
+                    want[i] = (want[i].astype(np.float64) - lr64 * row_grad(x_slots, X.offsets, u)).astype(np.float32)
+            hot_part = cand < hot_cap
+            got_hot = h.cache[torch.from_numpy(cand[hot_part]).to(device)].cpu().numpy()
+            assert_close(got_hot, want[hot_part], "sampled updated hot rows")
+            cold_ids = C[cand[~hot_part] - hot_cap]
+            assert_close(table.numpy()[cold_ids], want[~hot_part], "sampled written-back cold rows")
+            assert not np.array_equal(want[hot_part], rows_of(slot_row_id(cand[hot_part]))), "update changed nothing"
+            # rows nobody touched keep their bits
+            idle = np.flatnonzero(~(touched_by_o[:n_hot] | touched_by_x[:n_hot]))
+            idle = idle[rng.integers(0, len(idle), min(n_samples, len(idle)))] if len(idle) else idle
+            got = h.cache[torch.from_numpy(idle).to(device)].cpu().numpy()
+            assert np.array_equal(got.view(np.uint32), rows_of(hot_o[idle]).view(np.uint32)), "idle hot rows"
+            far = rng.integers(0, N, n_samples)
+            far = far[(remap_o[far] < 0) & ~np.isin(far, C)]
+            assert np.array_equal(table.numpy()[far].view(np.uint32), rows_of(far).view(np.uint32)), "idle host rows"
+            stats = dict(n_pop=n_pop_o, n_non=n_non_o, n_cold=len(C), n_hot=n_hot, N=N, batch=B)
+            if verbose:
+                print(f"[{spec.name} full size] {stats}")
+            return stats
+    finally:
+        if h is not None:
+            h.close()
+        torch.cuda.synchronize()
+        hl.hl_host_free(table.data_ptr())

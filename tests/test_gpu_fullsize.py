@@ -1,0 +1,35 @@
+"""The named configurations at (or near) their full sizes, in the launch configuration bench.py times."""
+import dataclasses
+
+import pytest
+
+import gen
+from tests.harness import run_config_check, run_fullsize_check
+
+pytestmark = pytest.mark.gpu
+
+
+def test_dlrm_large_full_size_sampled():
+    """26 tables, 257.5 M rows x dim 64 (61 GiB pinned host table), batch 16,384: integer results in full,
+    float results on samples."""
+    stats = run_fullsize_check("dlrm_large")
+    assert stats["N"] > 250_000_000 and 0 < stats["n_pop"] < stats["batch"] and stats["n_cold"] > 1000
+
+
+def test_tbsm_full_size_every_element():
+    """3 tables (1 M, 4 M, 10 k rows), 21 time steps, batch 2,048, 64 MB budget: every output element."""
+    stats = run_config_check("tbsm", steps=1)
+    assert stats["N"] == 5_010_000
+
+
+def test_dlrm_small_full_size_every_element():
+    """26 tables, 33.8 M rows x dim 16, batch 4,096, 256 MB budget, 256 profiling batches: every output element."""
+    stats = run_config_check("dlrm_small", steps=1)
+    assert stats["N"] > 33_000_000 and stats["n_pop"] > 0
+
+
+def test_multi_hot_full_batch_sampled():
+    """8 tables x dim 128, Poisson(20) bags capped at 64, the full batch of 65,536 inputs (10.5 M lookups); row
+    counts cut to an eighth (2.5 M rows per table, 9.5 GiB host table) to keep the test's set-up short."""
+    stats = run_fullsize_check("multi_hot", scale_rows=0.125, n_samples=600)
+    assert stats["batch"] == 65536
