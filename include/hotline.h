@@ -158,6 +158,14 @@ HL_API int32_t hl_profile_hot(hl_ctx* ctx, const hl_batch* b, int32_t reset, int
 HL_API int32_t hl_build_remap(hl_ctx* ctx, const int32_t* d_hot_rows, const int64_t* d_n_hot,
                        const float* host_table, float* d_cache, int32_t* d_remap_out, void* stream);
 
+/* Section V-B (the logger periodically returns to its learning phase to follow changes in popularity) and
+ * Section IV (popular rows live in GPU memory only): before a new popular set replaces the current one, the
+ * current values of the popular rows go back to the host table:
+ * host_table[d_hot_rows[i], :] = cache[i, :] for i < *d_n_hot.  Afterwards the host table holds every row's
+ * current value (a consistent snapshot), and hl_profile_hot / hl_build_remap may install another set. */
+HL_API int32_t hl_flush_hot(hl_ctx* ctx, const float* d_cache, const int32_t* d_hot_rows, const int64_t* d_n_hot,
+                            float* host_table, void* stream);
+
 /* ---------------------------------------------------------------------------------------------------------
  * Acceleration phase
  * ------------------------------------------------------------------------------------------------------- */

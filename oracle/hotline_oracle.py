@@ -192,6 +192,14 @@ def scatter_cold(table: np.ndarray, C: np.ndarray, staging: np.ndarray) -> None:
     table[np.asarray(C, dtype=np.int64)] = staging[: len(C)]
 
 
+def flush_hot(table: np.ndarray, cache: np.ndarray, hot_rows: np.ndarray) -> None:
+    """table[hot_rows[i], :] = cache[i, :]: before the popular set is re-learned (the logger periodically goes
+    back to its learning phase, Section V-B), the popular rows' current values return to CPU memory, the only
+    place that holds every row."""
+    hot_rows = np.asarray(hot_rows, dtype=np.int64)
+    table[hot_rows] = cache[: len(hot_rows)]
+
+
 # ----------------------------------------------------------------------------------------------------------
 # embedding bag: sum pooling forward (the Reducer, Section V-D) and scatter-add + SGD backward
 # ----------------------------------------------------------------------------------------------------------

@@ -19,7 +19,7 @@ EXPORTS = (
     "hl_workspace_bytes", "hl_create", "hl_destroy", "hl_status", "hl_strerror", "hl_launch_count", "hl_timing_enable", "hl_timing_read", "hl_host_alloc",
     "hl_host_free", "hl_profile_hot",
     "hl_build_remap", "hl_fragment", "hl_embbag_fwd", "hl_embbag_bwd_sgd", "hl_gather_cold", "hl_scatter_cold",
-    "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at",
+    "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at", "hl_flush_hot",
 )
 
 
@@ -93,6 +93,8 @@ def _load() -> ctypes.CDLL:
     lib.hl_forward_cold.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     lib.hl_scatter_cold_at.restype = i32
     lib.hl_scatter_cold_at.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
+    lib.hl_flush_hot.restype = i32
+    lib.hl_flush_hot.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.hl_embbag_bwd_sgd_static.restype = i32
     lib.hl_embbag_bwd_sgd_static.argtypes = [vp, i64, i32, vp, vp, i32, i64, vp, ctypes.c_float, vp, vp]
     return lib
@@ -285,3 +287,8 @@ def hl_scatter_cold_at(ctx: int, d_cache, stage_row0: int, stage_rows: int, d_co
                        stream: int) -> None:
     _check("hl_scatter_cold_at", _lib.hl_scatter_cold_at(ctx, _ptr(d_cache), int(stage_row0), int(stage_rows),
                                                          _ptr(d_cold_rows), _ptr(d_n_cold), _ptr(host_table), stream))
+
+
+def hl_flush_hot(ctx: int, d_cache, d_hot_rows, d_n_hot, host_table, stream: int) -> None:
+    _check("hl_flush_hot", _lib.hl_flush_hot(ctx, _ptr(d_cache), _ptr(d_hot_rows), _ptr(d_n_hot), _ptr(host_table),
+                                             stream))

@@ -471,3 +471,11 @@ extern "C" int32_t hl_scatter_cold(hl_ctx* ctx, const float* d_cache, const int3
     if (!ctx) return HL_EINVAL;
     return hl_scatter_cold_at(ctx, d_cache, 0, ctx->staging_cap, d_cold_rows, d_n_cold, host_table, stream_);
 }
+
+extern "C" int32_t hl_flush_hot(hl_ctx* ctx, const float* d_cache, const int32_t* d_hot_rows, const int64_t* d_n_hot,
+                                float* host_table, void* stream_) {
+    if (!ctx || !d_cache || !d_hot_rows || !d_n_hot || !host_table) return HL_EINVAL;
+    // runs between learning phases, with nothing else on the chip: the mover at the link's full rate
+    return launch_move_rows<true>(const_cast<float*>(d_cache), 0, host_table, d_hot_rows, d_n_hot, ctx->hot_cap, ctx->N,
+                                  ctx->D, nullptr, 2 * kSMs, ctx->r.status, static_cast<cudaStream_t>(stream_));
+}

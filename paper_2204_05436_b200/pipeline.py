@@ -112,6 +112,10 @@ class Hotline:
         B.hl_build_remap(self.ctx, self.hot_rows, self.n_hot, self.host_table if load_rows else None, self.cache,
                          remap_out, self.main.cuda_stream)
 
+    def flush_hot(self) -> None:
+        """Writes the popular rows' current values back to the host table (do this before re-learning the set)."""
+        B.hl_flush_hot(self.ctx, self.cache, self.hot_rows, self.n_hot, self.host_table, self.main.cuda_stream)
+
     # ---- acceleration phase: single calls ---------------------------------------------------------------------
     def fragment(self, indices, offsets, batch: int, dense: Optional[torch.Tensor] = None) -> None:
         B.hl_fragment(self.ctx, self._batch(indices, offsets, batch), dense, self.n_dense if dense is not None else 0,

@@ -471,3 +471,65 @@ def run_fullsize_check(spec, scale_rows: float = 1.0, n_samples: int = 1500, pro
             h.close()
         torch.cuda.synchronize()
         hl.hl_host_free(table.data_ptr())
+
+
+def run_recalibration_check(spec, steps_per_phase: int = 2, device: str = "cuda:0"):
+    """Learning phase, some mini-batches, flush of the popular rows, a second learning phase over a later window of
+    mini-batches (another popular set), more mini-batches, flush: after each flush the host table must equal the
+    oracle's table.  Integer data, so every comparison is exact."""
+    import paper_2204_05436_b200 as hl
+
+    if isinstance(spec, str):
+        spec = gen.CONFIGS[spec]
+    geom = gen.make_geometry(spec)
+    T, D, S, B = geom.num_tables, geom.dim, geom.bags_per_sample, spec.batch
+    N, n_bags, P, lr = geom.total_rows, T * B * S, spec.profile_batches, 0.125
+    max_nnz = max_nnz_of(spec, geom, B)
+    K = orc.hot_capacity(spec.hot_policy, N, D)
+    hot_cap, staging_cap = max(1, min(K, N)), max(1, min(N, max_nnz))
+    table_o = gen.table_values(np.arange(N), D, spec.seed, integer=True)
+    host_table = torch.from_numpy(table_o.copy()).pin_memory()
+    h = hl.Hotline(geom.table_rows, D, S, B, max_nnz, hot_cap, staging_cap, host_table, device=device)
+    pol, p_num, p_den = policy_args(spec.hot_policy)
+    hot_sets = []
+    try:
+        with torch.cuda.stream(h.main):
+            next_batch = 0
+            for phase in range(2):
+                # learning phase over the next P mini-batches, scaled differently per phase so the sets differ
+                prof = [gen.make_batch(spec, geom, next_batch + i) for i in range(P if phase == 0 else max(1, P // 3))]
+                next_batch += len(prof)
+                cnt = orc.access_counts([(b.indices, b.offsets) for b in prof], B, geom.table_rows, S)
+                hot_o = orc.select_hot(cnt, min(K, hot_cap))
+                hot_sets.append(hot_o)
+                remap_o = orc.build_remap(hot_o, N)
+                cache_o = np.zeros((hot_cap + staging_cap, D), dtype=np.float32)
+                cache_o[:len(hot_o)] = orc.load_hot_cache(table_o, hot_o)
+                for i, b in enumerate(prof):
+                    h.profile(_t(b.indices, device), _t(b.offsets, device), B, reset=(i == 0))
+                h.profile(None, None, finalize=True, policy=pol, p_num=p_num, p_den=p_den)
+                h.build_remap(load_rows=True)
+                h.status()
+                assert np.array_equal(h.hot_rows[:len(hot_o)].cpu().numpy(), hot_o.astype(np.int32)), ("hot", phase)
+                for step in range(steps_per_phase):
+                    batch = gen.make_batch(spec, geom, next_batch)
+                    grad_full = gen.grad_values(spec.seed, next_batch, 2, n_bags, D, integer=True)
+                    next_batch += 1
+                    perm_o, n_pop_o, _, _, _ = orc.fragment(batch.indices, batch.offsets, B, geom.table_rows, remap_o, S)
+                    g_pop, _ = mu_grad(grad_full, perm_o[:n_pop_o], T, B, S)
+                    g_non, _ = mu_grad(grad_full, perm_o[n_pop_o:], T, B, S)
+                    orc.hotline_step(table_o, cache_o, hot_cap, remap_o, batch.indices, batch.offsets, B,
+                                     geom.table_rows, S, g_pop, g_non, lr)
+                    gp = torch.zeros((n_bags, D), dtype=torch.float32, device=device)
+                    gn = torch.zeros((n_bags, D), dtype=torch.float32, device=device)
+                    gp[:len(g_pop)] = _t(g_pop, device)
+                    gn[:len(g_non)] = _t(g_non, device)
+                    h.step(_t(batch.indices, device), _t(batch.offsets, device), B, gp, gn, lr)
+                    h.status()
+                orc.flush_hot(table_o, cache_o, hot_o)
+                h.flush_hot()
+                h.status()
+                assert np.array_equal(h.host_table.numpy(), table_o), ("host table after flush", phase)
+    finally:
+        h.close()
+    return dict(hot_sets_differ=not np.array_equal(hot_sets[0], hot_sets[1]), n_hot=[len(x) for x in hot_sets])

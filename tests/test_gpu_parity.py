@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import gen
-from tests.harness import run_config_check, run_pipelined_check
+from tests.harness import run_config_check, run_pipelined_check, run_recalibration_check
 
 pytestmark = pytest.mark.gpu
 
@@ -112,3 +112,9 @@ def test_pipelined_multi_hot_integer_data():
                                hot_policy=("fraction", 40, 100), profile_batches=2)
     stats = run_pipelined_check(spec, steps=5, integer=True)
     assert stats["shared_cold_rows"] > 100
+
+
+def test_flush_and_second_learning_phase():
+    """Re-calibration: flush the popular rows, learn another popular set from later mini-batches, carry on."""
+    stats = run_recalibration_check("tiny")
+    assert stats["hot_sets_differ"]

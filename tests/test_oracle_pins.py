@@ -507,3 +507,17 @@ def test_input_record_size_matches_the_papers_buffer_sizing():
     per_input = int(2.5 * 2 ** 20) // (16 * 1024)
     assert per_input == 160 == 26 * 4 + 13 * 4 + 4
     assert gen.make_batch(gen.CONFIGS["tiny"], gen.make_geometry(gen.CONFIGS["tiny"]), 0).indices.itemsize == 4
+
+
+def test_flush_hot_gives_a_consistent_table():
+    rng = np.random.default_rng(71)
+    table = rng.standard_normal((30, 3)).astype(np.float32)
+    hot = np.array([2, 5, 11, 29])
+    cache = np.zeros((6, 3), dtype=np.float32)
+    cache[:4] = orc.load_hot_cache(table, hot) + 1.0          # the cache moved on; the host copies are stale
+    cache[4:] = 99.0                                          # unused slots and staging must not leak
+    before = table.copy()
+    orc.flush_hot(table, cache, hot)
+    assert np.array_equal(table[hot], before[hot] + 1.0)
+    rest = np.setdiff1d(np.arange(30), hot)
+    assert np.array_equal(table[rest].view(np.uint32), before[rest].view(np.uint32))
