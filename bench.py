@@ -298,10 +298,10 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
     n_batches = 8
     wl = Workload(name, scale, n_batches, args.profile_batches, device, args.threads)
     T, D, S, B = wl.T, wl.D, wl.S, wl.B
-    pipelined = args.pipeline
+    pipelined = not args.no_pipeline
     if pipelined:
         h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
-                                n_dense=wl.spec.n_dense, device=str(device))
+                                n_dense=wl.spec.n_dense, device=str(device), overlap_link=args.overlap_link)
     else:
         h = hl.Hotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
                        n_dense=wl.spec.n_dense, device=str(device))
@@ -487,22 +487,32 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         breakdown = {k: round(mean_us(k), 2) for k in timers}
         used = [sizes[(first_timed + i) % n_batches] for i in range(args.steps)]
         mean = lambda key: sum(u[key] for u in used) / len(used)   # noqa: E731
-        # roofline of the popular micro-batch's embedding-bag forward (one kernel per call): per lookup a row
-        # (4*D bytes) and its slot (4 bytes) are read, per bag a pooled row (4*D) is written and an offset read.
+        # roofline of the embedding-bag forward (one kernel per call): per lookup a row (4*D bytes) and its slot
+        # (4 bytes) are read, per bag a pooled row (4*D) is written and an offset read.  Of the two launches per
+        # mini-batch the one over the non-popular micro-batch is reported: it is the larger one here, and in the
+        # pipelined schedule it runs with the chip to itself, while the popular one shares it on purpose with the
+        # host reads and the next mini-batch's fragment (its contended time is given beside it).
         bags_pop = T * mean("n_pop") * S
-        fwd_bytes = mean("L_pop") * (4 * D + 4) + bags_pop * (4 * D + 4)
-        fwd_us = mean_us("fwd_pop")
+        bags_non = T * mean("n_non") * S
+        pop_bytes = mean("L_pop") * (4 * D + 4) + bags_pop * (4 * D + 4)
+        pop_us = mean_us("fwd_pop")
+        fwd_bytes = mean("L_non") * (4 * D + 4) + bags_non * (4 * D + 4)
+        fwd_us = mean_us("fwd_non")
         peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
         if os.path.exists(peaks_path):
             peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
         else:
             peak, peak_src = FALLBACK_HBM_GBS, "fallback"
         achieved = fwd_bytes / (fwd_us * 1e-6) / 1e9 if fwd_us > 0 else 0.0
-        roofline = {"kernel": "k_embbag_fwd (popular micro-batch)", "bound": "hbm", "achieved": achieved,
+        roofline = {"kernel": "k_embbag_fwd (non-popular micro-batch: hot rows + staged rows, all in HBM)",
+                    "bound": "hbm", "achieved": achieved,
                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                    "traffic": (NCU_FWD_TRAFFIC_BYTES_PER_BAG[D] * bags_pop if D in NCU_FWD_TRAFFIC_BYTES_PER_BAG else None),
+                    "traffic": (NCU_FWD_TRAFFIC_BYTES_PER_BAG[D] * bags_non if D in NCU_FWD_TRAFFIC_BYTES_PER_BAG else None),
                     "traffic_source": "ncu capture of the hot-only micro case, scaled by bags", "algorithmic_bytes_per_launch": fwd_bytes,
-                    "us_per_launch": fwd_us}
+                    "us_per_launch": fwd_us,
+                    "popular_launch": {"algorithmic_bytes_per_launch": pop_bytes, "us_per_launch": pop_us,
+                                       "achieved": pop_bytes / (pop_us * 1e-6) / 1e9 if pop_us > 0 else 0.0,
+                                       "frac": (pop_bytes / (pop_us * 1e-6) / 1e9 / peak) if pop_us > 0 else 0.0}}
         link_us = mean_us("gather_cold")
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -516,8 +526,9 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                              f"({(2 * wl.n_bags * D * 4 + fwd_bytes) / 2**20:.0f} MB of pooled vectors, gradients and rows)"
                              if 2 * wl.n_bags * D * 4 > L2_BYTES else
                              "per-step working set is smaller than L2 on this workload; batches rotate over 8 buffers",
-                       "schedule": ("software-pipelined across mini-batches (PipelinedHotline)" if pipelined else
-                                    "one mini-batch after the other (Hotline.step)"),
+                       "schedule": ("software-pipelined across mini-batches (PipelinedHotline"
+                                    + (", overlapping host reads and write-backs)" if args.overlap_link else ")")
+                                    if pipelined else "one mini-batch after the other (Hotline.step)"),
                        "replicas": "independent replica per GPU, no collective"},
             "clocks": clock_info, "gpu_launches": int(launches),
             "launches_per_step": launches / args.steps, "breakdown_us": breakdown, "roofline": roofline,
@@ -677,10 +688,12 @@ def main() -> None:
     ap.add_argument("--profile-batches", type=int, default=None)
     ap.add_argument("--threads", type=int, default=min(16, os.cpu_count() or 1))
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--pipeline", action="store_true",
-                    help="software-pipeline the mini-batches (PipelinedHotline) instead of running one after the "
-                         "other (Hotline.step); kernels of different mini-batches then overlap, so the per-call "
-                         "times no longer describe a kernel running alone")
+    ap.add_argument("--no-pipeline", action="store_true",
+                    help="run one mini-batch after the other (Hotline.step) instead of the software pipeline "
+                         "(PipelinedHotline), in which the next mini-batch's fragment, cold-row search and host reads "
+                         "run under this one's execution")
+    ap.add_argument("--overlap-link", action="store_true",
+                    help="pipeline variant that also overlaps host reads with write-backs (forwarding shared rows)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather"],
                     help="time one library call in isolation")

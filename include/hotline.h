@@ -236,6 +236,21 @@ HL_API int32_t hl_gather_cold_ahead(hl_ctx* ctx, hl_ubatch* non, const int32_t* 
                                     int32_t* d_fwd_src, void* record_after_index, void* wait_before_move_a,
                                     void* wait_before_move_b, void* stream);
 
+/* The two halves of hl_gather_cold_ahead as separate calls, so that they can go to different streams: hl_index_cold
+ * does everything up to and including d_cold_rows, *d_n_cold, d_fwd_src and the unified slots in non->ids (device
+ * work only; scratch: the cold region); hl_stage_cold then reads the host rows into the staging window (rows with
+ * d_fwd_src[i] >= 0 are left out; d_fwd_src may be NULL).  Issue hl_stage_cold on the stream that also carries the
+ * write-backs: stream order then puts the read behind the previous write-back without a stream sitting in an event
+ * wait while rows move over the link (on the bench platform a stream blocked in such a wait slowed the write-back
+ * running next to it by a factor of five). */
+HL_API int32_t hl_index_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, int64_t stage_row0,
+                             int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold,
+                             const int32_t* d_prev_cold_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
+                             void* stream);
+HL_API int32_t hl_stage_cold(hl_ctx* ctx, const float* host_table, float* d_cache, int64_t stage_row0,
+                             int64_t stage_rows, const int32_t* d_cold_rows, const int64_t* d_n_cold,
+                             const int32_t* d_fwd_src, void* stream);
+
 /* cache[hot_cap + to_stage_row0 + i, :] = cache[hot_cap + from_stage_row0 + d_fwd_src[i], :] for every
  * i < *d_n_cold with d_fwd_src[i] >= 0 (device-to-device; run it after the earlier mini-batch's backward). */
 HL_API int32_t hl_forward_cold(hl_ctx* ctx, float* d_cache, int64_t from_stage_row0, int64_t to_stage_row0,

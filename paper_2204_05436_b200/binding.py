@@ -19,7 +19,7 @@ EXPORTS = (
     "hl_workspace_bytes", "hl_create", "hl_destroy", "hl_status", "hl_strerror", "hl_launch_count", "hl_timing_enable", "hl_timing_read", "hl_host_alloc",
     "hl_host_free", "hl_profile_hot",
     "hl_build_remap", "hl_fragment", "hl_embbag_fwd", "hl_embbag_bwd_sgd", "hl_gather_cold", "hl_scatter_cold",
-    "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at", "hl_flush_hot",
+    "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at", "hl_flush_hot", "hl_index_cold", "hl_stage_cold",
 )
 
 
@@ -93,6 +93,10 @@ def _load() -> ctypes.CDLL:
     lib.hl_forward_cold.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     lib.hl_scatter_cold_at.restype = i32
     lib.hl_scatter_cold_at.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
+    lib.hl_index_cold.restype = i32
+    lib.hl_index_cold.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, i64, i64, vp, vp, vp, vp, vp, vp]
+    lib.hl_stage_cold.restype = i32
+    lib.hl_stage_cold.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp, vp]
     lib.hl_flush_hot.restype = i32
     lib.hl_flush_hot.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.hl_embbag_bwd_sgd_static.restype = i32
@@ -292,3 +296,16 @@ def hl_scatter_cold_at(ctx: int, d_cache, stage_row0: int, stage_rows: int, d_co
 def hl_flush_hot(ctx: int, d_cache, d_hot_rows, d_n_hot, host_table, stream: int) -> None:
     _check("hl_flush_hot", _lib.hl_flush_hot(ctx, _ptr(d_cache), _ptr(d_hot_rows), _ptr(d_n_hot), _ptr(host_table),
                                              stream))
+
+
+def hl_index_cold(ctx: int, non: hl_ubatch, d_n_non, stage_row0: int, stage_rows: int, d_cold_rows, d_n_cold,
+                  d_prev_cold_rows, d_n_prev, d_fwd_src, stream: int) -> None:
+    _check("hl_index_cold", _lib.hl_index_cold(ctx, ctypes.byref(non), _ptr(d_n_non), int(stage_row0), int(stage_rows),
+                                               _ptr(d_cold_rows), _ptr(d_n_cold), _ptr(d_prev_cold_rows), _ptr(d_n_prev),
+                                               _ptr(d_fwd_src), stream))
+
+
+def hl_stage_cold(ctx: int, host_table, d_cache, stage_row0: int, stage_rows: int, d_cold_rows, d_n_cold, d_fwd_src,
+                  stream: int) -> None:
+    _check("hl_stage_cold", _lib.hl_stage_cold(ctx, _ptr(host_table), _ptr(d_cache), int(stage_row0), int(stage_rows),
+                                               _ptr(d_cold_rows), _ptr(d_n_cold), _ptr(d_fwd_src), stream))

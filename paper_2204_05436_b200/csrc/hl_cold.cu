@@ -357,8 +357,18 @@ namespace {
 int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const float* host_table, float* d_cache,
                     int64_t stage_row0, int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold,
                     const int32_t* d_prev_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
-                    cudaEvent_t record_after_index, cudaEvent_t wait_a, cudaEvent_t wait_b, cudaStream_t stream) {
+                    cudaEvent_t record_after_index, cudaEvent_t wait_a, cudaEvent_t wait_b, bool do_index,
+                    bool do_move, cudaStream_t stream) {
     Regions& r = ctx->r;
+    if (!do_index) {
+        if (ctx->max_nnz == 0) return HL_OK;
+        timer_mark(ctx, HL_TIMER_GATHER_MOVE, 0, stream);
+        const int32_t st = launch_move_rows<false>(d_cache, ctx->hot_cap + stage_row0,
+                                                   const_cast<float*>(host_table), d_cold_rows, d_n_cold, stage_rows,
+                                                   ctx->N, ctx->D, d_fwd_src, kBulkCtas, r.status, stream);
+        timer_mark(ctx, HL_TIMER_GATHER_MOVE, 1, stream);
+        return st;
+    }
     if (ctx->max_nnz == 0) {
         HL_CUDA_TRY(cudaMemsetAsync(d_n_cold, 0, sizeof(int64_t), stream));
         if (record_after_index) HL_CUDA_TRY(cudaEventRecord(record_after_index, stream));
@@ -393,6 +403,7 @@ int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const f
         HL_LAUNCH_CHECK();
     }
     if (record_after_index) HL_CUDA_TRY(cudaEventRecord(record_after_index, stream));
+    if (!do_move) return HL_OK;
     if (wait_a) HL_CUDA_TRY(cudaStreamWaitEvent(stream, wait_a, 0));
     if (wait_b) HL_CUDA_TRY(cudaStreamWaitEvent(stream, wait_b, 0));
     timer_mark(ctx, HL_TIMER_GATHER_MOVE, 0, stream);
@@ -415,7 +426,7 @@ extern "C" int32_t hl_gather_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_
     if (!ctx || !non || !non->offsets || !d_n_non || !host_table || !d_cache || !d_cold_rows || !d_n_cold)
         return HL_EINVAL;
     return gather_impl(ctx, non, d_n_non, host_table, d_cache, 0, ctx->staging_cap, d_cold_rows, d_n_cold, nullptr,
-                       nullptr, nullptr, nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream_));
+                       nullptr, nullptr, nullptr, nullptr, nullptr, true, true, static_cast<cudaStream_t>(stream_));
 }
 
 extern "C" int32_t hl_gather_cold_ahead(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const float* host_table,
@@ -429,7 +440,30 @@ extern "C" int32_t hl_gather_cold_ahead(hl_ctx* ctx, hl_ubatch* non, const int32
     if ((d_prev_cold_rows != nullptr) != (d_n_prev != nullptr) || (d_prev_cold_rows && !d_fwd_src)) return HL_EINVAL;
     return gather_impl(ctx, non, d_n_non, host_table, d_cache, stage_row0, stage_rows, d_cold_rows, d_n_cold,
                        d_prev_cold_rows, d_n_prev, d_fwd_src, static_cast<cudaEvent_t>(record_after_index),
-                       static_cast<cudaEvent_t>(wait_before_move_a), static_cast<cudaEvent_t>(wait_before_move_b),
+                       static_cast<cudaEvent_t>(wait_before_move_a), static_cast<cudaEvent_t>(wait_before_move_b), true,
+                       true, static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int32_t hl_index_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, int64_t stage_row0,
+                                 int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold,
+                                 const int32_t* d_prev_cold_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
+                                 void* stream_) {
+    if (!ctx || !non || !non->offsets || !d_n_non || !d_cold_rows || !d_n_cold) return HL_EINVAL;
+    if (!window_ok(ctx, stage_row0, stage_rows)) return HL_EINVAL;
+    if ((d_prev_cold_rows != nullptr) != (d_n_prev != nullptr) || (d_prev_cold_rows && !d_fwd_src)) return HL_EINVAL;
+    return gather_impl(ctx, non, d_n_non, nullptr, nullptr, stage_row0, stage_rows, d_cold_rows, d_n_cold,
+                       d_prev_cold_rows, d_n_prev, d_fwd_src, nullptr, nullptr, nullptr, true, false,
+                       static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int32_t hl_stage_cold(hl_ctx* ctx, const float* host_table, float* d_cache, int64_t stage_row0,
+                                 int64_t stage_rows, const int32_t* d_cold_rows, const int64_t* d_n_cold,
+                                 const int32_t* d_fwd_src, void* stream_) {
+    if (!ctx || !host_table || !d_cache || !d_cold_rows || !d_n_cold) return HL_EINVAL;
+    if (!window_ok(ctx, stage_row0, stage_rows)) return HL_EINVAL;
+    return gather_impl(ctx, nullptr, nullptr, host_table, d_cache, stage_row0, stage_rows,
+                       const_cast<int32_t*>(d_cold_rows), const_cast<int64_t*>(d_n_cold), nullptr, nullptr,
+                       const_cast<int32_t*>(d_fwd_src), nullptr, nullptr, nullptr, false, true,
                        static_cast<cudaStream_t>(stream_));
 }
 

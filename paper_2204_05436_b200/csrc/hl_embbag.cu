@@ -324,7 +324,7 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
                                                         const int32_t* __restrict__ d_n_lookups, int D4,
                                                         int64_t n_slots, float lr, const float* __restrict__ part) {
     constexpr int GW = 32 / G;   // groups per warp
-    constexpr int U = NV >= 4 ? 1 : (NV >= 2 ? 2 : 4);
+    constexpr int U = NV >= 8 ? 2 : (NV >= 4 ? 4 : (NV >= 2 ? 8 : 16));   // partial sums in flight per lane
     const int64_t n = d_n_lookups[0];
     const int lane = threadIdx.x & 31;
     const int sub = lane % G, gi = lane / G;

@@ -208,18 +208,30 @@ __global__ void __launch_bounds__(kThreads) k_sort_pass(const int32_t* __restric
     uint32_t* my = tstat + tile * 256 + d;
     if (tile > 0) {
         st_relaxed(my, kFlagAgg | total);
-        for (int64_t t = tile - 1; t >= 0; --t) {
-            uint32_t w = 0;
-            int polls = 0;
-            while (((w = ld_relaxed(tstat + t * 256 + d)) & (kFlagAgg | kFlagPrefix)) == 0) {
-                if (++polls > kMaxPolls) {
-                    set_status(status, HL_ETIMEOUT);
-                    break;
+        // walk back kLook tiles at a time: the kLook status words are requested together, then consumed from the
+        // nearest tile outwards until one of them already carries an inclusive prefix
+        constexpr int kLook = 8;
+        bool found = false, gave_up = false;
+        for (int64_t t0 = tile - 1; t0 >= 0 && !found && !gave_up; t0 -= kLook) {
+            uint32_t w[kLook];
+#pragma unroll
+            for (int k = 0; k < kLook; ++k) w[k] = t0 - k >= 0 ? ld_relaxed(tstat + (t0 - k) * 256 + d) : kFlagPrefix;
+#pragma unroll
+            for (int k = 0; k < kLook; ++k) {
+                if (found || gave_up) break;
+                int polls = 0;
+                while ((w[k] & (kFlagAgg | kFlagPrefix)) == 0) {
+                    if (++polls > kMaxPolls) {
+                        set_status(status, HL_ETIMEOUT);
+                        gave_up = true;
+                        break;
+                    }
+                    __nanosleep(20);
+                    w[k] = ld_relaxed(tstat + (t0 - k) * 256 + d);
                 }
-                __nanosleep(20);
+                before += w[k] & kValueMask;
+                found = (w[k] & kFlagPrefix) != 0;
             }
-            before += w & kValueMask;
-            if ((w & kFlagPrefix) || polls > kMaxPolls) break;
         }
     }
     st_relaxed(my, kFlagPrefix | ((before + total) & kValueMask));

@@ -212,7 +212,8 @@ class _BatchSet:
         self.ev_forward = torch.cuda.Event()
         self.ev_x = torch.cuda.Event()
         self.ev_scatter = torch.cuda.Event()
-        for e in (self.ev_index, self.ev_gather, self.ev_forward, self.ev_x, self.ev_scatter):
+        self.ev_inputs = torch.cuda.Event()
+        for e in (self.ev_index, self.ev_gather, self.ev_forward, self.ev_x, self.ev_scatter, self.ev_inputs):
             e.record(h.main)
 
 
@@ -225,6 +226,13 @@ class PipelinedHotline(Hotline):
 
     Three sets of index buffers rotate over the mini-batches, two windows of the staging area alternate.
 
+    ``overlap_link=False`` (default): the host rows of mini-batch j+1 are read after mini-batch j's write-back has
+    finished, so the two transfers follow each other on the link and no forwarding is needed; fragment and the
+    search for the distinct cold rows of j+1 still run under j's execution.  ``overlap_link=True``: the read of
+    j+1 starts as soon as j-1's write-back is done and overlaps j's execution and write-back, with shared rows
+    forwarded between the staging windows (on a platform where random host rows are bound by address translation
+    the two transfers then compete and nothing is gained).
+
         p.start(idx0, off0, B)                       # ahead-work of mini-batch 0
         for j in range(n):
             s = p.step(grad_pop, grad_non, lr, next_batch=(idx, off, B, dense) or None)
@@ -233,14 +241,14 @@ class PipelinedHotline(Hotline):
     """
 
     def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
-                 n_dense: int = 0, device: str = "cuda:0"):
+                 n_dense: int = 0, device: str = "cuda:0", overlap_link: bool = False):
+        self.overlap_link = bool(overlap_link)
         self.window_rows = int(window_rows)
         super().__init__(table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, 2 * self.window_rows,
                          host_table, n_dense=n_dense, device=device)
         self.sets = [_BatchSet(self) for _ in range(3)]
         self.sides = [self.side, torch.cuda.Stream(device=self.device)]
         self.wb = torch.cuda.Stream(device=self.device)
-        self._ev_inputs = torch.cuda.Event()
         self.j_submitted = 0      # mini-batches whose ahead-work has been issued
         self.j_done = 0           # mini-batches whose main work has been issued
         torch.cuda.synchronize(self.device)
@@ -259,29 +267,52 @@ class PipelinedHotline(Hotline):
     def _submit(self, indices, offsets, batch: int, dense=None, timers=None) -> None:
         j = self.j_submitted
         st, side = self.sets[j % 3], self.sides[j % 2]
-        self._ev_inputs.record(self.main)                # the caller prepared the inputs on the main stream
-        side.wait_event(self._ev_inputs)
+        side.wait_event(st.ev_inputs)                    # the caller prepared the inputs on the main stream
         if j >= 3:
             side.wait_event(st.ev_scatter)               # set j%3 was mini-batch j-3's: long done, stated anyway
         prev = self.sets[(j - 1) % 3] if j >= 1 else None
         if prev is not None:
             side.wait_event(prev.ev_index)               # its cold set is final; fragment/cold scratch is free
+        if self.overlap_link:
+            excl = prev
+            wait_a = self.sets[(j - 2) % 3].ev_scatter if j >= 2 else None   # host rows of j-2 are final
+            wait_b = prev.ev_forward if prev is not None else None           # j-1 took what it needs from the window
+        else:
+            excl = None
+            wait_a = wait_b = None
+            if j >= 2:
+                # Keep this mini-batch's fragment / index kernels away from the write-back of mini-batch j-2: they
+                # then run next to the read of j-1's host rows instead.  (Measured: a write-back that shares the
+                # chip with them takes 650-870 us instead of 125 us; the read, which pays an address-translation
+                # miss per row anyway, does not care.)
+                side.wait_event(self.sets[(j - 2) % 3].ev_scatter)
         self._timed(timers, "fragment", side, lambda: B.hl_fragment(
             self.ctx, self._batch(indices, offsets, batch), dense, self.n_dense if dense is not None else 0,
             st.perm, st.counts, st.pop, st.non, st.dense_out if dense is not None else None, side.cuda_stream))
-        self._timed(timers, "gather_cold", side, lambda: B.hl_gather_cold_ahead(
-            self.ctx, st.non, st.counts[1:], self.host_table, self.cache, (j % 2) * self.window_rows,
-            self.window_rows, st.cold_rows, st.n_cold,
-            prev.cold_rows if prev is not None else None, prev.n_cold if prev is not None else None, st.fwd_src,
-            st.ev_index,
-            self.sets[(j - 2) % 3].ev_scatter if j >= 2 else None,     # host rows of j-2 are final after its write-back
-            prev.ev_forward if prev is not None else None,             # j-1 has copied what it needs out of this window
-            side.cuda_stream))
-        st.ev_gather.record(side)
+        if self.overlap_link:
+            self._timed(timers, "gather_cold", side, lambda: B.hl_gather_cold_ahead(
+                self.ctx, st.non, st.counts[1:], self.host_table, self.cache, (j % 2) * self.window_rows,
+                self.window_rows, st.cold_rows, st.n_cold,
+                excl.cold_rows if excl is not None else None, excl.n_cold if excl is not None else None, st.fwd_src,
+                st.ev_index, wait_a, wait_b, side.cuda_stream))
+            st.ev_gather.record(side)
+        else:
+            # index work on the side stream; the read of the host rows on the write-back stream, behind the
+            # write-back of the mini-batch before (stream order, no stream parked in an event wait meanwhile)
+            self._timed(timers, "index_cold", side, lambda: B.hl_index_cold(
+                self.ctx, st.non, st.counts[1:], (j % 2) * self.window_rows, self.window_rows, st.cold_rows,
+                st.n_cold, None, None, None, side.cuda_stream))
+            st.ev_index.record(side)
+            self.wb.wait_event(st.ev_index)
+            self._timed(timers, "gather_cold", self.wb, lambda: B.hl_stage_cold(
+                self.ctx, self.host_table, self.cache, (j % 2) * self.window_rows, self.window_rows, st.cold_rows,
+                st.n_cold, None, self.wb.cuda_stream))
+            st.ev_gather.record(self.wb)
         self.j_submitted += 1
 
     def start(self, indices, offsets, batch: int, dense=None) -> None:
         assert self.j_submitted == self.j_done, "start() only with nothing in flight"
+        self.sets[self.j_submitted % 3].ev_inputs.record(self.main)
         self._submit(indices, offsets, batch, dense)
 
     def step(self, grad_pop: torch.Tensor, grad_non: torch.Tensor, lr: float, next_batch=None, timers=None) -> int:
@@ -293,11 +324,20 @@ class PipelinedHotline(Hotline):
         st, m = self.sets[j % 3], self.main
         s_main = m.cuda_stream
         w0, w1 = (j % 2) * self.window_rows, ((j + 1) % 2) * self.window_rows
+        if next_batch is not None:
+            self.sets[(j + 1) % 3].ev_inputs.record(m)   # the next mini-batch's inputs are ready at this point
         m.wait_event(st.ev_index)
-        if j >= 1:   # rows shared with mini-batch j-1 come from its staging window (its backward ran on this stream)
+        if not self.overlap_link and j >= 1:
+            # The write-back of mini-batch j-1 gets the chip to itself: its 256-byte row writes reach the link as
+            # whole rows only while nothing else churns the L2 (measured: 125 us alone, 550-870 us next to the
+            # popular micro-batch's kernels).  This mini-batch's popular work starts when it is done, next to the
+            # read of its own cold rows, which does not mind.
+            m.wait_event(self.sets[(j - 1) % 3].ev_scatter)
+        if self.overlap_link and j >= 1:
+            # rows shared with mini-batch j-1 come from its staging window (its backward ran on this stream)
             B.hl_forward_cold(self.ctx, self.cache, w1, w0, self.window_rows, st.fwd_src, st.n_cold, s_main)
         st.ev_forward.record(m)
-        if next_batch is not None:
+        if next_batch is not None and self.overlap_link:
             self._submit(*next_batch, timers=timers)
         t = lambda name, stream, fn: self._timed(timers, name, stream, fn)   # noqa: E731
         t("fwd_pop", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.pop, st.counts, st.pooled_pop, s_main))
@@ -312,6 +352,8 @@ class PipelinedHotline(Hotline):
             self.ctx, self.cache, w0, self.window_rows, st.cold_rows, st.n_cold, self.host_table,
             self.wb.cuda_stream))
         st.ev_scatter.record(self.wb)
+        if next_batch is not None and not self.overlap_link:
+            self._submit(*next_batch, timers=timers)     # its host rows are read after the write-back just queued
         self.j_done += 1
         return j % 3
 

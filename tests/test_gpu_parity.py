@@ -103,6 +103,14 @@ def test_pipelined_steps_equal_sequential_steps_integer_data():
     assert stats["shared_cold_rows"] > 50
 
 
+def test_pipelined_steps_with_serialised_link_integer_data():
+    """The default schedule of the pipeline: the next mini-batch's host rows are read after this one's write-back."""
+    run_pipelined_check("tiny", steps=6, integer=True, overlap_link=False)
+    spec = dataclasses.replace(gen.CONFIGS["multi_hot"], batch=512, dim=32, rows=("fixed", 2000),
+                               hot_policy=("fraction", 40, 100), profile_batches=2)
+    run_pipelined_check(spec, steps=4, integer=True, overlap_link=False)
+
+
 def test_pipelined_steps_real_data_and_dense_features():
     run_pipelined_check("dlrm_small", steps=3, scale_rows=0.02, integer=False, profile_batches=6)
 
