@@ -280,6 +280,25 @@ def run_reference(args, rank: int, world: int) -> None:
 
 
 # ----------------------------------------------------------------------------------------------------------
+# ranks: independent replicas, one per GPU; the only exchange is the barrier and the max of the timings
+# ----------------------------------------------------------------------------------------------------------
+def max_over_ranks(values, world: int, device="cpu"):
+    """Element-wise maximum of ``values`` (floats) over all ranks of the default process group."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def whole_job_value(batch: int, steps: int, world: int, ms_total_max: float) -> float:
+    """Samples per second of the whole job: every rank processed batch*steps inputs in the slowest rank's time."""
+    return batch * world * steps / (ms_total_max * 1e-3)
+
+
+# ----------------------------------------------------------------------------------------------------------
 # CUDA arm
 # ----------------------------------------------------------------------------------------------------------
 def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
@@ -469,16 +488,14 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         h.status()
 
     # ---- reduce over ranks (max time) ----
-    if world > 1:
-        t = torch.tensor([ms_total, e2e["ms_total"] if e2e else 0.0], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t[0])
-        if e2e:
-            e2e["ms_total"] = float(t[1])
+    red = max_over_ranks([ms_total, e2e["ms_total"] if e2e else 0.0], world, device)
+    ms_total = red[0]
+    if e2e:
+        e2e["ms_total"] = red[1]
 
     if rank == 0:
         ms_per_step = ms_total / args.steps
-        value = B * world * args.steps / (ms_total * 1e-3)
+        value = whole_job_value(B, args.steps, world, ms_total)
 
         def mean_us(name):
             ev = timers.get(name, [])
