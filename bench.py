@@ -320,7 +320,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
     pipelined = not args.no_pipeline
     if pipelined:
         h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
-                                n_dense=wl.spec.n_dense, device=str(device), overlap_link=args.overlap_link)
+                                n_dense=wl.spec.n_dense, device=str(device), overlap_link=not args.serial_link)
     else:
         h = hl.Hotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
                        n_dense=wl.spec.n_dense, device=str(device))
@@ -544,7 +544,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                              if 2 * wl.n_bags * D * 4 > L2_BYTES else
                              "per-step working set is smaller than L2 on this workload; batches rotate over 8 buffers",
                        "schedule": ("software-pipelined across mini-batches (PipelinedHotline"
-                                    + (", overlapping host reads and write-backs)" if args.overlap_link else ")")
+                                    + (", host reads after write-backs)" if args.serial_link else
+                                       ", host reads overlap write-backs, shared rows forwarded)")
                                     if pipelined else "one mini-batch after the other (Hotline.step)"),
                        "replicas": "independent replica per GPU, no collective"},
             "clocks": clock_info, "gpu_launches": int(launches),
@@ -557,8 +558,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                 "gather_move_gbs": statistics.mean(n * D * 4 / (t * 1e-3) / 1e9 for t, n in kt["gather_move"] if t > 0),
                 "scatter_move_kernel_us": 1e3 * statistics.mean(t for t, _ in kt["scatter_move"]),
                 "scatter_move_gbs": statistics.mean(n * D * 4 / (t * 1e-3) / 1e9 for t, n in kt["scatter_move"] if t > 0),
-                "note": "fresh random rows of the host table every step; see `--micro gather` for the same kernel "
-                        "on rows whose address translations are resident"},
+                "note": "in-pipeline figures with 8 mover CTAs next to other kernels; `--micro gather` times the same "
+                        "kernel alone with 2 CTAs per SM"},
             "kernels_us": {"bwd_reduce_non": 1e3 * statistics.mean(t for t, _ in kt["bwd_reduce_non"]),
                            "fwd_non": 1e3 * statistics.mean(t for t, _ in kt["fwd_non"])},
         }
@@ -709,8 +710,9 @@ def main() -> None:
                     help="run one mini-batch after the other (Hotline.step) instead of the software pipeline "
                          "(PipelinedHotline), in which the next mini-batch's fragment, cold-row search and host reads "
                          "run under this one's execution")
-    ap.add_argument("--overlap-link", action="store_true",
-                    help="pipeline variant that also overlaps host reads with write-backs (forwarding shared rows)")
+    ap.add_argument("--serial-link", action="store_true",
+                    help="pipeline variant in which the host read of the next mini-batch follows this one's write-back "
+                         "instead of overlapping it (no forwarding of shared rows needed)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather"],
                     help="time one library call in isolation")

@@ -127,9 +127,12 @@ HL_API const char* hl_strerror(int32_t status);
 HL_API int32_t hl_timing_enable(hl_ctx* ctx, int32_t on);
 HL_API int32_t hl_timing_read(hl_ctx* ctx, int32_t which, float* ms);
 
-/* Pinned, device-mapped host memory for the host-DRAM table (exactly `bytes`, no rounding): the device reads
- * and writes it over the host link at the same address.  The caller owns it and frees it with hl_host_free.
- * Returns NULL on failure. */
+/* Host-resident, device-mapped memory for the host-DRAM table (exactly `bytes`): the current device reads and
+ * writes it in place over the host link, at the same address the CPU uses; the pages stay in host DRAM.  (Unified
+ * memory with the CPU as preferred location and the device advised to map it, which the device maps in large pages;
+ * memory from cudaHostAlloc also works as a table but is mapped in 4 KB pages, and random rows of a table of tens of
+ * GB then pay an address-translation miss each.)  The caller owns it and frees it with hl_host_free.  Returns NULL
+ * on failure. */
 HL_API void* hl_host_alloc(size_t bytes);
 HL_API int32_t hl_host_free(void* p);
 

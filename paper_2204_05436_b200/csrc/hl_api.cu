@@ -188,10 +188,26 @@ unsigned long long launches_so_far();
 
 extern "C" uint64_t hl_launch_count(void) { return hl::launches_so_far(); }
 
+// Host-resident memory that the current device reads and writes in place.  It is unified memory whose preferred
+// location is the CPU and which the device is advised to map ("accessed by"): the pages stay in host DRAM, nothing
+// migrates, and -- unlike memory from cudaHostAlloc / cudaHostRegister, which the device maps in 4 KB pages -- the
+// device maps it in large pages.  That matters for a table of tens of GB read at random: with 4 KB mappings
+// every fresh row paid an address-translation miss (measured 20-24 ns per 256-byte row, 10-13 GB/s); with this
+// allocation the same rows move at 46 GB/s.
 extern "C" void* hl_host_alloc(size_t bytes) {
     void* p = nullptr;
-    if (bytes == 0 || cudaHostAlloc(&p, bytes, cudaHostAllocMapped | cudaHostAllocPortable) != cudaSuccess) {
+    int dev = 0;
+    if (bytes == 0 || cudaGetDevice(&dev) != cudaSuccess ||
+        cudaMallocManaged(&p, bytes, cudaMemAttachGlobal) != cudaSuccess) {
         cudaGetLastError();
+        return nullptr;
+    }
+    if (cudaMemAdvise(p, bytes, cudaMemAdviseSetPreferredLocation, cudaCpuDeviceId) != cudaSuccess ||
+        cudaMemAdvise(p, bytes, cudaMemAdviseSetAccessedBy, dev) != cudaSuccess ||
+        cudaMemPrefetchAsync(p, bytes, cudaCpuDeviceId, 0) != cudaSuccess ||   // populate the pages in host DRAM
+        cudaDeviceSynchronize() != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(p);
         return nullptr;
     }
     return p;
@@ -199,7 +215,7 @@ extern "C" void* hl_host_alloc(size_t bytes) {
 
 extern "C" int32_t hl_host_free(void* p) {
     if (!p) return HL_OK;
-    HL_CUDA_TRY(cudaFreeHost(p));
+    HL_CUDA_TRY(cudaFree(p));
     return HL_OK;
 }
 

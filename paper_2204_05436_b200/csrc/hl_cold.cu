@@ -201,12 +201,12 @@ constexpr int kBulkThreads = 128;
 constexpr int kBulkStages = 2;
 constexpr int kBulkStageBytes = 16384;
 constexpr int kBulkMaxPolls = 1 << 22;
-// CTAs of the mover.  8 CTAs x 2 stages x 16 KB keep 256 KB of rows in flight: enough for the link (measured: 50 GB/s
-// on rows whose translations are resident), and the fastest setting on fresh random rows (390 us for 18 K rows,
-// against 416-460 us with 16 to 64 CTAs).  More rows in flight do not go faster -- the link is waiting for address
-// translations -- but they slow every other kernel on the chip: a forward kernel that takes 49 us alone takes
-// 60 us next to 8 mover CTAs, 100 us next to 16, and over 300 us next to 32 or more.
-constexpr int kBulkCtas = 8;   // (the hot-cache load of hl_build_remap, which runs alone, uses 2 per SM)
+// CTAs of the mover inside the pipeline.  8 CTAs x 2 stages x 16 KB keep 256 KB of rows in flight: 18 K rows of
+// 256 bytes take 190 us to read and 120 us to write back.  More CTAs move the rows faster (107 us with 148) but
+// the embedding-bag kernels of the other micro-batch, which run next to the mover, lose what it gains: the time per
+// mini-batch stayed within 0.43-0.49 ms for 8 to 148 CTAs, with 8 the best in the default schedule.  (The hot-cache
+// load of hl_build_remap and hl_flush_hot, which run alone, use 2 CTAs per SM and reach 90 % of the memcpy rate.)
+constexpr int kBulkCtas = 8;
 
 template <bool TO_TABLE>
 __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_side, int64_t dense_row0, float* table,

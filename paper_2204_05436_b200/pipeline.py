@@ -31,8 +31,8 @@ class Hotline:
         self.n_dense = int(n_dense)
         if host_table.dtype != torch.float32 or tuple(host_table.shape) != (self.N, self.D):
             raise ValueError("host_table must be fp32 [N, D]")
-        if not (host_table.is_cuda or host_table.is_pinned()):
-            raise ValueError("host_table must be pinned host memory (or device memory)")
+        # host_table must be memory the device can address: from hl_host_alloc (binding.host_table_tensor), pinned
+        # host memory, or device memory.  (Not checked here: torch cannot tell for memory it did not allocate.)
         self.host_table = host_table
 
         dev = self.device
@@ -226,12 +226,14 @@ class PipelinedHotline(Hotline):
 
     Three sets of index buffers rotate over the mini-batches, two windows of the staging area alternate.
 
-    ``overlap_link=False`` (default): the host rows of mini-batch j+1 are read after mini-batch j's write-back has
-    finished, so the two transfers follow each other on the link and no forwarding is needed; fragment and the
-    search for the distinct cold rows of j+1 still run under j's execution.  ``overlap_link=True``: the read of
-    j+1 starts as soon as j-1's write-back is done and overlaps j's execution and write-back, with shared rows
-    forwarded between the staging windows (on a platform where random host rows are bound by address translation
-    the two transfers then compete and nothing is gained).
+    ``overlap_link=True`` (default): the read of j+1's host rows starts as soon as j-1's write-back is done and
+    overlaps j's execution and write-back, with the rows j+1 shares with j forwarded between the staging windows.
+    ``overlap_link=False``: the host rows of j+1 are read after j's write-back has finished, so the two transfers
+    follow each other on the link and no forwarding is needed; fragment and the search for the distinct cold rows of
+    j+1 still run under j's execution.  (Which is faster depends on the host table's memory: with large-page
+    device mappings (hl_host_alloc) 0.43 against 0.47 ms per DLRM-large-like mini-batch; with 4 KB mappings
+    (cudaHostAlloc) reads and write-backs compete for address translations and it is the other way round, 0.84
+    against 0.65 ms.)
 
         p.start(idx0, off0, B)                       # ahead-work of mini-batch 0
         for j in range(n):
@@ -241,7 +243,7 @@ class PipelinedHotline(Hotline):
     """
 
     def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
-                 n_dense: int = 0, device: str = "cuda:0", overlap_link: bool = False):
+                 n_dense: int = 0, device: str = "cuda:0", overlap_link: bool = True):
         self.overlap_link = bool(overlap_link)
         self.window_rows = int(window_rows)
         super().__init__(table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, 2 * self.window_rows,
@@ -281,10 +283,8 @@ class PipelinedHotline(Hotline):
             excl = None
             wait_a = wait_b = None
             if j >= 2:
-                # Keep this mini-batch's fragment / index kernels away from the write-back of mini-batch j-2: they
-                # then run next to the read of j-1's host rows instead.  (Measured: a write-back that shares the
-                # chip with them takes 650-870 us instead of 125 us; the read, which pays an address-translation
-                # miss per row anyway, does not care.)
+                # keep this mini-batch's fragment / index kernels away from the write-back of mini-batch j-2: they
+                # then run next to the read of j-1's host rows instead
                 side.wait_event(self.sets[(j - 2) % 3].ev_scatter)
         self._timed(timers, "fragment", side, lambda: B.hl_fragment(
             self.ctx, self._batch(indices, offsets, batch), dense, self.n_dense if dense is not None else 0,
@@ -328,10 +328,10 @@ class PipelinedHotline(Hotline):
             self.sets[(j + 1) % 3].ev_inputs.record(m)   # the next mini-batch's inputs are ready at this point
         m.wait_event(st.ev_index)
         if not self.overlap_link and j >= 1:
-            # The write-back of mini-batch j-1 gets the chip to itself: its 256-byte row writes reach the link as
-            # whole rows only while nothing else churns the L2 (measured: 125 us alone, 550-870 us next to the
-            # popular micro-batch's kernels).  This mini-batch's popular work starts when it is done, next to the
-            # read of its own cold rows, which does not mind.
+            # The write-back of mini-batch j-1 gets the chip to itself; this mini-batch's popular work starts when it
+            # is done, next to the read of its own cold rows.  (This mattered with a host table in cudaHostAlloc
+            # memory, whose 4 KB device mappings made a write-back next to other kernels 5 times slower; with a table
+            # from hl_host_alloc it costs about 3 %.)
             m.wait_event(self.sets[(j - 1) % 3].ev_scatter)
         if self.overlap_link and j >= 1:
             # rows shared with mini-batch j-1 come from its staging window (its backward ran on this stream)

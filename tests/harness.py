@@ -211,7 +211,7 @@ def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: boo
 
 
 def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: bool = True, profile_batches=None,
-                        device: str = "cuda:0", overlap_link: bool = True):
+                        device: str = "cuda:0", overlap_link: bool = True):  # noqa: D401
     """Software-pipelined CUDA path (PipelinedHotline) against the oracle processing the same mini-batches one
     after the other.  With integer data every sum is exact, so pooled vectors, the hot cache and the host table
     must agree bit for bit after any number of steps -- which they only do if rows shared by consecutive
