@@ -45,6 +45,7 @@ class Hotline:
         self.n_hot = torch.zeros(1, dtype=i64, device=dev)
         self.perm = torch.zeros(self.max_batch, dtype=i32, device=dev)
         self.counts = torch.zeros(4, dtype=i32, device=dev)          # n_pop, n_non, L_pop, L_non
+        self.counts_non = self.counts[1:]                            # view: pointer to n_non
         ids_cap = max(1, self.max_nnz)
         self.pop_offsets = torch.zeros(self.max_bags + 1, dtype=i32, device=dev)
         self.pop_ids = torch.zeros(ids_cap, dtype=i32, device=dev)
@@ -124,20 +125,20 @@ class Hotline:
 
     def gather_cold(self, stream: Optional[torch.cuda.Stream] = None) -> None:
         s = stream or self.main
-        B.hl_gather_cold(self.ctx, self.non, self.counts[1:], self.host_table, self.cache, self.cold_rows,
+        B.hl_gather_cold(self.ctx, self.non, self.counts_non, self.host_table, self.cache, self.cold_rows,
                          self.n_cold, s.cuda_stream)
 
     def fwd_pop(self) -> None:
         B.hl_embbag_fwd(self.ctx, self.cache, self.pop, self.counts, self.pooled_pop, self.main.cuda_stream)
 
     def fwd_non(self) -> None:
-        B.hl_embbag_fwd(self.ctx, self.cache, self.non, self.counts[1:], self.pooled_non, self.main.cuda_stream)
+        B.hl_embbag_fwd(self.ctx, self.cache, self.non, self.counts_non, self.pooled_non, self.main.cuda_stream)
 
     def bwd_pop(self, grad: torch.Tensor, lr: float) -> None:
         B.hl_embbag_bwd_sgd(self.ctx, self.cache, self.pop, self.counts, grad, lr, self.main.cuda_stream)
 
     def bwd_non(self, grad: torch.Tensor, lr: float) -> None:
-        B.hl_embbag_bwd_sgd(self.ctx, self.cache, self.non, self.counts[1:], grad, lr, self.main.cuda_stream)
+        B.hl_embbag_bwd_sgd(self.ctx, self.cache, self.non, self.counts_non, grad, lr, self.main.cuda_stream)
 
     def scatter_cold(self) -> None:
         B.hl_scatter_cold(self.ctx, self.cache, self.cold_rows, self.n_cold, self.host_table, self.main.cuda_stream)
@@ -152,7 +153,7 @@ class Hotline:
         that receives, per call name, a list of (start, end) CUDA events recorded on the stream of that call."""
 
         def timed(name, stream, fn):
-            if timers is None:
+            if timers is None or ("only" in timers and name not in timers["only"]):
                 fn()
                 return
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -194,6 +195,7 @@ class _BatchSet:
         ids_cap = max(1, h.max_nnz)
         self.perm = torch.zeros(h.max_batch, dtype=i32, device=dev)
         self.counts = torch.zeros(4, dtype=i32, device=dev)
+        self.counts_non = self.counts[1:]
         self.pop_offsets = torch.zeros(h.max_bags + 1, dtype=i32, device=dev)
         self.pop_ids = torch.zeros(ids_cap, dtype=i32, device=dev)
         self.non_offsets = torch.zeros(h.max_bags + 1, dtype=i32, device=dev)
@@ -257,7 +259,7 @@ class PipelinedHotline(Hotline):
 
     @staticmethod
     def _timed(timers, name, stream, fn):
-        if timers is None:
+        if timers is None or ("only" in timers and name not in timers["only"]):
             fn()
             return
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -291,7 +293,7 @@ class PipelinedHotline(Hotline):
             st.perm, st.counts, st.pop, st.non, st.dense_out if dense is not None else None, side.cuda_stream))
         if self.overlap_link:
             self._timed(timers, "gather_cold", side, lambda: B.hl_gather_cold_ahead(
-                self.ctx, st.non, st.counts[1:], self.host_table, self.cache, (j % 2) * self.window_rows,
+                self.ctx, st.non, st.counts_non, self.host_table, self.cache, (j % 2) * self.window_rows,
                 self.window_rows, st.cold_rows, st.n_cold,
                 excl.cold_rows if excl is not None else None, excl.n_cold if excl is not None else None, st.fwd_src,
                 st.ev_index, wait_a, wait_b, side.cuda_stream))
@@ -300,7 +302,7 @@ class PipelinedHotline(Hotline):
             # index work on the side stream; the read of the host rows on the write-back stream, behind the
             # write-back of the mini-batch before (stream order, no stream parked in an event wait meanwhile)
             self._timed(timers, "index_cold", side, lambda: B.hl_index_cold(
-                self.ctx, st.non, st.counts[1:], (j % 2) * self.window_rows, self.window_rows, st.cold_rows,
+                self.ctx, st.non, st.counts_non, (j % 2) * self.window_rows, self.window_rows, st.cold_rows,
                 st.n_cold, None, None, None, side.cuda_stream))
             st.ev_index.record(side)
             self.wb.wait_event(st.ev_index)
@@ -343,8 +345,8 @@ class PipelinedHotline(Hotline):
         t("fwd_pop", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.pop, st.counts, st.pooled_pop, s_main))
         t("bwd_pop", m, lambda: B.hl_embbag_bwd_sgd(self.ctx, self.cache, st.pop, st.counts, grad_pop, lr, s_main))
         m.wait_event(st.ev_gather)
-        t("fwd_non", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.non, st.counts[1:], st.pooled_non, s_main))
-        t("bwd_non", m, lambda: B.hl_embbag_bwd_sgd(self.ctx, self.cache, st.non, st.counts[1:], grad_non, lr,
+        t("fwd_non", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.non, st.counts_non, st.pooled_non, s_main))
+        t("bwd_non", m, lambda: B.hl_embbag_bwd_sgd(self.ctx, self.cache, st.non, st.counts_non, grad_non, lr,
                                                     s_main))
         st.ev_x.record(m)
         self.wb.wait_event(st.ev_x)
