@@ -704,6 +704,97 @@ def run_micro(args) -> None:
     hl.hl_destroy(ctx)
 
 
+# ----------------------------------------------------------------------------------------------------------
+# sensitivity sweeps on synthetic data (the paper's Section VII-F studies: popular / non-popular ratio, batch size)
+# ----------------------------------------------------------------------------------------------------------
+def run_sweep(args) -> None:
+    """`--sweep`: (1) the hot-cache budget is cut from the configuration's value down to 1/64 of it, which moves
+    the ratio of popular to non-popular inputs; (2) the mini-batch size is varied at the full budget.  Every point:
+    10 warm-up and 60 timed mini-batches through the default pipeline, CUDA events.  One JSON line."""
+    import dataclasses
+    import torch
+    import paper_2204_05436_b200 as hl
+    device = torch.device("cuda:0")
+    torch.cuda.set_device(device)
+    name, scale = pick_workload(args.workload, 1)
+    wl = Workload(name, scale, 8, args.profile_batches, device, args.threads)
+    T, D, S = wl.T, wl.D, wl.S
+    points = []
+
+    def measure(h, batches, B, n_bags, label):
+        d_in = [(torch.from_numpy(b.indices).to(device), torch.from_numpy(b.offsets).to(device), B,
+                 torch.from_numpy(b.dense).to(device) if b.dense is not None else None) for b in batches]
+        d_grad = torch.randn((n_bags, D), device=device, dtype=torch.float32)
+        torch.cuda.synchronize()
+        n = len(d_in)
+        it = [0]
+
+        def step():
+            i = it[0]
+            it[0] += 1
+            if h.j_submitted == h.j_done:
+                h.start(*d_in[i % n])
+            return h.sets[h.step(d_grad, d_grad, wl.spec.lr, next_batch=d_in[(i + 1) % n])]
+
+        pops, colds = [], []
+        for _ in range(n):
+            st = step()
+            h.drain()
+            pops.append(int(st.counts[0].item()))
+            colds.append(int(st.n_cold.item()))
+        for _ in range(10):
+            step()
+        h.drain()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(h.main)
+        for _ in range(60):
+            step()
+        h.main.wait_stream(h.wb)
+        e1.record(h.main)
+        h.drain()
+        h.status()
+        ms = e0.elapsed_time(e1) / 60
+        points.append(dict(label, batch=B, popular_fraction=sum(pops) / (len(pops) * B),
+                           cold_rows_per_step=sum(colds) / len(colds), ms_per_step=ms, samples_per_s=B / ms * 1e3))
+        log(f"[sweep] {points[-1]}")
+
+    def learn(h, k_rows):
+        for i, b in enumerate(wl.profile):
+            h.profile(torch.from_numpy(b.indices).to(device), torch.from_numpy(b.offsets).to(device), wl.B, reset=(i == 0))
+        h.profile(None, None, finalize=True, policy=hl.HL_HOT_TOPK_ROWS, p_num=k_rows)
+        h.build_remap(load_rows=True)
+        h.status()
+        return int(h.n_hot.item())
+
+    # (1) budget / ratio sweep
+    h = hl.PipelinedHotline(wl.geom.table_rows, D, S, wl.B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
+                            n_dense=wl.spec.n_dense, device=str(device))
+    with torch.cuda.stream(h.main):
+        for div in (1, 2, 4, 16, 64):
+            n_hot = learn(h, max(1, wl.hot_cap // div))
+            measure(h, wl.batches, wl.B, wl.n_bags, dict(sweep="budget", budget_fraction=1.0 / div, hot_rows=n_hot))
+            h.flush_hot()            # the host table gets the popular rows back before the set changes
+            h.status()
+    h.close()
+    # (2) batch-size sweep at the full budget
+    for B in (2048, 4096, 8192, 32768):
+        spec = dataclasses.replace(wl.spec, batch=B)
+        batches = [gen.make_batch(spec, wl.geom, 100_000 + i, args.threads) for i in range(8)]
+        n_bags = T * B * S
+        mb = max(B, wl.B)
+        h = hl.PipelinedHotline(wl.geom.table_rows, D, S, mb, T * mb * S if wl.spec.pooling[0] == "one" else
+                                T * mb * S * int(wl.spec.pooling[2]), wl.hot_cap, wl.staging_cap, wl.table,
+                                n_dense=wl.spec.n_dense, device=str(device))
+        with torch.cuda.stream(h.main):
+            n_hot = learn(h, wl.hot_cap)
+            measure(h, batches, B, n_bags, dict(sweep="batch", budget_fraction=1.0, hot_rows=n_hot))
+            h.flush_hot()
+            h.status()
+        h.close()
+    print(json.dumps({"sweep": wl.name, "unit": "ms per mini-batch, samples/s", "points": points}), flush=True)
+    wl.free()
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -727,7 +818,11 @@ def main() -> None:
     ap.add_argument("--micro-dist", default="uniform", choices=["uniform", "zipf"])
     ap.add_argument("--micro-batch", type=int, default=16384)
     ap.add_argument("--micro-dim", type=int, default=64)
+    ap.add_argument("--sweep", action="store_true", help="hot-budget (popular ratio) and batch-size sweeps")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.micro == "gather":
         run_micro_gather(args)
         return
