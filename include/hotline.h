@@ -202,6 +202,20 @@ HL_API int32_t hl_embbag_fwd(hl_ctx* ctx, const float* d_cache, const hl_ubatch*
 HL_API int32_t hl_embbag_bwd_sgd(hl_ctx* ctx, float* d_cache, const hl_ubatch* ub, const int32_t* d_n_samples,
                           const float* d_grad_out, float lr, void* stream);
 
+/* The two halves of hl_embbag_bwd_sgd as separate calls.  hl_embbag_bwd_prepare does the part that depends only on
+ * the micro-batch's ids: the (slot, bag) pair of every lookup, stably sorted by slot, into d_sorted_slots /
+ * d_sorted_bags [cap_ids each], their number into *d_n_lookups.  It can therefore run ahead, on another stream, as
+ * soon as the ids are final (for X: after hl_gather_cold / hl_index_cold), which takes the sort off the path between
+ * a forward and its backward.  hl_embbag_bwd_apply then sums the gradient rows per run of equal slots and applies the
+ * one SGD update per row.  Scratch: prepare uses the sort buffers of the backward region (as hl_embbag_bwd_sgd does:
+ * do not overlap two of them), apply the partial-sum buffer of the backward region (do not overlap two applies). */
+HL_API int32_t hl_embbag_bwd_prepare(hl_ctx* ctx, const hl_ubatch* ub, const int32_t* d_n_samples,
+                                     int32_t* d_sorted_slots, int32_t* d_sorted_bags, int32_t* d_n_lookups,
+                                     void* stream);
+HL_API int32_t hl_embbag_bwd_apply(hl_ctx* ctx, float* d_cache, const int32_t* d_sorted_slots,
+                                   const int32_t* d_sorted_bags, const int32_t* d_n_lookups, const float* d_grad_out,
+                                   float lr, void* stream);
+
 /* Sections IV and V-A (dma_rd of non-popular rows; popular rows of X are read from GPU memory).
  * In:  non->ids = global rows of X (from hl_fragment), *d_n_non = inputs in X.
  * Out: d_cold_rows[0 .. *d_n_cold) = the distinct non-popular rows referenced by X, ascending (each staged

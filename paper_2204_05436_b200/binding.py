@@ -19,7 +19,7 @@ EXPORTS = (
     "hl_workspace_bytes", "hl_create", "hl_destroy", "hl_status", "hl_strerror", "hl_launch_count", "hl_timing_enable", "hl_timing_read", "hl_host_alloc",
     "hl_host_free", "hl_profile_hot",
     "hl_build_remap", "hl_fragment", "hl_embbag_fwd", "hl_embbag_bwd_sgd", "hl_gather_cold", "hl_scatter_cold",
-    "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at", "hl_flush_hot", "hl_index_cold", "hl_stage_cold",
+    "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at", "hl_flush_hot", "hl_index_cold", "hl_stage_cold", "hl_embbag_bwd_prepare", "hl_embbag_bwd_apply",
 )
 
 
@@ -97,6 +97,10 @@ def _load() -> ctypes.CDLL:
     lib.hl_index_cold.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, i64, i64, vp, vp, vp, vp, vp, vp]
     lib.hl_stage_cold.restype = i32
     lib.hl_stage_cold.argtypes = [vp, vp, vp, i64, i64, vp, vp, vp, vp]
+    lib.hl_embbag_bwd_prepare.restype = i32
+    lib.hl_embbag_bwd_prepare.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, vp, vp, vp, vp]
+    lib.hl_embbag_bwd_apply.restype = i32
+    lib.hl_embbag_bwd_apply.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp]
     lib.hl_flush_hot.restype = i32
     lib.hl_flush_hot.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.hl_embbag_bwd_sgd_static.restype = i32
@@ -309,3 +313,17 @@ def hl_stage_cold(ctx: int, host_table, d_cache, stage_row0: int, stage_rows: in
                   stream: int) -> None:
     _check("hl_stage_cold", _lib.hl_stage_cold(ctx, _ptr(host_table), _ptr(d_cache), int(stage_row0), int(stage_rows),
                                                _ptr(d_cold_rows), _ptr(d_n_cold), _ptr(d_fwd_src), stream))
+
+
+def hl_embbag_bwd_prepare(ctx: int, ub: hl_ubatch, d_n_samples, d_sorted_slots, d_sorted_bags, d_n_lookups,
+                          stream: int) -> None:
+    _check("hl_embbag_bwd_prepare", _lib.hl_embbag_bwd_prepare(ctx, ctypes.byref(ub), _ptr(d_n_samples),
+                                                               _ptr(d_sorted_slots), _ptr(d_sorted_bags),
+                                                               _ptr(d_n_lookups), stream))
+
+
+def hl_embbag_bwd_apply(ctx: int, d_cache, d_sorted_slots, d_sorted_bags, d_n_lookups, d_grad_out, lr: float,
+                        stream: int) -> None:
+    _check("hl_embbag_bwd_apply", _lib.hl_embbag_bwd_apply(ctx, _ptr(d_cache), _ptr(d_sorted_slots),
+                                                           _ptr(d_sorted_bags), _ptr(d_n_lookups), _ptr(d_grad_out),
+                                                           float(lr), stream))

@@ -427,17 +427,17 @@ int32_t launch_fwd(hl_ctx* ctx, const float* cache, const hl_ubatch* ub, const i
 }
 
 template <int G, int NV>
-int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t* vals, const float* grad, float lr,
-                   cudaStream_t stream) {
+int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t* vals, const int32_t* d_n_lookups,
+                   const float* grad, float lr, cudaStream_t stream) {
     const int64_t max_chunks = div_up(ctx->max_nnz, kBwdChunk);
     const int grid = grid_for(max_chunks * G, kThreads, kMaxGrid);
     const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 0, stream);
-    k_bwd_chunks<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, vals, ctx->r.bwd_n, grad, ctx->D / 4, n_slots,
+    k_bwd_chunks<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, vals, d_n_lookups, grad, ctx->D / 4, n_slots,
                                                       lr, ctx->r.bwd_part);
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 1, stream);
     const int span_grid = grid_for(max_chunks * 32, kThreads, kMaxGrid);   // one warp per chunk
-    k_bwd_spans<G, NV><<<span_grid, kThreads, 0, stream>>>(cache, keys, ctx->r.bwd_n, ctx->D / 4, n_slots, lr,
+    k_bwd_spans<G, NV><<<span_grid, kThreads, 0, stream>>>(cache, keys, d_n_lookups, ctx->D / 4, n_slots, lr,
                                                           ctx->r.bwd_part);
     note_launches(2);
     HL_LAUNCH_CHECK();
@@ -477,30 +477,79 @@ extern "C" int32_t hl_embbag_fwd(hl_ctx* ctx, const float* d_cache, const hl_uba
 #undef HL_FWD
 }
 
+namespace hl {
+namespace {
+
+// (slot, bag) pairs of the micro-batch, sorted by slot (stable).  The result lands in out_keys / out_vals: either
+// the caller's arrays (which then serve as one half of the sort's ping-pong buffers) or, if they are null, whichever
+// scratch buffer the last pass wrote.
+int32_t sort_lookups(hl_ctx* ctx, const hl_ubatch* ub, const int32_t* d_n_samples, int32_t* caller_keys,
+                     int32_t* caller_vals, int32_t* d_n_lookups, int32_t** out_keys, int32_t** out_vals,
+                     cudaStream_t stream) {
+    Regions& r = ctx->r;
+    const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
+    const int key_bits = bits_for(n_slots);
+    const int passes = (key_bits + 7) / 8;
+    int32_t* keys[2] = {r.bwd_keys[0], r.bwd_keys[1]};
+    int32_t* vals[2] = {r.bwd_vals[0], r.bwd_vals[1]};
+    if (caller_keys) {   // make the buffer the last pass writes the caller's
+        keys[passes & 1] = caller_keys;
+        vals[passes & 1] = caller_vals;
+    }
+    const bool short_bags = ctx->max_nnz <= 4 * ctx->max_bags;
+    if (short_bags)
+        k_bwd_pairs<1><<<grid_for(ctx->max_bags, kThreads, kMaxGrid), kThreads, 0, stream>>>(
+            ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, keys[0], vals[0],
+            d_n_lookups, r.status);
+    else
+        k_bwd_pairs<32><<<grid_for(ctx->max_bags, kThreads / 32, kMaxGrid), kThreads, 0, stream>>>(
+            ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, keys[0], vals[0],
+            d_n_lookups, r.status);
+    note_launches(1);
+    HL_LAUNCH_CHECK();
+    return radix_sort_pairs(keys, vals, d_n_lookups, ctx->max_nnz, key_bits, r.bwd_hist, r.status, out_keys, out_vals,
+                            stream);
+}
+
+}  // namespace
+}  // namespace hl
+
 extern "C" int32_t hl_embbag_bwd_sgd(hl_ctx* ctx, float* d_cache, const hl_ubatch* ub, const int32_t* d_n_samples,
                                      const float* d_grad_out, float lr, void* stream_) {
     if (!ctx || !d_cache || !ub || !ub->offsets || !d_n_samples || !d_grad_out) return HL_EINVAL;
     if (ctx->max_nnz == 0) return HL_OK;
     if (!ub->ids) return HL_EINVAL;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    Regions& r = ctx->r;
-    const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
-    const bool short_bags = ctx->max_nnz <= 4 * ctx->max_bags;
-    if (short_bags)
-        k_bwd_pairs<1><<<grid_for(ctx->max_bags, kThreads, kMaxGrid), kThreads, 0, stream>>>(
-            ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, r.bwd_keys[0],
-            r.bwd_vals[0], r.bwd_n, r.status);
-    else
-        k_bwd_pairs<32><<<grid_for(ctx->max_bags, kThreads / 32, kMaxGrid), kThreads, 0, stream>>>(
-            ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, r.bwd_keys[0],
-            r.bwd_vals[0], r.bwd_n, r.status);
-    note_launches(1);
-    HL_LAUNCH_CHECK();
     int32_t *keys, *vals;
-    int32_t st = radix_sort_pairs(r.bwd_keys, r.bwd_vals, r.bwd_n, ctx->max_nnz, bits_for(n_slots), r.bwd_hist,
-                                  r.status, &keys, &vals, stream);
+    int32_t st = sort_lookups(ctx, ub, d_n_samples, nullptr, nullptr, ctx->r.bwd_n, &keys, &vals, stream);
     if (st != HL_OK) return st;
-#define HL_BWD(G, NV) launch_bwd<G, NV>(ctx, d_cache, keys, vals, d_grad_out, lr, stream)
+#define HL_BWD(G, NV) launch_bwd<G, NV>(ctx, d_cache, keys, vals, ctx->r.bwd_n, d_grad_out, lr, stream)
+    HL_DISPATCH_ROW_SHAPE(ctx->D / 4, HL_BWD);
+#undef HL_BWD
+}
+
+extern "C" int32_t hl_embbag_bwd_prepare(hl_ctx* ctx, const hl_ubatch* ub, const int32_t* d_n_samples,
+                                         int32_t* d_sorted_slots, int32_t* d_sorted_bags, int32_t* d_n_lookups,
+                                         void* stream_) {
+    if (!ctx || !ub || !ub->offsets || !d_n_samples || !d_n_lookups) return HL_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (ctx->max_nnz == 0) {
+        HL_CUDA_TRY(cudaMemsetAsync(d_n_lookups, 0, sizeof(int32_t), stream));
+        return HL_OK;
+    }
+    if (!ub->ids || !d_sorted_slots || !d_sorted_bags) return HL_EINVAL;
+    int32_t *keys, *vals;
+    return sort_lookups(ctx, ub, d_n_samples, d_sorted_slots, d_sorted_bags, d_n_lookups, &keys, &vals, stream);
+}
+
+extern "C" int32_t hl_embbag_bwd_apply(hl_ctx* ctx, float* d_cache, const int32_t* d_sorted_slots,
+                                       const int32_t* d_sorted_bags, const int32_t* d_n_lookups,
+                                       const float* d_grad_out, float lr, void* stream_) {
+    if (!ctx || !d_cache || !d_n_lookups || !d_grad_out) return HL_EINVAL;
+    if (ctx->max_nnz == 0) return HL_OK;
+    if (!d_sorted_slots || !d_sorted_bags) return HL_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+#define HL_BWD(G, NV) launch_bwd<G, NV>(ctx, d_cache, d_sorted_slots, d_sorted_bags, d_n_lookups, d_grad_out, lr, stream)
     HL_DISPATCH_ROW_SHAPE(ctx->D / 4, HL_BWD);
 #undef HL_BWD
 }

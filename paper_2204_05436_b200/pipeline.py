@@ -215,8 +215,17 @@ class _BatchSet:
         self.ev_x = torch.cuda.Event()
         self.ev_scatter = torch.cuda.Event()
         self.ev_inputs = torch.cuda.Event()
-        for e in (self.ev_index, self.ev_gather, self.ev_forward, self.ev_x, self.ev_scatter, self.ev_inputs):
+        self.ev_frag = torch.cuda.Event()
+        self.ev_prep_pop = torch.cuda.Event()
+        self.ev_prep_non = torch.cuda.Event()
+        for e in (self.ev_index, self.ev_gather, self.ev_forward, self.ev_x, self.ev_scatter, self.ev_inputs,
+                  self.ev_frag, self.ev_prep_pop, self.ev_prep_non):
             e.record(h.main)
+        # (slot, bag) pairs of both micro-batches sorted by slot, prepared ahead of the backward passes
+        self.sorted_pop = (torch.zeros(ids_cap, dtype=i32, device=dev), torch.zeros(ids_cap, dtype=i32, device=dev),
+                           torch.zeros(1, dtype=i32, device=dev))
+        self.sorted_non = (torch.zeros(ids_cap, dtype=i32, device=dev), torch.zeros(ids_cap, dtype=i32, device=dev),
+                           torch.zeros(1, dtype=i32, device=dev))
 
 
 class PipelinedHotline(Hotline):
@@ -245,14 +254,19 @@ class PipelinedHotline(Hotline):
     """
 
     def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
-                 n_dense: int = 0, device: str = "cuda:0", overlap_link: bool = True):
+                 n_dense: int = 0, device: str = "cuda:0", overlap_link: bool = True, sort_ahead: bool = True):
         self.overlap_link = bool(overlap_link)
+        # sort_ahead (with overlap_link): the sorts of the two backward passes, which depend on the ids only, are
+        # part of the ahead-work (hl_embbag_bwd_prepare on a side stream); the main stream keeps the forwards and
+        # the gradient sums + updates (hl_embbag_bwd_apply)
+        self.sort_ahead = bool(sort_ahead) and self.overlap_link
         self.window_rows = int(window_rows)
         super().__init__(table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, 2 * self.window_rows,
                          host_table, n_dense=n_dense, device=device)
         self.sets = [_BatchSet(self) for _ in range(3)]
         self.sides = [self.side, torch.cuda.Stream(device=self.device)]
         self.wb = torch.cuda.Stream(device=self.device)
+        self.link = torch.cuda.Stream(device=self.device)
         self.j_submitted = 0      # mini-batches whose ahead-work has been issued
         self.j_done = 0           # mini-batches whose main work has been issued
         torch.cuda.synchronize(self.device)
@@ -268,7 +282,79 @@ class PipelinedHotline(Hotline):
         b.record(stream)
         timers.setdefault(name, []).append((a, b))
 
+    def _submit_sorted(self, indices, offsets, batch: int, dense=None, timers=None) -> None:
+        """Ahead-work of mini-batch j in the sort_ahead schedule.  Stream A: fragment, cold-row search.  Stream B:
+        the backward sorts of O (after fragment) and X (after the cold-row search).  Link stream: the host read."""
+        j = self.j_submitted
+        st, sa, sb, lk = self.sets[j % 3], self.sides[0], self.sides[1], self.link
+        prev = self.sets[(j - 1) % 3] if j >= 1 else None
+        w = (j % 2) * self.window_rows
+        sa.wait_event(st.ev_inputs)
+        if j >= 3:
+            sa.wait_event(st.ev_scatter)                 # the buffers of set j%3 were mini-batch j-3's
+        self._timed(timers, "fragment", sa, lambda: B.hl_fragment(
+            self.ctx, self._batch(indices, offsets, batch), dense, self.n_dense if dense is not None else 0,
+            st.perm, st.counts, st.pop, st.non, st.dense_out if dense is not None else None, sa.cuda_stream))
+        st.ev_frag.record(sa)
+        self._timed(timers, "index_cold", sa, lambda: B.hl_index_cold(
+            self.ctx, st.non, st.counts_non, w, self.window_rows, st.cold_rows, st.n_cold,
+            prev.cold_rows if prev is not None else None, prev.n_cold if prev is not None else None, st.fwd_src,
+            sa.cuda_stream))
+        st.ev_index.record(sa)
+        sb.wait_event(st.ev_frag)
+        self._timed(timers, "sort_pop", sb, lambda: B.hl_embbag_bwd_prepare(
+            self.ctx, st.pop, st.counts, st.sorted_pop[0], st.sorted_pop[1], st.sorted_pop[2], sb.cuda_stream))
+        st.ev_prep_pop.record(sb)
+        sb.wait_event(st.ev_index)
+        self._timed(timers, "sort_non", sb, lambda: B.hl_embbag_bwd_prepare(
+            self.ctx, st.non, st.counts_non, st.sorted_non[0], st.sorted_non[1], st.sorted_non[2], sb.cuda_stream))
+        st.ev_prep_non.record(sb)
+        lk.wait_event(st.ev_index)
+        if j >= 2:
+            lk.wait_event(self.sets[(j - 2) % 3].ev_scatter)    # host rows of j-2 are final; its window is free
+        if prev is not None:
+            lk.wait_event(prev.ev_forward)                       # j-1 took what it needs out of this window
+        self._timed(timers, "gather_cold", lk, lambda: B.hl_stage_cold(
+            self.ctx, self.host_table, self.cache, w, self.window_rows, st.cold_rows, st.n_cold,
+            st.fwd_src if prev is not None else None, lk.cuda_stream))
+        st.ev_gather.record(lk)
+        self.j_submitted += 1
+
+    def _step_sorted(self, grad_pop, grad_non, lr, next_batch, timers) -> int:
+        j = self.j_done
+        st, m = self.sets[j % 3], self.main
+        s_main = m.cuda_stream
+        w0, w1 = (j % 2) * self.window_rows, ((j + 1) % 2) * self.window_rows
+        if next_batch is not None:
+            self.sets[(j + 1) % 3].ev_inputs.record(m)
+        m.wait_event(st.ev_index)
+        if j >= 1:
+            B.hl_forward_cold(self.ctx, self.cache, w1, w0, self.window_rows, st.fwd_src, st.n_cold, s_main)
+        st.ev_forward.record(m)
+        if next_batch is not None:
+            self._submit_sorted(*next_batch, timers=timers)
+        t = lambda name, stream, fn: self._timed(timers, name, stream, fn)   # noqa: E731
+        t("fwd_pop", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.pop, st.counts, st.pooled_pop, s_main))
+        m.wait_event(st.ev_prep_pop)
+        t("bwd_pop", m, lambda: B.hl_embbag_bwd_apply(self.ctx, self.cache, st.sorted_pop[0], st.sorted_pop[1],
+                                                      st.sorted_pop[2], grad_pop, lr, s_main))
+        m.wait_event(st.ev_gather)
+        t("fwd_non", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.non, st.counts_non, st.pooled_non, s_main))
+        m.wait_event(st.ev_prep_non)
+        t("bwd_non", m, lambda: B.hl_embbag_bwd_apply(self.ctx, self.cache, st.sorted_non[0], st.sorted_non[1],
+                                                      st.sorted_non[2], grad_non, lr, s_main))
+        st.ev_x.record(m)
+        self.wb.wait_event(st.ev_x)
+        t("scatter_cold", self.wb, lambda: B.hl_scatter_cold_at(
+            self.ctx, self.cache, w0, self.window_rows, st.cold_rows, st.n_cold, self.host_table,
+            self.wb.cuda_stream))
+        st.ev_scatter.record(self.wb)
+        self.j_done += 1
+        return j % 3
+
     def _submit(self, indices, offsets, batch: int, dense=None, timers=None) -> None:
+        if self.sort_ahead:
+            return self._submit_sorted(indices, offsets, batch, dense, timers)
         j = self.j_submitted
         st, side = self.sets[j % 3], self.sides[j % 2]
         side.wait_event(st.ev_inputs)                    # the caller prepared the inputs on the main stream
@@ -323,6 +409,8 @@ class PipelinedHotline(Hotline):
         that holds this mini-batch's outputs."""
         j = self.j_done
         assert self.j_submitted == j + 1, "call start() first"
+        if self.sort_ahead:
+            return self._step_sorted(grad_pop, grad_non, lr, next_batch, timers)
         st, m = self.sets[j % 3], self.main
         s_main = m.cuda_stream
         w0, w1 = (j % 2) * self.window_rows, ((j + 1) % 2) * self.window_rows
@@ -361,5 +449,5 @@ class PipelinedHotline(Hotline):
 
     def drain(self) -> None:
         """Waits until everything issued so far, write-backs included, has finished."""
-        for s in [self.main, self.wb] + self.sides:
+        for s in [self.main, self.wb, self.link] + self.sides:
             s.synchronize()

@@ -103,6 +103,12 @@ def test_pipelined_steps_equal_sequential_steps_integer_data():
     assert stats["shared_cold_rows"] > 50
 
 
+def test_pipelined_steps_without_sorting_ahead_integer_data():
+    """The pipeline with the backward sorts left on the main stream (hl_embbag_bwd_sgd instead of prepare/apply)."""
+    stats = run_pipelined_check("tiny", steps=6, integer=True, sort_ahead=False)
+    assert stats["shared_cold_rows"] > 50
+
+
 def test_pipelined_steps_with_serialised_link_integer_data():
     """The default schedule of the pipeline: the next mini-batch's host rows are read after this one's write-back."""
     run_pipelined_check("tiny", steps=6, integer=True, overlap_link=False)
