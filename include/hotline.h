@@ -131,8 +131,9 @@ HL_API int32_t hl_timing_read(hl_ctx* ctx, int32_t which, float* ms);
  * writes it in place over the host link, at the same address the CPU uses; the pages stay in host DRAM.  (Unified
  * memory with the CPU as preferred location and the device advised to map it, which the device maps in large pages;
  * memory from cudaHostAlloc also works as a table but is mapped in 4 KB pages, and random rows of a table of tens of
- * GB then pay an address-translation miss each.)  The caller owns it and frees it with hl_host_free.  Returns NULL
- * on failure. */
+ * GB then pay an address-translation miss each.  If unified memory refuses the size -- on the bench platform a single
+ * allocation stops between 66 and 70 GB -- the call falls back to such memory.)  The caller owns it and frees it
+ * with hl_host_free.  Returns NULL on failure. */
 HL_API void* hl_host_alloc(size_t bytes);
 HL_API int32_t hl_host_free(void* p);
 

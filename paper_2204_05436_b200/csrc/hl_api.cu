@@ -197,17 +197,22 @@ extern "C" uint64_t hl_launch_count(void) { return hl::launches_so_far(); }
 extern "C" void* hl_host_alloc(size_t bytes) {
     void* p = nullptr;
     int dev = 0;
-    if (bytes == 0 || cudaGetDevice(&dev) != cudaSuccess ||
-        cudaMallocManaged(&p, bytes, cudaMemAttachGlobal) != cudaSuccess) {
-        cudaGetLastError();
-        return nullptr;
-    }
-    if (cudaMemAdvise(p, bytes, cudaMemAdviseSetPreferredLocation, cudaCpuDeviceId) != cudaSuccess ||
-        cudaMemAdvise(p, bytes, cudaMemAdviseSetAccessedBy, dev) != cudaSuccess ||
-        cudaMemPrefetchAsync(p, bytes, cudaCpuDeviceId, 0) != cudaSuccess ||   // populate the pages in host DRAM
-        cudaDeviceSynchronize() != cudaSuccess) {
+    if (bytes == 0 || cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    if (cudaMallocManaged(&p, bytes, cudaMemAttachGlobal) == cudaSuccess) {
+        if (cudaMemAdvise(p, bytes, cudaMemAdviseSetPreferredLocation, cudaCpuDeviceId) == cudaSuccess &&
+            cudaMemAdvise(p, bytes, cudaMemAdviseSetAccessedBy, dev) == cudaSuccess &&
+            cudaMemPrefetchAsync(p, bytes, cudaCpuDeviceId, 0) == cudaSuccess &&   // populate the pages in host DRAM
+            cudaDeviceSynchronize() == cudaSuccess)
+            return p;
         cudaGetLastError();
         cudaFree(p);
+    }
+    cudaGetLastError();
+    // Unified memory refused the size (on the bench platform one allocation stops between 66 and 70 GB): plain
+    // pinned, mapped host memory still works as a table, with 4 KB device mappings.
+    p = nullptr;
+    if (cudaHostAlloc(&p, bytes, cudaHostAllocMapped | cudaHostAllocPortable) != cudaSuccess) {
+        cudaGetLastError();
         return nullptr;
     }
     return p;
@@ -215,7 +220,13 @@ extern "C" void* hl_host_alloc(size_t bytes) {
 
 extern "C" int32_t hl_host_free(void* p) {
     if (!p) return HL_OK;
-    HL_CUDA_TRY(cudaFree(p));
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, p) != cudaSuccess) {
+        cudaGetLastError();
+        return HL_ECUDA;
+    }
+    if (attr.type == cudaMemoryTypeManaged) HL_CUDA_TRY(cudaFree(p));
+    else HL_CUDA_TRY(cudaFreeHost(p));
     return HL_OK;
 }
 
