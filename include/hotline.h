@@ -217,6 +217,18 @@ HL_API int32_t hl_embbag_bwd_apply(hl_ctx* ctx, float* d_cache, const int32_t* d
                                    const int32_t* d_sorted_bags, const int32_t* d_n_lookups, const float* d_grad_out,
                                    float lr, void* stream);
 
+/* One sort for both micro-batches of a mini-batch: hl_embbag_bwd_prepare2 sorts the (slot, bag) pairs of O and X
+ * together (X's keys offset by the number of cache slots, so that O's pairs come first), which costs one three-pass
+ * sort instead of two; d_n_lookups[0..2] = lookups of O, lookups of X, their sum.  O's ids must all be valid slots.
+ * hl_embbag_bwd_apply2(which = 0 for O, 1 for X) is hl_embbag_bwd_apply on that micro-batch's part of the arrays.
+ * d_sorted_slots / d_sorted_bags hold cap_ids(pop) + cap_ids(non) <= max_nnz entries.  Scratch as for prepare / apply. */
+HL_API int32_t hl_embbag_bwd_prepare2(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_n_pop, const hl_ubatch* non,
+                                      const int32_t* d_n_non, int32_t* d_sorted_slots, int32_t* d_sorted_bags,
+                                      int32_t* d_n_lookups, void* stream);
+HL_API int32_t hl_embbag_bwd_apply2(hl_ctx* ctx, float* d_cache, const int32_t* d_sorted_slots,
+                                    const int32_t* d_sorted_bags, const int32_t* d_n_lookups, int32_t which,
+                                    const float* d_grad_out, float lr, void* stream);
+
 /* Sections IV and V-A (dma_rd of non-popular rows; popular rows of X are read from GPU memory).
  * In:  non->ids = global rows of X (from hl_fragment), *d_n_non = inputs in X.
  * Out: d_cold_rows[0 .. *d_n_cold) = the distinct non-popular rows referenced by X, ascending (each staged

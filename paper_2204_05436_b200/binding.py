@@ -20,6 +20,7 @@ EXPORTS = (
     "hl_host_free", "hl_profile_hot",
     "hl_build_remap", "hl_fragment", "hl_embbag_fwd", "hl_embbag_bwd_sgd", "hl_gather_cold", "hl_scatter_cold",
     "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at", "hl_flush_hot", "hl_index_cold", "hl_stage_cold", "hl_embbag_bwd_prepare", "hl_embbag_bwd_apply",
+    "hl_embbag_bwd_prepare2", "hl_embbag_bwd_apply2",
 )
 
 
@@ -101,6 +102,10 @@ def _load() -> ctypes.CDLL:
     lib.hl_embbag_bwd_prepare.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, vp, vp, vp, vp]
     lib.hl_embbag_bwd_apply.restype = i32
     lib.hl_embbag_bwd_apply.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, vp]
+    lib.hl_embbag_bwd_prepare2.restype = i32
+    lib.hl_embbag_bwd_prepare2.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, ctypes.POINTER(hl_ubatch), vp, vp, vp, vp, vp]
+    lib.hl_embbag_bwd_apply2.restype = i32
+    lib.hl_embbag_bwd_apply2.argtypes = [vp, vp, vp, vp, vp, i32, vp, ctypes.c_float, vp]
     lib.hl_flush_hot.restype = i32
     lib.hl_flush_hot.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.hl_embbag_bwd_sgd_static.restype = i32
@@ -327,3 +332,17 @@ def hl_embbag_bwd_apply(ctx: int, d_cache, d_sorted_slots, d_sorted_bags, d_n_lo
     _check("hl_embbag_bwd_apply", _lib.hl_embbag_bwd_apply(ctx, _ptr(d_cache), _ptr(d_sorted_slots),
                                                            _ptr(d_sorted_bags), _ptr(d_n_lookups), _ptr(d_grad_out),
                                                            float(lr), stream))
+
+
+def hl_embbag_bwd_prepare2(ctx: int, pop: hl_ubatch, d_n_pop, non: hl_ubatch, d_n_non, d_sorted_slots, d_sorted_bags,
+                           d_n_lookups, stream: int) -> None:
+    _check("hl_embbag_bwd_prepare2", _lib.hl_embbag_bwd_prepare2(
+        ctx, ctypes.byref(pop), _ptr(d_n_pop), ctypes.byref(non), _ptr(d_n_non), _ptr(d_sorted_slots),
+        _ptr(d_sorted_bags), _ptr(d_n_lookups), stream))
+
+
+def hl_embbag_bwd_apply2(ctx: int, d_cache, d_sorted_slots, d_sorted_bags, d_n_lookups, which: int, d_grad_out,
+                         lr: float, stream: int) -> None:
+    _check("hl_embbag_bwd_apply2", _lib.hl_embbag_bwd_apply2(
+        ctx, _ptr(d_cache), _ptr(d_sorted_slots), _ptr(d_sorted_bags), _ptr(d_n_lookups), int(which),
+        _ptr(d_grad_out), float(lr), stream))

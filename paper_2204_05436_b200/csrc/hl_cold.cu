@@ -1,6 +1,7 @@
 // The non-popular micro-batch's working set: classify its lookups, find the distinct cold rows, stage them from
 // the host-DRAM table (zero-copy 128-bit loads over the host link) behind the hot cache, and write them back.
 #include "hl_common.cuh"
+#include <cstdlib>
 
 namespace hl {
 namespace {
@@ -206,7 +207,17 @@ constexpr int kBulkMaxPolls = 1 << 22;
 // the embedding-bag kernels of the other micro-batch, which run next to the mover, lose what it gains: the time per
 // mini-batch stayed within 0.43-0.49 ms for 8 to 148 CTAs, with 8 the best in the default schedule.  (The hot-cache
 // load of hl_build_remap and hl_flush_hot, which run alone, use 2 CTAs per SM and reach 90 % of the memcpy rate.)
-constexpr int kBulkCtas = 8;
+constexpr int kBulkCtasDefault = 8;
+// HOTLINE_MOVER_CTAS in the environment (read once) overrides the count, for tuning on other hosts.
+static int bulk_ctas_setting() {
+    static const int v = [] {
+        const char* e = getenv("HOTLINE_MOVER_CTAS");
+        const int n = e ? atoi(e) : 0;
+        return n >= 1 && n <= 4 * kSMs ? n : kBulkCtasDefault;
+    }();
+    return v;
+}
+#define kBulkCtas bulk_ctas_setting()
 
 template <bool TO_TABLE>
 __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_side, int64_t dense_row0, float* table,

@@ -154,27 +154,34 @@ __global__ void __launch_bounds__(kThreads) k_bwd_pairs(const int32_t* __restric
                                                         const int32_t* __restrict__ d_n_samples, int max_batch,
                                                         int bags_per_sample_all, int64_t n_slots, int64_t max_nnz,
                                                         int32_t* __restrict__ keys, int32_t* __restrict__ vals,
-                                                        int32_t* __restrict__ d_n_lookups, int32_t* status) {
+                                                        int32_t* __restrict__ d_n_lookups,
+                                                        const int32_t* __restrict__ d_pos0, int32_t key_bias,
+                                                        int32_t sentinel, int32_t* __restrict__ d_total,
+                                                        int32_t* status) {
+    // pairs go to positions pos0 + j (pos0 = *d_pos0 or 0) with key = slot + key_bias; *d_n_lookups = this
+    // micro-batch's lookups, *d_total (if given) = pos0 + that
+    const int64_t pos0 = d_pos0 ? d_pos0[0] : 0;
     const int64_t n_bags = (int64_t)clamp_samples(d_n_samples, max_batch) * bags_per_sample_all;
     const int sub = threadIdx.x % GROUP;
     const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / GROUP;
     const int64_t n_groups = (int64_t)gridDim.x * kThreads / GROUP;
     if (group == 0 && sub == 0) {
         int32_t L = offsets[n_bags];
-        if (L > max_nnz) {
+        if (pos0 + L > max_nnz) {
             set_status(status, HL_ECAPACITY);
-            L = (int32_t)max_nnz;
+            L = (int32_t)(max_nnz - pos0);
         }
         d_n_lookups[0] = L;
+        if (d_total) d_total[0] = (int32_t)(pos0 + L);
     }
     for (int64_t bag = group; bag < n_bags; bag += n_groups) {
         const int32_t lo = offsets[bag], hi = offsets[bag + 1];
         for (int32_t j = lo + sub; j < hi; j += GROUP) {
-            if (j >= max_nnz) break;
+            if (pos0 + j >= max_nnz) break;
             const int32_t id = ids[j];
             if (id >= n_slots) set_status(status, HL_EBOUNDS);
-            keys[j] = (id < 0 || id >= n_slots) ? (int32_t)n_slots : id;
-            vals[j] = (int32_t)bag;
+            keys[pos0 + j] = (id < 0 || id >= n_slots) ? sentinel : id + key_bias;
+            vals[pos0 + j] = (int32_t)bag;
         }
     }
 }
@@ -195,11 +202,15 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
                                                          const int32_t* __restrict__ vals,
                                                          const int32_t* __restrict__ d_n_lookups,
                                                          const float* __restrict__ grad_out, int D4, int64_t n_slots,
-                                                         float lr, float* __restrict__ part) {
+                                                         float lr, float* __restrict__ part,
+                                                         const int32_t* __restrict__ d_first, int32_t key_bias) {
+    // the lookups of this call are positions [first, first + *d_n_lookups) of the sorted arrays; their keys are
+    // slot + key_bias
     constexpr int KPL = kBwdChunk / G;                       // pairs held per lane
     constexpr int U = NV >= 4 ? 1 : (NV >= 2 ? 2 : 4);       // lookups in flight per lane
     static_assert(G % U == 0, "batch must divide the group");
-    const int64_t n = d_n_lookups[0];
+    const int64_t first = d_first ? d_first[0] : 0;
+    const int64_t n = first + d_n_lookups[0];
     const int lane = threadIdx.x & 31;
     const int sub = lane % G;
     const unsigned gmask = G == 32 ? 0xffffffffu : (((1u << G) - 1u) << (lane / G * G));
@@ -209,8 +220,8 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
     float4* cache4 = reinterpret_cast<float4*>(cache);
     float4* __restrict__ part4 = reinterpret_cast<float4*>(part);
 
-    for (int64_t chunk = group; chunk * kBwdChunk < n; chunk += n_groups) {
-        const int64_t start = chunk * kBwdChunk;
+    for (int64_t chunk = group; first + chunk * kBwdChunk < n; chunk += n_groups) {
+        const int64_t start = first + chunk * kBwdChunk;
         const int64_t end = min(start + (int64_t)kBwdChunk, n);
         int32_t kk[KPL], vv[KPL];
 #pragma unroll
@@ -219,7 +230,7 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
             kk[i] = p < end ? keys[p] : -1;
             vv[i] = p < end ? vals[p] : 0;
         }
-        const int32_t prev_key = start > 0 ? keys[start - 1] : -3;   // -3: equal to no key
+        const int32_t prev_key = start > first ? keys[start - 1] : -3;   // -3: equal to no key
         const int32_t next_key = end < n ? keys[end] : -2;
 
         int32_t cur = prev_key;        // slot of the segment being summed
@@ -237,7 +248,8 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
         }
 
         auto flush = [&](bool right_open) {
-            if (seg_count == 0 || cur >= n_slots) return;   // nothing summed, or the sentinel of skipped lookups
+            const int64_t row = (int64_t)cur - key_bias;
+            if (seg_count == 0 || row < 0 || row >= n_slots) return;   // nothing summed, or a skipped lookup's sentinel
             if (!seg_left_open && !right_open) {
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
@@ -248,7 +260,7 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
                         w.y -= lr * (float)acc[v][1];
                         w.z -= lr * (float)acc[v][2];
                         w.w -= lr * (float)acc[v][3];
-                        cache4[(int64_t)cur * D4 + c] = w;
+                        cache4[row * D4 + c] = w;
                     }
                 }
             } else {
@@ -278,12 +290,13 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
                 float4 g[U][NV], wn[U][NV];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    const bool ok = k[u] >= 0 && k[u] < n_slots;
+                    const int64_t row = (int64_t)k[u] - key_bias;
+                    const bool ok = k[u] >= 0 && row >= 0 && row < n_slots;
 #pragma unroll
                     for (int v = 0; v < NV; ++v) {
                         const int c = sub + v * G;
                         g[u][v] = (ok && c < D4) ? __ldg(&grad4[(int64_t)b[u] * D4 + c]) : f4_zero();
-                        wn[u][v] = (ok && head[u] && c < D4) ? cache4[(int64_t)k[u] * D4 + c] : f4_zero();
+                        wn[u][v] = (ok && head[u] && c < D4) ? cache4[row * D4 + c] : f4_zero();
                     }
                 }
 #pragma unroll
@@ -322,10 +335,12 @@ __global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cac
 template <int G, int NV>
 __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cache, const int32_t* __restrict__ keys,
                                                         const int32_t* __restrict__ d_n_lookups, int D4,
-                                                        int64_t n_slots, float lr, const float* __restrict__ part) {
+                                                        int64_t n_slots, float lr, const float* __restrict__ part,
+                                                        const int32_t* __restrict__ d_first, int32_t key_bias) {
     constexpr int GW = 32 / G;   // groups per warp
     constexpr int U = NV >= 8 ? 2 : (NV >= 4 ? 4 : (NV >= 2 ? 8 : 16));   // partial sums in flight per lane
-    const int64_t n = d_n_lookups[0];
+    const int64_t first = d_first ? d_first[0] : 0;
+    const int64_t n = first + d_n_lookups[0];
     const int lane = threadIdx.x & 31;
     const int sub = lane % G, gi = lane / G;
     const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
@@ -333,27 +348,28 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
     const float4* __restrict__ part4 = reinterpret_cast<const float4*>(part);
     float4* cache4 = reinterpret_cast<float4*>(cache);
 
-    for (int64_t chunk = warp; chunk * kBwdChunk < n; chunk += n_warps) {
-        const int64_t start = chunk * kBwdChunk;
+    for (int64_t chunk = warp; first + chunk * kBwdChunk < n; chunk += n_warps) {
+        const int64_t start = first + chunk * kBwdChunk;
         const int64_t end = min(start + (int64_t)kBwdChunk, n);
         if (end >= n) continue;
         const int32_t key = keys[end - 1];
-        if (key >= n_slots || keys[end] != key) continue;                         // not right-open
-        if (keys[start] == key && start > 0 && keys[start - 1] == key) continue;    // run started earlier
+        const int64_t row = (int64_t)key - key_bias;
+        if (row < 0 || row >= n_slots || keys[end] != key) continue;                    // not right-open
+        if (keys[start] == key && start > first && keys[start - 1] == key) continue;    // run started earlier
 
         // last chunk that holds a piece of the run: a later chunk lies wholly inside the run iff its last slot is
         // the run's slot
         int64_t last_chunk;
         for (int64_t base = chunk + 1;; base += 32) {
             const int64_t cc = base + lane;
-            const bool in_range = cc * kBwdChunk < n;
-            const int64_t last_pos = min((cc + 1) * (int64_t)kBwdChunk, n) - 1;
+            const bool in_range = first + cc * kBwdChunk < n;
+            const int64_t last_pos = min(first + (cc + 1) * (int64_t)kBwdChunk, n) - 1;
             const bool whole = in_range && keys[last_pos] == key;
             const unsigned m = __ballot_sync(0xffffffffu, whole);
             if (m == 0xffffffffu) continue;
             const int first_not = __ffs(~m) - 1;
             const int64_t cand = base + first_not;   // first chunk not wholly inside the run
-            last_chunk = (cand * kBwdChunk < n && keys[cand * kBwdChunk] == key) ? cand : cand - 1;
+            last_chunk = (first + cand * kBwdChunk < n && keys[first + cand * kBwdChunk] == key) ? cand : cand - 1;
             break;
         }
 
@@ -398,12 +414,12 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
             for (int v = 0; v < NV; ++v) {
                 const int c = sub + v * G;
                 if (c < D4) {
-                    float4 w = cache4[(int64_t)key * D4 + c];
+                    float4 w = cache4[row * D4 + c];
                     w.x -= lr * (float)dacc[v][0];
                     w.y -= lr * (float)dacc[v][1];
                     w.z -= lr * (float)dacc[v][2];
                     w.w -= lr * (float)dacc[v][3];
-                    cache4[(int64_t)key * D4 + c] = w;
+                    cache4[row * D4 + c] = w;
                 }
             }
         }
@@ -428,17 +444,18 @@ int32_t launch_fwd(hl_ctx* ctx, const float* cache, const hl_ubatch* ub, const i
 
 template <int G, int NV>
 int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t* vals, const int32_t* d_n_lookups,
-                   const float* grad, float lr, cudaStream_t stream) {
+                   const float* grad, float lr, cudaStream_t stream, const int32_t* d_first = nullptr,
+                   int32_t key_bias = 0) {
     const int64_t max_chunks = div_up(ctx->max_nnz, kBwdChunk);
     const int grid = grid_for(max_chunks * G, kThreads, kMaxGrid);
     const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 0, stream);
     k_bwd_chunks<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, vals, d_n_lookups, grad, ctx->D / 4, n_slots,
-                                                      lr, ctx->r.bwd_part);
+                                                      lr, ctx->r.bwd_part, d_first, key_bias);
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 1, stream);
     const int span_grid = grid_for(max_chunks * 32, kThreads, kMaxGrid);   // one warp per chunk
     k_bwd_spans<G, NV><<<span_grid, kThreads, 0, stream>>>(cache, keys, d_n_lookups, ctx->D / 4, n_slots, lr,
-                                                          ctx->r.bwd_part);
+                                                          ctx->r.bwd_part, d_first, key_bias);
     note_launches(2);
     HL_LAUNCH_CHECK();
     return HL_OK;
@@ -500,11 +517,11 @@ int32_t sort_lookups(hl_ctx* ctx, const hl_ubatch* ub, const int32_t* d_n_sample
     if (short_bags)
         k_bwd_pairs<1><<<grid_for(ctx->max_bags, kThreads, kMaxGrid), kThreads, 0, stream>>>(
             ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, keys[0], vals[0],
-            d_n_lookups, r.status);
+            d_n_lookups, nullptr, 0, (int32_t)n_slots, nullptr, r.status);
     else
         k_bwd_pairs<32><<<grid_for(ctx->max_bags, kThreads / 32, kMaxGrid), kThreads, 0, stream>>>(
             ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, keys[0], vals[0],
-            d_n_lookups, r.status);
+            d_n_lookups, nullptr, 0, (int32_t)n_slots, nullptr, r.status);
     note_launches(1);
     HL_LAUNCH_CHECK();
     return radix_sort_pairs(keys, vals, d_n_lookups, ctx->max_nnz, key_bits, r.bwd_hist, r.status, out_keys, out_vals,
@@ -540,6 +557,67 @@ extern "C" int32_t hl_embbag_bwd_prepare(hl_ctx* ctx, const hl_ubatch* ub, const
     if (!ub->ids || !d_sorted_slots || !d_sorted_bags) return HL_EINVAL;
     int32_t *keys, *vals;
     return sort_lookups(ctx, ub, d_n_samples, d_sorted_slots, d_sorted_bags, d_n_lookups, &keys, &vals, stream);
+}
+
+extern "C" int32_t hl_embbag_bwd_prepare2(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_n_pop,
+                                          const hl_ubatch* non, const int32_t* d_n_non, int32_t* d_sorted_slots,
+                                          int32_t* d_sorted_bags, int32_t* d_n_lookups, void* stream_) {
+    if (!ctx || !pop || !non || !pop->offsets || !non->offsets || !d_n_pop || !d_n_non || !d_n_lookups)
+        return HL_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (ctx->max_nnz == 0) {
+        HL_CUDA_TRY(cudaMemsetAsync(d_n_lookups, 0, 4 * sizeof(int32_t), stream));
+        return HL_OK;
+    }
+    if (!pop->ids || !non->ids || !d_sorted_slots || !d_sorted_bags) return HL_EINVAL;
+    Regions& r = ctx->r;
+    const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
+    if (2 * n_slots + 1 >= (int64_t(1) << 31)) return HL_EINVAL;
+    const int key_bits = bits_for(2 * n_slots);          // O's keys are slots, X's are n_slots + slot
+    const int passes = (key_bits + 7) / 8;
+    int32_t* keys[2] = {r.bwd_keys[0], r.bwd_keys[1]};
+    int32_t* vals[2] = {r.bwd_vals[0], r.bwd_vals[1]};
+    keys[passes & 1] = d_sorted_slots;
+    vals[passes & 1] = d_sorted_bags;
+    const int32_t sentinel = (int32_t)(2 * n_slots);
+    const bool short_bags = ctx->max_nnz <= 4 * ctx->max_bags;
+    const int per_block = short_bags ? kThreads : kThreads / 32;
+    const int grid = grid_for(ctx->max_bags, per_block, kMaxGrid);
+    const hl_ubatch* ubs[2] = {pop, non};
+    const int32_t* ns[2] = {d_n_pop, d_n_non};
+    for (int m = 0; m < 2; ++m) {
+        const int32_t* pos0 = m == 0 ? nullptr : d_n_lookups;
+        const int32_t bias = m == 0 ? 0 : (int32_t)n_slots;
+        if (short_bags)
+            k_bwd_pairs<1><<<grid, kThreads, 0, stream>>>(ubs[m]->ids, ubs[m]->offsets, ns[m], ctx->max_batch,
+                                                         ctx->T * ctx->S, n_slots, ctx->max_nnz, keys[0], vals[0],
+                                                         d_n_lookups + m, pos0, bias, sentinel, d_n_lookups + 2,
+                                                         r.status);
+        else
+            k_bwd_pairs<32><<<grid, kThreads, 0, stream>>>(ubs[m]->ids, ubs[m]->offsets, ns[m], ctx->max_batch,
+                                                          ctx->T * ctx->S, n_slots, ctx->max_nnz, keys[0], vals[0],
+                                                          d_n_lookups + m, pos0, bias, sentinel, d_n_lookups + 2,
+                                                          r.status);
+    }
+    note_launches(2);
+    HL_LAUNCH_CHECK();
+    int32_t *ok, *ov;
+    return radix_sort_pairs(keys, vals, d_n_lookups + 2, ctx->max_nnz, key_bits, r.bwd_hist, r.status, &ok, &ov, stream);
+}
+
+extern "C" int32_t hl_embbag_bwd_apply2(hl_ctx* ctx, float* d_cache, const int32_t* d_sorted_slots,
+                                        const int32_t* d_sorted_bags, const int32_t* d_n_lookups, int32_t which,
+                                        const float* d_grad_out, float lr, void* stream_) {
+    if (!ctx || !d_cache || !d_n_lookups || !d_grad_out || (which != 0 && which != 1)) return HL_EINVAL;
+    if (ctx->max_nnz == 0) return HL_OK;
+    if (!d_sorted_slots || !d_sorted_bags) return HL_EINVAL;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int32_t* d_first = which == 0 ? nullptr : d_n_lookups;             // X's block starts behind O's
+    const int32_t bias = which == 0 ? 0 : (int32_t)(ctx->hot_cap + ctx->staging_cap);
+#define HL_BWD(G, NV) \
+    launch_bwd<G, NV>(ctx, d_cache, d_sorted_slots, d_sorted_bags, d_n_lookups + which, d_grad_out, lr, stream, d_first, bias)
+    HL_DISPATCH_ROW_SHAPE(ctx->D / 4, HL_BWD);
+#undef HL_BWD
 }
 
 extern "C" int32_t hl_embbag_bwd_apply(hl_ctx* ctx, float* d_cache, const int32_t* d_sorted_slots,

@@ -226,6 +226,9 @@ class _BatchSet:
                            torch.zeros(1, dtype=i32, device=dev))
         self.sorted_non = (torch.zeros(ids_cap, dtype=i32, device=dev), torch.zeros(ids_cap, dtype=i32, device=dev),
                            torch.zeros(1, dtype=i32, device=dev))
+        # the pairs of O and X sorted together (O's block first); [2] = lookups of O, of X, and their sum
+        self.sorted_all = (torch.zeros(ids_cap, dtype=i32, device=dev), torch.zeros(ids_cap, dtype=i32, device=dev),
+                           torch.zeros(4, dtype=i32, device=dev))
 
 
 class PipelinedHotline(Hotline):
@@ -254,12 +257,15 @@ class PipelinedHotline(Hotline):
     """
 
     def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
-                 n_dense: int = 0, device: str = "cuda:0", overlap_link: bool = True, sort_ahead: bool = True):
+                 n_dense: int = 0, device: str = "cuda:0", overlap_link: bool = True, sort_ahead: bool = True,
+                 combined_sort: bool = True):
         self.overlap_link = bool(overlap_link)
         # sort_ahead (with overlap_link): the sorts of the two backward passes, which depend on the ids only, are
         # part of the ahead-work (hl_embbag_bwd_prepare on a side stream); the main stream keeps the forwards and
         # the gradient sums + updates (hl_embbag_bwd_apply)
         self.sort_ahead = bool(sort_ahead) and self.overlap_link
+        # combined_sort (with sort_ahead): one sort over the pairs of O and X (hl_embbag_bwd_prepare2) instead of two
+        self.combined_sort = bool(combined_sort) and self.sort_ahead
         self.window_rows = int(window_rows)
         super().__init__(table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, 2 * self.window_rows,
                          host_table, n_dense=n_dense, device=device)
@@ -301,14 +307,23 @@ class PipelinedHotline(Hotline):
             prev.cold_rows if prev is not None else None, prev.n_cold if prev is not None else None, st.fwd_src,
             sa.cuda_stream))
         st.ev_index.record(sa)
-        sb.wait_event(st.ev_frag)
-        self._timed(timers, "sort_pop", sb, lambda: B.hl_embbag_bwd_prepare(
-            self.ctx, st.pop, st.counts, st.sorted_pop[0], st.sorted_pop[1], st.sorted_pop[2], sb.cuda_stream))
-        st.ev_prep_pop.record(sb)
-        sb.wait_event(st.ev_index)
-        self._timed(timers, "sort_non", sb, lambda: B.hl_embbag_bwd_prepare(
-            self.ctx, st.non, st.counts_non, st.sorted_non[0], st.sorted_non[1], st.sorted_non[2], sb.cuda_stream))
-        st.ev_prep_non.record(sb)
+        if self.combined_sort:
+            sb.wait_event(st.ev_index)
+            self._timed(timers, "sort_all", sb, lambda: B.hl_embbag_bwd_prepare2(
+                self.ctx, st.pop, st.counts, st.non, st.counts_non, st.sorted_all[0], st.sorted_all[1],
+                st.sorted_all[2], sb.cuda_stream))
+            st.ev_prep_pop.record(sb)
+            st.ev_prep_non.record(sb)
+        else:
+            sb.wait_event(st.ev_frag)
+            self._timed(timers, "sort_pop", sb, lambda: B.hl_embbag_bwd_prepare(
+                self.ctx, st.pop, st.counts, st.sorted_pop[0], st.sorted_pop[1], st.sorted_pop[2], sb.cuda_stream))
+            st.ev_prep_pop.record(sb)
+            sb.wait_event(st.ev_index)
+            self._timed(timers, "sort_non", sb, lambda: B.hl_embbag_bwd_prepare(
+                self.ctx, st.non, st.counts_non, st.sorted_non[0], st.sorted_non[1], st.sorted_non[2],
+                sb.cuda_stream))
+            st.ev_prep_non.record(sb)
         lk.wait_event(st.ev_index)
         if j >= 2:
             lk.wait_event(self.sets[(j - 2) % 3].ev_scatter)    # host rows of j-2 are final; its window is free
@@ -336,13 +351,22 @@ class PipelinedHotline(Hotline):
         t = lambda name, stream, fn: self._timed(timers, name, stream, fn)   # noqa: E731
         t("fwd_pop", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.pop, st.counts, st.pooled_pop, s_main))
         m.wait_event(st.ev_prep_pop)
-        t("bwd_pop", m, lambda: B.hl_embbag_bwd_apply(self.ctx, self.cache, st.sorted_pop[0], st.sorted_pop[1],
-                                                      st.sorted_pop[2], grad_pop, lr, s_main))
+        if self.combined_sort:
+            sa_ = st.sorted_all
+            t("bwd_pop", m, lambda: B.hl_embbag_bwd_apply2(self.ctx, self.cache, sa_[0], sa_[1], sa_[2], 0, grad_pop,
+                                                           lr, s_main))
+        else:
+            t("bwd_pop", m, lambda: B.hl_embbag_bwd_apply(self.ctx, self.cache, st.sorted_pop[0], st.sorted_pop[1],
+                                                          st.sorted_pop[2], grad_pop, lr, s_main))
         m.wait_event(st.ev_gather)
         t("fwd_non", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.non, st.counts_non, st.pooled_non, s_main))
         m.wait_event(st.ev_prep_non)
-        t("bwd_non", m, lambda: B.hl_embbag_bwd_apply(self.ctx, self.cache, st.sorted_non[0], st.sorted_non[1],
-                                                      st.sorted_non[2], grad_non, lr, s_main))
+        if self.combined_sort:
+            t("bwd_non", m, lambda: B.hl_embbag_bwd_apply2(self.ctx, self.cache, sa_[0], sa_[1], sa_[2], 1, grad_non,
+                                                           lr, s_main))
+        else:
+            t("bwd_non", m, lambda: B.hl_embbag_bwd_apply(self.ctx, self.cache, st.sorted_non[0], st.sorted_non[1],
+                                                          st.sorted_non[2], grad_non, lr, s_main))
         st.ev_x.record(m)
         self.wb.wait_event(st.ev_x)
         t("scatter_cold", self.wb, lambda: B.hl_scatter_cold_at(

@@ -109,6 +109,15 @@ def test_pipelined_steps_without_sorting_ahead_integer_data():
     assert stats["shared_cold_rows"] > 50
 
 
+def test_pipelined_steps_with_one_sort_per_micro_batch_integer_data():
+    """Sorting ahead with hl_embbag_bwd_prepare / apply per micro-batch instead of the combined sort of O and X."""
+    stats = run_pipelined_check("tiny", steps=6, integer=True, combined_sort=False)
+    assert stats["shared_cold_rows"] > 50
+    spec = dataclasses.replace(gen.CONFIGS["multi_hot"], batch=512, dim=32, rows=("fixed", 2000),
+                               hot_policy=("fraction", 40, 100), profile_batches=2)
+    run_pipelined_check(spec, steps=4, integer=True, combined_sort=False)
+
+
 def test_pipelined_steps_with_serialised_link_integer_data():
     """The default schedule of the pipeline: the next mini-batch's host rows are read after this one's write-back."""
     run_pipelined_check("tiny", steps=6, integer=True, overlap_link=False)
