@@ -364,8 +364,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             k = i % n_batches
             if pipelined:
                 if h.j_submitted == h.j_done:
-                    h.start(*batch_args(k))
-                s = h.step(d_grad, d_grad, lr, next_batch=batch_args((i + 1) % n_batches), timers=timers)
+                    h.start(*batch_args(k), more=[batch_args((i + a) % n_batches) for a in range(1, h.lookahead)])
+                s = h.step(d_grad, d_grad, lr, next_batch=batch_args((i + h.lookahead) % n_batches), timers=timers)
                 return k, h.sets[s]
             h.step(d_idx[k], d_off[k], B, d_grad, d_grad, lr, dense=d_dense[k], timers=timers)
             return k, h
@@ -459,7 +459,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                 # the inputs copied here are those of the mini-batch whose ahead-work this step issues (pipelined)
                 # or of this step's own mini-batch (sequential); the gradients are this step's
                 nonlocal h2d, d2h
-                k = ((cursor[0] + 1) if pipelined else cursor[0]) % n_batches
+                k = ((cursor[0] + h.lookahead) if pipelined else cursor[0]) % n_batches
                 d_idx[k].copy_(h_idx[k], non_blocking=True)
                 d_off[k].copy_(h_off[k], non_blocking=True)
                 h2d_now = h_idx[k].numel() * 4 + h_off[k].numel() * 4 + h_grad.numel() * 4
@@ -733,8 +733,8 @@ def run_sweep(args) -> None:
             i = it[0]
             it[0] += 1
             if h.j_submitted == h.j_done:
-                h.start(*d_in[i % n])
-            return h.sets[h.step(d_grad, d_grad, wl.spec.lr, next_batch=d_in[(i + 1) % n])]
+                h.start(*d_in[i % n], more=[d_in[(i + a) % n] for a in range(1, h.lookahead)])
+            return h.sets[h.step(d_grad, d_grad, wl.spec.lr, next_batch=d_in[(i + h.lookahead) % n])]
 
         pops, colds = [], []
         for _ in range(n):

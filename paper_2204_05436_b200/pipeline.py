@@ -14,6 +14,12 @@ import torch
 from . import binding as B
 
 
+def _side_priority() -> int:
+    """Priority of the streams that carry ahead-work and host-link transfers (-1 = above the main stream's)."""
+    import os
+    return int(os.environ.get("HOTLINE_SIDE_PRIORITY", "-1"))
+
+
 class Hotline:
     def __init__(self, table_rows: Sequence[int], dim: int, bags_per_sample: int, max_batch: int, max_nnz: int,
                  hot_cap_rows: int, staging_cap_rows: int, host_table: torch.Tensor, n_dense: int = 0,
@@ -59,7 +65,7 @@ class Hotline:
         self.pooled_non = torch.zeros((self.max_bags, self.D), dtype=f32, device=dev)
         self.dense_out = torch.zeros((self.max_batch, self.n_dense), dtype=f32, device=dev) if n_dense else None
         self.main = torch.cuda.Stream(device=dev)
-        self.side = torch.cuda.Stream(device=dev)
+        self.side = torch.cuda.Stream(device=dev, priority=_side_priority())
         self.ev_frag = torch.cuda.Event()
         self.ev_gather = torch.cuda.Event()
         self.ev_pop_done = torch.cuda.Event()
@@ -258,7 +264,7 @@ class PipelinedHotline(Hotline):
 
     def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
                  n_dense: int = 0, device: str = "cuda:0", overlap_link: bool = True, sort_ahead: bool = True,
-                 combined_sort: bool = True):
+                 combined_sort: bool = True, lookahead: int = 2):
         self.overlap_link = bool(overlap_link)
         # sort_ahead (with overlap_link): the sorts of the two backward passes, which depend on the ids only, are
         # part of the ahead-work (hl_embbag_bwd_prepare on a side stream); the main stream keeps the forwards and
@@ -266,14 +272,21 @@ class PipelinedHotline(Hotline):
         self.sort_ahead = bool(sort_ahead) and self.overlap_link
         # combined_sort (with sort_ahead): one sort over the pairs of O and X (hl_embbag_bwd_prepare2) instead of two
         self.combined_sort = bool(combined_sort) and self.sort_ahead
+        # lookahead (with sort_ahead): the index-only part of the ahead-work (fragment, cold-row search, sort) runs
+        # this many mini-batches ahead of the main stream; the read of the host rows stays one mini-batch ahead, but
+        # no longer has that index work in front of it.  start() takes lookahead mini-batches, step() the one
+        # lookahead places after the mini-batch it executes.
+        self.lookahead = max(1, int(lookahead)) if self.sort_ahead else 1
         self.window_rows = int(window_rows)
         super().__init__(table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, 2 * self.window_rows,
                          host_table, n_dense=n_dense, device=device)
-        self.sets = [_BatchSet(self) for _ in range(3)]
-        self.sides = [self.side, torch.cuda.Stream(device=self.device)]
-        self.wb = torch.cuda.Stream(device=self.device)
-        self.link = torch.cuda.Stream(device=self.device)
-        self.j_submitted = 0      # mini-batches whose ahead-work has been issued
+        self.n_sets = self.lookahead + 2
+        self.sets = [_BatchSet(self) for _ in range(self.n_sets)]
+        self.sides = [self.side, torch.cuda.Stream(device=self.device, priority=_side_priority())]
+        self.wb = torch.cuda.Stream(device=self.device, priority=_side_priority())
+        self.link = torch.cuda.Stream(device=self.device, priority=_side_priority())
+        self.j_submitted = 0      # mini-batches whose ahead-work (host read included) has been issued
+        self.j_indexed = 0        # sort_ahead schedule: mini-batches whose index-only ahead-work has been issued
         self.j_done = 0           # mini-batches whose main work has been issued
         torch.cuda.synchronize(self.device)
 
@@ -288,16 +301,16 @@ class PipelinedHotline(Hotline):
         b.record(stream)
         timers.setdefault(name, []).append((a, b))
 
-    def _submit_sorted(self, indices, offsets, batch: int, dense=None, timers=None) -> None:
-        """Ahead-work of mini-batch j in the sort_ahead schedule.  Stream A: fragment, cold-row search.  Stream B:
-        the backward sorts of O (after fragment) and X (after the cold-row search).  Link stream: the host read."""
-        j = self.j_submitted
-        st, sa, sb, lk = self.sets[j % 3], self.sides[0], self.sides[1], self.link
-        prev = self.sets[(j - 1) % 3] if j >= 1 else None
+    def _submit_index(self, indices, offsets, batch: int, dense=None, timers=None) -> None:
+        """Index-only ahead-work of the next mini-batch in the sort_ahead schedule.  Stream A: fragment, cold-row
+        search.  Stream B: the backward sorts (after the cold-row search, or O's after fragment)."""
+        j, n = self.j_indexed, self.n_sets
+        st, sa, sb = self.sets[j % n], self.sides[0], self.sides[1]
+        prev = self.sets[(j - 1) % n] if j >= 1 else None
         w = (j % 2) * self.window_rows
         sa.wait_event(st.ev_inputs)
-        if j >= 3:
-            sa.wait_event(st.ev_scatter)                 # the buffers of set j%3 were mini-batch j-3's
+        if j >= n:
+            sa.wait_event(st.ev_scatter)                 # the buffers of this set were mini-batch j-n_sets's
         self._timed(timers, "fragment", sa, lambda: B.hl_fragment(
             self.ctx, self._batch(indices, offsets, batch), dense, self.n_dense if dense is not None else 0,
             st.perm, st.counts, st.pop, st.non, st.dense_out if dense is not None else None, sa.cuda_stream))
@@ -324,9 +337,18 @@ class PipelinedHotline(Hotline):
                 self.ctx, st.non, st.counts_non, st.sorted_non[0], st.sorted_non[1], st.sorted_non[2],
                 sb.cuda_stream))
             st.ev_prep_non.record(sb)
+        self.j_indexed += 1
+
+    def _submit_link(self, timers=None) -> None:
+        """The host read of the oldest indexed mini-batch whose rows are not staged yet (link stream)."""
+        j, n = self.j_submitted, self.n_sets
+        assert j < self.j_indexed
+        st, lk = self.sets[j % n], self.link
+        prev = self.sets[(j - 1) % n] if j >= 1 else None
+        w = (j % 2) * self.window_rows
         lk.wait_event(st.ev_index)
         if j >= 2:
-            lk.wait_event(self.sets[(j - 2) % 3].ev_scatter)    # host rows of j-2 are final; its window is free
+            lk.wait_event(self.sets[(j - 2) % n].ev_scatter)    # host rows of j-2 are final; its window is free
         if prev is not None:
             lk.wait_event(prev.ev_forward)                       # j-1 took what it needs out of this window
         self._timed(timers, "gather_cold", lk, lambda: B.hl_stage_cold(
@@ -336,18 +358,22 @@ class PipelinedHotline(Hotline):
         self.j_submitted += 1
 
     def _step_sorted(self, grad_pop, grad_non, lr, next_batch, timers) -> int:
-        j = self.j_done
-        st, m = self.sets[j % 3], self.main
+        j, n = self.j_done, self.n_sets
+        st, m = self.sets[j % n], self.main
         s_main = m.cuda_stream
         w0, w1 = (j % 2) * self.window_rows, ((j + 1) % 2) * self.window_rows
         if next_batch is not None:
-            self.sets[(j + 1) % 3].ev_inputs.record(m)
+            self.sets[self.j_indexed % n].ev_inputs.record(m)
         m.wait_event(st.ev_index)
         if j >= 1:
             B.hl_forward_cold(self.ctx, self.cache, w1, w0, self.window_rows, st.fwd_src, st.n_cold, s_main)
         st.ev_forward.record(m)
+        if self.j_submitted < self.j_indexed:
+            self._submit_link(timers)                    # mini-batch j+1, indexed during an earlier step
         if next_batch is not None:
-            self._submit_sorted(*next_batch, timers=timers)
+            self._submit_index(*next_batch, timers=timers)
+            if self.j_submitted == j + 1:
+                self._submit_link(timers)                # lookahead 1: j+1 was indexed only just now
         t = lambda name, stream, fn: self._timed(timers, name, stream, fn)   # noqa: E731
         t("fwd_pop", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.pop, st.counts, st.pooled_pop, s_main))
         m.wait_event(st.ev_prep_pop)
@@ -374,11 +400,14 @@ class PipelinedHotline(Hotline):
             self.wb.cuda_stream))
         st.ev_scatter.record(self.wb)
         self.j_done += 1
-        return j % 3
+        return j % n
 
     def _submit(self, indices, offsets, batch: int, dense=None, timers=None) -> None:
         if self.sort_ahead:
-            return self._submit_sorted(indices, offsets, batch, dense, timers)
+            self._submit_index(indices, offsets, batch, dense, timers)
+            if self.j_submitted == self.j_done:
+                self._submit_link(timers)
+            return
         j = self.j_submitted
         st, side = self.sets[j % 3], self.sides[j % 2]
         side.wait_event(st.ev_inputs)                    # the caller prepared the inputs on the main stream
@@ -422,17 +451,24 @@ class PipelinedHotline(Hotline):
             st.ev_gather.record(self.wb)
         self.j_submitted += 1
 
-    def start(self, indices, offsets, batch: int, dense=None) -> None:
+    def start(self, indices, offsets, batch: int, dense=None, more=()) -> None:
+        """Ahead-work of the first mini-batch; ``more`` = the (indices, offsets, batch, dense) tuples of the
+        lookahead - 1 mini-batches after it (fewer if the run is shorter)."""
         assert self.j_submitted == self.j_done, "start() only with nothing in flight"
-        self.sets[self.j_submitted % 3].ev_inputs.record(self.main)
-        self._submit(indices, offsets, batch, dense)
+        assert len(more) <= self.lookahead - 1
+        if self.sort_ahead:
+            self.j_indexed = self.j_submitted
+        for nb in [(indices, offsets, batch, dense)] + [tuple(x) for x in more]:
+            k = self.j_indexed if self.sort_ahead else self.j_submitted
+            self.sets[k % self.n_sets].ev_inputs.record(self.main)
+            self._submit(*nb)
 
     def step(self, grad_pop: torch.Tensor, grad_non: torch.Tensor, lr: float, next_batch=None, timers=None) -> int:
         """Main work of the oldest submitted mini-batch; ``next_batch`` = (indices, offsets, batch, dense) of
-        the one after it (its ahead-work is issued here), or None at the end.  Returns the index of the buffer set
-        that holds this mini-batch's outputs."""
+        the mini-batch ``lookahead`` places after it (its ahead-work is issued here), or None at the end.  Returns
+        the index of the buffer set that holds this mini-batch's outputs."""
         j = self.j_done
-        assert self.j_submitted == j + 1, "call start() first"
+        assert self.j_submitted >= j + 1, "call start() first"
         if self.sort_ahead:
             return self._step_sorted(grad_pop, grad_non, lr, next_batch, timers)
         st, m = self.sets[j % 3], self.main

@@ -212,7 +212,7 @@ def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: boo
 
 def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: bool = True, profile_batches=None,
                         device: str = "cuda:0", overlap_link: bool = True, sort_ahead: bool = True,
-                        combined_sort: bool = True):
+                        combined_sort: bool = True, lookahead: int = 2):
     """Software-pipelined CUDA path (PipelinedHotline) against the oracle processing the same mini-batches one
     after the other.  With integer data every sum is exact, so pooled vectors, the hot cache and the host table
     must agree bit for bit after any number of steps -- which they only do if rows shared by consecutive
@@ -266,7 +266,7 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
     host_table = torch.from_numpy(table0.copy()).pin_memory()
     p = hl.PipelinedHotline(geom.table_rows, D, S, B, max_nnz, hot_cap, window, host_table, n_dense=spec.n_dense,
                             device=device, overlap_link=overlap_link, sort_ahead=sort_ahead,
-                            combined_sort=combined_sort)
+                            combined_sort=combined_sort, lookahead=lookahead)
     got = []
     try:
         with torch.cuda.stream(p.main):
@@ -282,9 +282,10 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
                 gn[:len(g_non)] = _t(g_non, device)
                 d_grads.append((gp, gn))
             torch.cuda.synchronize()
-            p.start(*d_batches[0])
+            ahead = p.lookahead
+            p.start(*d_batches[0], more=d_batches[1:ahead])
             for step in range(steps):
-                nxt = d_batches[step + 1] if step + 1 < steps else None
+                nxt = d_batches[step + ahead] if step + ahead < steps else None
                 s = p.step(d_grads[step][0], d_grads[step][1], lr, next_batch=nxt)
                 st = p.sets[s]
                 got.append((st.perm.clone(), st.counts.clone(), st.pooled_pop.clone(), st.pooled_non.clone(),

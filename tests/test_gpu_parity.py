@@ -109,6 +109,14 @@ def test_pipelined_steps_without_sorting_ahead_integer_data():
     assert stats["shared_cold_rows"] > 50
 
 
+def test_pipelined_steps_with_index_work_one_mini_batch_ahead_integer_data():
+    """lookahead=1: fragment, cold-row search and sort of mini-batch j+1 are issued during mini-batch j (the default
+    issues them during j-1)."""
+    stats = run_pipelined_check("tiny", steps=6, integer=True, lookahead=1)
+    assert stats["shared_cold_rows"] > 50
+    run_pipelined_check("dlrm_small", steps=3, scale_rows=0.02, integer=False, profile_batches=6, lookahead=1)
+
+
 def test_pipelined_steps_with_one_sort_per_micro_batch_integer_data():
     """Sorting ahead with hl_embbag_bwd_prepare / apply per micro-batch instead of the combined sort of O and X."""
     stats = run_pipelined_check("tiny", steps=6, integer=True, combined_sort=False)
