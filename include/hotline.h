@@ -153,6 +153,33 @@ HL_API int32_t hl_profile_hot(hl_ctx* ctx, const hl_batch* b, int32_t reset, int
                        int32_t policy, int64_t p_num, int64_t p_den,
                        int32_t* d_hot_rows, int64_t* d_n_hot, void* stream);
 
+/* Section V-B "Efficient Embedding Tracking" (the access logger as the paper builds it) with the randomizer of
+ * Section V-C: a set-associative table of n_sets x ways blocks, each a row tag (global row id, -1 = empty) and a
+ * 2-bit re-reference prediction value (RRPV), replaced by SRRIP: a hit sets the block's RRPV to 0; a miss takes the
+ * first way, from way 0, whose RRPV is 3 (empty ways hold 3), incrementing every RRPV of the set until there is one,
+ * and inserts the row with RRPV 2.  A row's set is randomizer(row) mod n_sets, the randomizer a 4-round Feistel
+ * network on the 16-bit halves of the row id with round function F_r(x) = upper 16 bits of
+ * (x * 0x9E3779B1 + K_r) mod 2^32, K = {0x85EBCA6B, 0xC2B2AE35, 0x27D4EB2F, 0x165667B1}.  (The paper fixes the
+ * policy, the counter width and the insertion value; associativity, victim order and the rounds are this library's.)
+ * The state lives in caller-owned device arrays d_tags [n_sets*ways] int32 and d_rrpv [n_sets*ways] uint8
+ * (1 <= ways <= 32); d_hits (may be NULL) accumulates the number of hits.
+ *
+ * hl_tracker_reset   empties the logger (and clears *d_hits).
+ * hl_tracker_update  presents every lookup of the mini-batch to the logger; the result is that of serving them one
+ *                    after the other in the order of the layout (position 0 .. nnz-1 of `indices`).  Lookups outside
+ *                    their table are skipped (HL_EBOUNDS).  Scratch: the backward region.
+ * hl_tracker_export  writes what the logger holds into the context's access counters -- counter = 4 - RRPV for a
+ *                    tracked row, 0 for every other row -- after which hl_profile_hot(b = NULL, reset = 0,
+ *                    finalize = 1, ...) selects the popular rows among the tracked ones by its usual rules (all of
+ *                    them if the capacity allows, the most recently re-referenced first otherwise).
+ * None of the three may overlap with other calls on this context. */
+HL_API int32_t hl_tracker_reset(hl_ctx* ctx, int32_t* d_tags, uint8_t* d_rrpv, int64_t n_sets, int32_t ways,
+                                unsigned long long* d_hits, void* stream);
+HL_API int32_t hl_tracker_update(hl_ctx* ctx, const hl_batch* b, int32_t* d_tags, uint8_t* d_rrpv, int64_t n_sets,
+                                 int32_t ways, unsigned long long* d_hits, void* stream);
+HL_API int32_t hl_tracker_export(hl_ctx* ctx, const int32_t* d_tags, const uint8_t* d_rrpv, int64_t n_sets,
+                                 int32_t ways, void* stream);
+
 /* Section IV: popular rows are replicated in GPU memory, the classifier keeps only their indices.
  * Builds the lookup structure for the popular set d_hot_rows[0 .. *d_n_hot) (strictly ascending global ids;
  * any such set is allowed, misclassification never affects fidelity): the cache slot of a popular row is its

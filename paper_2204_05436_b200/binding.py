@@ -21,6 +21,7 @@ EXPORTS = (
     "hl_build_remap", "hl_fragment", "hl_embbag_fwd", "hl_embbag_bwd_sgd", "hl_gather_cold", "hl_scatter_cold",
     "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at", "hl_flush_hot", "hl_index_cold", "hl_stage_cold", "hl_embbag_bwd_prepare", "hl_embbag_bwd_apply",
     "hl_embbag_bwd_prepare2", "hl_embbag_bwd_apply2",
+    "hl_tracker_reset", "hl_tracker_update", "hl_tracker_export",
 )
 
 
@@ -106,6 +107,12 @@ def _load() -> ctypes.CDLL:
     lib.hl_embbag_bwd_prepare2.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, ctypes.POINTER(hl_ubatch), vp, vp, vp, vp, vp]
     lib.hl_embbag_bwd_apply2.restype = i32
     lib.hl_embbag_bwd_apply2.argtypes = [vp, vp, vp, vp, vp, i32, vp, ctypes.c_float, vp]
+    lib.hl_tracker_reset.restype = i32
+    lib.hl_tracker_reset.argtypes = [vp, vp, vp, i64, i32, vp, vp]
+    lib.hl_tracker_update.restype = i32
+    lib.hl_tracker_update.argtypes = [vp, ctypes.POINTER(hl_batch), vp, vp, i64, i32, vp, vp]
+    lib.hl_tracker_export.restype = i32
+    lib.hl_tracker_export.argtypes = [vp, vp, vp, i64, i32, vp]
     lib.hl_flush_hot.restype = i32
     lib.hl_flush_hot.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.hl_embbag_bwd_sgd_static.restype = i32
@@ -346,3 +353,18 @@ def hl_embbag_bwd_apply2(ctx: int, d_cache, d_sorted_slots, d_sorted_bags, d_n_l
     _check("hl_embbag_bwd_apply2", _lib.hl_embbag_bwd_apply2(
         ctx, _ptr(d_cache), _ptr(d_sorted_slots), _ptr(d_sorted_bags), _ptr(d_n_lookups), int(which),
         _ptr(d_grad_out), float(lr), stream))
+
+
+def hl_tracker_reset(ctx: int, d_tags, d_rrpv, n_sets: int, ways: int, d_hits, stream: int) -> None:
+    _check("hl_tracker_reset", _lib.hl_tracker_reset(ctx, _ptr(d_tags), _ptr(d_rrpv), int(n_sets), int(ways),
+                                                     _ptr(d_hits), stream))
+
+
+def hl_tracker_update(ctx: int, batch: hl_batch, d_tags, d_rrpv, n_sets: int, ways: int, d_hits, stream: int) -> None:
+    _check("hl_tracker_update", _lib.hl_tracker_update(ctx, ctypes.byref(batch), _ptr(d_tags), _ptr(d_rrpv),
+                                                       int(n_sets), int(ways), _ptr(d_hits), stream))
+
+
+def hl_tracker_export(ctx: int, d_tags, d_rrpv, n_sets: int, ways: int, stream: int) -> None:
+    _check("hl_tracker_export", _lib.hl_tracker_export(ctx, _ptr(d_tags), _ptr(d_rrpv), int(n_sets), int(ways),
+                                                       stream))

@@ -107,6 +107,28 @@ class Hotline:
         B.hl_profile_hot(self.ctx, b, reset, finalize, policy, p_num, p_den, self.hot_rows, self.n_hot,
                          self.main.cuda_stream)
 
+    def tracker_init(self, n_sets: int, ways: int = 16) -> None:
+        """The approximate access logger (SRRIP table of n_sets x ways row tags) instead of the exact counters:
+        tracker_init, tracker_update per sampled mini-batch, then tracker_select."""
+        self.trk_shape = (int(n_sets), int(ways))
+        self.trk_tags = torch.empty(n_sets * ways, dtype=torch.int32, device=self.device)
+        self.trk_rrpv = torch.empty(n_sets * ways, dtype=torch.uint8, device=self.device)
+        self.trk_hits = torch.zeros(1, dtype=torch.int64, device=self.device)
+        B.hl_tracker_reset(self.ctx, self.trk_tags, self.trk_rrpv, n_sets, ways, self.trk_hits,
+                           self.main.cuda_stream)
+
+    def tracker_update(self, indices: torch.Tensor, offsets: torch.Tensor, batch: int) -> None:
+        n_sets, ways = self.trk_shape
+        B.hl_tracker_update(self.ctx, self._batch(indices, offsets, batch), self.trk_tags, self.trk_rrpv, n_sets,
+                            ways, self.trk_hits, self.main.cuda_stream)
+
+    def tracker_select(self, policy: int = B.HL_HOT_TOPK_ROWS, p_num: int = 0, p_den: int = 1) -> None:
+        """The popular set = the rows the logger holds, clipped by the policy (most recently re-referenced first)."""
+        n_sets, ways = self.trk_shape
+        B.hl_tracker_export(self.ctx, self.trk_tags, self.trk_rrpv, n_sets, ways, self.main.cuda_stream)
+        B.hl_profile_hot(self.ctx, None, False, True, policy, p_num, p_den, self.hot_rows, self.n_hot,
+                         self.main.cuda_stream)
+
     def set_hot_rows(self, rows: torch.Tensor) -> None:
         """Installs a caller-chosen popular set (ascending global ids) instead of a profiled one."""
         n = rows.numel()
