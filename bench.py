@@ -643,6 +643,90 @@ def run_micro_gather(args) -> None:
     hl.hl_host_free(table.data_ptr())
 
 
+def run_micro_tracker(args) -> None:
+    """`--micro tracker`: the approximate access logger (hl_tracker_*) next to the exact counters on the learning
+    phase of the chosen workload (`--workload`, `--profile-batches` mini-batches): time per mini-batch of both, and
+    how much of the exact popular set the logger finds -- for loggers of 1, 2 and 4 M blocks (16 ways; the paper's
+    has 2 M blocks), each asked for 70 % of its blocks, against the exact top rows of the same number."""
+    import torch
+    import paper_2204_05436_b200 as hl
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    spec = gen.CONFIGS["dlrm_large" if args.workload in (None, "auto") else args.workload]
+    geom = gen.make_geometry(spec, 1.0)
+    T, D, S, B = geom.num_tables, spec.dim, geom.bags_per_sample, spec.batch
+    N = int(sum(geom.table_rows))
+    n_bags = T * B * S
+    max_nnz = n_bags if spec.pooling[0] == "one" else n_bags * int(spec.pooling[2])
+    P = args.profile_batches or 64
+    block_counts = [1 << 20, 1 << 21, 1 << 22]
+    hot_cap = int(0.7 * max(block_counts))
+    g = hl.make_geometry(geom.table_rows, D, S)
+    ws_bytes = hl.hl_workspace_bytes(g, B, max_nnz, hot_cap, 0)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    ctx = hl.hl_create(g, B, max_nnz, hot_cap, 0, ws, ws_bytes)
+    stream = torch.cuda.current_stream().cuda_stream
+    base = torch.from_numpy(np.concatenate([[0], np.cumsum(geom.table_rows)]).astype(np.int64)).to(dev)
+    batches = [gen.make_batch(spec, geom, i, args.threads) for i in range(P)]
+    d_in = [(torch.from_numpy(b.indices).to(dev), torch.from_numpy(b.offsets).to(dev)) for b in batches]
+    cnt = torch.zeros(N, dtype=torch.int64, device=dev)        # exact counts kept here too, to weigh the sets
+    for idx, off in d_in:
+        sizes = (off[1:] - off[:-1]).to(torch.int64)
+        table = torch.arange(n_bags, device=dev) // (B * S)
+        rows = base[torch.repeat_interleave(table, sizes)] + idx.to(torch.int64)
+        cnt += torch.bincount(rows, minlength=N)
+    total = float(cnt.sum().item())
+    hot_rows = torch.zeros(hot_cap, dtype=torch.int32, device=dev)
+    n_hot = torch.zeros(1, dtype=torch.int64, device=dev)
+
+    def timed(fn):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3
+
+    def batch_of(i):
+        return hl.make_batch(d_in[i][0], d_in[i][1], B, int(d_in[i][0].numel()))
+
+    exact_us = [timed(lambda i=i: hl.hl_profile_hot(ctx, batch_of(i), int(i == 0), 0, 0, 0, 1, hot_rows, n_hot, stream))
+                for i in range(P)]
+    res = {"micro": "tracker", "workload": spec.name, "total_rows": N, "mini_batches": P, "lookups_per_mini_batch":
+           int(d_in[0][0].numel()), "exact_counter_us_per_mini_batch": statistics.median(exact_us), "loggers": []}
+    exact_sets = {}
+    for blocks in block_counts:
+        k = int(0.7 * blocks)
+        hl.hl_profile_hot(ctx, None, 0, 1, hl.HL_HOT_TOPK_ROWS, k, 1, hot_rows, n_hot, stream)
+        torch.cuda.synchronize()
+        exact_sets[blocks] = hot_rows[:int(n_hot.item())].to(torch.int64).clone()
+    for blocks in block_counts:
+        ways, n_sets, k = 16, blocks // 16, int(0.7 * blocks)
+        tags = torch.empty(blocks, dtype=torch.int32, device=dev)
+        rrpv = torch.empty(blocks, dtype=torch.uint8, device=dev)
+        hits = torch.zeros(1, dtype=torch.int64, device=dev)
+        hl.hl_tracker_reset(ctx, tags, rrpv, n_sets, ways, hits, stream)
+        us = [timed(lambda i=i: hl.hl_tracker_update(ctx, batch_of(i), tags, rrpv, n_sets, ways, hits, stream))
+              for i in range(P)]
+        hl.hl_tracker_export(ctx, tags, rrpv, n_sets, ways, stream)
+        hl.hl_profile_hot(ctx, None, 0, 1, hl.HL_HOT_TOPK_ROWS, k, 1, hot_rows, n_hot, stream)
+        torch.cuda.synchronize()
+        tracked = hot_rows[:int(n_hot.item())].to(torch.int64)
+        exact = exact_sets[blocks]
+        mass_t, mass_e = float(cnt[tracked].sum().item()) / total, float(cnt[exact].sum().item()) / total
+        common = int(torch.isin(tracked, exact).sum().item())
+        res["loggers"].append({
+            "blocks": blocks, "ways": ways, "asked_rows": k, "tracked_rows": int((tags >= 0).sum().item()),
+            "selected_rows": int(tracked.numel()), "exact_rows": int(exact.numel()),
+            "update_us_per_mini_batch": statistics.median(us), "update_us_max": max(us),
+            "hit_rate": float(hits.item()) / (P * d_in[0][0].numel()),
+            "captured_mass": mass_t, "exact_mass": mass_e, "mass_vs_exact": mass_t / mass_e if mass_e else None,
+            "exact_rows_found": common / max(1, int(exact.numel()))})
+    hl.hl_status(ctx)
+    hl.hl_destroy(ctx)
+    print(json.dumps(res), flush=True)
+
+
 def run_micro(args) -> None:
     """`--micro fwd|bwd`: one library call in isolation on an all-popular ("hot-only") micro-batch with the
     DLRM-large-like shape (26 tables x `--micro-batch` inputs, dim 64, one lookup per bag) over a 1 GiB cache.
@@ -813,7 +897,7 @@ def main() -> None:
                     help="pipeline variant in which the host read of the next mini-batch follows this one's write-back "
                          "instead of overlapping it (no forwarding of shared rows needed)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather"],
+    ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather", "tracker"],
                     help="time one library call in isolation")
     ap.add_argument("--micro-dist", default="uniform", choices=["uniform", "zipf"])
     ap.add_argument("--micro-batch", type=int, default=16384)
@@ -822,6 +906,9 @@ def main() -> None:
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+        return
+    if args.micro == "tracker":
+        run_micro_tracker(args)
         return
     if args.micro == "gather":
         run_micro_gather(args)
