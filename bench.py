@@ -393,6 +393,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             dist.barrier()
         timers = {"only": ("fwd_pop", "fwd_non")}   # the roofline kernel's launches; every call is timed further down
         launches0 = hl.hl_launch_count()
+        log(f"[bench] library kernel launches before the timed region: {launches0}")
         clocks = ClockSampler(local_rank)
         clocks.start()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -431,6 +432,20 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             kt["bwd_reduce_non"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_BWD_REDUCE), sizes[k]["L_non"]))
             kt["fwd_non"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_FWD), sizes[k]["L_non"]))
         hl.hl_timing_enable(h.ctx, False)
+        # ---- the roofline kernel with the chip to itself: the forward over the last mini-batch's X again, after
+        # a 256 MB write that leaves nothing of it in the L2 ----
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        alone_us = []
+        for _ in range(10):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(h.main)
+            hl.hl_embbag_fwd(h.ctx, h.cache, _o.non, _o.counts_non, _o.pooled_non, h.main.cuda_stream)
+            b.record(h.main)
+            h.main.synchronize()
+            alone_us.append(a.elapsed_time(b) * 1e3)
+        alone_L, alone_bags = sizes[k]["L_non"], T * sizes[k]["n_non"] * S
+        del flush
         link = {}
         buf_h = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
         buf_d = torch.empty(256 << 20, dtype=torch.uint8, device=device)
@@ -535,6 +550,12 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                     "traffic": (NCU_FWD_TRAFFIC_BYTES_PER_BAG[D] * bags_non if D in NCU_FWD_TRAFFIC_BYTES_PER_BAG else None),
                     "traffic_source": "ncu capture of the hot-only micro case, scaled by bags", "algorithmic_bytes_per_launch": fwd_bytes,
                     "us_per_launch": fwd_us,
+                    "alone": {"note": "the same kernel over one mini-batch's X with no other kernel running, L2 flushed",
+                              "us_per_launch": statistics.median(alone_us),
+                              "achieved": (alone_L * (4 * D + 4) + alone_bags * (4 * D + 4))
+                              / (statistics.median(alone_us) * 1e-6) / 1e9,
+                              "frac": (alone_L * (4 * D + 4) + alone_bags * (4 * D + 4))
+                              / (statistics.median(alone_us) * 1e-6) / 1e9 / peak},
                     "popular_launch": {"algorithmic_bytes_per_launch": pop_bytes, "us_per_launch": pop_us,
                                        "achieved": pop_bytes / (pop_us * 1e-6) / 1e9 if pop_us > 0 else 0.0,
                                        "frac": (pop_bytes / (pop_us * 1e-6) / 1e9 / peak) if pop_us > 0 else 0.0}}
@@ -566,7 +587,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                 "gather_move_gbs": statistics.mean(n * D * 4 / (t * 1e-3) / 1e9 for t, n in kt["gather_move"] if t > 0),
                 "scatter_move_kernel_us": 1e3 * statistics.mean(t for t, _ in kt["scatter_move"]),
                 "scatter_move_gbs": statistics.mean(n * D * 4 / (t * 1e-3) / 1e9 for t, n in kt["scatter_move"] if t > 0),
-                "note": "in-pipeline figures with 8 mover CTAs next to other kernels; `--micro gather` times the same "
+                "note": "in-pipeline figures with 16 mover CTAs (HOTLINE_MOVER_CTAS) next to other kernels; `--micro gather` times the same "
                         "kernel alone with 2 CTAs per SM"},
             "kernels_us": {"bwd_reduce_non": 1e3 * statistics.mean(t for t, _ in kt["bwd_reduce_non"]),
                            "fwd_non": 1e3 * statistics.mean(t for t, _ in kt["fwd_non"])},

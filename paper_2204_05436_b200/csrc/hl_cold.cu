@@ -202,12 +202,14 @@ constexpr int kBulkThreads = 128;
 constexpr int kBulkStages = 2;
 constexpr int kBulkStageBytes = 16384;
 constexpr int kBulkMaxPolls = 1 << 22;
-// CTAs of the mover inside the pipeline.  8 CTAs x 2 stages x 16 KB keep 256 KB of rows in flight: 18 K rows of
-// 256 bytes take 190 us to read and 120 us to write back.  More CTAs move the rows faster (107 us with 148) but
-// the embedding-bag kernels of the other micro-batch, which run next to the mover, lose what it gains: the time per
-// mini-batch stayed within 0.43-0.49 ms for 8 to 148 CTAs, with 8 the best in the default schedule.  (The hot-cache
-// load of hl_build_remap and hl_flush_hot, which run alone, use 2 CTAs per SM and reach 90 % of the memcpy rate.)
-constexpr int kBulkCtasDefault = 8;
+// CTAs of the mover inside the pipeline.  16 CTAs x 16 KB keep 256 KB of rows in flight: 18 K rows of 256 bytes
+// take about 160 us to read and 125 us to write back next to the other streams' kernels.  More CTAs move the rows
+// faster (about 100 us with 2 per SM, alone) but every kernel that runs next to the mover slows down with the
+// number of host-link requests in flight -- with the movers switched off the same mini-batch takes 0.21 instead of
+// 0.31 ms -- and placing all mover CTAs on one GPC (one thread-block cluster) does not change that: 8, 16, 32 and 64
+// CTAs gave 0.335, 0.309, 0.38 and 0.39 ms per mini-batch.  (The hot-cache load of hl_build_remap and hl_flush_hot,
+// which run alone, use 2 CTAs per SM and reach 90 % of the memcpy rate.)
+constexpr int kBulkCtasDefault = 16;
 // HOTLINE_MOVER_CTAS in the environment (read once) overrides the count, for tuning on other hosts.
 static int bulk_ctas_setting() {
     static const int v = [] {

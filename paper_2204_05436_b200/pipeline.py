@@ -304,7 +304,8 @@ class PipelinedHotline(Hotline):
                          host_table, n_dense=n_dense, device=device)
         self.n_sets = self.lookahead + 2
         self.sets = [_BatchSet(self) for _ in range(self.n_sets)]
-        self.sides = [self.side, torch.cuda.Stream(device=self.device, priority=_side_priority())]
+        self.sides = [self.side] + [torch.cuda.Stream(device=self.device, priority=_side_priority())
+                                    for _ in range(2)]
         self.wb = torch.cuda.Stream(device=self.device, priority=_side_priority())
         self.link = torch.cuda.Stream(device=self.device, priority=_side_priority())
         self.j_submitted = 0      # mini-batches whose ahead-work (host read included) has been issued
@@ -324,10 +325,11 @@ class PipelinedHotline(Hotline):
         timers.setdefault(name, []).append((a, b))
 
     def _submit_index(self, indices, offsets, batch: int, dense=None, timers=None) -> None:
-        """Index-only ahead-work of the next mini-batch in the sort_ahead schedule.  Stream A: fragment, cold-row
-        search.  Stream B: the backward sorts (after the cold-row search, or O's after fragment)."""
+        """Index-only ahead-work of the next mini-batch in the sort_ahead schedule.  Stream A: fragment.  Stream C:
+        cold-row search (after fragment).  Stream B: the backward sorts (after the cold-row search, or O's after
+        fragment).  Three streams, so that the three chains of small kernels of successive mini-batches overlap."""
         j, n = self.j_indexed, self.n_sets
-        st, sa, sb = self.sets[j % n], self.sides[0], self.sides[1]
+        st, sa, sb, sc = self.sets[j % n], self.sides[0], self.sides[1], self.sides[2]
         prev = self.sets[(j - 1) % n] if j >= 1 else None
         w = (j % 2) * self.window_rows
         sa.wait_event(st.ev_inputs)
@@ -337,11 +339,14 @@ class PipelinedHotline(Hotline):
             self.ctx, self._batch(indices, offsets, batch), dense, self.n_dense if dense is not None else 0,
             st.perm, st.counts, st.pop, st.non, st.dense_out if dense is not None else None, sa.cuda_stream))
         st.ev_frag.record(sa)
-        self._timed(timers, "index_cold", sa, lambda: B.hl_index_cold(
+        sc.wait_event(st.ev_frag)
+        if j >= n:
+            sc.wait_event(st.ev_scatter)
+        self._timed(timers, "index_cold", sc, lambda: B.hl_index_cold(
             self.ctx, st.non, st.counts_non, w, self.window_rows, st.cold_rows, st.n_cold,
             prev.cold_rows if prev is not None else None, prev.n_cold if prev is not None else None, st.fwd_src,
-            sa.cuda_stream))
-        st.ev_index.record(sa)
+            sc.cuda_stream))
+        st.ev_index.record(sc)
         if self.combined_sort:
             sb.wait_event(st.ev_index)
             self._timed(timers, "sort_all", sb, lambda: B.hl_embbag_bwd_prepare2(
