@@ -87,6 +87,9 @@ def test_geometry_of_the_named_configs():
     assert min(small.table_rows) >= 4 and max(small.table_rows) <= 10_000_000
     assert min(large.table_rows) >= 10 and max(large.table_rows) <= 40_000_000
     assert gen.make_geometry(gen.CONFIGS["tiny"]).base[-1] == 80_000
+    avazu = gen.make_geometry(gen.CONFIGS["avazu_like"])
+    assert avazu.num_tables == 21 and abs(avazu.total_rows - 9.3e6) / 9.3e6 < 0.01
+    assert gen.CONFIGS["avazu_like"].n_dense == 1 and gen.CONFIGS["avazu_like"].dim == 16
 
 
 def test_grad_values_streams():

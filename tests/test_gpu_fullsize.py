@@ -4,7 +4,7 @@ import dataclasses
 import pytest
 
 import gen
-from tests.harness import run_config_check, run_fullsize_check
+from tests.harness import run_config_check, run_fullsize_check, run_pipelined_check
 
 pytestmark = pytest.mark.gpu
 
@@ -26,6 +26,14 @@ def test_dlrm_small_full_size_every_element():
     """26 tables, 33.8 M rows x dim 16, batch 4,096, 256 MB budget, 256 profiling batches: every output element."""
     stats = run_config_check("dlrm_small", steps=1)
     assert stats["N"] > 33_000_000 and stats["n_pop"] > 0
+
+
+def test_avazu_like_full_size_every_element():
+    """21 tables, 9.3 M rows x dim 16, one dense feature, batch 4,096, 128 MB budget: every output element, then
+    three more mini-batches through the pipelined schedule."""
+    stats = run_config_check("avazu_like", steps=1, profile_batches=32)
+    assert abs(stats["N"] - 9.3e6) / 9.3e6 < 0.01 and stats["n_pop"] > 0
+    run_pipelined_check("avazu_like", steps=3, integer=False, profile_batches=8)
 
 
 def test_multi_hot_full_batch_sampled():
