@@ -320,7 +320,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
     pipelined = not args.no_pipeline
     if pipelined:
         h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
-                                n_dense=wl.spec.n_dense, device=str(device), overlap_link=not args.serial_link)
+                                n_dense=wl.spec.n_dense, device=str(device), overlap_link=not args.serial_link,
+                                lookahead=args.lookahead)
     else:
         h = hl.Hotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
                        n_dense=wl.spec.n_dense, device=str(device))
@@ -917,6 +918,8 @@ def main() -> None:
     ap.add_argument("--serial-link", action="store_true",
                     help="pipeline variant in which the host read of the next mini-batch follows this one's write-back "
                          "instead of overlapping it (no forwarding of shared rows needed)")
+    ap.add_argument("--lookahead", type=int, default=2,
+                    help="mini-batches by which the index-only ahead-work of the pipelined schedule runs ahead")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather", "tracker"],
                     help="time one library call in isolation")

@@ -1,6 +1,7 @@
 // The non-popular micro-batch's working set: classify its lookups, find the distinct cold rows, stage them from
 // the host-DRAM table (zero-copy 128-bit loads over the host link) behind the hot cache, and write them back.
 #include "hl_common.cuh"
+#include <cooperative_groups.h>
 #include <cstdlib>
 
 namespace hl {
@@ -73,9 +74,11 @@ __global__ void __launch_bounds__(kThreads) k_cold_assign(const int32_t* __restr
                                                           const int32_t* __restrict__ rank_excl, int64_t slot0,
                                                           int64_t staging_cap, int32_t* __restrict__ ids,
                                                           int32_t* __restrict__ cold_rows,
-                                                          int64_t* __restrict__ d_n_cold, int32_t* status) {
+                                                          int64_t* __restrict__ d_n_cold, int32_t* status,
+                                                          const int32_t* __restrict__ d_n_classified) {
     int64_t n = *d_n;
     n = n < n_max ? n : n_max;
+    if (n == 0 && d_n_classified[0] != 0) return;    // the one-cluster path has done all of this already
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         int64_t distinct = rank_excl[n];
         if (distinct > staging_cap) {
@@ -94,6 +97,199 @@ __global__ void __launch_bounds__(kThreads) k_cold_assign(const int32_t* __restr
             ids[vals[i]] = -1;   // no room to stage this row: the lookup is dropped and the status word says so
         }
     }
+}
+
+// ---- few cold lookups: one thread-block cluster does sort, distinct-row ranking and slot assignment ----------------
+// With at most kSmallCap cold lookups (a DLRM-large mini-batch has about 18 K) the chain of radix passes, head
+// flags, scan and assignment -- nine launches that each take longer to start than to run -- is one kernel of one
+// cluster of 8 CTAs.  CTA c owns positions [c * kSmallPerCta, (c + 1) * kSmallPerCta) of the list.  Every pass ranks
+// the pairs, held in registers, by one digit (per-warp digit counters, as in the tile kernel of the general sort),
+// adds up the digit counts of the 8 CTAs through distributed shared memory, and writes each pair into the shared
+// memory of the CTA that owns its new position.  The sorted list is then ranked and assigned in place.
+// Order of a CTA's items: position = warp * (32 * kSmallItems) + round * 32 + lane.
+// Larger inputs: the kernel hands the count to the general path (*d_n_general = n) and leaves; otherwise it sets
+// *d_n_general = 0, which turns the general path's kernels into no-ops.
+constexpr int kSmallCtas = 8;
+constexpr int kSmallThreads = 256;
+constexpr int kSmallItems = 10;
+constexpr int kSmallPerCta = kSmallThreads * kSmallItems;       // 2560
+constexpr int kSmallCap = kSmallCtas * kSmallPerCta;            // 20480
+constexpr int kSmallWarps = kSmallThreads / 32;
+
+__device__ __forceinline__ int block_scan_small(int v, int* smem33, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int o = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += o;
+    }
+    if (lane == 31) smem33[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const int w = lane < kSmallWarps ? smem33[lane] : 0;
+        int wi = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int o = __shfl_up_sync(0xffffffffu, wi, d);
+            if (lane >= d) wi += o;
+        }
+        if (lane < kSmallWarps) smem33[lane] = wi - w;
+        if (lane == 31) smem33[32] = wi;
+    }
+    __syncthreads();
+    const int res = smem33[warp] + incl - v;
+    total = smem33[32];
+    __syncthreads();
+    return res;
+}
+
+__global__ void __launch_bounds__(kSmallThreads) k_cold_small(const int32_t* __restrict__ keys_in,
+                                                              const int32_t* __restrict__ vals_in,
+                                                              const int32_t* __restrict__ d_n, int64_t n_max,
+                                                              int passes, int64_t slot0, int64_t staging_cap,
+                                                              int32_t* __restrict__ ids,
+                                                              int32_t* __restrict__ cold_rows,
+                                                              int64_t* __restrict__ d_n_cold,
+                                                              int32_t* __restrict__ d_n_general, int32_t* status) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    __shared__ int32_t s_key[kSmallPerCta];
+    __shared__ int32_t s_val[kSmallPerCta];
+    __shared__ uint32_t cnt[kSmallWarps * 256];
+    __shared__ uint32_t cta_hist[256];       // this CTA's digit counts, read by the other CTAs
+    __shared__ uint32_t digit_base[256];
+    __shared__ int cta_heads;                // this CTA's number of run heads, read by the other CTAs
+    __shared__ int scan_smem[33];
+    int64_t n64 = d_n[0];
+    n64 = n64 < 0 ? 0 : (n64 < n_max ? n64 : n_max);
+    const int cta = (int)cluster.block_rank();
+    if (n64 > kSmallCap) {                   // the same decision in all CTAs, before any cluster barrier
+        if (cta == 0 && threadIdx.x == 0) d_n_general[0] = (int32_t)n64;
+        return;
+    }
+    if (cta == 0 && threadIdx.x == 0) d_n_general[0] = 0;
+    const int n = (int)n64;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned lt = lanemask_lt();
+    const int cta_base = cta * kSmallPerCta;
+    const int warp_base = warp * (32 * kSmallItems);
+    int32_t key[kSmallItems];
+    uint32_t aux[kSmallItems];        // low 16 bits: where the pair's value sits in vals_in; high 16: rank in its warp
+#pragma unroll
+    for (int r = 0; r < kSmallItems; ++r) {
+        const int idx = cta_base + warp_base + r * 32 + lane;
+        key[r] = idx < n ? keys_in[idx] : 0x7fffffff;     // padding sorts behind every row id and stays there
+        aux[r] = (uint32_t)idx;
+    }
+    for (int p = 0; p < passes; ++p) {
+        const int shift = 8 * p;
+        for (int i = threadIdx.x; i < kSmallWarps * 256; i += kSmallThreads) cnt[i] = 0;
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < kSmallItems; ++r) {
+            const uint32_t d = ((uint32_t)key[r] >> shift) & 255u;
+            const unsigned peers = __match_any_sync(0xffffffffu, d);
+            const uint32_t before = cnt[warp * 256 + d];
+            __syncwarp();
+            aux[r] = (aux[r] & 0xffffu) | ((before + __popc(peers & lt)) << 16);
+            if ((peers & lt) == 0) cnt[warp * 256 + d] = before + __popc(peers);
+            __syncwarp();
+        }
+        __syncthreads();
+        {   // thread d: prefix of digit d over this CTA's warps; publish the CTA's count
+            const int d = threadIdx.x;
+            uint32_t total = 0;
+#pragma unroll
+            for (int w = 0; w < kSmallWarps; ++w) {
+                const uint32_t c = cnt[w * 256 + d];
+                cnt[w * 256 + d] = total;
+                total += c;
+            }
+            cta_hist[d] = total;
+        }
+        cluster.sync();     // all counts published; all CTAs have taken the previous pass's pairs out of shared memory
+        {
+            const int d = threadIdx.x;
+            uint32_t before_me = 0, all_ctas = 0;
+#pragma unroll
+            for (int c = 0; c < kSmallCtas; ++c) {
+                const uint32_t v = *cluster.map_shared_rank(&cta_hist[d], c);
+                if (c < cta) before_me += v;
+                all_ctas += v;
+            }
+            int whole;
+            const int smaller = block_scan_small((int)all_ctas, scan_smem, whole);     // pairs with a smaller digit
+            digit_base[d] = (uint32_t)smaller + before_me;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < kSmallItems; ++r) {
+            const uint32_t d = ((uint32_t)key[r] >> shift) & 255u;
+            const uint32_t pos = digit_base[d] + cnt[warp * 256 + d] + (aux[r] >> 16);
+            const unsigned owner = pos / kSmallPerCta, off = pos % kSmallPerCta;
+            *cluster.map_shared_rank(&s_key[off], owner) = key[r];
+            *cluster.map_shared_rank(&s_val[off], owner) = (int32_t)(aux[r] & 0xffffu);
+        }
+        cluster.sync();     // every pair has arrived
+#pragma unroll
+        for (int r = 0; r < kSmallItems; ++r) {
+            const int idx = warp_base + r * 32 + lane;
+            key[r] = s_key[idx];
+            aux[r] = (uint32_t)s_val[idx];
+        }
+    }
+    // The sorted pairs are in the CTAs' shared memory (the last barrier above made them visible).  Thread t of CTA c
+    // ranks positions cta_base + [t * kSmallItems, (t + 1) * kSmallItems).
+    const int i0 = threadIdx.x * kSmallItems;
+    int32_t mine[kSmallItems + 1];           // mine[0] = the key before my first position
+    mine[0] = -1;
+    if (i0 > 0) mine[0] = s_key[i0 - 1];
+    else if (cta > 0) mine[0] = *cluster.map_shared_rank(&s_key[kSmallPerCta - 1], cta - 1);
+    int32_t where[kSmallItems];
+    int heads = 0;
+#pragma unroll
+    for (int u = 0; u < kSmallItems; ++u) {
+        const int i = cta_base + i0 + u;
+        mine[u + 1] = s_key[i0 + u];
+        where[u] = i < n ? vals_in[s_val[i0 + u]] : -1;          // the lookup's position in X's ids
+        if (i < n && (i == 0 || mine[u + 1] != mine[u])) ++heads;
+    }
+    int cta_total;
+    int rank = block_scan_small(heads, scan_smem, cta_total);    // heads before my first position, within the CTA
+    if (threadIdx.x == 0) cta_heads = cta_total;
+    cluster.sync();
+    int distinct = 0;
+#pragma unroll
+    for (int c = 0; c < kSmallCtas; ++c) {
+        const int v = *cluster.map_shared_rank(&cta_heads, c);
+        if (c < cta) rank += v;
+        distinct += v;
+    }
+    if (cta == 0 && threadIdx.x == 0) {
+        int64_t dn = distinct;
+        if (dn > staging_cap) {
+            set_status(status, HL_ECAPACITY);
+            dn = staging_cap;
+        }
+        *d_n_cold = dn;
+    }
+#pragma unroll
+    for (int u = 0; u < kSmallItems; ++u) {
+        const int i = cta_base + i0 + u;
+        if (i < n) {
+            const bool head = i == 0 || mine[u + 1] != mine[u];
+            const int my_rank = head ? rank : rank - 1;
+            if (head) ++rank;
+            if (my_rank < staging_cap) {
+                if (head) cold_rows[my_rank] = mine[u + 1];
+                ids[where[u]] = (int32_t)(slot0 + my_rank);
+            } else {
+                ids[where[u]] = -1;     // no room to stage this row: the lookup is dropped, the status word says so
+            }
+        }
+    }
+    cluster.sync();     // no CTA leaves while another may still read its shared memory
 }
 
 // dst[(dst_row0 + i), :] = table[rows[i], :] (or the other way round); G lanes per row, UR rows in flight per
@@ -204,11 +400,15 @@ constexpr int kBulkStageBytes = 16384;
 constexpr int kBulkMaxPolls = 1 << 22;
 // CTAs of the mover inside the pipeline.  16 CTAs x 16 KB keep 256 KB of rows in flight: 18 K rows of 256 bytes
 // take about 160 us to read and 125 us to write back next to the other streams' kernels.  More CTAs move the rows
-// faster (about 100 us with 2 per SM, alone) but every kernel that runs next to the mover slows down with the
-// number of host-link requests in flight -- with the movers switched off the same mini-batch takes 0.21 instead of
-// 0.31 ms -- and placing all mover CTAs on one GPC (one thread-block cluster) does not change that: 8, 16, 32 and 64
-// CTAs gave 0.335, 0.309, 0.38 and 0.39 ms per mini-batch.  (The hot-cache load of hl_build_remap and hl_flush_hot,
-// which run alone, use 2 CTAs per SM and reach 90 % of the memcpy rate.)
+// faster (about 100 us with 2 per SM, alone), fewer slower (one CTA writes back 64 rows every 3.4 us), but what the
+// transfers cost the kernels that run next to them does not depend on that: measured on DLRM-large-like
+// mini-batches, 0.31 ms per mini-batch with both transfers, 0.28 with the write-backs only, 0.22 with the reads only
+// and 0.21 with neither (the last two bound by the host's launch rate) -- the write-back of 4.7 MB costs every
+// concurrent kernel about as much time as the link needs to carry it, whether it is issued by 2, 4 or 16 CTAs, by
+// bulk copies or by plain stores, waiting for each stage to complete or not, spread over the chip or confined to one
+// GPC (all mover CTAs in one thread-block cluster).  8, 16, 32 and 64 CTAs gave 0.335, 0.309, 0.38 and 0.39 ms.
+// (The hot-cache load of hl_build_remap and hl_flush_hot, which run alone, use 2 CTAs per SM and reach 90 % of the
+// memcpy rate.)
 constexpr int kBulkCtasDefault = 16;
 // HOTLINE_MOVER_CTAS in the environment (read once) overrides the count, for tuning on other hosts.
 static int bulk_ctas_setting() {
@@ -395,20 +595,44 @@ int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const f
                                                    r.cold_n, ctx->max_nnz, r.status);
     note_launches(1);
     HL_LAUNCH_CHECK();
-    int32_t *keys, *vals;
-    int32_t st = radix_sort_pairs(r.cold_keys, r.cold_vals, r.cold_n, ctx->max_nnz, bits_for(ctx->N - 1),
-                                  r.cold_hist, r.status, &keys, &vals, stream);
-    if (st != HL_OK) return st;
-    k_cold_heads<<<grid, kThreads, 0, stream>>>(keys, r.cold_n, ctx->max_nnz, r.cold_rank);
+    // up to kSmallCap cold lookups: one cluster; more: the general path, whose count (cold_n[1]) that kernel sets
+    const int key_bits = bits_for(ctx->N - 1);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(kSmallCtas);
+        cfg.blockDim = dim3(kSmallThreads);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kSmallCtas;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        HL_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_cold_small, (const int32_t*)r.cold_keys[0],
+                                       (const int32_t*)r.cold_vals[0], (const int32_t*)r.cold_n, ctx->max_nnz,
+                                       (key_bits + 7) / 8, ctx->hot_cap + stage_row0, stage_rows, non->ids,
+                                       d_cold_rows, d_n_cold, r.cold_n + 1, r.status));
+    }
     note_launches(1);
     HL_LAUNCH_CHECK();
-    st = exclusive_scan_i32(r.cold_rank, r.cold_rank, r.cold_n, ctx->max_nnz, r.cold_tiles, r.status, stream);
-    if (st != HL_OK) return st;
-    k_cold_assign<<<grid, kThreads, 0, stream>>>(keys, vals, r.cold_n, ctx->max_nnz, r.cold_rank,
-                                                 ctx->hot_cap + stage_row0, stage_rows, non->ids, d_cold_rows,
-                                                 d_n_cold, r.status);
-    note_launches(1);
-    HL_LAUNCH_CHECK();
+    int32_t st = HL_OK;
+    if (ctx->max_nnz > kSmallCap) {
+        int32_t *keys, *vals;
+        st = radix_sort_pairs(r.cold_keys, r.cold_vals, r.cold_n + 1, ctx->max_nnz, key_bits, r.cold_hist, r.status,
+                              &keys, &vals, stream);
+        if (st != HL_OK) return st;
+        k_cold_heads<<<grid, kThreads, 0, stream>>>(keys, r.cold_n + 1, ctx->max_nnz, r.cold_rank);
+        note_launches(1);
+        HL_LAUNCH_CHECK();
+        st = exclusive_scan_i32(r.cold_rank, r.cold_rank, r.cold_n + 1, ctx->max_nnz, r.cold_tiles, r.status, stream);
+        if (st != HL_OK) return st;
+        k_cold_assign<<<grid, kThreads, 0, stream>>>(keys, vals, r.cold_n + 1, ctx->max_nnz, r.cold_rank,
+                                                     ctx->hot_cap + stage_row0, stage_rows, non->ids, d_cold_rows,
+                                                     d_n_cold, r.status, r.cold_n);
+        note_launches(1);
+        HL_LAUNCH_CHECK();
+    }
     if (d_prev_rows) {
         k_cold_match<<<grid_for(stage_rows, kThreads, kMaxGrid), kThreads, 0, stream>>>(
             d_cold_rows, d_n_cold, stage_rows, d_prev_rows, d_n_prev, ctx->staging_cap, d_fwd_src);
