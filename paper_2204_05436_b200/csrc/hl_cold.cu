@@ -420,6 +420,15 @@ static int bulk_ctas_setting() {
     return v;
 }
 #define kBulkCtas bulk_ctas_setting()
+// HOTLINE_SCATTER_CTAS: the same for the write-back alone (default: the mover's count).
+static int scatter_ctas_setting() {
+    static const int v = [] {
+        const char* e = getenv("HOTLINE_SCATTER_CTAS");
+        const int n = e ? atoi(e) : 0;
+        return n >= 1 && n <= 4 * kSMs ? n : bulk_ctas_setting();
+    }();
+    return v;
+}
 
 template <bool TO_TABLE>
 __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_side, int64_t dense_row0, float* table,
@@ -731,8 +740,8 @@ extern "C" int32_t hl_scatter_cold_at(hl_ctx* ctx, const float* d_cache, int64_t
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 0, stream);
     const int32_t st = launch_move_rows<true>(const_cast<float*>(d_cache), ctx->hot_cap + stage_row0, host_table,
-                                              d_cold_rows, d_n_cold, stage_rows, ctx->N, ctx->D, nullptr, kBulkCtas,
-                                              ctx->r.status, stream);
+                                              d_cold_rows, d_n_cold, stage_rows, ctx->N, ctx->D, nullptr,
+                                              scatter_ctas_setting(), ctx->r.status, stream);
     timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 1, stream);
     return st;
 }
