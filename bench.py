@@ -493,20 +493,82 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                 h.main.synchronize()
                 h2d, d2h = h2d_now, 16 + B * 4 + (bags_pop + bags_non) * D * 4
 
+            if pipelined:
+                # The copies are pipelined like the work: while mini-batch j executes, the gradients of j+1 and the
+                # indices of j+lookahead come in on one copy stream and the outputs of j-1 go out on another (the
+                # link carries both directions at once).  Every step's inputs and outputs cross the link inside the
+                # timed region; gradients and host output buffers are double-buffered.
+                s_in, s_out, s_cnt = (torch.cuda.Stream(device=device) for _ in range(3))
+                d_grads = [d_grad, torch.empty_like(d_grad)]
+                outs = [(out_pop, out_non, out_counts, out_perm),
+                        (torch.empty_like(out_pop).pin_memory(), torch.empty_like(out_non).pin_memory(),
+                         torch.empty_like(out_counts).pin_memory(), torch.empty_like(out_perm).pin_memory())]
+                ev_in = [torch.cuda.Event() for _ in range(2)]
+                ev_grad_free = [torch.cuda.Event() for _ in range(2)]
+                ev_out = [torch.cuda.Event() for _ in range(2)]
+                ev_done, ev_cnt = torch.cuda.Event(), torch.cuda.Event()
+                for e in ev_grad_free + ev_out:
+                    e.record(h.main)
+                L = h.lookahead
+
+                def e2e_pipe_step(i):
+                    nonlocal h2d, d2h
+                    j = cursor[0]
+                    cursor[0] += 1
+                    kin, g = (j + L) % n_batches, i % 2
+                    with torch.cuda.stream(s_in):
+                        s_in.wait_event(ev_grad_free[g])          # the backward of two steps ago has read this buffer
+                        d_idx[kin].copy_(h_idx[kin], non_blocking=True)
+                        d_off[kin].copy_(h_off[kin], non_blocking=True)
+                        h2d_now = h_idx[kin].numel() * 4 + h_off[kin].numel() * 4 + h_grad.numel() * 4
+                        if d_dense[kin] is not None:
+                            d_dense[kin].copy_(h_dense[kin], non_blocking=True)
+                            h2d_now += h_dense[kin].numel() * 4
+                        d_grads[g].copy_(h_grad, non_blocking=True)
+                        ev_in[g].record(s_in)
+                    h.main.wait_event(ev_in[g])
+                    if h.j_submitted == h.j_done:
+                        h.start(*batch_args(j % n_batches),
+                                more=[batch_args((j + a) % n_batches) for a in range(1, L)])
+                    st = h.sets[h.step(d_grads[g], d_grads[g], lr, next_batch=batch_args(kin))]
+                    ev_grad_free[g].record(h.main)
+                    ev_done.record(h.main)
+                    o_pop, o_non, o_counts, o_perm = outs[g]
+                    ev_out[g].synchronize()                       # the outputs of two steps ago have left this buffer
+                    with torch.cuda.stream(s_cnt):                # sizes of this mini-batch: known since its fragment
+                        s_cnt.wait_event(st.ev_index)
+                        o_counts.copy_(st.counts, non_blocking=True)
+                        ev_cnt.record(s_cnt)
+                    ev_cnt.synchronize()
+                    bags_pop, bags_non = T * int(o_counts[0]) * S, T * int(o_counts[1]) * S
+                    with torch.cuda.stream(s_out):
+                        s_out.wait_event(ev_done)
+                        o_perm.copy_(st.perm[:B], non_blocking=True)
+                        o_pop[:bags_pop].copy_(st.pooled_pop[:bags_pop], non_blocking=True)
+                        o_non[:bags_non].copy_(st.pooled_non[:bags_non], non_blocking=True)
+                        ev_out[g].record(s_out)
+                    h2d, d2h = h2d_now, 16 + B * 4 + (bags_pop + bags_non) * D * 4
+
+                step_fn = e2e_pipe_step
+            else:
+                step_fn = e2e_step
             for i in range(max(3, min(args.warmup, 5))):
-                e2e_step(i)
+                step_fn(i)
             torch.cuda.synchronize()
             if world > 1:
                 dist.barrier()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             finish()
+            torch.cuda.synchronize()
             e0.record(h.main)
             for i in range(args.steps):
-                e2e_step(args.warmup + i)
+                step_fn(args.warmup + i)
             if pipelined:
                 h.main.wait_stream(h.wb)
+                h.main.wait_stream(s_out)
             e1.record(h.main)
             finish()
+            torch.cuda.synchronize()
             e2e_ms = e0.elapsed_time(e1)
             e2e = {"ms_total": e2e_ms, "h2d": h2d, "d2h": d2h}
         h.status()
