@@ -12,12 +12,6 @@ constexpr int kThreads = 256;
 constexpr int kFwdTrips = 4;   // trips of the forward kernel per CTA
 
 __device__ __forceinline__ float4 f4_zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
-__device__ __forceinline__ void f4_add(float4& a, const float4& b) {
-    a.x += b.x;
-    a.y += b.y;
-    a.z += b.z;
-    a.w += b.w;
-}
 
 __device__ __forceinline__ int clamp_samples(const int32_t* d_n_samples, int max_batch) {
     int n = *d_n_samples;
@@ -197,7 +191,7 @@ __global__ void __launch_bounds__(kThreads) k_bwd_pairs(const int32_t* __restric
 // together with the cache row of every run that starts among those U lookups (the row is needed only when the
 // run closes, but asking for it up front takes its latency off the critical path).
 template <int G, int NV>
-__global__ void __launch_bounds__(kThreads) k_bwd_chunks(float* __restrict__ cache,
+__global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float* __restrict__ cache,
                                                          const int32_t* __restrict__ keys,
                                                          const int32_t* __restrict__ vals,
                                                          const int32_t* __restrict__ d_n_lookups,

@@ -103,27 +103,42 @@ __global__ void __launch_bounds__(kThreads) k_scan_chained(const int32_t* in, in
     }
     int total;
     int excl = block_exclusive_scan(s, smem, total);
-    if (threadIdx.x == 0) {
+    if (threadIdx.x < 32) {
+        // warp 0 walks back over the predecessors 32 tiles at a time: lane l looks at tile t0 - l; the sums up to
+        // and including the nearest tile that already knows its inclusive prefix are added
+        const int lane = threadIdx.x;
         long long before = 0;
         if (tile > 0) {
-            st_relaxed64(&st[1 + tile], kFlagAgg64 | (unsigned long long)total);
-            for (int64_t t = tile - 1; t >= 0; --t) {
-                unsigned long long w = 0;
-                int polls = 0;
-                while (((w = ld_relaxed64(&st[1 + t])) & (kFlagAgg64 | kFlagPrefix64)) == 0) {
-                    if (++polls > kMaxPolls) {
-                        set_status(status, HL_ETIMEOUT);
-                        break;
+            if (lane == 0) st_relaxed64(&st[1 + tile], kFlagAgg64 | (unsigned long long)total);
+            bool done = false;
+            for (int64_t t0 = tile - 1; t0 >= 0 && !done; t0 -= 32) {
+                const int64_t t = t0 - lane;
+                unsigned long long w = kFlagPrefix64;            // before tile 0: an empty prefix
+                if (t >= 0) {
+                    int polls = 0;
+                    while (((w = ld_relaxed64(&st[1 + t])) & (kFlagAgg64 | kFlagPrefix64)) == 0) {
+                        if (++polls > kMaxPolls) {               // give up: carry on with what there is
+                            set_status(status, HL_ETIMEOUT);
+                            w = kFlagPrefix64;
+                            break;
+                        }
+                        __nanosleep(20);
                     }
-                    __nanosleep(20);
                 }
-                before += (long long)(w & kValueMask64);
-                if ((w & kFlagPrefix64) || polls > kMaxPolls) break;
+                const unsigned with_prefix = __ballot_sync(0xffffffffu, (w & kFlagPrefix64) != 0);
+                const int stop = with_prefix ? __ffs(with_prefix) - 1 : 31;
+                long long val = lane <= stop ? (long long)(w & kValueMask64) : 0;
+#pragma unroll
+                for (int d = 16; d > 0; d >>= 1) val += __shfl_down_sync(0xffffffffu, val, d);
+                before += __shfl_sync(0xffffffffu, val, 0);
+                done = with_prefix != 0;
             }
         }
-        st_relaxed64(&st[1 + tile], kFlagPrefix64 | (unsigned long long)(before + total));
-        s_excl = before;
-        if (n < tile_base + kScanTile) out[n] = (int32_t)(before + total);
+        if (lane == 0) {
+            st_relaxed64(&st[1 + tile], kFlagPrefix64 | (unsigned long long)(before + total));
+            s_excl = before;
+            if (n < tile_base + kScanTile) out[n] = (int32_t)(before + total);
+        }
     }
     __syncthreads();
     excl += (int)s_excl;

@@ -7,6 +7,7 @@ stream, then the non-popular micro-batch, then the write-back of its cold rows. 
 """
 from __future__ import annotations
 
+import os
 from typing import Optional, Sequence
 
 import torch
@@ -15,8 +16,8 @@ from . import binding as B
 
 
 def _side_priority() -> int:
-    """Priority of the streams that carry ahead-work and host-link transfers (-1 = above the main stream's)."""
-    import os
+    """Priority of the streams that carry ahead-work and host-link transfers (-1 = above the main stream's;
+    HOTLINE_SIDE_PRIORITY in the environment overrides it)."""
     return int(os.environ.get("HOTLINE_SIDE_PRIORITY", "-1"))
 
 
