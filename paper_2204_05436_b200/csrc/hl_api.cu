@@ -58,7 +58,7 @@ size_t carve(char* base, const hl_geometry* g, int64_t N, int32_t max_batch, int
         r->bwd_vals[i] = c.take<int32_t>(nnz);
     }
     r->bwd_hist = c.take<uint32_t>(hist_words(nnz));
-    r->bwd_part = c.take<float>(2 * div_up(nnz, kBwdChunk) * D);
+    r->bwd_part = c.take<float>(2 * div_up(nnz, kBwdChunk) * D + bwd_span_list_words(nnz));
     r->bwd_n = c.take<int32_t>(4);
     for (int i = 0; i < 2; ++i) {
         r->cold_keys[i] = c.take<int32_t>(nnz);

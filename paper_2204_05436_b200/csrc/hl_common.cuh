@@ -158,6 +158,11 @@ constexpr int64_t sort_hist_words(int64_t max_nnz) {
     return 4 * 256 + 8 + 4 * n_tiles * 256;   // digit counts, tickets, tile status words for up to 4 passes
 }
 
+// ints behind the backward's partial sums: count words + (chunk, key) per chunk of kBwdChunk sorted lookups.
+constexpr int64_t bwd_span_list_words(int64_t max_nnz) {
+    return 8 + 2 * (((max_nnz > 0 ? max_nnz : 1) + kBwdChunk - 1) / kBwdChunk);
+}
+
 // ints of scratch exclusive_scan_i32 needs for at most n_max elements (64-bit ticket + status words).
 constexpr int64_t scan_tile_words(int64_t n_max) { return 2 * ((n_max > 0 ? n_max : 1) / kScanTile + 3); }
 

@@ -197,9 +197,12 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
                                                          const int32_t* __restrict__ d_n_lookups,
                                                          const float* __restrict__ grad_out, int D4, int64_t n_slots,
                                                          float lr, float* __restrict__ part,
-                                                         const int32_t* __restrict__ d_first, int32_t key_bias) {
+                                                         const int32_t* __restrict__ d_first, int32_t key_bias,
+                                                         int32_t* __restrict__ span_count,
+                                                         int32_t* __restrict__ span_list) {
     // the lookups of this call are positions [first, first + *d_n_lookups) of the sorted arrays; their keys are
-    // slot + key_bias
+    // slot + key_bias.  A chunk in which a run starts that goes on into the next chunk is appended to span_list
+    // (in any order): k_bwd_spans finishes those runs.
     constexpr int KPL = kBwdChunk / G;                       // pairs held per lane
     constexpr int U = NV >= 4 ? 1 : (NV >= 2 ? 2 : 4);       // lookups in flight per lane
     static_assert(G % U == 0, "batch must divide the group");
@@ -319,103 +322,200 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
             }
         }
         flush(next_key == cur);
+        if (sub == 0 && next_key == cur && !seg_left_open && seg_count > 0) {
+            const int64_t row = (int64_t)cur - key_bias;
+            if (row >= 0 && row < n_slots) {
+                const int32_t pos = atomicAdd(span_count, 1);
+                span_list[2 * pos] = (int32_t)chunk;
+                span_list[2 * pos + 1] = cur;
+            }
+        }
     }
 }
 
 // One WARP per chunk; it acts only if a run STARTS in its chunk and continues into the next one.  The lanes look
-// at the last slot of the next 32 chunks at once to find where the run ends, the warp's 32/G groups add the
-// run's continuation pieces in an interleaved, fixed order in fp64 (runs of many thousands of lookups occur), the
-// group sums are combined by shuffles in a fixed order, and group 0 applies the single SGD update of the row.
+// at the first slot of the next 32 chunks at once to find where the run ends (and, if it goes on, close in on the end
+// with a 32-way search over the rest of the list).  A run of up to kLongRun chunks is summed by its warp: the 32/G
+// groups add the run's continuation pieces in an interleaved, fixed order in fp64 (runs of many thousands of lookups
+// occur), the group sums are combined by shuffles in a fixed order, and group 0 applies the single SGD update of the
+// row.  Longer runs (a popular row can own hundreds of chunks) are queued in shared memory and then summed by the
+// whole CTA, every group taking every (8 * 32/G)-th piece, the group sums combined in a fixed order by one group.
+constexpr int kLongRun = 48;
+
 template <int G, int NV>
 __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cache, const int32_t* __restrict__ keys,
                                                         const int32_t* __restrict__ d_n_lookups, int D4,
                                                         int64_t n_slots, float lr, const float* __restrict__ part,
-                                                        const int32_t* __restrict__ d_first, int32_t key_bias) {
+                                                        const int32_t* __restrict__ d_first, int32_t key_bias,
+                                                        const int32_t* __restrict__ span_count,
+                                                        const int32_t* __restrict__ span_list) {
     constexpr int GW = 32 / G;   // groups per warp
-    constexpr int U = NV >= 8 ? 2 : (NV >= 4 ? 4 : (NV >= 2 ? 8 : 16));   // partial sums in flight per lane
+    constexpr int kWarps = kThreads / 32;
+    constexpr int U = NV >= 4 ? 2 : 4;   // partial sums in flight per lane (most runs end in the next chunk)
+    constexpr int UC = 8;                // the same in the CTA-wide sum
+    constexpr bool kCtaPath = NV == 1;   // the CTA-wide sum keeps one float4 column per lane
+    __shared__ int64_t q_chunk[kWarps], q_last[kWarps], q_row[kWarps];
+    __shared__ double s_sum[kCtaPath ? kThreads : 1][4];
     const int64_t first = d_first ? d_first[0] : 0;
     const int64_t n = first + d_n_lookups[0];
-    const int lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int sub = lane % G, gi = lane / G;
-    const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
-    const int64_t n_warps = ((int64_t)gridDim.x * kThreads) >> 5;
     const float4* __restrict__ part4 = reinterpret_cast<const float4*>(part);
     float4* cache4 = reinterpret_cast<float4*>(cache);
+    const int64_t n_chunks = (n - first + kBwdChunk - 1) / kBwdChunk;
 
-    for (int64_t chunk = warp; first + chunk * kBwdChunk < n; chunk += n_warps) {
-        const int64_t start = first + chunk * kBwdChunk;
-        const int64_t end = min(start + (int64_t)kBwdChunk, n);
-        if (end >= n) continue;
-        const int32_t key = keys[end - 1];
-        const int64_t row = (int64_t)key - key_bias;
-        if (row < 0 || row >= n_slots || keys[end] != key) continue;                    // not right-open
-        if (keys[start] == key && start > first && keys[start - 1] == key) continue;    // run started earlier
+    int64_t n_owned = span_count[0];     // chunks in which a run starts that goes on into the next chunk
+    n_owned = n_owned < 0 ? 0 : (n_owned < n_chunks ? n_owned : n_chunks);
 
-        // last chunk that holds a piece of the run: a later chunk lies wholly inside the run iff its last slot is
-        // the run's slot
-        int64_t last_chunk;
-        for (int64_t base = chunk + 1;; base += 32) {
-            const int64_t cc = base + lane;
-            const bool in_range = first + cc * kBwdChunk < n;
-            const int64_t last_pos = min(first + (cc + 1) * (int64_t)kBwdChunk, n) - 1;
-            const bool whole = in_range && keys[last_pos] == key;
-            const unsigned m = __ballot_sync(0xffffffffu, whole);
-            if (m == 0xffffffffu) continue;
-            const int first_not = __ffs(~m) - 1;
-            const int64_t cand = base + first_not;   // first chunk not wholly inside the run
-            last_chunk = (first + cand * kBwdChunk < n && keys[first + cand * kBwdChunk] == key) ? cand : cand - 1;
-            break;
+    // every warp of the CTA makes the same number of trips (there are block barriers inside)
+    for (int64_t base = (int64_t)blockIdx.x * kWarps; base < n_owned; base += (int64_t)gridDim.x * kWarps) {
+        if (kCtaPath && lane == 0) q_chunk[wib] = -1;
+        bool mine = false;
+        int32_t key = 0;
+        int64_t chunk = 0, row = 0, last_chunk = 0;
+        if (base + wib < n_owned) {
+            const int2 e = reinterpret_cast<const int2*>(span_list)[base + wib];     // (chunk, slot key of the run)
+            chunk = e.x;
+            key = e.y;
+            row = (int64_t)key - key_bias;
+            mine = chunk >= 0 && chunk + 1 < n_chunks && row >= 0 && row < n_slots;
         }
-
-        double dacc[NV][4];
+        // the row and the run's first piece are asked for now; they are needed after the search
+        float4 wrow[NV], piece0[NV];
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             const int c = sub + v * G;
-            const float4 t = (gi == 0 && c < D4) ? part4[(chunk * 2 + 1) * D4 + c] : f4_zero();
-            dacc[v][0] = t.x;
-            dacc[v][1] = t.y;
-            dacc[v][2] = t.z;
-            dacc[v][3] = t.w;
+            const bool ld = mine && gi == 0 && c < D4;
+            wrow[v] = ld ? cache4[row * D4 + c] : f4_zero();
+            piece0[v] = ld ? part4[(chunk * 2 + 1) * D4 + c] : f4_zero();
         }
-        for (int64_t c2 = chunk + 1 + gi; c2 <= last_chunk; c2 += (int64_t)GW * U) {
-            float4 t[U][NV];
+        if (mine) {
+            // last chunk that holds a piece of the run: chunk c > chunk holds one iff its first slot is the run's
+            int64_t lo = chunk + 1, hi = n_chunks;      // chunk lo holds a piece, chunk hi (if any) does not
+            {
+                const int64_t cc = lo + 1 + lane;       // the 32 chunks after lo
+                const bool t = cc < hi && keys[first + cc * kBwdChunk] == key;
+                const unsigned m = __ballot_sync(0xffffffffu, t);
+                const int cnt = __popc(m);              // sorted keys: the lanes that see the run form a prefix
+                lo += cnt;
+                if (cnt < 32) hi = min(hi, lo + 1);
+            }
+            while (hi - lo > 1) {
+                const int64_t step = (hi - lo + 31) / 32;
+                const int64_t cc = lo + (lane + 1) * step;
+                const bool t = cc < hi && keys[first + cc * kBwdChunk] == key;
+                const int cnt = __popc(__ballot_sync(0xffffffffu, t));
+                const int64_t new_hi = min(hi, lo + (cnt + 1) * step);
+                lo += cnt * step;
+                hi = new_hi;
+            }
+            last_chunk = lo;
+            if (kCtaPath && last_chunk - chunk > kLongRun) {
+                if (lane == 0) {
+                    q_chunk[wib] = chunk;
+                    q_last[wib] = last_chunk;
+                    q_row[wib] = row;
+                }
+                mine = false;        // summed by the whole CTA below
+            }
+        }
+        if (mine) {
+            double dacc[NV][4];
 #pragma unroll
-            for (int u = 0; u < U; ++u)
+            for (int v = 0; v < NV; ++v) {
+                dacc[v][0] = piece0[v].x;
+                dacc[v][1] = piece0[v].y;
+                dacc[v][2] = piece0[v].z;
+                dacc[v][3] = piece0[v].w;
+            }
+            for (int64_t c2 = chunk + 1 + gi; c2 <= last_chunk; c2 += (int64_t)GW * U) {
+                float4 t[U][NV];
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        const int c = sub + v * G;
+                        const int64_t cc = c2 + (int64_t)u * GW;
+                        t[u][v] = (cc <= last_chunk && c < D4) ? part4[(cc * 2) * D4 + c] : f4_zero();
+                    }
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) {
+                        dacc[v][0] += (double)t[u][v].x;
+                        dacc[v][1] += (double)t[u][v].y;
+                        dacc[v][2] += (double)t[u][v].z;
+                        dacc[v][3] += (double)t[u][v].w;
+                    }
+            }
+#pragma unroll
+            for (int off = G; off < 32; off <<= 1)
+#pragma unroll
+                for (int v = 0; v < NV; ++v)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) dacc[v][e] += __shfl_xor_sync(0xffffffffu, dacc[v][e], off);
+            if (gi == 0) {
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     const int c = sub + v * G;
-                    const int64_t cc = c2 + (int64_t)u * GW;
-                    t[u][v] = (cc <= last_chunk && c < D4) ? part4[(cc * 2) * D4 + c] : f4_zero();
-                }
-#pragma unroll
-            for (int u = 0; u < U; ++u)
-#pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    dacc[v][0] += (double)t[u][v].x;
-                    dacc[v][1] += (double)t[u][v].y;
-                    dacc[v][2] += (double)t[u][v].z;
-                    dacc[v][3] += (double)t[u][v].w;
-                }
-        }
-#pragma unroll
-        for (int off = G; off < 32; off <<= 1)
-#pragma unroll
-            for (int v = 0; v < NV; ++v)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) dacc[v][e] += __shfl_xor_sync(0xffffffffu, dacc[v][e], off);
-        if (gi == 0) {
-#pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                const int c = sub + v * G;
-                if (c < D4) {
-                    float4 w = cache4[row * D4 + c];
-                    w.x -= lr * (float)dacc[v][0];
-                    w.y -= lr * (float)dacc[v][1];
-                    w.z -= lr * (float)dacc[v][2];
-                    w.w -= lr * (float)dacc[v][3];
-                    cache4[row * D4 + c] = w;
+                    if (c < D4) {
+                        float4 w = wrow[v];
+                        w.x -= lr * (float)dacc[v][0];
+                        w.y -= lr * (float)dacc[v][1];
+                        w.z -= lr * (float)dacc[v][2];
+                        w.w -= lr * (float)dacc[v][3];
+                        cache4[row * D4 + c] = w;
+                    }
                 }
             }
+        }
+        if (kCtaPath) {
+            __syncthreads();
+            for (int qi = 0; qi < kWarps; ++qi) {
+                const int64_t qc = q_chunk[qi];
+                if (qc < 0) continue;                    // the same for all threads
+                const int64_t ql = q_last[qi], qrow = q_row[qi];
+                const int gg = wib * GW + gi;            // this group among the CTA's kWarps * GW groups
+                double d0 = 0.0, d1 = 0.0, d2 = 0.0, d3 = 0.0;
+                for (int64_t c2 = qc + 1 + gg; c2 <= ql; c2 += (int64_t)kWarps * GW * UC) {
+                    float4 t[UC];
+#pragma unroll
+                    for (int u = 0; u < UC; ++u) {
+                        const int64_t cc = c2 + (int64_t)u * kWarps * GW;
+                        t[u] = (cc <= ql && sub < D4) ? part4[(cc * 2) * D4 + sub] : f4_zero();
+                    }
+#pragma unroll
+                    for (int u = 0; u < UC; ++u) {
+                        d0 += (double)t[u].x;
+                        d1 += (double)t[u].y;
+                        d2 += (double)t[u].z;
+                        d3 += (double)t[u].w;
+                    }
+                }
+                s_sum[threadIdx.x][0] = d0;
+                s_sum[threadIdx.x][1] = d1;
+                s_sum[threadIdx.x][2] = d2;
+                s_sum[threadIdx.x][3] = d3;
+                __syncthreads();
+                if (threadIdx.x < G && sub < D4) {       // group 0 of warp 0: lane sub owns column sub
+                    const float4 p = part4[(qc * 2 + 1) * D4 + sub];      // the piece in the run's first chunk
+                    double a0 = p.x, a1 = p.y, a2 = p.z, a3 = p.w;
+                    for (int g2 = 0; g2 < kWarps * GW; ++g2) {
+                        a0 += s_sum[g2 * G + sub][0];
+                        a1 += s_sum[g2 * G + sub][1];
+                        a2 += s_sum[g2 * G + sub][2];
+                        a3 += s_sum[g2 * G + sub][3];
+                    }
+                    float4 w = cache4[qrow * D4 + sub];
+                    w.x -= lr * (float)a0;
+                    w.y -= lr * (float)a1;
+                    w.z -= lr * (float)a2;
+                    w.w -= lr * (float)a3;
+                    cache4[qrow * D4 + sub] = w;
+                }
+                __syncthreads();
+            }
+            __syncthreads();     // every warp has read the whole queue before any warp clears its entry again
         }
     }
 }
@@ -444,12 +544,16 @@ int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t
     const int grid = grid_for(max_chunks * G, kThreads, kMaxGrid);
     const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 0, stream);
+    // the list of chunks whose run goes on sits behind the partial sums: [count (8 ints)] [chunk ids]
+    int32_t* span_count = reinterpret_cast<int32_t*>(ctx->r.bwd_part + 2 * max_chunks * ctx->D);
+    int32_t* span_list = span_count + 8;
+    HL_CUDA_TRY(cudaMemsetAsync(span_count, 0, 8 * sizeof(int32_t), stream));
     k_bwd_chunks<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, vals, d_n_lookups, grad, ctx->D / 4, n_slots,
-                                                      lr, ctx->r.bwd_part, d_first, key_bias);
+                                                      lr, ctx->r.bwd_part, d_first, key_bias, span_count, span_list);
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 1, stream);
     const int span_grid = grid_for(max_chunks * 32, kThreads, kMaxGrid);   // one warp per chunk
     k_bwd_spans<G, NV><<<span_grid, kThreads, 0, stream>>>(cache, keys, d_n_lookups, ctx->D / 4, n_slots, lr,
-                                                          ctx->r.bwd_part, d_first, key_bias);
+                                                          ctx->r.bwd_part, d_first, key_bias, span_count, span_list);
     note_launches(2);
     HL_LAUNCH_CHECK();
     return HL_OK;
@@ -643,7 +747,8 @@ constexpr size_t kStaticPairBytes = align256(size_t(kStaticMaxNnz) * sizeof(int3
 constexpr int64_t kStaticHistWords = sort_hist_words(kStaticMaxNnz);
 constexpr size_t kStaticHistBytes = align256(size_t(kStaticHistWords) * sizeof(uint32_t));
 constexpr size_t kStaticPartBytes =
-    align256(size_t(2) * ((kStaticMaxNnz + kBwdChunk - 1) / kBwdChunk) * kStaticMaxDim * sizeof(float));
+    align256(size_t(2) * ((kStaticMaxNnz + kBwdChunk - 1) / kBwdChunk) * kStaticMaxDim * sizeof(float) +
+             bwd_span_list_words(kStaticMaxNnz) * sizeof(int32_t));
 constexpr size_t kStaticScratchBytes = kStaticHeaderBytes + 4 * kStaticPairBytes + kStaticHistBytes + kStaticPartBytes;
 
 // Lives in every device's copy of the library image from load to exit (about 3 MB).  The name below is only a
