@@ -13,6 +13,12 @@ constexpr int kFwdTrips = 4;   // trips of the forward kernel per CTA
 
 __device__ __forceinline__ float4 f4_zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
 
+// row[0..3] += v, done by the L2 (no value comes back, so nothing waits for the row)
+__device__ __forceinline__ void red_add_f4(float4* p, float4 v) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w)
+                 : "memory");
+}
+
 __device__ __forceinline__ int clamp_samples(const int32_t* d_n_samples, int max_batch) {
     int n = *d_n_samples;
     if (n < 0) n = 0;
@@ -204,7 +210,7 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
     // slot + key_bias.  A chunk in which a run starts that goes on into the next chunk is appended to span_list
     // (in any order): k_bwd_spans finishes those runs.
     constexpr int KPL = kBwdChunk / G;                       // pairs held per lane
-    constexpr int U = NV >= 4 ? 1 : (NV >= 2 ? 2 : 4);       // lookups in flight per lane
+    constexpr int U = NV >= 4 ? 2 : (NV >= 2 ? 4 : (G >= 8 ? 8 : 4));       // lookups in flight per lane
     static_assert(G % U == 0, "batch must divide the group");
     const int64_t first = d_first ? d_first[0] : 0;
     const int64_t n = first + d_n_lookups[0];
@@ -233,16 +239,11 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
         int32_t cur = prev_key;        // slot of the segment being summed
         bool seg_left_open = true;     // it continues a run from the previous chunk (until the slot changes)
         int seg_count = 0;             // lookups of this chunk summed into it so far
-        int32_t last_k = prev_key;     // slot of the previous lookup (to spot run heads)
         // a segment's sum is kept in fp64: a popular row can collect tens of thousands of gradient rows, and the
         // rounding of many fp32 partial sums would show in the updated row
         double acc[NV][4];
-        float4 wrow[NV];
 #pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0.0;
-            wrow[v] = f4_zero();
-        }
+        for (int v = 0; v < NV; ++v) acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0.0;
 
         auto flush = [&](bool right_open) {
             const int64_t row = (int64_t)cur - key_bias;
@@ -251,14 +252,10 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     const int c = sub + v * G;
-                    if (c < D4) {
-                        float4 w = wrow[v];
-                        w.x -= lr * (float)acc[v][0];
-                        w.y -= lr * (float)acc[v][1];
-                        w.z -= lr * (float)acc[v][2];
-                        w.w -= lr * (float)acc[v][3];
-                        cache4[row * D4 + c] = w;
-                    }
+                    if (c < D4)
+                        red_add_f4(&cache4[row * D4 + c],
+                                   make_float4(-(lr * (float)acc[v][0]), -(lr * (float)acc[v][1]),
+                                               -(lr * (float)acc[v][2]), -(lr * (float)acc[v][3])));
                 }
             } else {
                 const int64_t slot = chunk * 2 + (seg_left_open ? 0 : 1);
@@ -276,15 +273,12 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
         for (int i = 0; i < KPL; ++i) {
             for (int j = 0; j < G; j += U) {
                 int32_t k[U], b[U];
-                bool head[U];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     k[u] = __shfl_sync(gmask, kk[i], j + u, G);
                     b[u] = __shfl_sync(gmask, vv[i], j + u, G);
-                    head[u] = k[u] != last_k;
-                    last_k = k[u] >= 0 ? k[u] : last_k;
                 }
-                float4 g[U][NV], wn[U][NV];
+                float4 g[U][NV];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const int64_t row = (int64_t)k[u] - key_bias;
@@ -293,7 +287,6 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
                     for (int v = 0; v < NV; ++v) {
                         const int c = sub + v * G;
                         g[u][v] = (ok && c < D4) ? __ldg(&grad4[(int64_t)b[u] * D4 + c]) : f4_zero();
-                        wn[u][v] = (ok && head[u] && c < D4) ? cache4[row * D4 + c] : f4_zero();
                     }
                 }
 #pragma unroll
@@ -305,10 +298,7 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
                         seg_left_open = false;
                         seg_count = 0;
 #pragma unroll
-                        for (int v = 0; v < NV; ++v) {
-                            acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0.0;
-                            wrow[v] = wn[u][v];
-                        }
+                        for (int v = 0; v < NV; ++v) acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0.0;
                     }
 #pragma unroll
                     for (int v = 0; v < NV; ++v) {
@@ -380,13 +370,12 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
             row = (int64_t)key - key_bias;
             mine = chunk >= 0 && chunk + 1 < n_chunks && row >= 0 && row < n_slots;
         }
-        // the row and the run's first piece are asked for now; they are needed after the search
-        float4 wrow[NV], piece0[NV];
+        // the run's first piece is asked for now; it is needed after the search
+        float4 piece0[NV];
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             const int c = sub + v * G;
             const bool ld = mine && gi == 0 && c < D4;
-            wrow[v] = ld ? cache4[row * D4 + c] : f4_zero();
             piece0[v] = ld ? part4[(chunk * 2 + 1) * D4 + c] : f4_zero();
         }
         if (mine) {
@@ -458,14 +447,10 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
 #pragma unroll
                 for (int v = 0; v < NV; ++v) {
                     const int c = sub + v * G;
-                    if (c < D4) {
-                        float4 w = wrow[v];
-                        w.x -= lr * (float)dacc[v][0];
-                        w.y -= lr * (float)dacc[v][1];
-                        w.z -= lr * (float)dacc[v][2];
-                        w.w -= lr * (float)dacc[v][3];
-                        cache4[row * D4 + c] = w;
-                    }
+                    if (c < D4)
+                        red_add_f4(&cache4[row * D4 + c],
+                                   make_float4(-(lr * (float)dacc[v][0]), -(lr * (float)dacc[v][1]),
+                                               -(lr * (float)dacc[v][2]), -(lr * (float)dacc[v][3])));
                 }
             }
         }
@@ -506,12 +491,8 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
                         a2 += s_sum[g2 * G + sub][2];
                         a3 += s_sum[g2 * G + sub][3];
                     }
-                    float4 w = cache4[qrow * D4 + sub];
-                    w.x -= lr * (float)a0;
-                    w.y -= lr * (float)a1;
-                    w.z -= lr * (float)a2;
-                    w.w -= lr * (float)a3;
-                    cache4[qrow * D4 + sub] = w;
+                    red_add_f4(&cache4[qrow * D4 + sub], make_float4(-(lr * (float)a0), -(lr * (float)a1),
+                                                                     -(lr * (float)a2), -(lr * (float)a3)));
                 }
                 __syncthreads();
             }
