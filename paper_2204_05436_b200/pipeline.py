@@ -393,9 +393,14 @@ class PipelinedHotline(Hotline):
         if next_batch is not None:
             self.sets[self.j_indexed % n].ev_inputs.record(m)
         m.wait_event(st.ev_index)
+        # rows shared with mini-batch j-1 come out of its staging window once its backward is done; on the link
+        # stream, between the host reads of j and of j+1, so that O's work on the main stream does not wait for it
+        lk = self.link
         if j >= 1:
-            B.hl_forward_cold(self.ctx, self.cache, w1, w0, self.window_rows, st.fwd_src, st.n_cold, s_main)
-        st.ev_forward.record(m)
+            lk.wait_event(st.ev_index)
+            lk.wait_event(self.sets[(j - 1) % n].ev_x)
+            B.hl_forward_cold(self.ctx, self.cache, w1, w0, self.window_rows, st.fwd_src, st.n_cold, lk.cuda_stream)
+        st.ev_forward.record(lk)
         if self.j_submitted < self.j_indexed:
             self._submit_link(timers)                    # mini-batch j+1, indexed during an earlier step
         if next_batch is not None:
@@ -413,6 +418,7 @@ class PipelinedHotline(Hotline):
             t("bwd_pop", m, lambda: B.hl_embbag_bwd_apply(self.ctx, self.cache, st.sorted_pop[0], st.sorted_pop[1],
                                                           st.sorted_pop[2], grad_pop, lr, s_main))
         m.wait_event(st.ev_gather)
+        m.wait_event(st.ev_forward)
         t("fwd_non", m, lambda: B.hl_embbag_fwd(self.ctx, self.cache, st.non, st.counts_non, st.pooled_non, s_main))
         m.wait_event(st.ev_prep_non)
         if self.combined_sort:
