@@ -4,7 +4,7 @@
 //
 // The ASIC serves one access after the other; the result depends on that order only within a set.  So the lookups of
 // a mini-batch are keyed by their set and sorted stably (their order within a set stays the order of the layout),
-// and one warp per set replays its accesses in turn, the ways of the set held one per lane.
+// and a warp replays each set's run of the sorted list in turn, the ways of the set held one per lane.
 #include "hl_common.cuh"
 
 namespace hl {
@@ -63,7 +63,9 @@ __global__ void __launch_bounds__(kThreads) k_trk_keys(const int32_t* __restrict
     }
 }
 
-// One warp per set: lane w holds way w.  The set's accesses are the run of key s in the sorted list.
+// One warp per 32 positions of the sorted list: every position where a new set's run begins is a head, and the warp
+// replays, head after head, the accesses of that set (the run may reach far beyond the warp's own 32 positions; the
+// warps there find no head in it and leave it alone).  While a set is replayed lane w holds its way w.
 __global__ void __launch_bounds__(kThreads) k_trk_replay(const int32_t* __restrict__ keys,
                                                          const int32_t* __restrict__ vals,
                                                          const int32_t* __restrict__ d_n, int64_t n_max,
@@ -74,63 +76,66 @@ __global__ void __launch_bounds__(kThreads) k_trk_replay(const int32_t* __restri
     n = n < 0 ? 0 : (n < n_max ? n : n_max);
     const int lane = threadIdx.x & 31;
     const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    for (int64_t s = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); s < n_sets; s += n_warps) {
-        int64_t lo = 0, hi = n;              // first position whose key is >= s (the whole warp searches alike)
-        while (lo < hi) {
-            const int64_t mid = (lo + hi) >> 1;
-            if (keys[mid] < s) lo = mid + 1;
-            else hi = mid;
-        }
-        if (lo >= n || keys[lo] != s) continue;
-        int32_t tag = lane < ways ? tags[s * ways + lane] : -2;          // -2: matches no row
-        int rr = lane < ways ? (int)rrpv[s * ways + lane] : -1;          // -1: never a victim, never aged
-        int32_t last = -1;            // the row of the previous access
-        bool last_zero = false;       // ... which left that row at RRPV 0, so that repeating it changes nothing
-        unsigned long long hits = 0;
-        for (int64_t i = lo;; i += 32) {
-            const bool in = i + lane < n;
-            const int32_t k = in ? keys[i + lane] : -1;
-            const int32_t g = in ? vals[i + lane] : -1;
-            const int cnt = __popc(__ballot_sync(0xffffffffu, k == (int32_t)s));     // sorted: a prefix of the lanes
-            if (last_zero && __all_sync(0xffffffffu, lane >= cnt || g == last)) {
-                hits += cnt;                                                        // a burst of one popular row
-            } else {
-                for (int t = 0; t < cnt; ++t) {
-                    const int32_t gg = __shfl_sync(0xffffffffu, g, t);
-                    if (gg == last && last_zero) {
-                        ++hits;
-                        continue;
-                    }
-                    const unsigned hit = __ballot_sync(0xffffffffu, tag == gg);
-                    if (hit) {
-                        if (lane == __ffs(hit) - 1) rr = 0;
-                        last_zero = true;
-                        ++hits;
-                    } else {
-                        unsigned vm = __ballot_sync(0xffffffffu, rr == kRrpvMax);
-                        if (!vm) {   // age the whole set until its oldest block reaches the maximum
-                            const int add = __ballot_sync(0xffffffffu, rr == 2) ? 1
-                                            : __ballot_sync(0xffffffffu, rr == 1) ? 2 : 3;
-                            if (lane < ways) rr += add;
-                            vm = __ballot_sync(0xffffffffu, rr == kRrpvMax);
+    unsigned long long hits = 0;
+    for (int64_t w0 = ((int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * 32; w0 < n; w0 += n_warps * 32) {
+        const int64_t p = w0 + lane;
+        const int32_t kp = p < n ? keys[p] : -1;
+        const int32_t kprev = (p > 0 && p < n) ? keys[p - 1] : -1;
+        unsigned heads = __ballot_sync(0xffffffffu, p < n && kp >= 0 && kp < n_sets && kp != kprev);
+        while (heads) {
+            const int h = __ffs(heads) - 1;
+            heads &= heads - 1;
+            const int64_t s = __shfl_sync(0xffffffffu, kp, h);
+            int32_t tag = lane < ways ? tags[s * ways + lane] : -2;          // -2: matches no row
+            int rr = lane < ways ? (int)rrpv[s * ways + lane] : -1;          // -1: never a victim, never aged
+            int32_t last = -1;            // the row of the previous access
+            bool last_zero = false;       // ... which left that row at RRPV 0, so that repeating it changes nothing
+            for (int64_t i = w0 + h;; i += 32) {
+                const bool in = i + lane < n;
+                const int32_t k = in ? keys[i + lane] : -1;
+                const int32_t g = in ? vals[i + lane] : -1;
+                const int cnt = __ffs(~__ballot_sync(0xffffffffu, k == (int32_t)s)) - 1;   // leading lanes of the run
+                const int c = cnt < 0 ? 32 : cnt;
+                if (last_zero && __all_sync(0xffffffffu, lane >= c || g == last)) {
+                    hits += c;                                                    // a burst of one popular row
+                } else {
+                    for (int t = 0; t < c; ++t) {
+                        const int32_t gg = __shfl_sync(0xffffffffu, g, t);
+                        if (gg == last && last_zero) {
+                            ++hits;
+                            continue;
                         }
-                        if (lane == __ffs(vm) - 1) {
-                            tag = gg;
-                            rr = kRrpvInsert;
+                        const unsigned hit = __ballot_sync(0xffffffffu, tag == gg);
+                        if (hit) {
+                            if (lane == __ffs(hit) - 1) rr = 0;
+                            last_zero = true;
+                            ++hits;
+                        } else {
+                            unsigned vm = __ballot_sync(0xffffffffu, rr == kRrpvMax);
+                            if (!vm) {   // age the whole set until its oldest block reaches the maximum
+                                const int add = __ballot_sync(0xffffffffu, rr == 2) ? 1
+                                                : __ballot_sync(0xffffffffu, rr == 1) ? 2 : 3;
+                                if (lane < ways) rr += add;
+                                vm = __ballot_sync(0xffffffffu, rr == kRrpvMax);
+                            }
+                            if (lane == __ffs(vm) - 1) {
+                                tag = gg;
+                                rr = kRrpvInsert;
+                            }
+                            last_zero = false;
                         }
-                        last_zero = false;
+                        last = gg;
                     }
-                    last = gg;
                 }
+                if (c < 32) break;
             }
-            if (cnt < 32) break;
+            if (lane < ways) {
+                tags[s * ways + lane] = tag;
+                rrpv[s * ways + lane] = (uint8_t)rr;
+            }
         }
-        if (lane < ways) {
-            tags[s * ways + lane] = tag;
-            rrpv[s * ways + lane] = (uint8_t)rr;
-        }
-        if (lane == 0 && d_hits && hits) atomicAdd(d_hits, hits);
     }
+    if (lane == 0 && d_hits && hits) atomicAdd(d_hits, hits);
 }
 
 // counts[row] = 4 - RRPV for every tracked row (the counters were cleared before).
@@ -201,7 +206,7 @@ extern "C" int32_t hl_tracker_update(hl_ctx* ctx, const hl_batch* b, int32_t* d_
     const int32_t st = radix_sort_pairs(r.bwd_keys, r.bwd_vals, r.bwd_n, ctx->max_nnz, bits_for(n_sets), r.bwd_hist,
                                         r.status, &keys, &vals, stream);
     if (st != HL_OK) return st;
-    k_trk_replay<<<grid_for(n_sets, kThreads / 32, kMaxGrid), kThreads, 0, stream>>>(keys, vals, r.bwd_n, ctx->max_nnz,
+    k_trk_replay<<<grid_for(ctx->max_nnz, kThreads, kMaxGrid), kThreads, 0, stream>>>(keys, vals, r.bwd_n, ctx->max_nnz,
                                                                                     d_tags, d_rrpv, n_sets, ways,
                                                                                     d_hits);
     note_launches(1);
