@@ -319,9 +319,14 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
     T, D, S, B = wl.T, wl.D, wl.S, wl.B
     pipelined = not args.no_pipeline
     if pipelined:
-        h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
-                                n_dense=wl.spec.n_dense, device=str(device), overlap_link=not args.serial_link,
-                                lookahead=args.lookahead)
+        if args.python_pipeline or args.serial_link:
+            h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
+                                    n_dense=wl.spec.n_dense, device=str(device), overlap_link=not args.serial_link,
+                                    lookahead=args.lookahead)
+        else:
+            h = hl.NativePipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap,
+                                          wl.table, n_dense=wl.spec.n_dense, device=str(device),
+                                          lookahead=args.lookahead)
     else:
         h = hl.Hotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
                        n_dense=wl.spec.n_dense, device=str(device))
@@ -364,7 +369,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             cursor[0] += 1
             k = i % n_batches
             if pipelined:
-                if h.j_submitted == h.j_done:
+                if h.idle:
                     h.start(*batch_args(k), more=[batch_args((i + a) % n_batches) for a in range(1, h.lookahead)])
                 s = h.step(d_grad, d_grad, lr, next_batch=batch_args((i + h.lookahead) % n_batches), timers=timers)
                 return k, h.sets[s]
@@ -393,6 +398,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         if world > 1:
             dist.barrier()
         timers = {"only": ("fwd_pop", "fwd_non")}   # the roofline kernel's launches; every call is timed further down
+        if hasattr(h, "prepare_timers"):
+            h.prepare_timers(args.steps)
         launches0 = hl.hl_launch_count()
         log(f"[bench] library kernel launches before the timed region: {launches0}")
         clocks = ClockSampler(local_rank)
@@ -406,7 +413,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             one_step(timers)
         host_enqueue_us = (time.perf_counter() - host_t0) / args.steps * 1e6
         if pipelined:
-            h.main.wait_stream(h.wb)     # the last write-backs belong to the timed work
+            h.wait_outputs()     # the last write-backs belong to the timed work
         ev1.record(h.main)
         finish()
         if world > 1:
@@ -527,7 +534,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                         d_grads[g].copy_(h_grad, non_blocking=True)
                         ev_in[g].record(s_in)
                     h.main.wait_event(ev_in[g])
-                    if h.j_submitted == h.j_done:
+                    if h.idle:
                         h.start(*batch_args(j % n_batches),
                                 more=[batch_args((j + a) % n_batches) for a in range(1, L)])
                     st = h.sets[h.step(d_grads[g], d_grads[g], lr, next_batch=batch_args(kin))]
@@ -536,7 +543,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                     o_pop, o_non, o_counts, o_perm = outs[g]
                     ev_out[g].synchronize()                       # the outputs of two steps ago have left this buffer
                     with torch.cuda.stream(s_cnt):                # sizes of this mini-batch: known since its fragment
-                        s_cnt.wait_event(st.ev_index)
+                        h.wait_counts(s_cnt)
                         o_counts.copy_(st.counts, non_blocking=True)
                         ev_cnt.record(s_cnt)
                     ev_cnt.synchronize()
@@ -564,7 +571,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             for i in range(args.steps):
                 step_fn(args.warmup + i)
             if pipelined:
-                h.main.wait_stream(h.wb)
+                h.wait_outputs()
                 h.main.wait_stream(s_out)
             e1.record(h.main)
             finish()
@@ -635,7 +642,9 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                              f"({(2 * wl.n_bags * D * 4 + fwd_bytes) / 2**20:.0f} MB of pooled vectors, gradients and rows)"
                              if 2 * wl.n_bags * D * 4 > L2_BYTES else
                              "per-step working set is smaller than L2 on this workload; batches rotate over 8 buffers",
-                       "schedule": ("software-pipelined across mini-batches (PipelinedHotline"
+                       "schedule": ("software-pipelined across mini-batches ("
+                                    + ("PipelinedHotline, issued from Python" if args.python_pipeline or
+                                       args.serial_link else "hl_pipe_*, issued by the library")
                                     + (", host reads after write-backs)" if args.serial_link else
                                        ", host reads overlap write-backs, shared rows forwarded)")
                                     if pipelined else "one mini-batch after the other (Hotline.step)"),
@@ -900,7 +909,7 @@ def run_sweep(args) -> None:
         def step():
             i = it[0]
             it[0] += 1
-            if h.j_submitted == h.j_done:
+            if h.idle:
                 h.start(*d_in[i % n], more=[d_in[(i + a) % n] for a in range(1, h.lookahead)])
             return h.sets[h.step(d_grad, d_grad, wl.spec.lr, next_batch=d_in[(i + h.lookahead) % n])]
 
@@ -917,7 +926,7 @@ def run_sweep(args) -> None:
         e0.record(h.main)
         for _ in range(60):
             step()
-        h.main.wait_stream(h.wb)
+        h.wait_outputs()
         e1.record(h.main)
         h.drain()
         h.status()
@@ -935,8 +944,8 @@ def run_sweep(args) -> None:
         return int(h.n_hot.item())
 
     # (1) budget / ratio sweep
-    h = hl.PipelinedHotline(wl.geom.table_rows, D, S, wl.B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
-                            n_dense=wl.spec.n_dense, device=str(device))
+    h = hl.NativePipelinedHotline(wl.geom.table_rows, D, S, wl.B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
+                                  n_dense=wl.spec.n_dense, device=str(device))
     with torch.cuda.stream(h.main):
         for div in (1, 2, 4, 16, 64):
             n_hot = learn(h, max(1, wl.hot_cap // div))
@@ -950,9 +959,9 @@ def run_sweep(args) -> None:
         batches = [gen.make_batch(spec, wl.geom, 100_000 + i, args.threads) for i in range(8)]
         n_bags = T * B * S
         mb = max(B, wl.B)
-        h = hl.PipelinedHotline(wl.geom.table_rows, D, S, mb, T * mb * S if wl.spec.pooling[0] == "one" else
-                                T * mb * S * int(wl.spec.pooling[2]), wl.hot_cap, wl.staging_cap, wl.table,
-                                n_dense=wl.spec.n_dense, device=str(device))
+        h = hl.NativePipelinedHotline(wl.geom.table_rows, D, S, mb, T * mb * S if wl.spec.pooling[0] == "one" else
+                                      T * mb * S * int(wl.spec.pooling[2]), wl.hot_cap, wl.staging_cap, wl.table,
+                                      n_dense=wl.spec.n_dense, device=str(device))
         with torch.cuda.stream(h.main):
             n_hot = learn(h, wl.hot_cap)
             measure(h, batches, B, n_bags, dict(sweep="batch", budget_fraction=1.0, hot_rows=n_hot))
@@ -982,6 +991,9 @@ def main() -> None:
                          "instead of overlapping it (no forwarding of shared rows needed)")
     ap.add_argument("--lookahead", type=int, default=2,
                     help="mini-batches by which the index-only ahead-work of the pipelined schedule runs ahead")
+    ap.add_argument("--python-pipeline", action="store_true",
+                    help="issue the pipelined schedule from Python (PipelinedHotline) instead of the library's own "
+                         "scheduler (hl_pipe_*); gives a time for every call in breakdown_us")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather", "tracker"],
                     help="time one library call in isolation")

@@ -318,6 +318,68 @@ HL_API int32_t hl_scatter_cold_at(hl_ctx* ctx, const float* d_cache, int64_t sta
                                   const int32_t* d_cold_rows, const int64_t* d_n_cold, float* host_table,
                                   void* stream);
 
+/* ---------------------------------------------------------------------------------------------------------
+ * The pipelined schedule, issued from native code (Section IV: gathering the non-popular working parameters is
+ * pipelined with the execution of the popular micro-batch; here the pipeline also spans mini-batches)
+ * ------------------------------------------------------------------------------------------------------- */
+
+/* Buffers of one mini-batch in flight; all device memory, caller-owned, sized like the arguments of the calls
+ * they are passed to (perm [max_batch]; counts [4]; pop / non as for hl_fragment; cold_rows, fwd_src [window_rows];
+ * n_cold [1]; pooled_* [T*max_batch*S, D]; dense_out [max_batch, n_dense] or NULL; sorted_slots / sorted_bags
+ * [max_nnz]; sorted_n [4]). */
+typedef struct {
+    int32_t*  perm;
+    int32_t*  counts;
+    hl_ubatch pop, non;
+    int32_t*  cold_rows;
+    int64_t*  n_cold;
+    int32_t*  fwd_src;
+    float*    pooled_pop;
+    float*    pooled_non;
+    float*    dense_out;
+    int32_t*  sorted_slots;
+    int32_t*  sorted_bags;
+    int32_t*  sorted_n;
+} hl_pipe_set;
+
+typedef struct hl_pipe hl_pipe;
+
+/* A software pipeline over mini-batches on the context `ctx` (which it then uses exclusively): while mini-batch j
+ * executes on `main_stream`, the index-only work of mini-batch j + n_sets - 2 (hl_fragment, hl_index_cold,
+ * hl_embbag_bwd_prepare2), the host read of j + 1 (hl_stage_cold) and the write-back of j - 1 (hl_scatter_cold_at)
+ * run on streams the pipeline creates; rows that consecutive mini-batches share are forwarded between the two
+ * staging windows (hl_forward_cold).  The results are those of processing the mini-batches one after the other.
+ * d_cache [hot_cap + staging_cap, D] with staging_cap >= 2 * window_rows; host_table as for hl_gather_cold;
+ * sets[n_sets] (3 <= n_sets <= 16) are copied.  No device memory is allocated; streams and events are.
+ * Returns NULL on invalid arguments or if a stream or event cannot be created. */
+HL_API hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows, int32_t n_sets,
+                               const hl_pipe_set* sets, int32_t n_dense, void* main_stream);
+HL_API void hl_pipe_destroy(hl_pipe* p);
+
+/* Queues the ahead-work of the next mini-batch (its inputs must be complete in main_stream's order at the time of
+ * the call; d_dense may be NULL).  Call it n_sets - 2 times before the first hl_pipe_step; afterwards pass the next
+ * mini-batch to hl_pipe_step instead.  HL_ECAPACITY if every buffer set is in flight. */
+HL_API int32_t hl_pipe_submit(hl_pipe* p, const hl_batch* b, const float* d_dense);
+
+/* Queues the main work of the oldest submitted mini-batch: forward and update of O, forward and update of X with the
+ * upstream gradients d_grad_pop / d_grad_non ([bags of O, D] / [bags of X, D], in the micro-batches' bag order), and
+ * its write-back; and the ahead-work of `next` (may be NULL).  *set_index = which of the sets holds this mini-batch's
+ * perm, counts and pooled vectors; they are complete in main_stream's order, and the set is reused n_sets steps on.
+ * No call waits for the device. */
+HL_API int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float* d_grad_non, float lr,
+                            const hl_batch* next, const float* d_next_dense, int32_t* set_index);
+
+/* Measurement aid: the next hl_pipe_step (only that one) records these caller-owned events (cudaEvent_t, any may be
+ * NULL) on main_stream before and after the forward over O and before and after the forward over X. */
+HL_API int32_t hl_pipe_time_forward(hl_pipe* p, void* pop_begin, void* pop_end, void* non_begin, void* non_end);
+/* Makes `stream` wait for the write-back of the last mini-batch stepped (device-side wait). */
+HL_API int32_t hl_pipe_wait_outputs(hl_pipe* p, void* stream);
+/* Makes `stream` wait until perm and counts of the last mini-batch stepped are final (they are, long before its main
+ * work: hl_fragment runs n_sets - 2 mini-batches ahead). */
+HL_API int32_t hl_pipe_wait_counts(hl_pipe* p, void* stream);
+/* Host waits until everything queued so far has finished. */
+HL_API int32_t hl_pipe_drain(hl_pipe* p);
+
 /* No counterpart in the paper: an addition for callers that cannot allocate.
  *
  * Some callers have no way to hand the library a workspace: code that runs where device allocation is forbidden

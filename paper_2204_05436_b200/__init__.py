@@ -6,4 +6,4 @@ loudly if it has not been built (``python paper_2204_05436_b200/csrc/build.py``)
 """
 from . import binding  # noqa: F401  (loads the shared library)
 from .binding import *  # noqa: F401,F403
-from .pipeline import Hotline, PipelinedHotline  # noqa: F401
+from .pipeline import Hotline, NativePipelinedHotline, PipelinedHotline  # noqa: F401

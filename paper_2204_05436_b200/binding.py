@@ -22,6 +22,7 @@ EXPORTS = (
     "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at", "hl_flush_hot", "hl_index_cold", "hl_stage_cold", "hl_embbag_bwd_prepare", "hl_embbag_bwd_apply",
     "hl_embbag_bwd_prepare2", "hl_embbag_bwd_apply2",
     "hl_tracker_reset", "hl_tracker_update", "hl_tracker_export",
+    "hl_pipe_create", "hl_pipe_destroy", "hl_pipe_submit", "hl_pipe_step", "hl_pipe_wait_outputs", "hl_pipe_drain", "hl_pipe_time_forward", "hl_pipe_wait_counts",
 )
 
 
@@ -43,6 +44,13 @@ class hl_batch(ctypes.Structure):
 
 class hl_ubatch(ctypes.Structure):
     _fields_ = [("offsets", ctypes.c_void_p), ("ids", ctypes.c_void_p), ("cap_ids", ctypes.c_int64)]
+
+
+class hl_pipe_set(ctypes.Structure):
+    _fields_ = [("perm", ctypes.c_void_p), ("counts", ctypes.c_void_p), ("pop", hl_ubatch), ("non", hl_ubatch),
+                ("cold_rows", ctypes.c_void_p), ("n_cold", ctypes.c_void_p), ("fwd_src", ctypes.c_void_p),
+                ("pooled_pop", ctypes.c_void_p), ("pooled_non", ctypes.c_void_p), ("dense_out", ctypes.c_void_p),
+                ("sorted_slots", ctypes.c_void_p), ("sorted_bags", ctypes.c_void_p), ("sorted_n", ctypes.c_void_p)]
 
 
 def _load() -> ctypes.CDLL:
@@ -113,6 +121,22 @@ def _load() -> ctypes.CDLL:
     lib.hl_tracker_update.argtypes = [vp, ctypes.POINTER(hl_batch), vp, vp, i64, i32, vp, vp]
     lib.hl_tracker_export.restype = i32
     lib.hl_tracker_export.argtypes = [vp, vp, vp, i64, i32, vp]
+    lib.hl_pipe_create.restype = vp
+    lib.hl_pipe_create.argtypes = [vp, vp, vp, i64, i32, ctypes.POINTER(hl_pipe_set), i32, vp]
+    lib.hl_pipe_destroy.restype = None
+    lib.hl_pipe_destroy.argtypes = [vp]
+    lib.hl_pipe_submit.restype = i32
+    lib.hl_pipe_submit.argtypes = [vp, ctypes.POINTER(hl_batch), vp]
+    lib.hl_pipe_step.restype = i32
+    lib.hl_pipe_step.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.POINTER(hl_batch), vp, ctypes.POINTER(i32)]
+    lib.hl_pipe_wait_outputs.restype = i32
+    lib.hl_pipe_wait_outputs.argtypes = [vp, vp]
+    lib.hl_pipe_drain.restype = i32
+    lib.hl_pipe_drain.argtypes = [vp]
+    lib.hl_pipe_wait_counts.restype = i32
+    lib.hl_pipe_wait_counts.argtypes = [vp, vp]
+    lib.hl_pipe_time_forward.restype = i32
+    lib.hl_pipe_time_forward.argtypes = [vp, vp, vp, vp, vp]
     lib.hl_flush_hot.restype = i32
     lib.hl_flush_hot.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.hl_embbag_bwd_sgd_static.restype = i32
@@ -368,3 +392,47 @@ def hl_tracker_update(ctx: int, batch: hl_batch, d_tags, d_rrpv, n_sets: int, wa
 def hl_tracker_export(ctx: int, d_tags, d_rrpv, n_sets: int, ways: int, stream: int) -> None:
     _check("hl_tracker_export", _lib.hl_tracker_export(ctx, _ptr(d_tags), _ptr(d_rrpv), int(n_sets), int(ways),
                                                        stream))
+
+
+def hl_pipe_create(ctx: int, d_cache, host_table, window_rows: int, sets, n_dense: int, main_stream: int) -> int:
+    """``sets``: a list of hl_pipe_set.  Returns the pipeline handle."""
+    arr = (hl_pipe_set * len(sets))(*sets)
+    p = _lib.hl_pipe_create(ctx, _ptr(d_cache), _ptr(host_table), int(window_rows), len(sets), arr, int(n_dense),
+                            main_stream)
+    if not p:
+        raise HotlineError("hl_pipe_create", HL_EINVAL)
+    return p
+
+
+def hl_pipe_destroy(pipe: int) -> None:
+    _lib.hl_pipe_destroy(pipe)
+
+
+def hl_pipe_submit(pipe: int, batch: hl_batch, d_dense) -> None:
+    _check("hl_pipe_submit", _lib.hl_pipe_submit(pipe, ctypes.byref(batch), _ptr(d_dense)))
+
+
+def hl_pipe_step(pipe: int, d_grad_pop, d_grad_non, lr: float, next_batch: Optional[hl_batch], d_next_dense) -> int:
+    """Returns the index of the buffer set that holds the stepped mini-batch's outputs."""
+    out = ctypes.c_int32(-1)
+    _check("hl_pipe_step", _lib.hl_pipe_step(pipe, _ptr(d_grad_pop), _ptr(d_grad_non), float(lr),
+                                             ctypes.byref(next_batch) if next_batch is not None else None,
+                                             _ptr(d_next_dense), ctypes.byref(out)))
+    return int(out.value)
+
+
+def hl_pipe_wait_outputs(pipe: int, stream: int) -> None:
+    _check("hl_pipe_wait_outputs", _lib.hl_pipe_wait_outputs(pipe, stream))
+
+
+def hl_pipe_drain(pipe: int) -> None:
+    _check("hl_pipe_drain", _lib.hl_pipe_drain(pipe))
+
+
+def hl_pipe_time_forward(pipe: int, pop_begin, pop_end, non_begin, non_end) -> None:
+    _check("hl_pipe_time_forward", _lib.hl_pipe_time_forward(pipe, _ev(pop_begin), _ev(pop_end), _ev(non_begin),
+                                                             _ev(non_end)))
+
+
+def hl_pipe_wait_counts(pipe: int, stream: int) -> None:
+    _check("hl_pipe_wait_counts", _lib.hl_pipe_wait_counts(pipe, stream))

@@ -541,7 +541,108 @@ class PipelinedHotline(Hotline):
         self.j_done += 1
         return j % 3
 
+    @property
+    def idle(self) -> bool:
+        return self.j_submitted == self.j_done
+
+    def wait_outputs(self) -> None:
+        """The main stream waits for the last write-back (device-side)."""
+        self.main.wait_stream(self.wb)
+
+    def wait_counts(self, stream: torch.cuda.Stream) -> None:
+        """``stream`` waits until perm and counts of the mini-batch last stepped are final."""
+        if self.j_done >= 1:
+            stream.wait_event(self.sets[(self.j_done - 1) % self.n_sets].ev_index)
+
     def drain(self) -> None:
         """Waits until everything issued so far, write-backs included, has finished."""
         for s in [self.main, self.wb, self.link] + self.sides:
             s.synchronize()
+
+
+class NativePipelinedHotline(Hotline):
+    """The default schedule of :class:`PipelinedHotline` (index work ``lookahead`` mini-batches ahead on three
+    streams, one combined backward sort, host reads overlapping write-backs, shared rows forwarded), issued by the
+    library itself (hl_pipe_*): one C call per mini-batch instead of some sixty Python-level calls, which is what
+    bounds small mini-batches.  Same results, same buffers (``sets``), same call pattern:
+
+        p.start(idx0, off0, B, dense0, more=[(idx1, off1, B, dense1)])    # lookahead mini-batches
+        for j in range(n):
+            s = p.step(grad_pop, grad_non, lr, next_batch=(idx, off, B, dense) or None)
+        p.drain()
+    """
+
+    def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
+                 n_dense: int = 0, device: str = "cuda:0", lookahead: int = 2):
+        self.window_rows = int(window_rows)
+        self.lookahead = max(1, int(lookahead))
+        super().__init__(table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, 2 * self.window_rows,
+                         host_table, n_dense=n_dense, device=device)
+        self.n_sets = self.lookahead + 2
+        self.sets = [_BatchSet(self) for _ in range(self.n_sets)]
+        c_sets = []
+        for st in self.sets:
+            c_sets.append(B.hl_pipe_set(
+                B._ptr(st.perm), B._ptr(st.counts), st.pop, st.non, B._ptr(st.cold_rows), B._ptr(st.n_cold),
+                B._ptr(st.fwd_src), B._ptr(st.pooled_pop), B._ptr(st.pooled_non), B._ptr(st.dense_out),
+                B._ptr(st.sorted_all[0]), B._ptr(st.sorted_all[1]), B._ptr(st.sorted_all[2])))
+        torch.cuda.synchronize(self.device)
+        self.pipe = B.hl_pipe_create(self.ctx, self.cache, self.host_table, self.window_rows, c_sets, self.n_dense,
+                                     self.main.cuda_stream)
+        self.in_flight = 0
+        self._timer_pool = []
+
+    def _new_timer_events(self):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        for e in evs:
+            e.record(self.main)          # gives the event its handle
+        return evs
+
+    def prepare_timers(self, n: int) -> None:
+        """Creates the events of n timed steps ahead of time (step(timers=...) then only hands them to the library)."""
+        self._timer_pool.extend(self._new_timer_events() for _ in range(n))
+
+    def _hl_batch(self, nb):
+        indices, offsets, batch, dense = nb
+        return self._batch(indices, offsets, batch), (dense if self.n_dense else None)
+
+    def start(self, indices, offsets, batch: int, dense=None, more=()) -> None:
+        assert self.in_flight == 0, "start() only with nothing in flight"
+        for nb in [(indices, offsets, batch, dense)] + [tuple(x) for x in more]:
+            b, d = self._hl_batch(nb)
+            B.hl_pipe_submit(self.pipe, b, d)
+            self.in_flight += 1
+
+    def step(self, grad_pop: torch.Tensor, grad_non: torch.Tensor, lr: float, next_batch=None, timers=None) -> int:
+        b, d = self._hl_batch(next_batch) if next_batch is not None else (None, None)
+        if timers is not None:
+            # only the two forward calls can be timed from outside; the events are recorded inside the C call
+            evs = self._timer_pool.pop() if self._timer_pool else self._new_timer_events()
+            B.hl_pipe_time_forward(self.pipe, *evs)
+            timers.setdefault("fwd_pop", []).append((evs[0], evs[1]))
+            timers.setdefault("fwd_non", []).append((evs[2], evs[3]))
+        s = B.hl_pipe_step(self.pipe, grad_pop, grad_non, lr, b, d)
+        self.in_flight += (1 if next_batch is not None else 0) - 1
+        return s
+
+    @property
+    def idle(self) -> bool:
+        return self.in_flight == 0
+
+    def wait_outputs(self) -> None:
+        """The main stream waits for the last write-back (device-side)."""
+        B.hl_pipe_wait_outputs(self.pipe, self.main.cuda_stream)
+
+    def wait_counts(self, stream: torch.cuda.Stream) -> None:
+        """``stream`` waits until perm and counts of the mini-batch last stepped are final."""
+        B.hl_pipe_wait_counts(self.pipe, stream.cuda_stream)
+
+    def drain(self) -> None:
+        B.hl_pipe_drain(self.pipe)
+
+    def close(self) -> None:
+        if getattr(self, "pipe", None):
+            B.hl_pipe_drain(self.pipe)
+            B.hl_pipe_destroy(self.pipe)
+            self.pipe = None
+        super().close()

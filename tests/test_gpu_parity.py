@@ -154,6 +154,22 @@ def test_pipelined_multi_hot_integer_data():
     assert stats["shared_cold_rows"] > 100
 
 
+def test_native_pipeline_equals_sequential_steps_integer_data():
+    """The same schedule issued by the library itself (hl_pipe_*): bit-identical to the oracle's one-after-the-other
+    processing on integer data, with forwarding of shared cold rows, for index work one, two and three mini-batches
+    ahead."""
+    for ahead in (1, 2, 3):
+        stats = run_pipelined_check("tiny", steps=7, integer=True, native=True, lookahead=ahead)
+        assert stats["shared_cold_rows"] > 50
+    spec = dataclasses.replace(gen.CONFIGS["multi_hot"], batch=512, dim=32, rows=("fixed", 2000),
+                               hot_policy=("fraction", 40, 100), profile_batches=2)
+    run_pipelined_check(spec, steps=4, integer=True, native=True)
+
+
+def test_native_pipeline_real_data_and_dense_features():
+    run_pipelined_check("dlrm_small", steps=3, scale_rows=0.02, integer=False, profile_batches=6, native=True)
+
+
 def test_flush_and_second_learning_phase():
     """Re-calibration: flush the popular rows, learn another popular set from later mini-batches, carry on."""
     stats = run_recalibration_check("tiny")
