@@ -53,7 +53,7 @@ extern "C" {
 #define HL_EBOUNDS   (-2)   /* an index outside its table / a slot outside the cache (device; item skipped)      */
 #define HL_ECAPACITY (-3)   /* an output buffer, the hot cache or the staging area is too small (device; clamped)*/
 #define HL_ECUDA     (-4)   /* a CUDA runtime call failed                                                        */
-#define HL_ETIMEOUT  (-5)   /* reserved: a bounded device-side wait gave up                                      */
+#define HL_ETIMEOUT  (-5)   /* a bounded device-side wait (tile chaining of a scan or sort, a bulk copy) gave up  */
 
 typedef struct hl_ctx hl_ctx;
 

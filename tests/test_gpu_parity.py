@@ -166,6 +166,39 @@ def test_native_pipeline_equals_sequential_steps_integer_data():
     run_pipelined_check(spec, steps=4, integer=True, native=True)
 
 
+def test_native_pipeline_refuses_what_it_cannot_queue():
+    """hl_pipe_step before any hl_pipe_submit, and more submissions than there are spare buffer sets."""
+    import numpy as np
+    import torch
+    import paper_2204_05436_b200 as hl
+    spec = gen.CONFIGS["tiny"]
+    geom = gen.make_geometry(spec)
+    B, D = spec.batch, spec.dim
+    N = int(sum(geom.table_rows))
+    n_bags = geom.num_tables * B
+    table = torch.zeros((N, D), dtype=torch.float32).pin_memory()
+    p = hl.NativePipelinedHotline(geom.table_rows, D, 1, B, n_bags, 4096, 4096, table, lookahead=2)
+    try:
+        with torch.cuda.stream(p.main):
+            p.set_hot_rows(torch.arange(100, dtype=torch.int32, device="cuda:0"))
+            p.build_remap(load_rows=True)
+            b = gen.make_batch(spec, geom, 0)
+            idx = torch.from_numpy(b.indices).to("cuda:0")
+            off = torch.from_numpy(b.offsets).to("cuda:0")
+            grad = torch.zeros((n_bags, D), device="cuda:0")
+            with pytest.raises(hl.HotlineError):
+                p.step(grad, grad, 0.1)                       # nothing submitted
+            p.start(idx, off, B, None, more=[(idx, off, B, None), (idx, off, B, None)])   # 3 of 4 sets
+            with pytest.raises(hl.HotlineError):
+                hl.hl_pipe_submit(p.pipe, p._batch(idx, off, B), None)                   # no spare set left
+            for _ in range(3):
+                p.step(grad, grad, 0.1)
+            p.drain()
+            assert p.status() == hl.HL_OK
+    finally:
+        p.close()
+
+
 def test_native_pipeline_real_data_and_dense_features():
     run_pipelined_check("dlrm_small", steps=3, scale_rows=0.02, integer=False, profile_batches=6, native=True)
 
