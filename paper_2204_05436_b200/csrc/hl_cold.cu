@@ -1,5 +1,5 @@
 // The non-popular micro-batch's working set: classify its lookups, find the distinct cold rows, stage them from
-// the host-DRAM table (zero-copy 128-bit loads over the host link) behind the hot cache, and write them back.
+// the host-DRAM table (bulk copies over the host link, row by row) behind the hot cache, and write them back.
 #include "hl_common.cuh"
 #include <cooperative_groups.h>
 #include <cstdlib>
@@ -528,11 +528,8 @@ int32_t launch_move_rows(float* dense_side, int64_t dense_row0, float* table, co
         HL_LAUNCH_CHECK();
         return HL_OK;
     }
-    // Few CTAs with many rows in flight each.  Random rows of a table of tens of GB miss the address translation
-    // of the host link on almost every row, so the link needs about a megabyte in flight to reach its rate; but
-    // this kernel runs next to the embedding-bag kernels of another micro-batch, whose grids are sized to fill the
-    // chip: every SM it sits on takes CTA slots and load-store queue entries away from them for hundreds of
-    // microseconds.  48 CTAs x 16 groups x 16 rows keeps 12 K rows in flight on a third of the SMs.
+    // Rows wider than a stage of the bulk mover (16 KB): plain 128-bit loads and stores, 48 CTAs x 16 groups x 16 rows
+    // in flight on a third of the SMs, so that the kernels of the other streams keep CTA slots.
     const int grid = 48;
     if (D4 <= 4)
         k_move_rows<4, TO_TABLE><<<grid, kThreads, 0, stream>>>(dense_side, dense_row0, table, rows, d_n, n_max,

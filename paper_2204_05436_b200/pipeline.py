@@ -261,26 +261,28 @@ class _BatchSet:
 
 
 class PipelinedHotline(Hotline):
-    """The same path, software-pipelined across mini-batches: while mini-batch j executes on the main stream,
-    mini-batch j+1 is already fragmented and its cold rows staged on a side stream, and mini-batch j-1's cold rows
-    are written back on a third stream.  The result is that of processing the mini-batches one after the other:
-    a cold row that j+1 shares with j is not read from the host but copied from j's staging window after j's
-    backward (hl_forward_cold), and the host rows of j+1 are read only after j-1's write-back has finished.
+    """The same path, software-pipelined across mini-batches, issued from Python (NativePipelinedHotline issues the
+    default variant from C).  While mini-batch j executes on the main stream, the index-only work of mini-batch
+    j+lookahead (fragment, cold-row search, backward sort) runs on three side streams, the host rows of j+1 are read on
+    a link stream, and j-1's cold rows are written back on another.  The result is that of processing the mini-batches
+    one after the other: a cold row that j+1 shares with j is not read from the host but copied from j's staging
+    window after j's backward (hl_forward_cold), and the host rows of j+1 are read only after j-1's write-back has
+    finished.
 
-    Three sets of index buffers rotate over the mini-batches, two windows of the staging area alternate.
+    lookahead + 2 sets of index buffers rotate over the mini-batches, two windows of the staging area alternate.
 
     ``overlap_link=True`` (default): the read of j+1's host rows starts as soon as j-1's write-back is done and
     overlaps j's execution and write-back, with the rows j+1 shares with j forwarded between the staging windows.
     ``overlap_link=False``: the host rows of j+1 are read after j's write-back has finished, so the two transfers
     follow each other on the link and no forwarding is needed; fragment and the search for the distinct cold rows of
     j+1 still run under j's execution.  (Which is faster depends on the host table's memory: with large-page
-    device mappings (hl_host_alloc) 0.43 against 0.47 ms per DLRM-large-like mini-batch; with 4 KB mappings
-    (cudaHostAlloc) reads and write-backs compete for address translations and it is the other way round, 0.84
+    device mappings (hl_host_alloc) 0.30 against 0.43 ms per DLRM-large-like mini-batch; with 4 KB mappings
+    (cudaHostAlloc) reads and write-backs compete for address translations and it was the other way round, 0.84
     against 0.65 ms.)
 
-        p.start(idx0, off0, B)                       # ahead-work of mini-batch 0
+        p.start(idx0, off0, B, dense0, more=[(idx1, off1, B, dense1)])      # ahead-work of `lookahead` mini-batches
         for j in range(n):
-            s = p.step(grad_pop, grad_non, lr, next_batch=(idx, off, B, dense) or None)
+            s = p.step(grad_pop, grad_non, lr, next_batch=(idx, off, B, dense) or None)   # the next one not yet given
             ... p.sets[s].pooled_pop / pooled_non are mini-batch j's outputs once the main stream gets there
         p.drain()
     """
