@@ -370,8 +370,10 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             k = i % n_batches
             if pipelined:
                 if h.idle:
-                    h.start(*batch_args(k), more=[batch_args((i + a) % n_batches) for a in range(1, h.lookahead)])
-                s = h.step(d_grad, d_grad, lr, next_batch=batch_args((i + h.lookahead) % n_batches), timers=timers)
+                    h.start(*batch_args(k), more=[batch_args((i + a) % n_batches) for a in range(1, h.lookahead)],
+                            inputs_ready="resident")
+                s = h.step(d_grad, d_grad, lr, next_batch=batch_args((i + h.lookahead) % n_batches), timers=timers,
+                           inputs_ready="resident")      # the inputs of the timed region are in HBM already
                 return k, h.sets[s]
             h.step(d_idx[k], d_off[k], B, d_grad, d_grad, lr, dense=d_dense[k], timers=timers)
             return k, h
@@ -533,11 +535,11 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                             h2d_now += h_dense[kin].numel() * 4
                         d_grads[g].copy_(h_grad, non_blocking=True)
                         ev_in[g].record(s_in)
-                    h.main.wait_event(ev_in[g])
+                    h.main.wait_event(ev_in[g])               # this step's gradients
                     if h.idle:
                         h.start(*batch_args(j % n_batches),
                                 more=[batch_args((j + a) % n_batches) for a in range(1, L)])
-                    st = h.sets[h.step(d_grads[g], d_grads[g], lr, next_batch=batch_args(kin))]
+                    st = h.sets[h.step(d_grads[g], d_grads[g], lr, next_batch=batch_args(kin), inputs_ready=ev_in[g])]
                     ev_grad_free[g].record(h.main)
                     ev_done.record(h.main)
                     o_pop, o_non, o_counts, o_perm = outs[g]
@@ -910,8 +912,9 @@ def run_sweep(args) -> None:
             i = it[0]
             it[0] += 1
             if h.idle:
-                h.start(*d_in[i % n], more=[d_in[(i + a) % n] for a in range(1, h.lookahead)])
-            return h.sets[h.step(d_grad, d_grad, wl.spec.lr, next_batch=d_in[(i + h.lookahead) % n])]
+                h.start(*d_in[i % n], more=[d_in[(i + a) % n] for a in range(1, h.lookahead)], inputs_ready="resident")
+            return h.sets[h.step(d_grad, d_grad, wl.spec.lr, next_batch=d_in[(i + h.lookahead) % n],
+                                 inputs_ready="resident")]
 
         pops, colds = [], []
         for _ in range(n):

@@ -304,6 +304,19 @@ HL_API int32_t hl_index_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non
                              int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold,
                              const int32_t* d_prev_cold_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
                              void* stream);
+/* hl_index_cold in two halves, for a scheduler that can put other work between them.  hl_index_cold_begin classifies
+ * X's lookups and, if there are at most 20 480 cold ones, finds the distinct rows and assigns the slots at once; it
+ * leaves a verdict in the device word hl_index_cold_verdict(ctx): 0 = done, else the number of cold lookups.
+ * hl_index_cold_end does the rest (the general search, whose kernels find nothing to do after a verdict of 0, and the
+ * match against the previous cold rows); general_not_needed != 0 = the caller has read a verdict of 0 and spares the
+ * general search's launches.  Same arguments as hl_index_cold; both halves on one stream, nothing else of this
+ * context's cold-row search between them. */
+HL_API int32_t hl_index_cold_begin(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, int64_t stage_row0,
+                                   int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold, void* stream);
+HL_API const int32_t* hl_index_cold_verdict(hl_ctx* ctx);
+HL_API int32_t hl_index_cold_end(hl_ctx* ctx, hl_ubatch* non, int64_t stage_row0, int64_t stage_rows,
+                                 int32_t* d_cold_rows, int64_t* d_n_cold, const int32_t* d_prev_cold_rows,
+                                 const int64_t* d_n_prev, int32_t* d_fwd_src, int32_t general_not_needed, void* stream);
 HL_API int32_t hl_stage_cold(hl_ctx* ctx, const float* host_table, float* d_cache, int64_t stage_row0,
                              int64_t stage_rows, const int32_t* d_cold_rows, const int64_t* d_n_cold,
                              const int32_t* d_fwd_src, void* stream);
@@ -356,18 +369,22 @@ HL_API hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_table, i
                                const hl_pipe_set* sets, int32_t n_dense, void* main_stream);
 HL_API void hl_pipe_destroy(hl_pipe* p);
 
-/* Queues the ahead-work of the next mini-batch (its inputs must be complete in main_stream's order at the time of
- * the call; d_dense may be NULL).  Call it n_sets - 2 times before the first hl_pipe_step; afterwards pass the next
+/* Queues the ahead-work of the next mini-batch (d_dense may be NULL).  inputs_ready says when its indices, offsets and
+ * dense features are complete: NULL = in main_stream's order at the time of the call; a cudaEvent_t = when that event
+ * has happened; HL_PIPE_INPUTS_RESIDENT = they already are (the ahead-work then starts without waiting for whatever
+ * main_stream still has queued).  Call it n_sets - 2 times before the first hl_pipe_step; afterwards pass the next
  * mini-batch to hl_pipe_step instead.  HL_ECAPACITY if every buffer set is in flight. */
-HL_API int32_t hl_pipe_submit(hl_pipe* p, const hl_batch* b, const float* d_dense);
+#define HL_PIPE_INPUTS_RESIDENT ((void*)(intptr_t)-1)
+HL_API int32_t hl_pipe_submit(hl_pipe* p, const hl_batch* b, const float* d_dense, void* inputs_ready);
 
 /* Queues the main work of the oldest submitted mini-batch: forward and update of O, forward and update of X with the
  * upstream gradients d_grad_pop / d_grad_non ([bags of O, D] / [bags of X, D], in the micro-batches' bag order), and
- * its write-back; and the ahead-work of `next` (may be NULL).  *set_index = which of the sets holds this mini-batch's
+ * its write-back; and the ahead-work of `next` (may be NULL; next_inputs_ready as for hl_pipe_submit).  *set_index = which of the sets holds this mini-batch's
  * perm, counts and pooled vectors; they are complete in main_stream's order, and the set is reused n_sets steps on.
  * No call waits for the device. */
 HL_API int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float* d_grad_non, float lr,
-                            const hl_batch* next, const float* d_next_dense, int32_t* set_index);
+                            const hl_batch* next, const float* d_next_dense, void* next_inputs_ready,
+                            int32_t* set_index);
 
 /* Measurement aid: the next hl_pipe_step (only that one) records these caller-owned events (cudaEvent_t, any may be
  * NULL) on main_stream before and after the forward over O and before and after the forward over X. */

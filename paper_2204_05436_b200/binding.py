@@ -23,6 +23,7 @@ EXPORTS = (
     "hl_embbag_bwd_prepare2", "hl_embbag_bwd_apply2",
     "hl_tracker_reset", "hl_tracker_update", "hl_tracker_export",
     "hl_pipe_create", "hl_pipe_destroy", "hl_pipe_submit", "hl_pipe_step", "hl_pipe_wait_outputs", "hl_pipe_drain", "hl_pipe_time_forward", "hl_pipe_wait_counts",
+    "hl_index_cold_begin", "hl_index_cold_end", "hl_index_cold_verdict",
 )
 
 
@@ -126,13 +127,19 @@ def _load() -> ctypes.CDLL:
     lib.hl_pipe_destroy.restype = None
     lib.hl_pipe_destroy.argtypes = [vp]
     lib.hl_pipe_submit.restype = i32
-    lib.hl_pipe_submit.argtypes = [vp, ctypes.POINTER(hl_batch), vp]
+    lib.hl_pipe_submit.argtypes = [vp, ctypes.POINTER(hl_batch), vp, vp]
     lib.hl_pipe_step.restype = i32
-    lib.hl_pipe_step.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.POINTER(hl_batch), vp, ctypes.POINTER(i32)]
+    lib.hl_pipe_step.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.POINTER(hl_batch), vp, vp, ctypes.POINTER(i32)]
     lib.hl_pipe_wait_outputs.restype = i32
     lib.hl_pipe_wait_outputs.argtypes = [vp, vp]
     lib.hl_pipe_drain.restype = i32
     lib.hl_pipe_drain.argtypes = [vp]
+    lib.hl_index_cold_begin.restype = i32
+    lib.hl_index_cold_begin.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, i64, i64, vp, vp, vp]
+    lib.hl_index_cold_verdict.restype = vp
+    lib.hl_index_cold_verdict.argtypes = [vp]
+    lib.hl_index_cold_end.restype = i32
+    lib.hl_index_cold_end.argtypes = [vp, ctypes.POINTER(hl_ubatch), i64, i64, vp, vp, vp, vp, vp, i32, vp]
     lib.hl_pipe_wait_counts.restype = i32
     lib.hl_pipe_wait_counts.argtypes = [vp, vp]
     lib.hl_pipe_time_forward.restype = i32
@@ -408,16 +415,30 @@ def hl_pipe_destroy(pipe: int) -> None:
     _lib.hl_pipe_destroy(pipe)
 
 
-def hl_pipe_submit(pipe: int, batch: hl_batch, d_dense) -> None:
-    _check("hl_pipe_submit", _lib.hl_pipe_submit(pipe, ctypes.byref(batch), _ptr(d_dense)))
+HL_PIPE_INPUTS_RESIDENT = ctypes.c_void_p(-1).value
 
 
-def hl_pipe_step(pipe: int, d_grad_pop, d_grad_non, lr: float, next_batch: Optional[hl_batch], d_next_dense) -> int:
+def _ready(inputs_ready):
+    """None (main-stream order), "resident", a torch.cuda.Event or a raw cudaEvent_t."""
+    if inputs_ready is None:
+        return None
+    if isinstance(inputs_ready, str):
+        assert inputs_ready == "resident"
+        return HL_PIPE_INPUTS_RESIDENT
+    return _ev(inputs_ready)
+
+
+def hl_pipe_submit(pipe: int, batch: hl_batch, d_dense, inputs_ready=None) -> None:
+    _check("hl_pipe_submit", _lib.hl_pipe_submit(pipe, ctypes.byref(batch), _ptr(d_dense), _ready(inputs_ready)))
+
+
+def hl_pipe_step(pipe: int, d_grad_pop, d_grad_non, lr: float, next_batch: Optional[hl_batch], d_next_dense,
+                 next_inputs_ready=None) -> int:
     """Returns the index of the buffer set that holds the stepped mini-batch's outputs."""
     out = ctypes.c_int32(-1)
     _check("hl_pipe_step", _lib.hl_pipe_step(pipe, _ptr(d_grad_pop), _ptr(d_grad_non), float(lr),
                                              ctypes.byref(next_batch) if next_batch is not None else None,
-                                             _ptr(d_next_dense), ctypes.byref(out)))
+                                             _ptr(d_next_dense), _ready(next_inputs_ready), ctypes.byref(out)))
     return int(out.value)
 
 
@@ -436,3 +457,22 @@ def hl_pipe_time_forward(pipe: int, pop_begin, pop_end, non_begin, non_end) -> N
 
 def hl_pipe_wait_counts(pipe: int, stream: int) -> None:
     _check("hl_pipe_wait_counts", _lib.hl_pipe_wait_counts(pipe, stream))
+
+
+def hl_index_cold_begin(ctx: int, non: hl_ubatch, d_n_non, stage_row0: int, stage_rows: int, d_cold_rows, d_n_cold,
+                        stream: int) -> None:
+    _check("hl_index_cold_begin", _lib.hl_index_cold_begin(ctx, ctypes.byref(non), _ptr(d_n_non), int(stage_row0),
+                                                           int(stage_rows), _ptr(d_cold_rows), _ptr(d_n_cold), stream))
+
+
+def hl_index_cold_verdict(ctx: int) -> int:
+    """Device address of the verdict word (int32) of the last hl_index_cold_begin."""
+    return int(_lib.hl_index_cold_verdict(ctx) or 0)
+
+
+def hl_index_cold_end(ctx: int, non: hl_ubatch, stage_row0: int, stage_rows: int, d_cold_rows, d_n_cold, d_prev_cold_rows,
+                      d_n_prev, d_fwd_src, general_not_needed: bool, stream: int) -> None:
+    _check("hl_index_cold_end", _lib.hl_index_cold_end(ctx, ctypes.byref(non), int(stage_row0), int(stage_rows),
+                                                       _ptr(d_cold_rows), _ptr(d_n_cold), _ptr(d_prev_cold_rows),
+                                                       _ptr(d_n_prev), _ptr(d_fwd_src), int(bool(general_not_needed)),
+                                                       stream))

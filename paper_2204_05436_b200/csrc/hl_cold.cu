@@ -573,24 +573,14 @@ namespace {
 
 // Shared body of hl_gather_cold and hl_gather_cold_ahead.  Staging window: cache slots
 // [hot_cap + stage_row0, hot_cap + stage_row0 + stage_rows).
-int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const float* host_table, float* d_cache,
-                    int64_t stage_row0, int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold,
-                    const int32_t* d_prev_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
-                    cudaEvent_t record_after_index, cudaEvent_t wait_a, cudaEvent_t wait_b, bool do_index,
-                    bool do_move, cudaStream_t stream) {
+// First half of the cold-row search: classify X's lookups and let the one-cluster kernel try; it leaves its verdict in
+// cold_n[1] (0: done; else the number of cold lookups, for the general path).
+int32_t index_begin(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, int64_t stage_row0, int64_t stage_rows,
+                    int32_t* d_cold_rows, int64_t* d_n_cold, cudaStream_t stream) {
     Regions& r = ctx->r;
-    if (!do_index) {
-        if (ctx->max_nnz == 0) return HL_OK;
-        timer_mark(ctx, HL_TIMER_GATHER_MOVE, 0, stream);
-        const int32_t st = launch_move_rows<false>(d_cache, ctx->hot_cap + stage_row0,
-                                                   const_cast<float*>(host_table), d_cold_rows, d_n_cold, stage_rows,
-                                                   ctx->N, ctx->D, d_fwd_src, kBulkCtas, r.status, stream);
-        timer_mark(ctx, HL_TIMER_GATHER_MOVE, 1, stream);
-        return st;
-    }
     if (ctx->max_nnz == 0) {
         HL_CUDA_TRY(cudaMemsetAsync(d_n_cold, 0, sizeof(int64_t), stream));
-        if (record_after_index) HL_CUDA_TRY(cudaEventRecord(record_after_index, stream));
+        HL_CUDA_TRY(cudaMemsetAsync(r.cold_n, 0, 4 * sizeof(int32_t), stream));
         return HL_OK;
     }
     if (!non->ids) return HL_EINVAL;
@@ -603,27 +593,37 @@ int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const f
     HL_LAUNCH_CHECK();
     // up to kSmallCap cold lookups: one cluster; more: the general path, whose count (cold_n[1]) that kernel sets
     const int key_bits = bits_for(ctx->N - 1);
-    {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(kSmallCtas);
-        cfg.blockDim = dim3(kSmallThreads);
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = kSmallCtas;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        HL_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_cold_small, (const int32_t*)r.cold_keys[0],
-                                       (const int32_t*)r.cold_vals[0], (const int32_t*)r.cold_n, ctx->max_nnz,
-                                       (key_bits + 7) / 8, ctx->hot_cap + stage_row0, stage_rows, non->ids,
-                                       d_cold_rows, d_n_cold, r.cold_n + 1, r.status));
-    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kSmallCtas);
+    cfg.blockDim = dim3(kSmallThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kSmallCtas;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    HL_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_cold_small, (const int32_t*)r.cold_keys[0], (const int32_t*)r.cold_vals[0],
+                                   (const int32_t*)r.cold_n, ctx->max_nnz, (key_bits + 7) / 8,
+                                   ctx->hot_cap + stage_row0, stage_rows, non->ids, d_cold_rows, d_n_cold,
+                                   r.cold_n + 1, r.status));
     note_launches(1);
     HL_LAUNCH_CHECK();
+    return HL_OK;
+}
+
+// Second half: the general path (its kernels find nothing to do when the verdict is 0; `general_not_needed` = the
+// caller has read that verdict and spares the launches), then the match against the previous mini-batch's cold rows.
+int32_t index_end(hl_ctx* ctx, hl_ubatch* non, int64_t stage_row0, int64_t stage_rows, int32_t* d_cold_rows,
+                  int64_t* d_n_cold, const int32_t* d_prev_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
+                  bool general_not_needed, cudaStream_t stream) {
+    Regions& r = ctx->r;
+    if (ctx->max_nnz == 0) return HL_OK;
+    const int grid = grid_for(ctx->max_nnz, kThreads, kMaxGrid);
+    const int key_bits = bits_for(ctx->N - 1);
     int32_t st = HL_OK;
-    if (ctx->max_nnz > kSmallCap) {
+    if (ctx->max_nnz > kSmallCap && !general_not_needed) {
         int32_t *keys, *vals;
         st = radix_sort_pairs(r.cold_keys, r.cold_vals, r.cold_n + 1, ctx->max_nnz, key_bits, r.cold_hist, r.status,
                               &keys, &vals, stream);
@@ -645,6 +645,29 @@ int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const f
         note_launches(1);
         HL_LAUNCH_CHECK();
     }
+    return HL_OK;
+}
+
+int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const float* host_table, float* d_cache,
+                    int64_t stage_row0, int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold,
+                    const int32_t* d_prev_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
+                    cudaEvent_t record_after_index, cudaEvent_t wait_a, cudaEvent_t wait_b, bool do_index,
+                    bool do_move, cudaStream_t stream) {
+    Regions& r = ctx->r;
+    if (!do_index) {
+        if (ctx->max_nnz == 0) return HL_OK;
+        timer_mark(ctx, HL_TIMER_GATHER_MOVE, 0, stream);
+        const int32_t st = launch_move_rows<false>(d_cache, ctx->hot_cap + stage_row0,
+                                                   const_cast<float*>(host_table), d_cold_rows, d_n_cold, stage_rows,
+                                                   ctx->N, ctx->D, d_fwd_src, kBulkCtas, r.status, stream);
+        timer_mark(ctx, HL_TIMER_GATHER_MOVE, 1, stream);
+        return st;
+    }
+    int32_t st = index_begin(ctx, non, d_n_non, stage_row0, stage_rows, d_cold_rows, d_n_cold, stream);
+    if (st != HL_OK) return st;
+    st = index_end(ctx, non, stage_row0, stage_rows, d_cold_rows, d_n_cold, d_prev_rows, d_n_prev, d_fwd_src, false,
+                   stream);
+    if (st != HL_OK) return st;
     if (record_after_index) HL_CUDA_TRY(cudaEventRecord(record_after_index, stream));
     if (!do_move) return HL_OK;
     if (wait_a) HL_CUDA_TRY(cudaStreamWaitEvent(stream, wait_a, 0));
@@ -697,6 +720,27 @@ extern "C" int32_t hl_index_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n
     return gather_impl(ctx, non, d_n_non, nullptr, nullptr, stage_row0, stage_rows, d_cold_rows, d_n_cold,
                        d_prev_cold_rows, d_n_prev, d_fwd_src, nullptr, nullptr, nullptr, true, false,
                        static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" int32_t hl_index_cold_begin(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, int64_t stage_row0,
+                                       int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold, void* stream_) {
+    if (!ctx || !non || !non->offsets || !d_n_non || !d_cold_rows || !d_n_cold) return HL_EINVAL;
+    if (!window_ok(ctx, stage_row0, stage_rows)) return HL_EINVAL;
+    return index_begin(ctx, non, d_n_non, stage_row0, stage_rows, d_cold_rows, d_n_cold,
+                       static_cast<cudaStream_t>(stream_));
+}
+
+extern "C" const int32_t* hl_index_cold_verdict(hl_ctx* ctx) { return ctx ? ctx->r.cold_n + 1 : nullptr; }
+
+extern "C" int32_t hl_index_cold_end(hl_ctx* ctx, hl_ubatch* non, int64_t stage_row0, int64_t stage_rows,
+                                     int32_t* d_cold_rows, int64_t* d_n_cold, const int32_t* d_prev_cold_rows,
+                                     const int64_t* d_n_prev, int32_t* d_fwd_src, int32_t general_not_needed,
+                                     void* stream_) {
+    if (!ctx || !non || !d_cold_rows || !d_n_cold) return HL_EINVAL;
+    if (!window_ok(ctx, stage_row0, stage_rows)) return HL_EINVAL;
+    if ((d_prev_cold_rows != nullptr) != (d_n_prev != nullptr) || (d_prev_cold_rows && !d_fwd_src)) return HL_EINVAL;
+    return index_end(ctx, non, stage_row0, stage_rows, d_cold_rows, d_n_cold, d_prev_cold_rows, d_n_prev, d_fwd_src,
+                     general_not_needed != 0, static_cast<cudaStream_t>(stream_));
 }
 
 extern "C" int32_t hl_stage_cold(hl_ctx* ctx, const float* host_table, float* d_cache, int64_t stage_row0,

@@ -25,10 +25,13 @@ struct hl_pipe {
     std::vector<hl_pipe_set> sets;
     cudaStream_t main, sa, sb, sc, link, wb;
     struct Events {
-        cudaEvent_t inputs, frag, index, prep, gather, forward, x, scatter;
+        cudaEvent_t inputs, frag, index, prep, gather, forward, x, scatter, verdict;
     };
     std::vector<Events> ev;
-    int64_t j_indexed, j_submitted, j_done;
+    // mini-batches whose fragment + first half of the cold-row search are queued (begun), whose cold-row search and
+    // sort are queued in full (indexed), whose host read is queued (submitted), whose main work is queued (done)
+    int64_t j_begun, j_indexed, j_submitted, j_done;
+    int32_t* h_verdict;          // pinned host words, one per set: what the first half of the cold-row search found
     cudaEvent_t time_fwd[4];     // one-shot: recorded around the two forward calls of the next step
 };
 
@@ -43,29 +46,60 @@ namespace {
 int32_t wait(cudaStream_t s, cudaEvent_t e) { return cudaStreamWaitEvent(s, e, 0) == cudaSuccess ? HL_OK : HL_ECUDA; }
 int32_t record(cudaEvent_t e, cudaStream_t s) { return cudaEventRecord(e, s) == cudaSuccess ? HL_OK : HL_ECUDA; }
 
-// fragment, cold-row search and backward sort of the next mini-batch (index-only: nothing here touches a row)
-int32_t submit_index(hl_pipe* p, const hl_batch* b, const float* d_dense) {
+// Second half of the index-only work of the mini-batch begun last: the rest of the cold-row search and the backward
+// sort.  It is queued one call later than the first half whenever the schedule has that slack, because by then the
+// host can usually see (without waiting) that the one-cluster kernel has found the distinct rows itself, and the ten
+// launches of the general path need not be queued at all; if that is not known yet they are queued and decide on
+// the device.  (With steps issued back to back, as in the benchmark, the verdict of a mini-batch begun one step ago
+// is usually still on its way -- the chain of fragment and search kernels takes about as long as a step --, so the
+// saving shows when there is other work between the steps, as in training.)
+int32_t finish_index(hl_pipe* p) {
+    if (p->j_indexed == p->j_begun) return HL_OK;
     const int64_t j = p->j_indexed;
     const int n = p->n_sets;
     hl_pipe_set& st = p->sets[j % n];
     hl_pipe::Events& e = p->ev[j % n];
     hl_pipe_set* prev = j >= 1 ? &p->sets[(j - 1) % n] : nullptr;
     const int64_t w = (j % 2) * p->window_rows;
-    HL_PIPE_TRY(wait(p->sa, e.inputs));
-    if (j >= n) HL_PIPE_TRY(wait(p->sa, e.scatter));      // the buffers of this set were mini-batch j-n_sets's
-    HL_PIPE_TRY(hl_fragment(p->ctx, b, d_dense, d_dense ? p->n_dense : 0, st.perm, st.counts, &st.pop, &st.non,
-                            d_dense ? st.dense_out : nullptr, p->sa));
-    HL_PIPE_TRY(record(e.frag, p->sa));
-    HL_PIPE_TRY(wait(p->sc, e.frag));
-    if (j >= n) HL_PIPE_TRY(wait(p->sc, e.scatter));
-    HL_PIPE_TRY(hl_index_cold(p->ctx, &st.non, st.counts + 1, w, p->window_rows, st.cold_rows, st.n_cold,
-                              prev ? prev->cold_rows : nullptr, prev ? prev->n_cold : nullptr, st.fwd_src, p->sc));
+    const bool known_done = cudaEventQuery(e.verdict) == cudaSuccess && p->h_verdict[j % n] == 0;
+    HL_PIPE_TRY(hl_index_cold_end(p->ctx, &st.non, w, p->window_rows, st.cold_rows, st.n_cold,
+                                  prev ? prev->cold_rows : nullptr, prev ? prev->n_cold : nullptr, st.fwd_src,
+                                  known_done ? 1 : 0, p->sc));
     HL_PIPE_TRY(record(e.index, p->sc));
     HL_PIPE_TRY(wait(p->sb, e.index));
     HL_PIPE_TRY(hl_embbag_bwd_prepare2(p->ctx, &st.pop, st.counts, &st.non, st.counts + 1, st.sorted_slots,
                                        st.sorted_bags, st.sorted_n, p->sb));
     HL_PIPE_TRY(record(e.prep, p->sb));
     p->j_indexed += 1;
+    return HL_OK;
+}
+
+// fragment and the first half of the cold-row search of the next mini-batch (index-only: nothing here touches a row)
+int32_t begin_index(hl_pipe* p, const hl_batch* b, const float* d_dense, void* inputs_ready) {
+    HL_PIPE_TRY(finish_index(p));        // stream C: the mini-batch before ends its search before this one begins
+    const int64_t j = p->j_begun;
+    const int n = p->n_sets;
+    hl_pipe_set& st = p->sets[j % n];
+    hl_pipe::Events& e = p->ev[j % n];
+    const int64_t w = (j % 2) * p->window_rows;
+    if (inputs_ready == nullptr) {                        // the inputs are complete in main-stream order
+        HL_PIPE_TRY(record(e.inputs, p->main));
+        HL_PIPE_TRY(wait(p->sa, e.inputs));
+    } else if (inputs_ready != HL_PIPE_INPUTS_RESIDENT) {
+        HL_PIPE_TRY(wait(p->sa, static_cast<cudaEvent_t>(inputs_ready)));
+    }
+    if (j >= n) HL_PIPE_TRY(wait(p->sa, e.scatter));      // the buffers of this set were mini-batch j-n_sets's
+    HL_PIPE_TRY(hl_fragment(p->ctx, b, d_dense, d_dense ? p->n_dense : 0, st.perm, st.counts, &st.pop, &st.non,
+                            d_dense ? st.dense_out : nullptr, p->sa));
+    HL_PIPE_TRY(record(e.frag, p->sa));
+    HL_PIPE_TRY(wait(p->sc, e.frag));
+    if (j >= n) HL_PIPE_TRY(wait(p->sc, e.scatter));
+    HL_PIPE_TRY(hl_index_cold_begin(p->ctx, &st.non, st.counts + 1, w, p->window_rows, st.cold_rows, st.n_cold, p->sc));
+    if (cudaMemcpyAsync(p->h_verdict + (j % n), hl_index_cold_verdict(p->ctx), sizeof(int32_t), cudaMemcpyDeviceToHost,
+                        p->sc) != cudaSuccess)
+        return HL_ECUDA;
+    HL_PIPE_TRY(record(e.verdict, p->sc));
+    p->j_begun += 1;
     return HL_OK;
 }
 
@@ -109,7 +143,8 @@ extern "C" hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_tabl
     p->n_dense = n_dense;
     p->sets.assign(sets, sets + n_sets);
     p->main = static_cast<cudaStream_t>(main_stream);
-    p->j_indexed = p->j_submitted = p->j_done = 0;
+    p->j_begun = p->j_indexed = p->j_submitted = p->j_done = 0;
+    p->h_verdict = nullptr;
     for (auto& t : p->time_fwd) t = nullptr;
     int lo = 0, hi = 0;
     cudaDeviceGetStreamPriorityRange(&lo, &hi);          // hi = numerically lowest = highest priority
@@ -121,16 +156,20 @@ extern "C" hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_tabl
     }
     p->ev.resize(n_sets);
     for (auto& e : p->ev) {
-        cudaEvent_t* all[8] = {&e.inputs, &e.frag, &e.index, &e.prep, &e.gather, &e.forward, &e.x, &e.scatter};
+        cudaEvent_t* all[9] = {&e.inputs, &e.frag,    &e.index, &e.prep,   &e.gather,
+                               &e.forward, &e.x,      &e.scatter, &e.verdict};
         for (auto x : all) {
             *x = nullptr;
             ok = ok && cudaEventCreateWithFlags(x, cudaEventDisableTiming) == cudaSuccess;
         }
     }
+    ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&p->h_verdict), sizeof(int32_t) * n_sets, cudaHostAllocDefault) ==
+                   cudaSuccess;
     if (!ok) {
         hl_pipe_destroy(p);
         return nullptr;
     }
+    for (int i = 0; i < n_sets; ++i) p->h_verdict[i] = -1;
     return p;
 }
 
@@ -143,24 +182,28 @@ extern "C" void hl_pipe_destroy(hl_pipe* p) {
             cudaStreamDestroy(s);
         }
     for (auto& e : p->ev) {
-        cudaEvent_t all[8] = {e.inputs, e.frag, e.index, e.prep, e.gather, e.forward, e.x, e.scatter};
+        cudaEvent_t all[9] = {e.inputs, e.frag, e.index, e.prep, e.gather, e.forward, e.x, e.scatter, e.verdict};
         for (auto x : all)
             if (x) cudaEventDestroy(x);
     }
+    if (p->h_verdict) cudaFreeHost(p->h_verdict);
     delete p;
 }
 
-extern "C" int32_t hl_pipe_submit(hl_pipe* p, const hl_batch* b, const float* d_dense) {
+extern "C" int32_t hl_pipe_submit(hl_pipe* p, const hl_batch* b, const float* d_dense, void* inputs_ready) {
     if (!p || !b) return HL_EINVAL;
-    if (p->j_indexed - p->j_done >= p->n_sets - 1) return HL_ECAPACITY;    // every spare buffer set is in flight
-    HL_PIPE_TRY(record(p->ev[p->j_indexed % p->n_sets].inputs, p->main));   // the inputs are ready at this point
-    HL_PIPE_TRY(submit_index(p, b, d_dense));
-    if (p->j_submitted == p->j_done) HL_PIPE_TRY(submit_link(p));           // nothing staged ahead yet
+    if (p->j_begun - p->j_done >= p->n_sets - 1) return HL_ECAPACITY;      // every spare buffer set is in flight
+    HL_PIPE_TRY(begin_index(p, b, d_dense, inputs_ready));
+    if (p->j_submitted == p->j_done) {                                      // nothing staged ahead yet
+        HL_PIPE_TRY(finish_index(p));
+        HL_PIPE_TRY(submit_link(p));
+    }
     return HL_OK;
 }
 
 extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float* d_grad_non, float lr,
-                                const hl_batch* next, const float* d_next_dense, int32_t* set_index) {
+                                const hl_batch* next, const float* d_next_dense, void* next_inputs_ready,
+                                int32_t* set_index) {
     if (!p || !d_grad_pop || !d_grad_non) return HL_EINVAL;
     const int64_t j = p->j_done;
     if (p->j_submitted < j + 1) return HL_EINVAL;          // hl_pipe_submit first
@@ -168,10 +211,7 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
     hl_pipe_set& st = p->sets[j % n];
     hl_pipe::Events& e = p->ev[j % n];
     const int64_t w0 = (j % 2) * p->window_rows, w1 = ((j + 1) % 2) * p->window_rows;
-    if (next) {
-        if (p->j_indexed - j >= n - 1) return HL_ECAPACITY;
-        HL_PIPE_TRY(record(p->ev[p->j_indexed % n].inputs, p->main));
-    }
+    if (next && p->j_begun - j >= n - 1) return HL_ECAPACITY;
     HL_PIPE_TRY(wait(p->main, e.index));
     if (j >= 1) {
         // rows shared with mini-batch j-1 come out of its staging window once its backward is done
@@ -180,11 +220,7 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
         HL_PIPE_TRY(hl_forward_cold(p->ctx, p->cache, w1, w0, p->window_rows, st.fwd_src, st.n_cold, p->link));
     }
     HL_PIPE_TRY(record(e.forward, p->link));
-    if (p->j_submitted < p->j_indexed) HL_PIPE_TRY(submit_link(p));         // mini-batch j+1, indexed earlier
-    if (next) {
-        HL_PIPE_TRY(submit_index(p, next, d_next_dense));
-        if (p->j_submitted == j + 1) HL_PIPE_TRY(submit_link(p));           // j+1 was indexed only just now
-    }
+    if (p->j_submitted < p->j_indexed) HL_PIPE_TRY(submit_link(p));         // mini-batch j+1, if indexed in full
     if (p->time_fwd[0]) HL_PIPE_TRY(record(p->time_fwd[0], p->main));
     HL_PIPE_TRY(hl_embbag_fwd(p->ctx, p->cache, &st.pop, st.counts, st.pooled_pop, p->main));
     if (p->time_fwd[1]) HL_PIPE_TRY(record(p->time_fwd[1], p->main));
@@ -204,6 +240,16 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
     HL_PIPE_TRY(hl_scatter_cold_at(p->ctx, p->cache, w0, p->window_rows, st.cold_rows, st.n_cold, p->host_table,
                                    p->wb));
     HL_PIPE_TRY(record(e.scatter, p->wb));
+    // The ahead-work comes last: the later the pending cold-row search is ended, the likelier its verdict is known.
+    HL_PIPE_TRY(finish_index(p));                                           // the mini-batch begun one step ago
+    if (p->j_submitted == j + 1 && p->j_submitted < p->j_indexed) HL_PIPE_TRY(submit_link(p));   // mini-batch j+1
+    if (next) {
+        HL_PIPE_TRY(begin_index(p, next, d_next_dense, next_inputs_ready));
+        if (p->j_submitted == j + 1) {                                      // j+1 was begun only just now
+            HL_PIPE_TRY(finish_index(p));
+            HL_PIPE_TRY(submit_link(p));
+        }
+    }
     if (set_index) *set_index = (int32_t)(j % n);
     p->j_done += 1;
     return HL_OK;

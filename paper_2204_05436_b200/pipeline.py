@@ -487,9 +487,11 @@ class PipelinedHotline(Hotline):
             st.ev_gather.record(self.wb)
         self.j_submitted += 1
 
-    def start(self, indices, offsets, batch: int, dense=None, more=()) -> None:
+    def start(self, indices, offsets, batch: int, dense=None, more=(), inputs_ready=None) -> None:
         """Ahead-work of the first mini-batch; ``more`` = the (indices, offsets, batch, dense) tuples of the
-        lookahead - 1 mini-batches after it (fewer if the run is shorter)."""
+        lookahead - 1 mini-batches after it (fewer if the run is shorter).  (``inputs_ready`` is accepted for the
+        interface it shares with NativePipelinedHotline; this scheduler always orders the ahead-work after the main
+        stream.)"""
         assert self.j_submitted == self.j_done, "start() only with nothing in flight"
         assert len(more) <= self.lookahead - 1
         if self.sort_ahead:
@@ -499,7 +501,8 @@ class PipelinedHotline(Hotline):
             self.sets[k % self.n_sets].ev_inputs.record(self.main)
             self._submit(*nb)
 
-    def step(self, grad_pop: torch.Tensor, grad_non: torch.Tensor, lr: float, next_batch=None, timers=None) -> int:
+    def step(self, grad_pop: torch.Tensor, grad_non: torch.Tensor, lr: float, next_batch=None, timers=None,
+             inputs_ready=None) -> int:
         """Main work of the oldest submitted mini-batch; ``next_batch`` = (indices, offsets, batch, dense) of
         the mini-batch ``lookahead`` places after it (its ahead-work is issued here), or None at the end.  Returns
         the index of the buffer set that holds this mini-batch's outputs."""
@@ -608,14 +611,17 @@ class NativePipelinedHotline(Hotline):
         indices, offsets, batch, dense = nb
         return self._batch(indices, offsets, batch), (dense if self.n_dense else None)
 
-    def start(self, indices, offsets, batch: int, dense=None, more=()) -> None:
+    def start(self, indices, offsets, batch: int, dense=None, more=(), inputs_ready=None) -> None:
+        """``inputs_ready`` (also of step()): None = the inputs are complete in the main stream's order; "resident" =
+        they already are (the ahead-work need not wait for what the main stream still has queued); an event."""
         assert self.in_flight == 0, "start() only with nothing in flight"
         for nb in [(indices, offsets, batch, dense)] + [tuple(x) for x in more]:
             b, d = self._hl_batch(nb)
-            B.hl_pipe_submit(self.pipe, b, d)
+            B.hl_pipe_submit(self.pipe, b, d, inputs_ready)
             self.in_flight += 1
 
-    def step(self, grad_pop: torch.Tensor, grad_non: torch.Tensor, lr: float, next_batch=None, timers=None) -> int:
+    def step(self, grad_pop: torch.Tensor, grad_non: torch.Tensor, lr: float, next_batch=None, timers=None,
+             inputs_ready=None) -> int:
         b, d = self._hl_batch(next_batch) if next_batch is not None else (None, None)
         if timers is not None:
             # only the two forward calls can be timed from outside; the events are recorded inside the C call
@@ -623,7 +629,7 @@ class NativePipelinedHotline(Hotline):
             B.hl_pipe_time_forward(self.pipe, *evs)
             timers.setdefault("fwd_pop", []).append((evs[0], evs[1]))
             timers.setdefault("fwd_non", []).append((evs[2], evs[3]))
-        s = B.hl_pipe_step(self.pipe, grad_pop, grad_non, lr, b, d)
+        s = B.hl_pipe_step(self.pipe, grad_pop, grad_non, lr, b, d, inputs_ready)
         self.in_flight += (1 if next_batch is not None else 0) - 1
         return s
 
