@@ -212,7 +212,8 @@ def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: boo
 
 def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: bool = True, profile_batches=None,
                         device: str = "cuda:0", overlap_link: bool = True, sort_ahead: bool = True,
-                        combined_sort: bool = True, lookahead: int = 2, native: bool = False):
+                        combined_sort: bool = True, lookahead: int = 2, native: bool = False,
+                        drain_between: bool = False):
     """Software-pipelined CUDA path (PipelinedHotline) against the oracle processing the same mini-batches one
     after the other.  With integer data every sum is exact, so pooled vectors, the hot cache and the host table
     must agree bit for bit after any number of steps -- which they only do if rows shared by consecutive
@@ -287,15 +288,19 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
                 d_grads.append((gp, gn))
             torch.cuda.synchronize()
             ahead = p.lookahead
+            launches0 = hl.hl_launch_count()
             p.start(*d_batches[0], more=d_batches[1:ahead])
             for step in range(steps):
                 nxt = d_batches[step + ahead] if step + ahead < steps else None
+                if drain_between:
+                    p.drain()        # the device has caught up: what the ahead-work found is known to the host
                 s = p.step(d_grads[step][0], d_grads[step][1], lr, next_batch=nxt)
                 st = p.sets[s]
                 got.append((st.perm.clone(), st.counts.clone(), st.pooled_pop.clone(), st.pooled_non.clone(),
                             st.n_cold.clone()))
             p.drain()
             p.status()
+            launches = hl.hl_launch_count() - launches0
         for step in range(steps):
             perm_o, n_pop_o, pooled_pop_o, pooled_non_o, n_cold_o = expect[step]
             perm_g, counts_g, pp, pn, n_cold_g = [x.cpu().numpy() for x in got[step]]
@@ -318,7 +323,7 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
             assert_close(p.host_table.numpy(), table_o, "host table")
     finally:
         p.close()
-    return dict(shared_cold_rows=shared, steps=steps)
+    return dict(shared_cold_rows=shared, steps=steps, launches=int(launches))
 
 
 def run_fullsize_check(spec, scale_rows: float = 1.0, n_samples: int = 1500, profile_batches=None,

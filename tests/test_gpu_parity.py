@@ -166,6 +166,22 @@ def test_native_pipeline_equals_sequential_steps_integer_data():
     run_pipelined_check(spec, steps=4, integer=True, native=True)
 
 
+def test_native_pipeline_spares_the_general_cold_row_search_once_the_verdict_is_known():
+    """With the device caught up before every step the scheduler knows that the one-cluster kernel has found the
+    distinct cold rows of the mini-batch begun before, and does not queue the general search (8 launches fewer per
+    mini-batch) -- same results, also on a workload where some mini-batches have more cold lookups than that kernel
+    takes and need the general search."""
+    kw = dict(steps=6, scale_rows=0.02, integer=True, profile_batches=6, native=True)
+    known = run_pipelined_check("dlrm_small", drain_between=True, **kw)
+    # 32 kernels per mini-batch with the general search (4 sort passes, digit counts, heads, scan, assignment), 24 without
+    assert known["launches"] <= 6 * 24 + 8
+    spec = dataclasses.replace(gen.CONFIGS["multi_hot"], batch=512, dim=32, rows=("fixed", 2000),
+                               hot_policy=("fraction", 40, 100), profile_batches=2)
+    a = run_pipelined_check(spec, steps=4, integer=True, native=True)
+    b = run_pipelined_check(spec, steps=4, integer=True, native=True, drain_between=True)
+    assert b["launches"] <= a["launches"]          # mini-batches with more cold lookups keep the general search
+
+
 def test_native_pipeline_refuses_what_it_cannot_queue():
     """hl_pipe_step before any hl_pipe_submit, and more submissions than there are spare buffer sets."""
     import numpy as np
