@@ -550,6 +550,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                         ev_cnt.record(s_cnt)
                     ev_cnt.synchronize()
                     bags_pop, bags_non = T * int(o_counts[0]) * S, T * int(o_counts[1]) * S
+                    assert int(o_counts[0]) + int(o_counts[1]) == B, "fragment counts do not add up to the mini-batch"
                     with torch.cuda.stream(s_out):
                         s_out.wait_event(ev_done)
                         o_perm.copy_(st.perm[:B], non_blocking=True)
