@@ -182,6 +182,19 @@ def test_native_pipeline_spares_the_general_cold_row_search_once_the_verdict_is_
     assert b["launches"] <= a["launches"]          # mini-batches with more cold lookups keep the general search
 
 
+@pytest.mark.parametrize("native", [False, True])
+def test_pipelines_with_an_empty_micro_batch(native):
+    """No popular row at all (O is empty, every lookup is cold), and tables so small that the learning phase sees
+    every row (X is empty, nothing crosses the host link): both schedulers, bit-exact on integer data."""
+    none_hot = dataclasses.replace(gen.CONFIGS["tiny"], batch=256, hot_policy=("topk", 0), profile_batches=2)
+    stats = run_pipelined_check(none_hot, steps=4, integer=True, native=native)
+    assert stats["shared_cold_rows"] > 0
+    all_hot = dataclasses.replace(gen.CONFIGS["tiny"], batch=256, rows=("fixed", 40), hot_policy=("fraction", 100, 100),
+                                  profile_batches=8)
+    stats = run_pipelined_check(all_hot, steps=4, integer=True, native=native)
+    assert stats["shared_cold_rows"] == 0
+
+
 def test_native_pipeline_refuses_what_it_cannot_queue():
     """hl_pipe_step before any hl_pipe_submit, and more submissions than there are spare buffer sets."""
     import numpy as np
