@@ -398,6 +398,7 @@ constexpr int kBulkThreads = 128;
 constexpr int kBulkStages = 2;
 constexpr int kBulkStageBytes = 16384;
 constexpr int kBulkMaxPolls = 1 << 22;
+constexpr int kBulkStagesPerCta = 16;     // stages of rows per working CTA before another CTA joins in
 // CTAs of the mover inside the pipeline.  16 CTAs x 16 KB keep 256 KB of rows in flight: 18 K rows of 256 bytes
 // take about 160 us to read and 125 us to write back next to the other streams' kernels.  More CTAs move the rows
 // faster (about 100 us with 2 per SM, alone), fewer slower (one CTA writes back 64 rows every 3.4 us), but what the
@@ -436,7 +437,8 @@ __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_si
                                                                  const int64_t* __restrict__ d_n, int64_t n_max,
                                                                  int64_t table_rows, int row_bytes,
                                                                  int rows_per_stage,
-                                                                 const int32_t* __restrict__ skip, int32_t* status) {
+                                                                 const int32_t* __restrict__ skip, int32_t* status,
+                                                                 int min_ctas) {
     __shared__ __align__(128) unsigned char stage[kBulkStages][kBulkStageBytes];
     __shared__ __align__(8) uint64_t mbar[kBulkStages];
     __shared__ unsigned int stage_bytes[kBulkStages];
@@ -454,8 +456,16 @@ __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_si
     unsigned char* dense = reinterpret_cast<unsigned char*>(dense_side) + dense_row0 * row_bytes;
     unsigned char* tab = reinterpret_cast<unsigned char*>(table);
     const int64_t n_batches = (n + rows_per_stage - 1) / rows_per_stage;
+    // The launch has as many CTAs as the largest transfer could use; how many of them work is decided here, from the
+    // number of rows there really are: min_ctas for a mini-batch's worth of a DLRM-sized model (more would only slow
+    // the kernels that run beside the mover), up to all of them when a mini-batch moves hundreds of thousands of rows
+    // (the link is then all that matters): one more CTA for every kBulkStagesPerCta stages of rows.
+    int64_t active = n_batches / kBulkStagesPerCta;
+    active = active < min_ctas ? min_ctas : active;
+    active = active < (int64_t)gridDim.x ? active : (int64_t)gridDim.x;
+    if ((int64_t)blockIdx.x >= active) return;
     int it = 0;
-    for (int64_t b = blockIdx.x; b < n_batches; b += gridDim.x, ++it) {
+    for (int64_t b = blockIdx.x; b < n_batches; b += active, ++it) {
         const int s = it % kBulkStages;
         const uint32_t parity = (uint32_t)(it / kBulkStages) & 1u;
         const int64_t i0 = b * rows_per_stage;
@@ -520,10 +530,10 @@ int32_t launch_move_rows(float* dense_side, int64_t dense_row0, float* table, co
     const int row_bytes = D * 4;
     if (row_bytes <= kBulkStageBytes) {
         const int rows_per_stage = kBulkStageBytes / row_bytes;
-        const int grid = grid_for(n_max, rows_per_stage, bulk_ctas);
+        const int grid = grid_for(n_max, rows_per_stage, 2 * kSMs);
         k_move_rows_bulk<TO_TABLE><<<grid, kBulkThreads, 0, stream>>>(dense_side, dense_row0, table, rows, d_n, n_max,
                                                                      table_rows, row_bytes, rows_per_stage, skip,
-                                                                     status);
+                                                                     status, bulk_ctas < grid ? bulk_ctas : grid);
         note_launches(1);
         HL_LAUNCH_CHECK();
         return HL_OK;
