@@ -318,6 +318,9 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
     wl = Workload(name, scale, n_batches, args.profile_batches, device, args.threads)
     T, D, S, B = wl.T, wl.D, wl.S, wl.B
     pipelined = not args.no_pipeline
+    eq5 = args.order == "eq5"
+    if eq5 and (args.no_pipeline or args.python_pipeline or args.serial_link):
+        raise SystemExit("--order eq5 is a mode of the library's own scheduler")
     if pipelined:
         if args.python_pipeline or args.serial_link:
             h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
@@ -326,7 +329,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         else:
             h = hl.NativePipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap,
                                           wl.table, n_dense=wl.spec.n_dense, device=str(device),
-                                          lookahead=args.lookahead)
+                                          lookahead=args.lookahead, order=args.order)
     else:
         h = hl.Hotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
                        n_dense=wl.spec.n_dense, device=str(device))
@@ -372,8 +375,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                 if h.idle:
                     h.start(*batch_args(k), more=[batch_args((i + a) % n_batches) for a in range(1, h.lookahead)],
                             inputs_ready="resident")
-                s = h.step(d_grad, d_grad, lr, next_batch=batch_args((i + h.lookahead) % n_batches), timers=timers,
-                           inputs_ready="resident")      # the inputs of the timed region are in HBM already
+                s = h.step(d_grad, None if eq5 else d_grad, lr, next_batch=batch_args((i + h.lookahead) % n_batches),
+                           timers=timers, inputs_ready="resident")   # the timed region's inputs are in HBM already
                 return k, h.sets[s]
             h.step(d_idx[k], d_off[k], B, d_grad, d_grad, lr, dense=d_dense[k], timers=timers)
             return k, h
@@ -539,7 +542,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                     if h.idle:
                         h.start(*batch_args(j % n_batches),
                                 more=[batch_args((j + a) % n_batches) for a in range(1, L)])
-                    st = h.sets[h.step(d_grads[g], d_grads[g], lr, next_batch=batch_args(kin), inputs_ready=ev_in[g])]
+                    st = h.sets[h.step(d_grads[g], None if eq5 else d_grads[g], lr, next_batch=batch_args(kin),
+                                       inputs_ready=ev_in[g])]
                     ev_grad_free[g].record(h.main)
                     ev_done.record(h.main)
                     o_pop, o_non, o_counts, o_perm = outs[g]
@@ -650,6 +654,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                                        args.serial_link else "hl_pipe_*, issued by the library")
                                     + (", host reads after write-backs)" if args.serial_link else
                                        ", host reads overlap write-backs, shared rows forwarded)")
+                                    + ("; order of Eq. 5: both forwards, then one update per row and mini-batch"
+                                       if eq5 else "")
                                     if pipelined else "one mini-batch after the other (Hotline.step)"),
                        "replicas": "independent replica per GPU, no collective"},
             "clocks": clock_info, "gpu_launches": int(launches), "host_enqueue_us_per_step": host_enqueue_us,
@@ -998,6 +1004,9 @@ def main() -> None:
     ap.add_argument("--python-pipeline", action="store_true",
                     help="issue the pipelined schedule from Python (PipelinedHotline) instead of the library's own "
                          "scheduler (hl_pipe_*); gives a time for every call in breakdown_us")
+    ap.add_argument("--order", default="fig8", choices=["fig8", "eq5"],
+                    help="main work of a mini-batch: forward O, update O, forward X, update X (the paper's Fig. 8, "
+                         "default), or both forwards and then one update of every touched row (Eq. 5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather", "tracker"],
                     help="time one library call in isolation")

@@ -256,6 +256,16 @@ HL_API int32_t hl_embbag_bwd_apply2(hl_ctx* ctx, float* d_cache, const int32_t* 
                                     const int32_t* d_sorted_bags, const int32_t* d_n_lookups, int32_t which,
                                     const float* d_grad_out, float lr, void* stream);
 
+/* Section IV-A, Eq. 5 (the two micro-batches together give the mini-batch's gradient): hl_embbag_bwd_prepare_merged
+ * sorts the pairs of O and X in ONE key space, X's bags numbered behind O's, so that all lookups of a row, from either
+ * micro-batch, form one run.  hl_embbag_bwd_apply(ctx, cache, slots, bags, d_n_lookups + 2, d_grad_all, lr, stream) on
+ * the result, with d_grad_all = [gradients of O's bags; gradients of X's bags] (X's block starts at row
+ * T * (*d_n_pop) * S), then updates every row once with the whole mini-batch's gradient -- the result of the
+ * unfragmented step when both forwards ran before it.  Same arguments and scratch as hl_embbag_bwd_prepare2. */
+HL_API int32_t hl_embbag_bwd_prepare_merged(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_n_pop,
+                                            const hl_ubatch* non, const int32_t* d_n_non, int32_t* d_sorted_slots,
+                                            int32_t* d_sorted_bags, int32_t* d_n_lookups, void* stream);
+
 /* Sections IV and V-A (dma_rd of non-popular rows; popular rows of X are read from GPU memory).
  * In:  non->ids = global rows of X (from hl_fragment), *d_n_non = inputs in X.
  * Out: d_cold_rows[0 .. *d_n_cold) = the distinct non-popular rows referenced by X, ascending (each staged
@@ -368,6 +378,15 @@ typedef struct hl_pipe hl_pipe;
 HL_API hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows, int32_t n_sets,
                                const hl_pipe_set* sets, int32_t n_dense, void* main_stream);
 HL_API void hl_pipe_destroy(hl_pipe* p);
+
+/* Order of a mini-batch's main work.  HL_PIPE_ORDER_FIG8 (default): forward O, update O, forward X, update X, as the
+ * paper's Fig. 8 draws it.  HL_PIPE_ORDER_EQ5: forward O, forward X, then one update of every touched row with the
+ * gradient of the whole mini-batch (Section IV-A, Eq. 5) -- the unfragmented step's result; hl_pipe_step then takes the
+ * gradients of O's and X's bags in one array d_grad_pop = [O's bags; X's bags] and ignores d_grad_non.  Set it
+ * before the first hl_pipe_submit. */
+#define HL_PIPE_ORDER_FIG8 0
+#define HL_PIPE_ORDER_EQ5  1
+HL_API int32_t hl_pipe_set_order(hl_pipe* p, int32_t order);
 
 /* Queues the ahead-work of the next mini-batch (d_dense may be NULL).  inputs_ready says when its indices, offsets and
  * dense features are complete: NULL = in main_stream's order at the time of the call; a cudaEvent_t = when that event

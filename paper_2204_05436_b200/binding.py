@@ -24,6 +24,7 @@ EXPORTS = (
     "hl_tracker_reset", "hl_tracker_update", "hl_tracker_export",
     "hl_pipe_create", "hl_pipe_destroy", "hl_pipe_submit", "hl_pipe_step", "hl_pipe_wait_outputs", "hl_pipe_drain", "hl_pipe_time_forward", "hl_pipe_wait_counts",
     "hl_index_cold_begin", "hl_index_cold_end", "hl_index_cold_verdict",
+    "hl_embbag_bwd_prepare_merged", "hl_pipe_set_order",
 )
 
 
@@ -140,6 +141,10 @@ def _load() -> ctypes.CDLL:
     lib.hl_index_cold_verdict.argtypes = [vp]
     lib.hl_index_cold_end.restype = i32
     lib.hl_index_cold_end.argtypes = [vp, ctypes.POINTER(hl_ubatch), i64, i64, vp, vp, vp, vp, vp, i32, vp]
+    lib.hl_embbag_bwd_prepare_merged.restype = i32
+    lib.hl_embbag_bwd_prepare_merged.argtypes = [vp, ctypes.POINTER(hl_ubatch), vp, ctypes.POINTER(hl_ubatch), vp, vp, vp, vp, vp]
+    lib.hl_pipe_set_order.restype = i32
+    lib.hl_pipe_set_order.argtypes = [vp, i32]
     lib.hl_pipe_wait_counts.restype = i32
     lib.hl_pipe_wait_counts.argtypes = [vp, vp]
     lib.hl_pipe_time_forward.restype = i32
@@ -476,3 +481,17 @@ def hl_index_cold_end(ctx: int, non: hl_ubatch, stage_row0: int, stage_rows: int
                                                        _ptr(d_cold_rows), _ptr(d_n_cold), _ptr(d_prev_cold_rows),
                                                        _ptr(d_n_prev), _ptr(d_fwd_src), int(bool(general_not_needed)),
                                                        stream))
+
+
+HL_PIPE_ORDER_FIG8, HL_PIPE_ORDER_EQ5 = 0, 1
+
+
+def hl_embbag_bwd_prepare_merged(ctx: int, pop: hl_ubatch, d_n_pop, non: hl_ubatch, d_n_non, d_sorted_slots,
+                                 d_sorted_bags, d_n_lookups, stream: int) -> None:
+    _check("hl_embbag_bwd_prepare_merged", _lib.hl_embbag_bwd_prepare_merged(
+        ctx, ctypes.byref(pop), _ptr(d_n_pop), ctypes.byref(non), _ptr(d_n_non), _ptr(d_sorted_slots),
+        _ptr(d_sorted_bags), _ptr(d_n_lookups), stream))
+
+
+def hl_pipe_set_order(pipe: int, order: int) -> None:
+    _check("hl_pipe_set_order", _lib.hl_pipe_set_order(pipe, int(order)))

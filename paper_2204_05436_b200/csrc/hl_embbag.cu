@@ -157,10 +157,14 @@ __global__ void __launch_bounds__(kThreads) k_bwd_pairs(const int32_t* __restric
                                                         int32_t* __restrict__ d_n_lookups,
                                                         const int32_t* __restrict__ d_pos0, int32_t key_bias,
                                                         int32_t sentinel, int32_t* __restrict__ d_total,
-                                                        int32_t* status) {
-    // pairs go to positions pos0 + j (pos0 = *d_pos0 or 0) with key = slot + key_bias; *d_n_lookups = this
-    // micro-batch's lookups, *d_total (if given) = pos0 + that
+                                                        int32_t* status,
+                                                        const int32_t* __restrict__ d_bag_bias_samples = nullptr) {
+    // pairs go to positions pos0 + j (pos0 = *d_pos0 or 0) with key = slot + key_bias and value = bag (+ the bags of
+    // *d_bag_bias_samples inputs, if given); *d_n_lookups = this micro-batch's lookups, *d_total (if given) = pos0 +
+    // that
     const int64_t pos0 = d_pos0 ? d_pos0[0] : 0;
+    const int64_t bag_bias =
+        d_bag_bias_samples ? (int64_t)clamp_samples(d_bag_bias_samples, max_batch) * bags_per_sample_all : 0;
     const int64_t n_bags = (int64_t)clamp_samples(d_n_samples, max_batch) * bags_per_sample_all;
     const int sub = threadIdx.x % GROUP;
     const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / GROUP;
@@ -181,7 +185,7 @@ __global__ void __launch_bounds__(kThreads) k_bwd_pairs(const int32_t* __restric
             const int32_t id = ids[j];
             if (id >= n_slots) set_status(status, HL_EBOUNDS);
             keys[pos0 + j] = (id < 0 || id >= n_slots) ? sentinel : id + key_bias;
-            vals[pos0 + j] = (int32_t)bag;
+            vals[pos0 + j] = (int32_t)(bag + bag_bias);
         }
     }
 }
@@ -638,9 +642,12 @@ extern "C" int32_t hl_embbag_bwd_prepare(hl_ctx* ctx, const hl_ubatch* ub, const
     return sort_lookups(ctx, ub, d_n_samples, d_sorted_slots, d_sorted_bags, d_n_lookups, &keys, &vals, stream);
 }
 
-extern "C" int32_t hl_embbag_bwd_prepare2(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_n_pop,
-                                          const hl_ubatch* non, const int32_t* d_n_non, int32_t* d_sorted_slots,
-                                          int32_t* d_sorted_bags, int32_t* d_n_lookups, void* stream_) {
+static int32_t prepare_both(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_n_pop, const hl_ubatch* non,
+                            const int32_t* d_n_non, int32_t* d_sorted_slots, int32_t* d_sorted_bags,
+                            int32_t* d_n_lookups, bool merge, void* stream_) {
+    // merge = false: X's keys are offset by the number of slots, so that the sorted list is O's pairs, then X's;
+    // merge = true: one key space, and X's bags are numbered behind O's: the lookups of a row from both
+    // micro-batches form one run, over one gradient array [bags of O; bags of X]
     if (!ctx || !pop || !non || !pop->offsets || !non->offsets || !d_n_pop || !d_n_non || !d_n_lookups)
         return HL_EINVAL;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -652,13 +659,13 @@ extern "C" int32_t hl_embbag_bwd_prepare2(hl_ctx* ctx, const hl_ubatch* pop, con
     Regions& r = ctx->r;
     const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
     if (2 * n_slots + 1 >= (int64_t(1) << 31)) return HL_EINVAL;
-    const int key_bits = bits_for(2 * n_slots);          // O's keys are slots, X's are n_slots + slot
+    const int key_bits = bits_for(merge ? n_slots : 2 * n_slots);
     const int passes = (key_bits + 7) / 8;
     int32_t* keys[2] = {r.bwd_keys[0], r.bwd_keys[1]};
     int32_t* vals[2] = {r.bwd_vals[0], r.bwd_vals[1]};
     keys[passes & 1] = d_sorted_slots;
     vals[passes & 1] = d_sorted_bags;
-    const int32_t sentinel = (int32_t)(2 * n_slots);
+    const int32_t sentinel = (int32_t)(merge ? n_slots : 2 * n_slots);
     const bool short_bags = ctx->max_nnz <= 4 * ctx->max_bags;
     const int per_block = short_bags ? kThreads : kThreads / 32;
     const int grid = grid_for(ctx->max_bags, per_block, kMaxGrid);
@@ -666,22 +673,35 @@ extern "C" int32_t hl_embbag_bwd_prepare2(hl_ctx* ctx, const hl_ubatch* pop, con
     const int32_t* ns[2] = {d_n_pop, d_n_non};
     for (int m = 0; m < 2; ++m) {
         const int32_t* pos0 = m == 0 ? nullptr : d_n_lookups;
-        const int32_t bias = m == 0 ? 0 : (int32_t)n_slots;
+        const int32_t bias = (m == 0 || merge) ? 0 : (int32_t)n_slots;
+        const int32_t* bag_bias = (m == 1 && merge) ? d_n_pop : nullptr;
         if (short_bags)
             k_bwd_pairs<1><<<grid, kThreads, 0, stream>>>(ubs[m]->ids, ubs[m]->offsets, ns[m], ctx->max_batch,
                                                          ctx->T * ctx->S, n_slots, ctx->max_nnz, keys[0], vals[0],
                                                          d_n_lookups + m, pos0, bias, sentinel, d_n_lookups + 2,
-                                                         r.status);
+                                                         r.status, bag_bias);
         else
             k_bwd_pairs<32><<<grid, kThreads, 0, stream>>>(ubs[m]->ids, ubs[m]->offsets, ns[m], ctx->max_batch,
                                                           ctx->T * ctx->S, n_slots, ctx->max_nnz, keys[0], vals[0],
                                                           d_n_lookups + m, pos0, bias, sentinel, d_n_lookups + 2,
-                                                          r.status);
+                                                          r.status, bag_bias);
     }
     note_launches(2);
     HL_LAUNCH_CHECK();
     int32_t *ok, *ov;
     return radix_sort_pairs(keys, vals, d_n_lookups + 2, ctx->max_nnz, key_bits, r.bwd_hist, r.status, &ok, &ov, stream);
+}
+
+extern "C" int32_t hl_embbag_bwd_prepare2(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_n_pop,
+                                          const hl_ubatch* non, const int32_t* d_n_non, int32_t* d_sorted_slots,
+                                          int32_t* d_sorted_bags, int32_t* d_n_lookups, void* stream) {
+    return prepare_both(ctx, pop, d_n_pop, non, d_n_non, d_sorted_slots, d_sorted_bags, d_n_lookups, false, stream);
+}
+
+extern "C" int32_t hl_embbag_bwd_prepare_merged(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_n_pop,
+                                                const hl_ubatch* non, const int32_t* d_n_non, int32_t* d_sorted_slots,
+                                                int32_t* d_sorted_bags, int32_t* d_n_lookups, void* stream) {
+    return prepare_both(ctx, pop, d_n_pop, non, d_n_non, d_sorted_slots, d_sorted_bags, d_n_lookups, true, stream);
 }
 
 extern "C" int32_t hl_embbag_bwd_apply2(hl_ctx* ctx, float* d_cache, const int32_t* d_sorted_slots,

@@ -32,6 +32,7 @@ struct hl_pipe {
     // sort are queued in full (indexed), whose host read is queued (submitted), whose main work is queued (done)
     int64_t j_begun, j_indexed, j_submitted, j_done;
     int32_t* h_verdict;          // pinned host words, one per set: what the first half of the cold-row search found
+    int order;                   // HL_PIPE_ORDER_*
     cudaEvent_t time_fwd[4];     // one-shot: recorded around the two forward calls of the next step
 };
 
@@ -67,8 +68,12 @@ int32_t finish_index(hl_pipe* p) {
                                   known_done ? 1 : 0, p->sc));
     HL_PIPE_TRY(record(e.index, p->sc));
     HL_PIPE_TRY(wait(p->sb, e.index));
-    HL_PIPE_TRY(hl_embbag_bwd_prepare2(p->ctx, &st.pop, st.counts, &st.non, st.counts + 1, st.sorted_slots,
-                                       st.sorted_bags, st.sorted_n, p->sb));
+    if (p->order == HL_PIPE_ORDER_EQ5)
+        HL_PIPE_TRY(hl_embbag_bwd_prepare_merged(p->ctx, &st.pop, st.counts, &st.non, st.counts + 1, st.sorted_slots,
+                                                 st.sorted_bags, st.sorted_n, p->sb));
+    else
+        HL_PIPE_TRY(hl_embbag_bwd_prepare2(p->ctx, &st.pop, st.counts, &st.non, st.counts + 1, st.sorted_slots,
+                                           st.sorted_bags, st.sorted_n, p->sb));
     HL_PIPE_TRY(record(e.prep, p->sb));
     p->j_indexed += 1;
     return HL_OK;
@@ -145,6 +150,7 @@ extern "C" hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_tabl
     p->main = static_cast<cudaStream_t>(main_stream);
     p->j_begun = p->j_indexed = p->j_submitted = p->j_done = 0;
     p->h_verdict = nullptr;
+    p->order = HL_PIPE_ORDER_FIG8;
     for (auto& t : p->time_fwd) t = nullptr;
     int lo = 0, hi = 0;
     cudaDeviceGetStreamPriorityRange(&lo, &hi);          // hi = numerically lowest = highest priority
@@ -204,7 +210,7 @@ extern "C" int32_t hl_pipe_submit(hl_pipe* p, const hl_batch* b, const float* d_
 extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float* d_grad_non, float lr,
                                 const hl_batch* next, const float* d_next_dense, void* next_inputs_ready,
                                 int32_t* set_index) {
-    if (!p || !d_grad_pop || !d_grad_non) return HL_EINVAL;
+    if (!p || !d_grad_pop || (!d_grad_non && p->order != HL_PIPE_ORDER_EQ5)) return HL_EINVAL;
     const int64_t j = p->j_done;
     if (p->j_submitted < j + 1) return HL_EINVAL;          // hl_pipe_submit first
     const int n = p->n_sets;
@@ -224,17 +230,25 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
     if (p->time_fwd[0]) HL_PIPE_TRY(record(p->time_fwd[0], p->main));
     HL_PIPE_TRY(hl_embbag_fwd(p->ctx, p->cache, &st.pop, st.counts, st.pooled_pop, p->main));
     if (p->time_fwd[1]) HL_PIPE_TRY(record(p->time_fwd[1], p->main));
-    HL_PIPE_TRY(wait(p->main, e.prep));
-    HL_PIPE_TRY(hl_embbag_bwd_apply2(p->ctx, p->cache, st.sorted_slots, st.sorted_bags, st.sorted_n, 0, d_grad_pop, lr,
-                                     p->main));
+    if (p->order == HL_PIPE_ORDER_FIG8) {
+        HL_PIPE_TRY(wait(p->main, e.prep));
+        HL_PIPE_TRY(hl_embbag_bwd_apply2(p->ctx, p->cache, st.sorted_slots, st.sorted_bags, st.sorted_n, 0, d_grad_pop,
+                                         lr, p->main));
+    }
     HL_PIPE_TRY(wait(p->main, e.gather));
     HL_PIPE_TRY(wait(p->main, e.forward));
     if (p->time_fwd[2]) HL_PIPE_TRY(record(p->time_fwd[2], p->main));
     HL_PIPE_TRY(hl_embbag_fwd(p->ctx, p->cache, &st.non, st.counts + 1, st.pooled_non, p->main));
     if (p->time_fwd[3]) HL_PIPE_TRY(record(p->time_fwd[3], p->main));
     for (auto& t : p->time_fwd) t = nullptr;
-    HL_PIPE_TRY(hl_embbag_bwd_apply2(p->ctx, p->cache, st.sorted_slots, st.sorted_bags, st.sorted_n, 1, d_grad_non, lr,
-                                     p->main));
+    if (p->order == HL_PIPE_ORDER_FIG8) {
+        HL_PIPE_TRY(hl_embbag_bwd_apply2(p->ctx, p->cache, st.sorted_slots, st.sorted_bags, st.sorted_n, 1, d_grad_non,
+                                         lr, p->main));
+    } else {   // one update of every touched row with the gradient of the whole mini-batch
+        HL_PIPE_TRY(wait(p->main, e.prep));
+        HL_PIPE_TRY(hl_embbag_bwd_apply(p->ctx, p->cache, st.sorted_slots, st.sorted_bags, st.sorted_n + 2, d_grad_pop,
+                                        lr, p->main));
+    }
     HL_PIPE_TRY(record(e.x, p->main));
     HL_PIPE_TRY(wait(p->wb, e.x));
     HL_PIPE_TRY(hl_scatter_cold_at(p->ctx, p->cache, w0, p->window_rows, st.cold_rows, st.n_cold, p->host_table,
@@ -252,6 +266,13 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
     }
     if (set_index) *set_index = (int32_t)(j % n);
     p->j_done += 1;
+    return HL_OK;
+}
+
+extern "C" int32_t hl_pipe_set_order(hl_pipe* p, int32_t order) {
+    if (!p || (order != HL_PIPE_ORDER_FIG8 && order != HL_PIPE_ORDER_EQ5)) return HL_EINVAL;
+    if (p->j_begun != 0) return HL_EINVAL;       // the sorts queued so far were made for the other order
+    p->order = order;
     return HL_OK;
 }
 

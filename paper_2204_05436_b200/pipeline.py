@@ -578,7 +578,12 @@ class NativePipelinedHotline(Hotline):
     """
 
     def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
-                 n_dense: int = 0, device: str = "cuda:0", lookahead: int = 2):
+                 n_dense: int = 0, device: str = "cuda:0", lookahead: int = 2, order: str = "fig8"):
+        """``order``: "fig8" = forward O, update O, forward X, update X (the paper's Fig. 8); "eq5" = both forwards,
+        then one update of every touched row with the whole mini-batch's gradient (Eq. 5; the unfragmented step's
+        result): step() then takes ``grad_pop`` = [gradients of O's bags; gradients of X's bags] and no ``grad_non``."""
+        assert order in ("fig8", "eq5")
+        self.order = order
         self.window_rows = int(window_rows)
         self.lookahead = max(1, int(lookahead))
         super().__init__(table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, 2 * self.window_rows,
@@ -594,6 +599,8 @@ class NativePipelinedHotline(Hotline):
         torch.cuda.synchronize(self.device)
         self.pipe = B.hl_pipe_create(self.ctx, self.cache, self.host_table, self.window_rows, c_sets, self.n_dense,
                                      self.main.cuda_stream)
+        if order == "eq5":
+            B.hl_pipe_set_order(self.pipe, B.HL_PIPE_ORDER_EQ5)
         self.in_flight = 0
         self._timer_pool = []
 

@@ -213,7 +213,7 @@ def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: boo
 def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: bool = True, profile_batches=None,
                         device: str = "cuda:0", overlap_link: bool = True, sort_ahead: bool = True,
                         combined_sort: bool = True, lookahead: int = 2, native: bool = False,
-                        drain_between: bool = False):
+                        drain_between: bool = False, order: str = "fig8"):
     """Software-pipelined CUDA path (PipelinedHotline) against the oracle processing the same mini-batches one
     after the other.  With integer data every sum is exact, so pooled vectors, the hot cache and the host table
     must agree bit for bit after any number of steps -- which they only do if rows shared by consecutive
@@ -254,9 +254,22 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
         perm_o, n_pop_o, _, _, _ = orc.fragment(batch.indices, batch.offsets, B, geom.table_rows, remap_o, S)
         g_pop, _ = mu_grad(grad_full, perm_o[:n_pop_o], T, B, S)
         g_non, _ = mu_grad(grad_full, perm_o[n_pop_o:], T, B, S)
-        out = orc.hotline_step(table_o, cache_o, hot_cap, remap_o, batch.indices, batch.offsets, B, geom.table_rows,
-                               S, g_pop, g_non, lr)
-        _, _, _, _, C, pooled_pop_o, pooled_non_o = out
+        if order == "fig8":
+            out = orc.hotline_step(table_o, cache_o, hot_cap, remap_o, batch.indices, batch.offsets, B,
+                                   geom.table_rows, S, g_pop, g_non, lr)
+            _, _, _, _, C, pooled_pop_o, pooled_non_o = out
+        else:
+            # Eq. 5: both forwards, then ONE update of every touched row with the whole mini-batch's gradient --
+            # the oracle's steps put together: O's and X's lookups as one CSR over [O's bags; X's bags]
+            _, _, O, X, _ = orc.fragment(batch.indices, batch.offsets, B, geom.table_rows, remap_o, S)
+            C, x_slots = orc.gather_cold(X.ids, remap_o, hot_cap)
+            cache_o[hot_cap: hot_cap + len(C)] = orc.stage_cold_rows(table_o, C)
+            pooled_pop_o = orc.embbag_fwd(cache_o, O.ids, O.offsets)
+            pooled_non_o = orc.embbag_fwd(cache_o, x_slots, X.offsets)
+            ids_all = np.concatenate([O.ids, x_slots])
+            offsets_all = np.concatenate([O.offsets, X.offsets[1:] + len(O.ids)])
+            orc.embbag_bwd_sgd(cache_o, ids_all, offsets_all, np.concatenate([g_pop, g_non]), lr)
+            orc.scatter_cold(table_o, C, cache_o[hot_cap: hot_cap + len(C)])
         shared += len(np.intersect1d(C, prev_C))
         prev_C = C
         batches.append(batch)
@@ -267,7 +280,7 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
     host_table = torch.from_numpy(table0.copy()).pin_memory()
     if native:
         p = hl.NativePipelinedHotline(geom.table_rows, D, S, B, max_nnz, hot_cap, window, host_table,
-                                      n_dense=spec.n_dense, device=device, lookahead=lookahead)
+                                      n_dense=spec.n_dense, device=device, lookahead=lookahead, order=order)
     else:
         p = hl.PipelinedHotline(geom.table_rows, D, S, B, max_nnz, hot_cap, window, host_table, n_dense=spec.n_dense,
                                 device=device, overlap_link=overlap_link, sort_ahead=sort_ahead,
@@ -285,6 +298,9 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
                 gn = torch.zeros((n_bags, D), dtype=torch.float32, device=device)
                 gp[:len(g_pop)] = _t(g_pop, device)
                 gn[:len(g_non)] = _t(g_non, device)
+                if order == "eq5":       # one array: the gradients of O's bags, then those of X's bags
+                    gp[len(g_pop):len(g_pop) + len(g_non)] = _t(g_non, device)
+                    gn = None
                 d_grads.append((gp, gn))
             torch.cuda.synchronize()
             ahead = p.lookahead

@@ -195,6 +195,18 @@ def test_pipelines_with_an_empty_micro_batch(native):
     assert stats["shared_cold_rows"] == 0
 
 
+def test_native_pipeline_in_the_order_of_eq5_one_update_per_row_and_mini_batch():
+    """Both forwards, then one update of every touched row with the gradient of the whole mini-batch (the lookups of a
+    row from O and from X form one run of the merged sort): bit-exact on integer data, within the tolerance on real
+    data, with rows that O and X share (hot rows) and rows that consecutive mini-batches share (forwarded)."""
+    assert run_pipelined_check("tiny", steps=6, integer=True, native=True, order="eq5")["shared_cold_rows"] > 50
+    spec = dataclasses.replace(gen.CONFIGS["multi_hot"], batch=512, dim=32, rows=("fixed", 2000),
+                               hot_policy=("fraction", 40, 100), profile_batches=2)
+    run_pipelined_check(spec, steps=4, integer=True, native=True, order="eq5")
+    run_pipelined_check("dlrm_small", steps=3, scale_rows=0.02, integer=False, profile_batches=6, native=True,
+                        order="eq5")
+
+
 def test_native_pipeline_refuses_what_it_cannot_queue():
     """hl_pipe_step before any hl_pipe_submit, and more submissions than there are spare buffer sets."""
     import numpy as np
