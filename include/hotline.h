@@ -373,8 +373,8 @@ typedef struct hl_pipe hl_pipe;
  * run on streams the pipeline creates; rows that consecutive mini-batches share are forwarded between the two
  * staging windows (hl_forward_cold).  The results are those of processing the mini-batches one after the other.
  * d_cache [hot_cap + staging_cap, D] with staging_cap >= 2 * window_rows; host_table as for hl_gather_cold;
- * sets[n_sets] (3 <= n_sets <= 16) are copied.  No device memory is allocated; streams and events are.
- * Returns NULL on invalid arguments or if a stream or event cannot be created. */
+ * sets[n_sets] (3 <= n_sets <= 16) are copied.  No device memory is allocated; streams, events and a few pinned host
+ * words are.  Returns NULL on invalid arguments or if one of those cannot be created. */
 HL_API hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows, int32_t n_sets,
                                const hl_pipe_set* sets, int32_t n_dense, void* main_stream);
 HL_API void hl_pipe_destroy(hl_pipe* p);
@@ -398,9 +398,10 @@ HL_API int32_t hl_pipe_submit(hl_pipe* p, const hl_batch* b, const float* d_dens
 
 /* Queues the main work of the oldest submitted mini-batch: forward and update of O, forward and update of X with the
  * upstream gradients d_grad_pop / d_grad_non ([bags of O, D] / [bags of X, D], in the micro-batches' bag order), and
- * its write-back; and the ahead-work of `next` (may be NULL; next_inputs_ready as for hl_pipe_submit).  *set_index = which of the sets holds this mini-batch's
- * perm, counts and pooled vectors; they are complete in main_stream's order, and the set is reused n_sets steps on.
- * No call waits for the device. */
+ * its write-back; and the ahead-work of `next` (may be NULL; next_inputs_ready as for hl_pipe_submit).
+ * *set_index = which of the sets holds this mini-batch's perm, counts and pooled vectors; they are complete in
+ * main_stream's order, and the set is reused n_sets steps on.  HL_EINVAL if no mini-batch has been submitted,
+ * HL_ECAPACITY if `next` finds every buffer set in flight (nothing is queued then).  No call waits for the device. */
 HL_API int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float* d_grad_non, float lr,
                             const hl_batch* next, const float* d_next_dense, void* next_inputs_ready,
                             int32_t* set_index);
