@@ -314,7 +314,9 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         dist.init_process_group("nccl", device_id=device)
 
     name, scale = pick_workload(args.workload, world)
-    n_batches = 8
+    if args.row_scale is not None:
+        scale = args.row_scale       # a labelled variant: every table shrunk by this factor
+    n_batches = 16                   # distinct pre-generated mini-batches the timed steps rotate over
     wl = Workload(name, scale, n_batches, args.profile_batches, device, args.threads)
     T, D, S, B = wl.T, wl.D, wl.S, wl.B
     pipelined = not args.no_pipeline
@@ -990,6 +992,9 @@ def main() -> None:
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="auto", choices=["auto"] + sorted(gen.CONFIGS))
     ap.add_argument("--profile-batches", type=int, default=None)
+    ap.add_argument("--row-scale", type=float, default=None,
+                    help="shrink every table of the workload by this factor (a labelled variant, e.g. to reach the "
+                         "share of popular inputs the paper reports)")
     ap.add_argument("--threads", type=int, default=min(16, os.cpu_count() or 1))
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-pipeline", action="store_true",
