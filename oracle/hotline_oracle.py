@@ -55,7 +55,7 @@ def lookups_of(indices, offsets, batch: int, table_rows, bags_per_sample: int = 
 # ----------------------------------------------------------------------------------------------------------
 def access_counts(batches: Iterable, batch: int, table_rows, bags_per_sample: int = 1) -> np.ndarray:
     """cnt[g] = number of lookups of global row g over the profiled mini-batches; every occurrence counts,
-    also repeats inside one bag (the access logger "tracks the frequency of access", Section V-B; this is
+    also repeats inside one bag (the access logger keeps a per-row access frequency, Section V-B; this is
     the exact counter the paper calls the Oracle LFU logger)."""
     N = int(np.sum(np.asarray(table_rows, dtype=np.int64)))
     rows = [np.zeros(0, dtype=np.int64)]
@@ -102,7 +102,7 @@ def hot_capacity(policy: tuple, total_rows: int, dim: int) -> int:
 
 def build_remap(hot_rows: np.ndarray, total_rows: int) -> np.ndarray:
     """remap[g] = i if hot_rows[i] == g else -1: the slot of a popular row in the HBM cache is its rank among
-    the popular rows in ascending global id (the accelerator "stores only the indices", Section IV)."""
+    the popular rows in ascending global id (the access logger holds row indices, never row values: Section V-B)."""
     hot_rows = np.asarray(hot_rows, dtype=np.int64)
     assert (np.diff(hot_rows) > 0).all()
     remap = np.full(int(total_rows), -1, dtype=np.int32)
@@ -149,8 +149,8 @@ def fragment(indices, offsets, batch: int, table_rows, remap: np.ndarray, bags_p
     """Split mini-batch M into popular O and non-popular X.
 
     An input is popular iff *every* one of its lookups, over all tables and steps, addresses a popular row
-    (a single miss makes it non-popular, Section I; the Lookup Engine tests that "all embedding indices" are
-    logged, Section V-C); an input with no lookups is vacuously popular.  O and X partition M (Eq. 3); inside
+    (a single miss makes it non-popular, Section I; the Lookup Engine checks every index of the input against
+    the logger, Section V-C); an input with no lookups is vacuously popular.  O and X partition M (Eq. 3); inside
     each, inputs keep their order in M.  Returns (perm, n_pop, O, X, dense_out): perm lists O's inputs then
     X's; O.ids are cache slots, X.ids are global row ids; dense_out[i] = dense[perm[i]].
     """

@@ -500,6 +500,117 @@ def test_hand_worked_example():
     assert cache[:, 0].tolist() == g["cache_after"]
 
 
+def test_hand_worked_example_pins_the_order_of_a_step():
+    """hotline_step as a whole, in both orders, against tests/golden/worked_example_order.txt: X looks up popular
+    rows that O updates, so X's pooled vectors differ between the order of Fig. 8 (O forward, O update, X forward,
+    X update: the default) and the order of Eq. 5 (both forwards first)."""
+    g = _read_golden(os.path.join(GOLDEN, "worked_example_order.txt"))
+    tr, B, S = tuple(g["table_rows"]), g["batch"][0], 1
+    ind = np.asarray(g["indices"], dtype=np.int32)
+    off = np.asarray(g["offsets"], dtype=np.int32)
+    hot = np.asarray(g["hot_rows"], dtype=np.int64)
+    hot_cap = g["hot_cap"][0]
+    remap = orc.build_remap(hot, sum(tr))
+    gp = np.asarray(g["grad_pop"], dtype=np.float32).reshape(-1, 1)
+    gn = np.asarray(g["grad_non"], dtype=np.float32).reshape(-1, 1)
+    assert g["pooled_non_fig8"] != g["pooled_non_eq5"]
+    for deferred, key in ((False, "pooled_non_fig8"), (True, "pooled_non_eq5")):
+        table = np.asarray(g["table"], dtype=np.float32).reshape(sum(tr), 1)
+        cache = np.zeros((hot_cap + len(g["cold_rows"]), 1), dtype=np.float32)
+        cache[: len(hot)] = orc.load_hot_cache(table, hot)
+        perm, n_pop, O, X, C, pooled_pop, pooled_non = orc.hotline_step(
+            table, cache, hot_cap, remap, ind, off, B, tr, S, gp, gn, g["lr"][0], deferred=deferred)
+        assert perm.tolist() == g["perm"] and n_pop == g["n_pop"][0]
+        assert O.offsets.tolist() == g["pop_offsets"] and O.ids.tolist() == g["pop_slots"]
+        assert X.offsets.tolist() == g["non_offsets"] and X.ids.tolist() == g["non_slots"]
+        assert C.tolist() == g["cold_rows"]
+        assert pooled_pop[:, 0].tolist() == g["pooled_pop"]
+        assert pooled_non[:, 0].tolist() == g[key], (deferred, pooled_non[:, 0].tolist())
+        assert cache[:, 0].tolist() == g["cache_after"]
+        assert table[:, 0].tolist() == g["table_after"]
+    # the default is the order of Fig. 8
+    table = np.asarray(g["table"], dtype=np.float32).reshape(sum(tr), 1)
+    cache = np.zeros((hot_cap + len(g["cold_rows"]), 1), dtype=np.float32)
+    cache[: len(hot)] = orc.load_hot_cache(table, hot)
+    out = orc.hotline_step(table, cache, hot_cap, remap, ind, off, B, tr, S, gp, gn, g["lr"][0])
+    assert out[6][:, 0].tolist() == g["pooled_non_fig8"]
+
+
+def brute_step_fig8(table, indices, offsets, B, tr, S, hot_rows, grad_full, lr):
+    """The step of Fig. 8 with plain loops over a dict of rows, no cache and no slots: O's bags are pooled, O's
+    rows updated, then X's bags are pooled from the rows as they are now, then X's rows updated.  Returns pooled
+    vectors in the mini-batch's own bag order and the final rows (fp64 arithmetic, rounded to fp32 per update)."""
+    perm, n_pop, _, _ = brute_fragment(indices, offsets, B, tr, S, set(hot_rows))
+    T, D = len(tr), table.shape[1]
+    base = [0]
+    for r in tr:
+        base.append(base[-1] + r)
+    rows = {g: table[g].astype(np.float32).copy() for g in range(sum(tr))}
+    pooled = np.zeros((T * B * S, D), dtype=np.float32)
+    lr64 = float(np.float32(lr))
+    for samples in (perm[:n_pop], perm[n_pop:]):
+        bags = [(t, (t * B + b) * S + s) for t in range(T) for b in samples for s in range(S)]
+        for t, bag in bags:                                   # forward of this micro-batch
+            acc = np.zeros(D, dtype=np.float64)
+            for j in range(offsets[bag], offsets[bag + 1]):
+                acc += rows[base[t] + int(indices[j])].astype(np.float64)
+            pooled[bag] = acc.astype(np.float32)
+        G = {}
+        for t, bag in bags:                                   # its update: one per touched row
+            for j in range(offsets[bag], offsets[bag + 1]):
+                g = base[t] + int(indices[j])
+                G[g] = G.get(g, np.zeros(D, dtype=np.float64)) + grad_full[bag].astype(np.float64)
+        for g, grad in G.items():
+            rows[g] = (rows[g].astype(np.float64) - lr64 * grad).astype(np.float32)
+    return pooled, np.stack([rows[g] for g in range(sum(tr))])
+
+
+@pytest.mark.parametrize("case", CASES)
+def test_hotline_step_in_the_order_of_fig8_matches_a_brute_force_loop(case):
+    """The default order (deferred=False) on random mini-batches and hot sets: pooled vectors and final rows equal
+    a loop that runs O's forward and update before X's forward and update.  The hot sets are dense enough that X
+    reads rows O has just updated, so the other order gives other pooled vectors (checked)."""
+    rng = np.random.default_rng(67)
+    tr, B, S = case["table_rows"], case["B"], case["S"]
+    N, T, D = sum(tr), len(tr), 3
+    differs = 0
+    for trial in range(12):
+        ind, off = random_batch(rng, tr, B, S, case["max_pool"])
+        hot = np.asarray([g for g in range(N) if rng.random() < 0.75], dtype=np.int64)
+        table0 = gen.table_values(np.arange(N), D, 13 + trial, integer=False)
+        grad_full = gen.grad_values(5, trial, 2, T * B * S, D, integer=False)
+        lr = 0.25
+        want_pooled, want_rows = brute_step_fig8(table0, ind, off, B, tr, S, hot.tolist(), grad_full, lr)
+
+        remap = orc.build_remap(hot, N)
+        hot_cap = len(hot) + 2
+        perm, n_pop, _, _, _ = orc.fragment(ind, off, B, tr, remap, S)
+
+        def mu(samples):
+            src = ((np.arange(T)[:, None, None] * B + np.asarray(samples, dtype=np.int64)[None, :, None]) * S
+                   + np.arange(S)[None, None, :]).reshape(-1)
+            return grad_full[src], src
+
+        (g_pop, src_pop), (g_non, src_non) = mu(perm[:n_pop]), mu(perm[n_pop:])
+        results = {}
+        for deferred in (False, True):
+            table = table0.copy()
+            cache = np.zeros((hot_cap + N, D), dtype=np.float32)
+            cache[: len(hot)] = orc.load_hot_cache(table0, hot)
+            out = orc.hotline_step(table, cache, hot_cap, remap, ind, off, B, tr, S, g_pop, g_non, lr,
+                                   deferred=deferred)
+            pooled = np.zeros((T * B * S, D), dtype=np.float32)
+            pooled[src_pop], pooled[src_non] = out[5], out[6]
+            final = table.copy()
+            final[hot] = cache[: len(hot)]
+            results[deferred] = (pooled, final)
+        assert np.array_equal(results[False][0].view(np.uint32), want_pooled.view(np.uint32)), trial
+        assert np.array_equal(results[False][1].view(np.uint32), want_rows.view(np.uint32)), trial
+        differs += not np.array_equal(results[True][0], want_pooled)
+    # the two orders are told apart by these inputs (an input of X needs a popular and a non-popular lookup for that)
+    assert differs > 0 or T * S * case["max_pool"] == 1
+
+
 def test_input_record_size_matches_the_papers_buffer_sizing():
     """Section V-A: a 2.5 MB input buffer holds mini-batches of up to 16 K inputs, i.e. 160 bytes per input;
     26 four-byte sparse indices + 13 four-byte dense features + a four-byte label is exactly that, which is
