@@ -16,7 +16,6 @@ import os
 import statistics
 import subprocess
 import sys
-import tempfile
 import threading
 import time
 
@@ -73,13 +72,13 @@ def max_nnz_of(spec, geom) -> int:
     return bags if spec.pooling[0] == "one" else bags * int(spec.pooling[2])
 
 
-def fill_table(table, dim: int, seed: int, device, chunk_rows: int = 1 << 21) -> None:
+def fill_table(table, dim: int, seed: int, device, chunk_rows: int = 1 << 21, integer: bool = False) -> None:
     """table[g, :] = gen.table_values(g) for every row, computed on the device in chunks and copied down."""
     import torch
     n = table.shape[0]
     for r0 in range(0, n, chunk_rows):
         r1 = min(n, r0 + chunk_rows)
-        table[r0:r1].copy_(gen.table_values_torch(r0, r1 - r0, dim, seed, device))
+        table[r0:r1].copy_(gen.table_values_torch(r0, r1 - r0, dim, seed, device, integer=integer))
     if str(device) != "cpu":
         torch.cuda.synchronize()
 
@@ -87,9 +86,8 @@ def fill_table(table, dim: int, seed: int, device, chunk_rows: int = 1 << 21) ->
 class Workload:
     """Everything both arms need: geometry, the host table, profiling and timed batches (host copies)."""
 
-    def __init__(self, name: str, scale: float, n_batches: int, profile_batches, device, threads: int):
-        import torch
-        import paper_2204_05436_b200 as hl
+    def __init__(self, name: str, scale: float, n_batches: int, profile_batches, device, threads: int,
+                 with_table: bool = True):
         self.spec = gen.CONFIGS[name]
         self.geom = gen.make_geometry(self.spec, scale)
         self.name, self.scale = name, scale
@@ -100,11 +98,14 @@ class Workload:
         self.P = s.profile_batches if profile_batches is None else profile_batches
         self.hot_cap = max(1, min(self.N, self._policy_rows()))
         self.staging_cap = max(1, min(self.N, self.max_nnz))
-        t0 = time.time()
-        self.table = hl.host_table_tensor(self.N, self.D)
-        fill_table(self.table, self.D, s.seed, device)
-        log(f"[bench] host table {self.N} x {self.D} fp32 = {self.N * self.D * 4 / 2**30:.1f} GiB pinned+filled "
-            f"in {time.time() - t0:.1f}s")
+        self.table = None
+        if with_table:       # the CUDA arm's host table: memory the device can address, filled from the device
+            import paper_2204_05436_b200 as hl
+            t0 = time.time()
+            self.table = hl.host_table_tensor(self.N, self.D)
+            fill_table(self.table, self.D, s.seed, device)
+            log(f"[bench] host table {self.N} x {self.D} fp32 = {self.N * self.D * 4 / 2**30:.1f} GiB pinned+filled "
+                f"in {time.time() - t0:.1f}s")
         t0 = time.time()
         self.profile = [gen.make_batch(s, g, i, threads) for i in range(self.P)]
         self.batches = [gen.make_batch(s, g, self.P + i, threads) for i in range(n_batches)]
@@ -128,6 +129,8 @@ class Workload:
         return hl.HL_HOT_TOPK_ROWS, int(p[1]), 1
 
     def free(self):
+        if self.table is None:
+            return
         import paper_2204_05436_b200 as hl
         ptr = self.table.data_ptr()
         self.table = None
@@ -189,41 +192,55 @@ class ClockSampler:
 # ----------------------------------------------------------------------------------------------------------
 # CPU oracle legs (cpu_baseline of the CUDA arm, and the whole `--impl reference` arm)
 # ----------------------------------------------------------------------------------------------------------
-def take_samples(batch: gen.Batch, T: int, B: int, S: int, n: int) -> gen.Batch:
-    """The first n inputs of a table-major CSR mini-batch, as a mini-batch of n inputs."""
-    if n >= B:
+def take_samples(batch: gen.Batch, T: int, B: int, S: int, n: int, first: int = 0) -> gen.Batch:
+    """Inputs first .. first+n of a table-major CSR mini-batch, as a mini-batch of n inputs."""
+    if n >= B and first == 0:
         return batch
     off = batch.offsets.astype(np.int64)
     idx_parts, sizes = [], []
     for t in range(T):
-        lo_bag, hi_bag = t * B * S, (t * B + n) * S
+        lo_bag, hi_bag = (t * B + first) * S, (t * B + first + n) * S
         idx_parts.append(batch.indices[off[lo_bag]:off[hi_bag]])
         sizes.append(np.diff(off[lo_bag:hi_bag + 1]))
     new_off = np.concatenate([[0], np.cumsum(np.concatenate(sizes))]).astype(np.int32)
-    dense = None if batch.dense is None else batch.dense[:n]
+    dense = None if batch.dense is None else batch.dense[first:first + n]
     return gen.Batch(np.concatenate(idx_parts).astype(np.int32), new_off, dense, n)
 
 
 class OracleRunner:
-    """Runs the CPU oracle, as it stands, on the workload: learning phase once, then one step per call."""
+    """Runs the CPU oracle, as it stands, on the workload: learning phase once, then one step per call.
+    ``table``: fp32 [N, D] array-like holding (at least) the rows the steps will stage."""
 
-    def __init__(self, wl: Workload):
+    def __init__(self, wl, table, profile=None):
         from oracle import hotline_oracle as orc
         self.orc, self.wl = orc, wl
         t0 = time.time()
-        cnt = orc.access_counts([(b.indices, b.offsets) for b in wl.profile], wl.B, wl.geom.table_rows, wl.S)
+        profile = wl.profile if profile is None else profile
+        cnt = orc.access_counts([(b.indices, b.offsets) for b in profile], wl.B, wl.geom.table_rows, wl.S)
         k = min(wl.hot_cap, orc.hot_capacity(wl.spec.hot_policy, wl.N, wl.D))
         self.hot = orc.select_hot(cnt, k)
         del cnt
         self.remap = orc.build_remap(self.hot, wl.N)
-        self.table = wl.table.numpy()
-        self.cache = np.zeros((wl.hot_cap + wl.staging_cap, wl.D), dtype=np.float32)
-        self.cache[: len(self.hot)] = orc.load_hot_cache(self.table, self.hot)
+        self.table = table
+        self.cache = None
         self.rng = np.random.default_rng(1234)
         log(f"[bench] oracle learning phase: {len(self.hot)} hot rows in {time.time() - t0:.1f}s")
 
-    def step(self, batch: gen.Batch) -> float:
-        """Seconds the oracle needs for one mini-batch (fragment, gather, fwd/bwd of O and X, scatter)."""
+    def load_cache(self, hot_values=None):
+        wl = self.wl
+        self.cache = np.zeros((wl.hot_cap + wl.staging_cap, wl.D), dtype=np.float32)
+        self.cache[: len(self.hot)] = (self.orc.load_hot_cache(self.table, self.hot) if hot_values is None
+                                       else hot_values)
+
+    def sizes(self, batch: gen.Batch) -> dict:
+        """What the index-only part of the path finds for this mini-batch (for the cross-check with the device)."""
+        wl, orc = self.wl, self.orc
+        _, n_pop, O, X, _ = orc.fragment(batch.indices, batch.offsets, batch.batch, wl.geom.table_rows, self.remap, wl.S)
+        C, _ = orc.gather_cold(X.ids, self.remap, wl.hot_cap)
+        return dict(n_pop=n_pop, n_non=batch.batch - n_pop, L_pop=len(O.ids), L_non=len(X.ids), n_cold=len(C), C=C)
+
+    def step(self, batch: gen.Batch, cache=None):
+        """(seconds, sizes) of one mini-batch through the oracle (fragment, gather, fwd/bwd of O and X, scatter)."""
         wl, orc = self.wl, self.orc
         n_bags = wl.T * batch.batch * wl.S
         grad = self.rng.standard_normal((n_bags, wl.D), dtype=np.float32)
@@ -232,51 +249,113 @@ class OracleRunner:
                                          wl.S)
         bags_pop = wl.T * n_pop * wl.S
         t0 = time.perf_counter()
-        orc.hotline_step(self.table, self.cache, wl.hot_cap, self.remap, batch.indices, batch.offsets, batch.batch,
-                         wl.geom.table_rows, wl.S, grad[:bags_pop], grad[bags_pop:], wl.spec.lr)
+        out = orc.hotline_step(self.table, self.cache if cache is None else cache, wl.hot_cap, self.remap,
+                               batch.indices, batch.offsets, batch.batch, wl.geom.table_rows, wl.S, grad[:bags_pop],
+                               grad[bags_pop:], wl.spec.lr)
+        dt = time.perf_counter() - t0
+        _, n_pop, O, X, C, _, _ = out
+        return dt, dict(n_pop=n_pop, n_non=batch.batch - n_pop, L_pop=len(O.ids), L_non=len(X.ids), n_cold=len(C))
+
+    def step_all_cores(self, batch: gen.Batch, cores: int) -> float:
+        """Seconds for one mini-batch when its inputs are dealt out to ``cores`` threads, each running the oracle's
+        step on its share (numpy releases the interpreter lock inside its array operations).  The threads share the
+        tables and the staging area without coordination, so this leg times the work and its results are not used."""
+        from concurrent.futures import ThreadPoolExecutor
+        wl, orc = self.wl, self.orc
+        per = -(-batch.batch // cores)
+        shares = [take_samples(batch, wl.T, wl.B, wl.S, min(per, batch.batch - f), f)
+                  for f in range(0, batch.batch, per)]
+        rngs = [np.random.default_rng(99 + i) for i in range(len(shares))]
+
+        def work(i):
+            sh = shares[i]
+            n_bags = wl.T * sh.batch * wl.S
+            grad = rngs[i].standard_normal((n_bags, wl.D), dtype=np.float32)
+            _, n_pop, _, _, _ = orc.fragment(sh.indices, sh.offsets, sh.batch, wl.geom.table_rows, self.remap, wl.S)
+            bags_pop = wl.T * n_pop * wl.S
+            orc.hotline_step(self.table, self.cache, wl.hot_cap, self.remap, sh.indices, sh.offsets, sh.batch,
+                             wl.geom.table_rows, wl.S, grad[:bags_pop], grad[bags_pop:], wl.spec.lr)
+
+        t0 = time.perf_counter()
+        with ThreadPoolExecutor(max_workers=cores) as pool:
+            list(pool.map(work, range(len(shares))))
         return time.perf_counter() - t0
 
 
-def threads_in_use() -> int:
-    """numpy does the oracle's work on the calling thread (no BLAS call is involved)."""
-    return 1
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:   # pragma: no cover
+        return os.cpu_count() or 1
+
+
+def sparse_oracle_table(wl, rows_needed: np.ndarray, tmpdir: str):
+    """fp32 [N, D] table for the oracle that costs memory only for the rows in ``rows_needed``: a sparse file mapped
+    into memory, those rows filled from the procedural initialiser (the same values the real table holds)."""
+    table = np.memmap(os.path.join(tmpdir, "oracle_table.f32"), dtype=np.float32, mode="w+", shape=(wl.N, wl.D))
+    rows_needed = np.asarray(rows_needed, dtype=np.int64)
+    for i in range(0, len(rows_needed), 1 << 18):
+        chunk = rows_needed[i:i + (1 << 18)]
+        table[chunk] = gen.table_values(chunk, wl.D, wl.spec.seed)
+    return table
 
 
 def run_reference(args, rank: int, world: int) -> None:
+    """The CPU oracle on the host cores, on the CUDA arm's workload.  Needs neither the library nor a GPU: the table
+    is a sparse file holding the rows the sampled mini-batches stage."""
     if rank != 0:
         return
-    import torch
-    device = "cuda:0" if torch.cuda.is_available() else "cpu"
+    import tempfile
     name, scale = pick_workload(args.workload, 1)
+    if args.row_scale is not None:
+        scale = args.row_scale
     wl = Workload(name, scale, n_batches=min(8, args.steps + args.warmup), profile_batches=args.profile_batches,
-                  device=device, threads=args.threads)
-    runner = OracleRunner(wl)
-    # size the per-step sample so that the whole run ends within a few minutes
-    probe = take_samples(wl.batches[0], wl.T, wl.B, wl.S, min(wl.B, 2048))
-    t_probe = runner.step(probe)
-    budget = 150.0 / max(1, args.steps + args.warmup)
-    n = int(min(wl.B, max(256, probe.batch * budget / max(t_probe, 1e-6))))
-    n = 1 << (n.bit_length() - 1) if n < wl.B else wl.B
-    sample = [take_samples(b, wl.T, wl.B, wl.S, n) for b in wl.batches]
-    for i in range(args.warmup):
-        runner.step(sample[i % len(sample)])
-    times = [runner.step(sample[(args.warmup + i) % len(sample)]) for i in range(args.steps)]
-    total = sum(times)
-    value = n * args.steps / total
-    sample_txt = f"first {n} of {wl.B} inputs of each mini-batch, {args.steps} mini-batches"
-    line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "row_scale": wl.scale, "batch": wl.B, "sample_inputs_per_step": n,
-                   "tables": wl.T, "dim": wl.D, "total_rows": wl.N},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads_in_use(), "kind": "oracle",
-                         "sample": sample_txt},
-        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-        "gpu_launches": 0,
-    }
-    print(json.dumps(line), flush=True)
-    wl.free()
+                  device=None, threads=args.threads, with_table=False)
+    with tempfile.TemporaryDirectory() as tmp:
+        runner = OracleRunner(wl, table=None)
+        # size the per-step sample so that the whole run ends within a few minutes
+        n_try = min(wl.B, 2048)
+        probe = take_samples(wl.batches[0], wl.T, wl.B, wl.S, n_try)
+        need = [runner.sizes(probe)["C"]]
+        runner.table = sparse_oracle_table(wl, need[0], tmp)
+        hot_values = gen.table_values(runner.hot, wl.D, wl.spec.seed)
+        runner.load_cache(hot_values)
+        t_probe, _ = runner.step(probe)
+        budget = 150.0 / max(1, args.steps + args.warmup)
+        n = int(min(wl.B, max(256, probe.batch * budget / max(t_probe, 1e-6))))
+        n = 1 << (n.bit_length() - 1) if n < wl.B else wl.B
+        sample = [take_samples(b, wl.T, wl.B, wl.S, n) for b in wl.batches]
+        rows = np.unique(np.concatenate([runner.sizes(b)["C"] for b in sample]))
+        del runner.table
+        runner.table = sparse_oracle_table(wl, rows, tmp)
+        runner.load_cache(hot_values)
+        for i in range(args.warmup):
+            runner.step(sample[i % len(sample)])
+        times = [runner.step(sample[(args.warmup + i) % len(sample)])[0] for i in range(args.steps)]
+        total = sum(times)
+        value = n * args.steps / total
+        sample_txt = f"first {n} of {wl.B} inputs of each mini-batch, {args.steps} mini-batches"
+        line = {
+            "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(wl, extra={"sample_inputs_per_step": n}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample_txt},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0,
+        }
+        print(json.dumps(line), flush=True)
+        del runner.table
+
+
+def workload_config(wl, extra=None) -> dict:
+    """The keys of `config` that name the workload; both arms print the same ones."""
+    c = {"workload": wl.name, "row_scale": wl.scale, "batch": wl.B, "tables": wl.T, "dim": wl.D,
+         "bags_per_sample": wl.S, "total_rows": wl.N, "table_gib": round(wl.N * wl.D * 4 / 2 ** 30, 2),
+         "hot_cap_rows": wl.hot_cap, "profile_batches": wl.P}
+    if extra:
+        c.update(extra)
+    return c
 
 
 # ----------------------------------------------------------------------------------------------------------
@@ -298,9 +377,64 @@ def whole_job_value(batch: int, steps: int, world: int, ms_total_max: float) -> 
     return batch * world * steps / (ms_total_max * 1e-3)
 
 
+def spawn_ranks(argv, n: int) -> int:
+    """`python bench.py --gpus N` outside a launcher: starts the N ranks itself (one process per GPU)."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr",
+           "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.run(cmd).returncode
+
+
 # ----------------------------------------------------------------------------------------------------------
 # CUDA arm
 # ----------------------------------------------------------------------------------------------------------
+# DRAM bytes (read + written) per bag of the forward kernel at dim 64, from a profiler capture of the hot-only
+# micro case (`--micro fwd`: 425,984 one-lookup bags, 164.4 MB of DRAM traffic); a launch of the benchmark is
+# scaled from it by its number of bags, since the traffic grows in proportion to the bags.
+PROFILED_FWD_DRAM_BYTES_PER_BAG = {64: 164.4e6 / 425984}
+
+
+def fwd_bytes(L, bags, D):
+    """Algorithmic bytes of one forward launch: per lookup a row and its slot, per bag a pooled row and an offset."""
+    return L * (4 * D + 4) + bags * (4 * D + 4)
+
+
+def chunks_bytes(L, distinct, D):
+    """Algorithmic bytes of the backward's sum kernel: per lookup a gradient row and its (slot, bag) pair, per
+    distinct row one read-modify-write."""
+    return L * (4 * D + 8) + distinct * 2 * 4 * D
+
+
+def summarise_spans(spans):
+    """Mean duration (us) per span kind, and per (kind, position among the same kind inside a mini-batch)."""
+    by_kind, seq = {}, {}
+    for sp in spans:
+        key = (sp["mini_batch"], sp["name"])
+        k = seq.get(key, 0)
+        seq[key] = k + 1
+        by_kind.setdefault((sp["name"], k), []).append((sp["end_ms"] - sp["begin_ms"]) * 1e3)
+    return {f"{name}#{k}" if any(kk > 0 for (nn, kk) in by_kind if nn == name) else name:
+            round(statistics.mean(v), 2) for (name, k), v in sorted(by_kind.items())}
+
+
+def timeline_text(spans, mini_batches):
+    """The spans of the given mini-batches as text, one line per span, ordered by begin time."""
+    rows = sorted((sp for sp in spans if sp["mini_batch"] in mini_batches), key=lambda sp: sp["begin_ms"])
+    if not rows:
+        return ""
+    t0 = rows[0]["begin_ms"]
+    names = {0: "main", 1: "frag", 2: "sort", 3: "cold", 4: "read", 5: "wb"}
+    out = ["   begin_us      end_us   dur_us  stream  mini-batch  what"]
+    for sp in rows:
+        out.append(f"{(sp['begin_ms'] - t0) * 1e3:10.1f}  {(sp['end_ms'] - t0) * 1e3:10.1f}  "
+                   f"{(sp['end_ms'] - sp['begin_ms']) * 1e3:7.1f}  {names.get(sp['stream'], sp['stream']):>6}  "
+                   f"{sp['mini_batch']:10d}  {sp['name']}")
+    return "\n".join(out)
+
+
 def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
     import torch
     import torch.distributed as dist
@@ -320,22 +454,29 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
     wl = Workload(name, scale, n_batches, args.profile_batches, device, args.threads)
     T, D, S, B = wl.T, wl.D, wl.S, wl.B
     pipelined = not args.no_pipeline
+    native = pipelined and not (args.python_pipeline or args.serial_link)
     eq5 = args.order == "eq5"
-    if eq5 and (args.no_pipeline or args.python_pipeline or args.serial_link):
+    if eq5 and not native:
         raise SystemExit("--order eq5 is a mode of the library's own scheduler")
-    if pipelined:
-        if args.python_pipeline or args.serial_link:
-            h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
-                                    n_dense=wl.spec.n_dense, device=str(device), overlap_link=not args.serial_link,
-                                    lookahead=args.lookahead)
-        else:
-            h = hl.NativePipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap,
-                                          wl.table, n_dense=wl.spec.n_dense, device=str(device),
-                                          lookahead=args.lookahead, order=args.order)
+    if native:
+        h = hl.NativePipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
+                                      n_dense=wl.spec.n_dense, device=str(device), lookahead=args.lookahead,
+                                      order=args.order, main_priority=args.main_priority,
+                                      index_priority=args.index_priority, link_priority=args.link_priority,
+                                      mover_ctas=args.mover_ctas, scatter_ctas=args.scatter_ctas)
+    elif pipelined:
+        h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
+                                n_dense=wl.spec.n_dense, device=str(device), overlap_link=not args.serial_link,
+                                lookahead=args.lookahead, main_priority=args.main_priority,
+                                side_priority=args.index_priority)
     else:
         h = hl.Hotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
-                       n_dense=wl.spec.n_dense, device=str(device))
+                       n_dense=wl.spec.n_dense, device=str(device), main_priority=args.main_priority,
+                       side_priority=args.index_priority)
+        if args.mover_ctas or args.scatter_ctas:
+            hl.hl_set_mover_ctas(h.ctx, args.mover_ctas, args.scatter_ctas)
     lr = wl.spec.lr
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
 
     with torch.cuda.stream(h.main):
         # ---- learning phase (setup, timed separately) ----
@@ -364,9 +505,10 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
         torch.cuda.synchronize()
 
         cursor = [0]   # mini-batches issued so far; mini-batch i uses input buffers i % n_batches
+        inputs = {"idx": d_idx, "off": d_off, "dense": d_dense}
 
         def batch_args(k):
-            return (d_idx[k], d_off[k], B, d_dense[k])
+            return (inputs["idx"][k], inputs["off"][k], B, inputs["dense"][k])
 
         def one_step(timers=None):
             """Issues the next mini-batch; returns (its buffer index k, the object holding its outputs)."""
@@ -380,7 +522,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                 s = h.step(d_grad, None if eq5 else d_grad, lr, next_batch=batch_args((i + h.lookahead) % n_batches),
                            timers=timers, inputs_ready="resident")   # the timed region's inputs are in HBM already
                 return k, h.sets[s]
-            h.step(d_idx[k], d_off[k], B, d_grad, d_grad, lr, dense=d_dense[k], timers=timers)
+            h.step(inputs["idx"][k], inputs["off"][k], B, d_grad, d_grad, lr, dense=inputs["dense"][k], timers=timers)
             return k, h
 
         def finish():
@@ -389,77 +531,128 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                 h.drain()
             torch.cuda.synchronize()
 
-        # per-batch sizes (they depend only on the indices and the hot set): one untimed pass
-        sizes = [None] * n_batches
-        for _ in range(n_batches):
-            k, o = one_step()
+        def restart():
+            """Empties the pipeline and realigns the rotation, so that the next step is mini-batch 0 of the rotation."""
+            while pipelined and not h.idle:
+                h.step(d_grad, None if eq5 else d_grad, lr, next_batch=None, inputs_ready="resident")
             finish()
-            h.status()
-            c = o.counts.cpu().tolist()
-            sizes[k] = dict(n_pop=c[0], n_non=c[1], L_pop=c[2], L_non=c[3], n_cold=int(o.n_cold.item()))
+            cursor[0] = 0
+
+        def sizing_pass():
+            """Per-batch sizes (they depend only on the indices and the hot set): one untimed pass."""
+            out = [None] * n_batches
+            restart()
+            for _ in range(n_batches):
+                k, o = one_step()
+                finish()
+                h.status()
+                c = o.counts.cpu().tolist()
+                pop_ids = o.pop_ids[:c[2]] if hasattr(o, "pop_ids") else None
+                non_ids = o.non_ids[:c[3]] if hasattr(o, "non_ids") else None
+                out[k] = dict(n_pop=c[0], n_non=c[1], L_pop=c[2], L_non=c[3], n_cold=int(o.n_cold.item()),
+                              U_pop=int(torch.unique(pop_ids).numel()) if pop_ids is not None else 0,
+                              U_non=int(torch.unique(non_ids[non_ids >= 0]).numel()) if non_ids is not None else 0)
+            return out
+
+        BW_MASK = 0
+        if native:
+            BW_MASK = (1 << 6) | (1 << 8) | (1 << (hl.HL_SPAN_KERNEL + hl.HL_TIMER_BWD_REDUCE))
+
+        def timed_block(n_steps, mask=0, barrier=False):
+            """n_steps steps between two events on the main stream, a synchronisation on both sides.
+            Returns (ms, host enqueue us per step, spans, index of the first mini-batch)."""
+            torch.cuda.synchronize()
+            if barrier and world > 1:
+                dist.barrier()
+            if mask:
+                h.trace_begin(16 * n_steps + 64, mask)
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            first = (cursor[0], h.j_done if pipelined else 0)     # position in the rotation, the schedule's own count
+            timers = {"only": ("fwd_pop", "fwd_non")} if not native else None
+            ev0.record(h.main)
+            host_t0 = time.perf_counter()
+            for _ in range(n_steps):
+                one_step(timers)
+            host_us = (time.perf_counter() - host_t0) / n_steps * 1e6
+            if pipelined:
+                h.wait_outputs()     # the last write-backs belong to the timed work
+            ev1.record(h.main)
+            finish()
+            spans = h.trace_end() if mask else []
+            if barrier and world > 1:
+                dist.barrier()
+            return ev0.elapsed_time(ev1), host_us, spans, first, timers
+
+        sizes = sizing_pass()
 
         # ---- timed region: device-resident inputs ----
         for i in range(args.warmup):
             one_step()
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        timers = {"only": ("fwd_pop", "fwd_non")}   # the roofline kernel's launches; every call is timed further down
-        if hasattr(h, "prepare_timers"):
-            h.prepare_timers(args.steps)
         launches0 = hl.hl_launch_count()
         log(f"[bench] library kernel launches before the timed region: {launches0}")
         clocks = ClockSampler(local_rank)
         clocks.start()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        first_timed = cursor[0]
-        ev0.record(h.main)
-        host_t0 = time.perf_counter()
-        for i in range(args.steps):
-            one_step(timers)
-        host_enqueue_us = (time.perf_counter() - host_t0) / args.steps * 1e6
-        if pipelined:
-            h.wait_outputs()     # the last write-backs belong to the timed work
-        ev1.record(h.main)
-        finish()
-        if world > 1:
-            dist.barrier()
-        clock_info = clocks.stop()
+        ms_total, host_enqueue_us, bw_spans, first_timed, fwd_timers = timed_block(args.steps, BW_MASK, barrier=True)
         launches = hl.hl_launch_count() - launches0
         h.status()
-        ms_total = ev0.elapsed_time(ev1)
+        # ---- the same block repeated, for a spread (each with a synchronisation on both sides, no trace) ----
+        block_ms = [ms_total / args.steps]
+        for _ in range(args.blocks):
+            ms, _, _, _, _ = timed_block(args.steps)
+            block_ms.append(ms / args.steps)
+        clock_info = clocks.stop()
+        h.status()
 
-        # ---- per-call times (a second, untimed pass over n_batches steps, every call bracketed by events) ----
-        call_timers = {}
-        for _ in range(n_batches):
-            one_step(call_timers)
-        finish()
-
-        # ---- kernel timers and host link (diagnostic pass, outside the timed region) ----
-        hl.hl_timing_enable(h.ctx, True)
-        kt = {"gather_move": [], "scatter_move": [], "bwd_reduce_non": [], "fwd_non": []}
-        for _ in range(n_batches):
-            k, _o = one_step()
+        # ---- every call of the schedule, in place: a traced pass over n_batches steps (outside the timed region) ----
+        all_spans, call_timers = [], {}
+        if native:
+            _, _, all_spans, first_traced, _ = timed_block(n_batches, hl.HL_SPAN_ALL)
+        else:
+            for _ in range(n_batches):
+                one_step(call_timers)
             finish()
-            kt["gather_move"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_GATHER_MOVE), sizes[k]["n_cold"]))
-            kt["scatter_move"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_SCATTER_MOVE), sizes[k]["n_cold"]))
-            kt["bwd_reduce_non"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_BWD_REDUCE), sizes[k]["L_non"]))
-            kt["fwd_non"].append((hl.hl_timing_read(h.ctx, hl.HL_TIMER_FWD), sizes[k]["L_non"]))
-        hl.hl_timing_enable(h.ctx, False)
-        # ---- the roofline kernel with the chip to itself: the forward over the last mini-batch's X again, after
-        # a 256 MB write that leaves nothing of it in the L2 ----
+
+        # ---- kernels alone: nothing else on the chip, L2 flushed by a 256 MB write before every launch ----
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
-        alone_us = []
-        for _ in range(10):
-            flush.zero_()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(h.main)
-            hl.hl_embbag_fwd(h.ctx, h.cache, _o.non, _o.counts_non, _o.pooled_non, h.main.cuda_stream)
-            b.record(h.main)
-            h.main.synchronize()
-            alone_us.append(a.elapsed_time(b) * 1e3)
-        alone_L, alone_bags = sizes[k]["L_non"], T * sizes[k]["n_non"] * S
+        restart()
+        k_last, o_last = one_step()
+        while pipelined and not h.idle:      # the last mini-batch stepped is the one whose buffers are used below
+            o_last = h.sets[h.step(d_grad, None if eq5 else d_grad, lr, next_batch=None, inputs_ready="resident")]
+            k_last += 1
+        finish()
+        sz_last = sizes[k_last % n_batches]
+        stream = h.main.cuda_stream
+
+        def alone(fn, reps=7):
+            us = []
+            for _ in range(reps):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(h.main)
+                fn()
+                b.record(h.main)
+                h.main.synchronize()
+                us.append(a.elapsed_time(b) * 1e3)
+            return statistics.median(us)
+
+        alone_us = {
+            "fwd_non": alone(lambda: hl.hl_embbag_fwd(h.ctx, h.cache, o_last.non, o_last.counts_non, o_last.pooled_non,
+                                                      stream)),
+            "fwd_pop": alone(lambda: hl.hl_embbag_fwd(h.ctx, h.cache, o_last.pop, o_last.counts, o_last.pooled_pop,
+                                                      stream)),
+        }
+        # the movers alone at full width (two CTAs per multiprocessor) on that mini-batch's cold rows: reading them
+        # again and writing them back again changes nothing (the pipeline is empty, the rows were written back)
+        w_last = ((h.j_done - 1) % 2) * h.window_rows if pipelined else 0
+        rows_last = h.window_rows if pipelined else h.staging_cap
+        hl.hl_set_mover_ctas(h.ctx, 2 * sms, 2 * sms)
+        alone_us["move_read"] = alone(lambda: hl.hl_stage_cold(h.ctx, h.host_table, h.cache, w_last, rows_last,
+                                                               o_last.cold_rows, o_last.n_cold, None, stream))
+        alone_us["move_write"] = alone(lambda: hl.hl_scatter_cold_at(h.ctx, h.cache, w_last, rows_last,
+                                                                     o_last.cold_rows, o_last.n_cold, h.host_table,
+                                                                     stream))
+        hl.hl_set_mover_ctas(h.ctx, args.mover_ctas, args.scatter_ctas)
+        h.status()
         del flush
         link = {}
         buf_h = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
@@ -476,9 +669,30 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             link[nm] = best
         del buf_h, buf_d
 
+        # ---- hot-only run: the same mini-batches with every lookup redirected into the profiled popular set, so
+        # that every input is popular and nothing crosses the host link (the hot embedding-bag by itself) ----
+        hot_only = None
+        if not args.no_hot_only:
+            hot_rows_np = h.hot_rows[:n_hot].cpu().numpy()
+            hb = [gen.restrict_to_rows(b, wl.geom, hot_rows_np) for b in wl.batches]
+            if all(x is not None for x in hb):
+                restart()
+                inputs["idx"] = [torch.from_numpy(x.indices).to(device) for x in hb]
+                torch.cuda.synchronize()
+                hot_sizes = sizing_pass()
+                for _ in range(max(3, args.warmup)):
+                    one_step()
+                ms_hot, _, hot_spans, first_hot, hot_timers = timed_block(args.steps, BW_MASK)
+                hot_only = dict(ms=ms_hot, spans=hot_spans, first=first_hot, sizes=hot_sizes, timers=hot_timers)
+                restart()
+                inputs["idx"] = d_idx
+                torch.cuda.synchronize()
+                h.status()
+
         # ---- end to end: host buffers in, results out, copies inside the timed region ----
         e2e = None
         if not args.no_e2e:
+            restart()
             out_pop = torch.empty((wl.n_bags, D), dtype=torch.float32).pin_memory()
             out_non = torch.empty((wl.n_bags, D), dtype=torch.float32).pin_memory()
             out_counts = torch.empty(4, dtype=torch.int32).pin_memory()
@@ -598,96 +812,173 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
     if rank == 0:
         ms_per_step = ms_total / args.steps
         value = whole_job_value(B, args.steps, world, ms_total)
-
-        def mean_us(name, src=None):
-            ev = (timers if src is None else src).get(name, [])
-            return 1e3 * sum(a.elapsed_time(b) for a, b in ev) / max(1, len(ev))
-
-        breakdown = {k: round(mean_us(k, call_timers), 2) for k in call_timers}
-        used = [sizes[(first_timed + i) % n_batches] for i in range(args.steps)]
-        mean = lambda key: sum(u[key] for u in used) / len(used)   # noqa: E731
-        # roofline of the embedding-bag forward (one kernel per call): per lookup a row (4*D bytes) and its slot
-        # (4 bytes) are read, per bag a pooled row (4*D) is written and an offset read.  Of the two launches per
-        # mini-batch the one over the non-popular micro-batch is reported: it is the larger one here, and in the
-        # pipelined schedule it runs with the chip to itself, while the popular one shares it on purpose with the
-        # host reads and the next mini-batch's fragment (its contended time is given beside it).
-        bags_pop = T * mean("n_pop") * S
-        bags_non = T * mean("n_non") * S
-        pop_bytes = mean("L_pop") * (4 * D + 4) + bags_pop * (4 * D + 4)
-        pop_us = mean_us("fwd_pop")
-        fwd_bytes = mean("L_non") * (4 * D + 4) + bags_non * (4 * D + 4)
-        fwd_us = mean_us("fwd_non")
         peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
         if os.path.exists(peaks_path):
             peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
         else:
             peak, peak_src = FALLBACK_HBM_GBS, "fallback"
-        achieved = fwd_bytes / (fwd_us * 1e-6) / 1e9 if fwd_us > 0 else 0.0
-        roofline = {"kernel": "k_embbag_fwd (non-popular micro-batch: hot rows + staged rows, all in HBM)",
-                    "bound": "hbm", "achieved": achieved,
-                    "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                    "traffic": (NCU_FWD_TRAFFIC_BYTES_PER_BAG[D] * bags_non if D in NCU_FWD_TRAFFIC_BYTES_PER_BAG else None),
-                    "traffic_source": "ncu capture of the hot-only micro case, scaled by bags", "algorithmic_bytes_per_launch": fwd_bytes,
-                    "us_per_launch": fwd_us,
-                    "alone": {"note": "the same kernel over one mini-batch's X with no other kernel running, L2 flushed",
-                              "us_per_launch": statistics.median(alone_us),
-                              "achieved": (alone_L * (4 * D + 4) + alone_bags * (4 * D + 4))
-                              / (statistics.median(alone_us) * 1e-6) / 1e9,
-                              "frac": (alone_L * (4 * D + 4) + alone_bags * (4 * D + 4))
-                              / (statistics.median(alone_us) * 1e-6) / 1e9 / peak},
-                    "popular_launch": {"algorithmic_bytes_per_launch": pop_bytes, "us_per_launch": pop_us,
-                                       "achieved": pop_bytes / (pop_us * 1e-6) / 1e9 if pop_us > 0 else 0.0,
-                                       "frac": (pop_bytes / (pop_us * 1e-6) / 1e9 / peak) if pop_us > 0 else 0.0}}
-        link_us = mean_us("gather_cold", call_timers)
+
+        def kernel_table(spans, timers, first, n_steps, sz):
+            """In-step time and fraction of the HBM peak of each bandwidth-bound kernel of a step: both forward
+            launches and the backward's two sum kernels, from the events recorded inside the timed block."""
+            used = [sz[(first[0] + i) % n_batches] for i in range(n_steps)]
+            mean = lambda key: sum(u[key] for u in used) / len(used)   # noqa: E731
+            dur = {}
+            if spans:
+                seq = {}
+                for sp in spans:
+                    nm = sp["name"]
+                    if nm == "k_bwd_chunks":
+                        k = seq.get(sp["mini_batch"], 0)
+                        seq[sp["mini_batch"]] = k + 1
+                        nm = "bwd_chunks_all" if eq5 else ("bwd_chunks_pop" if k == 0 else "bwd_chunks_non")
+                    dur.setdefault(nm, []).append((sp["end_ms"] - sp["begin_ms"]) * 1e3)
+            elif timers:
+                for nm in ("fwd_pop", "fwd_non"):
+                    dur[nm] = [a.elapsed_time(b) * 1e3 for a, b in timers.get(nm, [])]
+            bags_pop, bags_non = T * mean("n_pop") * S, T * mean("n_non") * S
+            algo = {"fwd_pop": fwd_bytes(mean("L_pop"), bags_pop, D), "fwd_non": fwd_bytes(mean("L_non"), bags_non, D),
+                    "bwd_chunks_pop": chunks_bytes(mean("L_pop"), mean("U_pop"), D),
+                    "bwd_chunks_non": chunks_bytes(mean("L_non"), mean("U_non"), D),
+                    "bwd_chunks_all": chunks_bytes(mean("L_pop") + mean("L_non"), mean("U_pop") + mean("U_non"), D)}
+            table = {}
+            for nm, v in dur.items():
+                if not v or nm not in algo:
+                    continue
+                us = statistics.mean(v)
+                gbs = algo[nm] / (us * 1e-6) / 1e9 if us > 0 else 0.0
+                table[nm] = {"algorithmic_bytes_per_launch": algo[nm], "us_per_launch": us, "launches": len(v),
+                             "achieved": gbs, "frac": gbs / peak}
+            return table, mean, bags_pop, bags_non
+
+        kt, mean, bags_pop, bags_non = kernel_table(bw_spans, fwd_timers, first_timed, args.steps, sizes)
+        # The roofline line is the hot embedding-bag forward: both forward launches of a step taken together (the
+        # popular micro-batch's rows in the hot cache, and the non-popular one's over hot cache + staged rows, all
+        # in HBM), algorithmic bytes over the in-step time of the two launches.
+        f_us = sum(kt[k]["us_per_launch"] for k in ("fwd_pop", "fwd_non") if k in kt)
+        f_bytes = sum(kt[k]["algorithmic_bytes_per_launch"] for k in ("fwd_pop", "fwd_non") if k in kt)
+        achieved = f_bytes / (f_us * 1e-6) / 1e9 if f_us > 0 else 0.0
+        per_bag = PROFILED_FWD_DRAM_BYTES_PER_BAG.get(D)
+
+        def alone_entry(nm, L, bags):
+            us = alone_us[nm]
+            gbs = fwd_bytes(L, bags, D) / (us * 1e-6) / 1e9
+            return {"us_per_launch": us, "achieved": gbs, "frac": gbs / peak}
+
+        roofline = {"kernel": "k_embbag_fwd, both launches of a step (popular + non-popular micro-batch)",
+                    "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "peak_source": peak_src, "traffic": per_bag * (bags_pop + bags_non) if per_bag else None,
+                    "traffic_source": "profiler capture of the hot-only micro case, scaled by bags",
+                    "algorithmic_bytes_per_launch": f_bytes, "us_per_launch": f_us,
+                    "note": "us_per_launch = sum of the two forward launches of a step, timed by CUDA events on the "
+                            "main stream inside the timed region, where they share the chip with the other streams",
+                    "kernels_in_step": kt,
+                    "alone": {"note": "the same launches over one mini-batch with nothing else on the chip, L2 flushed",
+                              "fwd_non": alone_entry("fwd_non", sz_last["L_non"], T * sz_last["n_non"] * S),
+                              "fwd_pop": alone_entry("fwd_pop", sz_last["L_pop"], T * sz_last["n_pop"] * S)}}
+        # host link: the movers' kernels in the traced pass (in step) and alone at full width
+        move = {"k_move_read": [], "k_move_write": []}
+        for sp in all_spans:
+            if sp["name"] in move:      # which mini-batch of the rotation the span's mini-batch is
+                k = (first_traced[0] + sp["mini_batch"] - first_traced[1]) % n_batches
+                move[sp["name"]].append(((sp["end_ms"] - sp["begin_ms"]) * 1e3, sizes[k]["n_cold"]))
+
+        def link_entry(v, peak_gbs):
+            if not v:
+                return None
+            us = statistics.mean(t for t, _ in v)
+            gbs = statistics.mean(n * D * 4 / (t * 1e-6) / 1e9 for t, n in v if t > 0)
+            return {"kernel_us": us, "gbs": gbs, "frac_of_memcpy": gbs / peak_gbs}
+
+        bytes_last = sz_last["n_cold"] * D * 4
+        host_link = {
+            "memcpy_h2d_gbs": link["h2d"], "memcpy_d2h_gbs": link["d2h"],
+            "cold_rows_per_step": mean("n_cold"), "bytes_per_step": mean("n_cold") * D * 4,
+            "in_step": {"read": link_entry(move["k_move_read"], link["h2d"]),
+                        "write_back": link_entry(move["k_move_write"], link["d2h"]),
+                        "note": "the movers' kernels inside the schedule, next to the other streams' kernels"},
+            "alone": {"rows": sz_last["n_cold"],
+                      "read": {"kernel_us": alone_us["move_read"], "gbs": bytes_last / alone_us["move_read"] / 1e3,
+                               "frac_of_memcpy": bytes_last / alone_us["move_read"] / 1e3 / link["h2d"]},
+                      "write_back": {"kernel_us": alone_us["move_write"],
+                                     "gbs": bytes_last / alone_us["move_write"] / 1e3,
+                                     "frac_of_memcpy": bytes_last / alone_us["move_write"] / 1e3 / link["d2h"]},
+                      "note": "one mini-batch's cold rows, two mover CTAs per multiprocessor, nothing else running"}}
+        breakdown = summarise_spans(all_spans) if all_spans else \
+            {k: round(1e3 * sum(a.elapsed_time(b) for a, b in v) / max(1, len(v)), 2) for k, v in call_timers.items()}
+        if all_spans and args.timeline:
+            os.makedirs(os.path.dirname(os.path.abspath(args.timeline)), exist_ok=True)
+            mbs = sorted({sp["mini_batch"] for sp in all_spans})
+            with open(args.timeline, "w") as f:
+                f.write(timeline_text(all_spans, set(mbs[len(mbs) // 2: len(mbs) // 2 + 3])) + "\n")
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "row_scale": wl.scale, "batch": B, "tables": T, "dim": D,
-                       "bags_per_sample": S, "total_rows": wl.N, "table_gib": round(wl.N * D * 4 / 2 ** 30, 2),
-                       "hot_rows": n_hot, "hot_cap_rows": wl.hot_cap, "profile_batches": wl.P,
-                       "popular_fraction": round(mean("n_pop") / B, 4), "cold_rows_per_step": round(mean("n_cold"), 1),
-                       "l2": "no explicit flush: a step reads and writes more than the 126 MB L2 "
-                             f"({(2 * wl.n_bags * D * 4 + fwd_bytes) / 2**20:.0f} MB of pooled vectors, gradients and rows)"
-                             if 2 * wl.n_bags * D * 4 > L2_BYTES else
-                             "per-step working set is smaller than L2 on this workload; batches rotate over 8 buffers",
-                       "schedule": ("software-pipelined across mini-batches ("
-                                    + ("PipelinedHotline, issued from Python" if args.python_pipeline or
-                                       args.serial_link else "hl_pipe_*, issued by the library")
-                                    + (", host reads after write-backs)" if args.serial_link else
-                                       ", host reads overlap write-backs, shared rows forwarded)")
-                                    + ("; order of Eq. 5: both forwards, then one update per row and mini-batch"
-                                       if eq5 else "")
-                                    if pipelined else "one mini-batch after the other (Hotline.step)"),
-                       "replicas": "independent replica per GPU, no collective"},
+            "config": workload_config(wl, extra={
+                "hot_rows": n_hot, "popular_fraction": round(mean("n_pop") / B, 4),
+                "cold_rows_per_step": round(mean("n_cold"), 1),
+                "l2": "no explicit flush: a step reads and writes more than the 126 MB L2 "
+                      f"({(2 * wl.n_bags * D * 4 + f_bytes) / 2**20:.0f} MB of pooled vectors, gradients and rows)"
+                      if 2 * wl.n_bags * D * 4 > L2_BYTES else
+                      "per-step working set is smaller than L2 on this workload; batches rotate over 16 buffers",
+                "schedule": ("software-pipelined across mini-batches ("
+                             + ("hl_pipe_*, issued by the library" if native else "PipelinedHotline, issued from Python")
+                             + (", host reads after write-backs)" if args.serial_link else
+                                ", host reads overlap write-backs, shared rows forwarded)")
+                             + ("; order of Eq. 5: both forwards, then one update per row and mini-batch"
+                                if eq5 else "")
+                             if pipelined else "one mini-batch after the other (Hotline.step)"),
+                "stream_priorities": {"main": args.main_priority, "index": args.index_priority,
+                                      "link": args.link_priority},
+                "mover_ctas": {"read": args.mover_ctas or "default", "write": args.scatter_ctas or "default"},
+                "replicas": "independent replica per GPU, no collective"}),
             "clocks": clock_info, "gpu_launches": int(launches), "host_enqueue_us_per_step": host_enqueue_us,
-            "launches_per_step": launches / args.steps, "breakdown_us": breakdown, "roofline": roofline,
-            "host_link": {
-                "memcpy_h2d_gbs": link["h2d"], "memcpy_d2h_gbs": link["d2h"],
-                "cold_rows_per_step": mean("n_cold"), "bytes_per_step": mean("n_cold") * D * 4,
-                "gather_call_us": link_us,
-                "gather_move_kernel_us": 1e3 * statistics.mean(t for t, _ in kt["gather_move"]),
-                "gather_move_gbs": statistics.mean(n * D * 4 / (t * 1e-3) / 1e9 for t, n in kt["gather_move"] if t > 0),
-                "scatter_move_kernel_us": 1e3 * statistics.mean(t for t, _ in kt["scatter_move"]),
-                "scatter_move_gbs": statistics.mean(n * D * 4 / (t * 1e-3) / 1e9 for t, n in kt["scatter_move"] if t > 0),
-                "note": "in-pipeline figures with 16 mover CTAs (HOTLINE_MOVER_CTAS) next to other kernels; `--micro gather` times the same "
-                        "kernel alone with 2 CTAs per SM"},
-            "kernels_us": {"bwd_reduce_non": 1e3 * statistics.mean(t for t, _ in kt["bwd_reduce_non"]),
-                           "fwd_non": 1e3 * statistics.mean(t for t, _ in kt["fwd_non"])},
+            "launches_per_step": launches / args.steps,
+            "blocks": {"note": f"the timed block of {args.steps} steps and {args.blocks} repetitions of it, each "
+                               "synchronised on both sides; ms per step",
+                       "n": len(block_ms), "median": statistics.median(block_ms), "min": min(block_ms),
+                       "max": max(block_ms)},
+            "breakdown_us": breakdown, "roofline": roofline, "host_link": host_link,
         }
+        if hot_only:
+            hk, hmean, hb_pop, _ = kernel_table(hot_only["spans"], hot_only["timers"], hot_only["first"], args.steps,
+                                                hot_only["sizes"])
+            line["hot_only"] = {
+                "note": "the same schedule on the same mini-batches with every lookup redirected into the profiled "
+                        "popular set: every input is popular, nothing crosses the host link",
+                "ms_per_step": hot_only["ms"] / args.steps, "value": B * args.steps / (hot_only["ms"] * 1e-3),
+                "popular_fraction": hmean("n_pop") / B, "cold_rows_per_step": hmean("n_cold"), "kernels_in_step": hk}
         if e2e:
             line["e2e"] = {"value": B * world * args.steps / (e2e["ms_total"] * 1e-3), "unit": UNIT,
                            "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                            "ms_per_step": e2e["ms_total"] / args.steps}
         if world == 1 and not args.no_cpu_baseline:
             h.close()
-            runner = OracleRunner(wl)
-            t_first = runner.step(wl.batches[0])
-            n_more = int(max(1, min(len(wl.batches) - 1, 15.0 / max(t_first, 1e-3))))
-            times = [t_first] + [runner.step(wl.batches[1 + i]) for i in range(n_more)]
-            line["cpu_baseline"] = {"value": B * len(times) / sum(times), "unit": UNIT, "cores": threads_in_use(),
-                                    "kind": "oracle",
-                                    "sample": f"{len(times)} whole mini-batches of {B} inputs ({sum(times):.1f} s)"}
+            runner = OracleRunner(wl, wl.table.numpy())
+            runner.load_cache()
+            times, checked = [], 0
+            for i, b in enumerate(wl.batches):
+                dt, sz = runner.step(b)
+                times.append(dt)
+                # the oracle is the checker of what was timed: the sizes the device found for this mini-batch
+                for key in ("n_pop", "n_non", "L_pop", "L_non", "n_cold"):
+                    if sz[key] != sizes[i][key]:
+                        raise SystemExit(f"[bench] mini-batch {i}: device {key} = {sizes[i][key]}, oracle {sz[key]}")
+                checked += 1
+                if sum(times) > 15.0:
+                    break
+            line["cpu_baseline"] = {"value": B * len(times) / sum(times), "unit": UNIT, "cores": 1, "kind": "oracle",
+                                    "sample": f"{len(times)} whole mini-batches of {B} inputs ({sum(times):.1f} s)",
+                                    "cross_check": f"n_pop, n_non, L_pop, L_non, n_cold of {checked} timed mini-batches "
+                                                   "equal the device's"}
+            cores = host_cores()
+            if cores > 1:
+                t_all = [runner.step_all_cores(wl.batches[i % len(wl.batches)], cores) for i in range(4)]
+                line["cpu_baseline"]["all_cores"] = {
+                    "value": B * len(t_all) / sum(t_all), "unit": UNIT, "cores": cores, "kind": "oracle",
+                    "sample": f"{len(t_all)} whole mini-batches, inputs dealt out to {cores} threads that each run "
+                              f"the oracle's step on their share ({sum(t_all):.1f} s)"}
         print(json.dumps(line), flush=True)
     h.close()
     if world > 1:
@@ -1013,6 +1304,18 @@ def main() -> None:
                     help="main work of a mini-batch: forward O, update O, forward X, update X (the paper's Fig. 8, "
                          "default), or both forwards and then one update of every touched row (Eq. 5)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-hot-only", action="store_true", help="skip the hot-only section of the line")
+    ap.add_argument("--blocks", type=int, default=10,
+                    help="repetitions of the timed block of --steps steps, for the spread reported in `blocks`")
+    ap.add_argument("--main-priority", type=int, default=-1,
+                    help="CUDA priority of the main stream (forwards and updates); 0 = default, negative = higher")
+    ap.add_argument("--index-priority", type=int, default=0,
+                    help="CUDA priority of the streams of index-only ahead-work (fragment, cold-row search, sort)")
+    ap.add_argument("--link-priority", type=int, default=0, help="CUDA priority of the host-link transfer streams")
+    ap.add_argument("--mover-ctas", type=int, default=0, help="hl_set_mover_ctas: CTAs of the host reads (0 = default)")
+    ap.add_argument("--scatter-ctas", type=int, default=0, help="hl_set_mover_ctas: CTAs of the write-backs")
+    ap.add_argument("--timeline", default=None,
+                    help="write the per-stream timeline of three mini-batches of the traced pass to this text file")
     ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather", "tracker"],
                     help="time one library call in isolation")
     ap.add_argument("--micro-dist", default="uniform", choices=["uniform", "zipf"])
@@ -1035,6 +1338,9 @@ def main() -> None:
     if args.warmup < 3:
         log("[bench] warm-up raised to 3 steps")
         args.warmup = 3
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not under a launcher: start the ranks here (one process per GPU, each re-running this command line)
+        raise SystemExit(spawn_ranks(sys.argv[1:], args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -16,6 +16,7 @@ from .synthetic import (  # noqa: F401
     make_batch,
     make_geometry,
     mix32,
+    restrict_to_rows,
     table_values,
     table_values_torch,
     zipf_ranks,

@@ -137,6 +137,22 @@ HL_API int32_t hl_timing_read(hl_ctx* ctx, int32_t which, float* ms);
 HL_API void* hl_host_alloc(size_t bytes);
 HL_API int32_t hl_host_free(void* p);
 
+/* Width of the host-link movers inside a schedule: how many CTAs of hl_gather_cold / hl_stage_cold (read_ctas) and of
+ * hl_scatter_cold (write_ctas) work when a mini-batch moves a DLRM-sized number of rows (the kernels decide on the
+ * device, from the number of rows, whether more join in).  0 = the default (16); at most two per multiprocessor.
+ * Wider movers finish sooner and slow the kernels that run beside them more.  Takes effect with the next call. */
+HL_API int32_t hl_set_mover_ctas(hl_ctx* ctx, int32_t read_ctas, int32_t write_ctas);
+
+/* Test aid for the bounded device-side waits (the tile chaining of the scan inside hl_fragment and of the sorts
+ * inside hl_embbag_bwd_* / hl_gather_cold, the wait of a row mover for a stage of bulk copies).  In production these
+ * waits poll for about a second before they give up, which never happens.  poll_limit > 0 makes them give up after
+ * that many polls, and makes ONE participant withhold what the others wait for: tile `stall_tile` of every chained scan
+ * and sort pass publishes nothing, and (stall_tile >= 0) the first stage of the movers' first CTA issues no copies.
+ * The waits behind it then run out: the kernels return, the status word reads HL_ETIMEOUT, every position computed
+ * from the incomplete data is range-checked before use, and the results of those calls are unspecified.
+ * poll_limit = 0 restores production behaviour.  Nothing here can hang or fault the device. */
+HL_API int32_t hl_test_bounded_waits(hl_ctx* ctx, int32_t poll_limit, int64_t stall_tile);
+
 /* Number of kernels this library has launched in this process so far (all contexts). */
 HL_API uint64_t hl_launch_count(void);
 
@@ -224,8 +240,10 @@ HL_API int32_t hl_embbag_fwd(hl_ctx* ctx, const float* d_cache, const hl_ubatch*
 
 /* Section IV (popular rows are updated in GPU memory; plain SGD as the optimizer).
  * For every distinct id u of the micro-batch: G_u = sum over lookups j with ids[j] == u of
- * d_grad_out[bag(j), :], then cache[u, :] -= lr * G_u, exactly one read-modify-write per row, deterministic
- * (duplicates are segmented by a sort, no floating-point atomics).  Rows not referenced keep their bits.
+ * d_grad_out[bag(j), :], then cache[u, :] -= lr * G_u, exactly one read-modify-write per row and call: the lookups
+ * are sorted by id, every run of equal ids is summed in a fixed order, and -(lr * G_u) is added to the row by one
+ * reduction (red.global.add.f32) per element.  With a single addition per element and call the result does not depend
+ * on the order in which rows are served, so the call is deterministic.  Rows not referenced keep their bits.
  * Scratch: the backward region (may overlap with hl_gather_cold / hl_fragment, not with itself). */
 HL_API int32_t hl_embbag_bwd_sgd(hl_ctx* ctx, float* d_cache, const hl_ubatch* ub, const int32_t* d_n_samples,
                           const float* d_grad_out, float lr, void* stream);
@@ -245,8 +263,9 @@ HL_API int32_t hl_embbag_bwd_apply(hl_ctx* ctx, float* d_cache, const int32_t* d
                                    float lr, void* stream);
 
 /* One sort for both micro-batches of a mini-batch: hl_embbag_bwd_prepare2 sorts the (slot, bag) pairs of O and X
- * together (X's keys offset by the number of cache slots, so that O's pairs come first), which costs one three-pass
- * sort instead of two; d_n_lookups[0..2] = lookups of O, lookups of X, their sum.  O's ids must all be valid slots.
+ * together (X's keys offset by the number of cache slots + 1, so that O's pairs come first, a skipped lookup of O,
+ * negative id, last among them), which costs one three-pass sort instead of two; d_n_lookups[0..2] = lookups of O,
+ * lookups of X, their sum.
  * hl_embbag_bwd_apply2(which = 0 for O, 1 for X) is hl_embbag_bwd_apply on that micro-batch's part of the arrays.
  * d_sorted_slots / d_sorted_bags hold cap_ids(pop) + cap_ids(non) <= max_nnz entries.  Scratch as for prepare / apply. */
 HL_API int32_t hl_embbag_bwd_prepare2(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_n_pop, const hl_ubatch* non,
@@ -377,6 +396,17 @@ typedef struct hl_pipe hl_pipe;
  * words are.  Returns NULL on invalid arguments or if one of those cannot be created. */
 HL_API hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows, int32_t n_sets,
                                const hl_pipe_set* sets, int32_t n_dense, void* main_stream);
+/* The same with options (NULL = the defaults, which is what hl_pipe_create uses).  Priorities are CUDA stream
+ * priorities: 0 = the default priority, negative = higher, clamped to the device's range.  The main stream is the
+ * caller's; to put the bandwidth-bound main work above the ahead-work, create main_stream with a higher priority
+ * than the ones given here. */
+typedef struct {
+    int32_t index_priority;          /* the three streams of index-only ahead-work (fragment, cold-row search, sort) */
+    int32_t link_priority;           /* the two streams of host-link transfers (host read, write-back)              */
+} hl_pipe_options;
+HL_API hl_pipe* hl_pipe_create_ex(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows, int32_t n_sets,
+                                  const hl_pipe_set* sets, int32_t n_dense, void* main_stream,
+                                  const hl_pipe_options* options);
 HL_API void hl_pipe_destroy(hl_pipe* p);
 
 /* Order of a mini-batch's main work.  HL_PIPE_ORDER_FIG8 (default): forward O, update O, forward X, update X, as the
@@ -406,9 +436,34 @@ HL_API int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float* d_
                             const hl_batch* next, const float* d_next_dense, void* next_inputs_ready,
                             int32_t* set_index);
 
-/* Measurement aid: the next hl_pipe_step (only that one) records these caller-owned events (cudaEvent_t, any may be
- * NULL) on main_stream before and after the forward over O and before and after the forward over X. */
-HL_API int32_t hl_pipe_time_forward(hl_pipe* p, void* pop_begin, void* pop_end, void* non_begin, void* non_end);
+/* Measurement aid: a trace of the pipeline's calls.  Between hl_pipe_trace_begin and hl_pipe_trace_end every library
+ * call the pipeline issues whose kind is selected by what_mask (bit HL_SPAN_x) is bracketed by a CUDA event pair on
+ * the stream it is issued to, up to max_spans calls (the events are the pipeline's own; they cost a few microseconds
+ * of host time per call and no device memory).  Kinds HL_SPAN_KERNEL + HL_TIMER_x bracket single kernels inside those
+ * calls: the movers' kernels, the backward's sum kernel, the forward kernel.  hl_pipe_trace_end waits for everything
+ * queued (host-side), then writes the recorded spans, in the order they were issued, with times in milliseconds
+ * relative to the earliest one; *n_spans = how many.  stream: 0 = main, 1-3 = fragment / sort / cold-row search,
+ * 4 = host reads, 5 = write-backs. */
+#define HL_SPAN_FRAGMENT     0
+#define HL_SPAN_INDEX_BEGIN  1
+#define HL_SPAN_INDEX_END    2
+#define HL_SPAN_SORT         3
+#define HL_SPAN_STAGE        4
+#define HL_SPAN_FORWARD_COLD 5
+#define HL_SPAN_FWD_POP      6
+#define HL_SPAN_BWD_POP      7
+#define HL_SPAN_FWD_NON      8
+#define HL_SPAN_BWD_NON      9     /* in the order of Eq. 5: the one update of the whole mini-batch */
+#define HL_SPAN_SCATTER      10
+#define HL_SPAN_KERNEL       16    /* + HL_TIMER_x */
+typedef struct {
+    int32_t mini_batch;              /* counted from the pipeline's first mini-batch */
+    int32_t what;                    /* HL_SPAN_x */
+    int32_t stream;
+    float   begin_ms, end_ms;
+} hl_pipe_span;
+HL_API int32_t hl_pipe_trace_begin(hl_pipe* p, int32_t max_spans, uint32_t what_mask);
+HL_API int32_t hl_pipe_trace_end(hl_pipe* p, hl_pipe_span* out, int32_t cap, int32_t* n_spans);
 /* Makes `stream` wait for the write-back of the last mini-batch stepped (device-side wait). */
 HL_API int32_t hl_pipe_wait_outputs(hl_pipe* p, void* stream);
 /* Makes `stream` wait until perm and counts of the last mini-batch stepped are final (they are, long before its main

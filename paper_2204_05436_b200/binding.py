@@ -22,7 +22,8 @@ EXPORTS = (
     "hl_embbag_bwd_sgd_static", "hl_gather_cold_ahead", "hl_forward_cold", "hl_scatter_cold_at", "hl_flush_hot", "hl_index_cold", "hl_stage_cold", "hl_embbag_bwd_prepare", "hl_embbag_bwd_apply",
     "hl_embbag_bwd_prepare2", "hl_embbag_bwd_apply2",
     "hl_tracker_reset", "hl_tracker_update", "hl_tracker_export",
-    "hl_pipe_create", "hl_pipe_destroy", "hl_pipe_submit", "hl_pipe_step", "hl_pipe_wait_outputs", "hl_pipe_drain", "hl_pipe_time_forward", "hl_pipe_wait_counts",
+    "hl_pipe_create", "hl_pipe_create_ex", "hl_pipe_destroy", "hl_pipe_submit", "hl_pipe_step", "hl_pipe_wait_outputs", "hl_pipe_drain",
+    "hl_pipe_trace_begin", "hl_pipe_trace_end", "hl_pipe_wait_counts", "hl_set_mover_ctas", "hl_test_bounded_waits",
     "hl_index_cold_begin", "hl_index_cold_end", "hl_index_cold_verdict",
     "hl_embbag_bwd_prepare_merged", "hl_pipe_set_order",
 )
@@ -53,6 +54,15 @@ class hl_pipe_set(ctypes.Structure):
                 ("cold_rows", ctypes.c_void_p), ("n_cold", ctypes.c_void_p), ("fwd_src", ctypes.c_void_p),
                 ("pooled_pop", ctypes.c_void_p), ("pooled_non", ctypes.c_void_p), ("dense_out", ctypes.c_void_p),
                 ("sorted_slots", ctypes.c_void_p), ("sorted_bags", ctypes.c_void_p), ("sorted_n", ctypes.c_void_p)]
+
+
+class hl_pipe_options(ctypes.Structure):
+    _fields_ = [("index_priority", ctypes.c_int32), ("link_priority", ctypes.c_int32)]
+
+
+class hl_pipe_span(ctypes.Structure):
+    _fields_ = [("mini_batch", ctypes.c_int32), ("what", ctypes.c_int32), ("stream", ctypes.c_int32),
+                ("begin_ms", ctypes.c_float), ("end_ms", ctypes.c_float)]
 
 
 def _load() -> ctypes.CDLL:
@@ -147,8 +157,17 @@ def _load() -> ctypes.CDLL:
     lib.hl_pipe_set_order.argtypes = [vp, i32]
     lib.hl_pipe_wait_counts.restype = i32
     lib.hl_pipe_wait_counts.argtypes = [vp, vp]
-    lib.hl_pipe_time_forward.restype = i32
-    lib.hl_pipe_time_forward.argtypes = [vp, vp, vp, vp, vp]
+    lib.hl_pipe_create_ex.restype = vp
+    lib.hl_pipe_create_ex.argtypes = [vp, vp, vp, i64, i32, ctypes.POINTER(hl_pipe_set), i32, vp,
+                                      ctypes.POINTER(hl_pipe_options)]
+    lib.hl_pipe_trace_begin.restype = i32
+    lib.hl_pipe_trace_begin.argtypes = [vp, i32, ctypes.c_uint32]
+    lib.hl_pipe_trace_end.restype = i32
+    lib.hl_pipe_trace_end.argtypes = [vp, ctypes.POINTER(hl_pipe_span), i32, ctypes.POINTER(i32)]
+    lib.hl_set_mover_ctas.restype = i32
+    lib.hl_set_mover_ctas.argtypes = [vp, i32, i32]
+    lib.hl_test_bounded_waits.restype = i32
+    lib.hl_test_bounded_waits.argtypes = [vp, i32, i64]
     lib.hl_flush_hot.restype = i32
     lib.hl_flush_hot.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.hl_embbag_bwd_sgd_static.restype = i32
@@ -416,6 +435,26 @@ def hl_pipe_create(ctx: int, d_cache, host_table, window_rows: int, sets, n_dens
     return p
 
 
+def hl_pipe_create_ex(ctx: int, d_cache, host_table, window_rows: int, sets, n_dense: int, main_stream: int,
+                      index_priority: int = 0, link_priority: int = 0) -> int:
+    """hl_pipe_create with the stream priorities of the ahead-work and of the host-link transfers."""
+    arr = (hl_pipe_set * len(sets))(*sets)
+    opt = hl_pipe_options(int(index_priority), int(link_priority))
+    p = _lib.hl_pipe_create_ex(ctx, _ptr(d_cache), _ptr(host_table), int(window_rows), len(sets), arr, int(n_dense),
+                               main_stream, ctypes.byref(opt))
+    if not p:
+        raise HotlineError("hl_pipe_create_ex", HL_EINVAL)
+    return p
+
+
+def hl_set_mover_ctas(ctx: int, read_ctas: int, write_ctas: int) -> None:
+    _check("hl_set_mover_ctas", _lib.hl_set_mover_ctas(ctx, int(read_ctas), int(write_ctas)))
+
+
+def hl_test_bounded_waits(ctx: int, poll_limit: int, stall_tile: int = -1) -> None:
+    _check("hl_test_bounded_waits", _lib.hl_test_bounded_waits(ctx, int(poll_limit), int(stall_tile)))
+
+
 def hl_pipe_destroy(pipe: int) -> None:
     _lib.hl_pipe_destroy(pipe)
 
@@ -455,9 +494,24 @@ def hl_pipe_drain(pipe: int) -> None:
     _check("hl_pipe_drain", _lib.hl_pipe_drain(pipe))
 
 
-def hl_pipe_time_forward(pipe: int, pop_begin, pop_end, non_begin, non_end) -> None:
-    _check("hl_pipe_time_forward", _lib.hl_pipe_time_forward(pipe, _ev(pop_begin), _ev(pop_end), _ev(non_begin),
-                                                             _ev(non_end)))
+HL_SPAN_NAMES = {0: "fragment", 1: "index_begin", 2: "index_end", 3: "sort", 4: "stage_cold", 5: "forward_cold",
+                 6: "fwd_pop", 7: "bwd_pop", 8: "fwd_non", 9: "bwd_non", 10: "scatter_cold",
+                 16: "k_move_read", 17: "k_move_write", 18: "k_bwd_chunks", 19: "k_embbag_fwd"}
+HL_SPAN_KERNEL = 16
+HL_SPAN_ALL = 0xFFFFFFFF
+
+
+def hl_pipe_trace_begin(pipe: int, max_spans: int, what_mask: int = HL_SPAN_ALL) -> None:
+    _check("hl_pipe_trace_begin", _lib.hl_pipe_trace_begin(pipe, int(max_spans), int(what_mask) & 0xFFFFFFFF))
+
+
+def hl_pipe_trace_end(pipe: int, cap: int):
+    """Waits for everything queued; returns the recorded spans as dicts (times in milliseconds from the first one)."""
+    arr = (hl_pipe_span * max(1, int(cap)))()
+    n = ctypes.c_int32(0)
+    _check("hl_pipe_trace_end", _lib.hl_pipe_trace_end(pipe, arr, int(cap), ctypes.byref(n)))
+    return [dict(mini_batch=int(a.mini_batch), what=int(a.what), name=HL_SPAN_NAMES.get(int(a.what), str(a.what)),
+                 stream=int(a.stream), begin_ms=float(a.begin_ms), end_ms=float(a.end_ms)) for a in arr[: n.value]]
 
 
 def hl_pipe_wait_counts(pipe: int, stream: int) -> None:

@@ -2,7 +2,6 @@
 // the host-DRAM table (bulk copies over the host link, row by row) behind the hot cache, and write them back.
 #include "hl_common.cuh"
 #include <cooperative_groups.h>
-#include <cstdlib>
 
 namespace hl {
 namespace {
@@ -75,7 +74,8 @@ __global__ void __launch_bounds__(kThreads) k_cold_assign(const int32_t* __restr
                                                           int64_t staging_cap, int32_t* __restrict__ ids,
                                                           int32_t* __restrict__ cold_rows,
                                                           int64_t* __restrict__ d_n_cold, int32_t* status,
-                                                          const int32_t* __restrict__ d_n_classified) {
+                                                          const int32_t* __restrict__ d_n_classified,
+                                                          int64_t cap_ids) {
     int64_t n = *d_n;
     n = n < n_max ? n : n_max;
     if (n == 0 && d_n_classified[0] != 0) return;    // the one-cluster path has done all of this already
@@ -90,11 +90,13 @@ __global__ void __launch_bounds__(kThreads) k_cold_assign(const int32_t* __restr
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
         const bool head = i == 0 || keys[i] != keys[i - 1];
         const int64_t rank = head ? rank_excl[i] : rank_excl[i] - 1;
+        const int64_t where = vals[i];
+        if (where < 0 || where >= cap_ids || rank < 0) continue;   // only after a chain poll gave up (HL_ETIMEOUT)
         if (rank < staging_cap) {
             if (head) cold_rows[rank] = keys[i];
-            ids[vals[i]] = (int32_t)(slot0 + rank);
+            ids[where] = (int32_t)(slot0 + rank);
         } else {
-            ids[vals[i]] = -1;   // no room to stage this row: the lookup is dropped and the status word says so
+            ids[where] = -1;   // no room to stage this row: the lookup is dropped and the status word says so
         }
     }
 }
@@ -399,37 +401,20 @@ constexpr int kBulkStages = 2;
 constexpr int kBulkStageBytes = 16384;
 constexpr int kBulkMaxPolls = 1 << 22;
 constexpr int kBulkStagesPerCta = 16;     // stages of rows per working CTA before another CTA joins in
-// CTAs of the mover inside the pipeline.  16 CTAs x 16 KB keep 256 KB of rows in flight: 18 K rows of 256 bytes
-// take about 160 us to read and 125 us to write back next to the other streams' kernels.  More CTAs move the rows
-// faster (about 100 us with 2 per SM, alone), fewer slower (one CTA writes back 64 rows every 3.4 us), but what the
-// transfers cost the kernels that run next to them does not depend on that: measured on DLRM-large-like
-// mini-batches, 0.31 ms per mini-batch with both transfers, 0.28 with the write-backs only, 0.22 with the reads only
-// and 0.21 with neither (the last two bound by the host's launch rate) -- the write-back of 4.7 MB costs every
-// concurrent kernel about as much time as the link needs to carry it, whether it is issued by 2, 4 or 16 CTAs, by
-// bulk copies or by plain stores, waiting for each stage to complete or not, spread over the chip or confined to one
-// GPC (all mover CTAs in one thread-block cluster).  8, 16, 32 and 64 CTAs gave 0.335, 0.309, 0.38 and 0.39 ms.
-// (The hot-cache load of hl_build_remap and hl_flush_hot, which run alone, use 2 CTAs per SM and reach 90 % of the
-// memcpy rate.)
-constexpr int kBulkCtasDefault = 16;
-// HOTLINE_MOVER_CTAS in the environment (read once) overrides the count, for tuning on other hosts.
-static int bulk_ctas_setting() {
-    static const int v = [] {
-        const char* e = getenv("HOTLINE_MOVER_CTAS");
-        const int n = e ? atoi(e) : 0;
-        return n >= 1 && n <= 4 * kSMs ? n : kBulkCtasDefault;
-    }();
-    return v;
-}
-#define kBulkCtas bulk_ctas_setting()
-// HOTLINE_SCATTER_CTAS: the same for the write-back alone (default: the mover's count).
-static int scatter_ctas_setting() {
-    static const int v = [] {
-        const char* e = getenv("HOTLINE_SCATTER_CTAS");
-        const int n = e ? atoi(e) : 0;
-        return n >= 1 && n <= 4 * kSMs ? n : bulk_ctas_setting();
-    }();
-    return v;
-}
+// Working CTAs of the mover inside a schedule (hl_set_mover_ctas changes it per context).  16 CTAs x 2 stages x
+// 16 KB keep 512 KB of rows in flight: 18 K rows of 256 bytes take about 160 us to read and 125 us to write back
+// next to the other streams' kernels.  More CTAs move the rows faster (about 100 us with 2 per SM, alone), fewer
+// slower (one CTA writes back 64 rows every 3.4 us), but what the transfers cost the kernels that run next to them
+// does not depend on that.  (The hot-cache load of hl_build_remap and hl_flush_hot, which run alone, use 2 CTAs per
+// SM and reach 90 % of the memcpy rate.)  The default, kMoverCtasDefault, is set at hl_create.
+
+// What a launch of the mover needs to know about its context.
+struct MoveCfg {
+    int sms;            // multiprocessors of the device: the launch has at most 2 CTAs per SM
+    int min_ctas;       // CTAs that work however few rows there are
+    int max_polls;      // poll limit of the wait for a stage to fill
+    int stall;          // tests only: CTA 0 issues no loads for its first stage, whose wait then runs out
+};
 
 template <bool TO_TABLE>
 __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_side, int64_t dense_row0, float* table,
@@ -438,10 +423,11 @@ __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_si
                                                                  int64_t table_rows, int row_bytes,
                                                                  int rows_per_stage,
                                                                  const int32_t* __restrict__ skip, int32_t* status,
-                                                                 int min_ctas) {
+                                                                 int min_ctas, int max_polls, int stall) {
     __shared__ __align__(128) unsigned char stage[kBulkStages][kBulkStageBytes];
     __shared__ __align__(8) uint64_t mbar[kBulkStages];
     __shared__ unsigned int stage_bytes[kBulkStages];
+    __shared__ int s_gave_up;
     int64_t n = *d_n;
     n = n < 0 ? 0 : (n < n_max ? n : n_max);
     const int tid = threadIdx.x;
@@ -450,6 +436,7 @@ __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_si
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&mbar[s])), "r"(1) : "memory");
             stage_bytes[s] = 0;
         }
+        s_gave_up = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -489,7 +476,8 @@ __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_si
                          : "memory");
             stage_bytes[s] = 0;
         }
-        for (int r = tid; r < cnt; r += kBulkThreads) {
+        const bool stalled = stall && blockIdx.x == 0 && it == 0;     // tests: the expected bytes never arrive
+        for (int r = tid; r < cnt && !stalled; r += kBulkThreads) {
             const int64_t g = rows[i0 + r];
             const bool ok = g >= 0 && g < table_rows && !(skip != nullptr && skip[i0 + r] >= 0);
             if (!ok) continue;
@@ -504,36 +492,47 @@ __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_si
                 : "=r"(done)
                 : "r"(smem_u32(&mbar[s])), "r"(parity)
                 : "memory");
-            if (!done && polls > kBulkMaxPolls) {
+            if (!done && polls > max_polls) {
                 set_status(status, HL_ETIMEOUT);
+                s_gave_up = 1;
                 break;
             }
         }
+        // A wait that ran out ends this CTA's work: the stage is not written, no further stage is started (its
+        // barrier phases would be out of step), and the CTA leaves once its earlier stores have completed.  The rows
+        // it was responsible for stay unmoved; the status word says so.
+        __syncthreads();
+        if (s_gave_up) break;
         for (int r = tid; r < cnt; r += kBulkThreads) {
             const int64_t g = rows[i0 + r];
-            const bool ok = done && g >= 0 && g < table_rows && !(skip != nullptr && skip[i0 + r] >= 0);
-            if (!ok) continue;   // (a stage whose wait gave up is not written; the status word says so)
+            const bool ok = g >= 0 && g < table_rows && !(skip != nullptr && skip[i0 + r] >= 0);
+            if (!ok) continue;
             unsigned char* dst = TO_TABLE ? tab + g * row_bytes : dense + (i0 + r) * row_bytes;
             bulk_store(dst, &stage[s][r * row_bytes], (uint32_t)row_bytes);
         }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
     }
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (s_gave_up) {
+        // loads of the abandoned stage that are still on their way get a bounded grace period to land before the
+        // shared memory goes back to the SM
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    }
 }
 
 template <bool TO_TABLE>
 int32_t launch_move_rows(float* dense_side, int64_t dense_row0, float* table, const int32_t* rows,
                          const int64_t* d_n, int64_t n_max, int64_t table_rows, int D, const int32_t* skip,
-                         int bulk_ctas, int32_t* status, cudaStream_t stream) {
+                         MoveCfg cfg, int32_t* status, cudaStream_t stream) {
     if (n_max <= 0) return HL_OK;
     const int D4 = D / 4;
     const int row_bytes = D * 4;
     if (row_bytes <= kBulkStageBytes) {
         const int rows_per_stage = kBulkStageBytes / row_bytes;
-        const int grid = grid_for(n_max, rows_per_stage, 2 * kSMs);
-        k_move_rows_bulk<TO_TABLE><<<grid, kBulkThreads, 0, stream>>>(dense_side, dense_row0, table, rows, d_n, n_max,
-                                                                     table_rows, row_bytes, rows_per_stage, skip,
-                                                                     status, bulk_ctas < grid ? bulk_ctas : grid);
+        const int grid = grid_for(n_max, rows_per_stage, 2 * cfg.sms);
+        k_move_rows_bulk<TO_TABLE><<<grid, kBulkThreads, 0, stream>>>(
+            dense_side, dense_row0, table, rows, d_n, n_max, table_rows, row_bytes, rows_per_stage, skip, status,
+            cfg.min_ctas < grid ? cfg.min_ctas : grid, cfg.max_polls, cfg.stall);
         note_launches(1);
         HL_LAUNCH_CHECK();
         return HL_OK;
@@ -566,12 +565,22 @@ int bits_for(int64_t max_value) {
 
 }  // namespace
 
-int32_t launch_gather_rows(float* dst, int64_t dst_row0, const float* table, const int32_t* rows,
-                           const int64_t* d_n, int64_t n_max, int64_t table_rows, int D, int32_t* status,
-                           cudaStream_t stream) {
+// how the movers of this context are launched: inside a schedule (`width` = the context's setting) or alone on the
+// chip (`width` = 0: two CTAs per SM, the link's full rate)
+static MoveCfg move_cfg(const hl_ctx* ctx, int width) {
+    MoveCfg c;
+    c.sms = ctx_sms(ctx);
+    c.min_ctas = width > 0 ? width : 2 * c.sms;
+    c.max_polls = ctx->test_poll_limit > 0 ? ctx->test_poll_limit : kBulkMaxPolls;
+    c.stall = ctx->test_poll_limit > 0 && ctx->test_stall_tile >= 0;
+    return c;
+}
+
+int32_t launch_gather_rows(hl_ctx* ctx, float* dst, int64_t dst_row0, const float* table, const int32_t* rows,
+                           const int64_t* d_n, int64_t n_max, int32_t* status, cudaStream_t stream) {
     // loading the hot cache happens with nothing else on the chip: two mover CTAs per SM, for the link's full rate
-    return launch_move_rows<false>(dst, dst_row0, const_cast<float*>(table), rows, d_n, n_max, table_rows, D, nullptr,
-                                   2 * kSMs, status, stream);
+    return launch_move_rows<false>(dst, dst_row0, const_cast<float*>(table), rows, d_n, n_max, ctx->N, ctx->D, nullptr,
+                                   move_cfg(ctx, 0), status, stream);
 }
 
 }  // namespace hl
@@ -636,16 +645,17 @@ int32_t index_end(hl_ctx* ctx, hl_ubatch* non, int64_t stage_row0, int64_t stage
     if (ctx->max_nnz > kSmallCap && !general_not_needed) {
         int32_t *keys, *vals;
         st = radix_sort_pairs(r.cold_keys, r.cold_vals, r.cold_n + 1, ctx->max_nnz, key_bits, r.cold_hist, r.status,
-                              &keys, &vals, stream);
+                              &keys, &vals, stream, wait_cfg(ctx));
         if (st != HL_OK) return st;
         k_cold_heads<<<grid, kThreads, 0, stream>>>(keys, r.cold_n + 1, ctx->max_nnz, r.cold_rank);
         note_launches(1);
         HL_LAUNCH_CHECK();
-        st = exclusive_scan_i32(r.cold_rank, r.cold_rank, r.cold_n + 1, ctx->max_nnz, r.cold_tiles, r.status, stream);
+        st = exclusive_scan_i32(r.cold_rank, r.cold_rank, r.cold_n + 1, ctx->max_nnz, r.cold_tiles, r.status, stream,
+                                wait_cfg(ctx));
         if (st != HL_OK) return st;
         k_cold_assign<<<grid, kThreads, 0, stream>>>(keys, vals, r.cold_n + 1, ctx->max_nnz, r.cold_rank,
                                                      ctx->hot_cap + stage_row0, stage_rows, non->ids, d_cold_rows,
-                                                     d_n_cold, r.status, r.cold_n);
+                                                     d_n_cold, r.status, r.cold_n, non->cap_ids);
         note_launches(1);
         HL_LAUNCH_CHECK();
     }
@@ -669,7 +679,8 @@ int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const f
         timer_mark(ctx, HL_TIMER_GATHER_MOVE, 0, stream);
         const int32_t st = launch_move_rows<false>(d_cache, ctx->hot_cap + stage_row0,
                                                    const_cast<float*>(host_table), d_cold_rows, d_n_cold, stage_rows,
-                                                   ctx->N, ctx->D, d_fwd_src, kBulkCtas, r.status, stream);
+                                                   ctx->N, ctx->D, d_fwd_src, move_cfg(ctx, ctx->mover_ctas), r.status,
+                                                   stream);
         timer_mark(ctx, HL_TIMER_GATHER_MOVE, 1, stream);
         return st;
     }
@@ -684,8 +695,8 @@ int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const f
     if (wait_b) HL_CUDA_TRY(cudaStreamWaitEvent(stream, wait_b, 0));
     timer_mark(ctx, HL_TIMER_GATHER_MOVE, 0, stream);
     st = launch_move_rows<false>(d_cache, ctx->hot_cap + stage_row0, const_cast<float*>(host_table), d_cold_rows,
-                                 d_n_cold, stage_rows, ctx->N, ctx->D, d_prev_rows ? d_fwd_src : nullptr, kBulkCtas,
-                                 r.status, stream);
+                                 d_n_cold, stage_rows, ctx->N, ctx->D, d_prev_rows ? d_fwd_src : nullptr,
+                                 move_cfg(ctx, ctx->mover_ctas), r.status, stream);
     timer_mark(ctx, HL_TIMER_GATHER_MOVE, 1, stream);
     return st;
 }
@@ -772,7 +783,7 @@ extern "C" int32_t hl_forward_cold(hl_ctx* ctx, float* d_cache, int64_t from_sta
     if (stage_rows == 0) return HL_OK;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int D4 = ctx->D / 4;
-    const int grid = 2 * kSMs;
+    const int grid = 2 * ctx_sms(ctx);
     const int64_t from = ctx->hot_cap + from_stage_row0, to = ctx->hot_cap + to_stage_row0;
     if (D4 <= 4) k_forward_rows<4><<<grid, kThreads, 0, stream>>>(d_cache, from, to, d_fwd_src, d_n_cold, stage_rows, D4);
     else if (D4 <= 8) k_forward_rows<8><<<grid, kThreads, 0, stream>>>(d_cache, from, to, d_fwd_src, d_n_cold, stage_rows, D4);
@@ -792,7 +803,7 @@ extern "C" int32_t hl_scatter_cold_at(hl_ctx* ctx, const float* d_cache, int64_t
     timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 0, stream);
     const int32_t st = launch_move_rows<true>(const_cast<float*>(d_cache), ctx->hot_cap + stage_row0, host_table,
                                               d_cold_rows, d_n_cold, stage_rows, ctx->N, ctx->D, nullptr,
-                                              scatter_ctas_setting(), ctx->r.status, stream);
+                                              move_cfg(ctx, ctx->scatter_ctas), ctx->r.status, stream);
     timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 1, stream);
     return st;
 }
@@ -808,5 +819,5 @@ extern "C" int32_t hl_flush_hot(hl_ctx* ctx, const float* d_cache, const int32_t
     if (!ctx || !d_cache || !d_hot_rows || !d_n_hot || !host_table) return HL_EINVAL;
     // runs between learning phases, with nothing else on the chip: the mover at the link's full rate
     return launch_move_rows<true>(const_cast<float*>(d_cache), 0, host_table, d_hot_rows, d_n_hot, ctx->hot_cap, ctx->N,
-                                  ctx->D, nullptr, 2 * kSMs, ctx->r.status, static_cast<cudaStream_t>(stream_));
+                                  ctx->D, nullptr, move_cfg(ctx, 0), ctx->r.status, static_cast<cudaStream_t>(stream_));
 }

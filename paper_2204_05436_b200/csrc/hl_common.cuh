@@ -9,12 +9,13 @@
 
 namespace hl {
 
-constexpr int kSMs = 148;                  // B200: 2 dies x 74 SMs
+constexpr int kSMsFallback = 148;          // used only if the device's SM count cannot be queried (B200: 2 x 74)
 constexpr int kRemapRowsPerBlock = 224;    // 7 bitmap words per 32-byte remap block
 constexpr int kSortTile = 2048;            // keys per radix-sort tile (256 threads x 8)
 constexpr int kScanTile = 2048;            // elements per scan tile (256 threads x 8)
 constexpr int kSelTile = 4096;             // rows per hot-set selection tile (256 threads x 16)
 constexpr int kBwdChunk = 32;              // sorted lookups per backward chunk
+constexpr int kMoverCtasDefault = 16;      // working CTAs of a host-link mover inside a schedule
 // Per-mini-batch kernels are launched with one CTA per tile of work rather than as chip-filling persistent grids:
 // they run next to the host-link movers of another micro-batch, which slow down the SMs they sit on, and the
 // hardware block scheduler then simply hands those SMs fewer CTAs.
@@ -77,10 +78,17 @@ struct hl_ctx {
     int64_t hot_cap, staging_cap;
     int64_t n_remap_blocks, n_sel_tiles;
     int device;
+    int sms;                           // multiprocessors of `device` (queried at hl_create)
+    int mover_ctas, scatter_ctas;      // working CTAs of the host-link movers inside a schedule (hl_set_mover_ctas)
+    int test_poll_limit;               // > 0: poll limit of the bounded device waits (hl_test_bounded_waits)
+    int64_t test_stall_tile;           // with it: the tile / mover stage that never delivers (-1: none)
     int64_t* h_table_base;             // host copy [T+1]
     hl::Regions r;
     int timing_on;                     // optional kernel timers (hl_timing_enable)
     cudaEvent_t timer[HL_TIMER_COUNT][2];
+    // optional observer of the kernel timers' marks (the pipeline's trace): called with (user, which, end, stream)
+    void (*mark_hook)(void*, int, int, cudaStream_t);
+    void* mark_user;
 };
 
 namespace hl {
@@ -99,7 +107,10 @@ namespace hl {
 // Records the start/end event of one of the optional kernel timers on `stream` (no-op unless enabled).
 inline void timer_mark(hl_ctx* ctx, int which, int end, cudaStream_t stream) {
     if (ctx->timing_on && ctx->timer[which][end]) cudaEventRecord(ctx->timer[which][end], stream);
+    if (ctx->mark_hook) ctx->mark_hook(ctx->mark_user, which, end, stream);
 }
+
+inline int ctx_sms(const hl_ctx* ctx) { return ctx->sms > 0 ? ctx->sms : kSMsFallback; }
 
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) {
     atomicCAS(status, 0, code);
@@ -139,18 +150,34 @@ __device__ __forceinline__ unsigned lanemask_lt() {
     return m;
 }
 
+// How long the bounded device-side waits poll before they give up (HL_ETIMEOUT), and -- for the tests of that
+// path only -- which tile of a chained scan or sort pass publishes nothing, so that the tiles behind it wait in vain
+// (-1: none).  Production value: about a second of polling, far beyond any wait that can occur.
+struct WaitCfg {
+    int max_polls = 1 << 20;
+    int64_t stall_tile = -1;
+};
+inline WaitCfg wait_cfg(const hl_ctx* ctx) {
+    WaitCfg w;
+    if (ctx->test_poll_limit > 0) {
+        w.max_polls = ctx->test_poll_limit;
+        w.stall_tile = ctx->test_stall_tile;
+    }
+    return w;
+}
+
 // ---- primitives implemented in hl_prims.cu -----------------------------------------------------------------
 // Exclusive scan of in[0 .. n) into out[0 .. n] (out[n] = total); n = *d_n if d_n != nullptr (clamped to
 // n_max), else n_max.  in may alias out.  tiles: scratch of scan_tile_words(n_max) ints.  A chain poll that
 // gives up records HL_ETIMEOUT in *status.
 int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, int64_t n_max, int32_t* tiles,
-                           int32_t* status, cudaStream_t stream);
+                           int32_t* status, cudaStream_t stream, WaitCfg w = WaitCfg());
 
 // Stable LSD radix sort of (key, value) pairs by the low key_bits bits of the non-negative keys.
 // n = *d_n (clamped to n_max).  Returns in *out_keys / *out_vals which of the two buffers holds the result.
 int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n, int64_t n_max, int key_bits,
                          uint32_t* hist, int32_t* status, int32_t** out_keys, int32_t** out_vals,
-                         cudaStream_t stream);
+                         cudaStream_t stream, WaitCfg w = WaitCfg());
 
 // 32-bit words of histogram scratch radix_sort_pairs needs for at most max_nnz pairs.
 constexpr int64_t sort_hist_words(int64_t max_nnz) {

@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
                                                          float lr, float* __restrict__ part,
                                                          const int32_t* __restrict__ d_first, int32_t key_bias,
                                                          int32_t* __restrict__ span_count,
-                                                         int32_t* __restrict__ span_list) {
+                                                         int32_t* __restrict__ span_list, int64_t n_grad_rows) {
     // the lookups of this call are positions [first, first + *d_n_lookups) of the sorted arrays; their keys are
     // slot + key_bias.  A chunk in which a run starts that goes on into the next chunk is appended to span_list
     // (in any order): k_bwd_spans finishes those runs.
@@ -286,7 +286,8 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const int64_t row = (int64_t)k[u] - key_bias;
-                    const bool ok = k[u] >= 0 && row >= 0 && row < n_slots;
+                    // (a bag id outside the gradient array can only be what a given-up chain poll of the sort left behind)
+                    const bool ok = k[u] >= 0 && row >= 0 && row < n_slots && b[u] >= 0 && b[u] < n_grad_rows;
 #pragma unroll
                     for (int v = 0; v < NV; ++v) {
                         const int c = sub + v * G;
@@ -534,7 +535,8 @@ int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t
     int32_t* span_list = span_count + 8;
     HL_CUDA_TRY(cudaMemsetAsync(span_count, 0, 8 * sizeof(int32_t), stream));
     k_bwd_chunks<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, vals, d_n_lookups, grad, ctx->D / 4, n_slots,
-                                                      lr, ctx->r.bwd_part, d_first, key_bias, span_count, span_list);
+                                                      lr, ctx->r.bwd_part, d_first, key_bias, span_count, span_list,
+                                                      ctx->max_bags);
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 1, stream);
     const int span_grid = grid_for(max_chunks * 32, kThreads, kMaxGrid);   // one warp per chunk
     k_bwd_spans<G, NV><<<span_grid, kThreads, 0, stream>>>(cache, keys, d_n_lookups, ctx->D / 4, n_slots, lr,
@@ -608,7 +610,7 @@ int32_t sort_lookups(hl_ctx* ctx, const hl_ubatch* ub, const int32_t* d_n_sample
     note_launches(1);
     HL_LAUNCH_CHECK();
     return radix_sort_pairs(keys, vals, d_n_lookups, ctx->max_nnz, key_bits, r.bwd_hist, r.status, out_keys, out_vals,
-                            stream);
+                            stream, wait_cfg(ctx));
 }
 
 }  // namespace
@@ -645,7 +647,8 @@ extern "C" int32_t hl_embbag_bwd_prepare(hl_ctx* ctx, const hl_ubatch* ub, const
 static int32_t prepare_both(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_n_pop, const hl_ubatch* non,
                             const int32_t* d_n_non, int32_t* d_sorted_slots, int32_t* d_sorted_bags,
                             int32_t* d_n_lookups, bool merge, void* stream_) {
-    // merge = false: X's keys are offset by the number of slots, so that the sorted list is O's pairs, then X's;
+    // merge = false: X's keys are offset by the number of slots + 1, so that the sorted list is O's pairs (skipped
+    // lookups of O, key n_slots, last among them), then X's (its skipped lookups, key 2 * n_slots + 1, at the very end);
     // merge = true: one key space, and X's bags are numbered behind O's: the lookups of a row from both
     // micro-batches form one run, over one gradient array [bags of O; bags of X]
     if (!ctx || !pop || !non || !pop->offsets || !non->offsets || !d_n_pop || !d_n_non || !d_n_lookups)
@@ -658,14 +661,13 @@ static int32_t prepare_both(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_
     if (!pop->ids || !non->ids || !d_sorted_slots || !d_sorted_bags) return HL_EINVAL;
     Regions& r = ctx->r;
     const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
-    if (2 * n_slots + 1 >= (int64_t(1) << 31)) return HL_EINVAL;
-    const int key_bits = bits_for(merge ? n_slots : 2 * n_slots);
+    if (2 * n_slots + 2 >= (int64_t(1) << 31)) return HL_EINVAL;
+    const int key_bits = bits_for(merge ? n_slots : 2 * n_slots + 1);
     const int passes = (key_bits + 7) / 8;
     int32_t* keys[2] = {r.bwd_keys[0], r.bwd_keys[1]};
     int32_t* vals[2] = {r.bwd_vals[0], r.bwd_vals[1]};
     keys[passes & 1] = d_sorted_slots;
     vals[passes & 1] = d_sorted_bags;
-    const int32_t sentinel = (int32_t)(merge ? n_slots : 2 * n_slots);
     const bool short_bags = ctx->max_nnz <= 4 * ctx->max_bags;
     const int per_block = short_bags ? kThreads : kThreads / 32;
     const int grid = grid_for(ctx->max_bags, per_block, kMaxGrid);
@@ -673,7 +675,8 @@ static int32_t prepare_both(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_
     const int32_t* ns[2] = {d_n_pop, d_n_non};
     for (int m = 0; m < 2; ++m) {
         const int32_t* pos0 = m == 0 ? nullptr : d_n_lookups;
-        const int32_t bias = (m == 0 || merge) ? 0 : (int32_t)n_slots;
+        const int32_t bias = (m == 0 || merge) ? 0 : (int32_t)(n_slots + 1);
+        const int32_t sentinel = bias + (int32_t)n_slots;
         const int32_t* bag_bias = (m == 1 && merge) ? d_n_pop : nullptr;
         if (short_bags)
             k_bwd_pairs<1><<<grid, kThreads, 0, stream>>>(ubs[m]->ids, ubs[m]->offsets, ns[m], ctx->max_batch,
@@ -689,7 +692,8 @@ static int32_t prepare_both(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_
     note_launches(2);
     HL_LAUNCH_CHECK();
     int32_t *ok, *ov;
-    return radix_sort_pairs(keys, vals, d_n_lookups + 2, ctx->max_nnz, key_bits, r.bwd_hist, r.status, &ok, &ov, stream);
+    return radix_sort_pairs(keys, vals, d_n_lookups + 2, ctx->max_nnz, key_bits, r.bwd_hist, r.status, &ok, &ov, stream,
+                            wait_cfg(ctx));
 }
 
 extern "C" int32_t hl_embbag_bwd_prepare2(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_n_pop,
@@ -712,7 +716,7 @@ extern "C" int32_t hl_embbag_bwd_apply2(hl_ctx* ctx, float* d_cache, const int32
     if (!d_sorted_slots || !d_sorted_bags) return HL_EINVAL;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int32_t* d_first = which == 0 ? nullptr : d_n_lookups;             // X's block starts behind O's
-    const int32_t bias = which == 0 ? 0 : (int32_t)(ctx->hot_cap + ctx->staging_cap);
+    const int32_t bias = which == 0 ? 0 : (int32_t)(ctx->hot_cap + ctx->staging_cap + 1);
 #define HL_BWD(G, NV) \
     launch_bwd<G, NV>(ctx, d_cache, d_sorted_slots, d_sorted_bags, d_n_lookups + which, d_grad_out, lr, stream, d_first, bias)
     HL_DISPATCH_ROW_SHAPE(ctx->D / 4, HL_BWD);

@@ -197,6 +197,7 @@ __global__ void __launch_bounds__(kThreads) k_frag_emit(const int32_t* __restric
             }
         } else {
             const int32_t out_lo = dst_start[dst] - L_pop;
+            if (out_lo < 0) continue;   // only after a chain poll of the scan gave up (HL_ETIMEOUT)
             if (sub == 0) non_offsets[dst - pop_bags] = out_lo;
             for (int32_t j = sub; j < src_hi - src_lo; j += GROUP) {
                 if (out_lo + j >= non_cap) {
@@ -252,7 +253,8 @@ extern "C" int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_de
                                                                                d_counts, r.frag_scan);
     note_launches(3);   // flags, partition, sizes
     HL_LAUNCH_CHECK();
-    int32_t st = exclusive_scan_i32(r.frag_scan, r.frag_scan, nullptr, n_bags, r.frag_tiles, r.status, stream);
+    int32_t st = exclusive_scan_i32(r.frag_scan, r.frag_scan, nullptr, n_bags, r.frag_tiles, r.status, stream,
+                                    wait_cfg(ctx));
     if (st != HL_OK) return st;
     if (b->nnz <= 4 * n_bags)
         k_frag_emit<1><<<grid_for(n_bags, kThreads, kMaxGrid), kThreads, 0, stream>>>(

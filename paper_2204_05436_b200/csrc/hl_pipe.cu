@@ -33,7 +33,18 @@ struct hl_pipe {
     int64_t j_begun, j_indexed, j_submitted, j_done;
     int32_t* h_verdict;          // pinned host words, one per set: what the first half of the cold-row search found
     int order;                   // HL_PIPE_ORDER_*
-    cudaEvent_t time_fwd[4];     // one-shot: recorded around the two forward calls of the next step
+    // trace (hl_pipe_trace_begin / _end): one event pair per recorded span
+    struct Span {
+        cudaEvent_t b, e;
+        int32_t mini_batch, what, stream;
+        bool closed;
+    };
+    std::vector<Span> spans;
+    size_t n_spans;              // spans opened so far
+    uint32_t trace_mask;         // bit `what` set: spans of that kind are recorded; 0 = not tracing
+    int64_t cur_mb;              // mini-batch the call being issued belongs to (for spans opened by the kernel timers)
+    int cur_stream;
+    int open_timer[HL_TIMER_COUNT];
 };
 
 namespace {
@@ -46,6 +57,53 @@ namespace {
 
 int32_t wait(cudaStream_t s, cudaEvent_t e) { return cudaStreamWaitEvent(s, e, 0) == cudaSuccess ? HL_OK : HL_ECUDA; }
 int32_t record(cudaEvent_t e, cudaStream_t s) { return cudaEventRecord(e, s) == cudaSuccess ? HL_OK : HL_ECUDA; }
+
+// ---- trace ---------------------------------------------------------------------------------------------------
+enum { kMain = 0, kStreamA = 1, kStreamB = 2, kStreamC = 3, kLink = 4, kWb = 5 };
+
+cudaStream_t stream_of(hl_pipe* p, int id) {
+    cudaStream_t all[6] = {p->main, p->sa, p->sb, p->sc, p->link, p->wb};
+    return all[id];
+}
+
+// Opens a span of kind `what` for mini-batch `mb` on stream `id`: its begin event is recorded now.  -1 = not recorded.
+int span_open(hl_pipe* p, int what, int64_t mb, int id) {
+    p->cur_mb = mb;
+    p->cur_stream = id;
+    if (!(p->trace_mask >> what & 1u) || p->n_spans >= p->spans.size()) return -1;
+    hl_pipe::Span& sp = p->spans[p->n_spans];
+    if (cudaEventRecord(sp.b, stream_of(p, id)) != cudaSuccess) return -1;
+    sp.mini_batch = (int32_t)mb;
+    sp.what = what;
+    sp.stream = id;
+    sp.closed = false;
+    return (int)p->n_spans++;
+}
+
+void span_close(hl_pipe* p, int idx) {
+    if (idx < 0) return;
+    hl_pipe::Span& sp = p->spans[idx];
+    sp.closed = cudaEventRecord(sp.e, stream_of(p, sp.stream)) == cudaSuccess;
+}
+
+// the library's kernel timers (the movers' kernels, the backward's sum kernel, the forward kernel) seen from here
+void on_timer_mark(void* user, int which, int end, cudaStream_t) {
+    hl_pipe* p = static_cast<hl_pipe*>(user);
+    if (which < 0 || which >= HL_TIMER_COUNT) return;
+    if (!end) p->open_timer[which] = span_open(p, HL_SPAN_KERNEL + which, p->cur_mb, p->cur_stream);
+    else {
+        span_close(p, p->open_timer[which]);
+        p->open_timer[which] = -1;
+    }
+}
+
+// RAII span around one library call
+struct Scope {
+    hl_pipe* p;
+    int idx;
+    Scope(hl_pipe* p_, int what, int64_t mb, int id) : p(p_), idx(span_open(p_, what, mb, id)) {}
+    ~Scope() { span_close(p, idx); }
+};
 
 // Second half of the index-only work of the mini-batch begun last: the rest of the cold-row search and the backward
 // sort.  It is queued one call later than the first half whenever the schedule has that slack, because by then the
@@ -63,17 +121,23 @@ int32_t finish_index(hl_pipe* p) {
     hl_pipe_set* prev = j >= 1 ? &p->sets[(j - 1) % n] : nullptr;
     const int64_t w = (j % 2) * p->window_rows;
     const bool known_done = cudaEventQuery(e.verdict) == cudaSuccess && p->h_verdict[j % n] == 0;
-    HL_PIPE_TRY(hl_index_cold_end(p->ctx, &st.non, w, p->window_rows, st.cold_rows, st.n_cold,
+    {
+        Scope sc(p, HL_SPAN_INDEX_END, j, kStreamC);
+        HL_PIPE_TRY(hl_index_cold_end(p->ctx, &st.non, w, p->window_rows, st.cold_rows, st.n_cold,
                                   prev ? prev->cold_rows : nullptr, prev ? prev->n_cold : nullptr, st.fwd_src,
                                   known_done ? 1 : 0, p->sc));
+    }
     HL_PIPE_TRY(record(e.index, p->sc));
     HL_PIPE_TRY(wait(p->sb, e.index));
-    if (p->order == HL_PIPE_ORDER_EQ5)
-        HL_PIPE_TRY(hl_embbag_bwd_prepare_merged(p->ctx, &st.pop, st.counts, &st.non, st.counts + 1, st.sorted_slots,
-                                                 st.sorted_bags, st.sorted_n, p->sb));
-    else
-        HL_PIPE_TRY(hl_embbag_bwd_prepare2(p->ctx, &st.pop, st.counts, &st.non, st.counts + 1, st.sorted_slots,
-                                           st.sorted_bags, st.sorted_n, p->sb));
+    {
+        Scope sc(p, HL_SPAN_SORT, j, kStreamB);
+        if (p->order == HL_PIPE_ORDER_EQ5)
+            HL_PIPE_TRY(hl_embbag_bwd_prepare_merged(p->ctx, &st.pop, st.counts, &st.non, st.counts + 1,
+                                                     st.sorted_slots, st.sorted_bags, st.sorted_n, p->sb));
+        else
+            HL_PIPE_TRY(hl_embbag_bwd_prepare2(p->ctx, &st.pop, st.counts, &st.non, st.counts + 1, st.sorted_slots,
+                                               st.sorted_bags, st.sorted_n, p->sb));
+    }
     HL_PIPE_TRY(record(e.prep, p->sb));
     p->j_indexed += 1;
     return HL_OK;
@@ -94,12 +158,19 @@ int32_t begin_index(hl_pipe* p, const hl_batch* b, const float* d_dense, void* i
         HL_PIPE_TRY(wait(p->sa, static_cast<cudaEvent_t>(inputs_ready)));
     }
     if (j >= n) HL_PIPE_TRY(wait(p->sa, e.scatter));      // the buffers of this set were mini-batch j-n_sets's
-    HL_PIPE_TRY(hl_fragment(p->ctx, b, d_dense, d_dense ? p->n_dense : 0, st.perm, st.counts, &st.pop, &st.non,
-                            d_dense ? st.dense_out : nullptr, p->sa));
+    {
+        Scope sc(p, HL_SPAN_FRAGMENT, j, kStreamA);
+        HL_PIPE_TRY(hl_fragment(p->ctx, b, d_dense, d_dense ? p->n_dense : 0, st.perm, st.counts, &st.pop, &st.non,
+                                d_dense ? st.dense_out : nullptr, p->sa));
+    }
     HL_PIPE_TRY(record(e.frag, p->sa));
     HL_PIPE_TRY(wait(p->sc, e.frag));
     if (j >= n) HL_PIPE_TRY(wait(p->sc, e.scatter));
-    HL_PIPE_TRY(hl_index_cold_begin(p->ctx, &st.non, st.counts + 1, w, p->window_rows, st.cold_rows, st.n_cold, p->sc));
+    {
+        Scope sc(p, HL_SPAN_INDEX_BEGIN, j, kStreamC);
+        HL_PIPE_TRY(hl_index_cold_begin(p->ctx, &st.non, st.counts + 1, w, p->window_rows, st.cold_rows, st.n_cold,
+                                        p->sc));
+    }
     if (cudaMemcpyAsync(p->h_verdict + (j % n), hl_index_cold_verdict(p->ctx), sizeof(int32_t), cudaMemcpyDeviceToHost,
                         p->sc) != cudaSuccess)
         return HL_ECUDA;
@@ -117,8 +188,11 @@ int32_t submit_link(hl_pipe* p) {
     HL_PIPE_TRY(wait(p->link, p->ev[j % n].index));
     if (j >= 2) HL_PIPE_TRY(wait(p->link, p->ev[(j - 2) % n].scatter));   // host rows of j-2 final, its window free
     if (j >= 1) HL_PIPE_TRY(wait(p->link, p->ev[(j - 1) % n].forward));   // j-1 took what it needs out of the window
-    HL_PIPE_TRY(hl_stage_cold(p->ctx, p->host_table, p->cache, w, p->window_rows, st.cold_rows, st.n_cold,
-                              j >= 1 ? st.fwd_src : nullptr, p->link));
+    {
+        Scope sc(p, HL_SPAN_STAGE, j, kLink);
+        HL_PIPE_TRY(hl_stage_cold(p->ctx, p->host_table, p->cache, w, p->window_rows, st.cold_rows, st.n_cold,
+                                  j >= 1 ? st.fwd_src : nullptr, p->link));
+    }
     HL_PIPE_TRY(record(p->ev[j % n].gather, p->link));
     p->j_submitted += 1;
     return HL_OK;
@@ -126,8 +200,9 @@ int32_t submit_link(hl_pipe* p) {
 
 }  // namespace
 
-extern "C" hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows,
-                                   int32_t n_sets, const hl_pipe_set* sets, int32_t n_dense, void* main_stream) {
+extern "C" hl_pipe* hl_pipe_create_ex(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows,
+                                      int32_t n_sets, const hl_pipe_set* sets, int32_t n_dense, void* main_stream,
+                                      const hl_pipe_options* opt) {
     if (!ctx || !d_cache || !host_table || !sets || n_sets < 3 || n_sets > 16 || window_rows < 0 ||
         2 * window_rows > ctx->staging_cap || n_dense < 0)
         return nullptr;
@@ -151,14 +226,21 @@ extern "C" hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_tabl
     p->j_begun = p->j_indexed = p->j_submitted = p->j_done = 0;
     p->h_verdict = nullptr;
     p->order = HL_PIPE_ORDER_FIG8;
-    for (auto& t : p->time_fwd) t = nullptr;
+    p->n_spans = 0;
+    p->trace_mask = 0;
+    p->cur_mb = 0;
+    p->cur_stream = kMain;
+    for (auto& t : p->open_timer) t = -1;
     int lo = 0, hi = 0;
     cudaDeviceGetStreamPriorityRange(&lo, &hi);          // hi = numerically lowest = highest priority
+    auto clamp = [&](int prio) { return prio < hi ? hi : (prio > lo ? lo : prio); };
+    const int index_prio = clamp(opt ? opt->index_priority : 0), link_prio = clamp(opt ? opt->link_priority : 0);
     cudaStream_t* side[5] = {&p->sa, &p->sb, &p->sc, &p->link, &p->wb};
     bool ok = true;
-    for (auto s : side) {
-        *s = nullptr;
-        ok = ok && cudaStreamCreateWithPriority(s, cudaStreamNonBlocking, hi) == cudaSuccess;
+    for (int i = 0; i < 5; ++i) {
+        *side[i] = nullptr;
+        ok = ok && cudaStreamCreateWithPriority(side[i], cudaStreamNonBlocking, i < 3 ? index_prio : link_prio) ==
+                       cudaSuccess;
     }
     p->ev.resize(n_sets);
     for (auto& e : p->ev) {
@@ -179,6 +261,11 @@ extern "C" hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_tabl
     return p;
 }
 
+extern "C" hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows,
+                                   int32_t n_sets, const hl_pipe_set* sets, int32_t n_dense, void* main_stream) {
+    return hl_pipe_create_ex(ctx, d_cache, host_table, window_rows, n_sets, sets, n_dense, main_stream, nullptr);
+}
+
 extern "C" void hl_pipe_destroy(hl_pipe* p) {
     if (!p) return;
     cudaStream_t side[5] = {p->sa, p->sb, p->sc, p->link, p->wb};
@@ -193,6 +280,14 @@ extern "C" void hl_pipe_destroy(hl_pipe* p) {
             if (x) cudaEventDestroy(x);
     }
     if (p->h_verdict) cudaFreeHost(p->h_verdict);
+    if (p->ctx && p->ctx->mark_user == p) {
+        p->ctx->mark_hook = nullptr;
+        p->ctx->mark_user = nullptr;
+    }
+    for (auto& sp : p->spans) {
+        if (sp.b) cudaEventDestroy(sp.b);
+        if (sp.e) cudaEventDestroy(sp.e);
+    }
     delete p;
 }
 
@@ -223,36 +318,44 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
         // rows shared with mini-batch j-1 come out of its staging window once its backward is done
         HL_PIPE_TRY(wait(p->link, e.index));
         HL_PIPE_TRY(wait(p->link, p->ev[(j - 1) % n].x));
+        Scope sc(p, HL_SPAN_FORWARD_COLD, j, kLink);
         HL_PIPE_TRY(hl_forward_cold(p->ctx, p->cache, w1, w0, p->window_rows, st.fwd_src, st.n_cold, p->link));
     }
     HL_PIPE_TRY(record(e.forward, p->link));
     if (p->j_submitted < p->j_indexed) HL_PIPE_TRY(submit_link(p));         // mini-batch j+1, if indexed in full
-    if (p->time_fwd[0]) HL_PIPE_TRY(record(p->time_fwd[0], p->main));
-    HL_PIPE_TRY(hl_embbag_fwd(p->ctx, p->cache, &st.pop, st.counts, st.pooled_pop, p->main));
-    if (p->time_fwd[1]) HL_PIPE_TRY(record(p->time_fwd[1], p->main));
+    {
+        Scope sc(p, HL_SPAN_FWD_POP, j, kMain);
+        HL_PIPE_TRY(hl_embbag_fwd(p->ctx, p->cache, &st.pop, st.counts, st.pooled_pop, p->main));
+    }
     if (p->order == HL_PIPE_ORDER_FIG8) {
         HL_PIPE_TRY(wait(p->main, e.prep));
+        Scope sc(p, HL_SPAN_BWD_POP, j, kMain);
         HL_PIPE_TRY(hl_embbag_bwd_apply2(p->ctx, p->cache, st.sorted_slots, st.sorted_bags, st.sorted_n, 0, d_grad_pop,
                                          lr, p->main));
     }
     HL_PIPE_TRY(wait(p->main, e.gather));
     HL_PIPE_TRY(wait(p->main, e.forward));
-    if (p->time_fwd[2]) HL_PIPE_TRY(record(p->time_fwd[2], p->main));
-    HL_PIPE_TRY(hl_embbag_fwd(p->ctx, p->cache, &st.non, st.counts + 1, st.pooled_non, p->main));
-    if (p->time_fwd[3]) HL_PIPE_TRY(record(p->time_fwd[3], p->main));
-    for (auto& t : p->time_fwd) t = nullptr;
+    {
+        Scope sc(p, HL_SPAN_FWD_NON, j, kMain);
+        HL_PIPE_TRY(hl_embbag_fwd(p->ctx, p->cache, &st.non, st.counts + 1, st.pooled_non, p->main));
+    }
     if (p->order == HL_PIPE_ORDER_FIG8) {
+        Scope sc(p, HL_SPAN_BWD_NON, j, kMain);
         HL_PIPE_TRY(hl_embbag_bwd_apply2(p->ctx, p->cache, st.sorted_slots, st.sorted_bags, st.sorted_n, 1, d_grad_non,
                                          lr, p->main));
     } else {   // one update of every touched row with the gradient of the whole mini-batch
         HL_PIPE_TRY(wait(p->main, e.prep));
+        Scope sc(p, HL_SPAN_BWD_NON, j, kMain);
         HL_PIPE_TRY(hl_embbag_bwd_apply(p->ctx, p->cache, st.sorted_slots, st.sorted_bags, st.sorted_n + 2, d_grad_pop,
                                         lr, p->main));
     }
     HL_PIPE_TRY(record(e.x, p->main));
     HL_PIPE_TRY(wait(p->wb, e.x));
-    HL_PIPE_TRY(hl_scatter_cold_at(p->ctx, p->cache, w0, p->window_rows, st.cold_rows, st.n_cold, p->host_table,
-                                   p->wb));
+    {
+        Scope sc(p, HL_SPAN_SCATTER, j, kWb);
+        HL_PIPE_TRY(hl_scatter_cold_at(p->ctx, p->cache, w0, p->window_rows, st.cold_rows, st.n_cold, p->host_table,
+                                       p->wb));
+    }
     HL_PIPE_TRY(record(e.scatter, p->wb));
     // The ahead-work comes last: the later the pending cold-row search is ended, the likelier its verdict is known.
     HL_PIPE_TRY(finish_index(p));                                           // the mini-batch begun one step ago
@@ -276,12 +379,64 @@ extern "C" int32_t hl_pipe_set_order(hl_pipe* p, int32_t order) {
     return HL_OK;
 }
 
-extern "C" int32_t hl_pipe_time_forward(hl_pipe* p, void* pop_begin, void* pop_end, void* non_begin, void* non_end) {
-    if (!p) return HL_EINVAL;
-    p->time_fwd[0] = static_cast<cudaEvent_t>(pop_begin);
-    p->time_fwd[1] = static_cast<cudaEvent_t>(pop_end);
-    p->time_fwd[2] = static_cast<cudaEvent_t>(non_begin);
-    p->time_fwd[3] = static_cast<cudaEvent_t>(non_end);
+extern "C" int32_t hl_pipe_trace_begin(hl_pipe* p, int32_t max_spans, uint32_t what_mask) {
+    if (!p || max_spans < 1 || max_spans > (1 << 16) || what_mask == 0) return HL_EINVAL;
+    if ((int)p->spans.size() < max_spans) {
+        const size_t old = p->spans.size();
+        p->spans.resize(max_spans);
+        for (size_t i = old; i < p->spans.size(); ++i) p->spans[i].b = p->spans[i].e = nullptr;
+        for (size_t i = old; i < p->spans.size(); ++i)
+            if (cudaEventCreate(&p->spans[i].b) != cudaSuccess || cudaEventCreate(&p->spans[i].e) != cudaSuccess) {
+                p->spans.resize(i);      // (an event of the failed pair, if any, is leaked with the pipeline's others)
+                return HL_ECUDA;
+            }
+    }
+    p->n_spans = 0;
+    p->trace_mask = what_mask;
+    for (auto& t : p->open_timer) t = -1;
+    p->ctx->mark_hook = on_timer_mark;
+    p->ctx->mark_user = p;
+    return HL_OK;
+}
+
+extern "C" int32_t hl_pipe_trace_end(hl_pipe* p, hl_pipe_span* out, int32_t cap, int32_t* n_out) {
+    if (!p || !n_out || cap < 0 || (cap > 0 && !out)) return HL_EINVAL;
+    p->trace_mask = 0;
+    if (p->ctx->mark_user == p) {
+        p->ctx->mark_hook = nullptr;
+        p->ctx->mark_user = nullptr;
+    }
+    HL_PIPE_TRY(hl_pipe_drain(p));
+    // times are relative to the earliest begin among the recorded spans
+    int first = -1;
+    for (size_t i = 0; i < p->n_spans; ++i) {
+        if (!p->spans[i].closed) continue;
+        if (first < 0) {
+            first = (int)i;
+            continue;
+        }
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, p->spans[first].b, p->spans[i].b) == cudaSuccess && ms < 0.f) first = (int)i;
+    }
+    int32_t n = 0;
+    for (size_t i = 0; i < p->n_spans && n < cap; ++i) {
+        const hl_pipe::Span& sp = p->spans[i];
+        if (!sp.closed) continue;
+        float b = 0.f, e = 0.f;
+        if (cudaEventElapsedTime(&b, p->spans[first].b, sp.b) != cudaSuccess ||
+            cudaEventElapsedTime(&e, p->spans[first].b, sp.e) != cudaSuccess) {
+            cudaGetLastError();
+            continue;
+        }
+        out[n].mini_batch = sp.mini_batch;
+        out[n].what = sp.what;
+        out[n].stream = sp.stream;
+        out[n].begin_ms = b;
+        out[n].end_ms = e;
+        ++n;
+    }
+    *n_out = n;
+    p->n_spans = 0;
     return HL_OK;
 }
 

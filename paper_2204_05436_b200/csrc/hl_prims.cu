@@ -62,7 +62,6 @@ __device__ __forceinline__ int64_t clamp_n(const int32_t* d_n, int64_t n_max) {
 // and a poll that runs out records HL_ETIMEOUT and carries on with what it has (positions are range-checked).
 constexpr uint32_t kFlagAgg = 1u << 30, kFlagPrefix = 1u << 31, kValueMask = kFlagAgg - 1u;
 constexpr unsigned long long kFlagAgg64 = 1ull << 62, kFlagPrefix64 = 1ull << 63, kValueMask64 = kFlagAgg64 - 1ull;
-constexpr int kMaxPolls = 1 << 20;
 
 __device__ __forceinline__ uint32_t ld_relaxed(const uint32_t* p) {
     uint32_t v;
@@ -83,8 +82,10 @@ __device__ __forceinline__ void st_relaxed64(unsigned long long* p, unsigned lon
 
 // ---- scan ---------------------------------------------------------------------------------------------------
 // st[0] = ticket counter, st[1 + tile] = status word of the tile; all zero on entry.
+// max_polls / stall_tile: see WaitCfg (a stalled tile publishes nothing, so that its successors' waits run out).
 __global__ void __launch_bounds__(kThreads) k_scan_chained(const int32_t* in, int32_t* out, const int32_t* d_n,
-                                                           int64_t n_max, unsigned long long* st, int32_t* status) {
+                                                           int64_t n_max, unsigned long long* st, int32_t* status,
+                                                           int max_polls, int64_t stall_tile) {
     __shared__ int smem[40];
     __shared__ long long s_tile, s_excl;
     if (threadIdx.x == 0) s_tile = (long long)atomicAdd(&st[0], 1ull);
@@ -109,7 +110,7 @@ __global__ void __launch_bounds__(kThreads) k_scan_chained(const int32_t* in, in
         const int lane = threadIdx.x;
         long long before = 0;
         if (tile > 0) {
-            if (lane == 0) st_relaxed64(&st[1 + tile], kFlagAgg64 | (unsigned long long)total);
+            if (lane == 0 && tile != stall_tile) st_relaxed64(&st[1 + tile], kFlagAgg64 | (unsigned long long)total);
             bool done = false;
             for (int64_t t0 = tile - 1; t0 >= 0 && !done; t0 -= 32) {
                 const int64_t t = t0 - lane;
@@ -117,7 +118,7 @@ __global__ void __launch_bounds__(kThreads) k_scan_chained(const int32_t* in, in
                 if (t >= 0) {
                     int polls = 0;
                     while (((w = ld_relaxed64(&st[1 + t])) & (kFlagAgg64 | kFlagPrefix64)) == 0) {
-                        if (++polls > kMaxPolls) {               // give up: carry on with what there is
+                        if (++polls > max_polls) {               // give up: carry on with what there is
                             set_status(status, HL_ETIMEOUT);
                             w = kFlagPrefix64;
                             break;
@@ -135,7 +136,7 @@ __global__ void __launch_bounds__(kThreads) k_scan_chained(const int32_t* in, in
             }
         }
         if (lane == 0) {
-            st_relaxed64(&st[1 + tile], kFlagPrefix64 | (unsigned long long)(before + total));
+            if (tile != stall_tile) st_relaxed64(&st[1 + tile], kFlagPrefix64 | (unsigned long long)(before + total));
             s_excl = before;
             if (n < tile_base + kScanTile) out[n] = (int32_t)(before + total);
         }
@@ -176,7 +177,8 @@ __global__ void __launch_bounds__(kThreads) k_sort_pass(const int32_t* __restric
                                                         int32_t* __restrict__ keys_out, int32_t* __restrict__ vals_out,
                                                         const int32_t* d_n, int64_t n_max, int shift,
                                                         const uint32_t* __restrict__ ghist, uint32_t* ticket,
-                                                        uint32_t* tstat, int32_t* status) {
+                                                        uint32_t* tstat, int32_t* status, int max_polls,
+                                                        int64_t stall_tile) {
     constexpr int kWarps = kThreads / 32;
     __shared__ uint32_t cnt[kWarps][256];
     __shared__ uint32_t digit_base[256];
@@ -222,7 +224,7 @@ __global__ void __launch_bounds__(kThreads) k_sort_pass(const int32_t* __restric
     uint32_t before = 0;
     uint32_t* my = tstat + tile * 256 + d;
     if (tile > 0) {
-        st_relaxed(my, kFlagAgg | total);
+        if (tile != stall_tile) st_relaxed(my, kFlagAgg | total);
         // walk back kLook tiles at a time (32 at a time was no faster and cost 16 registers): the kLook status
         // words are requested together, then consumed from the
         // nearest tile outwards until one of them already carries an inclusive prefix
@@ -237,7 +239,7 @@ __global__ void __launch_bounds__(kThreads) k_sort_pass(const int32_t* __restric
                 if (found || gave_up) break;
                 int polls = 0;
                 while ((w[k] & (kFlagAgg | kFlagPrefix)) == 0) {
-                    if (++polls > kMaxPolls) {
+                    if (++polls > max_polls) {
                         set_status(status, HL_ETIMEOUT);
                         gave_up = true;
                         break;
@@ -250,7 +252,7 @@ __global__ void __launch_bounds__(kThreads) k_sort_pass(const int32_t* __restric
             }
         }
     }
-    st_relaxed(my, kFlagPrefix | ((before + total) & kValueMask));
+    if (tile != stall_tile) st_relaxed(my, kFlagPrefix | ((before + total) & kValueMask));
     int all;
     const int gbase = block_exclusive_scan((int)ghist[d], scan_smem, all);   // keys with a smaller digit
     digit_base[d] = (uint32_t)gbase + before;
@@ -272,7 +274,7 @@ __global__ void __launch_bounds__(kThreads) k_sort_pass(const int32_t* __restric
 }  // namespace
 
 int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, int64_t n_max, int32_t* tiles,
-                           int32_t* status, cudaStream_t stream) {
+                           int32_t* status, cudaStream_t stream, WaitCfg w) {
     if (n_max <= 0) {
         HL_CUDA_TRY(cudaMemsetAsync(out, 0, sizeof(int32_t), stream));
         return HL_OK;
@@ -280,7 +282,8 @@ int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, 
     const int64_t n_tiles = n_max / kScanTile + 1;   // one more than needed when n is a multiple of the tile
     unsigned long long* st = reinterpret_cast<unsigned long long*>(tiles);
     HL_CUDA_TRY(cudaMemsetAsync(st, 0, sizeof(unsigned long long) * (n_tiles + 1), stream));
-    k_scan_chained<<<(unsigned)n_tiles, kThreads, 0, stream>>>(in, out, d_n, n_max, st, status);
+    k_scan_chained<<<(unsigned)n_tiles, kThreads, 0, stream>>>(in, out, d_n, n_max, st, status, w.max_polls,
+                                                               w.stall_tile);
     note_launches(1);
     HL_LAUNCH_CHECK();
     return HL_OK;
@@ -288,7 +291,7 @@ int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, 
 
 int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n, int64_t n_max, int key_bits,
                          uint32_t* hist, int32_t* status, int32_t** out_keys, int32_t** out_vals,
-                         cudaStream_t stream) {
+                         cudaStream_t stream, WaitCfg w) {
     int cur = 0;
     if (n_max > 0) {
         const int64_t n_tiles = div_up(n_max, kSortTile);
@@ -305,7 +308,8 @@ int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n,
         for (int p = 0; p < passes; ++p) {
             k_sort_pass<<<(unsigned)n_tiles, kThreads, 0, stream>>>(keys[cur], vals[cur], keys[cur ^ 1], vals[cur ^ 1],
                                                                     d_n, n_max, 8 * p, ghist + 256 * p, ticket + p,
-                                                                    tstat + (size_t)p * n_tiles * 256, status);
+                                                                    tstat + (size_t)p * n_tiles * 256, status,
+                                                                    w.max_polls, w.stall_tile);
             cur ^= 1;
         }
         note_launches(1 + passes);

@@ -311,9 +311,8 @@ __global__ void __launch_bounds__(kThreads) k_remap_dense(const RemapBlock* __re
 }  // namespace
 
 // implemented in hl_cold.cu: dst[(dst_row0 + i), :] = table[rows[i], :] for i < *d_n (clamped to n_max)
-int32_t launch_gather_rows(float* dst, int64_t dst_row0, const float* table, const int32_t* rows,
-                           const int64_t* d_n, int64_t n_max, int64_t table_rows, int D, int32_t* status,
-                           cudaStream_t stream);
+int32_t launch_gather_rows(hl_ctx* ctx, float* dst, int64_t dst_row0, const float* table, const int32_t* rows,
+                           const int64_t* d_n, int64_t n_max, int32_t* status, cudaStream_t stream);
 
 }  // namespace hl
 
@@ -335,7 +334,7 @@ extern "C" int32_t hl_profile_hot(hl_ctx* ctx, const hl_batch* b, int32_t reset,
             return HL_EINVAL;
         const int64_t bags_per_table = (int64_t)b->batch * ctx->S;
         const int64_t n_bags = bags_per_table * ctx->T;
-        k_count<<<grid_for(n_bags, kThreads, kSMs * 8), kThreads, 0, stream>>>(
+        k_count<<<grid_for(n_bags, kThreads, ctx_sms(ctx) * 8), kThreads, 0, stream>>>(
             b->indices, b->offsets, n_bags, bags_per_table, r.table_base, r.counts, r.sel, r.status);
         note_launches(1);
         HL_LAUNCH_CHECK();
@@ -361,7 +360,7 @@ extern "C" int32_t hl_profile_hot(hl_ctx* ctx, const hl_batch* b, int32_t reset,
         if (k < 0) return HL_EINVAL;
         if (k > ctx->hot_cap) k = ctx->hot_cap;
         k_select_begin<<<1, 256, 0, stream>>>(r.sel, (unsigned long long)k, share_num, share_den);
-        const int grid = grid_for(ctx->N, kThreads * 16, kSMs * 8);
+        const int grid = grid_for(ctx->N, kThreads * 16, ctx_sms(ctx) * 8);
         for (int shift = 24; shift >= 0; shift -= 8) {
             k_select_hist<<<grid, kThreads, 0, stream>>>(r.counts, ctx->N, shift, r.sel);
             k_select_pick<<<1, 256, 0, stream>>>(r.sel, shift);
@@ -385,19 +384,18 @@ extern "C" int32_t hl_build_remap(hl_ctx* ctx, const int32_t* d_hot_rows, const 
     Regions& r = ctx->r;
     HL_CUDA_TRY(cudaMemsetAsync(r.remap, 0, sizeof(RemapBlock) * ctx->n_remap_blocks, stream));
     if (ctx->hot_cap > 0) {
-        k_remap_bits<<<grid_for(ctx->hot_cap, kThreads, kSMs * 8), kThreads, 0, stream>>>(
+        k_remap_bits<<<grid_for(ctx->hot_cap, kThreads, ctx_sms(ctx) * 8), kThreads, 0, stream>>>(
             d_hot_rows, d_n_hot, ctx->hot_cap, ctx->N, r.remap, r.status);
         note_launches(1);
     }
-    k_remap_prefix<<<grid_for(ctx->n_remap_blocks, kThreads, kSMs * 8), kThreads, 0, stream>>>(
+    k_remap_prefix<<<grid_for(ctx->n_remap_blocks, kThreads, ctx_sms(ctx) * 8), kThreads, 0, stream>>>(
         d_hot_rows, d_n_hot, ctx->hot_cap, ctx->n_remap_blocks, r.remap);
     note_launches(d_remap_out ? 2 : 1);
     if (d_remap_out)
-        k_remap_dense<<<grid_for(ctx->N, kThreads * 4, kSMs * 16), kThreads, 0, stream>>>(r.remap, ctx->N,
+        k_remap_dense<<<grid_for(ctx->N, kThreads * 4, ctx_sms(ctx) * 16), kThreads, 0, stream>>>(r.remap, ctx->N,
                                                                                          d_remap_out);
     HL_LAUNCH_CHECK();
     if (host_table && ctx->hot_cap > 0)
-        return launch_gather_rows(d_cache, 0, host_table, d_hot_rows, d_n_hot, ctx->hot_cap, ctx->N, ctx->D,
-                                  r.status, stream);
+        return launch_gather_rows(ctx, d_cache, 0, host_table, d_hot_rows, d_n_hot, ctx->hot_cap, r.status, stream);
     return HL_OK;
 }

@@ -7,7 +7,6 @@ stream, then the non-popular micro-batch, then the write-back of its cold rows. 
 """
 from __future__ import annotations
 
-import os
 from typing import Optional, Sequence
 
 import torch
@@ -15,16 +14,12 @@ import torch
 from . import binding as B
 
 
-def _side_priority() -> int:
-    """Priority of the streams that carry ahead-work and host-link transfers (-1 = above the main stream's;
-    HOTLINE_SIDE_PRIORITY in the environment overrides it)."""
-    return int(os.environ.get("HOTLINE_SIDE_PRIORITY", "-1"))
-
-
 class Hotline:
     def __init__(self, table_rows: Sequence[int], dim: int, bags_per_sample: int, max_batch: int, max_nnz: int,
                  hot_cap_rows: int, staging_cap_rows: int, host_table: torch.Tensor, n_dense: int = 0,
-                 device: str = "cuda:0"):
+                 device: str = "cuda:0", main_priority: int = 0, side_priority: int = -1):
+        """``main_priority`` / ``side_priority``: CUDA stream priorities (0 = default, negative = higher) of the main
+        stream and of the streams that carry ahead-work and host-link transfers."""
         if not torch.cuda.is_available():
             raise RuntimeError("the Hotline library needs a CUDA device (there is no CPU fallback)")
         self.device = torch.device(device)
@@ -65,8 +60,9 @@ class Hotline:
         self.pooled_pop = torch.zeros((self.max_bags, self.D), dtype=f32, device=dev)
         self.pooled_non = torch.zeros((self.max_bags, self.D), dtype=f32, device=dev)
         self.dense_out = torch.zeros((self.max_batch, self.n_dense), dtype=f32, device=dev) if n_dense else None
-        self.main = torch.cuda.Stream(device=dev)
-        self.side = torch.cuda.Stream(device=dev, priority=_side_priority())
+        self.main_priority, self.side_priority = int(main_priority), int(side_priority)
+        self.main = torch.cuda.Stream(device=dev, priority=self.main_priority)
+        self.side = torch.cuda.Stream(device=dev, priority=self.side_priority)
         self.ev_frag = torch.cuda.Event()
         self.ev_gather = torch.cuda.Event()
         self.ev_pop_done = torch.cuda.Event()
@@ -289,7 +285,7 @@ class PipelinedHotline(Hotline):
 
     def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
                  n_dense: int = 0, device: str = "cuda:0", overlap_link: bool = True, sort_ahead: bool = True,
-                 combined_sort: bool = True, lookahead: int = 2):
+                 combined_sort: bool = True, lookahead: int = 2, main_priority: int = 0, side_priority: int = -1):
         self.overlap_link = bool(overlap_link)
         # sort_ahead (with overlap_link): the sorts of the two backward passes, which depend on the ids only, are
         # part of the ahead-work (hl_embbag_bwd_prepare on a side stream); the main stream keeps the forwards and
@@ -304,13 +300,14 @@ class PipelinedHotline(Hotline):
         self.lookahead = max(1, int(lookahead)) if self.sort_ahead else 1
         self.window_rows = int(window_rows)
         super().__init__(table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, 2 * self.window_rows,
-                         host_table, n_dense=n_dense, device=device)
+                         host_table, n_dense=n_dense, device=device, main_priority=main_priority,
+                         side_priority=side_priority)
         self.n_sets = self.lookahead + 2
         self.sets = [_BatchSet(self) for _ in range(self.n_sets)]
-        self.sides = [self.side] + [torch.cuda.Stream(device=self.device, priority=_side_priority())
+        self.sides = [self.side] + [torch.cuda.Stream(device=self.device, priority=self.side_priority)
                                     for _ in range(2)]
-        self.wb = torch.cuda.Stream(device=self.device, priority=_side_priority())
-        self.link = torch.cuda.Stream(device=self.device, priority=_side_priority())
+        self.wb = torch.cuda.Stream(device=self.device, priority=self.side_priority)
+        self.link = torch.cuda.Stream(device=self.device, priority=self.side_priority)
         self.j_submitted = 0      # mini-batches whose ahead-work (host read included) has been issued
         self.j_indexed = 0        # sort_ahead schedule: mini-batches whose index-only ahead-work has been issued
         self.j_done = 0           # mini-batches whose main work has been issued
@@ -578,16 +575,22 @@ class NativePipelinedHotline(Hotline):
     """
 
     def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
-                 n_dense: int = 0, device: str = "cuda:0", lookahead: int = 2, order: str = "fig8"):
+                 n_dense: int = 0, device: str = "cuda:0", lookahead: int = 2, order: str = "fig8",
+                 main_priority: int = -1, index_priority: int = 0, link_priority: int = 0, mover_ctas: int = 0,
+                 scatter_ctas: int = 0):
         """``order``: "fig8" = forward O, update O, forward X, update X (the paper's Fig. 8); "eq5" = both forwards,
         then one update of every touched row with the whole mini-batch's gradient (Eq. 5; the unfragmented step's
-        result): step() then takes ``grad_pop`` = [gradients of O's bags; gradients of X's bags] and no ``grad_non``."""
+        result): step() then takes ``grad_pop`` = [gradients of O's bags; gradients of X's bags] and no ``grad_non``.
+        ``main_priority`` / ``index_priority`` / ``link_priority``: CUDA stream priorities (0 = default, negative =
+        higher) of the main stream (bandwidth-bound forwards and updates), of the index-only ahead-work and of the
+        host-link transfers.  ``mover_ctas`` / ``scatter_ctas``: hl_set_mover_ctas (0 = the library's default)."""
         assert order in ("fig8", "eq5")
         self.order = order
         self.window_rows = int(window_rows)
         self.lookahead = max(1, int(lookahead))
         super().__init__(table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, 2 * self.window_rows,
-                         host_table, n_dense=n_dense, device=device)
+                         host_table, n_dense=n_dense, device=device, main_priority=main_priority,
+                         side_priority=index_priority)
         self.n_sets = self.lookahead + 2
         self.sets = [_BatchSet(self) for _ in range(self.n_sets)]
         c_sets = []
@@ -597,22 +600,24 @@ class NativePipelinedHotline(Hotline):
                 B._ptr(st.fwd_src), B._ptr(st.pooled_pop), B._ptr(st.pooled_non), B._ptr(st.dense_out),
                 B._ptr(st.sorted_all[0]), B._ptr(st.sorted_all[1]), B._ptr(st.sorted_all[2])))
         torch.cuda.synchronize(self.device)
-        self.pipe = B.hl_pipe_create(self.ctx, self.cache, self.host_table, self.window_rows, c_sets, self.n_dense,
-                                     self.main.cuda_stream)
+        if mover_ctas or scatter_ctas:
+            B.hl_set_mover_ctas(self.ctx, mover_ctas, scatter_ctas)
+        self.pipe = B.hl_pipe_create_ex(self.ctx, self.cache, self.host_table, self.window_rows, c_sets, self.n_dense,
+                                        self.main.cuda_stream, index_priority=index_priority,
+                                        link_priority=link_priority)
         if order == "eq5":
             B.hl_pipe_set_order(self.pipe, B.HL_PIPE_ORDER_EQ5)
         self.in_flight = 0
-        self._timer_pool = []
+        self.j_done = 0           # mini-batches stepped so far (mini-batch j stages its cold rows in window j % 2)
 
-    def _new_timer_events(self):
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-        for e in evs:
-            e.record(self.main)          # gives the event its handle
-        return evs
+    def trace_begin(self, max_spans: int, what_mask: int = B.HL_SPAN_ALL) -> None:
+        """Records a CUDA event pair around the library calls (and the timed kernels inside them) that the
+        following steps issue; trace_end() drains the pipeline and returns the spans."""
+        self._trace_cap = int(max_spans)
+        B.hl_pipe_trace_begin(self.pipe, max_spans, what_mask)
 
-    def prepare_timers(self, n: int) -> None:
-        """Creates the events of n timed steps ahead of time (step(timers=...) then only hands them to the library)."""
-        self._timer_pool.extend(self._new_timer_events() for _ in range(n))
+    def trace_end(self):
+        return B.hl_pipe_trace_end(self.pipe, self._trace_cap)
 
     def _hl_batch(self, nb):
         indices, offsets, batch, dense = nb
@@ -630,14 +635,9 @@ class NativePipelinedHotline(Hotline):
     def step(self, grad_pop: torch.Tensor, grad_non: torch.Tensor, lr: float, next_batch=None, timers=None,
              inputs_ready=None) -> int:
         b, d = self._hl_batch(next_batch) if next_batch is not None else (None, None)
-        if timers is not None:
-            # only the two forward calls can be timed from outside; the events are recorded inside the C call
-            evs = self._timer_pool.pop() if self._timer_pool else self._new_timer_events()
-            B.hl_pipe_time_forward(self.pipe, *evs)
-            timers.setdefault("fwd_pop", []).append((evs[0], evs[1]))
-            timers.setdefault("fwd_non", []).append((evs[2], evs[3]))
         s = B.hl_pipe_step(self.pipe, grad_pop, grad_non, lr, b, d, inputs_ready)
         self.in_flight += (1 if next_batch is not None else 0) - 1
+        self.j_done += 1
         return s
 
     @property

@@ -6,6 +6,8 @@ The oracle never sees a value produced by the CUDA path: both start from the sam
 """
 from __future__ import annotations
 
+import os
+
 import numpy as np
 import torch
 
@@ -499,6 +501,138 @@ def run_fullsize_check(spec, scale_rows: float = 1.0, n_samples: int = 1500, pro
             h.close()
         torch.cuda.synchronize()
         hl.hl_host_free(table.data_ptr())
+
+
+def run_native_fullsize_check(spec, steps: int = 4, scale_rows: float = 1.0, profile_batches=None, lookahead: int = 2,
+                              order: str = "fig8", device: str = "cuda:0", verbose: bool = False):
+    """The schedule the benchmark times (the library's own scheduler, hl_pipe_*, default lookahead and order) on a
+    workload too large to hold twice, over several mini-batches, against orc.hotline_step applied in sequence.
+
+    Integer-valued tables and gradients make every sum exact, so everything is compared bit for bit and in full:
+    perm, counts, the number of cold rows, both pooled arrays of every mini-batch, the whole hot cache at the end,
+    and every host row that any mini-batch wrote back; sampled host rows nobody touched must keep their bits.
+    The oracle's table is a sparse file mapped into memory (same shape as the real table, same global row ids):
+    only the rows the mini-batches stage are ever populated, with the values the procedural initialiser gives."""
+    import tempfile
+
+    import bench
+    import paper_2204_05436_b200 as hl
+
+    if isinstance(spec, str):
+        spec = gen.CONFIGS[spec]
+    geom = gen.make_geometry(spec, scale_rows)
+    T, D, S, B = geom.num_tables, geom.dim, geom.bags_per_sample, spec.batch
+    N = geom.total_rows
+    n_bags = T * B * S
+    P = spec.profile_batches if profile_batches is None else profile_batches
+    lr = 0.125
+    max_nnz = max_nnz_of(spec, geom, B)
+    K = orc.hot_capacity(spec.hot_policy, N, D)
+    hot_cap = max(1, min(K, N))
+    window = max(1, min(N, max_nnz))
+    rng = np.random.default_rng(spec.seed + 777)
+    rows_of = lambda g: gen.table_values(np.asarray(g, dtype=np.int64), D, spec.seed, integer=True)   # noqa: E731
+
+    table = hl.host_table_tensor(N, D)
+    p, table_o = None, None
+    tmp = tempfile.TemporaryDirectory()
+    try:
+        bench.fill_table(table, D, spec.seed, torch.device(device), integer=True)
+        probe = rng.integers(0, N, 64)
+        assert np.array_equal(table.numpy()[probe], rows_of(probe)), "table fill"
+
+        # ---- oracle: learning phase, then the mini-batches one after the other on the sparse table ----
+        prof = [gen.make_batch(spec, geom, i) for i in range(P)]
+        cnt = orc.access_counts([(b.indices, b.offsets) for b in prof], B, geom.table_rows, S)
+        hot_o = orc.select_hot(cnt, min(K, hot_cap))
+        del cnt
+        n_hot = len(hot_o)
+        remap_o = orc.build_remap(hot_o, N)
+        batches = [gen.make_batch(spec, geom, P + i) for i in range(steps)]
+        table_o = np.memmap(os.path.join(tmp.name, "oracle_table.f32"), dtype=np.float32, mode="w+", shape=(N, D))
+        staged_rows = np.zeros(0, dtype=np.int64)
+        for b in batches:                       # index-only pass: which rows will ever be staged
+            _, _, _, X, _ = orc.fragment(b.indices, b.offsets, B, geom.table_rows, remap_o, S)
+            C, _ = orc.gather_cold(X.ids, remap_o, hot_cap)
+            staged_rows = np.union1d(staged_rows, C)
+        table_o[staged_rows] = rows_of(staged_rows)
+        cache_o = np.zeros((hot_cap + window, D), dtype=np.float32)
+        cache_o[:n_hot] = rows_of(hot_o)
+        grads, expect, shared, prev_C = [], [], 0, np.zeros(0, dtype=np.int64)
+        for i, b in enumerate(batches):
+            grad_full = gen.grad_values(spec.seed, P + i, 2, n_bags, D, integer=True)
+            perm_o, n_pop_o, _, _, _ = orc.fragment(b.indices, b.offsets, B, geom.table_rows, remap_o, S)
+            g_pop, _ = mu_grad(grad_full, perm_o[:n_pop_o], T, B, S)
+            g_non, _ = mu_grad(grad_full, perm_o[n_pop_o:], T, B, S)
+            out = orc.hotline_step(table_o, cache_o, hot_cap, remap_o, b.indices, b.offsets, B, geom.table_rows, S,
+                                   g_pop, g_non, lr, deferred=(order == "eq5"))
+            _, _, O, X, C, pooled_pop_o, pooled_non_o = out
+            shared += len(np.intersect1d(C, prev_C))
+            prev_C = C
+            grads.append((g_pop, g_non))
+            expect.append((perm_o, n_pop_o, len(O.ids), len(X.ids), len(C), pooled_pop_o, pooled_non_o))
+
+        # ---- CUDA: the library's scheduler ----
+        p = hl.NativePipelinedHotline(geom.table_rows, D, S, B, max_nnz, hot_cap, window, table, n_dense=spec.n_dense,
+                                      device=device, lookahead=lookahead, order=order)
+        with torch.cuda.stream(p.main):
+            pol, p_num, p_den = policy_args(spec.hot_policy)
+            for i, b in enumerate(prof):
+                p.profile(_t(b.indices, device), _t(b.offsets, device), B, reset=(i == 0))
+            p.profile(None, None, finalize=True, policy=pol, p_num=p_num, p_den=p_den)
+            p.build_remap(load_rows=True)
+            p.status()
+            assert int(p.n_hot.item()) == n_hot, ("n_hot", int(p.n_hot.item()), n_hot)
+            assert np.array_equal(p.hot_rows[:n_hot].cpu().numpy(), hot_o.astype(np.int32)), "hot rows"
+            del prof
+            d_batches = [(_t(b.indices, device), _t(b.offsets, device), B,
+                          _t(b.dense, device) if b.dense is not None else None) for b in batches]
+            d_grads = []
+            for (g_pop, g_non) in grads:
+                gp = torch.zeros((n_bags, D), dtype=torch.float32, device=device)
+                gp[:len(g_pop)] = _t(g_pop, device)
+                if order == "eq5":
+                    gp[len(g_pop):len(g_pop) + len(g_non)] = _t(g_non, device)
+                    gn = None
+                else:
+                    gn = torch.zeros((n_bags, D), dtype=torch.float32, device=device)
+                    gn[:len(g_non)] = _t(g_non, device)
+                d_grads.append((gp, gn))
+            torch.cuda.synchronize()
+            # outputs are read back after every step's main work, while later mini-batches are already in flight
+            p.start(*d_batches[0], more=d_batches[1:lookahead])
+            for i in range(steps):
+                nxt = d_batches[i + lookahead] if i + lookahead < steps else None
+                st = p.sets[p.step(d_grads[i][0], d_grads[i][1], lr, next_batch=nxt)]
+                perm_o, n_pop_o, L_pop, L_non, n_cold_o, pooled_pop_o, pooled_non_o = expect[i]
+                p.main.synchronize()
+                assert st.counts.cpu().tolist() == [n_pop_o, B - n_pop_o, L_pop, L_non], ("counts", i)
+                assert np.array_equal(st.perm[:B].cpu().numpy(), perm_o), ("perm", i)
+                assert int(st.n_cold.item()) == n_cold_o, ("n_cold", i, int(st.n_cold.item()), n_cold_o)
+                bags_pop, bags_non = T * n_pop_o * S, T * (B - n_pop_o) * S
+                assert np.array_equal(st.pooled_pop[:bags_pop].cpu().numpy(), pooled_pop_o), ("pooled_pop", i)
+                assert np.array_equal(st.pooled_non[:bags_non].cpu().numpy(), pooled_non_o), ("pooled_non", i)
+            p.drain()
+            p.status()
+        assert np.array_equal(p.cache[:n_hot].cpu().numpy(), cache_o[:n_hot]), "hot cache"
+        host = table.numpy()
+        assert np.array_equal(host[staged_rows], np.asarray(table_o[staged_rows])), "written-back host rows"
+        assert not np.array_equal(np.asarray(table_o[staged_rows]), rows_of(staged_rows)), "the updates changed nothing"
+        far = rng.integers(0, N, 4096)
+        far = far[~np.isin(far, staged_rows)]
+        assert np.array_equal(host[far], rows_of(far)), "host rows nobody touched"
+        stats = dict(N=N, batch=B, steps=steps, n_hot=n_hot, n_pop=[e[1] for e in expect], n_cold=[e[4] for e in expect],
+                     shared_cold_rows=shared, staged_rows=len(staged_rows))
+        if verbose:
+            print(f"[{spec.name} full size, hl_pipe] {stats}")
+        return stats
+    finally:
+        if p is not None:
+            p.close()
+        torch.cuda.synchronize()
+        hl.hl_host_free(table.data_ptr())
+        del table_o
+        tmp.cleanup()
 
 
 def run_recalibration_check(spec, steps_per_phase: int = 2, device: str = "cuda:0"):

@@ -1,10 +1,12 @@
-"""The named configurations at (or near) their full sizes, in the launch configuration bench.py times."""
+"""The named configurations at (or near) their full sizes: call by call and through Hotline.step (one mini-batch
+after the other), and -- the DLRM-large-like one -- through the library's own scheduler, hl_pipe_*, which is the
+launch configuration bench.py times."""
 import dataclasses
 
 import pytest
 
 import gen
-from tests.harness import run_config_check, run_fullsize_check, run_pipelined_check
+from tests.harness import run_config_check, run_fullsize_check, run_native_fullsize_check, run_pipelined_check
 
 pytestmark = pytest.mark.gpu
 
@@ -14,6 +16,17 @@ def test_dlrm_large_full_size_sampled():
     float results on samples."""
     stats = run_fullsize_check("dlrm_large")
     assert stats["N"] > 250_000_000 and 0 < stats["n_pop"] < stats["batch"] and stats["n_cold"] > 1000
+
+
+def test_dlrm_large_full_size_through_the_benchmarked_schedule_bit_exact():
+    """The same workload through NativePipelinedHotline (hl_pipe_*, index work two mini-batches ahead, order of
+    Fig. 8) -- what bench.py times by default -- for five mini-batches on integer-valued tables and gradients:
+    perm, counts, cold-row counts, every pooled vector, the whole hot cache and every written-back host row bit for
+    bit against orc.hotline_step applied in sequence.  At this size the one-cluster cold-row search sees about
+    18 K cold lookups, the movers choose their number of working CTAs, and both staging windows are in use."""
+    stats = run_native_fullsize_check("dlrm_large", steps=5)
+    assert stats["N"] > 250_000_000 and min(stats["n_cold"]) > 10_000
+    assert all(0 < n < stats["batch"] for n in stats["n_pop"])
 
 
 def test_tbsm_full_size_every_element():
