@@ -31,6 +31,7 @@ METRIC = "samples/sec through fragment+embbag fwd/bwd"
 UNIT = "samples/s"
 L2_BYTES = 126 << 20
 FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+SINGLE_ALLOCATION_LIMIT = 64 << 30  # a larger host table is held as one allocation per table
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the forward kernel per bag at dim 64, from the ncu capture
 # summarised in profiles/k_embbag_fwd_micro_dim64.md (164.4 MB for 425,984 one-lookup bags).  The bench's own
@@ -72,13 +73,14 @@ def max_nnz_of(spec, geom) -> int:
     return bags if spec.pooling[0] == "one" else bags * int(spec.pooling[2])
 
 
-def fill_table(table, dim: int, seed: int, device, chunk_rows: int = 1 << 21, integer: bool = False) -> None:
-    """table[g, :] = gen.table_values(g) for every row, computed on the device in chunks and copied down."""
+def fill_table(table, dim: int, seed: int, device, chunk_rows: int = 1 << 21, integer: bool = False,
+               row0: int = 0) -> None:
+    """table[i, :] = gen.table_values(row0 + i) for every row, computed on the device in chunks and copied down."""
     import torch
     n = table.shape[0]
     for r0 in range(0, n, chunk_rows):
         r1 = min(n, r0 + chunk_rows)
-        table[r0:r1].copy_(gen.table_values_torch(r0, r1 - r0, dim, seed, device, integer=integer))
+        table[r0:r1].copy_(gen.table_values_torch(row0 + r0, r1 - r0, dim, seed, device, integer=integer))
     if str(device) != "cpu":
         torch.cuda.synchronize()
 
@@ -102,10 +104,17 @@ class Workload:
         if with_table:       # the CUDA arm's host table: memory the device can address, filled from the device
             import paper_2204_05436_b200 as hl
             t0 = time.time()
-            self.table = hl.host_table_tensor(self.N, self.D)
-            fill_table(self.table, self.D, s.seed, device)
-            log(f"[bench] host table {self.N} x {self.D} fp32 = {self.N * self.D * 4 / 2**30:.1f} GiB pinned+filled "
-                f"in {time.time() - t0:.1f}s")
+            if self.N * self.D * 4 > SINGLE_ALLOCATION_LIMIT:
+                # above what one large-page allocation takes: one allocation per table (hl_set_host_tables)
+                self.table = [hl.host_table_tensor(r, self.D) for r in g.table_rows]
+                for t, ten in enumerate(self.table):
+                    fill_table(ten, self.D, s.seed, device, row0=int(g.base[t]))
+            else:
+                self.table = hl.host_table_tensor(self.N, self.D)
+                fill_table(self.table, self.D, s.seed, device)
+            log(f"[bench] host table {self.N} x {self.D} fp32 = {self.N * self.D * 4 / 2**30:.1f} GiB "
+                f"({len(self.table) if isinstance(self.table, list) else 1} allocation(s)) filled in "
+                f"{time.time() - t0:.1f}s")
         t0 = time.time()
         self.profile = [gen.make_batch(s, g, i, threads) for i in range(self.P)]
         self.batches = [gen.make_batch(s, g, self.P + i, threads) for i in range(n_batches)]
@@ -132,9 +141,10 @@ class Workload:
         if self.table is None:
             return
         import paper_2204_05436_b200 as hl
-        ptr = self.table.data_ptr()
+        ptrs = [t.data_ptr() for t in (self.table if isinstance(self.table, list) else [self.table])]
         self.table = None
-        hl.hl_host_free(ptr)
+        for ptr in ptrs:
+            hl.hl_host_free(ptr)
 
 
 # ----------------------------------------------------------------------------------------------------------
@@ -463,7 +473,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                                       n_dense=wl.spec.n_dense, device=str(device), lookahead=args.lookahead,
                                       order=args.order, main_priority=args.main_priority,
                                       index_priority=args.index_priority, link_priority=args.link_priority,
-                                      mover_ctas=args.mover_ctas, scatter_ctas=args.scatter_ctas)
+                                      mover_ctas=args.mover_ctas, scatter_ctas=args.scatter_ctas,
+                                      exclusive_write_back=args.exclusive_write_back)
     elif pipelined:
         h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
                                 n_dense=wl.spec.n_dense, device=str(device), overlap_link=not args.serial_link,
@@ -477,6 +488,8 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
             hl.hl_set_mover_ctas(h.ctx, args.mover_ctas, args.scatter_ctas)
     lr = wl.spec.lr
     sms = torch.cuda.get_device_properties(device).multi_processor_count
+    if args.fwd_ctas or args.bwd_ctas:
+        hl.hl_set_kernel_width(h.ctx, args.fwd_ctas, args.bwd_ctas)
 
     with torch.cuda.stream(h.main):
         # ---- learning phase (setup, timed separately) ----
@@ -955,10 +968,21 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                            "ms_per_step": e2e["ms_total"] / args.steps}
         if world == 1 and not args.no_cpu_baseline:
             h.close()
-            runner = OracleRunner(wl, wl.table.numpy())
-            runner.load_cache()
+            if isinstance(wl.table, list):
+                # per-table allocations: the oracle gets a sparse table holding the rows its mini-batches stage
+                import tempfile
+                tmp = tempfile.TemporaryDirectory()
+                runner = OracleRunner(wl, None)
+                need = np.unique(np.concatenate([runner.sizes(b)["C"] for b in wl.batches[:2]]))
+                runner.table = sparse_oracle_table(wl, need, tmp.name)
+                runner.load_cache(gen.table_values(runner.hot, D, wl.spec.seed))
+                oracle_batches = wl.batches[:2]
+            else:
+                runner = OracleRunner(wl, wl.table.numpy())
+                runner.load_cache()
+                oracle_batches = wl.batches
             times, checked = [], 0
-            for i, b in enumerate(wl.batches):
+            for i, b in enumerate(oracle_batches):
                 dt, sz = runner.step(b)
                 times.append(dt)
                 # the oracle is the checker of what was timed: the sizes the device found for this mini-batch
@@ -972,7 +996,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                                     "sample": f"{len(times)} whole mini-batches of {B} inputs ({sum(times):.1f} s)",
                                     "cross_check": f"n_pop, n_non, L_pop, L_non, n_cold of {checked} timed mini-batches "
                                                    "equal the device's"}
-            cores = host_cores()
+            cores = min(host_cores(), 32)
             if cores > 1:
                 t_all = [runner.step_all_cores(wl.batches[i % len(wl.batches)], cores) for i in range(4)]
                 line["cpu_baseline"]["all_cores"] = {
@@ -1145,6 +1169,8 @@ def run_micro(args) -> None:
     ws_bytes = hl.hl_workspace_bytes(geom, n_bags, n_bags, H, 0)
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
     ctx = hl.hl_create(geom, n_bags, n_bags, H, 0, ws, ws_bytes)
+    if args.fwd_ctas or args.bwd_ctas:
+        hl.hl_set_kernel_width(ctx, args.fwd_ctas, args.bwd_ctas)
     cache = torch.rand((H, D), device=dev, dtype=torch.float32) - 0.5
     d_ids = torch.from_numpy(ids.astype(np.int32)).to(dev)
     d_off = torch.arange(n_bags + 1, dtype=torch.int32, device=dev)
@@ -1314,6 +1340,10 @@ def main() -> None:
     ap.add_argument("--link-priority", type=int, default=0, help="CUDA priority of the host-link transfer streams")
     ap.add_argument("--mover-ctas", type=int, default=0, help="hl_set_mover_ctas: CTAs of the host reads (0 = default)")
     ap.add_argument("--scatter-ctas", type=int, default=0, help="hl_set_mover_ctas: CTAs of the write-backs")
+    ap.add_argument("--exclusive-write-back", action="store_true",
+                    help="a mini-batch's main work waits for the previous write-back (hl_pipe_options)")
+    ap.add_argument("--fwd-ctas", type=int, default=0, help="hl_set_kernel_width: forward CTAs per multiprocessor")
+    ap.add_argument("--bwd-ctas", type=int, default=0, help="hl_set_kernel_width: backward-sum CTAs per multiprocessor")
     ap.add_argument("--timeline", default=None,
                     help="write the per-stream timeline of three mini-batches of the traced pass to this text file")
     ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather", "tracker"],

@@ -137,11 +137,26 @@ HL_API int32_t hl_timing_read(hl_ctx* ctx, int32_t which, float* ms);
 HL_API void* hl_host_alloc(size_t bytes);
 HL_API int32_t hl_host_free(void* p);
 
+/* Section V-A (the Data Dispatcher keeps one base address per table).  Installs one host-memory allocation per
+ * table instead of a single allocation that holds all tables back to back: h_table_bases is a HOST array of
+ * num_tables pointers, each to fp32 [table_rows[t], D] that the device can read and write (16-byte aligned).  From
+ * then on global row g of table t is at h_table_bases[t] + (g - base_t) * D, and the `host_table` argument of every
+ * other call only says whether the host table takes part (non-NULL) -- its value is not used.  NULL returns to the
+ * single-allocation form.  Synchronises the device.  (A table too large for one allocation of hl_host_alloc's
+ * large-page memory -- 8 x 9.5 GiB of the multi-hot configuration, say -- is held this way.) */
+HL_API int32_t hl_set_host_tables(hl_ctx* ctx, float* const* h_table_bases);
+
 /* Width of the host-link movers inside a schedule: how many CTAs of hl_gather_cold / hl_stage_cold (read_ctas) and of
  * hl_scatter_cold (write_ctas) work when a mini-batch moves a DLRM-sized number of rows (the kernels decide on the
  * device, from the number of rows, whether more join in).  0 = the default (16); at most two per multiprocessor.
  * Wider movers finish sooner and slow the kernels that run beside them more.  Takes effect with the next call. */
 HL_API int32_t hl_set_mover_ctas(hl_ctx* ctx, int32_t read_ctas, int32_t write_ctas);
+
+/* Grid size of the two bandwidth-bound kernels, in CTAs per multiprocessor: the forward kernel (hl_embbag_fwd) and
+ * the backward's sum kernel (hl_embbag_bwd_*).  Both deal their work out evenly over a fixed grid; fewer CTAs per
+ * multiprocessor leave registers and shared memory for the kernels of other streams (index work, movers) to run
+ * beside them, more give the kernel itself more loads in flight.  0 = the default (3 and 3). */
+HL_API int32_t hl_set_kernel_width(hl_ctx* ctx, int32_t fwd_ctas_per_sm, int32_t bwd_ctas_per_sm);
 
 /* Test aid for the bounded device-side waits (the tile chaining of the scan inside hl_fragment and of the sorts
  * inside hl_embbag_bwd_* / hl_gather_cold, the wait of a row mover for a stage of bulk copies).  In production these
@@ -403,6 +418,10 @@ HL_API hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_table, i
 typedef struct {
     int32_t index_priority;          /* the three streams of index-only ahead-work (fragment, cold-row search, sort) */
     int32_t link_priority;           /* the two streams of host-link transfers (host read, write-back)              */
+    int32_t exclusive_write_back;    /* != 0: the main work of mini-batch j starts only when the write-back of j - 1 has
+                                        finished, so that no bandwidth-bound kernel runs beside a write-back (which
+                                        slows such a kernel several times over); the index-only ahead-work and the
+                                        host read still overlap it                                                   */
 } hl_pipe_options;
 HL_API hl_pipe* hl_pipe_create_ex(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows, int32_t n_sets,
                                   const hl_pipe_set* sets, int32_t n_dense, void* main_stream,

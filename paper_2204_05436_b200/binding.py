@@ -23,7 +23,7 @@ EXPORTS = (
     "hl_embbag_bwd_prepare2", "hl_embbag_bwd_apply2",
     "hl_tracker_reset", "hl_tracker_update", "hl_tracker_export",
     "hl_pipe_create", "hl_pipe_create_ex", "hl_pipe_destroy", "hl_pipe_submit", "hl_pipe_step", "hl_pipe_wait_outputs", "hl_pipe_drain",
-    "hl_pipe_trace_begin", "hl_pipe_trace_end", "hl_pipe_wait_counts", "hl_set_mover_ctas", "hl_test_bounded_waits",
+    "hl_pipe_trace_begin", "hl_pipe_trace_end", "hl_pipe_wait_counts", "hl_set_mover_ctas", "hl_test_bounded_waits", "hl_set_host_tables", "hl_set_kernel_width",
     "hl_index_cold_begin", "hl_index_cold_end", "hl_index_cold_verdict",
     "hl_embbag_bwd_prepare_merged", "hl_pipe_set_order",
 )
@@ -57,7 +57,8 @@ class hl_pipe_set(ctypes.Structure):
 
 
 class hl_pipe_options(ctypes.Structure):
-    _fields_ = [("index_priority", ctypes.c_int32), ("link_priority", ctypes.c_int32)]
+    _fields_ = [("index_priority", ctypes.c_int32), ("link_priority", ctypes.c_int32),
+                ("exclusive_write_back", ctypes.c_int32)]
 
 
 class hl_pipe_span(ctypes.Structure):
@@ -166,6 +167,10 @@ def _load() -> ctypes.CDLL:
     lib.hl_pipe_trace_end.argtypes = [vp, ctypes.POINTER(hl_pipe_span), i32, ctypes.POINTER(i32)]
     lib.hl_set_mover_ctas.restype = i32
     lib.hl_set_mover_ctas.argtypes = [vp, i32, i32]
+    lib.hl_set_kernel_width.restype = i32
+    lib.hl_set_kernel_width.argtypes = [vp, i32, i32]
+    lib.hl_set_host_tables.restype = i32
+    lib.hl_set_host_tables.argtypes = [vp, ctypes.POINTER(vp)]
     lib.hl_test_bounded_waits.restype = i32
     lib.hl_test_bounded_waits.argtypes = [vp, i32, i64]
     lib.hl_flush_hot.restype = i32
@@ -436,10 +441,11 @@ def hl_pipe_create(ctx: int, d_cache, host_table, window_rows: int, sets, n_dens
 
 
 def hl_pipe_create_ex(ctx: int, d_cache, host_table, window_rows: int, sets, n_dense: int, main_stream: int,
-                      index_priority: int = 0, link_priority: int = 0) -> int:
-    """hl_pipe_create with the stream priorities of the ahead-work and of the host-link transfers."""
+                      index_priority: int = 0, link_priority: int = 0, exclusive_write_back: bool = False) -> int:
+    """hl_pipe_create with its options: the stream priorities of the ahead-work and of the host-link transfers, and
+    whether a mini-batch's main work waits for the previous write-back."""
     arr = (hl_pipe_set * len(sets))(*sets)
-    opt = hl_pipe_options(int(index_priority), int(link_priority))
+    opt = hl_pipe_options(int(index_priority), int(link_priority), int(bool(exclusive_write_back)))
     p = _lib.hl_pipe_create_ex(ctx, _ptr(d_cache), _ptr(host_table), int(window_rows), len(sets), arr, int(n_dense),
                                main_stream, ctypes.byref(opt))
     if not p:
@@ -449,6 +455,19 @@ def hl_pipe_create_ex(ctx: int, d_cache, host_table, window_rows: int, sets, n_d
 
 def hl_set_mover_ctas(ctx: int, read_ctas: int, write_ctas: int) -> None:
     _check("hl_set_mover_ctas", _lib.hl_set_mover_ctas(ctx, int(read_ctas), int(write_ctas)))
+
+
+def hl_set_kernel_width(ctx: int, fwd_ctas_per_sm: int, bwd_ctas_per_sm: int) -> None:
+    _check("hl_set_kernel_width", _lib.hl_set_kernel_width(ctx, int(fwd_ctas_per_sm), int(bwd_ctas_per_sm)))
+
+
+def hl_set_host_tables(ctx: int, tables) -> None:
+    """``tables``: one device-addressable fp32 [rows_t, D] tensor (or address) per table, or None for a single table."""
+    if tables is None:
+        _check("hl_set_host_tables", _lib.hl_set_host_tables(ctx, None))
+        return
+    arr = (ctypes.c_void_p * len(tables))(*[_ptr(t) for t in tables])
+    _check("hl_set_host_tables", _lib.hl_set_host_tables(ctx, arr))
 
 
 def hl_test_bounded_waits(ctx: int, poll_limit: int, stall_tile: int = -1) -> None:

@@ -18,8 +18,10 @@ OBJ_DIR = os.path.join(CSRC, "build")
 LIB_PATH = os.path.join(PKG_DIR, "libhotline.so")
 INCLUDE = os.path.join(ROOT, "include")
 
+# -rdc=true: the cold-row search launches its general path from the device (tail launches), so device code is
+# linked across files and against the device runtime
 NVCC_FLAGS = [
-    "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+    "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-rdc=true",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-I", INCLUDE, "-I", CSRC,
 ]
 
@@ -68,7 +70,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
                     print(log)
     objs = [os.path.join(OBJ_DIR, os.path.basename(s)[:-3] + ".o") for s in sources()]
     if force or jobs or _stale(LIB_PATH, objs):
-        run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_PATH] + objs)
+        run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_PATH] + objs + ["-lcudadevrt"])
     return LIB_PATH
 
 

@@ -45,6 +45,7 @@ size_t carve(char* base, const hl_geometry* g, int64_t N, int32_t max_batch, int
     *n_sel_tiles = div_up(N, kSelTile);
     r->status = c.take<int32_t>(8);
     r->table_base = c.take<int64_t>(T + 1);
+    r->table_ptrs = c.take<unsigned char*>(T);
     r->remap = c.take<RemapBlock>(*n_remap_blocks);
     r->counts = c.take<uint32_t>(N);
     r->sel = c.take<SelectState>(1);
@@ -148,11 +149,33 @@ extern "C" int32_t hl_create(hl_ctx** out, const hl_geometry* geom, int32_t max_
     return HL_OK;
 }
 
+extern "C" int32_t hl_set_host_tables(hl_ctx* ctx, float* const* h_table_bases) {
+    if (!ctx) return HL_EINVAL;
+    if (!h_table_bases) {
+        ctx->per_table = 0;
+        return HL_OK;
+    }
+    for (int t = 0; t < ctx->T; ++t)
+        if (!h_table_bases[t] || (reinterpret_cast<uintptr_t>(h_table_bases[t]) & 15)) return HL_EINVAL;
+    HL_CUDA_TRY(cudaDeviceSynchronize());      // no kernel may still be reading the previous addresses
+    HL_CUDA_TRY(cudaMemcpy(ctx->r.table_ptrs, h_table_bases, sizeof(float*) * ctx->T, cudaMemcpyHostToDevice));
+    ctx->per_table = 1;
+    return HL_OK;
+}
+
 extern "C" int32_t hl_set_mover_ctas(hl_ctx* ctx, int32_t read_ctas, int32_t write_ctas) {
     if (!ctx || read_ctas < 0 || write_ctas < 0) return HL_EINVAL;
     const int most = 2 * ctx_sms(ctx);
     ctx->mover_ctas = read_ctas == 0 ? kMoverCtasDefault : (read_ctas < most ? read_ctas : most);
     ctx->scatter_ctas = write_ctas == 0 ? kMoverCtasDefault : (write_ctas < most ? write_ctas : most);
+    return HL_OK;
+}
+
+extern "C" int32_t hl_set_kernel_width(hl_ctx* ctx, int32_t fwd_ctas_per_sm, int32_t bwd_ctas_per_sm) {
+    if (!ctx || fwd_ctas_per_sm < 0 || bwd_ctas_per_sm < 0 || fwd_ctas_per_sm > 32 || bwd_ctas_per_sm > 32)
+        return HL_EINVAL;
+    ctx->fwd_ctas = fwd_ctas_per_sm;
+    ctx->bwd_ctas = bwd_ctas_per_sm;
     return HL_OK;
 }
 

@@ -56,11 +56,8 @@ __global__ void __launch_bounds__(kThreads) k_cold_classify(int32_t* __restrict_
     }
 }
 
-__global__ void __launch_bounds__(kThreads) k_cold_heads(const int32_t* __restrict__ keys,
-                                                         const int32_t* __restrict__ d_n, int64_t n_max,
+__global__ void __launch_bounds__(kThreads) k_cold_heads(const int32_t* __restrict__ keys, int64_t n,
                                                          int32_t* __restrict__ heads) {
-    int64_t n = *d_n;
-    n = n < n_max ? n : n_max;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         heads[i] = (i == 0 || keys[i] != keys[i - 1]) ? 1 : 0;
 }
@@ -68,17 +65,12 @@ __global__ void __launch_bounds__(kThreads) k_cold_heads(const int32_t* __restri
 // rank_excl[i] = number of run heads before i; the row at i has rank rank_excl[i] if it is a head, else
 // rank_excl[i] - 1.  A row of rank r is staged at cache slot slot0 + r (slot0 = start of the staging window).
 __global__ void __launch_bounds__(kThreads) k_cold_assign(const int32_t* __restrict__ keys,
-                                                          const int32_t* __restrict__ vals,
-                                                          const int32_t* __restrict__ d_n, int64_t n_max,
+                                                          const int32_t* __restrict__ vals, int64_t n,
                                                           const int32_t* __restrict__ rank_excl, int64_t slot0,
                                                           int64_t staging_cap, int32_t* __restrict__ ids,
                                                           int32_t* __restrict__ cold_rows,
                                                           int64_t* __restrict__ d_n_cold, int32_t* status,
-                                                          const int32_t* __restrict__ d_n_classified,
                                                           int64_t cap_ids) {
-    int64_t n = *d_n;
-    n = n < n_max ? n : n_max;
-    if (n == 0 && d_n_classified[0] != 0) return;    // the one-cluster path has done all of this already
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         int64_t distinct = rank_excl[n];
         if (distinct > staging_cap) {
@@ -109,14 +101,28 @@ __global__ void __launch_bounds__(kThreads) k_cold_assign(const int32_t* __restr
 // adds up the digit counts of the 8 CTAs through distributed shared memory, and writes each pair into the shared
 // memory of the CTA that owns its new position.  The sorted list is then ranked and assigned in place.
 // Order of a CTA's items: position = warp * (32 * kSmallItems) + round * 32 + lane.
-// Larger inputs: the kernel hands the count to the general path (*d_n_general = n) and leaves; otherwise it sets
-// *d_n_general = 0, which turns the general path's kernels into no-ops.
+// Larger inputs: the kernel launches the general path itself (tile sort, head flags, scan, assignment) as tail
+// launches, which run after this grid and before anything the host queued behind it -- so the host queues the same
+// two kernels for every mini-batch and never needs to know which path ran.  *d_n_general = the number of cold lookups
+// handed to the general path (0: none).
 constexpr int kSmallCtas = 8;
 constexpr int kSmallThreads = 256;
 constexpr int kSmallItems = 10;
 constexpr int kSmallPerCta = kSmallThreads * kSmallItems;       // 2560
 constexpr int kSmallCap = kSmallCtas * kSmallPerCta;            // 20480
 constexpr int kSmallWarps = kSmallThreads / 32;
+
+// what the general path works on (device pointers into the context's cold region)
+struct GeneralArgs {
+    int32_t* keys[2];
+    int32_t* vals[2];
+    uint32_t* hist;
+    int32_t* rank;
+    int32_t* tiles;
+    int64_t cap_ids;
+    int key_bits;
+    int max_polls;
+};
 
 __device__ __forceinline__ int block_scan_small(int v, int* smem33, int& total) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -153,7 +159,8 @@ __global__ void __launch_bounds__(kSmallThreads) k_cold_small(const int32_t* __r
                                                               int32_t* __restrict__ ids,
                                                               int32_t* __restrict__ cold_rows,
                                                               int64_t* __restrict__ d_n_cold,
-                                                              int32_t* __restrict__ d_n_general, int32_t* status) {
+                                                              int32_t* __restrict__ d_n_general, int32_t* status,
+                                                              GeneralArgs ga) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ int32_t s_key[kSmallPerCta];
@@ -167,7 +174,22 @@ __global__ void __launch_bounds__(kSmallThreads) k_cold_small(const int32_t* __r
     n64 = n64 < 0 ? 0 : (n64 < n_max ? n64 : n_max);
     const int cta = (int)cluster.block_rank();
     if (n64 > kSmallCap) {                   // the same decision in all CTAs, before any cluster barrier
-        if (cta == 0 && threadIdx.x == 0) d_n_general[0] = (int32_t)n64;
+        if (cta == 0 && threadIdx.x == 0) {
+            d_n_general[0] = (int32_t)n64;
+            // the general path, queued behind this grid: stable sort of the (row, position) pairs by row, a flag at
+            // the head of every run, ranks by a scan of the flags, slots and distinct rows from the ranks
+            const int cur = radix_sort_pairs_tail(ga.keys[0], ga.keys[1], ga.vals[0], ga.vals[1], n64, ga.key_bits,
+                                                  ga.hist, status, ga.max_polls);
+            const int32_t* sk = ga.keys[cur];
+            const int32_t* sv = ga.vals[cur];
+            int64_t grid = (n64 + kThreads - 1) / kThreads;
+            grid = grid < 2048 ? grid : 2048;
+            k_cold_heads<<<(unsigned)grid, kThreads, 0, cudaStreamTailLaunch>>>(sk, n64, ga.rank);
+            exclusive_scan_i32_tail(ga.rank, ga.rank, n64, ga.tiles, status, ga.max_polls);
+            k_cold_assign<<<(unsigned)grid, kThreads, 0, cudaStreamTailLaunch>>>(
+                sk, sv, n64, ga.rank, slot0, staging_cap, ids, cold_rows, d_n_cold, status, ga.cap_ids);
+            if (cudaGetLastError() != cudaSuccess) set_status(status, HL_ECUDA);
+        }
         return;
     }
     if (cta == 0 && threadIdx.x == 0) d_n_general[0] = 0;
@@ -298,7 +320,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_cold_small(const int32_t* __r
 // group.  Rows i with skip[i] >= 0 are left alone.
 template <int G, bool TO_TABLE>
 __global__ void __launch_bounds__(kThreads) k_move_rows(float* __restrict__ dense_side, int64_t dense_row0,
-                                                        float* __restrict__ table, const int32_t* __restrict__ rows,
+                                                        TableMap table, const int32_t* __restrict__ rows,
                                                         const int64_t* __restrict__ d_n, int64_t n_max,
                                                         int64_t table_rows, int D4,
                                                         const int32_t* __restrict__ skip, int32_t* status) {
@@ -309,27 +331,27 @@ __global__ void __launch_bounds__(kThreads) k_move_rows(float* __restrict__ dens
     const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
     const int64_t n_groups = (int64_t)gridDim.x * kThreads / G;
     float4* dense4 = reinterpret_cast<float4*>(dense_side) + dense_row0 * D4;
-    float4* table4 = reinterpret_cast<float4*>(table);
     for (int64_t i0 = group * UR; i0 < n; i0 += n_groups * UR) {
-        int64_t g[UR];
+        float4* trow[UR];              // the row in the host table, nullptr = nothing to move
 #pragma unroll
         for (int u = 0; u < UR; ++u) {
-            g[u] = i0 + u < n ? (int64_t)rows[i0 + u] : -1;
-            if (skip != nullptr && g[u] >= 0 && skip[i0 + u] >= 0) g[u] = -1;   // row comes from elsewhere
-            if (g[u] >= table_rows) {
+            int64_t g = i0 + u < n ? (int64_t)rows[i0 + u] : -1;
+            if (skip != nullptr && g >= 0 && skip[i0 + u] >= 0) g = -1;   // row comes from elsewhere
+            if (g >= table_rows) {
                 set_status(status, HL_EBOUNDS);
-                g[u] = -1;
+                g = -1;
             }
+            trow[u] = g >= 0 ? reinterpret_cast<float4*>(row_address(table, g, D4 * 16)) : nullptr;
         }
         for (int c = sub; c < D4; c += G) {
             float4 v[UR];
 #pragma unroll
             for (int u = 0; u < UR; ++u)
-                if (g[u] >= 0) v[u] = TO_TABLE ? dense4[(i0 + u) * D4 + c] : table4[g[u] * D4 + c];
+                if (trow[u]) v[u] = TO_TABLE ? dense4[(i0 + u) * D4 + c] : trow[u][c];
 #pragma unroll
             for (int u = 0; u < UR; ++u)
-                if (g[u] >= 0) {
-                    if (TO_TABLE) table4[g[u] * D4 + c] = v[u];
+                if (trow[u]) {
+                    if (TO_TABLE) trow[u][c] = v[u];
                     else dense4[(i0 + u) * D4 + c] = v[u];
                 }
         }
@@ -417,7 +439,7 @@ struct MoveCfg {
 };
 
 template <bool TO_TABLE>
-__global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_side, int64_t dense_row0, float* table,
+__global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_side, int64_t dense_row0, TableMap table,
                                                                  const int32_t* __restrict__ rows,
                                                                  const int64_t* __restrict__ d_n, int64_t n_max,
                                                                  int64_t table_rows, int row_bytes,
@@ -441,7 +463,6 @@ __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_si
     }
     __syncthreads();
     unsigned char* dense = reinterpret_cast<unsigned char*>(dense_side) + dense_row0 * row_bytes;
-    unsigned char* tab = reinterpret_cast<unsigned char*>(table);
     const int64_t n_batches = (n + rows_per_stage - 1) / rows_per_stage;
     // The launch has as many CTAs as the largest transfer could use; how many of them work is decided here, from the
     // number of rows there really are: min_ctas for a mini-batch's worth of a DLRM-sized model (more would only slow
@@ -481,7 +502,7 @@ __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_si
             const int64_t g = rows[i0 + r];
             const bool ok = g >= 0 && g < table_rows && !(skip != nullptr && skip[i0 + r] >= 0);
             if (!ok) continue;
-            const unsigned char* src = TO_TABLE ? dense + (i0 + r) * row_bytes : tab + g * row_bytes;
+            const unsigned char* src = TO_TABLE ? dense + (i0 + r) * row_bytes : row_address(table, g, row_bytes);
             bulk_load(&stage[s][r * row_bytes], src, (uint32_t)row_bytes, &mbar[s]);
         }
         // wait for the stage to fill (bounded)
@@ -507,7 +528,7 @@ __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_si
             const int64_t g = rows[i0 + r];
             const bool ok = g >= 0 && g < table_rows && !(skip != nullptr && skip[i0 + r] >= 0);
             if (!ok) continue;
-            unsigned char* dst = TO_TABLE ? tab + g * row_bytes : dense + (i0 + r) * row_bytes;
+            unsigned char* dst = TO_TABLE ? row_address(table, g, row_bytes) : dense + (i0 + r) * row_bytes;
             bulk_store(dst, &stage[s][r * row_bytes], (uint32_t)row_bytes);
         }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -521,7 +542,7 @@ __global__ void __launch_bounds__(kBulkThreads) k_move_rows_bulk(float* dense_si
 }
 
 template <bool TO_TABLE>
-int32_t launch_move_rows(float* dense_side, int64_t dense_row0, float* table, const int32_t* rows,
+int32_t launch_move_rows(float* dense_side, int64_t dense_row0, TableMap table, const int32_t* rows,
                          const int64_t* d_n, int64_t n_max, int64_t table_rows, int D, const int32_t* skip,
                          MoveCfg cfg, int32_t* status, cudaStream_t stream) {
     if (n_max <= 0) return HL_OK;
@@ -565,6 +586,17 @@ int bits_for(int64_t max_value) {
 
 }  // namespace
 
+// the host table as the movers see it: `host_table` itself, or the per-table allocations installed by
+// hl_set_host_tables (then `host_table` only says that there is a table)
+static TableMap table_map(const hl_ctx* ctx, const float* host_table) {
+    TableMap m;
+    m.single = reinterpret_cast<unsigned char*>(const_cast<float*>(host_table));
+    m.ptrs = ctx->per_table ? ctx->r.table_ptrs : nullptr;
+    m.base = ctx->r.table_base;
+    m.T = ctx->T;
+    return m;
+}
+
 // how the movers of this context are launched: inside a schedule (`width` = the context's setting) or alone on the
 // chip (`width` = 0: two CTAs per SM, the link's full rate)
 static MoveCfg move_cfg(const hl_ctx* ctx, int width) {
@@ -579,7 +611,7 @@ static MoveCfg move_cfg(const hl_ctx* ctx, int width) {
 int32_t launch_gather_rows(hl_ctx* ctx, float* dst, int64_t dst_row0, const float* table, const int32_t* rows,
                            const int64_t* d_n, int64_t n_max, int32_t* status, cudaStream_t stream) {
     // loading the hot cache happens with nothing else on the chip: two mover CTAs per SM, for the link's full rate
-    return launch_move_rows<false>(dst, dst_row0, const_cast<float*>(table), rows, d_n, n_max, ctx->N, ctx->D, nullptr,
+    return launch_move_rows<false>(dst, dst_row0, table_map(ctx, table), rows, d_n, n_max, ctx->N, ctx->D, nullptr,
                                    move_cfg(ctx, 0), status, stream);
 }
 
@@ -592,8 +624,8 @@ namespace {
 
 // Shared body of hl_gather_cold and hl_gather_cold_ahead.  Staging window: cache slots
 // [hot_cap + stage_row0, hot_cap + stage_row0 + stage_rows).
-// First half of the cold-row search: classify X's lookups and let the one-cluster kernel try; it leaves its verdict in
-// cold_n[1] (0: done; else the number of cold lookups, for the general path).
+// First half of the cold-row search: classify X's lookups, then the one-cluster kernel, which either finishes the
+// search or launches the general path behind itself; cold_n[1] says which (0, or the number of cold lookups).
 int32_t index_begin(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, int64_t stage_row0, int64_t stage_rows,
                     int32_t* d_cold_rows, int64_t* d_n_cold, cudaStream_t stream) {
     Regions& r = ctx->r;
@@ -604,14 +636,24 @@ int32_t index_begin(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, int64_t
     }
     if (!non->ids) return HL_EINVAL;
     HL_CUDA_TRY(cudaMemsetAsync(r.cold_n, 0, 4 * sizeof(int32_t), stream));
-    const int grid = grid_for(ctx->max_nnz, kThreads, kMaxGrid);
+    const int grid = grid_for(ctx->max_nnz, kThreads, 4 * ctx_sms(ctx));
     k_cold_classify<<<grid, kThreads, 0, stream>>>(non->ids, non->offsets, d_n_non, ctx->max_batch, ctx->T * ctx->S,
                                                    non->cap_ids, ctx->N, r.remap, r.cold_keys[0], r.cold_vals[0],
                                                    r.cold_n, ctx->max_nnz, r.status);
     note_launches(1);
     HL_LAUNCH_CHECK();
-    // up to kSmallCap cold lookups: one cluster; more: the general path, whose count (cold_n[1]) that kernel sets
     const int key_bits = bits_for(ctx->N - 1);
+    GeneralArgs ga;
+    for (int i = 0; i < 2; ++i) {
+        ga.keys[i] = r.cold_keys[i];
+        ga.vals[i] = r.cold_vals[i];
+    }
+    ga.hist = r.cold_hist;
+    ga.rank = r.cold_rank;
+    ga.tiles = r.cold_tiles;
+    ga.cap_ids = non->cap_ids;
+    ga.key_bits = key_bits;
+    ga.max_polls = wait_cfg(ctx).max_polls;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kSmallCtas);
     cfg.blockDim = dim3(kSmallThreads);
@@ -626,41 +668,19 @@ int32_t index_begin(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, int64_t
     HL_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_cold_small, (const int32_t*)r.cold_keys[0], (const int32_t*)r.cold_vals[0],
                                    (const int32_t*)r.cold_n, ctx->max_nnz, (key_bits + 7) / 8,
                                    ctx->hot_cap + stage_row0, stage_rows, non->ids, d_cold_rows, d_n_cold,
-                                   r.cold_n + 1, r.status));
+                                   r.cold_n + 1, r.status, ga));
     note_launches(1);
     HL_LAUNCH_CHECK();
     return HL_OK;
 }
 
-// Second half: the general path (its kernels find nothing to do when the verdict is 0; `general_not_needed` = the
-// caller has read that verdict and spares the launches), then the match against the previous mini-batch's cold rows.
-int32_t index_end(hl_ctx* ctx, hl_ubatch* non, int64_t stage_row0, int64_t stage_rows, int32_t* d_cold_rows,
-                  int64_t* d_n_cold, const int32_t* d_prev_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
-                  bool general_not_needed, cudaStream_t stream) {
-    Regions& r = ctx->r;
+// Second half: the match against the previous mini-batch's cold rows.  (Whatever the search needed beyond its
+// one-cluster kernel was launched by that kernel and has run by the time anything queued here starts.)
+int32_t index_end(hl_ctx* ctx, int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold,
+                  const int32_t* d_prev_rows, const int64_t* d_n_prev, int32_t* d_fwd_src, cudaStream_t stream) {
     if (ctx->max_nnz == 0) return HL_OK;
-    const int grid = grid_for(ctx->max_nnz, kThreads, kMaxGrid);
-    const int key_bits = bits_for(ctx->N - 1);
-    int32_t st = HL_OK;
-    if (ctx->max_nnz > kSmallCap && !general_not_needed) {
-        int32_t *keys, *vals;
-        st = radix_sort_pairs(r.cold_keys, r.cold_vals, r.cold_n + 1, ctx->max_nnz, key_bits, r.cold_hist, r.status,
-                              &keys, &vals, stream, wait_cfg(ctx));
-        if (st != HL_OK) return st;
-        k_cold_heads<<<grid, kThreads, 0, stream>>>(keys, r.cold_n + 1, ctx->max_nnz, r.cold_rank);
-        note_launches(1);
-        HL_LAUNCH_CHECK();
-        st = exclusive_scan_i32(r.cold_rank, r.cold_rank, r.cold_n + 1, ctx->max_nnz, r.cold_tiles, r.status, stream,
-                                wait_cfg(ctx));
-        if (st != HL_OK) return st;
-        k_cold_assign<<<grid, kThreads, 0, stream>>>(keys, vals, r.cold_n + 1, ctx->max_nnz, r.cold_rank,
-                                                     ctx->hot_cap + stage_row0, stage_rows, non->ids, d_cold_rows,
-                                                     d_n_cold, r.status, r.cold_n, non->cap_ids);
-        note_launches(1);
-        HL_LAUNCH_CHECK();
-    }
     if (d_prev_rows) {
-        k_cold_match<<<grid_for(stage_rows, kThreads, kMaxGrid), kThreads, 0, stream>>>(
+        k_cold_match<<<grid_for(stage_rows, kThreads, 2 * ctx_sms(ctx)), kThreads, 0, stream>>>(
             d_cold_rows, d_n_cold, stage_rows, d_prev_rows, d_n_prev, ctx->staging_cap, d_fwd_src);
         note_launches(1);
         HL_LAUNCH_CHECK();
@@ -678,7 +698,7 @@ int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const f
         if (ctx->max_nnz == 0) return HL_OK;
         timer_mark(ctx, HL_TIMER_GATHER_MOVE, 0, stream);
         const int32_t st = launch_move_rows<false>(d_cache, ctx->hot_cap + stage_row0,
-                                                   const_cast<float*>(host_table), d_cold_rows, d_n_cold, stage_rows,
+                                                   table_map(ctx, host_table), d_cold_rows, d_n_cold, stage_rows,
                                                    ctx->N, ctx->D, d_fwd_src, move_cfg(ctx, ctx->mover_ctas), r.status,
                                                    stream);
         timer_mark(ctx, HL_TIMER_GATHER_MOVE, 1, stream);
@@ -686,15 +706,14 @@ int32_t gather_impl(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, const f
     }
     int32_t st = index_begin(ctx, non, d_n_non, stage_row0, stage_rows, d_cold_rows, d_n_cold, stream);
     if (st != HL_OK) return st;
-    st = index_end(ctx, non, stage_row0, stage_rows, d_cold_rows, d_n_cold, d_prev_rows, d_n_prev, d_fwd_src, false,
-                   stream);
+    st = index_end(ctx, stage_rows, d_cold_rows, d_n_cold, d_prev_rows, d_n_prev, d_fwd_src, stream);
     if (st != HL_OK) return st;
     if (record_after_index) HL_CUDA_TRY(cudaEventRecord(record_after_index, stream));
     if (!do_move) return HL_OK;
     if (wait_a) HL_CUDA_TRY(cudaStreamWaitEvent(stream, wait_a, 0));
     if (wait_b) HL_CUDA_TRY(cudaStreamWaitEvent(stream, wait_b, 0));
     timer_mark(ctx, HL_TIMER_GATHER_MOVE, 0, stream);
-    st = launch_move_rows<false>(d_cache, ctx->hot_cap + stage_row0, const_cast<float*>(host_table), d_cold_rows,
+    st = launch_move_rows<false>(d_cache, ctx->hot_cap + stage_row0, table_map(ctx, host_table), d_cold_rows,
                                  d_n_cold, stage_rows, ctx->N, ctx->D, d_prev_rows ? d_fwd_src : nullptr,
                                  move_cfg(ctx, ctx->mover_ctas), r.status, stream);
     timer_mark(ctx, HL_TIMER_GATHER_MOVE, 1, stream);
@@ -760,8 +779,9 @@ extern "C" int32_t hl_index_cold_end(hl_ctx* ctx, hl_ubatch* non, int64_t stage_
     if (!ctx || !non || !d_cold_rows || !d_n_cold) return HL_EINVAL;
     if (!window_ok(ctx, stage_row0, stage_rows)) return HL_EINVAL;
     if ((d_prev_cold_rows != nullptr) != (d_n_prev != nullptr) || (d_prev_cold_rows && !d_fwd_src)) return HL_EINVAL;
-    return index_end(ctx, non, stage_row0, stage_rows, d_cold_rows, d_n_cold, d_prev_cold_rows, d_n_prev, d_fwd_src,
-                     general_not_needed != 0, static_cast<cudaStream_t>(stream_));
+    (void)general_not_needed;
+    return index_end(ctx, stage_rows, d_cold_rows, d_n_cold, d_prev_cold_rows, d_n_prev, d_fwd_src,
+                     static_cast<cudaStream_t>(stream_));
 }
 
 extern "C" int32_t hl_stage_cold(hl_ctx* ctx, const float* host_table, float* d_cache, int64_t stage_row0,
@@ -801,7 +821,8 @@ extern "C" int32_t hl_scatter_cold_at(hl_ctx* ctx, const float* d_cache, int64_t
     if (!window_ok(ctx, stage_row0, stage_rows)) return HL_EINVAL;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 0, stream);
-    const int32_t st = launch_move_rows<true>(const_cast<float*>(d_cache), ctx->hot_cap + stage_row0, host_table,
+    const int32_t st = launch_move_rows<true>(const_cast<float*>(d_cache), ctx->hot_cap + stage_row0,
+                                              table_map(ctx, host_table),
                                               d_cold_rows, d_n_cold, stage_rows, ctx->N, ctx->D, nullptr,
                                               move_cfg(ctx, ctx->scatter_ctas), ctx->r.status, stream);
     timer_mark(ctx, HL_TIMER_SCATTER_MOVE, 1, stream);
@@ -818,6 +839,7 @@ extern "C" int32_t hl_flush_hot(hl_ctx* ctx, const float* d_cache, const int32_t
                                 float* host_table, void* stream_) {
     if (!ctx || !d_cache || !d_hot_rows || !d_n_hot || !host_table) return HL_EINVAL;
     // runs between learning phases, with nothing else on the chip: the mover at the link's full rate
-    return launch_move_rows<true>(const_cast<float*>(d_cache), 0, host_table, d_hot_rows, d_n_hot, ctx->hot_cap, ctx->N,
+    return launch_move_rows<true>(const_cast<float*>(d_cache), 0, table_map(ctx, host_table), d_hot_rows, d_n_hot,
+                                  ctx->hot_cap, ctx->N,
                                   ctx->D, nullptr, move_cfg(ctx, 0), ctx->r.status, static_cast<cudaStream_t>(stream_));
 }

@@ -43,6 +43,7 @@ struct Regions {
     // common
     int32_t* status;                   // [8]  status[0] = first device error
     int64_t* table_base;               // [T+1]
+    unsigned char** table_ptrs;        // [T] host-memory base of every table (hl_set_host_tables), device copy
     RemapBlock* remap;                 // [n_remap_blocks]
     // profile
     uint32_t* counts;                  // [N]
@@ -80,9 +81,11 @@ struct hl_ctx {
     int device;
     int sms;                           // multiprocessors of `device` (queried at hl_create)
     int mover_ctas, scatter_ctas;      // working CTAs of the host-link movers inside a schedule (hl_set_mover_ctas)
+    int fwd_ctas, bwd_ctas;            // CTAs per multiprocessor of the forward / backward-sum kernel (0 = default)
     int test_poll_limit;               // > 0: poll limit of the bounded device waits (hl_test_bounded_waits)
     int64_t test_stall_tile;           // with it: the tile / mover stage that never delivers (-1: none)
     int64_t* h_table_base;             // host copy [T+1]
+    int per_table;                     // 1: the host table is one allocation per table (r.table_ptrs is set)
     hl::Regions r;
     int timing_on;                     // optional kernel timers (hl_timing_enable)
     cudaEvent_t timer[HL_TIMER_COUNT][2];
@@ -111,6 +114,9 @@ inline void timer_mark(hl_ctx* ctx, int which, int end, cudaStream_t stream) {
 }
 
 inline int ctx_sms(const hl_ctx* ctx) { return ctx->sms > 0 ? ctx->sms : kSMsFallback; }
+// CTAs per multiprocessor of the two bandwidth-bound kernels (hl_set_kernel_width; defaults chosen by measurement)
+inline int fwd_ctas_per_sm(const hl_ctx* ctx) { return ctx->fwd_ctas > 0 ? ctx->fwd_ctas : 3; }
+inline int bwd_ctas_per_sm(const hl_ctx* ctx) { return ctx->bwd_ctas > 0 ? ctx->bwd_ctas : 3; }
 
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) {
     atomicCAS(status, 0, code);
@@ -142,6 +148,27 @@ __device__ __forceinline__ int32_t remap_slot(const RemapBlock* __restrict__ rem
     if (!((word >> bit) & 1u)) return -1;
     slot += __popc(word & ((1u << bit) - 1u));
     return (int32_t)slot;
+}
+
+// Where the host-DRAM table's rows are: one allocation holding all tables back to back (ptrs == nullptr: row g at
+// single + g * row_bytes), or one allocation per table (the address registers of the paper's Data Dispatcher,
+// Section V-A): row g of table t at ptrs[t] + (g - base[t]) * row_bytes.
+struct TableMap {
+    unsigned char* single;
+    unsigned char* const* ptrs;
+    const int64_t* base;               // [T+1]
+    int T;
+};
+
+__device__ __forceinline__ unsigned char* row_address(const TableMap& m, int64_t g, int row_bytes) {
+    if (m.ptrs == nullptr) return m.single + g * row_bytes;
+    int lo = 0, hi = m.T;              // base[lo] <= g < base[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(&m.base[mid]) <= g) lo = mid;
+        else hi = mid;
+    }
+    return m.ptrs[lo] + (g - __ldg(&m.base[lo])) * row_bytes;
 }
 
 __device__ __forceinline__ unsigned lanemask_lt() {
@@ -178,6 +205,13 @@ int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, 
 int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n, int64_t n_max, int key_bits,
                          uint32_t* hist, int32_t* status, int32_t** out_keys, int32_t** out_vals,
                          cudaStream_t stream, WaitCfg w = WaitCfg());
+
+// The same from the device (one thread calls; the launches run after the calling grid, in order: see hl_prims.cu).
+// radix_sort_pairs_tail returns which buffer (0 / 1) will hold the result.
+__device__ int radix_sort_pairs_tail(int32_t* keys0, int32_t* keys1, int32_t* vals0, int32_t* vals1, int64_t n,
+                                     int key_bits, uint32_t* hist, int32_t* status, int max_polls);
+__device__ void exclusive_scan_i32_tail(const int32_t* in, int32_t* out, int64_t n, int32_t* tiles, int32_t* status,
+                                        int max_polls);
 
 // 32-bit words of histogram scratch radix_sort_pairs needs for at most max_nnz pairs.
 constexpr int64_t sort_hist_words(int64_t max_nnz) {

@@ -9,7 +9,6 @@ namespace hl {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kFwdTrips = 4;   // trips of the forward kernel per CTA
 
 __device__ __forceinline__ float4 f4_zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
 
@@ -97,11 +96,18 @@ __global__ void __launch_bounds__(kThreads) k_embbag_fwd(const float* __restrict
         for (int u = 0; u < UB; ++u) id1[u] = len[u] == 1 ? __ldg(&ids[lo[u]]) : -1;
     };
 
-    // this CTA's tile: kFwdTrips consecutive trips of (groups per CTA) x UB bags
+    // This CTA's share: the bags are dealt out in trips of (groups per CTA) x UB consecutive bags, every CTA gets a
+    // contiguous run of trips, and the counts differ by at most one trip -- the grid is a fixed number of CTAs per
+    // multiprocessor, whatever the number of bags.
     constexpr int kGroups = kThreads / G;
     int32_t lo[UB], len[UB], id1[UB];
-    const int64_t tile0 = (int64_t)blockIdx.x * kFwdTrips * kGroups * UB;
-    const int64_t tile_end = min(n_bags, tile0 + (int64_t)kFwdTrips * kGroups * UB);
+    const int64_t trip_bags = (int64_t)kGroups * UB;
+    const int64_t trips_all = (n_bags + trip_bags - 1) / trip_bags;
+    const int64_t q = trips_all / gridDim.x, rem = trips_all % gridDim.x;
+    const int64_t my_first = (int64_t)blockIdx.x * q + min((int64_t)blockIdx.x, rem);
+    const int64_t my_trips = q + ((int64_t)blockIdx.x < rem ? 1 : 0);
+    const int64_t tile0 = my_first * trip_bags;
+    const int64_t tile_end = min(n_bags, tile0 + my_trips * trip_bags);
     int64_t bag0 = tile0 + (int64_t)(threadIdx.x / G) * UB;
     if (bag0 < tile_end) load_index(bag0, lo, len, id1);
     for (; bag0 < tile_end; bag0 += kGroups * UB) {
@@ -510,8 +516,8 @@ template <int G, int NV>
 int32_t launch_fwd(hl_ctx* ctx, const float* cache, const hl_ubatch* ub, const int32_t* d_n, float* out,
                    cudaStream_t stream) {
     constexpr int UB = NV >= 4 ? 1 : (NV >= 2 ? 2 : 4);
-    const int64_t bags_per_cta = (int64_t)kFwdTrips * (kThreads / G) * UB;
-    const int grid = grid_for(ctx->max_bags, (int)bags_per_cta, kMaxGrid);
+    const int64_t bags_per_trip = (int64_t)(kThreads / G) * UB;
+    const int grid = grid_for(ctx->max_bags, (int)bags_per_trip, fwd_ctas_per_sm(ctx) * ctx_sms(ctx));
     timer_mark(ctx, HL_TIMER_FWD, 0, stream);
     k_embbag_fwd<G, NV, UB><<<grid, kThreads, 0, stream>>>(cache, ub->ids, ub->offsets, d_n, ctx->max_batch,
                                                           ctx->T * ctx->S, ctx->D / 4,
@@ -527,7 +533,9 @@ int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t
                    const float* grad, float lr, cudaStream_t stream, const int32_t* d_first = nullptr,
                    int32_t key_bias = 0) {
     const int64_t max_chunks = div_up(ctx->max_nnz, kBwdChunk);
-    const int grid = grid_for(max_chunks * G, kThreads, kMaxGrid);
+    // a fixed number of CTAs per multiprocessor (the groups stride over the chunks), so that kernels of other
+    // streams find room beside this one
+    const int grid = grid_for(max_chunks * G, kThreads, bwd_ctas_per_sm(ctx) * ctx_sms(ctx));
     const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 0, stream);
     // the list of chunks whose run goes on sits behind the partial sums: [count (8 ints)] [chunk ids]
@@ -538,7 +546,7 @@ int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t
                                                       lr, ctx->r.bwd_part, d_first, key_bias, span_count, span_list,
                                                       ctx->max_bags);
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 1, stream);
-    const int span_grid = grid_for(max_chunks * 32, kThreads, kMaxGrid);   // one warp per chunk
+    const int span_grid = grid_for(max_chunks * 32, kThreads, 4 * ctx_sms(ctx));   // the warps stride over the listed runs
     k_bwd_spans<G, NV><<<span_grid, kThreads, 0, stream>>>(cache, keys, d_n_lookups, ctx->D / 4, n_slots, lr,
                                                           ctx->r.bwd_part, d_first, key_bias, span_count, span_list);
     note_launches(2);
@@ -600,11 +608,11 @@ int32_t sort_lookups(hl_ctx* ctx, const hl_ubatch* ub, const int32_t* d_n_sample
     }
     const bool short_bags = ctx->max_nnz <= 4 * ctx->max_bags;
     if (short_bags)
-        k_bwd_pairs<1><<<grid_for(ctx->max_bags, kThreads, kMaxGrid), kThreads, 0, stream>>>(
+        k_bwd_pairs<1><<<grid_for(ctx->max_bags, kThreads, 4 * ctx_sms(ctx)), kThreads, 0, stream>>>(
             ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, keys[0], vals[0],
             d_n_lookups, nullptr, 0, (int32_t)n_slots, nullptr, r.status);
     else
-        k_bwd_pairs<32><<<grid_for(ctx->max_bags, kThreads / 32, kMaxGrid), kThreads, 0, stream>>>(
+        k_bwd_pairs<32><<<grid_for(ctx->max_bags, kThreads / 32, 8 * ctx_sms(ctx)), kThreads, 0, stream>>>(
             ub->ids, ub->offsets, d_n_samples, ctx->max_batch, ctx->T * ctx->S, n_slots, ctx->max_nnz, keys[0], vals[0],
             d_n_lookups, nullptr, 0, (int32_t)n_slots, nullptr, r.status);
     note_launches(1);
@@ -670,7 +678,7 @@ static int32_t prepare_both(hl_ctx* ctx, const hl_ubatch* pop, const int32_t* d_
     vals[passes & 1] = d_sorted_bags;
     const bool short_bags = ctx->max_nnz <= 4 * ctx->max_bags;
     const int per_block = short_bags ? kThreads : kThreads / 32;
-    const int grid = grid_for(ctx->max_bags, per_block, kMaxGrid);
+    const int grid = grid_for(ctx->max_bags, per_block, (short_bags ? 4 : 8) * ctx_sms(ctx));
     const hl_ubatch* ubs[2] = {pop, non};
     const int32_t* ns[2] = {d_n_pop, d_n_non};
     for (int m = 0; m < 2; ++m) {

@@ -241,7 +241,8 @@ extern "C" int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_de
     const int64_t n_bags = (int64_t)T * B * S;
     const bool short_bags = b->nnz <= 4 * (int64_t)T * B;   // on average at most 4 lookups per input and table
 
-    const int flag_grid = grid_for(B, kThreads / 32, kMaxGrid);
+    const int cap = 4 * ctx_sms(ctx);      // CTAs of every kernel here: they stride over their work
+    const int flag_grid = grid_for(B, kThreads / 32, 2 * cap);
     if (short_bags)
         k_frag_flags<true><<<flag_grid, kThreads, 0, stream>>>(b->indices, b->offsets, B, T, S, r.table_base,
                                                                r.remap, r.frag_flags, r.status);
@@ -249,7 +250,7 @@ extern "C" int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_de
         k_frag_flags<false><<<flag_grid, kThreads, 0, stream>>>(b->indices, b->offsets, B, T, S, r.table_base,
                                                                 r.remap, r.frag_flags, r.status);
     k_frag_partition<<<1, 1024, 0, stream>>>(r.frag_flags, B, d_perm, d_counts);
-    k_frag_sizes<<<grid_for(n_bags, kThreads, kMaxGrid), kThreads, 0, stream>>>(b->offsets, B, T, S, d_perm,
+    k_frag_sizes<<<grid_for(n_bags, kThreads, cap), kThreads, 0, stream>>>(b->offsets, B, T, S, d_perm,
                                                                                d_counts, r.frag_scan);
     note_launches(3);   // flags, partition, sizes
     HL_LAUNCH_CHECK();
@@ -257,15 +258,15 @@ extern "C" int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_de
                                     wait_cfg(ctx));
     if (st != HL_OK) return st;
     if (b->nnz <= 4 * n_bags)
-        k_frag_emit<1><<<grid_for(n_bags, kThreads, kMaxGrid), kThreads, 0, stream>>>(
+        k_frag_emit<1><<<grid_for(n_bags, kThreads, cap), kThreads, 0, stream>>>(
             b->indices, b->offsets, B, T, S, d_perm, d_counts, r.frag_scan, r.table_base, r.remap, pop->offsets,
             pop->ids, pop->cap_ids, non->offsets, non->ids, non->cap_ids, r.status);
     else
-        k_frag_emit<32><<<grid_for(n_bags, kThreads / 32, kMaxGrid), kThreads, 0, stream>>>(
+        k_frag_emit<32><<<grid_for(n_bags, kThreads / 32, 2 * cap), kThreads, 0, stream>>>(
             b->indices, b->offsets, B, T, S, d_perm, d_counts, r.frag_scan, r.table_base, r.remap, pop->offsets,
             pop->ids, pop->cap_ids, non->offsets, non->ids, non->cap_ids, r.status);
     if (d_dense)
-        k_permute_dense<<<grid_for((int64_t)B * n_dense, kThreads, kMaxGrid), kThreads, 0, stream>>>(
+        k_permute_dense<<<grid_for((int64_t)B * n_dense, kThreads, cap), kThreads, 0, stream>>>(
             d_dense, B, n_dense, d_perm, d_dense_out);
     note_launches(d_dense ? 2 : 1);   // emit (+ dense permutation)
     HL_LAUNCH_CHECK();

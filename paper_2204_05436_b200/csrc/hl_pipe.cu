@@ -25,14 +25,14 @@ struct hl_pipe {
     std::vector<hl_pipe_set> sets;
     cudaStream_t main, sa, sb, sc, link, wb;
     struct Events {
-        cudaEvent_t inputs, frag, index, prep, gather, forward, x, scatter, verdict;
+        cudaEvent_t inputs, frag, index, prep, gather, forward, x, scatter;
     };
     std::vector<Events> ev;
     // mini-batches whose fragment + first half of the cold-row search are queued (begun), whose cold-row search and
     // sort are queued in full (indexed), whose host read is queued (submitted), whose main work is queued (done)
     int64_t j_begun, j_indexed, j_submitted, j_done;
-    int32_t* h_verdict;          // pinned host words, one per set: what the first half of the cold-row search found
     int order;                   // HL_PIPE_ORDER_*
+    int exclusive_wb;            // main work of j waits for the write-back of j - 1
     // trace (hl_pipe_trace_begin / _end): one event pair per recorded span
     struct Span {
         cudaEvent_t b, e;
@@ -105,13 +105,8 @@ struct Scope {
     ~Scope() { span_close(p, idx); }
 };
 
-// Second half of the index-only work of the mini-batch begun last: the rest of the cold-row search and the backward
-// sort.  It is queued one call later than the first half whenever the schedule has that slack, because by then the
-// host can usually see (without waiting) that the one-cluster kernel has found the distinct rows itself, and the ten
-// launches of the general path need not be queued at all; if that is not known yet they are queued and decide on
-// the device.  (With steps issued back to back, as in the benchmark, the verdict of a mini-batch begun one step ago
-// is usually still on its way -- the chain of fragment and search kernels takes about as long as a step --, so the
-// saving shows when there is other work between the steps, as in training.)
+// Second half of the index-only work of the mini-batch begun last: the match of its cold rows against the mini-batch
+// before (stream C, in order behind that mini-batch's search) and the backward sort (stream B).
 int32_t finish_index(hl_pipe* p) {
     if (p->j_indexed == p->j_begun) return HL_OK;
     const int64_t j = p->j_indexed;
@@ -120,12 +115,11 @@ int32_t finish_index(hl_pipe* p) {
     hl_pipe::Events& e = p->ev[j % n];
     hl_pipe_set* prev = j >= 1 ? &p->sets[(j - 1) % n] : nullptr;
     const int64_t w = (j % 2) * p->window_rows;
-    const bool known_done = cudaEventQuery(e.verdict) == cudaSuccess && p->h_verdict[j % n] == 0;
     {
         Scope sc(p, HL_SPAN_INDEX_END, j, kStreamC);
         HL_PIPE_TRY(hl_index_cold_end(p->ctx, &st.non, w, p->window_rows, st.cold_rows, st.n_cold,
-                                  prev ? prev->cold_rows : nullptr, prev ? prev->n_cold : nullptr, st.fwd_src,
-                                  known_done ? 1 : 0, p->sc));
+                                      prev ? prev->cold_rows : nullptr, prev ? prev->n_cold : nullptr, st.fwd_src, 0,
+                                      p->sc));
     }
     HL_PIPE_TRY(record(e.index, p->sc));
     HL_PIPE_TRY(wait(p->sb, e.index));
@@ -145,7 +139,7 @@ int32_t finish_index(hl_pipe* p) {
 
 // fragment and the first half of the cold-row search of the next mini-batch (index-only: nothing here touches a row)
 int32_t begin_index(hl_pipe* p, const hl_batch* b, const float* d_dense, void* inputs_ready) {
-    HL_PIPE_TRY(finish_index(p));        // stream C: the mini-batch before ends its search before this one begins
+    HL_PIPE_TRY(finish_index(p));        // (nothing pending in the usual order of calls)
     const int64_t j = p->j_begun;
     const int n = p->n_sets;
     hl_pipe_set& st = p->sets[j % n];
@@ -171,12 +165,8 @@ int32_t begin_index(hl_pipe* p, const hl_batch* b, const float* d_dense, void* i
         HL_PIPE_TRY(hl_index_cold_begin(p->ctx, &st.non, st.counts + 1, w, p->window_rows, st.cold_rows, st.n_cold,
                                         p->sc));
     }
-    if (cudaMemcpyAsync(p->h_verdict + (j % n), hl_index_cold_verdict(p->ctx), sizeof(int32_t), cudaMemcpyDeviceToHost,
-                        p->sc) != cudaSuccess)
-        return HL_ECUDA;
-    HL_PIPE_TRY(record(e.verdict, p->sc));
     p->j_begun += 1;
-    return HL_OK;
+    return finish_index(p);
 }
 
 // the host read of the oldest indexed mini-batch whose rows are not staged yet
@@ -224,8 +214,8 @@ extern "C" hl_pipe* hl_pipe_create_ex(hl_ctx* ctx, float* d_cache, float* host_t
     p->sets.assign(sets, sets + n_sets);
     p->main = static_cast<cudaStream_t>(main_stream);
     p->j_begun = p->j_indexed = p->j_submitted = p->j_done = 0;
-    p->h_verdict = nullptr;
     p->order = HL_PIPE_ORDER_FIG8;
+    p->exclusive_wb = opt ? opt->exclusive_write_back : 0;
     p->n_spans = 0;
     p->trace_mask = 0;
     p->cur_mb = 0;
@@ -244,20 +234,16 @@ extern "C" hl_pipe* hl_pipe_create_ex(hl_ctx* ctx, float* d_cache, float* host_t
     }
     p->ev.resize(n_sets);
     for (auto& e : p->ev) {
-        cudaEvent_t* all[9] = {&e.inputs, &e.frag,    &e.index, &e.prep,   &e.gather,
-                               &e.forward, &e.x,      &e.scatter, &e.verdict};
+        cudaEvent_t* all[8] = {&e.inputs, &e.frag, &e.index, &e.prep, &e.gather, &e.forward, &e.x, &e.scatter};
         for (auto x : all) {
             *x = nullptr;
             ok = ok && cudaEventCreateWithFlags(x, cudaEventDisableTiming) == cudaSuccess;
         }
     }
-    ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&p->h_verdict), sizeof(int32_t) * n_sets, cudaHostAllocDefault) ==
-                   cudaSuccess;
     if (!ok) {
         hl_pipe_destroy(p);
         return nullptr;
     }
-    for (int i = 0; i < n_sets; ++i) p->h_verdict[i] = -1;
     return p;
 }
 
@@ -275,11 +261,10 @@ extern "C" void hl_pipe_destroy(hl_pipe* p) {
             cudaStreamDestroy(s);
         }
     for (auto& e : p->ev) {
-        cudaEvent_t all[9] = {e.inputs, e.frag, e.index, e.prep, e.gather, e.forward, e.x, e.scatter, e.verdict};
+        cudaEvent_t all[8] = {e.inputs, e.frag, e.index, e.prep, e.gather, e.forward, e.x, e.scatter};
         for (auto x : all)
             if (x) cudaEventDestroy(x);
     }
-    if (p->h_verdict) cudaFreeHost(p->h_verdict);
     if (p->ctx && p->ctx->mark_user == p) {
         p->ctx->mark_hook = nullptr;
         p->ctx->mark_user = nullptr;
@@ -314,6 +299,7 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
     const int64_t w0 = (j % 2) * p->window_rows, w1 = ((j + 1) % 2) * p->window_rows;
     if (next && p->j_begun - j >= n - 1) return HL_ECAPACITY;
     HL_PIPE_TRY(wait(p->main, e.index));
+    if (p->exclusive_wb && j >= 1) HL_PIPE_TRY(wait(p->main, p->ev[(j - 1) % n].scatter));
     if (j >= 1) {
         // rows shared with mini-batch j-1 come out of its staging window once its backward is done
         HL_PIPE_TRY(wait(p->link, e.index));
@@ -357,8 +343,7 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
                                        p->wb));
     }
     HL_PIPE_TRY(record(e.scatter, p->wb));
-    // The ahead-work comes last: the later the pending cold-row search is ended, the likelier its verdict is known.
-    HL_PIPE_TRY(finish_index(p));                                           // the mini-batch begun one step ago
+    HL_PIPE_TRY(finish_index(p));
     if (p->j_submitted == j + 1 && p->j_submitted < p->j_indexed) HL_PIPE_TRY(submit_link(p));   // mini-batch j+1
     if (next) {
         HL_PIPE_TRY(begin_index(p, next, d_next_dense, next_inputs_ready));

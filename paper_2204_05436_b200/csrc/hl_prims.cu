@@ -271,7 +271,55 @@ __global__ void __launch_bounds__(kThreads) k_sort_pass(const int32_t* __restric
     }
 }
 
+__global__ void __launch_bounds__(kThreads) k_zero_words(uint32_t* p, int64_t n) {
+    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n; i += (int64_t)gridDim.x * kThreads) p[i] = 0u;
+}
+
 }  // namespace
+
+// ---- the same two primitives, launched from the device --------------------------------------------------------
+// For a kernel that learns on the device that follow-up work is needed (the cold-row search beyond its one-cluster
+// path): ONE thread calls these; every launch goes to the tail-launch stream of the calling grid, i.e. runs after
+// that grid has finished, one launch after the other, before anything the host queued behind the grid.  n is known
+// here, so the grids are exact.  A launch the device runtime refuses sets HL_ECUDA in *status.
+__device__ static void tail_check(int32_t* status) {
+    if (cudaGetLastError() != cudaSuccess) set_status(status, HL_ECUDA);
+}
+
+__device__ int radix_sort_pairs_tail(int32_t* keys0, int32_t* keys1, int32_t* vals0, int32_t* vals1, int64_t n,
+                                     int key_bits, uint32_t* hist, int32_t* status, int max_polls) {
+    if (n <= 0) return 0;
+    const int64_t n_tiles = (n + kSortTile - 1) / kSortTile;
+    const int passes = (key_bits + 7) / 8;
+    uint32_t* ghist = hist;
+    uint32_t* ticket = hist + 4 * 256;
+    uint32_t* tstat = hist + 4 * 256 + 8;
+    const int64_t words = 4 * 256 + 8 + (int64_t)passes * n_tiles * 256;
+    int64_t zero_grid = (words + kThreads * 8 - 1) / (kThreads * 8);
+    k_zero_words<<<(unsigned)(zero_grid < 1024 ? zero_grid : 1024), kThreads, 0, cudaStreamTailLaunch>>>(hist, words);
+    int64_t hist_grid = (n + kThreads * 8 - 1) / (kThreads * 8);
+    k_sort_digit_hist<<<(unsigned)hist_grid, kThreads, 0, cudaStreamTailLaunch>>>(keys0, nullptr, n, passes, ghist);
+    int32_t* k[2] = {keys0, keys1};
+    int32_t* v[2] = {vals0, vals1};
+    int cur = 0;
+    for (int p = 0; p < passes; ++p) {
+        k_sort_pass<<<(unsigned)n_tiles, kThreads, 0, cudaStreamTailLaunch>>>(
+            k[cur], v[cur], k[cur ^ 1], v[cur ^ 1], nullptr, n, 8 * p, ghist + 256 * p, ticket + p,
+            tstat + (size_t)p * n_tiles * 256, status, max_polls, (int64_t)-1);
+        cur ^= 1;
+    }
+    tail_check(status);
+    return cur;
+}
+
+__device__ void exclusive_scan_i32_tail(const int32_t* in, int32_t* out, int64_t n, int32_t* tiles, int32_t* status,
+                                        int max_polls) {
+    const int64_t n_tiles = n / kScanTile + 1;
+    k_zero_words<<<1, kThreads, 0, cudaStreamTailLaunch>>>(reinterpret_cast<uint32_t*>(tiles), 2 * (n_tiles + 1));
+    k_scan_chained<<<(unsigned)n_tiles, kThreads, 0, cudaStreamTailLaunch>>>(
+        in, out, nullptr, n, reinterpret_cast<unsigned long long*>(tiles), status, max_polls, (int64_t)-1);
+    tail_check(status);
+}
 
 int32_t exclusive_scan_i32(const int32_t* in, int32_t* out, const int32_t* d_n, int64_t n_max, int32_t* tiles,
                            int32_t* status, cudaStream_t stream, WaitCfg w) {
@@ -303,7 +351,7 @@ int32_t radix_sort_pairs(int32_t* keys[2], int32_t* vals[2], const int32_t* d_n,
         uint32_t* tstat = hist + 4 * 256 + 8;
         HL_CUDA_TRY(cudaMemsetAsync(hist, 0, sizeof(uint32_t) * (4 * 256 + 8 + (size_t)passes * n_tiles * 256),
                                     stream));
-        k_sort_digit_hist<<<grid_for(n_max, kThreads * 8, kMaxGrid), kThreads, 0, stream>>>(keys[0], d_n, n_max,
+        k_sort_digit_hist<<<grid_for(n_max, kThreads * 8, 1024), kThreads, 0, stream>>>(keys[0], d_n, n_max,
                                                                                             passes, ghist);
         for (int p = 0; p < passes; ++p) {
             k_sort_pass<<<(unsigned)n_tiles, kThreads, 0, stream>>>(keys[cur], vals[cur], keys[cur ^ 1], vals[cur ^ 1],

@@ -31,10 +31,19 @@ class Hotline:
         self.hot_cap, self.staging_cap = int(hot_cap_rows), int(staging_cap_rows)
         self.max_bags = self.T * self.max_batch * self.S
         self.n_dense = int(n_dense)
-        if host_table.dtype != torch.float32 or tuple(host_table.shape) != (self.N, self.D):
+        # host_table: fp32 [N, D], or a list of one fp32 [rows_t, D] tensor per table (a table too large for one
+        # allocation).  It must be memory the device can address: from hl_host_alloc (binding.host_table_tensor),
+        # pinned host memory, or device memory.  (Not checked here: torch cannot tell for memory it did not allocate.)
+        self.host_tables = None
+        if isinstance(host_table, (list, tuple)):
+            self.host_tables = list(host_table)
+            if len(self.host_tables) != self.T or any(
+                    t.dtype != torch.float32 or tuple(t.shape) != (r, self.D)
+                    for t, r in zip(self.host_tables, self.table_rows)):
+                raise ValueError("host_table must be one fp32 [rows_t, D] tensor per table")
+            host_table = self.host_tables[0]     # only says "there is a host table" once the per-table bases are set
+        elif host_table.dtype != torch.float32 or tuple(host_table.shape) != (self.N, self.D):
             raise ValueError("host_table must be fp32 [N, D]")
-        # host_table must be memory the device can address: from hl_host_alloc (binding.host_table_tensor), pinned
-        # host memory, or device memory.  (Not checked here: torch cannot tell for memory it did not allocate.)
         self.host_table = host_table
 
         dev = self.device
@@ -68,6 +77,8 @@ class Hotline:
         self.ev_pop_done = torch.cuda.Event()
         self.ctx = B.hl_create(self.geom, self.max_batch, self.max_nnz, self.hot_cap, self.staging_cap,
                                self.workspace, self.ws_bytes)
+        if self.host_tables is not None:
+            B.hl_set_host_tables(self.ctx, self.host_tables)
 
     # ---- life cycle ------------------------------------------------------------------------------------------
     def close(self) -> None:
@@ -577,13 +588,14 @@ class NativePipelinedHotline(Hotline):
     def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
                  n_dense: int = 0, device: str = "cuda:0", lookahead: int = 2, order: str = "fig8",
                  main_priority: int = -1, index_priority: int = 0, link_priority: int = 0, mover_ctas: int = 0,
-                 scatter_ctas: int = 0):
+                 scatter_ctas: int = 0, exclusive_write_back: bool = False):
         """``order``: "fig8" = forward O, update O, forward X, update X (the paper's Fig. 8); "eq5" = both forwards,
         then one update of every touched row with the whole mini-batch's gradient (Eq. 5; the unfragmented step's
         result): step() then takes ``grad_pop`` = [gradients of O's bags; gradients of X's bags] and no ``grad_non``.
         ``main_priority`` / ``index_priority`` / ``link_priority``: CUDA stream priorities (0 = default, negative =
         higher) of the main stream (bandwidth-bound forwards and updates), of the index-only ahead-work and of the
-        host-link transfers.  ``mover_ctas`` / ``scatter_ctas``: hl_set_mover_ctas (0 = the library's default)."""
+        host-link transfers.  ``mover_ctas`` / ``scatter_ctas``: hl_set_mover_ctas (0 = the library's default).
+        ``exclusive_write_back``: a mini-batch's main work waits for the previous mini-batch's write-back."""
         assert order in ("fig8", "eq5")
         self.order = order
         self.window_rows = int(window_rows)
@@ -604,7 +616,7 @@ class NativePipelinedHotline(Hotline):
             B.hl_set_mover_ctas(self.ctx, mover_ctas, scatter_ctas)
         self.pipe = B.hl_pipe_create_ex(self.ctx, self.cache, self.host_table, self.window_rows, c_sets, self.n_dense,
                                         self.main.cuda_stream, index_priority=index_priority,
-                                        link_priority=link_priority)
+                                        link_priority=link_priority, exclusive_write_back=exclusive_write_back)
         if order == "eq5":
             B.hl_pipe_set_order(self.pipe, B.HL_PIPE_ORDER_EQ5)
         self.in_flight = 0

@@ -52,12 +52,13 @@ def assert_close(got, want, what):
 
 def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: bool = False, hot_override=None,
                      deferred: bool = False, overlap: bool = True, profile_batches=None, verbose: bool = False,
-                     device: str = "cuda:0", resync: bool = True):
+                     device: str = "cuda:0", resync: bool = True, per_table: bool = False):
     """Profiles, builds the remap, then runs ``steps`` mini-batches: the first call by call with a comparison
     after every call, the others through Hotline.step().  ``hot_override``: None (profiled), "empty", "full",
     or ("random", fraction).  With ``resync`` every step after the first starts from the oracle's tables
     (copied to the device and the host table), so that each step is a parity check on identical inputs; without
-    it the two sides drift apart by their accumulated fp32 rounding.  Returns a dict of workload statistics."""
+    it the two sides drift apart by their accumulated fp32 rounding.  ``per_table``: the host table is one allocation
+    per table (hl_set_host_tables) instead of one for all.  Returns a dict of workload statistics."""
     import paper_2204_05436_b200 as hl
 
     if isinstance(spec, str):
@@ -74,9 +75,17 @@ def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: boo
     staging_cap = max(1, min(N, max_nnz))
 
     table0 = gen.table_values(np.arange(N), D, spec.seed, integer=integer)
-    host_table = torch.from_numpy(table0.copy()).pin_memory()
+    if per_table:
+        base = geom.base
+        host_table = [torch.from_numpy(table0[base[t]:base[t + 1]].copy()).pin_memory() for t in range(T)]
+    else:
+        host_table = torch.from_numpy(table0.copy()).pin_memory()
     h = hl.Hotline(geom.table_rows, D, S, B, max_nnz, hot_cap, staging_cap, host_table, n_dense=spec.n_dense,
                    device=device)
+
+    def host_rows():
+        return np.concatenate([t.numpy() for t in h.host_tables]) if per_table else h.host_table.numpy()
+
     stats = {}
     try:
         with torch.cuda.stream(h.main):
@@ -120,7 +129,11 @@ def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: boo
                 bid = P + step
                 if step > 0 and resync:
                     h.cache.copy_(_t(cache_o, device))
-                    h.host_table.copy_(torch.from_numpy(table_o))
+                    if per_table:
+                        for t in range(T):
+                            h.host_tables[t].copy_(torch.from_numpy(table_o[geom.base[t]:geom.base[t + 1]]))
+                    else:
+                        h.host_table.copy_(torch.from_numpy(table_o))
                     torch.cuda.synchronize()
                 batch = gen.make_batch(spec, geom, bid)
                 grad_full = gen.grad_values(spec.seed, bid, 2, n_bags, D, integer=integer)
@@ -191,17 +204,17 @@ def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: boo
                 assert_close(h.cache[:n_hot].cpu().numpy(), cache_o[:n_hot], "hot rows after update")
                 assert_close(h.cache[hot_cap:hot_cap + len(C)].cpu().numpy(), cache_o[hot_cap:hot_cap + len(C)],
                              "staged rows after update")
-                assert_close(h.host_table.numpy(), table_o, "host table after scatter")
+                assert_close(host_rows(), table_o, "host table after scatter")
                 if integer:
                     assert np.array_equal(pp, pooled_pop_o) and np.array_equal(pn, pooled_non_o), "integer pooled"
                     assert np.array_equal(h.cache[:n_hot].cpu().numpy(), cache_o[:n_hot]), "integer hot rows"
-                    assert np.array_equal(h.host_table.numpy(), table_o), "integer host table"
+                    assert np.array_equal(host_rows(), table_o), "integer host table"
                 if spec.pooling[0] == "one" and step == 0:   # a bag of one lookup is a row copy: bit-exact
                     assert np.array_equal(pp.view(np.uint32), pooled_pop_o.view(np.uint32)), "pooled_pop bits"
                 # rows nobody touched keep their bits
                 touched = np.zeros(N, dtype=bool)
                 touched[C] = True
-                assert np.array_equal(h.host_table.numpy()[~touched].view(np.uint32), table0[~touched].view(np.uint32)) \
+                assert np.array_equal(host_rows()[~touched].view(np.uint32), table0[~touched].view(np.uint32)) \
                     or step > 0, "untouched host rows"
                 stats = dict(n_pop=n_pop_o, n_non=n_non_o, n_cold=len(C), n_hot=n_hot, L_pop=len(O.ids), L_non=len(X.ids),
                              batch=B, N=N)
@@ -215,7 +228,7 @@ def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: boo
 def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: bool = True, profile_batches=None,
                         device: str = "cuda:0", overlap_link: bool = True, sort_ahead: bool = True,
                         combined_sort: bool = True, lookahead: int = 2, native: bool = False,
-                        drain_between: bool = False, order: str = "fig8"):
+                        drain_between: bool = False, order: str = "fig8", per_table: bool = False):
     """Software-pipelined CUDA path (PipelinedHotline) against the oracle processing the same mini-batches one
     after the other.  With integer data every sum is exact, so pooled vectors, the hot cache and the host table
     must agree bit for bit after any number of steps -- which they only do if rows shared by consecutive
@@ -279,7 +292,14 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
         expect.append((perm_o, n_pop_o, pooled_pop_o, pooled_non_o, len(C)))
 
     # ---- CUDA: pipelined ----
-    host_table = torch.from_numpy(table0.copy()).pin_memory()
+    if per_table:      # one host allocation per table (hl_set_host_tables)
+        host_table = [torch.from_numpy(table0[geom.base[t]:geom.base[t + 1]].copy()).pin_memory() for t in range(T)]
+    else:
+        host_table = torch.from_numpy(table0.copy()).pin_memory()
+
+    def host_rows():
+        return np.concatenate([t.numpy() for t in p.host_tables]) if per_table else p.host_table.numpy()
+
     if native:
         p = hl.NativePipelinedHotline(geom.table_rows, D, S, B, max_nnz, hot_cap, window, host_table,
                                       n_dense=spec.n_dense, device=device, lookahead=lookahead, order=order)
@@ -335,24 +355,64 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
         hot_g = p.cache[:n_hot].cpu().numpy()
         if integer:
             assert np.array_equal(hot_g, cache_o[:n_hot]), "hot cache"
-            assert np.array_equal(p.host_table.numpy(), table_o), "host table"
+            assert np.array_equal(host_rows(), table_o), "host table"
         else:
             assert_close(hot_g, cache_o[:n_hot], "hot cache")
-            assert_close(p.host_table.numpy(), table_o, "host table")
+            assert_close(host_rows(), table_o, "host table")
     finally:
         p.close()
     return dict(shared_cold_rows=shared, steps=steps, launches=int(launches))
 
 
+class _HostTable:
+    """The host-DRAM table of a full-size check: one allocation of device-addressable memory, or one per table
+    (for a table above what a single allocation takes).  Rows are read by global id."""
+
+    def __init__(self, hl, geom, per_table: bool):
+        self.base, self.per_table = geom.base, per_table
+        if per_table:
+            self.tensors = [hl.host_table_tensor(r, geom.dim) for r in geom.table_rows]
+        else:
+            self.tensors = [hl.host_table_tensor(geom.total_rows, geom.dim)]
+
+    def for_library(self):
+        return self.tensors if self.per_table else self.tensors[0]
+
+    def fill(self, seed, device, integer=False):
+        for t, ten in enumerate(self.tensors):
+            row0 = int(self.base[t]) if self.per_table else 0
+            for r0 in range(0, ten.shape[0], 1 << 21):      # rows row0 + r0 ... of the whole table
+                n = min(1 << 21, ten.shape[0] - r0)
+                ten[r0:r0 + n].copy_(gen.table_values_torch(row0 + r0, n, ten.shape[1], seed, device, integer=integer))
+        torch.cuda.synchronize()
+
+    def rows(self, g):
+        g = np.asarray(g, dtype=np.int64)
+        if not self.per_table:
+            return self.tensors[0].numpy()[g]
+        t = np.searchsorted(self.base, g, side="right") - 1
+        out = np.empty((len(g), self.tensors[0].shape[1]), dtype=np.float32)
+        for tt in np.unique(t):
+            sel = t == tt
+            out[sel] = self.tensors[tt].numpy()[g[sel] - self.base[tt]]
+        return out
+
+    def free(self, hl):
+        ptrs = [ten.data_ptr() for ten in self.tensors]
+        self.tensors = []
+        for ptr in ptrs:
+            hl.hl_host_free(ptr)
+
+
 def run_fullsize_check(spec, scale_rows: float = 1.0, n_samples: int = 1500, profile_batches=None,
-                       device: str = "cuda:0", verbose: bool = False):
+                       device: str = "cuda:0", verbose: bool = False, per_table: bool = False):
     """A workload too large for an element-by-element float comparison, run in the launch configuration the
     benchmark times (Hotline.step, cold gather on the side stream).  Every integer result is compared in full
     (hot set, perm, counts, both CSRs, cold rows, unified slots); float results are compared on sampled outputs
     that the oracle's definitions give one by one: sampled pooled vectors, sampled updated hot rows, sampled
     written-back cold rows, and sampled rows nobody touched (which must keep their bits).  The host table lives in
-    pinned memory and is filled on the device from the same counter hash the oracle evaluates row by row."""
-    import bench
+    pinned memory and is filled on the device from the same counter hash the oracle evaluates row by row.
+    ``per_table``: one host allocation per table (hl_set_host_tables)."""
     import paper_2204_05436_b200 as hl
 
     if isinstance(spec, str):
@@ -370,14 +430,14 @@ def run_fullsize_check(spec, scale_rows: float = 1.0, n_samples: int = 1500, pro
     rng = np.random.default_rng(spec.seed + 4242)
     rows_of = lambda g: gen.table_values(np.asarray(g, dtype=np.int64), D, spec.seed)   # noqa: E731
 
-    table = hl.host_table_tensor(N, D)
+    table = _HostTable(hl, geom, per_table)
     h = None
     try:
-        bench.fill_table(table, D, spec.seed, torch.device(device))
+        table.fill(spec.seed, torch.device(device))
         probe = rng.integers(0, N, 64)
-        assert np.array_equal(table.numpy()[probe].view(np.uint32), rows_of(probe).view(np.uint32)), "table fill"
-        h = hl.Hotline(geom.table_rows, D, S, B, max_nnz, hot_cap, staging_cap, table, n_dense=spec.n_dense,
-                       device=device)
+        assert np.array_equal(table.rows(probe).view(np.uint32), rows_of(probe).view(np.uint32)), "table fill"
+        h = hl.Hotline(geom.table_rows, D, S, B, max_nnz, hot_cap, staging_cap, table.for_library(),
+                       n_dense=spec.n_dense, device=device)
         with torch.cuda.stream(h.main):
             # ---- learning phase: full comparison ----
             prof = [gen.make_batch(spec, geom, i) for i in range(P)]
@@ -482,7 +542,7 @@ def run_fullsize_check(spec, scale_rows: float = 1.0, n_samples: int = 1500, pro
             got_hot = h.cache[torch.from_numpy(cand[hot_part]).to(device)].cpu().numpy()
             assert_close(got_hot, want[hot_part], "sampled updated hot rows")
             cold_ids = C[cand[~hot_part] - hot_cap]
-            assert_close(table.numpy()[cold_ids], want[~hot_part], "sampled written-back cold rows")
+            assert_close(table.rows(cold_ids), want[~hot_part], "sampled written-back cold rows")
             assert not np.array_equal(want[hot_part], rows_of(slot_row_id(cand[hot_part]))), "update changed nothing"
             # rows nobody touched keep their bits
             idle = np.flatnonzero(~(touched_by_o[:n_hot] | touched_by_x[:n_hot]))
@@ -491,7 +551,7 @@ def run_fullsize_check(spec, scale_rows: float = 1.0, n_samples: int = 1500, pro
             assert np.array_equal(got.view(np.uint32), rows_of(hot_o[idle]).view(np.uint32)), "idle hot rows"
             far = rng.integers(0, N, n_samples)
             far = far[(remap_o[far] < 0) & ~np.isin(far, C)]
-            assert np.array_equal(table.numpy()[far].view(np.uint32), rows_of(far).view(np.uint32)), "idle host rows"
+            assert np.array_equal(table.rows(far).view(np.uint32), rows_of(far).view(np.uint32)), "idle host rows"
             stats = dict(n_pop=n_pop_o, n_non=n_non_o, n_cold=len(C), n_hot=n_hot, N=N, batch=B)
             if verbose:
                 print(f"[{spec.name} full size] {stats}")
@@ -500,7 +560,7 @@ def run_fullsize_check(spec, scale_rows: float = 1.0, n_samples: int = 1500, pro
         if h is not None:
             h.close()
         torch.cuda.synchronize()
-        hl.hl_host_free(table.data_ptr())
+        table.free(hl)
 
 
 def run_native_fullsize_check(spec, steps: int = 4, scale_rows: float = 1.0, profile_batches=None, lookahead: int = 2,

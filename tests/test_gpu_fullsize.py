@@ -49,8 +49,8 @@ def test_avazu_like_full_size_every_element():
     run_pipelined_check("avazu_like", steps=3, integer=False, profile_batches=8)
 
 
-def test_multi_hot_full_batch_sampled():
-    """8 tables x dim 128, Poisson(20) bags capped at 64, the full batch of 65,536 inputs (10.5 M lookups); row
-    counts cut to an eighth (2.5 M rows per table, 9.5 GiB host table) to keep the test's set-up short."""
-    stats = run_fullsize_check("multi_hot", scale_rows=0.125, n_samples=600)
-    assert stats["batch"] == 65536
+def test_multi_hot_full_size_sampled():
+    """8 tables x 20 M rows x dim 128 (76.3 GiB, one host allocation of 9.5 GiB per table), Poisson(20) bags capped
+    at 64, the full batch of 65,536 inputs (10.5 M lookups): integer results in full, float results on samples."""
+    stats = run_fullsize_check("multi_hot", n_samples=600, per_table=True)
+    assert stats["batch"] == 65536 and stats["N"] == 160_000_000 and stats["n_cold"] > 1_000_000

@@ -50,6 +50,16 @@ def test_cold_row_search_at_the_limit_of_its_one_cluster_path(batch):
     assert stats["n_pop"] == 0 and stats["n_cold"] > 5_000        # distinct rows; the lookups are 8 * batch
 
 
+def test_one_host_allocation_per_table():
+    """hl_set_host_tables: every table in an allocation of its own (ragged sizes), the call-by-call path and the
+    library's scheduler both bit-exact on integer data."""
+    spec = gen.WorkloadSpec(name="ragged_tables", num_tables=11, dim=32, batch=777, rows=("loguniform", 4, 30_000, 3),
+                            alpha=tuple([1.1] * 11), hot_policy=("fraction", 10, 100), profile_batches=4, seed=23)
+    run_config_check(spec, steps=2, integer=True, per_table=True)
+    run_config_check(spec, steps=1, per_table=True)
+    run_pipelined_check(spec, steps=5, integer=True, native=True, per_table=True)
+
+
 def test_min_share_policy():
     spec = dataclasses.replace(gen.CONFIGS["tiny"], hot_policy=("share", 1, 2000))
     run_config_check(spec, steps=1)
