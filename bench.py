@@ -1215,18 +1215,26 @@ def run_micro(args) -> None:
 def run_sweep(args) -> None:
     """`--sweep`: (1) the hot-cache budget is cut from the configuration's value down to 1/64 of it, which moves
     the ratio of popular to non-popular inputs; (2) the mini-batch size is varied at the full budget.  Every point:
-    10 warm-up and 60 timed mini-batches through the default pipeline, CUDA events.  One JSON line."""
+    10 warm-up and 60 timed mini-batches through the default pipeline, CUDA events.  Budget points also get the
+    overlap efficiency of the host link (the paper's Section VII-F claim is that the gather stays hidden as the share
+    of popular inputs falls): the same steps are timed with the whole table resident in HBM (the movers then move
+    rows inside the device, which costs next to nothing), and the movers are timed alone on one mini-batch's rows;
+    efficiency = 1 - (time with the host table - time with the resident table) / (read alone + write-back alone),
+    i.e. the share of the transfers' own time that the schedule hides.  One JSON line."""
     import dataclasses
     import torch
     import paper_2204_05436_b200 as hl
     device = torch.device("cuda:0")
     torch.cuda.set_device(device)
     name, scale = pick_workload(args.workload, 1)
+    if args.row_scale is not None:
+        scale = args.row_scale
     wl = Workload(name, scale, 8, args.profile_batches, device, args.threads)
     T, D, S = wl.T, wl.D, wl.S
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
     points = []
 
-    def measure(h, batches, B, n_bags, label):
+    def measure(h, batches, B, n_bags, movers_alone=False):
         d_in = [(torch.from_numpy(b.indices).to(device), torch.from_numpy(b.offsets).to(device), B,
                  torch.from_numpy(b.dense).to(device) if b.dense is not None else None) for b in batches]
         d_grad = torch.randn((n_bags, D), device=device, dtype=torch.float32)
@@ -1234,12 +1242,12 @@ def run_sweep(args) -> None:
         n = len(d_in)
         it = [0]
 
-        def step():
+        def step(last=False):
             i = it[0]
             it[0] += 1
             if h.idle:
                 h.start(*d_in[i % n], more=[d_in[(i + a) % n] for a in range(1, h.lookahead)], inputs_ready="resident")
-            return h.sets[h.step(d_grad, d_grad, wl.spec.lr, next_batch=d_in[(i + h.lookahead) % n],
+            return h.sets[h.step(d_grad, d_grad, wl.spec.lr, next_batch=None if last else d_in[(i + h.lookahead) % n],
                                  inputs_ready="resident")]
 
         pops, colds = [], []
@@ -1259,10 +1267,37 @@ def run_sweep(args) -> None:
         e1.record(h.main)
         h.drain()
         h.status()
-        ms = e0.elapsed_time(e1) / 60
-        points.append(dict(label, batch=B, popular_fraction=sum(pops) / (len(pops) * B),
-                           cold_rows_per_step=sum(colds) / len(colds), ms_per_step=ms, samples_per_s=B / ms * 1e3))
-        log(f"[sweep] {points[-1]}")
+        out = dict(batch=B, popular_fraction=sum(pops) / (len(pops) * B), cold_rows_per_step=sum(colds) / len(colds),
+                   ms_per_step=e0.elapsed_time(e1) / 60)
+        while not h.idle:                 # empty the pipeline: the last mini-batch stepped is used below
+            st = step(last=True)
+        h.drain()
+        if movers_alone:
+            flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+            w = ((h.j_done - 1) % 2) * h.window_rows
+            hl.hl_set_mover_ctas(h.ctx, 2 * sms, 2 * sms)
+
+            def alone(fn):
+                us = []
+                for _ in range(5):
+                    flush.zero_()
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(h.main)
+                    fn()
+                    b.record(h.main)
+                    h.main.synchronize()
+                    us.append(a.elapsed_time(b) * 1e3)
+                return statistics.median(us)
+
+            s_ = h.main.cuda_stream
+            out["read_alone_us"] = alone(lambda: hl.hl_stage_cold(h.ctx, h.host_table, h.cache, w, h.window_rows,
+                                                                  st.cold_rows, st.n_cold, None, s_))
+            out["write_back_alone_us"] = alone(lambda: hl.hl_scatter_cold_at(h.ctx, h.cache, w, h.window_rows,
+                                                                             st.cold_rows, st.n_cold, h.host_table, s_))
+            out["alone_rows"] = int(st.n_cold.item())
+            hl.hl_set_mover_ctas(h.ctx, 0, 0)
+            h.status()
+        return out
 
     def learn(h, k_rows):
         for i, b in enumerate(wl.profile):
@@ -1272,32 +1307,64 @@ def run_sweep(args) -> None:
         h.status()
         return int(h.n_hot.item())
 
-    # (1) budget / ratio sweep
-    h = hl.NativePipelinedHotline(wl.geom.table_rows, D, S, wl.B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
-                                  n_dense=wl.spec.n_dense, device=str(device))
-    with torch.cuda.stream(h.main):
-        for div in (1, 2, 4, 16, 64):
-            n_hot = learn(h, max(1, wl.hot_cap // div))
-            measure(h, wl.batches, wl.B, wl.n_bags, dict(sweep="budget", budget_fraction=1.0 / div, hot_rows=n_hot))
+    def make(table, max_batch=None):
+        mb = wl.B if max_batch is None else max_batch
+        nnz = T * mb * S if wl.spec.pooling[0] == "one" else T * mb * S * int(wl.spec.pooling[2])
+        return hl.NativePipelinedHotline(wl.geom.table_rows, D, S, mb, nnz, wl.hot_cap, min(wl.N, nnz), table,
+                                         n_dense=wl.spec.n_dense, device=str(device))
+
+    # (1) budget / ratio sweep, with the overlap efficiency of the link
+    resident = None
+    if not isinstance(wl.table, list):
+        try:
+            resident = torch.empty((wl.N, D), dtype=torch.float32, device=device)
+            resident.copy_(wl.table, non_blocking=False)
+        except RuntimeError:      # no room for a copy of the table in HBM: the sweep goes without the efficiency
+            resident = None
+    h = make(wl.table)
+    h_res = make(resident) if resident is not None else None
+    for div in (1, 2, 4, 16, 64):
+        k = max(1, wl.hot_cap // div)
+        with torch.cuda.stream(h.main):
+            n_hot = learn(h, k)
+            pt = measure(h, wl.batches, wl.B, wl.n_bags, movers_alone=True)
             h.flush_hot()            # the host table gets the popular rows back before the set changes
             h.status()
+        pt.update(sweep="budget", budget_fraction=1.0 / div, hot_rows=n_hot, samples_per_s=wl.B / pt["ms_per_step"] * 1e3)
+        if h_res is not None:
+            with torch.cuda.stream(h_res.main):
+                learn(h_res, k)
+                res = measure(h_res, wl.batches, wl.B, wl.n_bags)
+                h_res.flush_hot()
+                h_res.status()
+            scale_rows = pt["cold_rows_per_step"] / max(1, pt["alone_rows"])     # the alone run moved one mini-batch's rows
+            t_link = (pt["read_alone_us"] + pt["write_back_alone_us"]) * 1e-3 * scale_rows
+            pt["ms_per_step_table_resident"] = res["ms_per_step"]
+            pt["link_alone_ms_per_step"] = t_link
+            pt["overlap_efficiency"] = 1.0 - (pt["ms_per_step"] - res["ms_per_step"]) / t_link if t_link > 0 else None
+        points.append(pt)
+        log(f"[sweep] {pt}")
     h.close()
+    if h_res is not None:
+        h_res.close()
+    del resident
+    torch.cuda.empty_cache()
     # (2) batch-size sweep at the full budget
     for B in (2048, 4096, 8192, 32768):
         spec = dataclasses.replace(wl.spec, batch=B)
         batches = [gen.make_batch(spec, wl.geom, 100_000 + i, args.threads) for i in range(8)]
-        n_bags = T * B * S
-        mb = max(B, wl.B)
-        h = hl.NativePipelinedHotline(wl.geom.table_rows, D, S, mb, T * mb * S if wl.spec.pooling[0] == "one" else
-                                      T * mb * S * int(wl.spec.pooling[2]), wl.hot_cap, wl.staging_cap, wl.table,
-                                      n_dense=wl.spec.n_dense, device=str(device))
+        h = make(wl.table, max(B, wl.B))
         with torch.cuda.stream(h.main):
             n_hot = learn(h, wl.hot_cap)
-            measure(h, batches, B, n_bags, dict(sweep="batch", budget_fraction=1.0, hot_rows=n_hot))
+            pt = measure(h, batches, B, T * B * S)
             h.flush_hot()
             h.status()
+        pt.update(sweep="batch", budget_fraction=1.0, hot_rows=n_hot, samples_per_s=B / pt["ms_per_step"] * 1e3)
+        points.append(pt)
+        log(f"[sweep] {pt}")
         h.close()
-    print(json.dumps({"sweep": wl.name, "unit": "ms per mini-batch, samples/s", "points": points}), flush=True)
+    print(json.dumps({"sweep": wl.name, "row_scale": wl.scale, "unit": "ms per mini-batch, samples/s",
+                      "points": points}), flush=True)
     wl.free()
 
 
