@@ -491,6 +491,47 @@ HL_API int32_t hl_pipe_wait_counts(hl_pipe* p, void* stream);
 /* Host waits until everything queued so far has finished. */
 HL_API int32_t hl_pipe_drain(hl_pipe* p);
 
+/* ---------------------------------------------------------------------------------------------------------
+ * Models with 2^31 rows and more (Section VII-F "Varying Model Size": the synthetic models of 196 to 390 GB), and
+ * the hashed lookup of Section V-C: the index-only calls of the path with 64-bit global row ids.
+ *
+ * Every table still has fewer than 2^31 rows (table-local indices stay int32, the mini-batch layout is unchanged), but
+ * the tables together may have more, so popular rows, X's row ids and cold rows are int64.  Nothing is sized by the
+ * number of rows: accesses are counted in an open-addressing table of `counter_slots` entries (rounded up to a power
+ * of two; it must hold every distinct row the profiled mini-batches touch, HL_ECAPACITY otherwise), and the popular
+ * set is an open-addressing table row -> slot of at least 2 * hot_cap_rows entries.  Both are addressed by the
+ * randomizer (a 4-round Feistel network on the 32-bit halves of the row id) with linear probing.  Results are those
+ * of the dense structures: hl_wide_profile_hot selects by hl_profile_hot's rules (one ranking, count descending, id
+ * ascending), popular rows get their slots in ascending id order, hl_wide_fragment and hl_wide_index_cold give
+ * hl_fragment's and hl_index_cold's outputs.  The slots they produce feed hl_embbag_fwd / hl_embbag_bwd_* of an
+ * ordinary context over the same cache.  Scratch: the caller's workspace (hl_wide_workspace_bytes); the calls of one
+ * context must not overlap.
+ * ------------------------------------------------------------------------------------------------------- */
+typedef struct hl_wide hl_wide;
+HL_API size_t hl_wide_workspace_bytes(const hl_geometry* geom, int32_t max_batch, int64_t max_nnz,
+                                      int64_t hot_cap_rows, int64_t staging_cap_rows, int64_t counter_slots);
+HL_API int32_t hl_wide_create(hl_wide** out, const hl_geometry* geom, int32_t max_batch, int64_t max_nnz,
+                              int64_t hot_cap_rows, int64_t staging_cap_rows, int64_t counter_slots,
+                              void* d_workspace, size_t ws_bytes);
+HL_API int32_t hl_wide_destroy(hl_wide* w);
+HL_API int32_t hl_wide_status(hl_wide* w);     /* as hl_status */
+/* As hl_profile_hot; d_hot_rows is int64 [hot_cap_rows]; row_bytes is the row payload HL_HOT_BUDGET_BYTES divides by. */
+HL_API int32_t hl_wide_profile_hot(hl_wide* w, const hl_batch* b, int32_t reset, int32_t finalize, int32_t policy,
+                                   int64_t p_num, int64_t p_den, int32_t row_bytes, int64_t* d_hot_rows,
+                                   int64_t* d_n_hot, void* stream);
+/* As hl_build_remap without the row load: the hashed remap for d_hot_rows[0 .. *d_n_hot) (strictly ascending). */
+HL_API int32_t hl_wide_build_remap(hl_wide* w, const int64_t* d_hot_rows, const int64_t* d_n_hot, void* stream);
+/* As hl_fragment (no dense features); X's offsets go to d_non_offsets [T*max_batch*S + 1], its global row ids (int64,
+ * -1 for an index outside its table) to d_non_rows [non_cap]. */
+HL_API int32_t hl_wide_fragment(hl_wide* w, const hl_batch* b, int32_t* d_perm, int32_t* d_counts, hl_ubatch* pop,
+                                int32_t* d_non_offsets, int64_t* d_non_rows, int64_t non_cap, void* stream);
+/* As hl_index_cold without windows: d_cold_rows (int64 [staging_cap_rows]) = the distinct non-popular rows of X,
+ * ascending; d_non_slots [non_cap] = the unified slot of every lookup of X (hot slot, or hot_cap_rows + rank in
+ * d_cold_rows; -1 for a skipped lookup). */
+HL_API int32_t hl_wide_index_cold(hl_wide* w, const int32_t* d_non_offsets, const int64_t* d_non_rows, int64_t non_cap,
+                                  const int32_t* d_n_non, int32_t* d_non_slots, int64_t* d_cold_rows,
+                                  int64_t* d_n_cold, void* stream);
+
 /* No counterpart in the paper: an addition for callers that cannot allocate.
  *
  * Some callers have no way to hand the library a workspace: code that runs where device allocation is forbidden

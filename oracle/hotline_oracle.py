@@ -122,10 +122,10 @@ def load_hot_cache(table: np.ndarray, hot_rows: np.ndarray) -> np.ndarray:
 class MicroBatch:
     samples: np.ndarray      # int64 [n]   ids (positions in M) of the inputs, ascending
     offsets: np.ndarray      # int32 [T*n*S + 1]
-    ids: np.ndarray          # int32 [L_mu]  cache slots (O) or global rows (X)
+    ids: np.ndarray          # [L_mu]  cache slots (O, int32) or global rows (X; int64 once the model has 2^31 rows)
 
 
-def _emit_microbatch(samples, per_lookup_value, offsets, T, B, S) -> MicroBatch:
+def _emit_microbatch(samples, per_lookup_value, offsets, T, B, S, id_dtype=np.int32) -> MicroBatch:
     """Re-lay the bags of the chosen inputs table-major, bag (t*n + i)*S + s <- bag (t*B + samples[i])*S + s,
     each bag's lookups kept in their original order."""
     samples = np.asarray(samples, dtype=np.int64)
@@ -140,7 +140,7 @@ def _emit_microbatch(samples, per_lookup_value, offsets, T, B, S) -> MicroBatch:
     total = int(new_off[-1])
     within = np.arange(total, dtype=np.int64) - np.repeat(new_off[:-1], sizes)
     src_pos = np.repeat(offsets[src_bags], sizes) + within
-    ids = np.asarray(per_lookup_value)[src_pos].astype(np.int32)
+    ids = np.asarray(per_lookup_value)[src_pos].astype(id_dtype)
     return MicroBatch(samples=samples, offsets=new_off.astype(np.int32), ids=ids)
 
 
@@ -163,7 +163,8 @@ def fragment(indices, offsets, batch: int, table_rows, remap: np.ndarray, bags_p
     x_samples = np.flatnonzero(~popular)
     perm = np.concatenate([o_samples, x_samples]).astype(np.int32)
     O = _emit_microbatch(o_samples, slot, offsets, T, B, S)
-    X = _emit_microbatch(x_samples, g, offsets, T, B, S)
+    # global row ids need 64 bits once the tables together have 2^31 rows (the paper's largest synthetic models)
+    X = _emit_microbatch(x_samples, g, offsets, T, B, S, np.int64 if remap.shape[0] >= 2 ** 31 else np.int32)
     dense_out = None if dense is None else np.asarray(dense)[perm].copy()
     return perm, int(o_samples.shape[0]), O, X, dense_out
 

@@ -24,6 +24,8 @@ EXPORTS = (
     "hl_tracker_reset", "hl_tracker_update", "hl_tracker_export",
     "hl_pipe_create", "hl_pipe_create_ex", "hl_pipe_destroy", "hl_pipe_submit", "hl_pipe_step", "hl_pipe_wait_outputs", "hl_pipe_drain",
     "hl_pipe_trace_begin", "hl_pipe_trace_end", "hl_pipe_wait_counts", "hl_set_mover_ctas", "hl_test_bounded_waits", "hl_set_host_tables", "hl_set_kernel_width",
+    "hl_wide_workspace_bytes", "hl_wide_create", "hl_wide_destroy", "hl_wide_status", "hl_wide_profile_hot",
+    "hl_wide_build_remap", "hl_wide_fragment", "hl_wide_index_cold",
     "hl_index_cold_begin", "hl_index_cold_end", "hl_index_cold_verdict",
     "hl_embbag_bwd_prepare_merged", "hl_pipe_set_order",
 )
@@ -167,6 +169,22 @@ def _load() -> ctypes.CDLL:
     lib.hl_pipe_trace_end.argtypes = [vp, ctypes.POINTER(hl_pipe_span), i32, ctypes.POINTER(i32)]
     lib.hl_set_mover_ctas.restype = i32
     lib.hl_set_mover_ctas.argtypes = [vp, i32, i32]
+    lib.hl_wide_workspace_bytes.restype = ctypes.c_size_t
+    lib.hl_wide_workspace_bytes.argtypes = [geo, i32, i64, i64, i64, i64]
+    lib.hl_wide_create.restype = i32
+    lib.hl_wide_create.argtypes = [ctypes.POINTER(vp), geo, i32, i64, i64, i64, i64, vp, ctypes.c_size_t]
+    lib.hl_wide_destroy.restype = i32
+    lib.hl_wide_destroy.argtypes = [vp]
+    lib.hl_wide_status.restype = i32
+    lib.hl_wide_status.argtypes = [vp]
+    lib.hl_wide_profile_hot.restype = i32
+    lib.hl_wide_profile_hot.argtypes = [vp, ctypes.POINTER(hl_batch), i32, i32, i32, i64, i64, i32, vp, vp, vp]
+    lib.hl_wide_build_remap.restype = i32
+    lib.hl_wide_build_remap.argtypes = [vp, vp, vp, vp]
+    lib.hl_wide_fragment.restype = i32
+    lib.hl_wide_fragment.argtypes = [vp, ctypes.POINTER(hl_batch), vp, vp, ctypes.POINTER(hl_ubatch), vp, vp, i64, vp]
+    lib.hl_wide_index_cold.restype = i32
+    lib.hl_wide_index_cold.argtypes = [vp, vp, vp, i64, vp, vp, vp, vp, vp]
     lib.hl_set_kernel_width.restype = i32
     lib.hl_set_kernel_width.argtypes = [vp, i32, i32]
     lib.hl_set_host_tables.restype = i32
@@ -455,6 +473,59 @@ def hl_pipe_create_ex(ctx: int, d_cache, host_table, window_rows: int, sets, n_d
 
 def hl_set_mover_ctas(ctx: int, read_ctas: int, write_ctas: int) -> None:
     _check("hl_set_mover_ctas", _lib.hl_set_mover_ctas(ctx, int(read_ctas), int(write_ctas)))
+
+
+def hl_wide_workspace_bytes(geom: hl_geometry, max_batch: int, max_nnz: int, hot_cap_rows: int, staging_cap_rows: int,
+                            counter_slots: int) -> int:
+    n = _lib.hl_wide_workspace_bytes(ctypes.byref(geom), max_batch, max_nnz, hot_cap_rows, staging_cap_rows,
+                                     counter_slots)
+    if n == 0:
+        raise HotlineError("hl_wide_workspace_bytes", HL_EINVAL)
+    return int(n)
+
+
+def hl_wide_create(geom: hl_geometry, max_batch: int, max_nnz: int, hot_cap_rows: int, staging_cap_rows: int,
+                   counter_slots: int, d_workspace, ws_bytes: int) -> int:
+    w = ctypes.c_void_p()
+    _check("hl_wide_create", _lib.hl_wide_create(ctypes.byref(w), ctypes.byref(geom), max_batch, max_nnz, hot_cap_rows,
+                                                 staging_cap_rows, counter_slots, _ptr(d_workspace), ws_bytes))
+    return w.value
+
+
+def hl_wide_destroy(w: int) -> None:
+    _check("hl_wide_destroy", _lib.hl_wide_destroy(w))
+
+
+def hl_wide_status(w: int, raise_on_error: bool = True) -> int:
+    st = _lib.hl_wide_status(w)
+    if raise_on_error:
+        _check("hl_wide_status", st)
+    return st
+
+
+def hl_wide_profile_hot(w: int, batch: Optional[hl_batch], reset: bool, finalize: bool, policy: int, p_num: int,
+                        p_den: int, row_bytes: int, d_hot_rows, d_n_hot, stream: int) -> None:
+    b = ctypes.byref(batch) if batch is not None else None
+    _check("hl_wide_profile_hot", _lib.hl_wide_profile_hot(w, b, int(reset), int(finalize), policy, p_num, p_den,
+                                                           int(row_bytes), _ptr(d_hot_rows), _ptr(d_n_hot), stream))
+
+
+def hl_wide_build_remap(w: int, d_hot_rows, d_n_hot, stream: int) -> None:
+    _check("hl_wide_build_remap", _lib.hl_wide_build_remap(w, _ptr(d_hot_rows), _ptr(d_n_hot), stream))
+
+
+def hl_wide_fragment(w: int, batch: hl_batch, d_perm, d_counts, pop: hl_ubatch, d_non_offsets, d_non_rows,
+                     non_cap: int, stream: int) -> None:
+    _check("hl_wide_fragment", _lib.hl_wide_fragment(w, ctypes.byref(batch), _ptr(d_perm), _ptr(d_counts),
+                                                     ctypes.byref(pop), _ptr(d_non_offsets), _ptr(d_non_rows),
+                                                     int(non_cap), stream))
+
+
+def hl_wide_index_cold(w: int, d_non_offsets, d_non_rows, non_cap: int, d_n_non, d_non_slots, d_cold_rows, d_n_cold,
+                       stream: int) -> None:
+    _check("hl_wide_index_cold", _lib.hl_wide_index_cold(w, _ptr(d_non_offsets), _ptr(d_non_rows), int(non_cap),
+                                                         _ptr(d_n_non), _ptr(d_non_slots), _ptr(d_cold_rows),
+                                                         _ptr(d_n_cold), stream))
 
 
 def hl_set_kernel_width(ctx: int, fwd_ctas_per_sm: int, bwd_ctas_per_sm: int) -> None:

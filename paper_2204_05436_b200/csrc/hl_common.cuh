@@ -94,6 +94,40 @@ struct hl_ctx {
     void* mark_user;
 };
 
+// Context of the wide-id index path (hl_wide_*): global row ids are 64-bit, every table still has fewer than 2^31
+// rows.  Popularity is counted in a hashed counter and the popular rows are found through a hashed remap, so nothing
+// here is sized by the number of rows.
+struct hl_wide {
+    int32_t T, S;
+    int64_t N;
+    int32_t max_batch;
+    int64_t max_nnz, max_bags, hot_cap, staging_cap;
+    int64_t counter_slots, remap_slots;     // powers of two
+    int sms;
+    int64_t* h_table_base;
+    // device regions (carved from the caller's workspace)
+    int32_t* status;
+    int64_t* table_base;                     // [T+1]
+    long long* c_keys;                       // [counter_slots] row id or -1
+    uint32_t* c_cnt;                         // [counter_slots]
+    hl::SelectState* sel;
+    uint32_t *sel_gt, *sel_eq;               // [counter_slots / kSelTile + 2]
+    int32_t* n_seen;                         // [4]
+    int32_t *e_tab, *e_idx;                  // [counter_slots] table and table-local index of every counted row
+    uint32_t *e_cnt, *s_cnt;                 // [counter_slots] its count; the counts in row order
+    int32_t* s_ent;                          // [counter_slots] entry behind every position of the row order
+    int32_t* sel_idx;                        // [hot_cap] selected positions
+    long long* r_keys;                       // [remap_slots] popular row or -1
+    int32_t* r_vals;                         // [remap_slots] its slot
+    int32_t* sort_keys[2];                   // [max(counter_slots, max_nnz)]
+    int32_t* sort_vals[2];
+    uint32_t* sort_hist;
+    uint8_t* frag_flags;                     // [max_batch]
+    int32_t *frag_scan, *frag_tiles;
+    int32_t *cold_tab, *cold_idx, *cold_pos; // [max_nnz] cold lookups: table, index, position in X
+    int32_t *cold_rank, *cold_tiles, *cold_n;
+};
+
 namespace hl {
 
 #define HL_CUDA_TRY(expr)                         \
@@ -171,6 +205,49 @@ __device__ __forceinline__ unsigned char* row_address(const TableMap& m, int64_t
     return m.ptrs[lo] + (g - __ldg(&m.base[lo])) * row_bytes;
 }
 
+// ---- the hashed lookup structures of the wide-id path (global row ids beyond 2^31, hl_wide_*) ------------------
+// Randomizer of Section V-C on a 64-bit row id: a 4-round Feistel network on its 32-bit halves (a bijection, so
+// distinct rows never collide before the reduction to the table size), round function (x * 0x9E3779B1 + K_r)
+// rotated by 15 bits.
+__host__ __device__ __forceinline__ uint64_t randomize64(uint64_t g) {
+    uint32_t l = (uint32_t)(g >> 32), r = (uint32_t)g;
+    const uint32_t k[4] = {0x85EBCA6Bu, 0xC2B2AE35u, 0x27D4EB2Fu, 0x165667B1u};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        uint32_t f = r * 0x9E3779B1u + k[i];
+        f = (f << 15) | (f >> 17);
+        const uint32_t nl = r;
+        r = l ^ f;
+        l = nl;
+    }
+    return ((uint64_t)l << 32) | r;
+}
+
+// Open-addressing table row id -> value (linear probing from randomize64(row) & mask; an empty entry holds -1).
+struct HashProbe {
+    const long long* keys;
+    const int32_t* vals;
+    uint64_t mask;
+    __device__ __forceinline__ int32_t slot(int64_t g) const {
+        uint64_t h = randomize64((uint64_t)g) & mask;
+        for (uint64_t tries = 0; tries <= mask; ++tries) {
+            const long long k = __ldg(&keys[h]);
+            if (k == g) return __ldg(&vals[h]);
+            if (k < 0) return -1;
+            h = (h + 1) & mask;
+        }
+        return -1;
+    }
+    __device__ __forceinline__ bool hit(int64_t g) const { return slot(g) >= 0; }
+};
+
+// The dense form used by the 32-bit path: one 32-byte block per 224 rows (see RemapBlock).
+struct BitmapProbe {
+    const RemapBlock* remap;
+    __device__ __forceinline__ int32_t slot(int64_t g) const { return remap_slot(remap, g); }
+    __device__ __forceinline__ bool hit(int64_t g) const { return remap_hit(remap, g); }
+};
+
 __device__ __forceinline__ unsigned lanemask_lt() {
     unsigned m;
     asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
@@ -226,6 +303,11 @@ constexpr int64_t bwd_span_list_words(int64_t max_nnz) {
 
 // ints of scratch exclusive_scan_i32 needs for at most n_max elements (64-bit ticket + status words).
 constexpr int64_t scan_tile_words(int64_t n_max) { return 2 * ((n_max > 0 ? n_max : 1) / kScanTile + 3); }
+
+// Selection of the rows with the k largest counts (implemented in hl_profile.cu; see there).
+int32_t select_rows_by_count(const uint32_t* counts, int64_t n, SelectState* sel, uint32_t* sel_gt, uint32_t* sel_eq,
+                             long long k, long long share_num, long long share_den, int64_t cap, int32_t* out_idx,
+                             int64_t* d_n_out, int32_t* status, int sms, cudaStream_t stream);
 
 // Process-wide count of kernels this library has launched (read by hl_launch_count).
 void note_launches(int n);

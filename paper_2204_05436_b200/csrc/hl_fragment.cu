@@ -15,11 +15,12 @@ constexpr int kThreads = 256;
 // LANE_PER_TABLE: lane l walks the lookups of tables l, l+32, ... of its input (short bags: pooling 1).
 // otherwise the warp walks table after table with the lanes striding over the table's lookups of the input
 // (its S bags are contiguous in the table-major layout).
-template <bool LANE_PER_TABLE>
+// Probe: how a global row is looked up in the popular set (BitmapProbe: the dense bitmap of the 32-bit path;
+// HashProbe: the hashed remap of the wide-id path).
+template <bool LANE_PER_TABLE, class Probe>
 __global__ void __launch_bounds__(kThreads) k_frag_flags(const int32_t* __restrict__ indices,
                                                          const int32_t* __restrict__ offsets, int B, int T, int S,
-                                                         const int64_t* __restrict__ table_base,
-                                                         const RemapBlock* __restrict__ remap,
+                                                         const int64_t* __restrict__ table_base, Probe remap,
                                                          uint8_t* __restrict__ flags, int32_t* status) {
     const int lane = threadIdx.x & 31;
     const int warps_per_block = kThreads / 32;
@@ -35,7 +36,7 @@ __global__ void __launch_bounds__(kThreads) k_frag_flags(const int32_t* __restri
                     if (idx < 0 || idx >= rows) {
                         set_status(status, HL_EBOUNDS);
                         miss = true;
-                    } else if (!remap_hit(remap, base + idx)) {
+                    } else if (!remap.hit(base + idx)) {
                         miss = true;
                     }
                 }
@@ -50,7 +51,7 @@ __global__ void __launch_bounds__(kThreads) k_frag_flags(const int32_t* __restri
                     if (idx < 0 || idx >= rows) {
                         set_status(status, HL_EBOUNDS);
                         miss = true;
-                    } else if (!remap_hit(remap, base + idx)) {
+                    } else if (!remap.hit(base + idx)) {
                         miss = true;
                     }
                 }
@@ -154,18 +155,18 @@ __global__ void __launch_bounds__(kThreads) k_frag_sizes(const int32_t* __restri
     }
 }
 
-// GROUP lanes cooperate on one destination bag (1 for short bags, 32 for long ones).
-template <int GROUP>
+// GROUP lanes cooperate on one destination bag (1 for short bags, 32 for long ones).  NonId: type of X's global row
+// ids (int32_t, or int64_t on the wide-id path).
+template <int GROUP, class Probe, typename NonId>
 __global__ void __launch_bounds__(kThreads) k_frag_emit(const int32_t* __restrict__ indices,
                                                         const int32_t* __restrict__ offsets, int B, int T, int S,
                                                         const int32_t* __restrict__ perm,
                                                         int32_t* __restrict__ counts,
                                                         const int32_t* __restrict__ dst_start,   // scanned sizes
-                                                        const int64_t* __restrict__ table_base,
-                                                        const RemapBlock* __restrict__ remap,
+                                                        const int64_t* __restrict__ table_base, Probe remap,
                                                         int32_t* __restrict__ pop_offsets, int32_t* __restrict__ pop_ids,
                                                         int64_t pop_cap, int32_t* __restrict__ non_offsets,
-                                                        int32_t* __restrict__ non_ids, int64_t non_cap,
+                                                        NonId* __restrict__ non_ids, int64_t non_cap,
                                                         int32_t* status) {
     const int n_pop = counts[0];
     const int64_t n_bags = (int64_t)T * B * S, pop_bags = (int64_t)T * n_pop * S;
@@ -193,7 +194,7 @@ __global__ void __launch_bounds__(kThreads) k_frag_emit(const int32_t* __restric
                 }
                 const int32_t idx = indices[src_lo + j];
                 // every lookup of a popular input was tested to be in range and popular
-                pop_ids[out_lo + j] = remap_slot(remap, base + idx);
+                pop_ids[out_lo + j] = remap.slot(base + idx);
             }
         } else {
             const int32_t out_lo = dst_start[dst] - L_pop;
@@ -205,7 +206,7 @@ __global__ void __launch_bounds__(kThreads) k_frag_emit(const int32_t* __restric
                     break;
                 }
                 const int32_t idx = indices[src_lo + j];
-                non_ids[out_lo + j] = (idx < 0 || idx >= rows) ? -1 : (int32_t)(base + idx);
+                non_ids[out_lo + j] = (idx < 0 || idx >= rows) ? (NonId)-1 : (NonId)(base + idx);
             }
         }
     }
@@ -226,6 +227,52 @@ __global__ void __launch_bounds__(kThreads) k_permute_dense(const float* __restr
 
 using namespace hl;
 
+namespace hl {
+namespace {
+
+// The launches of a fragment call, for either lookup structure.  scratch: flags [max_batch], scan [n_bags + 2],
+// tiles [scan_tile_words(n_bags)].
+template <class Probe, typename NonId>
+int32_t fragment_launch(const hl_batch* b, int T, int S, int sms, const int64_t* table_base, Probe probe,
+                        uint8_t* flags, int32_t* scan, int32_t* tiles, int32_t* status, WaitCfg waits,
+                        const float* d_dense, int32_t n_dense, int32_t* d_perm, int32_t* d_counts, hl_ubatch* pop,
+                        int32_t* non_offsets, NonId* non_ids, int64_t non_cap, float* d_dense_out, cudaStream_t stream) {
+    const int B = b->batch;
+    const int64_t n_bags = (int64_t)T * B * S;
+    const bool short_bags = b->nnz <= 4 * (int64_t)T * B;   // on average at most 4 lookups per input and table
+    const int cap = 4 * sms;               // CTAs of every kernel here: they stride over their work
+    const int flag_grid = grid_for(B, kThreads / 32, 2 * cap);
+    if (short_bags)
+        k_frag_flags<true, Probe><<<flag_grid, kThreads, 0, stream>>>(b->indices, b->offsets, B, T, S, table_base, probe,
+                                                                      flags, status);
+    else
+        k_frag_flags<false, Probe><<<flag_grid, kThreads, 0, stream>>>(b->indices, b->offsets, B, T, S, table_base,
+                                                                       probe, flags, status);
+    k_frag_partition<<<1, 1024, 0, stream>>>(flags, B, d_perm, d_counts);
+    k_frag_sizes<<<grid_for(n_bags, kThreads, cap), kThreads, 0, stream>>>(b->offsets, B, T, S, d_perm, d_counts, scan);
+    note_launches(3);   // flags, partition, sizes
+    HL_LAUNCH_CHECK();
+    int32_t st = exclusive_scan_i32(scan, scan, nullptr, n_bags, tiles, status, stream, waits);
+    if (st != HL_OK) return st;
+    if (b->nnz <= 4 * n_bags)
+        k_frag_emit<1, Probe, NonId><<<grid_for(n_bags, kThreads, cap), kThreads, 0, stream>>>(
+            b->indices, b->offsets, B, T, S, d_perm, d_counts, scan, table_base, probe, pop->offsets, pop->ids,
+            pop->cap_ids, non_offsets, non_ids, non_cap, status);
+    else
+        k_frag_emit<32, Probe, NonId><<<grid_for(n_bags, kThreads / 32, 2 * cap), kThreads, 0, stream>>>(
+            b->indices, b->offsets, B, T, S, d_perm, d_counts, scan, table_base, probe, pop->offsets, pop->ids,
+            pop->cap_ids, non_offsets, non_ids, non_cap, status);
+    if (d_dense)
+        k_permute_dense<<<grid_for((int64_t)B * n_dense, kThreads, cap), kThreads, 0, stream>>>(d_dense, B, n_dense,
+                                                                                              d_perm, d_dense_out);
+    note_launches(d_dense ? 2 : 1);   // emit (+ dense permutation)
+    HL_LAUNCH_CHECK();
+    return HL_OK;
+}
+
+}  // namespace
+}  // namespace hl
+
 extern "C" int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_dense, int32_t n_dense,
                                int32_t* d_perm, int32_t* d_counts, hl_ubatch* pop, hl_ubatch* non,
                                float* d_dense_out, void* stream_) {
@@ -235,40 +282,23 @@ extern "C" int32_t hl_fragment(hl_ctx* ctx, const hl_batch* b, const float* d_de
         return HL_EINVAL;
     if (!pop->offsets || !non->offsets || (b->nnz > 0 && (!pop->ids || !non->ids))) return HL_EINVAL;
     if ((d_dense == nullptr) != (d_dense_out == nullptr) || (d_dense && n_dense < 1)) return HL_EINVAL;
-    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     Regions& r = ctx->r;
-    const int B = b->batch, T = ctx->T, S = ctx->S;
-    const int64_t n_bags = (int64_t)T * B * S;
-    const bool short_bags = b->nnz <= 4 * (int64_t)T * B;   // on average at most 4 lookups per input and table
+    return fragment_launch<BitmapProbe, int32_t>(b, ctx->T, ctx->S, ctx_sms(ctx), r.table_base, BitmapProbe{r.remap},
+                                                 r.frag_flags, r.frag_scan, r.frag_tiles, r.status, wait_cfg(ctx),
+                                                 d_dense, n_dense, d_perm, d_counts, pop, non->offsets, non->ids,
+                                                 non->cap_ids, d_dense_out, static_cast<cudaStream_t>(stream_));
+}
 
-    const int cap = 4 * ctx_sms(ctx);      // CTAs of every kernel here: they stride over their work
-    const int flag_grid = grid_for(B, kThreads / 32, 2 * cap);
-    if (short_bags)
-        k_frag_flags<true><<<flag_grid, kThreads, 0, stream>>>(b->indices, b->offsets, B, T, S, r.table_base,
-                                                               r.remap, r.frag_flags, r.status);
-    else
-        k_frag_flags<false><<<flag_grid, kThreads, 0, stream>>>(b->indices, b->offsets, B, T, S, r.table_base,
-                                                                r.remap, r.frag_flags, r.status);
-    k_frag_partition<<<1, 1024, 0, stream>>>(r.frag_flags, B, d_perm, d_counts);
-    k_frag_sizes<<<grid_for(n_bags, kThreads, cap), kThreads, 0, stream>>>(b->offsets, B, T, S, d_perm,
-                                                                               d_counts, r.frag_scan);
-    note_launches(3);   // flags, partition, sizes
-    HL_LAUNCH_CHECK();
-    int32_t st = exclusive_scan_i32(r.frag_scan, r.frag_scan, nullptr, n_bags, r.frag_tiles, r.status, stream,
-                                    wait_cfg(ctx));
-    if (st != HL_OK) return st;
-    if (b->nnz <= 4 * n_bags)
-        k_frag_emit<1><<<grid_for(n_bags, kThreads, cap), kThreads, 0, stream>>>(
-            b->indices, b->offsets, B, T, S, d_perm, d_counts, r.frag_scan, r.table_base, r.remap, pop->offsets,
-            pop->ids, pop->cap_ids, non->offsets, non->ids, non->cap_ids, r.status);
-    else
-        k_frag_emit<32><<<grid_for(n_bags, kThreads / 32, 2 * cap), kThreads, 0, stream>>>(
-            b->indices, b->offsets, B, T, S, d_perm, d_counts, r.frag_scan, r.table_base, r.remap, pop->offsets,
-            pop->ids, pop->cap_ids, non->offsets, non->ids, non->cap_ids, r.status);
-    if (d_dense)
-        k_permute_dense<<<grid_for((int64_t)B * n_dense, kThreads, cap), kThreads, 0, stream>>>(
-            d_dense, B, n_dense, d_perm, d_dense_out);
-    note_launches(d_dense ? 2 : 1);   // emit (+ dense permutation)
-    HL_LAUNCH_CHECK();
-    return HL_OK;
+extern "C" int32_t hl_wide_fragment(hl_wide* w, const hl_batch* b, int32_t* d_perm, int32_t* d_counts, hl_ubatch* pop,
+                                    int32_t* d_non_offsets, int64_t* d_non_rows, int64_t non_cap, void* stream_) {
+    if (!w || !b || !d_perm || !d_counts || !pop || !d_non_offsets) return HL_EINVAL;
+    if (b->batch < 1 || b->batch > w->max_batch || b->nnz < 0 || b->nnz > w->max_nnz || !b->offsets ||
+        (b->nnz > 0 && !b->indices))
+        return HL_EINVAL;
+    if (!pop->offsets || (b->nnz > 0 && (!pop->ids || !d_non_rows))) return HL_EINVAL;
+    const HashProbe probe{w->r_keys, w->r_vals, (uint64_t)(w->remap_slots - 1)};
+    return fragment_launch<HashProbe, long long>(b, w->T, w->S, w->sms, w->table_base, probe, w->frag_flags,
+                                                 w->frag_scan, w->frag_tiles, w->status, WaitCfg(), nullptr, 0, d_perm,
+                                                 d_counts, pop, d_non_offsets, reinterpret_cast<long long*>(d_non_rows),
+                                                 non_cap, nullptr, static_cast<cudaStream_t>(stream_));
 }

@@ -314,6 +314,29 @@ __global__ void __launch_bounds__(kThreads) k_remap_dense(const RemapBlock* __re
 int32_t launch_gather_rows(hl_ctx* ctx, float* dst, int64_t dst_row0, const float* table, const int32_t* rows,
                            const int64_t* d_n, int64_t n_max, int32_t* status, cudaStream_t stream);
 
+
+// The rows [0, n) whose counts are among the k largest (count >= 1, and count * share_den >= total * share_num if
+// share_num > 0; sel->total holds the total), ties at the threshold going to the smaller index; their indices, in
+// ascending order, to out_idx [cap], their number to *d_n_out.  sel_gt / sel_eq: div_up(n, kSelTile) + 2 words each.
+int32_t select_rows_by_count(const uint32_t* counts, int64_t n, SelectState* sel, uint32_t* sel_gt, uint32_t* sel_eq,
+                             long long k, long long share_num, long long share_den, int64_t cap, int32_t* out_idx,
+                             int64_t* d_n_out, int32_t* status, int sms, cudaStream_t stream) {
+    const int64_t n_tiles = div_up(n, kSelTile);
+    k_select_begin<<<1, 256, 0, stream>>>(sel, (unsigned long long)k, share_num, share_den);
+    const int grid = grid_for(n, kThreads * 16, sms * 8);
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        k_select_hist<<<grid, kThreads, 0, stream>>>(counts, n, shift, sel);
+        k_select_pick<<<1, 256, 0, stream>>>(sel, shift);
+    }
+    k_select_tile_counts<<<(unsigned)n_tiles, kThreads, 0, stream>>>(counts, n, sel, sel_gt, sel_eq);
+    k_select_spine<<<1, 1024, 0, stream>>>(sel_gt, sel_eq, n_tiles);
+    k_select_emit<<<(unsigned)n_tiles, kThreads, 0, stream>>>(counts, n, sel, sel_gt, sel_eq, n_tiles, cap, out_idx,
+                                                             d_n_out, status);
+    note_launches(12);   // begin, 4 x (histogram, pick), tile counts, spine, emit
+    HL_LAUNCH_CHECK();
+    return HL_OK;
+}
+
 }  // namespace hl
 
 using namespace hl;
@@ -359,19 +382,8 @@ extern "C" int32_t hl_profile_hot(hl_ctx* ctx, const hl_batch* b, int32_t reset,
         }
         if (k < 0) return HL_EINVAL;
         if (k > ctx->hot_cap) k = ctx->hot_cap;
-        k_select_begin<<<1, 256, 0, stream>>>(r.sel, (unsigned long long)k, share_num, share_den);
-        const int grid = grid_for(ctx->N, kThreads * 16, ctx_sms(ctx) * 8);
-        for (int shift = 24; shift >= 0; shift -= 8) {
-            k_select_hist<<<grid, kThreads, 0, stream>>>(r.counts, ctx->N, shift, r.sel);
-            k_select_pick<<<1, 256, 0, stream>>>(r.sel, shift);
-        }
-        const unsigned tiles = (unsigned)ctx->n_sel_tiles;
-        k_select_tile_counts<<<tiles, kThreads, 0, stream>>>(r.counts, ctx->N, r.sel, r.sel_gt, r.sel_eq);
-        k_select_spine<<<1, 1024, 0, stream>>>(r.sel_gt, r.sel_eq, ctx->n_sel_tiles);
-        k_select_emit<<<tiles, kThreads, 0, stream>>>(r.counts, ctx->N, r.sel, r.sel_gt, r.sel_eq, ctx->n_sel_tiles,
-                                                      ctx->hot_cap, d_hot_rows, d_n_hot, r.status);
-        note_launches(12);   // begin, 4 x (histogram, pick), tile counts, spine, emit
-        HL_LAUNCH_CHECK();
+        return select_rows_by_count(r.counts, ctx->N, r.sel, r.sel_gt, r.sel_eq, k, share_num, share_den, ctx->hot_cap,
+                                    d_hot_rows, d_n_hot, r.status, ctx_sms(ctx), stream);
     }
     return HL_OK;
 }

@@ -218,6 +218,30 @@ def test_fragment_degenerate_hot_sets():
     assert check_fragment(ind2, off2, B, tr, S, []) == empty_inputs
 
 
+def test_fragment_and_cold_rows_keep_64_bit_row_ids_beyond_2_to_31():
+    """Two tables with 2^31 + 90 rows together: the second table's rows have global ids that do not fit 32 bits.
+    X's row ids, the cold rows and the unified slots against values worked out with Python integers."""
+    tr = (2 ** 31 - 10, 100)
+    N = sum(tr)
+    B = 4
+    # table 0: indices near both ends; table 1: every global id is >= 2^31 - 10
+    ind = np.array([5, 2 ** 31 - 11, 7, 5, 0, 99, 50, 99], dtype=np.int32)
+    off = np.arange(9, dtype=np.int32)
+    hot = np.array([5, 2 ** 31 - 10 + 99], dtype=np.int64)          # one popular row per table
+    remap = orc.build_remap(hot, N)
+    perm, n_pop, O, X, _ = orc.fragment(ind, off, B, tr, remap, 1)
+    # inputs: 0 -> rows (5, base+0), 1 -> (2^31-11, base+99), 2 -> (7, base+50), 3 -> (5, base+99): only input 3 is popular
+    base1 = 2 ** 31 - 10
+    assert perm.tolist() == [3, 0, 1, 2] and n_pop == 1
+    assert O.ids.tolist() == [0, 1]
+    assert X.ids.dtype == np.int64
+    assert [int(v) for v in X.ids] == [5, 2 ** 31 - 11, 7, base1 + 0, base1 + 99, base1 + 50]
+    C, slots = orc.gather_cold(X.ids, remap, 2)
+    assert [int(v) for v in C] == [7, 2 ** 31 - 11, base1 + 0, base1 + 50]
+    assert slots.tolist() == [0, 3, 2, 4, 1, 5]
+    del remap
+
+
 def test_fragment_dense_rows_follow_perm():
     rng = np.random.default_rng(8)
     tr, B = (5, 5), 9
