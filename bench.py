@@ -33,11 +33,6 @@ L2_BYTES = 126 << 20
 FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
 SINGLE_ALLOCATION_LIMIT = 64 << 30  # a larger host table is held as one allocation per table
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the forward kernel per bag at dim 64, from the ncu capture
-# summarised in profiles/k_embbag_fwd_micro_dim64.md (164.4 MB for 425,984 one-lookup bags).  The bench's own
-# launch is scaled from it by the number of bags it processes (traffic grows in proportion to the bags).
-NCU_FWD_TRAFFIC_BYTES_PER_BAG = {64: 164.4e6 / 425984}
-
 
 def log(*a):
     print(*a, file=sys.stderr, flush=True)
@@ -1025,7 +1020,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
 
 
 # ----------------------------------------------------------------------------------------------------------
-# single-call micro runs (the small cases the ncu captures under profiles/ are taken on)
+# single-call micro runs (small cases: one library call in isolation, sized for a profiler capture)
 # ----------------------------------------------------------------------------------------------------------
 def run_micro_gather(args) -> None:
     """`--micro gather`: the row-move kernel alone, host table -> HBM, 65,536 rows of 256 bytes from a 16 GiB

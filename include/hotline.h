@@ -132,8 +132,9 @@ HL_API int32_t hl_timing_read(hl_ctx* ctx, int32_t which, float* ms);
  * memory with the CPU as preferred location and the device advised to map it, which the device maps in large pages;
  * memory from cudaHostAlloc also works as a table but is mapped in 4 KB pages, and random rows of a table of tens of
  * GB then pay an address-translation miss each.  If unified memory refuses the size -- on the bench platform a single
- * allocation stops between 66 and 70 GB -- the call falls back to such memory.)  The caller owns it and frees it
- * with hl_host_free.  Returns NULL on failure. */
+ * allocation stops between 66 and 70 GB -- the call falls back to such memory; a larger table is better held as one
+ * allocation per table, see hl_set_host_tables.)  The caller owns it and frees it with hl_host_free.  Returns NULL on
+ * failure. */
 HL_API void* hl_host_alloc(size_t bytes);
 HL_API int32_t hl_host_free(void* p);
 
@@ -168,7 +169,8 @@ HL_API int32_t hl_set_kernel_width(hl_ctx* ctx, int32_t fwd_ctas_per_sm, int32_t
  * poll_limit = 0 restores production behaviour.  Nothing here can hang or fault the device. */
 HL_API int32_t hl_test_bounded_waits(hl_ctx* ctx, int32_t poll_limit, int64_t stall_tile);
 
-/* Number of kernels this library has launched in this process so far (all contexts). */
+/* Number of kernels this library has launched from the host in this process so far (all contexts; the general cold-row
+ * search that a kernel launches from the device is not counted). */
 HL_API uint64_t hl_launch_count(void);
 
 /* ---------------------------------------------------------------------------------------------------------
@@ -348,13 +350,14 @@ HL_API int32_t hl_index_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non
                              int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold,
                              const int32_t* d_prev_cold_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
                              void* stream);
-/* hl_index_cold in two halves, for a scheduler that can put other work between them.  hl_index_cold_begin classifies
- * X's lookups and, if there are at most 20 480 cold ones, finds the distinct rows and assigns the slots at once; it
- * leaves a verdict in the device word hl_index_cold_verdict(ctx): 0 = done, else the number of cold lookups.
- * hl_index_cold_end does the rest (the general search, whose kernels find nothing to do after a verdict of 0, and the
- * match against the previous cold rows); general_not_needed != 0 = the caller has read a verdict of 0 and spares the
- * general search's launches.  Same arguments as hl_index_cold; both halves on one stream, nothing else of this
- * context's cold-row search between them. */
+/* hl_index_cold in two halves.  hl_index_cold_begin classifies X's lookups and finds the distinct cold rows and the
+ * slots: with at most 20 480 cold lookups one thread-block cluster does all of it in one kernel; with more, that
+ * kernel launches the general search (tile sort, head flags, scan, assignment) from the device, behind itself and
+ * ahead of whatever the host queued next -- so the host queues the same two kernels for every mini-batch and never
+ * needs to know the count.  The device word hl_index_cold_verdict(ctx) says afterwards which it was: 0 = the cluster
+ * kernel, else the number of cold lookups handed on.  hl_index_cold_end does the match against the previous cold rows
+ * (general_not_needed is ignored; it dates from when the host queued the general search).  Same arguments as
+ * hl_index_cold; both halves on one stream, nothing else of this context's cold-row search between them. */
 HL_API int32_t hl_index_cold_begin(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, int64_t stage_row0,
                                    int64_t stage_rows, int32_t* d_cold_rows, int64_t* d_n_cold, void* stream);
 HL_API const int32_t* hl_index_cold_verdict(hl_ctx* ctx);

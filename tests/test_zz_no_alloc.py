@@ -4,9 +4,9 @@ Some users of the library cannot allocate device memory at all (a plug-in inside
 GPU's memory, a loop that must stay out of the allocator), so they cannot give the library a workspace.  For them
 the library carries a fixed scratch array in its own image.  This test calls that entry point through the C
 boundary twice in a row, with different shapes, and checks each result against hl_embbag_bwd_sgd on the same
-inputs (and against the CPU oracle).  It lives in a file that pytest collects last, so that a run stopping at
-the first failure has already been through every other test; it sets up everything it needs itself, so it also
-passes when run alone in a fresh process.
+inputs (and against the CPU oracle).  The second call finds the first call's data still in the array, which is the
+case the entry point has to cope with; the test creates every buffer and context it uses, so it does not depend on
+what ran before it.
 """
 import numpy as np
 import pytest
