@@ -198,14 +198,19 @@ __global__ void __launch_bounds__(kThreads) k_bwd_pairs(const int32_t* __restric
 
 // The sorted lookups are cut into chunks of kBwdChunk.  One group per chunk sums, in order, the gradient rows of
 // each run of equal slots inside its chunk.  A run that lies wholly inside the chunk is finished here (one
-// read-modify-write of its row).  A run that crosses a chunk border leaves a partial sum: part[chunk][0] for the
+// reduction into its row).  A run that crosses a chunk border leaves a partial sum: part[chunk][0] for the
 // piece that continues a run from the previous chunk, part[chunk][1] for the piece that starts a run continuing
 // into the next chunk.  k_bwd_spans adds those up.
 //
-// The group reads its chunk's 32 (slot, bag) pairs with one coalesced load per lane and passes them round by
-// shuffles, so that all gradient-row addresses are known at once; gradient rows are then loaded U at a time,
-// together with the cache row of every run that starts among those U lookups (the row is needed only when the
-// run closes, but asking for it up front takes its latency off the critical path).
+// The group reads its chunk's 32 (slot, bag) pairs with one coalesced load per lane.  Where runs begin and end is
+// then settled once for the whole chunk: every lane compares its pairs' slots with their neighbours' (shuffles, the
+// slots just outside the chunk for the ends) and two ballots per 32 pairs give a mask of run heads and a mask of
+// run tails.  The loop over the lookups is driven by those two masks alone, and a lookup costs two shuffles, one
+// address, one 128-bit load per column and the additions; everything that checks a pair (position inside the call,
+// bag inside the gradient array) is done by the lane that loaded the pair, once.  Gradient rows are loaded U at a
+// time.  The instruction count matters: this kernel issues about as many cycles as it waits for memory.
+static_assert(kBwdChunk == 32, "the head and tail masks of a chunk are 32-bit words");
+
 template <int G, int NV>
 __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float* __restrict__ cache,
                                                          const int32_t* __restrict__ keys,
@@ -226,12 +231,25 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
     const int64_t n = first + d_n_lookups[0];
     const int lane = threadIdx.x & 31;
     const int sub = lane % G;
-    const unsigned gmask = G == 32 ? 0xffffffffu : (((1u << G) - 1u) << (lane / G * G));
+    const unsigned gshift = G == 32 ? 0u : (unsigned)(lane / G * G);
+    constexpr unsigned gbits = G == 32 ? 0xffffffffu : ((1u << G) - 1u);
+    const unsigned gmask = gbits << gshift;
     const int64_t group = ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
     const int64_t n_groups = (int64_t)gridDim.x * kThreads / G;
-    const float4* __restrict__ grad4 = reinterpret_cast<const float4*>(grad_out);
     float4* cache4 = reinterpret_cast<float4*>(cache);
     float4* __restrict__ part4 = reinterpret_cast<float4*>(part);
+    // slots and bags are 32-bit numbers, so one unsigned comparison tells whether one lies inside its array
+    const uint32_t n_rows_u = (uint32_t)(n_slots < 0x7fffffff ? n_slots : 0x7fffffff);
+    const uint32_t n_grad_u = (uint32_t)(n_grad_rows < 0x7fffffff ? n_grad_rows : 0x7fffffff);
+    // this lane's columns; a lane beyond the row's width reads column 0 and writes nothing
+    bool on[NV];
+    const float4* gcol[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c = sub + v * G;
+        on[v] = c < D4;
+        gcol[v] = reinterpret_cast<const float4*>(grad_out) + (on[v] ? c : 0);
+    }
 
     for (int64_t chunk = group; first + chunk * kBwdChunk < n; chunk += n_groups) {
         const int64_t start = first + chunk * kBwdChunk;
@@ -240,74 +258,86 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
 #pragma unroll
         for (int i = 0; i < KPL; ++i) {
             const int64_t p = start + i * G + sub;
-            kk[i] = p < end ? keys[p] : -1;
-            vv[i] = p < end ? vals[p] : 0;
+            const bool in = p < end;
+            kk[i] = in ? keys[p] : -1;                       // -1: past the end; no slot has this key
+            const int32_t bag = in ? vals[p] : 0;
+            // (a bag id outside the gradient array can only be what a given-up chain poll of the sort left behind;
+            // such a call has its error status set, and reads bag 0 instead)
+            vv[i] = (uint32_t)bag < n_grad_u ? bag : 0;
         }
         const int32_t prev_key = start > first ? keys[start - 1] : -3;   // -3: equal to no key
         const int32_t next_key = end < n ? keys[end] : -2;
 
-        int32_t cur = prev_key;        // slot of the segment being summed
-        bool seg_left_open = true;     // it continues a run from the previous chunk (until the slot changes)
-        int seg_count = 0;             // lookups of this chunk summed into it so far
+        // bit q of `heads`: lookup q of the chunk begins a run; of `tails`: it ends one
+        uint32_t heads = 0, tails = 0;
+#pragma unroll
+        for (int i = 0; i < KPL; ++i) {
+            const int32_t up = __shfl_up_sync(gmask, kk[i], 1, G);
+            const int32_t dn = __shfl_down_sync(gmask, kk[i], 1, G);
+            const int32_t before = i > 0 ? __shfl_sync(gmask, kk[i > 0 ? i - 1 : 0], G - 1, G) : prev_key;
+            const int32_t after = i + 1 < KPL ? __shfl_sync(gmask, kk[i + 1 < KPL ? i + 1 : i], 0, G) : next_key;
+            const int32_t pred = sub > 0 ? up : before;
+            const int32_t succ = sub < G - 1 ? dn : after;
+            const uint32_t hb = (__ballot_sync(gmask, kk[i] != pred) >> gshift) & gbits;
+            const uint32_t tb = (__ballot_sync(gmask, kk[i] != succ) >> gshift) & gbits;
+            heads |= hb << (i * G);
+            tails |= tb << (i * G);
+        }
+
+        // the run being summed continues one from the previous chunk until the first head
+        bool left_open = true;
         // a segment's sum is kept in fp64: a popular row can collect tens of thousands of gradient rows, and the
         // rounding of many fp32 partial sums would show in the updated row
         double acc[NV][4];
 #pragma unroll
         for (int v = 0; v < NV; ++v) acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0.0;
 
-        auto flush = [&](bool right_open) {
-            const int64_t row = (int64_t)cur - key_bias;
-            if (seg_count == 0 || row < 0 || row >= n_slots) return;   // nothing summed, or a skipped lookup's sentinel
-            if (!seg_left_open && !right_open) {
+        // the run whose last lookup in this chunk has key `key` is complete in acc
+        auto emit = [&](int32_t key, bool right_open) {
+            const uint32_t row = (uint32_t)(key - key_bias);
+            if (row >= n_rows_u) return;                     // a skipped lookup's sentinel, or past the end
+            if (!left_open && !right_open) {
 #pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    const int c = sub + v * G;
-                    if (c < D4)
-                        red_add_f4(&cache4[row * D4 + c],
+                for (int v = 0; v < NV; ++v)
+                    if (on[v])
+                        red_add_f4(&cache4[(int64_t)row * D4 + sub + v * G],
                                    make_float4(-(lr * (float)acc[v][0]), -(lr * (float)acc[v][1]),
                                                -(lr * (float)acc[v][2]), -(lr * (float)acc[v][3])));
-                }
             } else {
-                const int64_t slot = chunk * 2 + (seg_left_open ? 0 : 1);
+                const int64_t slot = chunk * 2 + (left_open ? 0 : 1);
 #pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    const int c = sub + v * G;
-                    if (c < D4)
-                        part4[slot * D4 + c] =
+                for (int v = 0; v < NV; ++v)
+                    if (on[v])
+                        part4[slot * D4 + sub + v * G] =
                             make_float4((float)acc[v][0], (float)acc[v][1], (float)acc[v][2], (float)acc[v][3]);
+                if (right_open && !left_open && sub == 0) {
+                    const int32_t pos = atomicAdd(span_count, 1);
+                    span_list[2 * pos] = (int32_t)chunk;
+                    span_list[2 * pos + 1] = key;
                 }
             }
         };
 
 #pragma unroll
         for (int i = 0; i < KPL; ++i) {
+            // (kept rolled: with all 32 lookups unrolled the kernel is tens of KB of straight-line code that every
+            // warp runs through about once, and it waits for instructions)
+#pragma unroll 1
             for (int j = 0; j < G; j += U) {
-                int32_t k[U], b[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    k[u] = __shfl_sync(gmask, kk[i], j + u, G);
-                    b[u] = __shfl_sync(gmask, vv[i], j + u, G);
-                }
+                int32_t k[U];
                 float4 g[U][NV];
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    const int64_t row = (int64_t)k[u] - key_bias;
-                    // (a bag id outside the gradient array can only be what a given-up chain poll of the sort left behind)
-                    const bool ok = k[u] >= 0 && row >= 0 && row < n_slots && b[u] >= 0 && b[u] < n_grad_rows;
+                    k[u] = __shfl_sync(gmask, kk[i], j + u, G);
+                    const int32_t bag = __shfl_sync(gmask, vv[i], j + u, G);
 #pragma unroll
-                    for (int v = 0; v < NV; ++v) {
-                        const int c = sub + v * G;
-                        g[u][v] = (ok && c < D4) ? __ldg(&grad4[(int64_t)b[u] * D4 + c]) : f4_zero();
-                    }
+                    for (int v = 0; v < NV; ++v) g[u][v] = __ldg(gcol[v] + (int64_t)bag * D4);
                 }
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
-                    if (k[u] < 0) continue;   // past the end of the last chunk
-                    if (k[u] != cur) {
-                        flush(false);
-                        cur = k[u];
-                        seg_left_open = false;
-                        seg_count = 0;
+                    const int q = i * G + j + u;
+                    if ((heads >> q) & 1u) {
+                        left_open = false;
 #pragma unroll
                         for (int v = 0; v < NV; ++v) acc[v][0] = acc[v][1] = acc[v][2] = acc[v][3] = 0.0;
                     }
@@ -318,19 +348,13 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
                         acc[v][2] += (double)g[u][v].z;
                         acc[v][3] += (double)g[u][v].w;
                     }
-                    ++seg_count;
+                    if ((tails >> q) & 1u) emit(k[u], false);
                 }
             }
         }
-        flush(next_key == cur);
-        if (sub == 0 && next_key == cur && !seg_left_open && seg_count > 0) {
-            const int64_t row = (int64_t)cur - key_bias;
-            if (row >= 0 && row < n_slots) {
-                const int32_t pos = atomicAdd(span_count, 1);
-                span_list[2 * pos] = (int32_t)chunk;
-                span_list[2 * pos + 1] = cur;
-            }
-        }
+        // the chunk's last lookup does not end its run: the run goes on in the next chunk (only a full chunk has a
+        // next one)
+        if (!((tails >> (kBwdChunk - 1)) & 1u)) emit(__shfl_sync(gmask, kk[KPL - 1], G - 1, G), true);
     }
 }
 
