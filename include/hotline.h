@@ -351,7 +351,8 @@ HL_API int32_t hl_index_cold(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non
                              const int32_t* d_prev_cold_rows, const int64_t* d_n_prev, int32_t* d_fwd_src,
                              void* stream);
 /* hl_index_cold in two halves.  hl_index_cold_begin classifies X's lookups and finds the distinct cold rows and the
- * slots: with at most 20 480 cold lookups one thread-block cluster does all of it in one kernel; with more, that
+ * slots: with at most 40 960 cold lookups (20 480 on a device that cannot place a cluster of 16 CTAs) one
+ * thread-block cluster does all of it in one kernel; with more, that
  * kernel launches the general search (tile sort, head flags, scan, assignment) from the device, behind itself and
  * ahead of whatever the host queued next -- so the host queues the same two kernels for every mini-batch and never
  * needs to know the count.  The device word hl_index_cold_verdict(ctx) says afterwards which it was: 0 = the cluster

@@ -94,22 +94,21 @@ __global__ void __launch_bounds__(kThreads) k_cold_assign(const int32_t* __restr
 }
 
 // ---- few cold lookups: one thread-block cluster does sort, distinct-row ranking and slot assignment ----------------
-// With at most kSmallCap cold lookups (a DLRM-large mini-batch has about 18 K) the chain of radix passes, head
-// flags, scan and assignment -- nine launches that each take longer to start than to run -- is one kernel of one
-// cluster of 8 CTAs.  CTA c owns positions [c * kSmallPerCta, (c + 1) * kSmallPerCta) of the list.  Every pass ranks
+// With at most CTAS * kSmallPerCta cold lookups (a DLRM-large mini-batch has about 18 K) the chain of radix passes,
+// head flags, scan and assignment -- nine launches that each take longer to start than to run -- is one kernel of
+// one cluster of CTAS CTAs: 16 (40 960 lookups; a cluster size the kernel has to opt in to) where the device can
+// place such a cluster, else 8 (20 480).  CTA c owns positions [c * kSmallPerCta, (c + 1) * kSmallPerCta) of the list.  Every pass ranks
 // the pairs, held in registers, by one digit (per-warp digit counters, as in the tile kernel of the general sort),
-// adds up the digit counts of the 8 CTAs through distributed shared memory, and writes each pair into the shared
+// adds up the digit counts of the cluster's CTAs through distributed shared memory, and writes each pair into the shared
 // memory of the CTA that owns its new position.  The sorted list is then ranked and assigned in place.
 // Order of a CTA's items: position = warp * (32 * kSmallItems) + round * 32 + lane.
 // Larger inputs: the kernel launches the general path itself (tile sort, head flags, scan, assignment) as tail
 // launches, which run after this grid and before anything the host queued behind it -- so the host queues the same
 // two kernels for every mini-batch and never needs to know which path ran.  *d_n_general = the number of cold lookups
 // handed to the general path (0: none).
-constexpr int kSmallCtas = 8;
 constexpr int kSmallThreads = 256;
 constexpr int kSmallItems = 10;
 constexpr int kSmallPerCta = kSmallThreads * kSmallItems;       // 2560
-constexpr int kSmallCap = kSmallCtas * kSmallPerCta;            // 20480
 constexpr int kSmallWarps = kSmallThreads / 32;
 
 // what the general path works on (device pointers into the context's cold region)
@@ -152,6 +151,7 @@ __device__ __forceinline__ int block_scan_small(int v, int* smem33, int& total) 
     return res;
 }
 
+template <int CTAS>
 __global__ void __launch_bounds__(kSmallThreads) k_cold_small(const int32_t* __restrict__ keys_in,
                                                               const int32_t* __restrict__ vals_in,
                                                               const int32_t* __restrict__ d_n, int64_t n_max,
@@ -173,7 +173,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_cold_small(const int32_t* __r
     int64_t n64 = d_n[0];
     n64 = n64 < 0 ? 0 : (n64 < n_max ? n64 : n_max);
     const int cta = (int)cluster.block_rank();
-    if (n64 > kSmallCap) {                   // the same decision in all CTAs, before any cluster barrier
+    if (n64 > CTAS * kSmallPerCta) {         // the same decision in all CTAs, before any cluster barrier
         if (cta == 0 && threadIdx.x == 0) {
             d_n_general[0] = (int32_t)n64;
             // the general path, queued behind this grid: stable sort of the (row, position) pairs by row, a flag at
@@ -237,7 +237,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_cold_small(const int32_t* __r
             const int d = threadIdx.x;
             uint32_t before_me = 0, all_ctas = 0;
 #pragma unroll
-            for (int c = 0; c < kSmallCtas; ++c) {
+            for (int c = 0; c < CTAS; ++c) {
                 const uint32_t v = *cluster.map_shared_rank(&cta_hist[d], c);
                 if (c < cta) before_me += v;
                 all_ctas += v;
@@ -285,7 +285,7 @@ __global__ void __launch_bounds__(kSmallThreads) k_cold_small(const int32_t* __r
     cluster.sync();
     int distinct = 0;
 #pragma unroll
-    for (int c = 0; c < kSmallCtas; ++c) {
+    for (int c = 0; c < CTAS; ++c) {
         const int v = *cluster.map_shared_rank(&cta_heads, c);
         if (c < cta) rank += v;
         distinct += v;
@@ -654,18 +654,38 @@ int32_t index_begin(hl_ctx* ctx, hl_ubatch* non, const int32_t* d_n_non, int64_t
     ga.cap_ids = non->cap_ids;
     ga.key_bits = key_bits;
     ga.max_polls = wait_cfg(ctx).max_polls;
+    // the widest cluster the device can place: 16 CTAs (a non-portable size) or 8; asked once per context
+    if (ctx->cold_cluster == 0) {
+        ctx->cold_cluster = 8;
+        cudaLaunchConfig_t probe = {};
+        probe.gridDim = dim3(16);
+        probe.blockDim = dim3(kSmallThreads);
+        cudaLaunchAttribute pa[1];
+        pa[0].id = cudaLaunchAttributeClusterDimension;
+        pa[0].val.clusterDim.x = 16;
+        pa[0].val.clusterDim.y = pa[0].val.clusterDim.z = 1;
+        probe.attrs = pa;
+        probe.numAttrs = 1;
+        int clusters = 0;
+        if (cudaFuncSetAttribute(k_cold_small<16>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+            cudaOccupancyMaxActiveClusters(&clusters, k_cold_small<16>, &probe) == cudaSuccess && clusters >= 1)
+            ctx->cold_cluster = 16;
+        (void)cudaGetLastError();
+    }
+    const int ctas = ctx->cold_cluster;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(kSmallCtas);
+    cfg.gridDim = dim3(ctas);
     cfg.blockDim = dim3(kSmallThreads);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = kSmallCtas;
+    attr[0].val.clusterDim.x = ctas;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    HL_CUDA_TRY(cudaLaunchKernelEx(&cfg, k_cold_small, (const int32_t*)r.cold_keys[0], (const int32_t*)r.cold_vals[0],
+    HL_CUDA_TRY(cudaLaunchKernelEx(&cfg, ctas == 16 ? k_cold_small<16> : k_cold_small<8>,
+                                   (const int32_t*)r.cold_keys[0], (const int32_t*)r.cold_vals[0],
                                    (const int32_t*)r.cold_n, ctx->max_nnz, (key_bits + 7) / 8,
                                    ctx->hot_cap + stage_row0, stage_rows, non->ids, d_cold_rows, d_n_cold,
                                    r.cold_n + 1, r.status, ga));

@@ -82,6 +82,7 @@ struct hl_ctx {
     int sms;                           // multiprocessors of `device` (queried at hl_create)
     int mover_ctas, scatter_ctas;      // working CTAs of the host-link movers inside a schedule (hl_set_mover_ctas)
     int fwd_ctas, bwd_ctas;            // CTAs per multiprocessor of the forward / backward-sum kernel (0 = default)
+    int cold_cluster;                  // CTAs of the one-cluster cold-row search (0 = not asked yet; 8 or 16)
     int test_poll_limit;               // > 0: poll limit of the bounded device waits (hl_test_bounded_waits)
     int64_t test_stall_tile;           // with it: the tile / mover stage that never delivers (-1: none)
     int64_t* h_table_base;             // host copy [T+1]

@@ -41,10 +41,11 @@ def test_arbitrary_hot_sets(hot):
         assert stats["n_non"] == 0 and stats["n_cold"] == 0
 
 
-@pytest.mark.parametrize("batch", [2559, 2560, 2561, 3000])
+@pytest.mark.parametrize("batch", [2559, 2560, 2561, 3000, 5119, 5120, 5121, 6000])
 def test_cold_row_search_at_the_limit_of_its_one_cluster_path(batch):
-    """Empty hot set, 8 tables: every lookup is cold, 8 * batch of them.  20 480 is the most the one-cluster kernel
-    takes; one more and the general path (tile sort, head flags, scan, assignment) does the work."""
+    """Empty hot set, 8 tables: every lookup is cold, 8 * batch of them.  The one-cluster kernel takes at most 40 960
+    (a cluster of 16 CTAs; 20 480 where the device places only 8); one more and the general path (tile sort, head
+    flags, scan, assignment), launched from the device, does the work."""
     spec = dataclasses.replace(gen.CONFIGS["tiny"], batch=batch, hot_policy=("topk", 80_000))
     stats = run_config_check(spec, steps=2, hot_override="empty", integer=True)
     assert stats["n_pop"] == 0 and stats["n_cold"] > 5_000        # distinct rows; the lookups are 8 * batch
