@@ -46,3 +46,20 @@ def test_single_rank_helpers():
     import bench
     assert bench.max_over_ranks([1.5, 2.5], 1) == [1.5, 2.5]
     assert abs(bench.whole_job_value(16384, 100, 1, 64.6) - 16384 * 100 / 0.0646) < 1e-3
+
+
+def test_reference_arm_under_two_ranks_runs_on_rank_zero_alone():
+    """`bench.py --impl reference` launched as two ranks: rank 0 times the oracle and prints the one JSON line, the
+    other rank leaves with exit code 0 and prints nothing; neither loads the CUDA library."""
+    import json
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1")
+    out = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+                          "--master-addr", "127.0.0.1", "--master-port", "29733", os.path.join(ROOT, "bench.py"),
+                          "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "3", "--workload", "tiny"],
+                         capture_output=True, text=True, env=env, timeout=600, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    res = json.loads(lines[0])
+    assert res["impl"] == "reference" and res["n_gpus"] == 2 and res["value"] > 0
+    assert res["cpu_baseline"]["kind"] == "oracle" and res["e2e"]["h2d_bytes_per_step"] == 0
