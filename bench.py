@@ -1154,6 +1154,116 @@ def run_micro_tracker(args) -> None:
     print(json.dumps(res), flush=True)
 
 
+def run_micro_wide(args) -> None:
+    """`--micro wide`: the index part of the path (learning phase, remap, fragment, cold-row search) through the
+    wide-id calls (64-bit row ids, hashed counter, hashed remap) next to the same calls of the 32-bit path (dense
+    counter, bitmap remap) on the same mini-batches of the chosen workload: time per call, CUDA events, and the
+    outputs of the two paths compared (popular set, perm, counts, cold rows)."""
+    import torch
+    import paper_2204_05436_b200 as hl
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    n_timed = 8
+    wl = Workload("dlrm_large" if args.workload in (None, "auto") else args.workload,
+                  1.0 if args.row_scale is None else args.row_scale, n_timed, args.profile_batches or 64, dev,
+                  args.threads, with_table=False)
+    spec, geom = wl.spec, wl.geom
+    T, D, S, B, N, P = wl.T, wl.D, wl.S, wl.B, wl.N, wl.P
+    n_bags, max_nnz, hot_cap, staging = wl.n_bags, wl.max_nnz, wl.hot_cap, wl.staging_cap
+    stream = torch.cuda.current_stream().cuda_stream
+    i32, i64 = torch.int32, torch.int64
+    batches = wl.profile + wl.batches
+    d_in = [(torch.from_numpy(b.indices).to(dev), torch.from_numpy(b.offsets).to(dev)) for b in batches]
+    policy, p_num, p_den = wl.policy_args()
+
+    def batch_of(i):
+        return hl.make_batch(d_in[i][0], d_in[i][1], B, int(d_in[i][0].numel()))
+
+    def timed(fn):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3
+
+    z = lambda n, dt: torch.zeros(max(1, n), dtype=dt, device=dev)   # noqa: E731
+    # ---- 32-bit path ----
+    g = hl.make_geometry(geom.table_rows, D, S)
+    ws_bytes = hl.hl_workspace_bytes(g, B, max_nnz, hot_cap, staging)
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    ctx = hl.hl_create(g, B, max_nnz, hot_cap, staging, ws, ws_bytes)
+    hot32, n_hot32 = z(hot_cap, i32), z(1, i64)
+    perm, counts = z(B, i32), z(4, i32)
+    pop_off, pop_ids = z(n_bags + 1, i32), z(max_nnz, i32)
+    non_off, non_ids = z(n_bags + 1, i32), z(max_nnz, i32)
+    cold32, n_cold32 = z(staging, i32), z(1, i64)
+    pop, non = hl.make_ubatch(pop_off, pop_ids, max_nnz), hl.make_ubatch(non_off, non_ids, max_nnz)
+    t32 = {"profile": [timed(lambda i=i: hl.hl_profile_hot(ctx, batch_of(i), int(i == 0), 0, 0, 0, 1, hot32, n_hot32,
+                                                           stream)) for i in range(P)]}
+    t32["select"] = [timed(lambda: hl.hl_profile_hot(ctx, None, 0, 1, policy, p_num, p_den, hot32, n_hot32, stream))]
+    t32["remap"] = [timed(lambda: hl.hl_build_remap(ctx, hot32, n_hot32, None, None, None, stream))]
+    t32["fragment"], t32["index_cold"], out32 = [], [], []
+    for rep in range(3):
+        for i in range(P, P + n_timed):
+            t32["fragment"].append(timed(lambda i=i: hl.hl_fragment(ctx, batch_of(i), None, 0, perm, counts, pop, non,
+                                                                    None, stream)))
+            t32["index_cold"].append(timed(lambda: hl.hl_index_cold(ctx, non, counts[1:], 0, staging, cold32, n_cold32,
+                                                                    None, None, None, stream)))
+            if rep == 0:
+                nc = int(n_cold32.item())
+                out32.append((perm.clone(), counts.clone(), cold32[:nc].to(i64).clone()))
+    hl.hl_status(ctx)
+    n_hot = int(n_hot32.item())
+    hot32_rows = hot32[:n_hot].to(i64).clone()
+    hl.hl_destroy(ctx)
+    del ws
+    # ---- wide path ----
+    seen = int(torch.unique(torch.cat([_global_rows(torch, geom, B, S, idx, off, dev) for idx, off in d_in[:P]])).numel())
+    counter_slots = 1 << max(16, (4 * seen - 1).bit_length())
+    wws_bytes = hl.hl_wide_workspace_bytes(g, B, max_nnz, hot_cap, staging, counter_slots)
+    wws = torch.empty(wws_bytes, dtype=torch.uint8, device=dev)
+    w = hl.hl_wide_create(g, B, max_nnz, hot_cap, staging, counter_slots, wws, wws_bytes)
+    hot64, n_hot64 = z(hot_cap, i64), z(1, i64)
+    non_rows, non_slots = z(max_nnz, i64), z(max_nnz, i32)
+    cold64, n_cold64 = z(staging, i64), z(1, i64)
+    tw = {"profile": [timed(lambda i=i: hl.hl_wide_profile_hot(w, batch_of(i), i == 0, False, 0, 0, 1, 4 * D, hot64,
+                                                               n_hot64, stream)) for i in range(P)]}
+    tw["select"] = [timed(lambda: hl.hl_wide_profile_hot(w, None, False, True, policy, p_num, p_den, 4 * D, hot64,
+                                                         n_hot64, stream))]
+    tw["remap"] = [timed(lambda: hl.hl_wide_build_remap(w, hot64, n_hot64, stream))]
+    tw["fragment"], tw["index_cold"] = [], []
+    same = int(n_hot64.item()) == n_hot and bool(torch.equal(hot64[:n_hot], hot32_rows))
+    for rep in range(3):
+        for k, i in enumerate(range(P, P + n_timed)):
+            tw["fragment"].append(timed(lambda i=i: hl.hl_wide_fragment(w, batch_of(i), perm, counts, pop, non_off,
+                                                                        non_rows, max_nnz, stream)))
+            tw["index_cold"].append(timed(lambda: hl.hl_wide_index_cold(w, non_off, non_rows, max_nnz, counts[1:],
+                                                                        non_slots, cold64, n_cold64, stream)))
+            if rep == 0:
+                nc = int(n_cold64.item())
+                same = same and bool(torch.equal(perm, out32[k][0]) and torch.equal(counts, out32[k][1])
+                                     and torch.equal(cold64[:nc], out32[k][2]))
+    hl.hl_wide_status(w)
+    hl.hl_wide_destroy(w)
+    med = lambda d: {k: round(statistics.median(v), 2) for k, v in d.items()}   # noqa: E731
+    print(json.dumps({"micro": "wide", "workload": spec.name, "total_rows": N, "profile_mini_batches": P,
+                      "lookups_per_mini_batch": int(d_in[0][0].numel()), "distinct_rows_seen": seen,
+                      "counter_slots": counter_slots, "hot_rows": n_hot,
+                      "cold_rows_per_mini_batch": round(statistics.mean(int(o[2].numel()) for o in out32), 1),
+                      "us_per_call_32bit": med(t32), "us_per_call_wide": med(tw),
+                      "same_results": same}), flush=True)
+
+
+def _global_rows(torch, geom, B, S, idx, off, dev):
+    """Global row id (table base + index) of every lookup of a table-major mini-batch."""
+    base = torch.from_numpy(np.concatenate([[0], np.cumsum(geom.table_rows)]).astype(np.int64)).to(dev)
+    n_bags = geom.num_tables * B * S
+    sizes = (off[1:] - off[:-1]).to(torch.int64)
+    table = torch.arange(n_bags, device=dev) // (B * S)
+    return base[torch.repeat_interleave(table, sizes)] + idx.to(torch.int64)
+
+
 def run_micro(args) -> None:
     """`--micro fwd|bwd`: one library call in isolation on an all-popular ("hot-only") micro-batch with the
     DLRM-large-like shape (26 tables x `--micro-batch` inputs, dim 64, one lookup per bag) over a 1 GiB cache.
@@ -1421,7 +1531,7 @@ def main() -> None:
     ap.add_argument("--bwd-ctas", type=int, default=0, help="hl_set_kernel_width: backward-sum CTAs per multiprocessor")
     ap.add_argument("--timeline", default=None,
                     help="write the per-stream timeline of three mini-batches of the traced pass to this text file")
-    ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather", "tracker"],
+    ap.add_argument("--micro", default=None, choices=["fwd", "bwd", "gather", "tracker", "wide"],
                     help="time one library call in isolation")
     ap.add_argument("--micro-dist", default="uniform", choices=["uniform", "zipf"])
     ap.add_argument("--micro-batch", type=int, default=16384)
@@ -1433,6 +1543,9 @@ def main() -> None:
         return
     if args.micro == "tracker":
         run_micro_tracker(args)
+        return
+    if args.micro == "wide":
+        run_micro_wide(args)
         return
     if args.micro == "gather":
         run_micro_gather(args)
