@@ -297,9 +297,16 @@ constexpr int64_t sort_hist_words(int64_t max_nnz) {
     return 4 * 256 + 8 + 4 * n_tiles * 256;   // digit counts, tickets, tile status words for up to 4 passes
 }
 
-// ints behind the backward's partial sums: count words + (chunk, key) per chunk of kBwdChunk sorted lookups.
+// ints behind the backward's partial sums: count words + (chunk, key, last chunk of the run or -1, unused) per chunk
+// of kBwdChunk sorted lookups.
 constexpr int64_t bwd_span_list_words(int64_t max_nnz) {
-    return 8 + 2 * (((max_nnz > 0 ? max_nnz : 1) + kBwdChunk - 1) / kBwdChunk);
+    return 8 + 4 * (((max_nnz > 0 ? max_nnz : 1) + kBwdChunk - 1) / kBwdChunk);
+}
+
+// where those ints start
+inline int32_t* span_count_of(const hl_ctx* ctx) {
+    const int64_t max_chunks = ((ctx->max_nnz > 0 ? ctx->max_nnz : 1) + kBwdChunk - 1) / kBwdChunk;
+    return reinterpret_cast<int32_t*>(ctx->r.bwd_part + 2 * max_chunks * ctx->D);
 }
 
 // ints of scratch exclusive_scan_i32 needs for at most n_max elements (64-bit ticket + status words).

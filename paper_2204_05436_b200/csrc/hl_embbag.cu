@@ -310,10 +310,20 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
                     if (on[v])
                         part4[slot * D4 + sub + v * G] =
                             make_float4((float)acc[v][0], (float)acc[v][1], (float)acc[v][2], (float)acc[v][3]);
-                if (right_open && !left_open && sub == 0) {
-                    const int32_t pos = atomicAdd(span_count, 1);
-                    span_list[2 * pos] = (int32_t)chunk;
-                    span_list[2 * pos + 1] = key;
+                if (right_open && !left_open) {
+                    // a run starts here and goes on: list it, with its last chunk if that is among the next G (chunk
+                    // c > chunk holds a piece of the run iff its first slot is the run's; sorted keys: those chunks
+                    // form a prefix).  Nearly every run ends there, and k_bwd_spans then has nothing to search.
+                    const int64_t n_chunks = (n - first + kBwdChunk - 1) / kBwdChunk;
+                    const int64_t cc = chunk + 1 + sub;
+                    const bool goes_on = cc < n_chunks && keys[first + cc * kBwdChunk] == key;
+                    const uint32_t m = (__ballot_sync(gmask, goes_on) >> gshift) & gbits;
+                    const int cnt = __ffs((int)~m) - 1;      // m == gbits (all G go on): -1 for G == 32, else G
+                    if (sub == 0) {
+                        const int32_t pos = atomicAdd(span_count, 1);
+                        reinterpret_cast<int4*>(span_list)[pos] =
+                            make_int4((int32_t)chunk, key, (cnt >= 1 && cnt < G) ? (int32_t)(chunk + cnt) : -1, 0);
+                    }
                 }
             }
         };
@@ -365,18 +375,18 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
 // occur), the group sums are combined by shuffles in a fixed order, and group 0 applies the single SGD update of the
 // row.  Longer runs (a popular row can own hundreds of chunks) are queued in shared memory and then summed by the
 // whole CTA, every group taking every (8 * 32/G)-th piece, the group sums combined in a fixed order by one group.
-constexpr int kLongRun = 48;
+constexpr int kLongRun = 32;
 
 template <int G, int NV>
 __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cache, const int32_t* __restrict__ keys,
                                                         const int32_t* __restrict__ d_n_lookups, int D4,
                                                         int64_t n_slots, float lr, const float* __restrict__ part,
                                                         const int32_t* __restrict__ d_first, int32_t key_bias,
-                                                        const int32_t* __restrict__ span_count,
-                                                        const int32_t* __restrict__ span_list) {
+                                                        int32_t* span_count,
+                                                        const int32_t* __restrict__ span_list, int64_t max_entries) {
     constexpr int GW = 32 / G;   // groups per warp
     constexpr int kWarps = kThreads / 32;
-    constexpr int U = NV >= 4 ? 2 : 4;   // partial sums in flight per lane (most runs end in the next chunk)
+    constexpr int U = NV >= 4 ? 2 : (NV >= 2 ? 4 : 8);   // partial sums in flight per lane
     constexpr int UC = 8;                // the same in the CTA-wide sum
     constexpr bool kCtaPath = NV == 1;   // the CTA-wide sum keeps one float4 column per lane
     __shared__ int64_t q_chunk[kWarps], q_last[kWarps], q_row[kWarps];
@@ -391,6 +401,7 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
 
     int64_t n_owned = span_count[0];     // chunks in which a run starts that goes on into the next chunk
     n_owned = n_owned < 0 ? 0 : (n_owned < n_chunks ? n_owned : n_chunks);
+    n_owned = n_owned < max_entries ? n_owned : max_entries;
 
     // every warp of the CTA makes the same number of trips (there are block barriers inside)
     for (int64_t base = (int64_t)blockIdx.x * kWarps; base < n_owned; base += (int64_t)gridDim.x * kWarps) {
@@ -398,12 +409,15 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
         bool mine = false;
         int32_t key = 0;
         int64_t chunk = 0, row = 0, last_chunk = 0;
+        int64_t known_last = -1;
         if (base + wib < n_owned) {
-            const int2 e = reinterpret_cast<const int2*>(span_list)[base + wib];     // (chunk, slot key of the run)
+            // (chunk, slot key of the run, its last chunk if the sum kernel has found it)
+            const int4 e = reinterpret_cast<const int4*>(span_list)[base + wib];
             chunk = e.x;
             key = e.y;
             row = (int64_t)key - key_bias;
             mine = chunk >= 0 && chunk + 1 < n_chunks && row >= 0 && row < n_slots;
+            if (e.z > e.x && e.z < n_chunks) known_last = e.z;
         }
         // the run's first piece is asked for now; it is needed after the search
         float4 piece0[NV];
@@ -416,7 +430,10 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
         if (mine) {
             // last chunk that holds a piece of the run: chunk c > chunk holds one iff its first slot is the run's
             int64_t lo = chunk + 1, hi = n_chunks;      // chunk lo holds a piece, chunk hi (if any) does not
-            {
+            if (known_last >= 0) {
+                lo = known_last;
+                hi = known_last + 1;
+            } else {
                 const int64_t cc = lo + 1 + lane;       // the 32 chunks after lo
                 const bool t = cc < hi && keys[first + cc * kBwdChunk] == key;
                 const unsigned m = __ballot_sync(0xffffffffu, t);
@@ -534,6 +551,17 @@ __global__ void __launch_bounds__(kThreads) k_bwd_spans(float* __restrict__ cach
             __syncthreads();     // every warp has read the whole queue before any warp clears its entry again
         }
     }
+    // The list is empty again for the next call: the last CTA to get here clears the count (word 0) and the tally of
+    // finished CTAs (word 2).  Every CTA read the count when it started, and the next call's kernels start after this
+    // grid has ended.
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int32_t finished = atomicAdd(&span_count[2], 1);
+        if (finished == (int32_t)gridDim.x - 1) {
+            span_count[0] = 0;
+            span_count[2] = 0;
+        }
+    }
 }
 
 template <int G, int NV>
@@ -562,17 +590,18 @@ int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t
     const int grid = grid_for(max_chunks * G, kThreads, bwd_ctas_per_sm(ctx) * ctx_sms(ctx));
     const int64_t n_slots = ctx->hot_cap + ctx->staging_cap;
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 0, stream);
-    // the list of chunks whose run goes on sits behind the partial sums: [count (8 ints)] [chunk ids]
-    int32_t* span_count = reinterpret_cast<int32_t*>(ctx->r.bwd_part + 2 * max_chunks * ctx->D);
+    // the list of runs that cross a chunk border sits behind the partial sums: [count words (8 ints)] [entries].
+    // The count is zero between calls: hl_create clears it and k_bwd_spans clears it again when it is done.
+    int32_t* span_count = span_count_of(ctx);
     int32_t* span_list = span_count + 8;
-    HL_CUDA_TRY(cudaMemsetAsync(span_count, 0, 8 * sizeof(int32_t), stream));
     k_bwd_chunks<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, vals, d_n_lookups, grad, ctx->D / 4, n_slots,
                                                       lr, ctx->r.bwd_part, d_first, key_bias, span_count, span_list,
                                                       ctx->max_bags);
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 1, stream);
     const int span_grid = grid_for(max_chunks * 32, kThreads, 4 * ctx_sms(ctx));   // the warps stride over the listed runs
     k_bwd_spans<G, NV><<<span_grid, kThreads, 0, stream>>>(cache, keys, d_n_lookups, ctx->D / 4, n_slots, lr,
-                                                          ctx->r.bwd_part, d_first, key_bias, span_count, span_list);
+                                                          ctx->r.bwd_part, d_first, key_bias, span_count,
+                                                          (const int32_t*)span_list, max_chunks);
     note_launches(2);
     HL_LAUNCH_CHECK();
     return HL_OK;
@@ -795,9 +824,12 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 std::mutex g_static_mutex;
 unsigned char* g_static_ptr[64] = {};   // device address of g_static_scratch, per device ordinal
 
-__global__ void k_static_begin(int32_t* header, int32_t n_bags) {
+__global__ void k_static_begin(int32_t* header, int32_t n_bags, int32_t* span_count) {
     header[0] = 0;        // status word: every call starts clean
     header[8] = n_bags;   // the backward kernels read their bag count from device memory
+    // the count words of the backward's run list: their place in the array depends on the call's sizes, so an earlier
+    // call may have left partial sums there
+    for (int i = 0; i < 8; ++i) span_count[i] = 0;
 }
 
 __global__ void k_static_end(const int32_t* header, int32_t* d_status) { *d_status = header[0]; }
@@ -860,7 +892,7 @@ extern "C" int32_t hl_embbag_bwd_sgd_static(float* d_cache, int64_t cache_rows, 
     p += kStaticHistBytes;
     tmp.r.bwd_part = reinterpret_cast<float*>(p);
 
-    k_static_begin<<<1, 1, 0, stream>>>(header, n_bags);
+    k_static_begin<<<1, 1, 0, stream>>>(header, n_bags, span_count_of(&tmp));
     note_launches(1);
     HL_LAUNCH_CHECK();
     hl_ubatch ub{const_cast<int32_t*>(d_offsets), const_cast<int32_t*>(d_ids), nnz};
