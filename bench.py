@@ -469,7 +469,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                                       order=args.order, main_priority=args.main_priority,
                                       index_priority=args.index_priority, link_priority=args.link_priority,
                                       mover_ctas=args.mover_ctas, scatter_ctas=args.scatter_ctas,
-                                      exclusive_write_back=args.exclusive_write_back)
+                                      write_back=args.write_back)
     elif pipelined:
         h = hl.PipelinedHotline(wl.geom.table_rows, D, S, B, wl.max_nnz, wl.hot_cap, wl.staging_cap, wl.table,
                                 n_dense=wl.spec.n_dense, device=str(device), overlap_link=not args.serial_link,
@@ -953,6 +953,7 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
                 "stream_priorities": {"main": args.main_priority, "index": args.index_priority,
                                       "link": args.link_priority},
                 "mover_ctas": {"read": args.mover_ctas or "default", "write": args.scatter_ctas or "default"},
+                "write_back": args.write_back,
                 "replicas": "independent replica per GPU, no collective"}),
             "clocks": clock_info, "gpu_launches": int(launches), "host_enqueue_us_per_step": host_enqueue_us,
             "launches_per_step": launches / args.steps,
@@ -1525,8 +1526,8 @@ def main() -> None:
     ap.add_argument("--link-priority", type=int, default=0, help="CUDA priority of the host-link transfer streams")
     ap.add_argument("--mover-ctas", type=int, default=0, help="hl_set_mover_ctas: CTAs of the host reads (0 = default)")
     ap.add_argument("--scatter-ctas", type=int, default=0, help="hl_set_mover_ctas: CTAs of the write-backs")
-    ap.add_argument("--exclusive-write-back", action="store_true",
-                    help="a mini-batch's main work waits for the previous write-back (hl_pipe_options)")
+    ap.add_argument("--write-back", choices=("overlap", "exclusive", "after_forward"), default="overlap",
+                    help="hl_pipe_options.write_back: when a mini-batch's write-back runs")
     ap.add_argument("--fwd-ctas", type=int, default=0, help="hl_set_kernel_width: forward CTAs per multiprocessor")
     ap.add_argument("--bwd-ctas", type=int, default=0, help="hl_set_kernel_width: backward-sum CTAs per multiprocessor")
     ap.add_argument("--timeline", default=None,

@@ -149,8 +149,9 @@ HL_API int32_t hl_set_host_tables(hl_ctx* ctx, float* const* h_table_bases);
 
 /* Width of the host-link movers inside a schedule: how many CTAs of hl_gather_cold / hl_stage_cold (read_ctas) and of
  * hl_scatter_cold (write_ctas) work when a mini-batch moves a DLRM-sized number of rows (the kernels decide on the
- * device, from the number of rows, whether more join in).  0 = the default (16); at most two per multiprocessor.
- * Wider movers finish sooner and slow the kernels that run beside them more.  Takes effect with the next call. */
+ * device, from the number of rows, whether more join in).  0 = the default (24 for reads, 16 for write-backs); at
+ * most two per multiprocessor.  Wider movers finish sooner and slow the kernels that run beside them more.  Takes
+ * effect with the next call. */
 HL_API int32_t hl_set_mover_ctas(hl_ctx* ctx, int32_t read_ctas, int32_t write_ctas);
 
 /* Grid size of the two bandwidth-bound kernels, in CTAs per multiprocessor: the forward kernel (hl_embbag_fwd) and
@@ -422,11 +423,18 @@ HL_API hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_table, i
 typedef struct {
     int32_t index_priority;          /* the three streams of index-only ahead-work (fragment, cold-row search, sort) */
     int32_t link_priority;           /* the two streams of host-link transfers (host read, write-back)              */
-    int32_t exclusive_write_back;    /* != 0: the main work of mini-batch j starts only when the write-back of j - 1 has
-                                        finished, so that no bandwidth-bound kernel runs beside a write-back (which
-                                        slows such a kernel several times over); the index-only ahead-work and the
-                                        host read still overlap it                                                   */
+    int32_t write_back;              /* HL_PIPE_WB_x: when the write-back of mini-batch j runs                       */
 } hl_pipe_options;
+/* HL_PIPE_WB_OVERLAP (default): as soon as j's backward is over, beside the main work of j + 1.
+ * HL_PIPE_WB_EXCLUSIVE: the same, and the main work of j + 1 starts only when it has finished, so that no
+ *   bandwidth-bound kernel runs beside a write-back (the index-only ahead-work and the host read still do).
+ * HL_PIPE_WB_AFTER_FORWARD: when the popular forward of j + 1 is over (the kernel of the main stream that loses most
+ *   next to a write-back); hl_pipe_step then holds j's write-back over until the next hl_pipe_step, or until
+ *   hl_pipe_wait_outputs / hl_pipe_drain, whichever comes first (the last step of a run, the one without a next
+ *   mini-batch, queues it at once).  The results are the same in all three. */
+#define HL_PIPE_WB_OVERLAP       0
+#define HL_PIPE_WB_EXCLUSIVE     1
+#define HL_PIPE_WB_AFTER_FORWARD 2
 HL_API hl_pipe* hl_pipe_create_ex(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows, int32_t n_sets,
                                   const hl_pipe_set* sets, int32_t n_dense, void* main_stream,
                                   const hl_pipe_options* options);

@@ -60,7 +60,7 @@ class hl_pipe_set(ctypes.Structure):
 
 class hl_pipe_options(ctypes.Structure):
     _fields_ = [("index_priority", ctypes.c_int32), ("link_priority", ctypes.c_int32),
-                ("exclusive_write_back", ctypes.c_int32)]
+                ("write_back", ctypes.c_int32)]
 
 
 class hl_pipe_span(ctypes.Structure):
@@ -459,11 +459,11 @@ def hl_pipe_create(ctx: int, d_cache, host_table, window_rows: int, sets, n_dens
 
 
 def hl_pipe_create_ex(ctx: int, d_cache, host_table, window_rows: int, sets, n_dense: int, main_stream: int,
-                      index_priority: int = 0, link_priority: int = 0, exclusive_write_back: bool = False) -> int:
+                      index_priority: int = 0, link_priority: int = 0, write_back: int = 0) -> int:
     """hl_pipe_create with its options: the stream priorities of the ahead-work and of the host-link transfers, and
-    whether a mini-batch's main work waits for the previous write-back."""
+    when a mini-batch's write-back runs (HL_PIPE_WB_*)."""
     arr = (hl_pipe_set * len(sets))(*sets)
-    opt = hl_pipe_options(int(index_priority), int(link_priority), int(bool(exclusive_write_back)))
+    opt = hl_pipe_options(int(index_priority), int(link_priority), int(write_back))
     p = _lib.hl_pipe_create_ex(ctx, _ptr(d_cache), _ptr(host_table), int(window_rows), len(sets), arr, int(n_dense),
                                main_stream, ctypes.byref(opt))
     if not p:
@@ -628,6 +628,7 @@ def hl_index_cold_end(ctx: int, non: hl_ubatch, stage_row0: int, stage_rows: int
 
 
 HL_PIPE_ORDER_FIG8, HL_PIPE_ORDER_EQ5 = 0, 1
+HL_PIPE_WB_OVERLAP, HL_PIPE_WB_EXCLUSIVE, HL_PIPE_WB_AFTER_FORWARD = 0, 1, 2
 
 
 def hl_embbag_bwd_prepare_merged(ctx: int, pop: hl_ubatch, d_n_pop, non: hl_ubatch, d_n_non, d_sorted_slots,

@@ -122,7 +122,8 @@ extern "C" int32_t hl_create(hl_ctx** out, const hl_geometry* geom, int32_t max_
         free(ctx);
         return HL_ECUDA;
     }
-    ctx->mover_ctas = ctx->scatter_ctas = kMoverCtasDefault;
+    ctx->mover_ctas = kReadCtasDefault;
+    ctx->scatter_ctas = kMoverCtasDefault;
     ctx->test_poll_limit = 0;
     ctx->test_stall_tile = -1;
     ctx->h_table_base = static_cast<int64_t*>(malloc(sizeof(int64_t) * (ctx->T + 1)));
@@ -167,7 +168,7 @@ extern "C" int32_t hl_set_host_tables(hl_ctx* ctx, float* const* h_table_bases) 
 extern "C" int32_t hl_set_mover_ctas(hl_ctx* ctx, int32_t read_ctas, int32_t write_ctas) {
     if (!ctx || read_ctas < 0 || write_ctas < 0) return HL_EINVAL;
     const int most = 2 * ctx_sms(ctx);
-    ctx->mover_ctas = read_ctas == 0 ? kMoverCtasDefault : (read_ctas < most ? read_ctas : most);
+    ctx->mover_ctas = read_ctas == 0 ? kReadCtasDefault : (read_ctas < most ? read_ctas : most);
     ctx->scatter_ctas = write_ctas == 0 ? kMoverCtasDefault : (write_ctas < most ? write_ctas : most);
     return HL_OK;
 }

@@ -428,7 +428,7 @@ constexpr int kBulkStagesPerCta = 16;     // stages of rows per working CTA befo
 // next to the other streams' kernels.  More CTAs move the rows faster (about 100 us with 2 per SM, alone), fewer
 // slower (one CTA writes back 64 rows every 3.4 us), but what the transfers cost the kernels that run next to them
 // does not depend on that.  (The hot-cache load of hl_build_remap and hl_flush_hot, which run alone, use 2 CTAs per
-// SM and reach 90 % of the memcpy rate.)  The default, kMoverCtasDefault, is set at hl_create.
+// SM and reach 90 % of the memcpy rate.)  The defaults, kReadCtasDefault and kMoverCtasDefault, are set at hl_create.
 
 // What a launch of the mover needs to know about its context.
 struct MoveCfg {

@@ -15,7 +15,8 @@ constexpr int kSortTile = 2048;            // keys per radix-sort tile (256 thre
 constexpr int kScanTile = 2048;            // elements per scan tile (256 threads x 8)
 constexpr int kSelTile = 4096;             // rows per hot-set selection tile (256 threads x 16)
 constexpr int kBwdChunk = 32;              // sorted lookups per backward chunk
-constexpr int kMoverCtasDefault = 16;      // working CTAs of a host-link mover inside a schedule
+constexpr int kMoverCtasDefault = 16;      // working CTAs of a host-link mover inside a schedule: write-backs
+constexpr int kReadCtasDefault = 24;       // ... and host reads (a wider read finishes sooner and costs the step nothing)
 // Per-mini-batch kernels are launched with one CTA per tile of work rather than as chip-filling persistent grids:
 // they run next to the host-link movers of another micro-batch, which slow down the SMs they sit on, and the
 // hardware block scheduler then simply hands those SMs fewer CTAs.

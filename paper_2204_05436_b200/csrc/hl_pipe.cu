@@ -25,14 +25,15 @@ struct hl_pipe {
     std::vector<hl_pipe_set> sets;
     cudaStream_t main, sa, sb, sc, link, wb;
     struct Events {
-        cudaEvent_t inputs, frag, index, prep, gather, forward, x, scatter;
+        cudaEvent_t inputs, frag, index, prep, gather, forward, x, scatter, fwd_pop;
     };
     std::vector<Events> ev;
     // mini-batches whose fragment + first half of the cold-row search are queued (begun), whose cold-row search and
     // sort are queued in full (indexed), whose host read is queued (submitted), whose main work is queued (done)
     int64_t j_begun, j_indexed, j_submitted, j_done;
     int order;                   // HL_PIPE_ORDER_*
-    int exclusive_wb;            // main work of j waits for the write-back of j - 1
+    int wb_mode;                 // HL_PIPE_WB_*
+    bool wb_pending;             // HL_PIPE_WB_AFTER_FORWARD: the write-back of mini-batch j_done - 1 is not queued yet
     // trace (hl_pipe_trace_begin / _end): one event pair per recorded span
     struct Span {
         cudaEvent_t b, e;
@@ -188,6 +189,28 @@ int32_t submit_link(hl_pipe* p) {
     return HL_OK;
 }
 
+// the write-back of mini-batch j (whose main work is queued), behind its backward
+int32_t queue_scatter(hl_pipe* p, int64_t j) {
+    const int n = p->n_sets;
+    hl_pipe_set& st = p->sets[j % n];
+    hl_pipe::Events& e = p->ev[j % n];
+    const int64_t w0 = (j % 2) * p->window_rows;
+    HL_PIPE_TRY(wait(p->wb, e.x));
+    {
+        Scope sc(p, HL_SPAN_SCATTER, j, kWb);
+        HL_PIPE_TRY(hl_scatter_cold_at(p->ctx, p->cache, w0, p->window_rows, st.cold_rows, st.n_cold, p->host_table,
+                                       p->wb));
+    }
+    return record(e.scatter, p->wb);
+}
+
+// HL_PIPE_WB_AFTER_FORWARD: the write-back held over from the previous hl_pipe_step, if there is one
+int32_t flush_scatter(hl_pipe* p) {
+    if (!p->wb_pending) return HL_OK;
+    p->wb_pending = false;
+    return queue_scatter(p, p->j_done - 1);
+}
+
 }  // namespace
 
 extern "C" hl_pipe* hl_pipe_create_ex(hl_ctx* ctx, float* d_cache, float* host_table, int64_t window_rows,
@@ -203,6 +226,7 @@ extern "C" hl_pipe* hl_pipe_create_ex(hl_ctx* ctx, float* d_cache, float* host_t
             return nullptr;
         if (ctx->max_nnz > 0 && (!s.pop.ids || !s.non.ids || !s.sorted_slots || !s.sorted_bags)) return nullptr;
     }
+    if (opt && (opt->write_back < HL_PIPE_WB_OVERLAP || opt->write_back > HL_PIPE_WB_AFTER_FORWARD)) return nullptr;
     hl_pipe* p = new (std::nothrow) hl_pipe();
     if (!p) return nullptr;
     p->ctx = ctx;
@@ -215,7 +239,8 @@ extern "C" hl_pipe* hl_pipe_create_ex(hl_ctx* ctx, float* d_cache, float* host_t
     p->main = static_cast<cudaStream_t>(main_stream);
     p->j_begun = p->j_indexed = p->j_submitted = p->j_done = 0;
     p->order = HL_PIPE_ORDER_FIG8;
-    p->exclusive_wb = opt ? opt->exclusive_write_back : 0;
+    p->wb_mode = opt ? opt->write_back : HL_PIPE_WB_OVERLAP;
+    p->wb_pending = false;
     p->n_spans = 0;
     p->trace_mask = 0;
     p->cur_mb = 0;
@@ -234,7 +259,8 @@ extern "C" hl_pipe* hl_pipe_create_ex(hl_ctx* ctx, float* d_cache, float* host_t
     }
     p->ev.resize(n_sets);
     for (auto& e : p->ev) {
-        cudaEvent_t* all[8] = {&e.inputs, &e.frag, &e.index, &e.prep, &e.gather, &e.forward, &e.x, &e.scatter};
+        cudaEvent_t* all[9] = {&e.inputs, &e.frag,    &e.index, &e.prep,   &e.gather,
+                               &e.forward, &e.x,      &e.scatter, &e.fwd_pop};
         for (auto x : all) {
             *x = nullptr;
             ok = ok && cudaEventCreateWithFlags(x, cudaEventDisableTiming) == cudaSuccess;
@@ -299,7 +325,7 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
     const int64_t w0 = (j % 2) * p->window_rows, w1 = ((j + 1) % 2) * p->window_rows;
     if (next && p->j_begun - j >= n - 1) return HL_ECAPACITY;
     HL_PIPE_TRY(wait(p->main, e.index));
-    if (p->exclusive_wb && j >= 1) HL_PIPE_TRY(wait(p->main, p->ev[(j - 1) % n].scatter));
+    if (p->wb_mode == HL_PIPE_WB_EXCLUSIVE && j >= 1) HL_PIPE_TRY(wait(p->main, p->ev[(j - 1) % n].scatter));
     if (j >= 1) {
         // rows shared with mini-batch j-1 come out of its staging window once its backward is done
         HL_PIPE_TRY(wait(p->link, e.index));
@@ -308,10 +334,19 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
         HL_PIPE_TRY(hl_forward_cold(p->ctx, p->cache, w1, w0, p->window_rows, st.fwd_src, st.n_cold, p->link));
     }
     HL_PIPE_TRY(record(e.forward, p->link));
-    if (p->j_submitted < p->j_indexed) HL_PIPE_TRY(submit_link(p));         // mini-batch j+1, if indexed in full
+    // (the host read of j+1 waits for the write-back of j-1, so it is queued behind a write-back that was held over)
+    if (!p->wb_pending && p->j_submitted < p->j_indexed) HL_PIPE_TRY(submit_link(p));   // j+1, if indexed in full
     {
         Scope sc(p, HL_SPAN_FWD_POP, j, kMain);
         HL_PIPE_TRY(hl_embbag_fwd(p->ctx, p->cache, &st.pop, st.counts, st.pooled_pop, p->main));
+    }
+    if (p->wb_pending) {
+        // the write-back of j-1 starts when the popular forward of j is over: of all kernels of the main stream that
+        // one loses most next to a write-back
+        HL_PIPE_TRY(record(e.fwd_pop, p->main));
+        HL_PIPE_TRY(wait(p->wb, e.fwd_pop));
+        HL_PIPE_TRY(flush_scatter(p));
+        if (p->j_submitted < p->j_indexed) HL_PIPE_TRY(submit_link(p));
     }
     if (p->order == HL_PIPE_ORDER_FIG8) {
         HL_PIPE_TRY(wait(p->main, e.prep));
@@ -336,13 +371,11 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
                                         lr, p->main));
     }
     HL_PIPE_TRY(record(e.x, p->main));
-    HL_PIPE_TRY(wait(p->wb, e.x));
-    {
-        Scope sc(p, HL_SPAN_SCATTER, j, kWb);
-        HL_PIPE_TRY(hl_scatter_cold_at(p->ctx, p->cache, w0, p->window_rows, st.cold_rows, st.n_cold, p->host_table,
-                                       p->wb));
-    }
-    HL_PIPE_TRY(record(e.scatter, p->wb));
+    p->j_done += 1;
+    if (p->wb_mode == HL_PIPE_WB_AFTER_FORWARD && next)
+        p->wb_pending = true;            // queued by the next hl_pipe_step (or by whatever call comes instead)
+    else
+        HL_PIPE_TRY(queue_scatter(p, j));
     HL_PIPE_TRY(finish_index(p));
     if (p->j_submitted == j + 1 && p->j_submitted < p->j_indexed) HL_PIPE_TRY(submit_link(p));   // mini-batch j+1
     if (next) {
@@ -353,7 +386,6 @@ extern "C" int32_t hl_pipe_step(hl_pipe* p, const float* d_grad_pop, const float
         }
     }
     if (set_index) *set_index = (int32_t)(j % n);
-    p->j_done += 1;
     return HL_OK;
 }
 
@@ -429,6 +461,7 @@ extern "C" int32_t hl_pipe_wait_outputs(hl_pipe* p, void* stream) {
     // makes `stream` wait for the last write-back issued (the main stream's own work it sees in order)
     if (!p) return HL_EINVAL;
     if (p->j_done == 0) return HL_OK;
+    HL_PIPE_TRY(flush_scatter(p));
     return wait(static_cast<cudaStream_t>(stream), p->ev[(p->j_done - 1) % p->n_sets].scatter);
 }
 
@@ -441,6 +474,7 @@ extern "C" int32_t hl_pipe_wait_counts(hl_pipe* p, void* stream) {
 
 extern "C" int32_t hl_pipe_drain(hl_pipe* p) {
     if (!p) return HL_EINVAL;
+    HL_PIPE_TRY(flush_scatter(p));
     cudaStream_t all[6] = {p->main, p->sa, p->sb, p->sc, p->link, p->wb};
     for (auto s : all)
         if (cudaStreamSynchronize(s) != cudaSuccess) return HL_ECUDA;

@@ -588,15 +588,20 @@ class NativePipelinedHotline(Hotline):
     def __init__(self, table_rows, dim, bags_per_sample, max_batch, max_nnz, hot_cap_rows, window_rows, host_table,
                  n_dense: int = 0, device: str = "cuda:0", lookahead: int = 2, order: str = "fig8",
                  main_priority: int = -1, index_priority: int = 0, link_priority: int = 0, mover_ctas: int = 0,
-                 scatter_ctas: int = 0, exclusive_write_back: bool = False):
+                 scatter_ctas: int = 0, write_back: str = "overlap"):
         """``order``: "fig8" = forward O, update O, forward X, update X (the paper's Fig. 8); "eq5" = both forwards,
         then one update of every touched row with the whole mini-batch's gradient (Eq. 5; the unfragmented step's
         result): step() then takes ``grad_pop`` = [gradients of O's bags; gradients of X's bags] and no ``grad_non``.
         ``main_priority`` / ``index_priority`` / ``link_priority``: CUDA stream priorities (0 = default, negative =
         higher) of the main stream (bandwidth-bound forwards and updates), of the index-only ahead-work and of the
         host-link transfers.  ``mover_ctas`` / ``scatter_ctas``: hl_set_mover_ctas (0 = the library's default).
-        ``exclusive_write_back``: a mini-batch's main work waits for the previous mini-batch's write-back."""
+        ``write_back``: when a mini-batch's write-back runs: "overlap" = right after its backward, beside the next
+        mini-batch's main work; "exclusive" = the same, and the next mini-batch's main work waits for it;
+        "after_forward" = when the next mini-batch's popular forward is over."""
         assert order in ("fig8", "eq5")
+        wb_modes = {"overlap": B.HL_PIPE_WB_OVERLAP, "exclusive": B.HL_PIPE_WB_EXCLUSIVE,
+                    "after_forward": B.HL_PIPE_WB_AFTER_FORWARD}
+        assert write_back in wb_modes
         self.order = order
         self.window_rows = int(window_rows)
         self.lookahead = max(1, int(lookahead))
@@ -616,7 +621,7 @@ class NativePipelinedHotline(Hotline):
             B.hl_set_mover_ctas(self.ctx, mover_ctas, scatter_ctas)
         self.pipe = B.hl_pipe_create_ex(self.ctx, self.cache, self.host_table, self.window_rows, c_sets, self.n_dense,
                                         self.main.cuda_stream, index_priority=index_priority,
-                                        link_priority=link_priority, exclusive_write_back=exclusive_write_back)
+                                        link_priority=link_priority, write_back=wb_modes[write_back])
         if order == "eq5":
             B.hl_pipe_set_order(self.pipe, B.HL_PIPE_ORDER_EQ5)
         self.in_flight = 0

@@ -228,7 +228,8 @@ def run_config_check(spec, steps: int = 1, scale_rows: float = 1.0, integer: boo
 def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: bool = True, profile_batches=None,
                         device: str = "cuda:0", overlap_link: bool = True, sort_ahead: bool = True,
                         combined_sort: bool = True, lookahead: int = 2, native: bool = False,
-                        drain_between: bool = False, order: str = "fig8", per_table: bool = False):
+                        drain_between: bool = False, order: str = "fig8", per_table: bool = False,
+                        write_back: str = "overlap"):
     """Software-pipelined CUDA path (PipelinedHotline) against the oracle processing the same mini-batches one
     after the other.  With integer data every sum is exact, so pooled vectors, the hot cache and the host table
     must agree bit for bit after any number of steps -- which they only do if rows shared by consecutive
@@ -302,7 +303,8 @@ def run_pipelined_check(spec, steps: int = 6, scale_rows: float = 1.0, integer: 
 
     if native:
         p = hl.NativePipelinedHotline(geom.table_rows, D, S, B, max_nnz, hot_cap, window, host_table,
-                                      n_dense=spec.n_dense, device=device, lookahead=lookahead, order=order)
+                                      n_dense=spec.n_dense, device=device, lookahead=lookahead, order=order,
+                                      write_back=write_back)
     else:
         p = hl.PipelinedHotline(geom.table_rows, D, S, B, max_nnz, hot_cap, window, host_table, n_dense=spec.n_dense,
                                 device=device, overlap_link=overlap_link, sort_ahead=sort_ahead,

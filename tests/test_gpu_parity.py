@@ -204,6 +204,20 @@ def test_pipelines_with_an_empty_micro_batch(native):
     assert stats["shared_cold_rows"] == 0
 
 
+@pytest.mark.parametrize("write_back", ["exclusive", "after_forward"])
+def test_native_pipeline_write_back_modes(write_back):
+    """hl_pipe_options.write_back: the write-back of a mini-batch alone on the chip, or held over until the next
+    mini-batch's popular forward is over (queued by the next step, by a drain between steps, or at once by the last
+    step): the same results, bit for bit on integer data, with rows forwarded between consecutive mini-batches."""
+    assert run_pipelined_check("tiny", steps=7, integer=True, native=True, write_back=write_back)["shared_cold_rows"] > 50
+    run_pipelined_check("tiny", steps=5, integer=True, native=True, write_back=write_back, drain_between=True)
+    run_pipelined_check("tiny", steps=5, integer=True, native=True, write_back=write_back, lookahead=1)
+    run_pipelined_check("dlrm_small", steps=4, scale_rows=0.02, integer=True, profile_batches=6, native=True,
+                        write_back=write_back, lookahead=3)
+    if write_back == "after_forward":
+        run_pipelined_check("tiny", steps=6, integer=True, native=True, write_back=write_back, order="eq5")
+
+
 def test_native_pipeline_in_the_order_of_eq5_one_update_per_row_and_mini_batch():
     """Both forwards, then one update of every touched row with the gradient of the whole mini-batch (the lookups of a
     row from O and from X form one run of the merged sort): bit-exact on integer data, within the tolerance on real
