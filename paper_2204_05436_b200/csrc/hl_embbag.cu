@@ -220,7 +220,8 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
                                                          float lr, float* __restrict__ part,
                                                          const int32_t* __restrict__ d_first, int32_t key_bias,
                                                          int32_t* __restrict__ span_count,
-                                                         int32_t* __restrict__ span_list, int64_t n_grad_rows) {
+                                                         int32_t* __restrict__ span_list, int64_t n_grad_rows,
+                                                         int64_t max_entries, int32_t* status) {
     // the lookups of this call are positions [first, first + *d_n_lookups) of the sorted arrays; their keys are
     // slot + key_bias.  A chunk in which a run starts that goes on into the next chunk is appended to span_list
     // (in any order): k_bwd_spans finishes those runs.
@@ -321,8 +322,13 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
                     const int cnt = __ffs((int)~m) - 1;      // m == gbits (all G go on): -1 for G == 32, else G
                     if (sub == 0) {
                         const int32_t pos = atomicAdd(span_count, 1);
-                        reinterpret_cast<int4*>(span_list)[pos] =
-                            make_int4((int32_t)chunk, key, (cnt >= 1 && cnt < G) ? (int32_t)(chunk + cnt) : -1, 0);
+                        // (one entry per chunk at most, and the count is zero when a call starts: the list cannot
+                        // overflow unless an earlier call was cut short between its two kernels)
+                        if (pos >= 0 && pos < max_entries)
+                            reinterpret_cast<int4*>(span_list)[pos] =
+                                make_int4((int32_t)chunk, key, (cnt >= 1 && cnt < G) ? (int32_t)(chunk + cnt) : -1, 0);
+                        else
+                            set_status(status, HL_ECAPACITY);
                     }
                 }
             }
@@ -596,7 +602,7 @@ int32_t launch_bwd(hl_ctx* ctx, float* cache, const int32_t* keys, const int32_t
     int32_t* span_list = span_count + 8;
     k_bwd_chunks<G, NV><<<grid, kThreads, 0, stream>>>(cache, keys, vals, d_n_lookups, grad, ctx->D / 4, n_slots,
                                                       lr, ctx->r.bwd_part, d_first, key_bias, span_count, span_list,
-                                                      ctx->max_bags);
+                                                      ctx->max_bags, max_chunks, ctx->r.status);
     timer_mark(ctx, HL_TIMER_BWD_REDUCE, 1, stream);
     const int span_grid = grid_for(max_chunks * 32, kThreads, 4 * ctx_sms(ctx));   // the warps stride over the listed runs
     k_bwd_spans<G, NV><<<span_grid, kThreads, 0, stream>>>(cache, keys, d_n_lookups, ctx->D / 4, n_slots, lr,
