@@ -424,11 +424,13 @@ constexpr int kBulkStageBytes = 16384;
 constexpr int kBulkMaxPolls = 1 << 22;
 constexpr int kBulkStagesPerCta = 16;     // stages of rows per working CTA before another CTA joins in
 // Working CTAs of the mover inside a schedule (hl_set_mover_ctas changes it per context).  16 CTAs x 2 stages x
-// 16 KB keep 512 KB of rows in flight: 18 K rows of 256 bytes take about 160 us to read and 125 us to write back
+// 16 KB keep 512 KB of rows in flight: 16 K rows of 256 bytes take about 150 us to read and 120 us to write back
 // next to the other streams' kernels.  More CTAs move the rows faster (about 100 us with 2 per SM, alone), fewer
-// slower (one CTA writes back 64 rows every 3.4 us), but what the transfers cost the kernels that run next to them
-// does not depend on that.  (The hot-cache load of hl_build_remap and hl_flush_hot, which run alone, use 2 CTAs per
-// SM and reach 90 % of the memcpy rate.)  The defaults, kReadCtasDefault and kMoverCtasDefault, are set at hl_create.
+// slower (one CTA writes back 64 rows every 3.4 us); what a transfer costs the kernels that run next to it hardly
+// depends on that, so the host read, which nothing else of its mini-batch waits for at once, runs on 24 CTAs (about
+// 135 us) and the write-back on 16.  (The hot-cache load of hl_build_remap and hl_flush_hot, which run alone, use
+// 2 CTAs per SM and reach 90 % of the memcpy rate.)  The defaults, kReadCtasDefault and kMoverCtasDefault, are set at
+// hl_create.
 
 // What a launch of the mover needs to know about its context.
 struct MoveCfg {
