@@ -157,7 +157,8 @@ HL_API int32_t hl_set_mover_ctas(hl_ctx* ctx, int32_t read_ctas, int32_t write_c
 /* Grid size of the two bandwidth-bound kernels, in CTAs per multiprocessor: the forward kernel (hl_embbag_fwd) and
  * the backward's sum kernel (hl_embbag_bwd_*).  Both deal their work out evenly over a fixed grid; fewer CTAs per
  * multiprocessor leave registers and shared memory for the kernels of other streams (index work, movers) to run
- * beside them, more give the kernel itself more loads in flight.  0 = the default (3 and 6). */
+ * beside them, more give the kernel itself more loads in flight.  0 = the default (4 for the forward, 3 for rows wider
+ * than 128 fp32; 6 for the sum kernel). */
 HL_API int32_t hl_set_kernel_width(hl_ctx* ctx, int32_t fwd_ctas_per_sm, int32_t bwd_ctas_per_sm);
 
 /* Test aid for the bounded device-side waits (the tile chaining of the scan inside hl_fragment and of the sorts

@@ -151,7 +151,8 @@ inline void timer_mark(hl_ctx* ctx, int which, int end, cudaStream_t stream) {
 
 inline int ctx_sms(const hl_ctx* ctx) { return ctx->sms > 0 ? ctx->sms : kSMsFallback; }
 // CTAs per multiprocessor of the two bandwidth-bound kernels (hl_set_kernel_width; defaults chosen by measurement)
-inline int fwd_ctas_per_sm(const hl_ctx* ctx) { return ctx->fwd_ctas > 0 ? ctx->fwd_ctas : 3; }
+// (rows of up to 128 fp32: the forward kernel is held to 64 registers, so four of its CTAs fit a multiprocessor)
+inline int fwd_ctas_per_sm(const hl_ctx* ctx) { return ctx->fwd_ctas > 0 ? ctx->fwd_ctas : (ctx->D <= 128 ? 4 : 3); }
 inline int bwd_ctas_per_sm(const hl_ctx* ctx) { return ctx->bwd_ctas > 0 ? ctx->bwd_ctas : 6; }
 
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) {

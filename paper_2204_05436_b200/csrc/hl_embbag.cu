@@ -72,7 +72,7 @@ __device__ __forceinline__ void pool_long_bag(const float4* __restrict__ rows, c
 // the NEXT trip are requested before those rows are consumed, so that the offsets -> id -> row chain of one trip
 // hides behind the rows of another.  Longer bags go through pool_long_bag one after the other.
 template <int G, int NV, int UB>
-__global__ void __launch_bounds__(kThreads) k_embbag_fwd(const float* __restrict__ cache,
+__global__ void __launch_bounds__(kThreads, NV == 1 ? 4 : 1) k_embbag_fwd(const float* __restrict__ cache,
                                                          const int32_t* __restrict__ ids,
                                                          const int32_t* __restrict__ offsets,
                                                          const int32_t* __restrict__ d_n_samples, int max_batch,
