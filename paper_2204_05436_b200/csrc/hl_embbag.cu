@@ -18,6 +18,14 @@ __device__ __forceinline__ void red_add_f4(float4* p, float4 v) {
                  : "memory");
 }
 
+template <int N>
+__device__ __forceinline__ int32_t pick(const int32_t (&a)[N], int i) {      // a[i] without indexing registers
+    int32_t r = a[0];
+#pragma unroll
+    for (int k = 1; k < N; ++k) r = i == k ? a[k] : r;
+    return r;
+}
+
 __device__ __forceinline__ int clamp_samples(const int32_t* d_n_samples, int max_batch) {
     int n = *d_n_samples;
     if (n < 0) n = 0;
@@ -209,6 +217,12 @@ __global__ void __launch_bounds__(kThreads) k_bwd_pairs(const int32_t* __restric
 // address, one 128-bit load per column and the additions; everything that checks a pair (position inside the call,
 // bag inside the gradient array) is done by the lane that loaded the pair, once.  Gradient rows are loaded U at a
 // time.  The instruction count matters: this kernel issues about as many cycles as it waits for memory.
+//
+// A run that starts in one chunk and ends in the next (most runs that cross a border do) is finished by the group of
+// the chunk it starts in, which reads on into the next chunk; the group of that next chunk leaves the run's lookups
+// alone.  Both decide from the sorted slots alone and by the same test -- the run's head lies in the first of the two
+// chunks, and the chunk after the second does not begin with the run's slot -- so exactly one of them sums each
+// lookup.  Only runs over three or more chunks go through partial sums and k_bwd_spans.
 static_assert(kBwdChunk == 32, "the head and tail masks of a chunk are 32-bit words");
 
 template <int G, int NV>
@@ -268,6 +282,9 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
         }
         const int32_t prev_key = start > first ? keys[start - 1] : -3;   // -3: equal to no key
         const int32_t next_key = end < n ? keys[end] : -2;
+        // the slot before the previous chunk, and the first slot of the chunk after the next one
+        const int32_t prev2_key = start - kBwdChunk > first ? keys[start - kBwdChunk - 1] : -3;
+        const int32_t next2_key = start + 2 * kBwdChunk < n ? keys[start + 2 * kBwdChunk] : -2;
 
         // bit q of `heads`: lookup q of the chunk begins a run; of `tails`: it ends one
         uint32_t heads = 0, tails = 0;
@@ -283,6 +300,22 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
             const uint32_t tb = (__ballot_sync(gmask, kk[i] != succ) >> gshift) & gbits;
             heads |= hb << (i * G);
             tails |= tb << (i * G);
+        }
+
+        const bool ends_open = !((tails >> (kBwdChunk - 1)) & 1u);   // the last run goes on in the next chunk
+        // A run that comes in from the previous chunk, began there and ends here was finished by that chunk's group:
+        // its lookups (up to its tail, the lowest tail bit) are not summed here -- their loads are pointed at the bag
+        // of the chunk's last lookup, which is loaded anyway, and the tail bit is cleared so that nothing is applied.
+        {
+            const int32_t key0 = __shfl_sync(gmask, kk[0], 0, G);
+            if (chunk >= 1 && !(heads & 1u) && tails != 0u && prev2_key != key0) {
+                const int t = __ffs((int)tails) - 1;
+                tails &= tails - 1u;
+                const int32_t last_bag = __shfl_sync(gmask, vv[KPL - 1], G - 1, G);
+#pragma unroll
+                for (int i = 0; i < KPL; ++i)
+                    if (i * G + sub <= t) vv[i] = last_bag;
+            }
         }
 
         // the run being summed continues one from the previous chunk until the first head
@@ -370,7 +403,52 @@ __global__ void __launch_bounds__(kThreads, NV == 1 ? 3 : 1) k_bwd_chunks(float*
         }
         // the chunk's last lookup does not end its run: the run goes on in the next chunk (only a full chunk has a
         // next one)
-        if (!((tails >> (kBwdChunk - 1)) & 1u)) emit(__shfl_sync(gmask, kk[KPL - 1], G - 1, G), true);
+        if (ends_open) {
+            const int32_t key = __shfl_sync(gmask, kk[KPL - 1], G - 1, G);
+            if (!left_open && next2_key != key && (uint32_t)(key - key_bias) < n_rows_u) {
+                // it began in this chunk and ends in the next: its lookups there are summed here as well (they are a
+                // prefix of that chunk: m of them), and the row gets its one update
+                const int64_t start2 = start + kBwdChunk;
+                const int64_t end2 = min(start2 + (int64_t)kBwdChunk, n);
+                int32_t vv2[KPL];
+                uint32_t same = 0;
+#pragma unroll
+                for (int i = 0; i < KPL; ++i) {
+                    const int64_t p = start2 + i * G + sub;
+                    const bool in = p < end2;
+                    const int32_t k2 = in ? keys[p] : -1;
+                    const int32_t bag = in ? vals[p] : 0;
+                    vv2[i] = (uint32_t)bag < n_grad_u ? bag : 0;
+                    same |= ((__ballot_sync(gmask, k2 == key) >> gshift) & gbits) << (i * G);
+                }
+                const int m = same == 0xffffffffu ? kBwdChunk : __ffs((int)~same) - 1;
+#pragma unroll 1
+                for (int q0 = 0; q0 < m; q0 += U) {
+                    float4 g[U][NV];
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        const int q = q0 + u < m ? q0 + u : m - 1;       // (past the run's end: a row already asked for)
+                        const int32_t bag = __shfl_sync(gmask, pick(vv2, q / G), q % G, G);
+#pragma unroll
+                        for (int v = 0; v < NV; ++v) g[u][v] = __ldg(gcol[v] + (int64_t)bag * D4);
+                    }
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if (q0 + u >= m) continue;
+#pragma unroll
+                        for (int v = 0; v < NV; ++v) {
+                            acc[v][0] += (double)g[u][v].x;
+                            acc[v][1] += (double)g[u][v].y;
+                            acc[v][2] += (double)g[u][v].z;
+                            acc[v][3] += (double)g[u][v].w;
+                        }
+                    }
+                }
+                emit(key, false);
+            } else {
+                emit(key, true);
+            }
+        }
     }
 }
 
