@@ -280,6 +280,7 @@ extern "C" hl_pipe* hl_pipe_create(hl_ctx* ctx, float* d_cache, float* host_tabl
 
 extern "C" void hl_pipe_destroy(hl_pipe* p) {
     if (!p) return;
+    if (p->wb_pending && p->wb) (void)flush_scatter(p);      // a write-back held over is not lost
     cudaStream_t side[5] = {p->sa, p->sb, p->sc, p->link, p->wb};
     for (auto s : side)
         if (s) {
@@ -287,7 +288,7 @@ extern "C" void hl_pipe_destroy(hl_pipe* p) {
             cudaStreamDestroy(s);
         }
     for (auto& e : p->ev) {
-        cudaEvent_t all[8] = {e.inputs, e.frag, e.index, e.prep, e.gather, e.forward, e.x, e.scatter};
+        cudaEvent_t all[9] = {e.inputs, e.frag, e.index, e.prep, e.gather, e.forward, e.x, e.scatter, e.fwd_pop};
         for (auto x : all)
             if (x) cudaEventDestroy(x);
     }
