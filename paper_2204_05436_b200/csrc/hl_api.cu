@@ -140,6 +140,7 @@ extern "C" int32_t hl_create(hl_ctx** out, const hl_geometry* geom, int32_t max_
     if (e == cudaSuccess) e = cudaMemset(ctx->r.remap, 0, sizeof(RemapBlock) * ctx->n_remap_blocks);
     if (e == cudaSuccess) e = cudaMemset(ctx->r.counts, 0, sizeof(uint32_t) * N);
     if (e == cudaSuccess) e = cudaMemset(ctx->r.sel, 0, sizeof(SelectState));
+    if (e == cudaSuccess) e = cudaMemset(ctx->r.frag_tiles, 0, sizeof(int32_t) * scan_tile_words(max_bags));
     if (e == cudaSuccess) e = cudaMemset(span_count_of(ctx), 0, 8 * sizeof(int32_t));   // kept zero between backward calls
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {

@@ -274,6 +274,7 @@ extern "C" int32_t hl_wide_create(hl_wide** out, const hl_geometry* geom, int32_
     if (e == cudaSuccess) e = cudaMemset(w->c_cnt, 0, sizeof(uint32_t) * w->counter_slots);
     if (e == cudaSuccess) e = cudaMemset(w->r_keys, 0xff, sizeof(long long) * w->remap_slots);
     if (e == cudaSuccess) e = cudaMemset(w->sel, 0, sizeof(SelectState));
+    if (e == cudaSuccess) e = cudaMemset(w->frag_tiles, 0, sizeof(int32_t) * scan_tile_words(w->max_bags));
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         free(w->h_table_base);
