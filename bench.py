@@ -1024,9 +1024,10 @@ def run_cuda(args, rank: int, local_rank: int, world: int) -> None:
 # single-call micro runs (small cases: one library call in isolation, sized for a profiler capture)
 # ----------------------------------------------------------------------------------------------------------
 def run_micro_gather(args) -> None:
-    """`--micro gather`: the row-move kernel alone, host table -> HBM, 65,536 rows of 256 bytes from a 16 GiB
-    pinned table: consecutive rows, random rows within the first 4 GiB, random rows over the whole table; each
-    pattern is gathered three times (the later repetitions find their address translations resident)."""
+    """`--micro gather`: the row-move kernel alone, host table -> HBM and back, 65,536 rows of 256 bytes of a 16 GiB
+    host table: consecutive rows, random rows within the first 4 GiB, random rows over the whole table; each
+    pattern is gathered three times (the later repetitions find their address translations resident) and then
+    written back three times (hl_flush_hot: the same mover in the other direction)."""
     import torch
     import paper_2204_05436_b200 as hl
     dev = torch.device("cuda:0")
@@ -1047,7 +1048,16 @@ def run_micro_gather(args) -> None:
         b.record()
         torch.cuda.synchronize()
         best = max(best, buf_h.numel() / (a.elapsed_time(b) * 1e-3) / 1e9)
-    res = {"micro": "gather", "rows": K, "row_bytes": 4 * D, "table_gib": N * D * 4 / 2 ** 30, "memcpy_h2d_gbs": best}
+    best_d2h = 0.0
+    for _ in range(5):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        buf_h.copy_(buf_d, non_blocking=True)
+        b.record()
+        torch.cuda.synchronize()
+        best_d2h = max(best_d2h, buf_h.numel() / (a.elapsed_time(b) * 1e-3) / 1e9)
+    res = {"micro": "gather", "rows": K, "row_bytes": 4 * D, "table_gib": N * D * 4 / 2 ** 30, "memcpy_h2d_gbs": best,
+           "memcpy_d2h_gbs": best_d2h}
 
     def timed(load):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -1065,6 +1075,16 @@ def run_micro_gather(args) -> None:
             runs = [timed(True) - base for _ in range(3)]
             res[name] = {"first_gbs": K * D * 4 / runs[0] / 1e6, "best_gbs": K * D * 4 / min(runs) / 1e6,
                          "best_frac_of_memcpy": K * D * 4 / min(runs) / 1e6 / best}
+            wb = []
+            for _ in range(3):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(h.main)
+                h.flush_hot()
+                b.record(h.main)
+                torch.cuda.synchronize()
+                wb.append(a.elapsed_time(b))
+            res[name]["write_back"] = {"first_gbs": K * D * 4 / wb[0] / 1e6, "best_gbs": K * D * 4 / min(wb) / 1e6,
+                                       "best_frac_of_memcpy": K * D * 4 / min(wb) / 1e6 / best_d2h}
     h.status()
     h.close()
     print(json.dumps(res), flush=True)
